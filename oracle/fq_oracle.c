@@ -1,0 +1,280 @@
+/*
+ * CPU oracle for the outlier-aware W4A16 decode matmul.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain, obviously-correct
+ * statement of what the method computes.  Only the test-suite, the smoke check
+ * and the benchmark's cpu_baseline / reference arm may build or call it.  It
+ * shares no code, header, table or helper with the CUDA library; the format
+ * decoders below are written from the packed-format description alone.
+ *
+ * What it states (paper passage for each):
+ *   - affine 4-bit group quantiser            Eq. 2 (q = round(w/s) + z) and the
+ *                                             formulas for s and z given with Eq. 3
+ *   - dequantisation  w^ = s (q - z)          Eq. 3
+ *   - result  Y = X deq(W_Q) + X W_O          Eq. 1
+ *   - Tile-COO arrays (tile_indptr, bucket_info, packed_outliers; four
+ *     outliers per 16-byte packet, u8 row index, u8 column index, BF16 value)
+ *                                             Section 3.2.1, Table 1
+ *
+ * Readings taken where the paper is silent (each also listed in the design
+ * notes): round = round-half-to-even; q and z clamped to [0,15]; the quantiser
+ * runs in IEEE binary32 with the BF16-rounded scale; the group range always
+ * contains 0; a degenerate group gets s = 1, z = 0, q = 0; an outlier slot holds
+ * q = z so that it dequantises to exactly 0 and W_O carries the full BF16
+ * weight; groups run along K.
+ *
+ * Floating point: everything after the quantiser is binary64, k ascending,
+ * no blocking, no reordering.  Build with -ffp-contract=off and without
+ * -ffast-math.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* ------------------------------------------------------------------ BF16 */
+
+/* binary32 -> bfloat16, round to nearest even; NaN stays NaN. */
+uint16_t orc_f32_to_bf16(float f) {
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x0040u);
+    uint32_t lsb = (u >> 16) & 1u;
+    u += 0x7fffu + lsb;
+    return (uint16_t)(u >> 16);
+}
+
+float orc_bf16_to_f32(uint16_t h) {
+    uint32_t u = ((uint32_t)h) << 16;
+    float f;
+    memcpy(&f, &u, 4);
+    return f;
+}
+
+int orc_num_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* ------------------------------------------------------------ quantiser */
+
+static int clamp_i(int v, int lo, int hi) { return v < lo ? lo : (v > hi ? hi : v); }
+
+/*
+ * Eq. 2 with b = 4, per (group of g rows along K, column n), over the weights
+ * that are not outliers.  W is K x N row-major binary32; mask is K x N (1 =
+ * outlier) or NULL.  Outputs: q K x N (one code per byte), scale and zero
+ * (K/g) x N as BF16 bit patterns.  Returns 0, or -1 on bad sizes.
+ */
+int orc_quantize(const float* W, const uint8_t* mask, uint32_t K, uint32_t N, uint32_t g,
+                 uint8_t* q, uint16_t* scale, uint16_t* zero) {
+    if (g == 0 || K % g != 0) return -1;
+    const uint32_t G = K / g;
+#pragma omp parallel for schedule(static)
+    for (int64_t n = 0; n < (int64_t)N; ++n) {
+        for (uint32_t gi = 0; gi < G; ++gi) {
+            float wmin = 0.0f, wmax = 0.0f; /* the range always contains 0 */
+            for (uint32_t k = gi * g; k < (gi + 1) * g; ++k) {
+                size_t idx = (size_t)k * N + (size_t)n;
+                if (mask && mask[idx]) continue;
+                float w = W[idx];
+                if (w < wmin) wmin = w;
+                if (w > wmax) wmax = w;
+            }
+            float s32 = (wmax - wmin) / 15.0f; /* s = (wmax - wmin) / (2^b - 1) */
+            uint16_t sb = orc_f32_to_bf16(s32);
+            float sf = orc_bf16_to_f32(sb);
+            int z;
+            if (!(sf > 0.0f)) { /* degenerate group */
+                sb = orc_f32_to_bf16(1.0f);
+                sf = 1.0f;
+                z = 0;
+                for (uint32_t k = gi * g; k < (gi + 1) * g; ++k) q[(size_t)k * N + (size_t)n] = 0;
+            } else {
+                z = clamp_i((int)nearbyintf(-wmin / sf), 0, 15); /* z = round(-wmin / s) */
+                for (uint32_t k = gi * g; k < (gi + 1) * g; ++k) {
+                    size_t idx = (size_t)k * N + (size_t)n;
+                    if (mask && mask[idx]) {
+                        q[idx] = (uint8_t)z; /* dequantises to exactly 0 */
+                    } else {
+                        int qi = (int)nearbyintf(W[idx] / sf) + z; /* q = round(w / s) + z */
+                        q[idx] = (uint8_t)clamp_i(qi, 0, 15);
+                    }
+                }
+            }
+            scale[(size_t)gi * N + (size_t)n] = sb;
+            zero[(size_t)gi * N + (size_t)n] = orc_f32_to_bf16((float)z);
+        }
+    }
+    return 0;
+}
+
+/* Eq. 3: What[k][n] = s[k/g][n] * (q[k][n] - z[k/g][n]), in binary64. */
+void orc_dequant(const uint8_t* q, const uint16_t* scale, const uint16_t* zero, uint32_t K,
+                 uint32_t N, uint32_t g, double* What) {
+#pragma omp parallel for schedule(static)
+    for (int64_t k = 0; k < (int64_t)K; ++k) {
+        const size_t gi = (size_t)k / g;
+        for (uint32_t n = 0; n < N; ++n) {
+            double s = (double)orc_bf16_to_f32(scale[gi * N + n]);
+            double z = (double)orc_bf16_to_f32(zero[gi * N + n]);
+            What[(size_t)k * N + n] = s * ((double)q[(size_t)k * N + n] - z);
+        }
+    }
+}
+
+/* --------------------------------------------------------------- result */
+
+/*
+ * Eq. 1 on a list of output columns (cols == NULL: all N columns, ncols == N).
+ *   Y[m][j]    = sum_k X[m][k] * s (q - z)  +  sum over outliers in column
+ *                cols[j] of X[m][k] * W_O[k][n]
+ *   Yabs[m][j] = the same sums with every product replaced by its magnitude
+ *                (NULL to skip); used only for condition-aware reporting.
+ * X is M x K BF16 bits, row-major.  Outliers come as COO (k, n, BF16 bits).
+ * Y and Yabs are M x ncols binary64, row-major.
+ */
+void orc_fused_matmul(const uint16_t* X, uint32_t M, uint32_t K, uint32_t N, uint32_t g,
+                      const uint8_t* q, const uint16_t* scale, const uint16_t* zero,
+                      const uint32_t* coo_k, const uint32_t* coo_n, const uint16_t* coo_v,
+                      size_t nnz, const uint32_t* cols, uint32_t ncols, double* Y, double* Yabs) {
+    /* dense part: X * dequant(W_Q) */
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < (int64_t)ncols; ++j) {
+        const uint32_t n = cols ? cols[j] : (uint32_t)j;
+        for (uint32_t m = 0; m < M; ++m) {
+            double acc = 0.0, accabs = 0.0;
+            for (uint32_t k = 0; k < K; ++k) {
+                const size_t gi = (size_t)k / g;
+                double s = (double)orc_bf16_to_f32(scale[gi * N + n]);
+                double z = (double)orc_bf16_to_f32(zero[gi * N + n]);
+                double w = s * ((double)q[(size_t)k * N + n] - z);
+                double x = (double)orc_bf16_to_f32(X[(size_t)m * K + k]);
+                acc += x * w;
+                accabs += fabs(x * w);
+            }
+            Y[(size_t)m * ncols + (size_t)j] = acc;
+            if (Yabs) Yabs[(size_t)m * ncols + (size_t)j] = accabs;
+        }
+    }
+    /* sparse part: X * W_O, one COO entry at a time */
+    int64_t* slot = NULL;
+    if (cols) {
+        slot = (int64_t*)malloc(sizeof(int64_t) * (size_t)N);
+        for (uint32_t n = 0; n < N; ++n) slot[n] = -1;
+        for (uint32_t j = 0; j < ncols; ++j) slot[cols[j]] = (int64_t)j;
+    }
+    for (size_t e = 0; e < nnz; ++e) {
+        int64_t j = cols ? slot[coo_n[e]] : (int64_t)coo_n[e];
+        if (j < 0) continue;
+        double v = (double)orc_bf16_to_f32(coo_v[e]);
+        for (uint32_t m = 0; m < M; ++m) {
+            double x = (double)orc_bf16_to_f32(X[(size_t)m * K + coo_k[e]]);
+            Y[(size_t)m * ncols + (size_t)j] += x * v;
+            if (Yabs) Yabs[(size_t)m * ncols + (size_t)j] += fabs(x * v);
+        }
+    }
+    free(slot);
+}
+
+/* ------------------------------------------------------ format decoders */
+
+/*
+ * Packed INT4 weight buffer -> q[K][N], from the format description:
+ *
+ *   The buffer is a sequence of chunks, one per (column tile tn, row tile kt),
+ *   ordered tn-major (chunk index tn * (K/128) + kt).  A chunk covers 128 rows
+ *   by BN columns and holds 16 * BN little-endian 32-bit words.  Word index
+ *   inside the chunk:
+ *        ((w * 4 + j) * 32 + lane) * 4 + c
+ *   with w = 32-column strip (0 .. BN/32-1), j = 0..3, lane = 0..31, c = 0..3.
+ *   Let ns = j >> 1, ks = (j & 1) * 4 + c, grp = lane >> 2, t = lane & 3.
+ *   Nibble p (bits 4p .. 4p+3) of that word, p = r + 4h with r = 0..3, h = 0..1,
+ *   is the code of
+ *        column  tn*BN + 32*w + 16*ns + grp + 8*(r & 1)
+ *        row     kt*128 + 32*(ks >> 1) + 8*t + 4*(ks & 1) + 2*(r >> 1) + h
+ */
+int orc_decode_wq(const uint32_t* wq, uint32_t K, uint32_t N, uint32_t BN, uint8_t* q) {
+    if (K % 128 != 0 || BN % 32 != 0 || N % BN != 0) return -1;
+    const uint32_t KT = K / 128, NT = N / BN, strips = BN / 32;
+    const size_t chunk_words = (size_t)16 * BN;
+    for (uint32_t tn = 0; tn < NT; ++tn)
+        for (uint32_t kt = 0; kt < KT; ++kt) {
+            const uint32_t* chunk = wq + ((size_t)tn * KT + kt) * chunk_words;
+            for (uint32_t w = 0; w < strips; ++w)
+                for (uint32_t j = 0; j < 4; ++j)
+                    for (uint32_t lane = 0; lane < 32; ++lane)
+                        for (uint32_t c = 0; c < 4; ++c) {
+                            uint32_t word = chunk[((w * 4 + j) * 32 + lane) * 4 + c];
+                            uint32_t ns = j >> 1, ks = (j & 1) * 4 + c;
+                            uint32_t grp = lane >> 2, t = lane & 3;
+                            for (uint32_t p = 0; p < 8; ++p) {
+                                uint32_t r = p & 3, h = p >> 2;
+                                uint32_t col = tn * BN + 32 * w + 16 * ns + grp + 8 * (r & 1);
+                                uint32_t row = kt * 128 + 32 * (ks >> 1) + 8 * t + 4 * (ks & 1) +
+                                               2 * (r >> 1) + h;
+                                q[(size_t)row * N + col] = (uint8_t)((word >> (4 * p)) & 0xfu);
+                            }
+                        }
+        }
+    return 0;
+}
+
+/*
+ * Tile-COO arrays -> COO list, from the format description:
+ *
+ *   Tiles are 128 rows by BN columns, tile index tn * (K/128) + kt.
+ *   tile_indptr[t] .. tile_indptr[t+1] is the tile's range of 16-byte packets
+ *   in packed_outliers.  bucket_info[t * NB + b] = offset | (count << 16):
+ *   bucket b of tile t owns packets [tile_indptr[t] + offset, + count).
+ *   A packet is: bytes 0-3 row index inside the tile of slots 0-3, bytes 4-7
+ *   column index inside the tile of slots 0-3, bytes 8-15 four BF16 values
+ *   (little-endian).  A slot whose value bits are 0x0000 is padding.
+ *
+ * out_* must have room for 4 * (number of packets) entries; *count receives the
+ * number of real entries.  Returns 0, or a negative code for a structural
+ * error (-2 indptr not monotone, -3 bucket range outside its tile, -4 index
+ * outside the tile).
+ */
+int orc_decode_tilecoo(const uint32_t* tile_indptr, const uint32_t* bucket_info,
+                       const uint8_t* packed, uint32_t K, uint32_t N, uint32_t BN, uint32_t NB,
+                       uint32_t* out_k, uint32_t* out_n, uint16_t* out_v, uint32_t* out_bucket,
+                       size_t* count) {
+    if (K % 128 != 0 || N % BN != 0) return -1;
+    const uint32_t KT = K / 128, NT = N / BN;
+    size_t c = 0;
+    for (uint32_t tn = 0; tn < NT; ++tn)
+        for (uint32_t kt = 0; kt < KT; ++kt) {
+            const size_t t = (size_t)tn * KT + kt;
+            const uint32_t p0 = tile_indptr[t], p1 = tile_indptr[t + 1];
+            if (p1 < p0) return -2;
+            for (uint32_t b = 0; b < NB; ++b) {
+                uint32_t info = bucket_info[t * NB + b];
+                uint32_t off = info & 0xffffu, cnt = info >> 16;
+                if ((size_t)p0 + off + cnt > (size_t)p1) return -3;
+                for (uint32_t i = 0; i < cnt; ++i) {
+                    const uint8_t* pk = packed + ((size_t)p0 + off + i) * 16;
+                    for (int sidx = 0; sidx < 4; ++sidx) {
+                        uint16_t v = (uint16_t)(pk[8 + 2 * sidx] | (pk[9 + 2 * sidx] << 8));
+                        if (v == 0) continue;
+                        uint32_t kk = pk[sidx], cc = pk[4 + sidx];
+                        if (kk >= 128 || cc >= BN) return -4;
+                        out_k[c] = kt * 128 + kk;
+                        out_n[c] = tn * BN + cc;
+                        out_v[c] = v;
+                        if (out_bucket) out_bucket[c] = (uint32_t)(t * NB + b);
+                        ++c;
+                    }
+                }
+            }
+        }
+    *count = c;
+    return 0;
+}

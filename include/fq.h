@@ -1,0 +1,211 @@
+/*
+ * fq.h -- C ABI of the fused outlier-aware W4A16 decode matmul for NVIDIA B200
+ * (sm_100a).
+ *
+ *      Y = X * dequant(W_Q) + X * W_O                                  (Eq. 1)
+ *
+ * X is a small-M BF16 activation block (M x K, row-major), W_Q is K x N
+ * group-quantised asymmetric INT4 (Eq. 2, Eq. 3; groups of 64 or 128 rows along
+ * K, BF16 scale and BF16-held integer zero-point per group and column) and W_O
+ * is a sparse BF16 outlier matrix in the Tile-COO encoding (Section 3.2.1,
+ * Table 1).  Y is M x N BF16, row-major, accumulated in FP32 and rounded once.
+ *
+ * Conventions
+ *   - Every function returns an fq_status_t; nothing throws across the ABI.
+ *     fq_last_error() gives a thread-local text for the last failure.
+ *   - "host" pointers are ordinary memory, "device" pointers are CUDA global
+ *     memory of the current device.  The caller owns every buffer; the library
+ *     allocates nothing that outlives a call.
+ *   - Device entry points only enqueue work on `cuda_stream` (a cudaStream_t
+ *     passed as void*; NULL = the legacy default stream) and return.  Argument
+ *     errors are reported synchronously and nothing is launched.  A device-side
+ *     wait that gave up is reported by fq_check_status().
+ *   - Device arrays must be 128-byte aligned (16 bytes for X and Y rows, which
+ *     follows from K % 8 == 0 and N % 8 == 0).
+ *
+ * Packed formats (the kernel's choice; the paper leaves them open)
+ *
+ *   INT4 weights.  BK = 128 rows, BN = 128 or 256 columns per tile.  The buffer
+ *   is a sequence of chunks, one per (column tile tn, row tile kt), chunk index
+ *   tn * (K/128) + kt, each 16 * BN little-endian 32-bit words.  Word index
+ *   inside a chunk is ((w*4 + j)*32 + lane)*4 + c  (w = 32-column strip,
+ *   j = 0..3, lane = 0..31, c = 0..3).  With ns = j>>1, ks = (j&1)*4 + c,
+ *   grp = lane>>2, t = lane&3, nibble p = r + 4h (r = 0..3, h = 0..1; bits
+ *   4p..4p+3) of that word is the code of
+ *       column tn*BN + 32w + 16ns + grp + 8(r&1)
+ *       row    kt*128 + 32(ks>>1) + 8t + 4(ks&1) + 2(r>>1) + h .
+ *   (One word is one thread's A-operand fragment of one m16n8k16 MMA; row order
+ *   inside a 32-row block follows the 16-byte activation loads of the kernel.)
+ *
+ *   Scale, zero.  (K/group) x N row-major BF16.  zero holds the integer 0..15.
+ *
+ *   Tile-COO.  Tiles are BK x BN, tile index t = tn * (K/128) + kt.
+ *   tile_indptr[t] .. tile_indptr[t+1]: the tile's range of 16-byte packets in
+ *   packed_outliers (N_tile + 1 entries, uint32).  bucket_info[t*NB + b] =
+ *   offset | count << 16 (two uint16): bucket b of tile t owns `count` packets
+ *   starting `offset` packets after the tile's first.  Buckets of one tile own
+ *   disjoint column sets.  A packet holds four outliers: bytes 0-3 row index in
+ *   the tile, bytes 4-7 column index in the tile, bytes 8-15 four BF16 values.
+ *   A slot with value bits 0x0000 is padding (its indices repeat the bucket's
+ *   last real entry).  Storage: (N_tile+1)*4 + N_tile*NB*4 + 16*packets bytes.
+ */
+#ifndef FQ_H_
+#define FQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t fq_status_t;
+#define FQ_OK 0
+#define FQ_ERR_INVALID_ARG (-1)       /* null or misaligned pointer, M out of range, bad layout */
+#define FQ_ERR_UNSUPPORTED_SHAPE (-2) /* K % 128, N % BN, group not 64/128, bucket count */
+#define FQ_ERR_BUFFER_TOO_SMALL (-3)
+#define FQ_ERR_CUDA (-4)              /* a CUDA runtime call failed; text in fq_last_error() */
+#define FQ_ERR_TIMEOUT (-5)           /* a bounded device-side wait expired */
+#define FQ_ERR_FORMAT (-6)            /* Tile-COO validator: bad indptr / offset / index */
+
+#define FQ_ABI_VERSION 1u
+#define FQ_MAX_M 128u
+#define FQ_BK 128u
+
+/* Plain data, caller-owned.  Filled by fq_get_layout(); fq_encode_tilecoo()
+ * writes max_tile_packets.  Pass the same struct to every later call. */
+typedef struct fq_layout {
+    uint32_t abi;
+    uint32_t K, N;
+    uint32_t group;            /* 64 or 128, along K */
+    uint32_t BK;               /* 128 */
+    uint32_t BN;               /* 128 or 256 */
+    uint32_t buckets_per_tile; /* NB: 32, 64 or 128 */
+    uint32_t wq_interleave;    /* 1: the MMA-fragment order described above */
+    uint32_t coo_unit_bytes;   /* 16 */
+    uint32_t max_tile_packets; /* largest tile of the encoded W_O, in packets; 0 = not encoded */
+    uint32_t reserved[6];
+} fq_layout_t;
+
+/* Choose tile sizes for a K x N layer.  bn_hint / nb_hint: 0 = library default,
+ * otherwise BN in {128, 256} and NB in {32, 64, 128}.  Errors:
+ * FQ_ERR_UNSUPPORTED_SHAPE for shapes the kernel cannot tile. */
+fq_status_t fq_get_layout(uint32_t K, uint32_t N, uint32_t group, uint32_t bn_hint, uint32_t nb_hint,
+                          fq_layout_t* out);
+
+/* ---------------------------------------------------------------- host, offline */
+
+/* Byte sizes of the three arrays fq_pack_int4 writes. */
+fq_status_t fq_pack_int4_sizes(const fq_layout_t* L, size_t* wq_bytes, size_t* scale_bytes,
+                               size_t* zero_bytes);
+
+/*
+ * Quantise and pack (Eq. 2 with b = 4, the formulas for s and z that follow
+ * Eq. 3).  W: host, K x N row-major binary32.  outlier_mask: host, K x N bytes,
+ * 1 = outlier (excluded from the group range, stored with code = zero-point so
+ * that it dequantises to 0), may be NULL.  Outputs (host): wq in the chunked
+ * order above, scale and zero as (K/group) x N BF16 bit patterns.  Readings
+ * where the paper is silent: round-half-to-even, codes and zero-point clamped to
+ * 0..15, binary32 arithmetic with the BF16-rounded scale, the group range always
+ * contains 0, a degenerate group gets scale 1 and zero 0.
+ */
+fq_status_t fq_pack_int4(const fq_layout_t* L, const float* W, const uint8_t* outlier_mask, void* wq,
+                         uint16_t* scale_bf16, uint16_t* zero_bf16);
+
+/* Inverse of the nibble interleave: wq (host) -> q_canon (host, K x N, one code per byte). */
+fq_status_t fq_unpack_int4(const fq_layout_t* L, const void* wq, uint8_t* q_canon);
+
+/*
+ * Tile-COO encoder (Section 3.2.1; column reordering and element reordering of
+ * Section 3.2.2).  Input: COO triplets on the host (k, n, BF16 value bits), any
+ * order; entries whose value is +-0 are dropped.  Per tile, columns are sorted
+ * by outlier count (descending) and assigned greedily to the least-loaded of NB
+ * buckets; inside a bucket, entries are ordered so that position i of bucket b
+ * prefers shared-memory bank group (i + b) mod 8 of the kernel's activation
+ * copy (bank group of row k = k mod 8), falling through to the next non-empty
+ * group; buckets are padded to whole packets.
+ *
+ * fq_encode_tilecoo_sizes: element counts of the three arrays (tile_indptr in
+ * uint32, bucket_info in uint32, packets in 16-byte units) and the largest
+ * tile.  fq_encode_tilecoo: writes them and stores max_tile_packets in *L.
+ */
+fq_status_t fq_encode_tilecoo_sizes(const fq_layout_t* L, const uint32_t* k, const uint32_t* n,
+                                    const uint16_t* val_bf16, size_t nnz, size_t* n_indptr,
+                                    size_t* n_bucket_info, size_t* n_packets,
+                                    uint32_t* max_tile_packets);
+fq_status_t fq_encode_tilecoo(fq_layout_t* L, const uint32_t* k, const uint32_t* n,
+                              const uint16_t* val_bf16, size_t nnz, uint32_t* tile_indptr,
+                              uint32_t* bucket_info, void* packed_outliers, size_t n_packets);
+
+/* Tile-COO -> COO (host).  *nnz_inout: capacity on entry, count on return. */
+fq_status_t fq_decode_tilecoo(const fq_layout_t* L, const uint32_t* tile_indptr,
+                              const uint32_t* bucket_info, const void* packed_outliers, uint32_t* k,
+                              uint32_t* n, uint16_t* val_bf16, size_t* nnz_inout);
+
+/* Structural check of host Tile-COO arrays before they are given to a kernel:
+ * monotone indptr ending at n_packets, bucket ranges inside their tile, indices
+ * inside the tile, bucket column sets disjoint.  FQ_ERR_FORMAT on violation. */
+fq_status_t fq_validate_tilecoo(const fq_layout_t* L, const uint32_t* tile_indptr,
+                                const uint32_t* bucket_info, const void* packed_outliers,
+                                size_t n_packets);
+
+/* --------------------------------------------------------------------- device */
+
+/* Bytes of caller-allocated device scratch for calls with this layout and M.
+ * The scratch must be zeroed once before its first use; every completed call
+ * leaves it ready for the next one on the same stream.  Calls that may overlap
+ * on the GPU need distinct scratch. */
+fq_status_t fq_workspace_bytes(const fq_layout_t* L, uint32_t M, size_t* bytes);
+
+/*
+ * The fused operator (Eq. 1; Sections 3.1 and 4.1): one launch per 32 rows of X
+ * reads X, W_Q and the Tile-COO tiles through a TMA/mbarrier ring, dequantises
+ * in registers into tensor-core accumulators, applies the tile's outliers
+ * against the same shared-memory activation tile, and writes Y once.
+ * X: device, M x K BF16.  M in [1, FQ_MAX_M].  Y: device, M x N BF16,
+ * overwritten.  All other arrays: device copies of the host packer/encoder
+ * output.  Work is split over persistent CTAs by contiguous ranges of (tile,
+ * k-step) units; tiles shared by several CTAs are summed in a fixed order, so
+ * results are run-to-run reproducible.
+ */
+fq_status_t fq_fused_w4a16_outlier_gemm(const fq_layout_t* L, const void* X, uint32_t M,
+                                        const void* wq, const void* scale, const void* zero,
+                                        const void* tile_indptr, const void* bucket_info,
+                                        const void* packed_outliers, void* Y, void* workspace,
+                                        size_t workspace_bytes, void* cuda_stream);
+
+/* Unfused baseline, dense half: Y = X * dequant(W_Q) (same kernel, sparse path
+ * compiled out). */
+fq_status_t fq_unfused_gemm(const fq_layout_t* L, const void* X, uint32_t M, const void* wq,
+                            const void* scale, const void* zero, void* Y, void* workspace,
+                            size_t workspace_bytes, void* cuda_stream);
+
+/* Unfused baseline, sparse half: Y += X * W_O as a separate launch that re-reads
+ * X and read-modify-writes the BF16 Y (the two-kernel scheme the paper compares
+ * against, Section 2.2). */
+fq_status_t fq_unfused_spmm(const fq_layout_t* L, const void* X, uint32_t M, const void* tile_indptr,
+                            const void* bucket_info, const void* packed_outliers, void* Y,
+                            void* cuda_stream);
+
+/* Same operator as fq_fused_w4a16_outlier_gemm, called with HOST X and HOST Y:
+ * copies X to x_dev, runs the kernel, copies Y back from y_dev and waits for
+ * the stream.  x_dev / y_dev are caller-allocated device staging buffers of
+ * M*K*2 and M*N*2 bytes. */
+fq_status_t fq_fused_host_io(const fq_layout_t* L, const void* X_host, uint32_t M, void* x_dev,
+                             const void* wq, const void* scale, const void* zero,
+                             const void* tile_indptr, const void* bucket_info,
+                             const void* packed_outliers, void* y_dev, void* Y_host, void* workspace,
+                             size_t workspace_bytes, void* cuda_stream);
+
+/* Synchronise the stream and return the scratch's status word: FQ_OK, or
+ * FQ_ERR_TIMEOUT if a bounded wait expired in a kernel (Y is then undefined);
+ * the word is cleared. */
+fq_status_t fq_check_status(void* workspace, void* cuda_stream);
+
+/* Thread-local description of the most recent error; valid until the next call. */
+const char* fq_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FQ_H_ */

@@ -1,0 +1,419 @@
+// Host side of the library: layout choice, INT4 group quantiser + packer (Eq. 2, Eq. 3),
+// Tile-COO encoder / decoder / validator (Section 3.2).  Plain C++, no CUDA.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <queue>
+#include <vector>
+
+#include "fq_internal.h"
+
+namespace fq {
+char* error_buffer() {
+    static thread_local char buf[512] = {0};
+    return buf;
+}
+
+static inline uint16_t f32_to_bf16_rne(float f) {
+    uint32_t u;
+    std::memcpy(&u, &f, 4);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x40u);
+    u += 0x7fffu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
+}
+static inline float bf16_to_f32(uint16_t h) {
+    uint32_t u = (uint32_t)h << 16;
+    float f;
+    std::memcpy(&f, &u, 4);
+    return f;
+}
+
+// Position of the code of (row kr, column cr) inside a 128 x BN chunk: word index and nibble.
+static inline void wq_slot(uint32_t kr, uint32_t cr, uint32_t& word, uint32_t& nib) {
+    const uint32_t w = cr >> 5, ns = (cr >> 4) & 1, rlo = (cr >> 3) & 1, grp = cr & 7;
+    const uint32_t kb = kr >> 5, t = (kr >> 3) & 3, odd = (kr >> 2) & 1, rhi = (kr >> 1) & 1, h = kr & 1;
+    const uint32_t ks = 2 * kb + odd;
+    const uint32_t j = ns * 2 + (ks >> 2), c = ks & 3, lane = grp * 4 + t;
+    word = ((w * 4 + j) * 32 + lane) * 4 + c;
+    nib = (rlo + 2 * rhi) + 4 * h;
+}
+}  // namespace fq
+
+using namespace fq;
+
+extern "C" {
+
+const char* fq_last_error(void) { return error_buffer(); }
+
+fq_status_t fq_get_layout(uint32_t K, uint32_t N, uint32_t group, uint32_t bn_hint, uint32_t nb_hint,
+                          fq_layout_t* out) {
+    if (!out) return fail(FQ_ERR_INVALID_ARG, "fq_get_layout: null output");
+    if (group != 64 && group != 128) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "group must be 64 or 128, got %u", group);
+    if (K == 0 || K % FQ_BK != 0) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "K = %u is not a multiple of 128", K);
+    uint32_t BN = bn_hint;
+    if (BN == 0) BN = (N % 256 == 0) ? 256 : 128;
+    if (BN != 128 && BN != 256) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "BN must be 128 or 256, got %u", BN);
+    if (N == 0 || N % BN != 0) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "N = %u is not a multiple of BN = %u", N, BN);
+    if (N / BN > kMaxTilesN) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "N = %u has too many column tiles", N);
+    uint32_t NB = nb_hint ? nb_hint : 32;
+    if (NB != 32 && NB != 64 && NB != 128) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "buckets per tile must be 32, 64 or 128, got %u", NB);
+    std::memset(out, 0, sizeof(*out));
+    out->abi = FQ_ABI_VERSION;
+    out->K = K;
+    out->N = N;
+    out->group = group;
+    out->BK = FQ_BK;
+    out->BN = BN;
+    out->buckets_per_tile = NB;
+    out->wq_interleave = 1;
+    out->coo_unit_bytes = 16;
+    return FQ_OK;
+}
+
+fq_status_t fq_pack_int4_sizes(const fq_layout_t* L, size_t* wq_bytes, size_t* scale_bytes, size_t* zero_bytes) {
+    if (!layout_ok(L)) return fail(FQ_ERR_INVALID_ARG, "bad layout");
+    if (wq_bytes) *wq_bytes = (size_t)L->K * L->N / 2;
+    if (scale_bytes) *scale_bytes = (size_t)(L->K / L->group) * L->N * 2;
+    if (zero_bytes) *zero_bytes = (size_t)(L->K / L->group) * L->N * 2;
+    return FQ_OK;
+}
+
+fq_status_t fq_pack_int4(const fq_layout_t* L, const float* W, const uint8_t* mask, void* wq_out,
+                         uint16_t* scale, uint16_t* zero) {
+    if (!layout_ok(L)) return fail(FQ_ERR_INVALID_ARG, "bad layout");
+    if (!W || !wq_out || !scale || !zero) return fail(FQ_ERR_INVALID_ARG, "fq_pack_int4: null pointer");
+    const uint32_t K = L->K, N = L->N, g = L->group, BN = L->BN;
+    const uint32_t KT = K / FQ_BK, NT = N / BN, gpc = FQ_BK / g;  // groups per chunk
+    uint32_t* wq = (uint32_t*)wq_out;
+    const size_t chunk_words = (size_t)16 * BN;
+#pragma omp parallel
+    {
+        std::vector<float> wmin(BN), wmax(BN), sf(BN);
+        std::vector<int> zz(BN);
+#pragma omp for schedule(dynamic, 4)
+        for (int64_t ch = 0; ch < (int64_t)NT * KT; ++ch) {
+            const uint32_t tn = (uint32_t)(ch / KT), kt = (uint32_t)(ch % KT);
+            uint32_t* chunk = wq + (size_t)ch * chunk_words;
+            std::memset(chunk, 0, chunk_words * 4);
+            const size_t n0 = (size_t)tn * BN;
+            for (uint32_t gi = 0; gi < gpc; ++gi) {
+                const uint32_t k0 = kt * FQ_BK + gi * g;
+                const size_t grow = (size_t)(k0 / g);
+                std::fill(wmin.begin(), wmin.end(), 0.0f);  // the range always contains 0
+                std::fill(wmax.begin(), wmax.end(), 0.0f);
+                for (uint32_t k = k0; k < k0 + g; ++k) {
+                    const float* wr = W + (size_t)k * N + n0;
+                    const uint8_t* mr = mask ? mask + (size_t)k * N + n0 : nullptr;
+                    for (uint32_t c = 0; c < BN; ++c) {
+                        if (mr && mr[c]) continue;
+                        float w = wr[c];
+                        if (w < wmin[c]) wmin[c] = w;
+                        if (w > wmax[c]) wmax[c] = w;
+                    }
+                }
+                for (uint32_t c = 0; c < BN; ++c) {
+                    float s32 = (wmax[c] - wmin[c]) / 15.0f;
+                    uint16_t sb = f32_to_bf16_rne(s32);
+                    float s = bf16_to_f32(sb);
+                    int z = 0;
+                    if (!(s > 0.0f)) {  // degenerate group
+                        sb = f32_to_bf16_rne(1.0f);
+                        s = 0.0f;       // marks "all codes 0" below
+                    } else {
+                        z = (int)nearbyintf(-wmin[c] / s);
+                        z = z < 0 ? 0 : (z > 15 ? 15 : z);
+                    }
+                    sf[c] = s;
+                    zz[c] = z;
+                    scale[grow * N + n0 + c] = sb;
+                    zero[grow * N + n0 + c] = f32_to_bf16_rne((float)z);
+                }
+                for (uint32_t k = k0; k < k0 + g; ++k) {
+                    const float* wr = W + (size_t)k * N + n0;
+                    const uint8_t* mr = mask ? mask + (size_t)k * N + n0 : nullptr;
+                    const uint32_t kr = k - kt * FQ_BK;
+                    for (uint32_t c = 0; c < BN; ++c) {
+                        int q;
+                        if (sf[c] == 0.0f) {
+                            q = 0;
+                        } else if (mr && mr[c]) {
+                            q = zz[c];
+                        } else {
+                            q = (int)nearbyintf(wr[c] / sf[c]) + zz[c];
+                            q = q < 0 ? 0 : (q > 15 ? 15 : q);
+                        }
+                        uint32_t word, nib;
+                        wq_slot(kr, c, word, nib);
+                        chunk[word] |= (uint32_t)q << (4 * nib);
+                    }
+                }
+            }
+        }
+    }
+    return FQ_OK;
+}
+
+fq_status_t fq_unpack_int4(const fq_layout_t* L, const void* wq_in, uint8_t* q) {
+    if (!layout_ok(L)) return fail(FQ_ERR_INVALID_ARG, "bad layout");
+    if (!wq_in || !q) return fail(FQ_ERR_INVALID_ARG, "fq_unpack_int4: null pointer");
+    const uint32_t K = L->K, N = L->N, BN = L->BN, KT = K / FQ_BK, NT = N / BN;
+    const uint32_t* wq = (const uint32_t*)wq_in;
+#pragma omp parallel for schedule(static)
+    for (int64_t ch = 0; ch < (int64_t)NT * KT; ++ch) {
+        const uint32_t tn = (uint32_t)(ch / KT), kt = (uint32_t)(ch % KT);
+        const uint32_t* chunk = wq + (size_t)ch * 16 * BN;
+        for (uint32_t kr = 0; kr < FQ_BK; ++kr)
+            for (uint32_t c = 0; c < BN; ++c) {
+                uint32_t word, nib;
+                wq_slot(kr, c, word, nib);
+                q[(size_t)(kt * FQ_BK + kr) * N + (size_t)tn * BN + c] = (uint8_t)((chunk[word] >> (4 * nib)) & 0xf);
+            }
+    }
+    return FQ_OK;
+}
+
+}  // extern "C"
+
+// ------------------------------------------------------------------ Tile-COO encoder
+
+namespace {
+
+struct Entry {
+    uint8_t k, c;
+    uint16_t v;
+};
+
+struct Encoded {
+    std::vector<uint32_t> indptr;   // N_tile + 1
+    std::vector<uint32_t> info;     // N_tile * NB
+    std::vector<uint8_t> packets;   // 16 * n_packets
+    uint32_t max_tile_packets = 0;
+};
+
+// Order one bucket's entries: position i of bucket b prefers bank group (i + b) % 8, where an
+// entry's bank group is k % 8 (one 16-byte row of the transposed activation copy per k).
+void order_bucket(std::vector<Entry>& e, uint32_t b, std::vector<Entry>& out) {
+    std::vector<Entry> grp[8];
+    for (const Entry& x : e) grp[x.k & 7].push_back(x);
+    size_t head[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    out.clear();
+    for (size_t i = 0; i < e.size(); ++i) {
+        uint32_t want = (uint32_t)((i + b) & 7);
+        for (uint32_t d = 0; d < 8; ++d) {
+            uint32_t gsel = (want + d) & 7;
+            if (head[gsel] < grp[gsel].size()) {
+                out.push_back(grp[gsel][head[gsel]++]);
+                break;
+            }
+        }
+    }
+}
+
+fq_status_t encode_impl(const fq_layout_t* L, const uint32_t* k, const uint32_t* n, const uint16_t* v,
+                        size_t nnz, Encoded& E) {
+    const uint32_t K = L->K, N = L->N, BN = L->BN, NB = L->buckets_per_tile;
+    const uint32_t KT = K / FQ_BK, NT = N / BN;
+    const size_t ntile = (size_t)KT * NT;
+    // counting sort of the entries by tile
+    std::vector<size_t> tstart(ntile + 1, 0);
+    for (size_t e = 0; e < nnz; ++e) {
+        if (k[e] >= K || n[e] >= N) return fq::fail(FQ_ERR_INVALID_ARG, "outlier %zu at (%u, %u) is outside the %u x %u matrix", e, k[e], n[e], K, N);
+        if ((v[e] & 0x7fffu) == 0) continue;  // +-0 is not an outlier
+        size_t t = (size_t)(n[e] / BN) * KT + k[e] / FQ_BK;
+        ++tstart[t + 1];
+    }
+    for (size_t t = 0; t < ntile; ++t) tstart[t + 1] += tstart[t];
+    std::vector<Entry> sorted(tstart[ntile]);
+    {
+        std::vector<size_t> fill(tstart.begin(), tstart.end() - 1);
+        for (size_t e = 0; e < nnz; ++e) {
+            if ((v[e] & 0x7fffu) == 0) continue;
+            size_t t = (size_t)(n[e] / BN) * KT + k[e] / FQ_BK;
+            sorted[fill[t]++] = Entry{(uint8_t)(k[e] % FQ_BK), (uint8_t)(n[e] % BN), v[e]};
+        }
+    }
+    // pass 1: per tile, packets per bucket
+    E.indptr.assign(ntile + 1, 0);
+    E.info.assign(ntile * NB, 0);
+    std::vector<uint8_t> col2bucket(ntile * BN);  // kept for pass 2
+    int bad = 0;
+#pragma omp parallel for schedule(dynamic, 16)
+    for (int64_t t = 0; t < (int64_t)ntile; ++t) {
+        uint32_t cnt[256] = {0};
+        for (size_t e = tstart[t]; e < tstart[t + 1]; ++e) ++cnt[sorted[e].c];
+        // columns by descending count (ties: lower column first), then least-loaded bucket
+        // (ties: lower bucket id) -- the greedy longest-processing-time rule
+        uint32_t order[256];
+        for (uint32_t c = 0; c < BN; ++c) order[c] = c;
+        std::stable_sort(order, order + BN, [&](uint32_t a, uint32_t b) { return cnt[a] > cnt[b]; });
+        typedef std::pair<uint32_t, uint32_t> LB;  // (load, bucket)
+        std::priority_queue<LB, std::vector<LB>, std::greater<LB>> heap;
+        for (uint32_t b = 0; b < NB; ++b) heap.push(LB(0, b));
+        uint32_t load[128] = {0};
+        uint8_t* c2b = &col2bucket[(size_t)t * BN];
+        for (uint32_t i = 0; i < BN; ++i) {
+            uint32_t c = order[i];
+            if (cnt[c] == 0) { c2b[c] = (uint8_t)(c % NB); continue; }
+            LB top = heap.top();
+            heap.pop();
+            c2b[c] = (uint8_t)top.second;
+            load[top.second] += cnt[c];
+            heap.push(LB(top.first + cnt[c], top.second));
+        }
+        uint32_t off = 0;
+        for (uint32_t b = 0; b < NB; ++b) {
+            uint32_t pk = (load[b] + 3) / 4;
+            if (off > 0xffffu || pk > 0xffffu) {
+#pragma omp atomic write
+                bad = 1;
+            }
+            E.info[(size_t)t * NB + b] = (off & 0xffffu) | (pk << 16);
+            off += pk;
+        }
+        E.indptr[t + 1] = off;
+    }
+    if (bad) return fq::fail(FQ_ERR_UNSUPPORTED_SHAPE, "a bucket exceeds the 16-bit packet offset/count range");
+    uint64_t total = 0;
+    for (size_t t = 0; t < ntile; ++t) {
+        uint32_t c = E.indptr[t + 1];
+        E.max_tile_packets = std::max(E.max_tile_packets, c);
+        total += c;
+        if (total > 0xffffffffull) return fq::fail(FQ_ERR_UNSUPPORTED_SHAPE, "more than 2^32 packets");
+        E.indptr[t + 1] = (uint32_t)total;
+    }
+    E.packets.assign((size_t)total * 16, 0);
+    // pass 2: order and write the packets
+#pragma omp parallel
+    {
+        std::vector<std::vector<Entry>> per(NB);
+        std::vector<Entry> ordered;
+#pragma omp for schedule(dynamic, 16)
+        for (int64_t t = 0; t < (int64_t)ntile; ++t) {
+            if (tstart[t] == tstart[t + 1]) continue;
+            for (auto& p : per) p.clear();
+            const uint8_t* c2b = &col2bucket[(size_t)t * BN];
+            for (size_t e = tstart[t]; e < tstart[t + 1]; ++e) per[c2b[sorted[e].c]].push_back(sorted[e]);
+            for (uint32_t b = 0; b < NB; ++b) {
+                if (per[b].empty()) continue;
+                // deterministic input order: by column, then row
+                std::sort(per[b].begin(), per[b].end(), [](const Entry& a, const Entry& c) {
+                    return a.c != c.c ? a.c < c.c : a.k < c.k;
+                });
+                order_bucket(per[b], b, ordered);
+                uint32_t info = E.info[(size_t)t * NB + b];
+                uint8_t* dst = &E.packets[((size_t)E.indptr[t] + (info & 0xffffu)) * 16];
+                const size_t cntp = info >> 16;
+                for (size_t s = 0; s < cntp * 4; ++s) {
+                    const bool real = s < ordered.size();
+                    const Entry& x = real ? ordered[s] : ordered.back();
+                    uint8_t* pk = dst + (s / 4) * 16;
+                    pk[s % 4] = x.k;
+                    pk[4 + s % 4] = x.c;
+                    uint16_t vv = real ? x.v : 0;
+                    pk[8 + 2 * (s % 4)] = (uint8_t)(vv & 0xff);
+                    pk[9 + 2 * (s % 4)] = (uint8_t)(vv >> 8);
+                }
+            }
+        }
+    }
+    return FQ_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+fq_status_t fq_encode_tilecoo_sizes(const fq_layout_t* L, const uint32_t* k, const uint32_t* n,
+                                    const uint16_t* v, size_t nnz, size_t* n_indptr, size_t* n_bucket_info,
+                                    size_t* n_packets, uint32_t* max_tile_packets) {
+    if (!layout_ok(L)) return fail(FQ_ERR_INVALID_ARG, "bad layout");
+    if (nnz && (!k || !n || !v)) return fail(FQ_ERR_INVALID_ARG, "fq_encode_tilecoo_sizes: null pointer");
+    Encoded E;
+    fq_status_t st = encode_impl(L, k, n, v, nnz, E);
+    if (st != FQ_OK) return st;
+    if (n_indptr) *n_indptr = E.indptr.size();
+    if (n_bucket_info) *n_bucket_info = E.info.size();
+    if (n_packets) *n_packets = E.packets.size() / 16;
+    if (max_tile_packets) *max_tile_packets = E.max_tile_packets;
+    return FQ_OK;
+}
+
+fq_status_t fq_encode_tilecoo(fq_layout_t* L, const uint32_t* k, const uint32_t* n, const uint16_t* v,
+                              size_t nnz, uint32_t* tile_indptr, uint32_t* bucket_info, void* packed,
+                              size_t n_packets) {
+    if (!layout_ok(L)) return fail(FQ_ERR_INVALID_ARG, "bad layout");
+    if ((nnz && (!k || !n || !v)) || !tile_indptr || !bucket_info) return fail(FQ_ERR_INVALID_ARG, "fq_encode_tilecoo: null pointer");
+    Encoded E;
+    fq_status_t st = encode_impl(L, k, n, v, nnz, E);
+    if (st != FQ_OK) return st;
+    if (E.packets.size() / 16 > n_packets) return fail(FQ_ERR_BUFFER_TOO_SMALL, "packed_outliers holds %zu packets, %zu needed", n_packets, E.packets.size() / 16);
+    if (!E.packets.empty() && !packed) return fail(FQ_ERR_INVALID_ARG, "fq_encode_tilecoo: null packet buffer");
+    std::memcpy(tile_indptr, E.indptr.data(), E.indptr.size() * 4);
+    std::memcpy(bucket_info, E.info.data(), E.info.size() * 4);
+    if (!E.packets.empty()) std::memcpy(packed, E.packets.data(), E.packets.size());
+    L->max_tile_packets = E.max_tile_packets;
+    return FQ_OK;
+}
+
+fq_status_t fq_decode_tilecoo(const fq_layout_t* L, const uint32_t* indptr, const uint32_t* info,
+                              const void* packed, uint32_t* k, uint32_t* n, uint16_t* v, size_t* nnz_inout) {
+    if (!layout_ok(L)) return fail(FQ_ERR_INVALID_ARG, "bad layout");
+    if (!indptr || !info || !nnz_inout) return fail(FQ_ERR_INVALID_ARG, "fq_decode_tilecoo: null pointer");
+    const uint32_t BN = L->BN, NB = L->buckets_per_tile, KT = L->K / FQ_BK, NT = L->N / BN;
+    const uint8_t* pk = (const uint8_t*)packed;
+    const size_t cap = *nnz_inout;
+    size_t c = 0;
+    for (uint32_t tn = 0; tn < NT; ++tn)
+        for (uint32_t kt = 0; kt < KT; ++kt) {
+            size_t t = (size_t)tn * KT + kt;
+            for (uint32_t b = 0; b < NB; ++b) {
+                uint32_t i0 = indptr[t] + (info[t * NB + b] & 0xffffu), cnt = info[t * NB + b] >> 16;
+                for (uint32_t i = 0; i < cnt; ++i)
+                    for (int s = 0; s < 4; ++s) {
+                        const uint8_t* p = pk + (size_t)(i0 + i) * 16;
+                        uint16_t val = (uint16_t)(p[8 + 2 * s] | (p[9 + 2 * s] << 8));
+                        if (val == 0) continue;
+                        if (c >= cap) return fail(FQ_ERR_BUFFER_TOO_SMALL, "decode buffer holds %zu entries", cap);
+                        k[c] = kt * FQ_BK + p[s];
+                        n[c] = tn * BN + p[4 + s];
+                        v[c] = val;
+                        ++c;
+                    }
+            }
+        }
+    *nnz_inout = c;
+    return FQ_OK;
+}
+
+fq_status_t fq_validate_tilecoo(const fq_layout_t* L, const uint32_t* indptr, const uint32_t* info,
+                                const void* packed, size_t n_packets) {
+    if (!layout_ok(L)) return fail(FQ_ERR_INVALID_ARG, "bad layout");
+    if (!indptr || !info || (n_packets && !packed)) return fail(FQ_ERR_INVALID_ARG, "fq_validate_tilecoo: null pointer");
+    const uint32_t BN = L->BN, NB = L->buckets_per_tile;
+    const size_t ntile = (size_t)(L->K / FQ_BK) * (L->N / BN);
+    const uint8_t* pk = (const uint8_t*)packed;
+    if (indptr[0] != 0) return fail(FQ_ERR_FORMAT, "tile_indptr[0] = %u, expected 0", indptr[0]);
+    for (size_t t = 0; t < ntile; ++t) {
+        if (indptr[t + 1] < indptr[t]) return fail(FQ_ERR_FORMAT, "tile_indptr decreases at tile %zu", t);
+        const uint32_t tile_pk = indptr[t + 1] - indptr[t];
+        if ((size_t)indptr[t + 1] > n_packets) return fail(FQ_ERR_FORMAT, "tile %zu ends at packet %u of %zu", t, indptr[t + 1], n_packets);
+        int16_t owner[256];
+        for (uint32_t c = 0; c < BN; ++c) owner[c] = -1;
+        for (uint32_t b = 0; b < NB; ++b) {
+            uint32_t off = info[t * NB + b] & 0xffffu, cnt = info[t * NB + b] >> 16;
+            if (off + cnt > tile_pk) return fail(FQ_ERR_FORMAT, "bucket %u of tile %zu covers packets [%u, %u) of %u", b, t, off, off + cnt, tile_pk);
+            for (uint32_t i = 0; i < cnt; ++i) {
+                const uint8_t* p = pk + (size_t)(indptr[t] + off + i) * 16;
+                for (int s = 0; s < 4; ++s) {
+                    if (p[s] >= FQ_BK || p[4 + s] >= BN) return fail(FQ_ERR_FORMAT, "index (%u, %u) outside the tile in tile %zu", p[s], p[4 + s], t);
+                    if (owner[p[4 + s]] >= 0 && owner[p[4 + s]] != (int16_t)b) return fail(FQ_ERR_FORMAT, "column %u of tile %zu appears in buckets %d and %u", p[4 + s], t, owner[p[4 + s]], b);
+                    owner[p[4 + s]] = (int16_t)b;
+                }
+            }
+        }
+    }
+    if ((size_t)indptr[ntile] != n_packets) return fail(FQ_ERR_FORMAT, "tile_indptr ends at %u, %zu packets given", indptr[ntile], n_packets);
+    return FQ_OK;
+}
+
+}  // extern "C"

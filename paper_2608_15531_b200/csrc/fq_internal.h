@@ -1,0 +1,37 @@
+// Internal declarations shared by the host packer/encoder and the CUDA launchers.
+#pragma once
+#include <cstdarg>
+#include <cstdint>
+#include <cstdio>
+
+#include "fq.h"
+
+namespace fq {
+
+// thread-local error text returned by fq_last_error()
+char* error_buffer();
+inline fq_status_t fail(fq_status_t code, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(error_buffer(), 512, fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+inline bool layout_ok(const fq_layout_t* L) {
+    if (!L || L->abi != FQ_ABI_VERSION) return false;
+    if (L->BK != FQ_BK || (L->BN != 128 && L->BN != 256)) return false;
+    if (L->group != 64 && L->group != 128) return false;
+    if (L->K == 0 || L->N == 0 || L->K % FQ_BK != 0 || L->N % L->BN != 0) return false;
+    if (L->buckets_per_tile != 32 && L->buckets_per_tile != 64 && L->buckets_per_tile != 128) return false;
+    if (L->wq_interleave != 1 || L->coo_unit_bytes != 16) return false;
+    return true;
+}
+
+// Upper bound on persistent CTAs per launch; sizes the scratch independently of the device.
+constexpr uint32_t kMaxCtas = 192;
+constexpr uint32_t kMaxTilesN = 2048;       // tile-arrival counters in the scratch
+constexpr size_t kWsHeaderBytes = 256;      // status word lives at offset 0
+constexpr size_t kWsCounterBytes = kMaxTilesN * 4;
+
+}  // namespace fq

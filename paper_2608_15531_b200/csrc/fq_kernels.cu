@@ -1,0 +1,771 @@
+// CUDA side of the library (sm_100a): the fused W4A16 + Tile-COO outlier decode matmul
+// (Eq. 1; Sections 3.1, 4.1, 4.2), its two unfused baselines and the launchers behind the C ABI.
+//
+// Kernel shape (one persistent CTA per SM):
+//   warp 0            producer: per (tile, k-step) unit, bulk-copies (cp.async.bulk + mbarrier
+//                     expect_tx) the unit's INT4 chunk, scale/zero rows, bucket_info slice, packet
+//                     range and the M activation rows into a ring of shared-memory stages
+//   warps 1..NDW      dense: each owns 32 output columns; one 32-bit word = one m16n8k16 A
+//                     fragment of codes, turned into BF16 (128 + q) with lop3 and fed to mma.sync
+//                     with the activations as the B operand; an all-ones A fragment yields the
+//                     per-group activation sums, so zero-point and scale are applied once per group
+//                     in FP32:  acc += s * (sum x (128+q) - (128+z) sum x)
+//   remaining warps   sparse: lane = bucket; transposes the activation tile to k-major, then for
+//                     each packet slot adds v * x[0..7][k] into the FP32 tile sh_c[col][m]
+//                     (buckets own disjoint columns, so no atomics)
+// Units are split over CTAs as contiguous ranges (stream-K).  A tile whose k-range is shared by
+// several CTAs is finished by the last CTA to arrive, which adds the FP32 partials in CTA order.
+// Every wait is bounded: on expiry the CTA raises the scratch status word and leaves.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstring>
+#include <mutex>
+
+#include "fq_internal.h"
+
+namespace fq {
+
+constexpr int kBK = 128;
+constexpr int kXRowBytes = 320;        // 256 B of activations + 64 B pad: conflict-free 16-byte fragment loads
+constexpr int kSmemBudget = 232448;    // 227 KB per CTA on sm_100
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+struct Params {
+    const uint16_t* X;
+    const uint8_t* wq;
+    const uint16_t* scale;
+    const uint16_t* zero;
+    const uint32_t* indptr;
+    const uint32_t* info;
+    const uint4* packed;
+    uint16_t* Y;
+    uint32_t* status;
+    uint32_t* counters;
+    float* partials;
+    uint32_t M, K, N, KT, NT;
+    uint32_t NB, coo_cap, stages, nsw;
+    // shared-memory offsets (bytes)
+    uint32_t stage_bytes, off_sz, off_x, off_info, off_coo;
+    uint32_t off_shc, off_xt, off_bar;
+};
+
+// ----------------------------------------------------------------------------- PTX helpers
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.shared::cta.b64 st, [%0];\n}" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n}" ::"r"(bar), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: false if this CTA is giving up (its own limit expired, or another warp's did).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          uint32_t* status) {
+    uint32_t spins = 0;
+    unsigned long long t0 = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 0xff) == 0) {
+            if (*abort_flag) return false;
+            unsigned long long now = globaltimer_ns();
+            if (t0 == 0) {
+                t0 = now;
+            } else if (now - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                atomicExch(status, (uint32_t)FQ_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// (w >> sh) & 0x000f000f | 0x43004300: two codes -> two BF16 values 128 + q
+__device__ __forceinline__ uint32_t codes_to_bf16x2(uint32_t w) {
+    uint32_t r;
+    asm("lop3.b32 %0, %1, 0x000f000f, 0x43004300, 0xea;" : "=r"(r) : "r"(w));
+    return r;
+}
+__device__ __forceinline__ float bf16lo(uint32_t v) { return __uint_as_float(v << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
+__device__ __forceinline__ float bf16_bits_to_float(uint16_t v) { return __uint_as_float((uint32_t)v << 16); }
+__device__ __forceinline__ uint16_t float_to_bf16_bits(float f) {
+    return __bfloat16_as_ushort(__float2bfloat16_rn(f));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr));
+}
+
+// Which CTA owns unit u when U units are dealt out as contiguous ranges, the first r CTAs one longer.
+__device__ __forceinline__ uint32_t cta_of_unit(uint32_t u, uint32_t q, uint32_t r) {
+    const uint32_t big = r * (q + 1);
+    return u < big ? u / (q + 1) : r + (u - big) / q;
+}
+__device__ __forceinline__ uint32_t unit_begin_of(uint32_t c, uint32_t q, uint32_t r) { return c * q + min(c, r); }
+
+// ----------------------------------------------------------------------------- sparse step
+
+// One bucket's packets against the k-major activation copy xt ([128][8] BF16, 16 B per row):
+// shc[col * ldc + 0..7] += v * x[0..7][k] for each slot (Section 4.2, without the per-column
+// padding: every slot carries its own column byte).
+__device__ __forceinline__ void apply_packet(const uint4 pk, const uint8_t* xt, float* shc_oct, uint32_t ldc) {
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+        const uint32_t k = (pk.x >> (8 * s)) & 0xffu;
+        const uint32_t c = (pk.y >> (8 * s)) & 0xffu;
+        const uint32_t vw = (s < 2) ? pk.z : pk.w;
+        const float v = (s & 1) ? bf16hi(vw) : bf16lo(vw);
+        const uint4 xv = *reinterpret_cast<const uint4*>(xt + k * 16);
+        float4* cp = reinterpret_cast<float4*>(shc_oct + c * ldc);
+        float4 c0 = cp[0], c1 = cp[1];
+        c0.x = fmaf(v, bf16lo(xv.x), c0.x);
+        c0.y = fmaf(v, bf16hi(xv.x), c0.y);
+        c0.z = fmaf(v, bf16lo(xv.y), c0.z);
+        c0.w = fmaf(v, bf16hi(xv.y), c0.w);
+        c1.x = fmaf(v, bf16lo(xv.z), c1.x);
+        c1.y = fmaf(v, bf16hi(xv.z), c1.y);
+        c1.z = fmaf(v, bf16lo(xv.w), c1.z);
+        c1.w = fmaf(v, bf16hi(xv.w), c1.w);
+        cp[0] = c0;
+        cp[1] = c1;
+    }
+}
+
+// Transpose 8 activation rows (row-major, kXRowBytes apart, 128 k each) into xt[k][8].
+__device__ __forceinline__ void transpose_octet(uint32_t xs_rows_u32, uint8_t* xt, int lane) {
+#pragma unroll
+    for (int kb = 0; kb < 4; ++kb) {
+        uint32_t r0, r1, r2, r3;
+        const uint32_t addr = xs_rows_u32 + (lane & 7) * kXRowBytes + (kb * 4 + (lane >> 3)) * 16;
+        ldmatrix_x4_trans(addr, r0, r1, r2, r3);
+        // thread T holds rows m = 2(T%4), 2(T%4)+1 of column k = 8*block + T/4
+        uint8_t* dst = xt + ((kb * 32) + (lane >> 2)) * 16 + (lane & 3) * 4;
+        *reinterpret_cast<uint32_t*>(dst) = r0;
+        *reinterpret_cast<uint32_t*>(dst + 8 * 16) = r1;
+        *reinterpret_cast<uint32_t*>(dst + 16 * 16) = r2;
+        *reinterpret_cast<uint32_t*>(dst + 24 * 16) = r3;
+    }
+}
+
+// ----------------------------------------------------------------------------- fused kernel
+
+template <int BN, int MO, int GROUP, bool SPARSE>
+__global__ void __launch_bounds__(32 * (1 + BN / 32 + 8), 1) fq_fused_kernel(const Params p) {
+    constexpr int NDW = BN / 32;
+    constexpr int GPS = kBK / GROUP;          // groups per k-step
+    constexpr int W_BYTES = 16 * BN * 4;
+    constexpr int SZ_ROW = BN * 2;
+    constexpr int LDC = 8 * MO;               // sh_c row: FP32 per batch row
+    extern __shared__ __align__(128) uint8_t smem[];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t S = p.stages;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
+    const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * S;
+    const uint32_t bar_sparse_done = bar_empty + 8 * S, bar_dense_done = bar_sparse_done + 8, bar_dense = bar_dense_done + 8;
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 2 * S + 3);
+    volatile uint32_t* last_flag = abort_flag + 1;
+    float* shc = reinterpret_cast<float*>(smem + p.off_shc);
+
+    const uint32_t nsw = SPARSE ? p.nsw : 0;
+    if (tid == 0) {
+        for (uint32_t s = 0; s < S; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, NDW + nsw);
+        }
+        mbar_init(bar_sparse_done, nsw ? nsw : 1);
+        mbar_init(bar_dense_done, NDW);
+        mbar_init(bar_dense, NDW);
+        *abort_flag = 0;
+        *last_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (SPARSE) {
+        for (uint32_t i = tid; i < (uint32_t)(BN * LDC); i += blockDim.x) shc[i] = 0.0f;
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncthreads();
+
+    // contiguous range of units for this CTA
+    const uint32_t U = p.NT * p.KT, P = gridDim.x, q = U / P, r = U % P;
+    const uint32_t u_begin = unit_begin_of(blockIdx.x, q, r);
+    const uint32_t u_end = u_begin + q + (blockIdx.x < r ? 1u : 0u);
+    const uint32_t KT = p.KT;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer
+        uint32_t ip_a = 0, ip_b = 0;
+        for (uint32_t u = u_begin, it = 0; u < u_end; ++u, ++it) {
+            const uint32_t s = it % S, ph = (it / S) & 1;
+            if (SPARSE && (it & 31) == 0) {  // this warp's next 32 packet ranges, one coalesced read
+                const uint32_t i = u + lane;
+                ip_a = (i <= U) ? __ldg(p.indptr + i) : 0;
+                ip_b = (i + 1 <= U) ? __ldg(p.indptr + i + 1) : 0;
+            }
+            uint32_t pk0 = 0, npk = 0;
+            if (SPARSE) {
+                pk0 = __shfl_sync(0xffffffffu, ip_a, it & 31);
+                npk = __shfl_sync(0xffffffffu, ip_b, it & 31) - pk0;
+                npk = min(npk, p.coo_cap);
+            }
+            if (!mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_flag, p.status)) {
+                // giving up: let the copies already issued land before the CTA's shared memory goes away
+                for (uint32_t j = (it > S ? it - S : 0); j < it; ++j)
+                    for (uint32_t spin = 0; spin < (1u << 20) && !mbar_try_wait(bar_full + 8 * (j % S), (j / S) & 1); ++spin) {}
+                return;
+            }
+            const uint32_t tn = u / KT, kt = u % KT;
+            const uint32_t full = bar_full + 8 * s;
+            const uint32_t st = smem_u32(smem) + s * p.stage_bytes;
+            if (lane == 0) {
+                uint32_t bytes = W_BYTES + 2 * GPS * SZ_ROW + p.M * 256;
+                if (SPARSE) bytes += p.NB * 4 + npk * 16;
+                mbar_arrive_expect_tx(full, bytes);
+            }
+            __syncwarp();
+            if (lane == 0) {
+                bulk_g2s(st, p.wq + (size_t)u * W_BYTES, W_BYTES, full);
+            } else if (lane == 1) {
+#pragma unroll
+                for (int gi = 0; gi < GPS; ++gi)
+                    bulk_g2s(st + p.off_sz + gi * SZ_ROW, p.scale + (size_t)(kt * GPS + gi) * p.N + (size_t)tn * BN, SZ_ROW, full);
+            } else if (lane == 2) {
+#pragma unroll
+                for (int gi = 0; gi < GPS; ++gi)
+                    bulk_g2s(st + p.off_sz + (GPS + gi) * SZ_ROW, p.zero + (size_t)(kt * GPS + gi) * p.N + (size_t)tn * BN, SZ_ROW, full);
+            } else if (lane == 3) {
+                if (SPARSE) bulk_g2s(st + p.off_info, p.info + (size_t)u * p.NB, p.NB * 4, full);
+            } else if (lane == 4) {
+                if (SPARSE && npk) bulk_g2s(st + p.off_coo, p.packed + pk0, npk * 16, full);
+            }
+            {
+                const uint32_t m = (lane + 27) & 31;  // rows start on lane 5
+                if (m < p.M) bulk_g2s(st + p.off_x + m * kXRowBytes, p.X + (size_t)m * p.K + (size_t)kt * kBK, 256, full);
+            }
+        }
+        return;
+    }
+
+    if (warp <= NDW) {
+        // ------------------------------------------------------------------ dense
+        const int dw = warp - 1, g = lane >> 2, t = lane & 3;
+        const int dtid = dw * 32 + lane;
+        float accf[2][MO][4];
+#pragma unroll
+        for (int a = 0; a < 2; ++a)
+#pragma unroll
+            for (int o = 0; o < MO; ++o)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) accf[a][o][i] = 0.0f;
+        const uint32_t ones[4] = {0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u};
+        uint32_t piece = 0, dense_phase = 0;
+
+        for (uint32_t u = u_begin, it = 0; u < u_end; ++u, ++it) {
+            const uint32_t s = it % S, ph = (it / S) & 1;
+            const uint32_t tn = u / KT, kt = u % KT;
+            const uint8_t* st = smem + s * p.stage_bytes;
+            if (!mbar_wait(bar_full + 8 * s, ph, abort_flag, p.status)) return;
+
+            const uint4* wp = reinterpret_cast<const uint4*>(st) + dw * 128 + lane;
+            uint4 wa[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) wa[j] = wp[j * 32];
+            const uint8_t* xrow = st + p.off_x + g * kXRowBytes + t * 16;
+            const uint16_t* sc = reinterpret_cast<const uint16_t*>(st + p.off_sz);
+
+#pragma unroll
+            for (int gi = 0; gi < GPS; ++gi) {
+                float accg[2][MO][4], xs[MO][4];
+#pragma unroll
+                for (int o = 0; o < MO; ++o)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        accg[0][o][i] = 0.0f;
+                        accg[1][o][i] = 0.0f;
+                        xs[o][i] = 0.0f;
+                    }
+#pragma unroll
+                for (int kb = gi * (4 / GPS); kb < (gi + 1) * (4 / GPS); ++kb) {
+                    uint4 xb[MO];
+#pragma unroll
+                    for (int o = 0; o < MO; ++o)
+                        xb[o] = *reinterpret_cast<const uint4*>(xrow + o * 8 * kXRowBytes + kb * 64);
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int ks = 2 * kb + e;
+#pragma unroll
+                        for (int ns = 0; ns < 2; ++ns) {
+                            const uint4 w4 = wa[ns * 2 + (ks >> 2)];
+                            const uint32_t w = (ks & 3) == 0 ? w4.x : (ks & 3) == 1 ? w4.y : (ks & 3) == 2 ? w4.z : w4.w;
+                            uint32_t a[4];
+                            a[0] = codes_to_bf16x2(w);
+                            a[1] = codes_to_bf16x2(w >> 4);
+                            a[2] = codes_to_bf16x2(w >> 8);
+                            a[3] = codes_to_bf16x2(w >> 12);
+#pragma unroll
+                            for (int o = 0; o < MO; ++o)
+                                mma_bf16(accg[ns][o], a, e ? xb[o].z : xb[o].x, e ? xb[o].w : xb[o].y);
+                        }
+#pragma unroll
+                        for (int o = 0; o < MO; ++o) mma_bf16(xs[o], ones, e ? xb[o].z : xb[o].x, e ? xb[o].w : xb[o].y);
+                    }
+                }
+                // once per group: acc += s * (sum x (128+q) - (128+z) sum x)     (Eq. 3 inside Eq. 1)
+#pragma unroll
+                for (int ns = 0; ns < 2; ++ns)
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int nl = dw * 32 + ns * 16 + h * 8 + g;
+                        const float sv = bf16_bits_to_float(sc[gi * BN + nl]);
+                        const float zc = -(128.0f + bf16_bits_to_float(sc[(GPS + gi) * BN + nl]));
+#pragma unroll
+                        for (int o = 0; o < MO; ++o) {
+                            accf[ns][o][2 * h + 0] = fmaf(sv, fmaf(zc, xs[o][0], accg[ns][o][2 * h + 0]), accf[ns][o][2 * h + 0]);
+                            accf[ns][o][2 * h + 1] = fmaf(sv, fmaf(zc, xs[o][1], accg[ns][o][2 * h + 1]), accf[ns][o][2 * h + 1]);
+                        }
+                    }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_empty + 8 * s);
+
+            if (kt == KT - 1 || u == u_end - 1) {
+                // ---------------------------------------------------------- end of a piece
+                if (SPARSE) {
+                    if (!mbar_wait(bar_sparse_done, piece & 1, abort_flag, p.status)) return;
+#pragma unroll
+                    for (int ns = 0; ns < 2; ++ns)
+#pragma unroll
+                        for (int h = 0; h < 2; ++h)
+#pragma unroll
+                            for (int o = 0; o < MO; ++o) {
+                                float2* cp = reinterpret_cast<float2*>(shc + (dw * 32 + ns * 16 + h * 8 + g) * LDC + o * 8 + 2 * t);
+                                const float2 v = *cp;
+                                accf[ns][o][2 * h + 0] += v.x;
+                                accf[ns][o][2 * h + 1] += v.y;
+                                *cp = make_float2(0.0f, 0.0f);
+                            }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_dense_done);
+                }
+                const uint32_t u_tile0 = tn * KT;
+                const uint32_t piece_k0 = max(u_tile0, u_begin) - u_tile0;
+                const bool full_piece = (piece_k0 == 0) && (kt == KT - 1);
+                bool write_y = full_piece;
+                if (!full_piece) {
+                    // FP32 partial in fragment order; the last CTA to arrive sums them in CTA order
+                    const uint32_t which = (u_begin / KT == tn) ? 0u : 1u;
+                    float* slot = p.partials + ((size_t)blockIdx.x * 2 + which) * (size_t)(BN * LDC);
+#pragma unroll
+                    for (int ns = 0; ns < 2; ++ns)
+#pragma unroll
+                        for (int o = 0; o < MO; ++o)
+#pragma unroll
+                            for (int i = 0; i < 4; ++i)
+                                __stcg(slot + (size_t)((ns * MO + o) * 4 + i) * (NDW * 32) + dtid, accf[ns][o][i]);
+                    __threadfence();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_dense);
+                    if (!mbar_wait(bar_dense, dense_phase & 1, abort_flag, p.status)) return;
+                    ++dense_phase;
+                    const uint32_t c_first = cta_of_unit(u_tile0, q, r), c_last = cta_of_unit(u_tile0 + KT - 1, q, r);
+                    if (dtid == 0) {
+                        const uint32_t old = atomicAdd(p.counters + tn, 1u);
+                        *last_flag = (old == c_last - c_first) ? 1u : 0u;
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_dense);
+                    if (!mbar_wait(bar_dense, dense_phase & 1, abort_flag, p.status)) return;
+                    ++dense_phase;
+                    if (*last_flag) {
+                        write_y = true;
+                        __threadfence();
+                        float tot[2][MO][4];
+#pragma unroll
+                        for (int ns = 0; ns < 2; ++ns)
+#pragma unroll
+                            for (int o = 0; o < MO; ++o)
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) tot[ns][o][i] = 0.0f;
+                        for (uint32_t c = c_first; c <= c_last; ++c) {
+                            const uint32_t wch = (unit_begin_of(c, q, r) / KT == tn) ? 0u : 1u;
+                            const float* sl = p.partials + ((size_t)c * 2 + wch) * (size_t)(BN * LDC);
+#pragma unroll
+                            for (int ns = 0; ns < 2; ++ns)
+#pragma unroll
+                                for (int o = 0; o < MO; ++o)
+#pragma unroll
+                                    for (int i = 0; i < 4; ++i)
+                                        tot[ns][o][i] += __ldcg(sl + (size_t)((ns * MO + o) * 4 + i) * (NDW * 32) + dtid);
+                        }
+#pragma unroll
+                        for (int ns = 0; ns < 2; ++ns)
+#pragma unroll
+                            for (int o = 0; o < MO; ++o)
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) accf[ns][o][i] = tot[ns][o][i];
+                        if (dtid == 0) p.counters[tn] = 0;  // ready for the next call
+                    }
+                }
+                if (write_y) {
+#pragma unroll
+                    for (int ns = 0; ns < 2; ++ns)
+#pragma unroll
+                        for (int h = 0; h < 2; ++h)
+#pragma unroll
+                            for (int o = 0; o < MO; ++o)
+#pragma unroll
+                                for (int j = 0; j < 2; ++j) {
+                                    const uint32_t m = o * 8 + 2 * t + j;
+                                    if (m < p.M)
+                                        p.Y[(size_t)m * p.N + (size_t)tn * BN + dw * 32 + ns * 16 + h * 8 + g] =
+                                            float_to_bf16_bits(accf[ns][o][2 * h + j]);
+                                }
+                }
+#pragma unroll
+                for (int ns = 0; ns < 2; ++ns)
+#pragma unroll
+                    for (int o = 0; o < MO; ++o)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) accf[ns][o][i] = 0.0f;
+                ++piece;
+            }
+        }
+        return;
+    }
+
+    if (SPARSE) {
+        // ------------------------------------------------------------------ sparse
+        const uint32_t sw = warp - 1 - NDW;
+        const uint32_t nbb = p.NB >> 5;            // blocks of 32 buckets
+        const uint32_t bb = sw % nbb, og = sw / nbb, n_og = nsw / nbb;
+        const uint32_t bucket = bb * 32 + lane;
+        uint8_t* xt = smem + p.off_xt + sw * 2048;
+        uint32_t piece = 0;
+        for (uint32_t u = u_begin, it = 0; u < u_end; ++u, ++it) {
+            const uint32_t s = it % S, ph = (it / S) & 1;
+            const uint32_t kt = u % KT;
+            const uint8_t* st = smem + s * p.stage_bytes;
+            if (!mbar_wait(bar_full + 8 * s, ph, abort_flag, p.status)) return;
+            const uint32_t info = reinterpret_cast<const uint32_t*>(st + p.off_info)[bucket];
+            const uint32_t off = info & 0xffffu, cnt = info >> 16;
+            const uint4* pk_s = reinterpret_cast<const uint4*>(st + p.off_coo);
+            const uint4* pk_g = nullptr;
+            if (off + cnt > p.coo_cap) pk_g = p.packed + __ldg(p.indptr + u);  // tail of an oversized tile
+            for (uint32_t o = og; o < (uint32_t)MO; o += n_og) {
+                transpose_octet(smem_u32(st + p.off_x) + o * 8 * kXRowBytes, xt, lane);
+                __syncwarp();
+                float* shc_o = shc + o * 8;
+                for (uint32_t i = 0; i < cnt; ++i) {
+                    const uint32_t idx = off + i;
+                    const uint4 pk = (idx < p.coo_cap) ? pk_s[idx] : __ldg(pk_g + idx);
+                    apply_packet(pk, xt, shc_o, LDC);
+                }
+                __syncwarp();
+            }
+            if (lane == 0) mbar_arrive(bar_empty + 8 * s);
+            if (kt == KT - 1 || u == u_end - 1) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_sparse_done);
+                if (!mbar_wait(bar_dense_done, piece & 1, abort_flag, p.status)) return;
+                ++piece;
+            }
+        }
+    }
+}
+
+// ----------------------------------------------------------------------------- unfused SpMM
+
+// Y += X * W_O as its own launch (the sparse half of the two-kernel baseline).  One CTA per column
+// tile walks all K/128 row tiles: stages the activation tile k-major in shared memory, applies the
+// tile's packets straight from global memory, and finally adds the FP32 tile to the BF16 Y.
+template <int BN>
+__global__ void __launch_bounds__(256) fq_spmm_kernel(const uint16_t* __restrict__ X, const uint32_t* __restrict__ indptr,
+                                                    const uint32_t* __restrict__ info, const uint4* __restrict__ packed,
+                                                    uint16_t* __restrict__ Y, uint32_t M, uint32_t K, uint32_t N,
+                                                    uint32_t NB, uint32_t MO) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    const uint32_t LDC = 8 * MO;
+    float* shc = reinterpret_cast<float*>(smem);                    // [BN][8 MO]
+    uint8_t* xt = smem + (size_t)BN * LDC * 4;                       // [MO][128][8] BF16
+    const uint32_t tn = blockIdx.x, KT = K / kBK;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (uint32_t i = tid; i < BN * LDC; i += blockDim.x) shc[i] = 0.0f;
+    for (uint32_t kt = 0; kt < KT; ++kt) {
+        __syncthreads();
+        // k-major copy of the activation tile, zero for rows >= M
+        for (uint32_t i = tid; i < 128 * LDC; i += blockDim.x) {
+            const uint32_t k = i / LDC, m = i % LDC;
+            const uint16_t v = (m < M) ? X[(size_t)m * K + (size_t)kt * kBK + k] : (uint16_t)0;
+            reinterpret_cast<uint16_t*>(xt)[((m >> 3) * 128 + k) * 8 + (m & 7)] = v;
+        }
+        __syncthreads();
+        const size_t t = (size_t)tn * KT + kt;
+        const uint4* pk = packed + indptr[t];
+        // (bucket block, octet) pairs dealt to the 8 warps
+        const uint32_t nbb = NB >> 5;
+        for (uint32_t w = warp; w < nbb * MO; w += 8) {
+            const uint32_t bb = w % nbb, o = w / nbb;
+            const uint32_t inf = info[t * NB + bb * 32 + lane];
+            const uint32_t off = inf & 0xffffu, cnt = inf >> 16;
+            for (uint32_t i = 0; i < cnt; ++i) apply_packet(__ldg(pk + off + i), xt + o * 2048, shc + o * 8, LDC);
+        }
+    }
+    __syncthreads();
+    for (uint32_t i = tid; i < BN * M; i += blockDim.x) {
+        const uint32_t m = i / BN, c = i % BN;
+        uint16_t* y = Y + (size_t)m * N + (size_t)tn * BN + c;
+        *y = float_to_bf16_bits(bf16_bits_to_float(*y) + shc[c * LDC + m]);
+    }
+}
+
+// ----------------------------------------------------------------------------- launch plumbing
+
+struct Plan {
+    Params p;
+    uint32_t threads, smem, grid;
+};
+
+static inline uint32_t round_up(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
+
+static int sm_count_cached() {
+    static int cached[64];
+    static std::once_flag once;
+    std::call_once(once, [] { std::memset(cached, 0, sizeof(cached)); });
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return -1;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -1;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
+static fq_status_t make_plan(const fq_layout_t* L, uint32_t M, bool sparse, Plan& pl) {
+    const uint32_t BN = L->BN, NB = L->buckets_per_tile, GPS = kBK / L->group;
+    const uint32_t MO = M <= 8 ? 1 : (M <= 16 ? 2 : 4);
+    const uint32_t NDW = BN / 32;
+    uint32_t nsw = 0;
+    if (sparse) nsw = std::min<uint32_t>(8, (NB / 32) * MO);
+    Params& p = pl.p;
+    std::memset(&p, 0, sizeof(p));
+    p.M = M; p.K = L->K; p.N = L->N; p.KT = L->K / kBK; p.NT = L->N / BN; p.NB = NB; p.nsw = nsw;
+    const uint32_t w_bytes = 16 * BN * 4, sz_bytes = 2 * GPS * BN * 2, x_bytes = 8 * MO * kXRowBytes;
+    const uint32_t fixed = (sparse ? BN * 8 * MO * 4 + nsw * 2048 : 0) + 1024;
+    uint32_t cap = 0;
+    if (sparse) {
+        cap = L->max_tile_packets ? round_up(L->max_tile_packets, 8) : 256;
+        cap = std::min<uint32_t>(cap, 1024);
+    }
+    uint32_t stage = 0, S = 0;
+    for (;;) {
+        p.off_sz = w_bytes;
+        p.off_x = p.off_sz + round_up(sz_bytes, 128);
+        p.off_info = p.off_x + round_up(x_bytes, 128);
+        p.off_coo = p.off_info + (sparse ? round_up(NB * 4, 128) : 0);
+        stage = p.off_coo + cap * 16;
+        stage = round_up(stage, 128);
+        S = std::min<uint32_t>(8, (kSmemBudget - fixed) / stage);
+        if (S >= 4 || cap <= 64) break;
+        cap = std::max<uint32_t>(64, cap / 2);  // oversized tiles read their tail from global memory
+    }
+    if (S < 2) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "shared-memory stages do not fit");
+    p.coo_cap = cap; p.stages = S; p.stage_bytes = stage;
+    p.off_shc = S * stage;
+    p.off_xt = p.off_shc + (sparse ? BN * 8 * MO * 4 : 0);
+    p.off_bar = p.off_xt + nsw * 2048;
+    pl.smem = p.off_bar + 1024;
+    pl.threads = 32 * (1 + NDW + nsw);
+    const int sms = sm_count_cached();
+    if (sms <= 0) return fail(FQ_ERR_CUDA, "no CUDA device: %s", cudaGetErrorString(cudaGetLastError()));
+    pl.grid = std::min<uint32_t>({(uint32_t)sms, kMaxCtas, p.NT * p.KT});
+    return FQ_OK;
+}
+
+typedef void (*KernelFn)(const Params);
+
+template <int BN, int MO, int G>
+static KernelFn pick_sparse(bool sparse) {
+    return sparse ? (KernelFn)fq_fused_kernel<BN, MO, G, true> : (KernelFn)fq_fused_kernel<BN, MO, G, false>;
+}
+template <int BN, int MO>
+static KernelFn pick_group(uint32_t g, bool sparse) {
+    return g == 64 ? pick_sparse<BN, MO, 64>(sparse) : pick_sparse<BN, MO, 128>(sparse);
+}
+template <int BN>
+static KernelFn pick_mo(uint32_t mo, uint32_t g, bool sparse) {
+    return mo == 1 ? pick_group<BN, 1>(g, sparse) : mo == 2 ? pick_group<BN, 2>(g, sparse) : pick_group<BN, 4>(g, sparse);
+}
+static KernelFn pick_kernel(uint32_t bn, uint32_t mo, uint32_t g, bool sparse) {
+    return bn == 128 ? pick_mo<128>(mo, g, sparse) : pick_mo<256>(mo, g, sparse);
+}
+
+static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, const void* wq, const void* scale,
+                               const void* zero, const void* indptr, const void* info, const void* packed, void* Y,
+                               void* workspace, size_t workspace_bytes, void* stream, bool sparse) {
+    if (!layout_ok(L)) return fail(FQ_ERR_INVALID_ARG, "bad layout");
+    if (M < 1 || M > FQ_MAX_M) return fail(FQ_ERR_INVALID_ARG, "M = %u outside [1, %u]", M, FQ_MAX_M);
+    if (!X || !wq || !scale || !zero || !Y || !workspace) return fail(FQ_ERR_INVALID_ARG, "null device pointer");
+    if (sparse && (!indptr || !info)) return fail(FQ_ERR_INVALID_ARG, "null Tile-COO pointer");
+    if (sparse && !packed && L->max_tile_packets) return fail(FQ_ERR_INVALID_ARG, "null packet pointer");
+    if (!aligned(X, 16) || !aligned(Y, 16) || !aligned(wq, 128) || !aligned(scale, 128) || !aligned(zero, 128) ||
+        !aligned(workspace, 128) || (sparse && (!aligned(indptr, 4) || !aligned(info, 128) || !aligned(packed, 128))))
+        return fail(FQ_ERR_INVALID_ARG, "misaligned device pointer");
+    size_t need = 0;
+    fq_status_t st = fq_workspace_bytes(L, M, &need);
+    if (st != FQ_OK) return st;
+    if (workspace_bytes < need) return fail(FQ_ERR_BUFFER_TOO_SMALL, "workspace holds %zu bytes, %zu needed", workspace_bytes, need);
+    for (uint32_t m0 = 0; m0 < M; m0 += 32) {
+        const uint32_t mb = std::min<uint32_t>(32, M - m0);
+        Plan pl;
+        st = make_plan(L, mb, sparse, pl);
+        if (st != FQ_OK) return st;
+        Params& p = pl.p;
+        p.X = (const uint16_t*)X + (size_t)m0 * L->K;
+        p.Y = (uint16_t*)Y + (size_t)m0 * L->N;
+        p.wq = (const uint8_t*)wq; p.scale = (const uint16_t*)scale; p.zero = (const uint16_t*)zero;
+        p.indptr = (const uint32_t*)indptr; p.info = (const uint32_t*)info; p.packed = (const uint4*)packed;
+        p.status = (uint32_t*)workspace;
+        p.counters = (uint32_t*)((uint8_t*)workspace + kWsHeaderBytes);
+        p.partials = (float*)((uint8_t*)workspace + kWsHeaderBytes + kWsCounterBytes);
+        const uint32_t MO = mb <= 8 ? 1 : (mb <= 16 ? 2 : 4);
+        KernelFn fn = pick_kernel(L->BN, MO, L->group, sparse);
+        cudaError_t e = cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget);
+        if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+        fn<<<pl.grid, pl.threads, pl.smem, (cudaStream_t)stream>>>(p);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
+    }
+    return FQ_OK;
+}
+
+}  // namespace fq
+
+using namespace fq;
+
+extern "C" {
+
+fq_status_t fq_workspace_bytes(const fq_layout_t* L, uint32_t M, size_t* bytes) {
+    if (!layout_ok(L) || !bytes) return fail(FQ_ERR_INVALID_ARG, "bad layout or null output");
+    if (M < 1 || M > FQ_MAX_M) return fail(FQ_ERR_INVALID_ARG, "M = %u outside [1, %u]", M, FQ_MAX_M);
+    const uint32_t mb = std::min<uint32_t>(M, 32);
+    const uint32_t MO = mb <= 8 ? 1 : (mb <= 16 ? 2 : 4);
+    *bytes = kWsHeaderBytes + kWsCounterBytes + (size_t)kMaxCtas * 2 * L->BN * 8 * MO * 4;
+    return FQ_OK;
+}
+
+fq_status_t fq_fused_w4a16_outlier_gemm(const fq_layout_t* L, const void* X, uint32_t M, const void* wq,
+                                        const void* scale, const void* zero, const void* tile_indptr,
+                                        const void* bucket_info, const void* packed_outliers, void* Y,
+                                        void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return launch_gemm(L, X, M, wq, scale, zero, tile_indptr, bucket_info, packed_outliers, Y, workspace,
+                       workspace_bytes, cuda_stream, true);
+}
+
+fq_status_t fq_unfused_gemm(const fq_layout_t* L, const void* X, uint32_t M, const void* wq, const void* scale,
+                            const void* zero, void* Y, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return launch_gemm(L, X, M, wq, scale, zero, nullptr, nullptr, nullptr, Y, workspace, workspace_bytes,
+                       cuda_stream, false);
+}
+
+fq_status_t fq_unfused_spmm(const fq_layout_t* L, const void* X, uint32_t M, const void* tile_indptr,
+                            const void* bucket_info, const void* packed_outliers, void* Y, void* cuda_stream) {
+    if (!layout_ok(L)) return fail(FQ_ERR_INVALID_ARG, "bad layout");
+    if (M < 1 || M > FQ_MAX_M) return fail(FQ_ERR_INVALID_ARG, "M = %u outside [1, %u]", M, FQ_MAX_M);
+    if (!X || !tile_indptr || !bucket_info || !Y) return fail(FQ_ERR_INVALID_ARG, "null device pointer");
+    if (!packed_outliers && L->max_tile_packets) return fail(FQ_ERR_INVALID_ARG, "null packet pointer");
+    for (uint32_t m0 = 0; m0 < M; m0 += 32) {
+        const uint32_t mb = std::min<uint32_t>(32, M - m0);
+        const uint32_t MO = (mb + 7) / 8;
+        const size_t smem = (size_t)L->BN * 8 * MO * 4 + (size_t)MO * 2048;
+        const uint16_t* x = (const uint16_t*)X + (size_t)m0 * L->K;
+        uint16_t* y = (uint16_t*)Y + (size_t)m0 * L->N;
+        cudaError_t e;
+        if (L->BN == 128) {
+            e = cudaFuncSetAttribute((const void*)fq_spmm_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 65536);
+            if (e == cudaSuccess)
+                fq_spmm_kernel<128><<<L->N / 128, 256, smem, (cudaStream_t)cuda_stream>>>(
+                    x, (const uint32_t*)tile_indptr, (const uint32_t*)bucket_info, (const uint4*)packed_outliers, y, mb,
+                    L->K, L->N, L->buckets_per_tile, MO);
+        } else {
+            e = cudaFuncSetAttribute((const void*)fq_spmm_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, 65536);
+            if (e == cudaSuccess)
+                fq_spmm_kernel<256><<<L->N / 256, 256, smem, (cudaStream_t)cuda_stream>>>(
+                    x, (const uint32_t*)tile_indptr, (const uint32_t*)bucket_info, (const uint4*)packed_outliers, y, mb,
+                    L->K, L->N, L->buckets_per_tile, MO);
+        }
+        if (e == cudaSuccess) e = cudaGetLastError();
+        if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "spmm launch: %s", cudaGetErrorString(e));
+    }
+    return FQ_OK;
+}
+
+fq_status_t fq_fused_host_io(const fq_layout_t* L, const void* X_host, uint32_t M, void* x_dev, const void* wq,
+                             const void* scale, const void* zero, const void* tile_indptr, const void* bucket_info,
+                             const void* packed_outliers, void* y_dev, void* Y_host, void* workspace,
+                             size_t workspace_bytes, void* cuda_stream) {
+    if (!layout_ok(L)) return fail(FQ_ERR_INVALID_ARG, "bad layout");
+    if (!X_host || !Y_host || !x_dev || !y_dev) return fail(FQ_ERR_INVALID_ARG, "null pointer");
+    if (M < 1 || M > FQ_MAX_M) return fail(FQ_ERR_INVALID_ARG, "M = %u outside [1, %u]", M, FQ_MAX_M);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    cudaError_t e = cudaMemcpyAsync(x_dev, X_host, (size_t)M * L->K * 2, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "copy of X: %s", cudaGetErrorString(e));
+    fq_status_t st = fq_fused_w4a16_outlier_gemm(L, x_dev, M, wq, scale, zero, tile_indptr, bucket_info,
+                                                 packed_outliers, y_dev, workspace, workspace_bytes, cuda_stream);
+    if (st != FQ_OK) return st;
+    e = cudaMemcpyAsync(Y_host, y_dev, (size_t)M * L->N * 2, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "copy of Y: %s", cudaGetErrorString(e));
+    return FQ_OK;
+}
+
+fq_status_t fq_check_status(void* workspace, void* cuda_stream) {
+    if (!workspace) return fail(FQ_ERR_INVALID_ARG, "null workspace");
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    uint32_t word = 0;
+    cudaError_t e = cudaMemcpyAsync(&word, workspace, 4, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "status read: %s", cudaGetErrorString(e));
+    if (word != 0) {
+        cudaMemsetAsync(workspace, 0, 4, s);
+        cudaStreamSynchronize(s);
+        return fail((fq_status_t)(int32_t)word, "a device-side wait expired (status word %d)", (int32_t)word);
+    }
+    return FQ_OK;
+}
+
+}  // extern "C"

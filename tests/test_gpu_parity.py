@@ -1,0 +1,199 @@
+"""Parity of the CUDA path against the CPU oracle, through the C ABI.  Needs a B200."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_15531_b200 import binding as fq
+from paper_2608_15531_b200 import synth
+
+import harness as H
+
+pytestmark = pytest.mark.gpu
+
+
+def _x(seed, M, K):
+    return synth.activations(seed, M, K)
+
+
+# ------------------------------------------------------------------ element-by-element, small
+
+@pytest.mark.parametrize("K,N,g,BN,NB,density,layout", [
+    (512, 512, 128, 256, 32, 0.01, "mixed"),       # 8 units: every CTA holds a partial piece
+    (512, 768, 64, 256, 64, 0.02, "uniform"),
+    (1024, 640, 128, 128, 32, 0.01, "mixed"),      # BN = 128 layout, ragged tile count
+    (2048, 1024, 64, 128, 128, 0.05, "clustered"),
+    (4096, 4096, 128, 256, 32, 0.01, "mixed"),     # configuration 1: 512 units over all SMs
+    (1536, 2304, 128, 256, 32, 0.0, "uniform"),    # no outliers at all
+])
+@pytest.mark.parametrize("M", [1, 5, 8, 16])
+def test_fused_matches_oracle(K, N, g, BN, NB, density, layout, M):
+    lay = synth.layer(synth.tensor_seed(9, K + N + g), K, N, density=density, layout=layout)
+    P = H.pack_layer(lay, g, BN, NB)
+    X = _x(lay.seed, M, K)
+    Y = H.run_fused(P, X)
+    Yref, Yabs = H.oracle_result(P, X)
+    stats = H.check_tolerances(Y, Yref, Yabs, K)
+    assert stats["mean_rel"] < H.MEAN_TOL
+
+
+@pytest.mark.parametrize("M", [17, 32, 33, 64, 100, 128])
+def test_fused_larger_batches(M):
+    K, N, g = 1024, 1024, 128
+    lay = synth.layer(synth.tensor_seed(9, M), K, N, density=0.01, layout="mixed")
+    P = H.pack_layer(lay, g)
+    X = _x(lay.seed, M, K)
+    Y = H.run_fused(P, X)
+    Yref, Yabs = H.oracle_result(P, X)
+    H.check_tolerances(Y, Yref, Yabs, K)
+
+
+# ------------------------------------------------------------------ bit-exact special cases
+
+@pytest.mark.parametrize("BN,g,M", [(256, 128, 8), (128, 64, 16), (256, 64, 32), (256, 128, 1)])
+def test_identity_rows_return_the_reconstructed_weights_bit_exact(BN, g, M):
+    # X = M rows of the identity: every other addend is exactly 0, so Y row = bf16(W^[k,:] + W_O[k,:])
+    K, N = 512, 768
+    lay = synth.layer(synth.tensor_seed(8, BN + g), K, N, density=0.03, layout="mixed")
+    P = H.pack_layer(lay, g, BN)
+    rows = (np.arange(M) * 37 + 5) % K
+    hot = np.argsort(lay.mask.sum(axis=1))[::-1][:M // 2]          # include outlier-heavy rows
+    rows[:len(hot)] = hot
+    X = np.zeros((M, K), dtype=np.uint16)
+    X[np.arange(M), rows] = 0x3F80
+    Y = H.run_fused(P, X)
+    Yref, _ = H.oracle_result(P, X)
+    assert np.array_equal(Y, H.f64_to_bf16_bits(Yref))
+    # one-hot times a power of two stays exact as well
+    X[np.arange(M), rows] = 0x4080                                   # 4.0
+    Y = H.run_fused(P, X)
+    assert np.array_equal(Y, H.f64_to_bf16_bits(4.0 * Yref))
+
+
+def test_zero_density_equals_the_dense_kernel_bit_for_bit():
+    K, N, g, M = 1024, 1536, 128, 8
+    lay = synth.layer(synth.tensor_seed(8, 1), K, N, density=0.0)
+    P = H.pack_layer(lay, g)
+    X = _x(3, M, K)
+    assert np.array_equal(H.run_fused(P, X), H.run_unfused(P, X, with_spmm=False))
+
+
+@pytest.mark.parametrize("M", [1, 8, 16, 40])
+def test_unfused_pair_matches_oracle_and_fused(M):
+    K, N, g = 1024, 1024, 128
+    lay = synth.layer(synth.tensor_seed(8, 2), K, N, density=0.02, layout="mixed")
+    P = H.pack_layer(lay, g)
+    X = _x(4, M, K)
+    Yd = H.run_unfused(P, X, with_spmm=False)
+    Yref_d, Yabs_d = H.oracle_result(P, X, dense_only=True)
+    H.check_tolerances(Yd, Yref_d, Yabs_d, K)
+    Yu = H.run_unfused(P, X, with_spmm=True)
+    Yref, Yabs = H.oracle_result(P, X)
+    # the two-kernel path rounds to BF16 twice (the dense result, then the sum): each element may be
+    # off by half a BF16 ulp of the dense part plus half an ulp of the total, plus FP32 accumulation
+    err = np.abs(H.bits_to_f64(Yu) - Yref)
+    bound = 2.0 ** -8 * (np.abs(Yref_d) + np.abs(Yref)) + K * 2.0 ** -24 * Yabs
+    assert np.all(err <= bound)
+    assert err.sum() / np.abs(Yref).sum() <= 4e-3
+    Yf = H.run_fused(P, X)
+    H.check_tolerances(Yf, Yref, Yabs, K)
+
+
+# ------------------------------------------------------------------ edge cases
+
+def test_oversized_tiles_fall_back_to_global_packets():
+    # one tile is completely dense in outliers (8192 packets, far above the staged capacity), one
+    # row and one column are hot; results must still match
+    K, N, g, BN = 256, 512, 128, 256
+    lay = synth.layer(synth.tensor_seed(8, 3), K, N, density=0.0)
+    mask = np.zeros((K, N), dtype=np.uint8)
+    mask[128:256, 0:256] = 1
+    mask[3, 256:512] = 1
+    mask[0:128, 400] = 1
+    kk, nn = np.nonzero(mask)
+    rng = np.random.default_rng(0)
+    vals = (rng.uniform(0.12, 0.4, size=kk.size) * rng.choice([-1, 1], size=kk.size)).astype(np.float32)
+    vb = (vals.view(np.uint32) >> 16).astype(np.uint16)
+    lay.mask, lay.coo_k, lay.coo_n, lay.coo_v = mask, kk.astype(np.uint32), nn.astype(np.uint32), vb
+    lay.W[kk, nn] = synth.bf16_bits_to_f32(vb)
+    P = H.pack_layer(lay, g, BN)
+    assert P.L.max_tile_packets == 8192
+    for M in (1, 8, 16):
+        X = _x(6, M, K)
+        Y = H.run_fused(P, X)
+        Yref, Yabs = H.oracle_result(P, X)
+        H.check_tolerances(Y, Yref, Yabs, K)
+
+
+def test_scratch_is_reusable_and_results_are_reproducible():
+    K, N, g = 2048, 1024, 128
+    lay = synth.layer(synth.tensor_seed(8, 4), K, N, density=0.01, layout="mixed")
+    P = H.pack_layer(lay, g)
+    outs = []
+    for M in (16, 1, 16, 8, 16):
+        outs.append((M, H.run_fused(P, _x(5, M, K))))
+    a = [y for m, y in outs if m == 16]
+    assert np.array_equal(a[0], a[1]) and np.array_equal(a[1], a[2])
+    # counters and status word are back to zero
+    head = P.ws[: 256 + 8192].cpu().numpy()
+    assert not head.any()
+
+
+def test_argument_errors_launch_nothing():
+    K, N, g = 512, 512, 128
+    lay = synth.layer(1, K, N, density=0.01)
+    P = H.pack_layer(lay, g)
+    X = H.to_dev(_x(1, 4, K))
+    Y = torch.zeros((4, N), dtype=torch.int16, device="cuda")
+    with pytest.raises(fq.FqError) as e:
+        fq.fq_fused_w4a16_outlier_gemm(P.L, X, 0, P.d["wq"], P.d["scale"], P.d["zero"], P.d["indptr"], P.d["info"],
+                                       P.d["packed"], Y, P.ws)
+    assert e.value.code == fq.FQ_ERR_INVALID_ARG
+    small = torch.zeros(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(fq.FqError) as e:
+        fq.fq_fused_w4a16_outlier_gemm(P.L, X, 4, P.d["wq"], P.d["scale"], P.d["zero"], P.d["indptr"], P.d["info"],
+                                       P.d["packed"], Y, small)
+    assert e.value.code == fq.FQ_ERR_BUFFER_TOO_SMALL
+    with pytest.raises(fq.FqError) as e:
+        fq.fq_fused_w4a16_outlier_gemm(P.L, None, 4, P.d["wq"], P.d["scale"], P.d["zero"], P.d["indptr"],
+                                       P.d["info"], P.d["packed"], Y, P.ws)
+    assert e.value.code == fq.FQ_ERR_INVALID_ARG
+    assert not Y.any()
+
+
+def test_host_io_entry_point_matches_device_entry_point():
+    K, N, g, M = 1024, 1024, 128, 16
+    lay = synth.layer(synth.tensor_seed(8, 5), K, N, density=0.01, layout="mixed")
+    P = H.pack_layer(lay, g)
+    Xb = _x(7, M, K)
+    Y_dev = H.run_fused(P, Xb)
+    xh = torch.from_numpy(Xb.view(np.int16)).pin_memory()
+    yh = torch.zeros((M, N), dtype=torch.int16).pin_memory()
+    xd = torch.empty((M, K), dtype=torch.int16, device="cuda")
+    yd = torch.empty((M, N), dtype=torch.int16, device="cuda")
+    fq.fq_fused_host_io(P.L, xh, M, xd, P.d["wq"], P.d["scale"], P.d["zero"], P.d["indptr"], P.d["info"],
+                        P.d["packed"], yd, yh, P.ws)
+    assert np.array_equal(yh.numpy().view(np.uint16), Y_dev)
+
+
+# ------------------------------------------------------------------ full-size, sampled columns
+
+FULL = [("8b_" + n, 2, i, K, N) for i, (n, K, N) in enumerate(synth.LLAMA3_8B)]
+
+
+@pytest.mark.parametrize("name,cfg,idx,K,N", FULL)
+def test_full_size_layers_on_sampled_columns(name, cfg, idx, K, N):
+    g = 128
+    lay = synth.layer(synth.tensor_seed(cfg, idx), K, N, density=0.01, layout="mixed")
+    P = H.pack_layer(lay, g)
+    rng = np.random.default_rng(idx)
+    BN = P.L.BN
+    # columns from the first, last and random tiles, plus the columns richest in outliers
+    cols = np.unique(np.concatenate([np.arange(0, 8), np.arange(N - 8, N), rng.integers(0, N, 80),
+                                     np.argsort(lay.mask.sum(axis=0))[::-1][:8]])).astype(np.uint32)
+    for M in (1, 8, 16):
+        X = _x(lay.seed, M, K)
+        Y = H.run_fused(P, X)
+        Yref, Yabs = H.oracle_result(P, X, cols=cols)
+        assert np.all(np.isfinite(H.bits_to_f64(Y)))
+        H.check_tolerances(Y[:, cols], Yref, Yabs, K)
+    del BN

@@ -1,0 +1,414 @@
+#!/usr/bin/env python
+"""Benchmark of the fused outlier-aware W4A16 decode matmul on B200.
+
+One step = one pass of the hot path over the LLaMA-3-8B-shaped decode layer set (qkv, o_proj,
+gate_up, down) at M in {1, 8, 16}: twelve calls of fq_fused_w4a16_outlier_gemm on seeded synthetic
+layers (INT4 g128, 1 % mixed-layout BF16 outliers).  The metric is effective HBM GB/s: the
+algorithmic bytes of those calls (packed INT4 + scale/zero + Tile-COO by the paper's storage
+formula with the true nnz + X + Y) divided by device time.  Weights are resident in HBM; every
+call reads a different packed copy of its layer so that no call finds its weights in L2.
+
+`--impl reference` times the CPU oracle instead (a deliberately plain program; a reported
+baseline, not a target).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+MS = (1, 8, 16)
+GROUP = 128
+DENSITY = 0.01
+CONFIG_ID = 2                      # the LLaMA-3-8B layer set
+L2_COVER_BYTES = 400 << 20         # rotating copies per layer cover at least this (L2 is 126 MB)
+METRIC = "effective_hbm_gbs_fused_w4a16_outlier_gemm_m1_8_16"
+
+
+def algorithmic_bytes(K, N, g, nnz, n_tile, n_bucket, M):
+    return K * N // 2 + 2 * (K // g) * N * 2 + (n_tile + 1) * 4 + n_bucket * 4 + 4 * nnz + 2 * M * K + 2 * M * N
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons, sampled while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            f = tempfile.NamedTemporaryFile(prefix="fq_clocks_", suffix=".csv", delete=False)
+            self.path = f.name
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=f,
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                parts = [x.strip() for x in line.split(",")]
+                if len(parts) < 7:
+                    continue
+                try:
+                    sm.append(float(parts[0]))
+                    mx.append(float(parts[1]))
+                except ValueError:
+                    continue
+                for nm, val in zip(names, parts[3:7]):
+                    if val.lower().startswith("active"):
+                        reasons.add(nm)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def build_workload(layers, log):
+    """Generate, pack and encode every layer on the host.  Returns a list of dicts."""
+    from paper_2608_15531_b200 import binding as fq
+    from paper_2608_15531_b200 import synth
+    out = []
+    for idx, (name, K, N) in enumerate(layers):
+        t0 = time.time()
+        lay = synth.layer(synth.tensor_seed(CONFIG_ID, idx), K, N, density=DENSITY, layout="mixed")
+        L = fq.fq_get_layout(K, N, GROUP)
+        wq, scale, zero = fq.fq_pack_int4(L, lay.W, lay.mask)
+        indptr, info, packed = fq.fq_encode_tilecoo(L, lay.coo_k, lay.coo_n, lay.coo_v)
+        n_tile = (K // 128) * (N // L.BN)
+        out.append(dict(name=name, K=K, N=N, L=L, lay=lay, wq=wq, scale=scale, zero=zero, indptr=indptr, info=info,
+                        packed=packed, n_tile=n_tile, n_bucket=n_tile * L.buckets_per_tile, nnz=lay.nnz,
+                        X=synth.activations(synth.tensor_seed(CONFIG_ID, idx), max(MS), K)))
+        log(f"packed {name} {K}x{N}: nnz={lay.nnz} packets={packed.shape[0]} max_tile={L.max_tile_packets} "
+            f"in {time.time() - t0:.1f}s")
+    return out
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2608_15531_b200 import binding as fq
+    from paper_2608_15531_b200 import synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the fused path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    fq.lib()                                     # fail loudly if the library is missing
+
+    def log(msg):
+        if rank == 0 and args.verbose:
+            print(f"[bench] {msg}", file=sys.stderr, flush=True)
+
+    work = build_workload(synth.LLAMA3_8B, log)
+    dev = torch.device("cuda", local)
+
+    def up(a):
+        a = np.ascontiguousarray(a)
+        if a.dtype == np.uint16:
+            a = a.view(np.int16)
+        elif a.dtype == np.uint32:
+            a = a.view(np.int32)
+        return torch.from_numpy(a).to(dev)
+
+    ws_bytes = max(fq.fq_workspace_bytes(w["L"], max(MS)) for w in work)
+    ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
+    calls = []                                   # (layer dict, M, bytes)
+    for w in work:
+        per_copy = w["wq"].nbytes + w["scale"].nbytes + w["zero"].nbytes + w["indptr"].nbytes + w["info"].nbytes + \
+            w["packed"].nbytes
+        ncopy = max(2, -(-L2_COVER_BYTES // per_copy))
+        base = dict(wq=up(w["wq"]), scale=up(w["scale"]), zero=up(w["zero"]), indptr=up(w["indptr"]),
+                    info=up(w["info"]), packed=up(w["packed"]))
+        w["copies"] = [base] + [{k: v.clone() for k, v in base.items()} for _ in range(ncopy - 1)]
+        w["Xd"] = {M: up(w["X"][:M]) for M in MS}
+        w["Yd"] = {M: torch.empty((M, w["N"]), dtype=torch.int16, device=dev) for M in MS}
+        w["turn"] = 0
+        for M in MS:
+            calls.append((w, M, algorithmic_bytes(w["K"], w["N"], GROUP, w["nnz"], w["n_tile"], w["n_bucket"], M)))
+    step_bytes = sum(c[2] for c in calls)
+    stream = torch.cuda.current_stream()
+
+    def one_call(w, M):
+        c = w["copies"][w["turn"] % len(w["copies"])]
+        w["turn"] += 1
+        fq.fq_fused_w4a16_outlier_gemm(w["L"], w["Xd"][M], M, c["wq"], c["scale"], c["zero"], c["indptr"], c["info"],
+                                       c["packed"], w["Yd"][M], ws, stream)
+
+    def step():
+        for w, M, _ in calls:
+            one_call(w, M)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    fq.fq_check_status(ws)
+    sampler = ClockSampler(local)
+    sync_all()
+    if rank == 0:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sync_all()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    sync_all()
+    clocks = sampler.stop() if rank == 0 else {}
+    ms = e0.elapsed_time(e1)
+    fq.fq_check_status(ws)
+    if world > 1:
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_per_step = ms / args.steps
+    value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
+
+    # ---- end to end: host X in, host Y out, through the C ABI, every call
+    xh = {(w["name"], M): torch.from_numpy(np.ascontiguousarray(w["X"][:M]).view(np.int16)).pin_memory()
+          for w, M, _ in calls}
+    yh = {(w["name"], M): torch.empty((M, w["N"]), dtype=torch.int16).pin_memory() for w, M, _ in calls}
+    xd = {k: torch.empty_like(v, device=dev) for k, v in xh.items()}
+
+    def e2e_step():
+        for w, M, _ in calls:
+            c = w["copies"][w["turn"] % len(w["copies"])]
+            w["turn"] += 1
+            key = (w["name"], M)
+            fq.fq_fused_host_io(w["L"], xh[key], M, xd[key], c["wq"], c["scale"], c["zero"], c["indptr"], c["info"],
+                                c["packed"], w["Yd"][M], yh[key], ws, stream)
+
+    for _ in range(3):
+        e2e_step()
+    sync_all()
+    e0.record(stream)
+    for _ in range(args.steps):
+        e2e_step()
+    e1.record(stream)
+    sync_all()
+    e2e_ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_value = world * step_bytes / (e2e_ms / args.steps * 1e-3) / 1e9
+    h2d = sum(2 * M * w["K"] for w, M, _ in calls)
+    d2h = sum(2 * M * w["N"] for w, M, _ in calls)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = peaks()
+
+    # ---- per call: fused, unfused pair, cuBLAS BF16 on pre-dequantised weights (context, N = 1 view)
+    def time_loop(fn, reps):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(reps):
+            fn()
+        b.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps * 1e3          # microseconds
+
+    per_call = []
+    reps = max(10, min(100, args.steps * 2))
+    for w, M, nbytes in calls:
+        def fused():
+            one_call(w, M)
+
+        def unfused():
+            c = w["copies"][w["turn"] % len(w["copies"])]
+            w["turn"] += 1
+            fq.fq_unfused_gemm(w["L"], w["Xd"][M], M, c["wq"], c["scale"], c["zero"], w["Yd"][M], ws, stream)
+            fq.fq_unfused_spmm(w["L"], w["Xd"][M], M, c["indptr"], c["info"], c["packed"], w["Yd"][M], stream)
+
+        us_f = time_loop(fused, reps)
+        us_u = time_loop(unfused, reps)
+        per_call.append(dict(layer=w["name"], K=w["K"], N=w["N"], M=M, bytes=nbytes, fused_us=round(us_f, 3),
+                             fused_gbs=round(nbytes / us_f / 1e3, 1), frac_of_peak=round(nbytes / us_f / 1e3 / peak, 4),
+                             unfused_us=round(us_u, 3)))
+    if args.cublas:
+        for w in work:
+            # BF16 GEMM on dequant(W_Q) + W_O, materialised with torch on the device (a baseline, not the path)
+            q = torch.from_numpy(fq.fq_unpack_int4(w["L"], w["wq"])).to(dev).float()
+            s = up(w["scale"]).view(torch.bfloat16).float().repeat_interleave(GROUP, 0)
+            z = up(w["zero"]).view(torch.bfloat16).float().repeat_interleave(GROUP, 0)
+            Wd = (s * (q - z))
+            Wd[torch.from_numpy(w["lay"].coo_k.astype(np.int64)).to(dev), torch.from_numpy(w["lay"].coo_n.astype(np.int64)).to(dev)] = \
+                up(w["lay"].coo_v).view(torch.bfloat16).float()
+            Wb = Wd.to(torch.bfloat16)
+            del q, s, z, Wd
+            ncopy = max(2, -(-L2_COVER_BYTES // (Wb.numel() * 2)))
+            Wc = [Wb] + [Wb.clone() for _ in range(ncopy - 1)]
+            for M in MS:
+                xb = w["Xd"][M].view(torch.bfloat16)
+                turn = [0]
+
+                def gemm():
+                    turn[0] += 1
+                    torch.matmul(xb, Wc[turn[0] % len(Wc)])
+
+                us = time_loop(gemm, reps)
+                for pc in per_call:
+                    if pc["layer"] == w["name"] and pc["M"] == M:
+                        pc["cublas_bf16_us"] = round(us, 3)
+            del Wc, Wb
+            torch.cuda.empty_cache()
+
+    cpu = cpu_baseline(work, budget_s=args.cpu_seconds) if args.cpu_seconds > 0 else None
+
+    line = {
+        "metric": METRIC, "value": round(value, 2), "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "configs[1]: LLaMA3-8B decode layer set qkv/o_proj/gate_up/down x M in {1,8,16}, "
+                               "INT4 g128, 1% mixed-layout BF16 outliers; one step = 12 fused calls",
+                   "l2": "inputs larger than L2: each call reads a different packed copy, copies per layer cover >= 400 MB",
+                   "replicas": "replicas only: each rank runs the same workload on its own GPU, no collective on the data path"},
+        "clocks": clocks,
+        "e2e": {"value": round(e2e_value, 2), "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": round(e2e_ms / args.steps, 5)},
+        "gpu_launches": args.steps * len(calls),
+        "roofline": {"bound": "hbm", "achieved": round(value / world, 2), "peak": peak, "unit": "GB/s",
+                     "frac": round(value / world / peak, 4), "traffic": None, "peak_kind": f"of {peak_kind}",
+                     "bytes_per_launch": step_bytes // len(calls), "us_per_launch": round(ms_per_step * 1e3 / len(calls), 3)},
+        "cpu_baseline": cpu,
+        "us_per_call": per_call,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def cpu_baseline(work, budget_s: float):
+    """The oracle as it stands on the host cores, on a bounded sample: every layer of the step at
+    M = 16, restricted to its first `f * N` output columns, f chosen from a short probe so that the
+    whole sample takes about `budget_s` seconds."""
+    import oracle
+    probe = work[1]                                # o_proj
+    cols = 128
+    lay = probe["lay"]
+    q, s, z = oracle.quantize(np.ascontiguousarray(lay.W[:, :cols]), np.ascontiguousarray(lay.mask[:, :cols]), GROUP)
+    sel = lay.coo_n < cols
+    t0 = time.time()
+    oracle.fused_matmul(probe["X"][:16], q, s, z, GROUP, lay.coo_k[sel], lay.coo_n[sel], lay.coo_v[sel])
+    rate = 16 * probe["K"] * cols / max(time.time() - t0, 1e-6)        # multiply-adds per second
+    total_mac = sum(16 * w["K"] * w["N"] for w in work)
+    f = min(1.0, budget_s * rate / total_mac)
+    t_total, bytes_total = 0.0, 0
+    for w in work:
+        lay = w["lay"]
+        ncols = max(64, int(f * w["N"]) // 64 * 64)
+        q, s, z = oracle.quantize(np.ascontiguousarray(lay.W[:, :ncols]), np.ascontiguousarray(lay.mask[:, :ncols]), GROUP)
+        sel = lay.coo_n < ncols
+        t0 = time.time()
+        oracle.fused_matmul(w["X"][:16], q, s, z, GROUP, lay.coo_k[sel], lay.coo_n[sel], lay.coo_v[sel])
+        t_total += time.time() - t0
+        frac = ncols / w["N"]
+        bytes_total += int(frac * algorithmic_bytes(w["K"], w["N"], GROUP, w["nnz"], w["n_tile"], w["n_bucket"], 16))
+    return {"value": round(bytes_total / t_total / 1e9, 4), "unit": "GB/s", "cores": oracle.num_threads(),
+            "kind": "oracle", "seconds": round(t_total, 2),
+            "sample": f"all four layers at M=16, first {f:.3f} of each layer's output columns (fp64 oracle, OpenMP over columns)"}
+
+
+def run_reference(args):
+    """The oracle arm: rank 0 times the CPU oracle on a bounded sample of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2608_15531_b200 import synth
+
+    def log(msg):
+        if args.verbose:
+            print(f"[bench] {msg}", file=sys.stderr, flush=True)
+
+    work = build_workload(synth.LLAMA3_8B, log)
+    steps = max(1, args.steps)
+    per_step_budget = max(2.0, min(20.0, 120.0 / (steps + args.warmup)))
+    for _ in range(args.warmup):
+        cpu_baseline(work, per_step_budget)
+    t0 = time.time()
+    res = None
+    for _ in range(steps):
+        res = cpu_baseline(work, per_step_budget)
+    dt = (time.time() - t0) / steps
+    line = {
+        "impl": "reference", "metric": METRIC, "value": res["value"], "unit": "GB/s",
+        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": steps, "warmup": args.warmup,
+        "ms_per_step": round(dt * 1e3, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "configs[1]: LLaMA3-8B decode layer set, bounded sample per step (see cpu_baseline.sample)"},
+        "cpu_baseline": res,
+        "e2e": {"value": res["value"], "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cpu-seconds", type=float, default=15.0, help="budget of the CPU-oracle baseline leg (0 = skip)")
+    ap.add_argument("--no-cublas", dest="cublas", action="store_false")
+    ap.add_argument("--verbose", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

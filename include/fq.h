@@ -28,14 +28,14 @@
  *   INT4 weights.  BK = 128 rows, BN = 128 or 256 columns per tile.  The buffer
  *   is a sequence of chunks, one per (column tile tn, row tile kt), chunk index
  *   tn * (K/128) + kt, each 16 * BN little-endian 32-bit words.  Word index
- *   inside a chunk is ((w*4 + j)*32 + lane)*4 + c  (w = 32-column strip,
- *   j = 0..3, lane = 0..31, c = 0..3).  With ns = j>>1, ks = (j&1)*4 + c,
- *   grp = lane>>2, t = lane&3, nibble p = r + 4h (r = 0..3, h = 0..1; bits
- *   4p..4p+3) of that word is the code of
- *       column tn*BN + 32w + 16ns + grp + 8(r&1)
- *       row    kt*128 + 32(ks>>1) + 8t + 4(ks&1) + 2(r>>1) + h .
- *   (One word is one thread's A-operand fragment of one m16n8k16 MMA; row order
- *   inside a 32-row block follows the 16-byte activation loads of the kernel.)
+ *   inside a chunk is (j*BN + t)*4 + w  (j = 0..3: 32-row block, t = column
+ *   inside the tile, w = 0..3: 8-row block).  Nibble p = i + 4h (i = 0..3,
+ *   h = 0..1; bits 4p..4p+3) of that word is the code of
+ *       column tn*BN + t
+ *       row    kt*128 + 32j + 8w + 2i + h .
+ *   (One thread owns one column: four 16-byte loads give its 128 codes of the
+ *   tile, and one shift-and-mask turns nibbles i and i+4 into a BF16 pair of
+ *   consecutive rows, which is the tensor-memory operand order.)
  *
  *   Scale, zero.  (K/group) x N row-major BF16.  zero holds the integer 0..15.
  *
@@ -81,7 +81,7 @@ typedef struct fq_layout {
     uint32_t BK;               /* 128 */
     uint32_t BN;               /* 128 or 256 */
     uint32_t buckets_per_tile; /* NB: 32, 64 or 128 */
-    uint32_t wq_interleave;    /* 1: the MMA-fragment order described above */
+    uint32_t wq_interleave;    /* 2: the column-per-thread order described above */
     uint32_t coo_unit_bytes;   /* 16 */
     uint32_t max_tile_packets; /* largest tile of the encoded W_O, in packets; 0 = not encoded */
     uint32_t reserved[6];
@@ -159,9 +159,10 @@ fq_status_t fq_workspace_bytes(const fq_layout_t* L, uint32_t M, size_t* bytes);
 
 /*
  * The fused operator (Eq. 1; Sections 3.1 and 4.1): one launch per 32 rows of X
- * reads X, W_Q and the Tile-COO tiles through a TMA/mbarrier ring, dequantises
- * in registers into tensor-core accumulators, applies the tile's outliers
- * against the same shared-memory activation tile, and writes Y once.
+ * reads X, W_Q and the Tile-COO tiles through a bulk-copy/mbarrier ring,
+ * dequantises in registers into the tensor-memory operand of tcgen05 MMAs,
+ * applies the tile's outliers against the same shared-memory activation tile,
+ * and writes Y once.
  * X: device, M x K BF16.  M in [1, FQ_MAX_M].  Y: device, M x N BF16,
  * overwritten.  All other arrays: device copies of the host packer/encoder
  * output.  Work is split over persistent CTAs by contiguous ranges of (tile,

@@ -192,37 +192,30 @@ void orc_fused_matmul(const uint16_t* X, uint32_t M, uint32_t K, uint32_t N, uin
  *   The buffer is a sequence of chunks, one per (column tile tn, row tile kt),
  *   ordered tn-major (chunk index tn * (K/128) + kt).  A chunk covers 128 rows
  *   by BN columns and holds 16 * BN little-endian 32-bit words.  Word index
- *   inside the chunk:
- *        ((w * 4 + j) * 32 + lane) * 4 + c
- *   with w = 32-column strip (0 .. BN/32-1), j = 0..3, lane = 0..31, c = 0..3.
- *   Let ns = j >> 1, ks = (j & 1) * 4 + c, grp = lane >> 2, t = lane & 3.
- *   Nibble p (bits 4p .. 4p+3) of that word, p = r + 4h with r = 0..3, h = 0..1,
- *   is the code of
- *        column  tn*BN + 32*w + 16*ns + grp + 8*(r & 1)
- *        row     kt*128 + 32*(ks >> 1) + 8*t + 4*(ks & 1) + 2*(r >> 1) + h
+ *   inside the chunk:  (j * BN + t) * 4 + w   with j = 0..3, t = 0..BN-1,
+ *   w = 0..3.  Nibble p (bits 4p .. 4p+3) of that word, p = i + 4h with
+ *   i = 0..3, h = 0..1, is the code of
+ *        column  tn*BN + t
+ *        row     kt*128 + 32*j + 8*w + 2*i + h
  */
 int orc_decode_wq(const uint32_t* wq, uint32_t K, uint32_t N, uint32_t BN, uint8_t* q) {
-    if (K % 128 != 0 || BN % 32 != 0 || N % BN != 0) return -1;
-    const uint32_t KT = K / 128, NT = N / BN, strips = BN / 32;
+    if (K % 128 != 0 || BN == 0 || N % BN != 0) return -1;
+    const uint32_t KT = K / 128, NT = N / BN;
     const size_t chunk_words = (size_t)16 * BN;
     for (uint32_t tn = 0; tn < NT; ++tn)
         for (uint32_t kt = 0; kt < KT; ++kt) {
             const uint32_t* chunk = wq + ((size_t)tn * KT + kt) * chunk_words;
-            for (uint32_t w = 0; w < strips; ++w)
-                for (uint32_t j = 0; j < 4; ++j)
-                    for (uint32_t lane = 0; lane < 32; ++lane)
-                        for (uint32_t c = 0; c < 4; ++c) {
-                            uint32_t word = chunk[((w * 4 + j) * 32 + lane) * 4 + c];
-                            uint32_t ns = j >> 1, ks = (j & 1) * 4 + c;
-                            uint32_t grp = lane >> 2, t = lane & 3;
-                            for (uint32_t p = 0; p < 8; ++p) {
-                                uint32_t r = p & 3, h = p >> 2;
-                                uint32_t col = tn * BN + 32 * w + 16 * ns + grp + 8 * (r & 1);
-                                uint32_t row = kt * 128 + 32 * (ks >> 1) + 8 * t + 4 * (ks & 1) +
-                                               2 * (r >> 1) + h;
-                                q[(size_t)row * N + col] = (uint8_t)((word >> (4 * p)) & 0xfu);
-                            }
+            for (uint32_t j = 0; j < 4; ++j)
+                for (uint32_t t = 0; t < BN; ++t)
+                    for (uint32_t w = 0; w < 4; ++w) {
+                        uint32_t word = chunk[(j * BN + t) * 4 + w];
+                        for (uint32_t p = 0; p < 8; ++p) {
+                            uint32_t i = p & 3, h = p >> 2;
+                            uint32_t col = tn * BN + t;
+                            uint32_t row = kt * 128 + 32 * j + 8 * w + 2 * i + h;
+                            q[(size_t)row * N + col] = (uint8_t)((word >> (4 * p)) & 0xfu);
                         }
+                    }
         }
     return 0;
 }

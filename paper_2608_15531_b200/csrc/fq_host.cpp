@@ -29,13 +29,10 @@ static inline float bf16_to_f32(uint16_t h) {
 }
 
 // Position of the code of (row kr, column cr) inside a 128 x BN chunk: word index and nibble.
-static inline void wq_slot(uint32_t kr, uint32_t cr, uint32_t& word, uint32_t& nib) {
-    const uint32_t w = cr >> 5, ns = (cr >> 4) & 1, rlo = (cr >> 3) & 1, grp = cr & 7;
-    const uint32_t kb = kr >> 5, t = (kr >> 3) & 3, odd = (kr >> 2) & 1, rhi = (kr >> 1) & 1, h = kr & 1;
-    const uint32_t ks = 2 * kb + odd;
-    const uint32_t j = ns * 2 + (ks >> 2), c = ks & 3, lane = grp * 4 + t;
-    word = ((w * 4 + j) * 32 + lane) * 4 + c;
-    nib = (rlo + 2 * rhi) + 4 * h;
+static inline void wq_slot(uint32_t kr, uint32_t cr, uint32_t BN, uint32_t& word, uint32_t& nib) {
+    const uint32_t j = kr >> 5, w = (kr >> 3) & 3, i = (kr >> 1) & 3, h = kr & 1;
+    word = (j * BN + cr) * 4 + w;
+    nib = i + 4 * h;
 }
 }  // namespace fq
 
@@ -65,7 +62,7 @@ fq_status_t fq_get_layout(uint32_t K, uint32_t N, uint32_t group, uint32_t bn_hi
     out->BK = FQ_BK;
     out->BN = BN;
     out->buckets_per_tile = NB;
-    out->wq_interleave = 1;
+    out->wq_interleave = 2;
     out->coo_unit_bytes = 16;
     return FQ_OK;
 }
@@ -143,7 +140,7 @@ fq_status_t fq_pack_int4(const fq_layout_t* L, const float* W, const uint8_t* ma
                             q = q < 0 ? 0 : (q > 15 ? 15 : q);
                         }
                         uint32_t word, nib;
-                        wq_slot(kr, c, word, nib);
+                        wq_slot(kr, c, BN, word, nib);
                         chunk[word] |= (uint32_t)q << (4 * nib);
                     }
                 }
@@ -165,7 +162,7 @@ fq_status_t fq_unpack_int4(const fq_layout_t* L, const void* wq_in, uint8_t* q) 
         for (uint32_t kr = 0; kr < FQ_BK; ++kr)
             for (uint32_t c = 0; c < BN; ++c) {
                 uint32_t word, nib;
-                wq_slot(kr, c, word, nib);
+                wq_slot(kr, c, BN, word, nib);
                 q[(size_t)(kt * FQ_BK + kr) * N + (size_t)tn * BN + c] = (uint8_t)((chunk[word] >> (4 * nib)) & 0xf);
             }
     }

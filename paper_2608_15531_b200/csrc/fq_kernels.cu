@@ -1,21 +1,25 @@
 // CUDA side of the library (sm_100a): the fused W4A16 + Tile-COO outlier decode matmul
 // (Eq. 1; Sections 3.1, 4.1, 4.2), its two unfused baselines and the launchers behind the C ABI.
 //
-// Kernel shape (one persistent CTA per SM):
-//   warp 0            producer: per (tile, k-step) unit, bulk-copies (cp.async.bulk + mbarrier
-//                     expect_tx) the unit's INT4 chunk, scale/zero rows, bucket_info slice, packet
-//                     range and the M activation rows into a ring of shared-memory stages
-//   warps 1..NDW      dense: each owns 32 output columns; one 32-bit word = one m16n8k16 A
-//                     fragment of codes, turned into BF16 (128 + q) with lop3 and fed to mma.sync
-//                     with the activations as the B operand; an all-ones A fragment yields the
-//                     per-group activation sums, so zero-point and scale are applied once per group
-//                     in FP32:  acc += s * (sum x (128+q) - (128+z) sum x)
-//   remaining warps   sparse: lane = bucket; transposes the activation tile to k-major, then for
-//                     each packet slot adds v * x[0..7][k] into the FP32 tile sh_c[col][m]
-//                     (buckets own disjoint columns, so no atomics)
+// Kernel shape (one persistent CTA per SM, warp-specialised):
+//   warp 0        producer: per (tile, k-step) unit, bulk-copies (cp.async.bulk + mbarrier expect_tx)
+//                 the unit's INT4 chunk, scale/zero rows, bucket_info slice, packet range and the M
+//                 activation rows into a ring of shared-memory stages
+//   warp 1        tensor: owns the TMEM allocation; per unit re-lays the activation rows into the
+//                 canonical K-major operand layout, computes the per-group activation sums, and
+//                 issues tcgen05.mma (A = dequantised weights in TMEM, B = activations in shared
+//                 memory, D = FP32 in TMEM); completion is signalled with tcgen05.commit
+//   dense warps   thread = output column: unpacks its 128 codes of the unit with lop3 into BF16
+//                 (128 + q), stores them as the A operand into TMEM (tcgen05.st), and one unit later
+//                 reads the FP32 group sums back (tcgen05.ld) and applies scale and zero-point once
+//                 per group in FP32:  acc[m] += s * (sum_k x (128+q) - (128+z) sum_k x)
+//   sparse warps  lane = bucket; transposes the activation tile to k-major, then for each packet
+//                 slot adds v * x[0..7][k] into the FP32 tile sh_c[col][m] (buckets own disjoint
+//                 columns, so no atomics); merged into the column owner's registers at tile end
 // Units are split over CTAs as contiguous ranges (stream-K).  A tile whose k-range is shared by
 // several CTAs is finished by the last CTA to arrive, which adds the FP32 partials in CTA order.
-// Every wait is bounded: on expiry the CTA raises the scratch status word and leaves.
+// Every wait on a barrier is bounded: on expiry the CTA raises the scratch status word, drains and
+// leaves through the common exit that frees its TMEM.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -28,9 +32,10 @@
 namespace fq {
 
 constexpr int kBK = 128;
-constexpr int kXRowBytes = 320;        // 256 B of activations + 64 B pad: conflict-free 16-byte fragment loads
+constexpr int kXRowBytes = 272;        // 256 B of activations + 16 B pad: conflict-free ldmatrix rows
 constexpr int kSmemBudget = 232448;    // 227 KB per CTA on sm_100
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+constexpr uint32_t kTmemCols = 512;
 
 struct Params {
     const uint16_t* X;
@@ -46,8 +51,8 @@ struct Params {
     float* partials;
     uint32_t M, K, N, KT, NT;
     uint32_t NB, coo_cap, stages, nsw;
-    // shared-memory offsets (bytes)
-    uint32_t stage_bytes, off_sz, off_x, off_info, off_coo;
+    // shared-memory offsets (bytes); the first five are relative to a stage
+    uint32_t stage_bytes, off_sz, off_xraw, off_xcan, off_xsum, off_info, off_coo;
     uint32_t off_shc, off_xt, off_bar;
 };
 
@@ -99,18 +104,16 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
     return true;
 }
+// Warp-uniform form: every lane waits, and the warp gives up together.
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t* status) {
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status));
+}
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                  "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
 }
-__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-// (w >> sh) & 0x000f000f | 0x43004300: two codes -> two BF16 values 128 + q
+// (w & 0x000f000f) | 0x43004300: two codes -> two BF16 values 128 + q
 __device__ __forceinline__ uint32_t codes_to_bf16x2(uint32_t w) {
     uint32_t r;
     asm("lop3.b32 %0, %1, 0x000f000f, 0x43004300, 0xea;" : "=r"(r) : "r"(w));
@@ -128,6 +131,55 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, u
                  : "r"(addr));
 }
 
+// ---- tcgen05 / tensor memory
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"r"(taddr), "r"(r[0]), "r"(r[1]),
+                 "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&d)[16]) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+    tmem_wait_ld();
+#pragma unroll
+    for (int i = 0; i < 16; ++i) d[i] = __uint_as_float(r[i]);
+}
+// D[128 x N] (+)= A[128 x 16] (TMEM) * B[16 x N] (shared-memory descriptor), BF16 in, FP32 out
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+        " tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// K-major, no swizzle: 8 rows x 16 B core matrices; LBO = step between the two K halves of one MMA,
+// SBO = step between 8-row groups.
+__device__ __forceinline__ uint64_t make_b_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    return (uint64_t)((saddr & 0x3ffffu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
+           (1ull << 46);
+}
+
 // Which CTA owns unit u when U units are dealt out as contiguous ranges, the first r CTAs one longer.
 __device__ __forceinline__ uint32_t cta_of_unit(uint32_t u, uint32_t q, uint32_t r) {
     const uint32_t big = r * (q + 1);
@@ -137,29 +189,61 @@ __device__ __forceinline__ uint32_t unit_begin_of(uint32_t c, uint32_t q, uint32
 
 // ----------------------------------------------------------------------------- sparse step
 
-// One bucket's packets against the k-major activation copy xt ([128][8] BF16, 16 B per row):
-// shc[col * ldc + 0..7] += v * x[0..7][k] for each slot (Section 4.2, without the per-column
-// padding: every slot carries its own column byte).
-__device__ __forceinline__ void apply_packet(const uint4 pk, const uint8_t* xt, float* shc_oct, uint32_t ldc) {
+__device__ __forceinline__ uint32_t has_zero_byte(uint32_t v) { return (v - 0x01010101u) & ~v & 0x80808080u; }
+
+__device__ __forceinline__ void fma8(float4& c0, float4& c1, float v, const uint4 xv) {
+    c0.x = fmaf(v, bf16lo(xv.x), c0.x);
+    c0.y = fmaf(v, bf16hi(xv.x), c0.y);
+    c0.z = fmaf(v, bf16lo(xv.y), c0.z);
+    c0.w = fmaf(v, bf16hi(xv.y), c0.w);
+    c1.x = fmaf(v, bf16lo(xv.z), c1.x);
+    c1.y = fmaf(v, bf16hi(xv.z), c1.y);
+    c1.z = fmaf(v, bf16lo(xv.w), c1.z);
+    c1.w = fmaf(v, bf16hi(xv.w), c1.w);
+}
+
+// One packet (four outliers) against the k-major activation copy xt ([128][8] BF16, 16 B per row):
+// shc[col * ldc + 0..7] += v * x[0..7][k] for each slot (Section 4.2, without the per-column padding:
+// every slot carries its own column byte).  When the four columns differ, all loads are issued
+// before the first store.
+__device__ __forceinline__ void apply_packet(const uint4 pk, const uint8_t* __restrict__ xt, float* shc_oct, uint32_t ldc) {
+    uint32_t k[4], c[4];
+    float v[4];
 #pragma unroll
     for (int s = 0; s < 4; ++s) {
-        const uint32_t k = (pk.x >> (8 * s)) & 0xffu;
-        const uint32_t c = (pk.y >> (8 * s)) & 0xffu;
-        const uint32_t vw = (s < 2) ? pk.z : pk.w;
-        const float v = (s & 1) ? bf16hi(vw) : bf16lo(vw);
-        const uint4 xv = *reinterpret_cast<const uint4*>(xt + k * 16);
-        float4* cp = reinterpret_cast<float4*>(shc_oct + c * ldc);
-        float4 c0 = cp[0], c1 = cp[1];
-        c0.x = fmaf(v, bf16lo(xv.x), c0.x);
-        c0.y = fmaf(v, bf16hi(xv.x), c0.y);
-        c0.z = fmaf(v, bf16lo(xv.y), c0.z);
-        c0.w = fmaf(v, bf16hi(xv.y), c0.w);
-        c1.x = fmaf(v, bf16lo(xv.z), c1.x);
-        c1.y = fmaf(v, bf16hi(xv.z), c1.y);
-        c1.z = fmaf(v, bf16lo(xv.w), c1.z);
-        c1.w = fmaf(v, bf16hi(xv.w), c1.w);
-        cp[0] = c0;
-        cp[1] = c1;
+        k[s] = (pk.x >> (8 * s)) & 0xffu;
+        c[s] = (pk.y >> (8 * s)) & 0xffu;
+    }
+    v[0] = bf16lo(pk.z); v[1] = bf16hi(pk.z); v[2] = bf16lo(pk.w); v[3] = bf16hi(pk.w);
+    uint4 xv[4];
+#pragma unroll
+    for (int s = 0; s < 4; ++s) xv[s] = *reinterpret_cast<const uint4*>(xt + k[s] * 16);
+    const uint32_t dup = has_zero_byte(pk.y ^ __byte_perm(pk.y, 0, 0x0321)) | has_zero_byte(pk.y ^ __byte_perm(pk.y, 0, 0x1032));
+    if (!dup) {
+        float4 c0[4], c1[4];
+#pragma unroll
+        for (int s = 0; s < 4; ++s) {
+            const float4* cp = reinterpret_cast<const float4*>(shc_oct + c[s] * ldc);
+            c0[s] = cp[0];
+            c1[s] = cp[1];
+        }
+#pragma unroll
+        for (int s = 0; s < 4; ++s) fma8(c0[s], c1[s], v[s], xv[s]);
+#pragma unroll
+        for (int s = 0; s < 4; ++s) {
+            float4* cp = reinterpret_cast<float4*>(shc_oct + c[s] * ldc);
+            cp[0] = c0[s];
+            cp[1] = c1[s];
+        }
+    } else {
+#pragma unroll
+        for (int s = 0; s < 4; ++s) {
+            float4* cp = reinterpret_cast<float4*>(shc_oct + c[s] * ldc);
+            float4 c0 = cp[0], c1 = cp[1];
+            fma8(c0, c1, v[s], xv[s]);
+            cp[0] = c0;
+            cp[1] = c1;
+        }
     }
 }
 
@@ -181,33 +265,47 @@ __device__ __forceinline__ void transpose_octet(uint32_t xs_rows_u32, uint8_t* x
 
 // ----------------------------------------------------------------------------- fused kernel
 
-template <int BN, int MO, int GROUP, bool SPARSE>
-__global__ void __launch_bounds__(32 * (1 + BN / 32 + 8), 1) fq_fused_kernel(const Params p) {
-    constexpr int NDW = BN / 32;
+// BN: tile columns (128 or 256).  NB16: batch columns of the MMA in units of 16 (1: M <= 16, 2: M <= 32).
+template <int BN, int NB16, int GROUP, bool SPARSE>
+__global__ void __launch_bounds__(32 * (4 + BN / 32 + 6), 1) fq_fused_kernel(const Params p) {
+    constexpr int NDW = BN / 32;              // dense warps: one thread per tile column
+    constexpr int NT128 = BN / 128;           // 128-row MMA tiles per unit
+    constexpr int NMMA = 16 * NB16;           // MMA N: batch rows, padded
     constexpr int GPS = kBK / GROUP;          // groups per k-step
+    constexpr int DCOLS = GPS * NMMA;         // accumulator columns per D buffer
     constexpr int W_BYTES = 16 * BN * 4;
     constexpr int SZ_ROW = BN * 2;
-    constexpr int LDC = 8 * MO;               // sh_c row: FP32 per batch row
+    constexpr int LDC = NMMA;                 // sh_c row: FP32 per batch row
+    constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NMMA >> 3) << 17) | (8u << 24);
     extern __shared__ __align__(128) uint8_t smem[];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t S = p.stages;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
     const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * S;
-    const uint32_t bar_sparse_done = bar_empty + 8 * S, bar_dense_done = bar_sparse_done + 8, bar_dense = bar_dense_done + 8;
-    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 2 * S + 3);
+    const uint32_t bar_a_ready = bar_empty + 8 * S;      // [2]
+    const uint32_t bar_d_ready = bar_a_ready + 16;       // [2]
+    const uint32_t bar_sparse_done = bar_d_ready + 16, bar_dense_done = bar_sparse_done + 8;
+    const uint32_t bar_dense = bar_dense_done + 8, bar_final = bar_dense + 8;
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 2 * S + 8);
     volatile uint32_t* last_flag = abort_flag + 1;
+    volatile uint32_t* tmem_slot = abort_flag + 2;
     float* shc = reinterpret_cast<float*>(smem + p.off_shc);
 
     const uint32_t nsw = SPARSE ? p.nsw : 0;
     if (tid == 0) {
         for (uint32_t s = 0; s < S; ++s) {
             mbar_init(bar_full + 8 * s, 1);
-            mbar_init(bar_empty + 8 * s, NDW + nsw);
+            mbar_init(bar_empty + 8 * s, NDW + nsw + 1);
         }
+        mbar_init(bar_a_ready, NDW);
+        mbar_init(bar_a_ready + 8, NDW);
+        mbar_init(bar_d_ready, 2);
+        mbar_init(bar_d_ready + 8, 2);
         mbar_init(bar_sparse_done, nsw ? nsw : 1);
         mbar_init(bar_dense_done, NDW);
         mbar_init(bar_dense, NDW);
+        mbar_init(bar_final, 1);
         *abort_flag = 0;
         *last_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -215,8 +313,15 @@ __global__ void __launch_bounds__(32 * (1 + BN / 32 + 8), 1) fq_fused_kernel(con
     if (SPARSE) {
         for (uint32_t i = tid; i < (uint32_t)(BN * LDC); i += blockDim.x) shc[i] = 0.0f;
     }
+    if (warp == 1) {
+        tmem_alloc(smem_u32((const void*)tmem_slot), kTmemCols);
+        tmem_relinquish();
+    }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    tc_fence_before();
     __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
 
     // contiguous range of units for this CTA
     const uint32_t U = p.NT * p.KT, P = gridDim.x, q = U / P, r = U % P;
@@ -226,7 +331,8 @@ __global__ void __launch_bounds__(32 * (1 + BN / 32 + 8), 1) fq_fused_kernel(con
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer
-        uint32_t ip_a = 0, ip_b = 0;
+        uint32_t ip_a = 0, ip_b = 0, issued = 0;
+        bool ok = true;
         for (uint32_t u = u_begin, it = 0; u < u_end; ++u, ++it) {
             const uint32_t s = it % S, ph = (it / S) & 1;
             if (SPARSE && (it & 31) == 0) {  // this warp's next 32 packet ranges, one coalesced read
@@ -240,12 +346,7 @@ __global__ void __launch_bounds__(32 * (1 + BN / 32 + 8), 1) fq_fused_kernel(con
                 npk = __shfl_sync(0xffffffffu, ip_b, it & 31) - pk0;
                 npk = min(npk, p.coo_cap);
             }
-            if (!mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_flag, p.status)) {
-                // giving up: let the copies already issued land before the CTA's shared memory goes away
-                for (uint32_t j = (it > S ? it - S : 0); j < it; ++j)
-                    for (uint32_t spin = 0; spin < (1u << 20) && !mbar_try_wait(bar_full + 8 * (j % S), (j / S) & 1); ++spin) {}
-                return;
-            }
+            if (!warp_wait(bar_empty + 8 * s, ph ^ 1, abort_flag, p.status)) { ok = false; break; }
             const uint32_t tn = u / KT, kt = u % KT;
             const uint32_t full = bar_full + 8 * s;
             const uint32_t st = smem_u32(smem) + s * p.stage_bytes;
@@ -272,110 +373,169 @@ __global__ void __launch_bounds__(32 * (1 + BN / 32 + 8), 1) fq_fused_kernel(con
             }
             {
                 const uint32_t m = (lane + 27) & 31;  // rows start on lane 5
-                if (m < p.M) bulk_g2s(st + p.off_x + m * kXRowBytes, p.X + (size_t)m * p.K + (size_t)kt * kBK, 256, full);
+                if (m < p.M) bulk_g2s(st + p.off_xraw + m * kXRowBytes, p.X + (size_t)m * p.K + (size_t)kt * kBK, 256, full);
             }
+            issued = it + 1;
         }
-        return;
-    }
-
-    if (warp <= NDW) {
-        // ------------------------------------------------------------------ dense
-        const int dw = warp - 1, g = lane >> 2, t = lane & 3;
-        const int dtid = dw * 32 + lane;
-        float accf[2][MO][4];
-#pragma unroll
-        for (int a = 0; a < 2; ++a)
-#pragma unroll
-            for (int o = 0; o < MO; ++o)
-#pragma unroll
-                for (int i = 0; i < 4; ++i) accf[a][o][i] = 0.0f;
-        const uint32_t ones[4] = {0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u};
-        uint32_t piece = 0, dense_phase = 0;
-
+        if (!ok) {
+            // giving up: let the copies already issued land before the CTA's shared memory goes away
+            for (uint32_t j = (issued > S ? issued - S : 0); j < issued; ++j)
+                for (uint32_t spin = 0; spin < (1u << 20) && !mbar_try_wait(bar_full + 8 * (j % S), (j / S) & 1); ++spin) {}
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ tensor warp
         for (uint32_t u = u_begin, it = 0; u < u_end; ++u, ++it) {
-            const uint32_t s = it % S, ph = (it / S) & 1;
-            const uint32_t tn = u / KT, kt = u % KT;
-            const uint8_t* st = smem + s * p.stage_bytes;
-            if (!mbar_wait(bar_full + 8 * s, ph, abort_flag, p.status)) return;
-
-            const uint4* wp = reinterpret_cast<const uint4*>(st) + dw * 128 + lane;
-            uint4 wa[4];
+            const uint32_t s = it % S, ph = (it / S) & 1, b = it & 1;
+            uint8_t* st = smem + s * p.stage_bytes;
+            if (!warp_wait(bar_full + 8 * s, ph, abort_flag, p.status)) break;
+            // activation rows -> canonical K-major core matrices (8 rows x 16 B each, chunk-major);
+            // rows beyond M are zero.  Per-group sums of each row go to xsum[group][row].
+            {
+                constexpr int LPR = 32 / (NMMA < 32 ? NMMA : 32);   // lanes per row: 2 (N = 16) or 1 (N = 32)
+                constexpr int CPL = 16 / LPR;                        // 16-byte chunks per lane
+                const int m = lane % NMMA, part = lane / NMMA;
+                const bool real = (uint32_t)m < p.M;
+                const uint8_t* src = st + p.off_xraw + m * kXRowBytes + part * CPL * 16;
+                uint8_t* dst = st + p.off_xcan + ((part * CPL) * (NMMA / 8) + (m >> 3)) * 128 + (m & 7) * 16;
+                float sum[2] = {0.0f, 0.0f};
 #pragma unroll
-            for (int j = 0; j < 4; ++j) wa[j] = wp[j * 32];
-            const uint8_t* xrow = st + p.off_x + g * kXRowBytes + t * 16;
-            const uint16_t* sc = reinterpret_cast<const uint16_t*>(st + p.off_sz);
-
-#pragma unroll
-            for (int gi = 0; gi < GPS; ++gi) {
-                float accg[2][MO][4], xs[MO][4];
-#pragma unroll
-                for (int o = 0; o < MO; ++o)
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        accg[0][o][i] = 0.0f;
-                        accg[1][o][i] = 0.0f;
-                        xs[o][i] = 0.0f;
-                    }
-#pragma unroll
-                for (int kb = gi * (4 / GPS); kb < (gi + 1) * (4 / GPS); ++kb) {
-                    uint4 xb[MO];
-#pragma unroll
-                    for (int o = 0; o < MO; ++o)
-                        xb[o] = *reinterpret_cast<const uint4*>(xrow + o * 8 * kXRowBytes + kb * 64);
-#pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        const int ks = 2 * kb + e;
-#pragma unroll
-                        for (int ns = 0; ns < 2; ++ns) {
-                            const uint4 w4 = wa[ns * 2 + (ks >> 2)];
-                            const uint32_t w = (ks & 3) == 0 ? w4.x : (ks & 3) == 1 ? w4.y : (ks & 3) == 2 ? w4.z : w4.w;
-                            uint32_t a[4];
-                            a[0] = codes_to_bf16x2(w);
-                            a[1] = codes_to_bf16x2(w >> 4);
-                            a[2] = codes_to_bf16x2(w >> 8);
-                            a[3] = codes_to_bf16x2(w >> 12);
-#pragma unroll
-                            for (int o = 0; o < MO; ++o)
-                                mma_bf16(accg[ns][o], a, e ? xb[o].z : xb[o].x, e ? xb[o].w : xb[o].y);
-                        }
-#pragma unroll
-                        for (int o = 0; o < MO; ++o) mma_bf16(xs[o], ones, e ? xb[o].z : xb[o].x, e ? xb[o].w : xb[o].y);
-                    }
+                for (int c = 0; c < CPL; ++c) {
+                    uint4 v = make_uint4(0, 0, 0, 0);
+                    if (real) v = *reinterpret_cast<const uint4*>(src + c * 16);
+                    *reinterpret_cast<uint4*>(dst + c * (NMMA / 8) * 128) = v;
+                    const float t = (bf16lo(v.x) + bf16hi(v.x)) + (bf16lo(v.y) + bf16hi(v.y)) + (bf16lo(v.z) + bf16hi(v.z)) +
+                                    (bf16lo(v.w) + bf16hi(v.w));
+                    sum[(LPR == 1 && c >= 8) ? 1 : 0] += t;
                 }
-                // once per group: acc += s * (sum x (128+q) - (128+z) sum x)     (Eq. 3 inside Eq. 1)
+                float* xsum = reinterpret_cast<float*>(st + p.off_xsum);
+                if (LPR == 2) {
+                    // lane `part` holds k 0..63 or 64..127 of its row
+                    const float other = __shfl_xor_sync(0xffffffffu, sum[0], 16);
+                    if (GPS == 2) xsum[part * NMMA + m] = sum[0];
+                    else if (part == 0) xsum[m] = sum[0] + other;
+                } else {
+                    if (GPS == 2) { xsum[m] = sum[0]; xsum[NMMA + m] = sum[1]; }
+                    else xsum[m] = sum[0] + sum[1];
+                }
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (!warp_wait(bar_a_ready + 8 * b, (it >> 1) & 1, abort_flag, p.status)) break;
+            tc_fence_after();
+            if (lane == 0) {
+                const uint32_t xcan = smem_u32(st + p.off_xcan);
 #pragma unroll
-                for (int ns = 0; ns < 2; ++ns)
+                for (int ti = 0; ti < NT128; ++ti)
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const int nl = dw * 32 + ns * 16 + h * 8 + g;
-                        const float sv = bf16_bits_to_float(sc[gi * BN + nl]);
-                        const float zc = -(128.0f + bf16_bits_to_float(sc[(GPS + gi) * BN + nl]));
-#pragma unroll
-                        for (int o = 0; o < MO; ++o) {
-                            accf[ns][o][2 * h + 0] = fmaf(sv, fmaf(zc, xs[o][0], accg[ns][o][2 * h + 0]), accf[ns][o][2 * h + 0]);
-                            accf[ns][o][2 * h + 1] = fmaf(sv, fmaf(zc, xs[o][1], accg[ns][o][2 * h + 1]), accf[ns][o][2 * h + 1]);
-                        }
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const int gi = ks / (8 / GPS);
+                        const uint32_t d = tmem_base + ti * 256 + 128 + b * DCOLS + gi * NMMA;
+                        const uint32_t a = tmem_base + ti * 256 + b * 64 + ks * 8;
+                        const uint64_t bd = make_b_desc(xcan + ks * 2 * (NMMA / 8) * 128, (NMMA / 8) * 128, 128);
+                        umma_ts(d, a, bd, IDESC, (ks % (8 / GPS)) != 0);
                     }
+                umma_commit(bar_d_ready + 8 * b);   // accumulators of this unit are complete
+                umma_commit(bar_empty + 8 * s);     // and the stage's activation operand has been read
+                mbar_arrive(bar_d_ready + 8 * b);   // release of the xsum stores above
             }
             __syncwarp();
+        }
+    } else if (warp >= 4 && warp < 4 + NDW) {
+        // ------------------------------------------------------------------ dense: thread = column
+        const int dw = warp - 4;
+        const int col = dw * 32 + lane;                       // column inside the tile
+        const uint32_t t_lane = ((uint32_t)((dw & 3) * 32)) << 16;
+        const uint32_t t_tile = tmem_base + (uint32_t)(dw >> 2) * 256 + t_lane;
+        float accf[NMMA];
+#pragma unroll
+        for (int i = 0; i < NMMA; ++i) accf[i] = 0.0f;
+        uint32_t piece = 0, dense_phase = 0;
+        bool ok = true;
+
+        // scale / zero-point / activation sums of one finished unit, then release its stage
+        auto epilogue = [&](uint32_t e) -> bool {
+            const uint32_t s = e % S, b = e & 1;
+            const uint8_t* st = smem + s * p.stage_bytes;
+            if (!warp_wait(bar_d_ready + 8 * b, (e >> 1) & 1, abort_flag, p.status)) return false;
+            tc_fence_after();
+            const uint16_t* sc = reinterpret_cast<const uint16_t*>(st + p.off_sz);
+            const float4* xsum = reinterpret_cast<const float4*>(st + p.off_xsum);
+#pragma unroll
+            for (int gi = 0; gi < GPS; ++gi) {
+                const float sv = bf16_bits_to_float(sc[gi * BN + col]);
+                const float zc = -(128.0f + bf16_bits_to_float(sc[(GPS + gi) * BN + col]));
+#pragma unroll
+                for (int h = 0; h < NB16; ++h) {
+                    float d[16];
+                    tmem_ld16(t_tile + 128 + b * DCOLS + gi * NMMA + h * 16, d);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const float4 xs = xsum[(gi * NMMA + h * 16) / 4 + i];
+                        accf[h * 16 + 4 * i + 0] = fmaf(sv, fmaf(zc, xs.x, d[4 * i + 0]), accf[h * 16 + 4 * i + 0]);
+                        accf[h * 16 + 4 * i + 1] = fmaf(sv, fmaf(zc, xs.y, d[4 * i + 1]), accf[h * 16 + 4 * i + 1]);
+                        accf[h * 16 + 4 * i + 2] = fmaf(sv, fmaf(zc, xs.z, d[4 * i + 2]), accf[h * 16 + 4 * i + 2]);
+                        accf[h * 16 + 4 * i + 3] = fmaf(sv, fmaf(zc, xs.w, d[4 * i + 3]), accf[h * 16 + 4 * i + 3]);
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
             if (lane == 0) mbar_arrive(bar_empty + 8 * s);
+            return true;
+        };
+
+        uint32_t pending = 0xffffffffu;      // unit whose epilogue has not run yet
+        for (uint32_t u = u_begin, it = 0; u < u_end && ok; ++u, ++it) {
+            const uint32_t s = it % S, ph = (it / S) & 1, b = it & 1;
+            const uint32_t tn = u / KT, kt = u % KT;
+            const uint8_t* st = smem + s * p.stage_bytes;
+            if (!warp_wait(bar_full + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
+            // unpack: four 16-byte chunks = 128 codes of this column -> A operand rows in TMEM
+            const uint4* wp = reinterpret_cast<const uint4*>(st) + col;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint4 w4 = wp[j * BN];
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    const uint32_t w0 = hf ? w4.z : w4.x, w1 = hf ? w4.w : w4.y;
+                    uint32_t a[8];
+                    a[0] = codes_to_bf16x2(w0);
+                    a[1] = codes_to_bf16x2(w0 >> 4);
+                    a[2] = codes_to_bf16x2(w0 >> 8);
+                    a[3] = codes_to_bf16x2(w0 >> 12);
+                    a[4] = codes_to_bf16x2(w1);
+                    a[5] = codes_to_bf16x2(w1 >> 4);
+                    a[6] = codes_to_bf16x2(w1 >> 8);
+                    a[7] = codes_to_bf16x2(w1 >> 12);
+                    tmem_st8(t_tile + b * 64 + (j * 2 + hf) * 8, a);
+                }
+            }
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_a_ready + 8 * b);
+            // while the tensor core works on this unit, finish the previous one
+            if (pending != 0xffffffffu) {
+                if (!epilogue(pending)) { ok = false; break; }
+            }
+            pending = it;
 
             if (kt == KT - 1 || u == u_end - 1) {
                 // ---------------------------------------------------------- end of a piece
+                if (!epilogue(pending)) { ok = false; break; }
+                pending = 0xffffffffu;
                 if (SPARSE) {
-                    if (!mbar_wait(bar_sparse_done, piece & 1, abort_flag, p.status)) return;
+                    if (!warp_wait(bar_sparse_done, piece & 1, abort_flag, p.status)) { ok = false; break; }
+                    float4* cp = reinterpret_cast<float4*>(shc + col * LDC);
 #pragma unroll
-                    for (int ns = 0; ns < 2; ++ns)
-#pragma unroll
-                        for (int h = 0; h < 2; ++h)
-#pragma unroll
-                            for (int o = 0; o < MO; ++o) {
-                                float2* cp = reinterpret_cast<float2*>(shc + (dw * 32 + ns * 16 + h * 8 + g) * LDC + o * 8 + 2 * t);
-                                const float2 v = *cp;
-                                accf[ns][o][2 * h + 0] += v.x;
-                                accf[ns][o][2 * h + 1] += v.y;
-                                *cp = make_float2(0.0f, 0.0f);
-                            }
+                    for (int i = 0; i < NMMA / 4; ++i) {
+                        const float4 v = cp[i];
+                        accf[4 * i + 0] += v.x;
+                        accf[4 * i + 1] += v.y;
+                        accf[4 * i + 2] += v.z;
+                        accf[4 * i + 3] += v.w;
+                        cp[i] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                    }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_dense_done);
                 }
@@ -384,124 +544,105 @@ __global__ void __launch_bounds__(32 * (1 + BN / 32 + 8), 1) fq_fused_kernel(con
                 const bool full_piece = (piece_k0 == 0) && (kt == KT - 1);
                 bool write_y = full_piece;
                 if (!full_piece) {
-                    // FP32 partial in fragment order; the last CTA to arrive sums them in CTA order
+                    // FP32 partial [m][column]; the last CTA to arrive sums them in CTA order
                     const uint32_t which = (u_begin / KT == tn) ? 0u : 1u;
                     float* slot = p.partials + ((size_t)blockIdx.x * 2 + which) * (size_t)(BN * LDC);
 #pragma unroll
-                    for (int ns = 0; ns < 2; ++ns)
-#pragma unroll
-                        for (int o = 0; o < MO; ++o)
-#pragma unroll
-                            for (int i = 0; i < 4; ++i)
-                                __stcg(slot + (size_t)((ns * MO + o) * 4 + i) * (NDW * 32) + dtid, accf[ns][o][i]);
+                    for (int m = 0; m < NMMA; ++m)
+                        if ((uint32_t)m < p.M) __stcg(slot + m * BN + col, accf[m]);
                     __threadfence();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_dense);
-                    if (!mbar_wait(bar_dense, dense_phase & 1, abort_flag, p.status)) return;
+                    if (!warp_wait(bar_dense, dense_phase & 1, abort_flag, p.status)) { ok = false; break; }
                     ++dense_phase;
                     const uint32_t c_first = cta_of_unit(u_tile0, q, r), c_last = cta_of_unit(u_tile0 + KT - 1, q, r);
-                    if (dtid == 0) {
+                    if (dw == 0 && lane == 0) {
                         const uint32_t old = atomicAdd(p.counters + tn, 1u);
                         *last_flag = (old == c_last - c_first) ? 1u : 0u;
                     }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_dense);
-                    if (!mbar_wait(bar_dense, dense_phase & 1, abort_flag, p.status)) return;
+                    if (!warp_wait(bar_dense, dense_phase & 1, abort_flag, p.status)) { ok = false; break; }
                     ++dense_phase;
                     if (*last_flag) {
                         write_y = true;
                         __threadfence();
-                        float tot[2][MO][4];
 #pragma unroll
-                        for (int ns = 0; ns < 2; ++ns)
-#pragma unroll
-                            for (int o = 0; o < MO; ++o)
-#pragma unroll
-                                for (int i = 0; i < 4; ++i) tot[ns][o][i] = 0.0f;
+                        for (int m = 0; m < NMMA; ++m) accf[m] = 0.0f;
                         for (uint32_t c = c_first; c <= c_last; ++c) {
                             const uint32_t wch = (unit_begin_of(c, q, r) / KT == tn) ? 0u : 1u;
                             const float* sl = p.partials + ((size_t)c * 2 + wch) * (size_t)(BN * LDC);
 #pragma unroll
-                            for (int ns = 0; ns < 2; ++ns)
-#pragma unroll
-                                for (int o = 0; o < MO; ++o)
-#pragma unroll
-                                    for (int i = 0; i < 4; ++i)
-                                        tot[ns][o][i] += __ldcg(sl + (size_t)((ns * MO + o) * 4 + i) * (NDW * 32) + dtid);
+                            for (int m = 0; m < NMMA; ++m)
+                                if ((uint32_t)m < p.M) accf[m] += __ldcg(sl + m * BN + col);
                         }
-#pragma unroll
-                        for (int ns = 0; ns < 2; ++ns)
-#pragma unroll
-                            for (int o = 0; o < MO; ++o)
-#pragma unroll
-                                for (int i = 0; i < 4; ++i) accf[ns][o][i] = tot[ns][o][i];
-                        if (dtid == 0) p.counters[tn] = 0;  // ready for the next call
+                        if (dw == 0 && lane == 0) p.counters[tn] = 0;  // ready for the next call
                     }
                 }
                 if (write_y) {
 #pragma unroll
-                    for (int ns = 0; ns < 2; ++ns)
-#pragma unroll
-                        for (int h = 0; h < 2; ++h)
-#pragma unroll
-                            for (int o = 0; o < MO; ++o)
-#pragma unroll
-                                for (int j = 0; j < 2; ++j) {
-                                    const uint32_t m = o * 8 + 2 * t + j;
-                                    if (m < p.M)
-                                        p.Y[(size_t)m * p.N + (size_t)tn * BN + dw * 32 + ns * 16 + h * 8 + g] =
-                                            float_to_bf16_bits(accf[ns][o][2 * h + j]);
-                                }
+                    for (int m = 0; m < NMMA; ++m)
+                        if ((uint32_t)m < p.M) p.Y[(size_t)m * p.N + (size_t)tn * BN + col] = float_to_bf16_bits(accf[m]);
                 }
 #pragma unroll
-                for (int ns = 0; ns < 2; ++ns)
-#pragma unroll
-                    for (int o = 0; o < MO; ++o)
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) accf[ns][o][i] = 0.0f;
+                for (int m = 0; m < NMMA; ++m) accf[m] = 0.0f;
                 ++piece;
             }
         }
-        return;
+    } else if (SPARSE && (warp == 2 || warp == 3 || warp >= 4 + NDW)) {
+        // ------------------------------------------------------------------ sparse
+        const uint32_t sw = warp < 4 ? warp - 2 : warp - (4 + NDW) + 2;
+        if (sw + 1 <= nsw) {
+            const uint32_t nbb = p.NB >> 5;            // blocks of 32 buckets
+            const uint32_t bb = sw % nbb, og = sw / nbb, n_og = nsw / nbb;
+            const uint32_t bucket = bb * 32 + lane;
+            const uint32_t n_oct = (p.M + 7) >> 3;
+            uint8_t* xt = smem + p.off_xt + sw * 2048;
+            uint32_t piece = 0;
+            for (uint32_t u = u_begin, it = 0; u < u_end; ++u, ++it) {
+                const uint32_t s = it % S, ph = (it / S) & 1;
+                const uint32_t kt = u % KT;
+                const uint8_t* st = smem + s * p.stage_bytes;
+                if (!warp_wait(bar_full + 8 * s, ph, abort_flag, p.status)) break;
+                const uint32_t info = reinterpret_cast<const uint32_t*>(st + p.off_info)[bucket];
+                const uint32_t off = info & 0xffffu, cnt = info >> 16;
+                const uint4* pk_s = reinterpret_cast<const uint4*>(st + p.off_coo);
+                const uint4* pk_g = nullptr;
+                if (off + cnt > p.coo_cap) pk_g = p.packed + __ldg(p.indptr + u);  // tail of an oversized tile
+                for (uint32_t o = og; o < n_oct; o += n_og) {
+                    transpose_octet(smem_u32(st + p.off_xraw) + o * 8 * kXRowBytes, xt, lane);
+                    __syncwarp();
+                    float* shc_o = shc + o * 8;
+                    for (uint32_t i = 0; i < cnt; ++i) {
+                        const uint32_t idx = off + i;
+                        const uint4 pk = (idx < p.coo_cap) ? pk_s[idx] : __ldg(pk_g + idx);
+                        apply_packet(pk, xt, shc_o, LDC);
+                    }
+                    __syncwarp();
+                }
+                if (lane == 0) mbar_arrive(bar_empty + 8 * s);
+                if (kt == KT - 1 || u == u_end - 1) {
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_sparse_done);
+                    if (!warp_wait(bar_dense_done, piece & 1, abort_flag, p.status)) break;
+                    ++piece;
+                }
+            }
+        }
     }
 
-    if (SPARSE) {
-        // ------------------------------------------------------------------ sparse
-        const uint32_t sw = warp - 1 - NDW;
-        const uint32_t nbb = p.NB >> 5;            // blocks of 32 buckets
-        const uint32_t bb = sw % nbb, og = sw / nbb, n_og = nsw / nbb;
-        const uint32_t bucket = bb * 32 + lane;
-        uint8_t* xt = smem + p.off_xt + sw * 2048;
-        uint32_t piece = 0;
-        for (uint32_t u = u_begin, it = 0; u < u_end; ++u, ++it) {
-            const uint32_t s = it % S, ph = (it / S) & 1;
-            const uint32_t kt = u % KT;
-            const uint8_t* st = smem + s * p.stage_bytes;
-            if (!mbar_wait(bar_full + 8 * s, ph, abort_flag, p.status)) return;
-            const uint32_t info = reinterpret_cast<const uint32_t*>(st + p.off_info)[bucket];
-            const uint32_t off = info & 0xffffu, cnt = info >> 16;
-            const uint4* pk_s = reinterpret_cast<const uint4*>(st + p.off_coo);
-            const uint4* pk_g = nullptr;
-            if (off + cnt > p.coo_cap) pk_g = p.packed + __ldg(p.indptr + u);  // tail of an oversized tile
-            for (uint32_t o = og; o < (uint32_t)MO; o += n_og) {
-                transpose_octet(smem_u32(st + p.off_x) + o * 8 * kXRowBytes, xt, lane);
-                __syncwarp();
-                float* shc_o = shc + o * 8;
-                for (uint32_t i = 0; i < cnt; ++i) {
-                    const uint32_t idx = off + i;
-                    const uint4 pk = (idx < p.coo_cap) ? pk_s[idx] : __ldg(pk_g + idx);
-                    apply_packet(pk, xt, shc_o, LDC);
-                }
-                __syncwarp();
-            }
-            if (lane == 0) mbar_arrive(bar_empty + 8 * s);
-            if (kt == KT - 1 || u == u_end - 1) {
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_sparse_done);
-                if (!mbar_wait(bar_dense_done, piece & 1, abort_flag, p.status)) return;
-                ++piece;
-            }
+    // ---------------------------------------------------------------------- common exit
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        // every tcgen05 operation of this CTA must have retired before its TMEM is released
+        if (lane == 0) {
+            umma_commit(bar_final);
+            for (uint32_t spin = 0; spin < (1u << 24) && !mbar_try_wait(bar_final, 0); ++spin) {}
         }
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
     }
 }
 
@@ -573,17 +714,22 @@ static int sm_count_cached() {
     return cached[dev];
 }
 
+static inline uint32_t nb16_of(uint32_t m) { return m <= 16 ? 1u : 2u; }
+
 static fq_status_t make_plan(const fq_layout_t* L, uint32_t M, bool sparse, Plan& pl) {
     const uint32_t BN = L->BN, NB = L->buckets_per_tile, GPS = kBK / L->group;
-    const uint32_t MO = M <= 8 ? 1 : (M <= 16 ? 2 : 4);
+    const uint32_t NMMA = 16 * nb16_of(M);
     const uint32_t NDW = BN / 32;
     uint32_t nsw = 0;
-    if (sparse) nsw = std::min<uint32_t>(8, (NB / 32) * MO);
+    if (sparse) {
+        const uint32_t nbb = NB / 32, n_oct = (M + 7) / 8;
+        nsw = nbb * std::min<uint32_t>(n_oct, std::max<uint32_t>(1, 8 / nbb));
+    }
     Params& p = pl.p;
     std::memset(&p, 0, sizeof(p));
     p.M = M; p.K = L->K; p.N = L->N; p.KT = L->K / kBK; p.NT = L->N / BN; p.NB = NB; p.nsw = nsw;
-    const uint32_t w_bytes = 16 * BN * 4, sz_bytes = 2 * GPS * BN * 2, x_bytes = 8 * MO * kXRowBytes;
-    const uint32_t fixed = (sparse ? BN * 8 * MO * 4 + nsw * 2048 : 0) + 1024;
+    const uint32_t w_bytes = 16 * BN * 4, sz_bytes = 2 * GPS * BN * 2;
+    const uint32_t fixed = (sparse ? BN * NMMA * 4 + nsw * 2048 : 0) + 1024;
     uint32_t cap = 0;
     if (sparse) {
         cap = L->max_tile_packets ? round_up(L->max_tile_packets, 8) : 256;
@@ -592,22 +738,23 @@ static fq_status_t make_plan(const fq_layout_t* L, uint32_t M, bool sparse, Plan
     uint32_t stage = 0, S = 0;
     for (;;) {
         p.off_sz = w_bytes;
-        p.off_x = p.off_sz + round_up(sz_bytes, 128);
-        p.off_info = p.off_x + round_up(x_bytes, 128);
+        p.off_xraw = p.off_sz + round_up(sz_bytes, 128);
+        p.off_xcan = p.off_xraw + round_up(NMMA * kXRowBytes, 128);
+        p.off_xsum = p.off_xcan + NMMA * 256;
+        p.off_info = p.off_xsum + round_up(GPS * NMMA * 4, 128);
         p.off_coo = p.off_info + (sparse ? round_up(NB * 4, 128) : 0);
-        stage = p.off_coo + cap * 16;
-        stage = round_up(stage, 128);
+        stage = round_up(p.off_coo + cap * 16, 128);
         S = std::min<uint32_t>(8, (kSmemBudget - fixed) / stage);
         if (S >= 4 || cap <= 64) break;
         cap = std::max<uint32_t>(64, cap / 2);  // oversized tiles read their tail from global memory
     }
-    if (S < 2) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "shared-memory stages do not fit");
+    if (S < 3) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "shared-memory stages do not fit");
     p.coo_cap = cap; p.stages = S; p.stage_bytes = stage;
     p.off_shc = S * stage;
-    p.off_xt = p.off_shc + (sparse ? BN * 8 * MO * 4 : 0);
+    p.off_xt = p.off_shc + (sparse ? BN * NMMA * 4 : 0);
     p.off_bar = p.off_xt + nsw * 2048;
     pl.smem = p.off_bar + 1024;
-    pl.threads = 32 * (1 + NDW + nsw);
+    pl.threads = 32 * (4 + NDW + (nsw > 2 ? nsw - 2 : 0));
     const int sms = sm_count_cached();
     if (sms <= 0) return fail(FQ_ERR_CUDA, "no CUDA device: %s", cudaGetErrorString(cudaGetLastError()));
     pl.grid = std::min<uint32_t>({(uint32_t)sms, kMaxCtas, p.NT * p.KT});
@@ -625,11 +772,28 @@ static KernelFn pick_group(uint32_t g, bool sparse) {
     return g == 64 ? pick_sparse<BN, MO, 64>(sparse) : pick_sparse<BN, MO, 128>(sparse);
 }
 template <int BN>
-static KernelFn pick_mo(uint32_t mo, uint32_t g, bool sparse) {
-    return mo == 1 ? pick_group<BN, 1>(g, sparse) : mo == 2 ? pick_group<BN, 2>(g, sparse) : pick_group<BN, 4>(g, sparse);
+static KernelFn pick_mo(uint32_t nb16, uint32_t g, bool sparse) {
+    return nb16 == 1 ? pick_group<BN, 1>(g, sparse) : pick_group<BN, 2>(g, sparse);
 }
 static KernelFn pick_kernel(uint32_t bn, uint32_t mo, uint32_t g, bool sparse) {
     return bn == 128 ? pick_mo<128>(mo, g, sparse) : pick_mo<256>(mo, g, sparse);
+}
+
+// cudaFuncSetAttribute costs several microseconds: do it once per (kernel, device).
+static cudaError_t ensure_smem_attr(const void* fn, int bytes) {
+    struct Seen { const void* fn; int dev; };
+    static Seen seen[256];
+    static int nseen = 0;
+    static std::mutex mu;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> lock(mu);
+    for (int i = 0; i < nseen; ++i)
+        if (seen[i].fn == fn && seen[i].dev == dev) return cudaSuccess;
+    e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess && nseen < 256) seen[nseen++] = Seen{fn, dev};
+    return e;
 }
 
 static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
@@ -662,9 +826,8 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
         p.status = (uint32_t*)workspace;
         p.counters = (uint32_t*)((uint8_t*)workspace + kWsHeaderBytes);
         p.partials = (float*)((uint8_t*)workspace + kWsHeaderBytes + kWsCounterBytes);
-        const uint32_t MO = mb <= 8 ? 1 : (mb <= 16 ? 2 : 4);
-        KernelFn fn = pick_kernel(L->BN, MO, L->group, sparse);
-        cudaError_t e = cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget);
+        KernelFn fn = pick_kernel(L->BN, nb16_of(mb), L->group, sparse);
+        cudaError_t e = ensure_smem_attr((const void*)fn, (int)kSmemBudget);
         if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
         fn<<<pl.grid, pl.threads, pl.smem, (cudaStream_t)stream>>>(p);
         e = cudaGetLastError();
@@ -683,8 +846,7 @@ fq_status_t fq_workspace_bytes(const fq_layout_t* L, uint32_t M, size_t* bytes) 
     if (!layout_ok(L) || !bytes) return fail(FQ_ERR_INVALID_ARG, "bad layout or null output");
     if (M < 1 || M > FQ_MAX_M) return fail(FQ_ERR_INVALID_ARG, "M = %u outside [1, %u]", M, FQ_MAX_M);
     const uint32_t mb = std::min<uint32_t>(M, 32);
-    const uint32_t MO = mb <= 8 ? 1 : (mb <= 16 ? 2 : 4);
-    *bytes = kWsHeaderBytes + kWsCounterBytes + (size_t)kMaxCtas * 2 * L->BN * 8 * MO * 4;
+    *bytes = kWsHeaderBytes + kWsCounterBytes + (size_t)kMaxCtas * 2 * L->BN * 16 * nb16_of(mb) * 4;
     return FQ_OK;
 }
 
@@ -716,13 +878,13 @@ fq_status_t fq_unfused_spmm(const fq_layout_t* L, const void* X, uint32_t M, con
         uint16_t* y = (uint16_t*)Y + (size_t)m0 * L->N;
         cudaError_t e;
         if (L->BN == 128) {
-            e = cudaFuncSetAttribute((const void*)fq_spmm_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 65536);
+            e = ensure_smem_attr((const void*)fq_spmm_kernel<128>, 65536);
             if (e == cudaSuccess)
                 fq_spmm_kernel<128><<<L->N / 128, 256, smem, (cudaStream_t)cuda_stream>>>(
                     x, (const uint32_t*)tile_indptr, (const uint32_t*)bucket_info, (const uint4*)packed_outliers, y, mb,
                     L->K, L->N, L->buckets_per_tile, MO);
         } else {
-            e = cudaFuncSetAttribute((const void*)fq_spmm_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, 65536);
+            e = ensure_smem_attr((const void*)fq_spmm_kernel<256>, 65536);
             if (e == cudaSuccess)
                 fq_spmm_kernel<256><<<L->N / 256, 256, smem, (cudaStream_t)cuda_stream>>>(
                     x, (const uint32_t*)tile_indptr, (const uint32_t*)bucket_info, (const uint4*)packed_outliers, y, mb,

@@ -249,23 +249,13 @@ def test_decode_wq_against_a_direct_packer():
     KT = K // 128
     for row in range(K):
         kt, kr = divmod(row, 128)
-        kb32, r32 = divmod(kr, 32)
-        t, r8 = divmod(r32, 8)
-        odd, r4 = divmod(r8, 4)
-        rhi, h = divmod(r4, 2)
-        ks = 2 * kb32 + odd
+        j, r32 = divmod(kr, 32)
+        w, r8 = divmod(r32, 8)
+        i, h = divmod(r8, 2)
         for col in range(N):
-            tn, cr = divmod(col, BN)
-            w, c32 = divmod(cr, 32)
-            ns, c16 = divmod(c32, 16)
-            rlo, grp = divmod(c16, 8)
-            r = rlo + 2 * rhi
-            p = r + 4 * h
-            j = ns * 2 + (ks >> 2)
-            c = ks & 3
-            lane = grp * 4 + t
-            idx = (tn * KT + kt) * 16 * BN + ((w * 4 + j) * 32 + lane) * 4 + c
-            words[idx] |= np.uint32(int(q[row, col]) << (4 * p))
+            tn, t = divmod(col, BN)
+            idx = (tn * KT + kt) * 16 * BN + (j * BN + t) * 4 + w
+            words[idx] |= np.uint32(int(q[row, col]) << (4 * (i + 4 * h)))
     assert np.array_equal(oracle.decode_wq(words, K, N, BN), q)
 
 

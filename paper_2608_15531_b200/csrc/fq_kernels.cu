@@ -3,12 +3,14 @@
 //
 // Kernel shape (one persistent CTA per SM, warp-specialised):
 //   warp 0        producer: per (tile, k-step) unit, bulk-copies (cp.async.bulk + mbarrier expect_tx)
-//                 the unit's INT4 chunk, scale/zero rows, bucket_info slice, packet range and the M
-//                 activation rows into a ring of shared-memory stages
-//   warp 1        tensor: owns the TMEM allocation; per unit re-lays the activation rows into the
-//                 canonical K-major operand layout, computes the per-group activation sums, and
-//                 issues tcgen05.mma (A = dequantised weights in TMEM, B = activations in shared
-//                 memory, D = FP32 in TMEM); completion is signalled with tcgen05.commit
+//                 the unit's INT4 chunk, scale/zero rows, bucket_info slice and packet range into a
+//                 ring of shared-memory stages
+//   warp 1        tensor: owns the TMEM allocation and issues tcgen05.mma (A = dequantised weights
+//                 in TMEM, B = activations in shared memory, D = FP32 in TMEM); completion is
+//                 signalled with tcgen05.commit
+//   warp 2        activations: reads the unit's M x 128 activation block from global memory (it
+//                 stays in L2), lays it out as the canonical K-major MMA operand in the stage, and
+//                 writes the per-group sums of each row
 //   dense warps   thread = output column: unpacks its 128 codes of the unit with lop3 into BF16
 //                 (128 + q), stores them as the A operand into TMEM (tcgen05.st), and one unit later
 //                 reads the FP32 group sums back (tcgen05.ld) and applies scale and zero-point once
@@ -32,10 +34,17 @@
 namespace fq {
 
 constexpr int kBK = 128;
-constexpr int kXRowBytes = 272;        // 256 B of activations + 16 B pad: conflict-free ldmatrix rows
 constexpr int kSmemBudget = 232448;    // 227 KB per CTA on sm_100
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 constexpr uint32_t kTmemCols = 512;
+
+#ifdef FQ_TRACE
+// Developer build only: cycle stamps of CTA 0's first iterations, [role][iteration][event].
+__device__ unsigned long long g_trace[4 * 64 * 8];
+#define FQ_STAMP(role, it, ev) do { if (blockIdx.x == 0 && (it) < 64 && lane == 0) g_trace[((role) * 64 + (it)) * 8 + (ev)] = clock64(); } while (0)
+#else
+#define FQ_STAMP(role, it, ev) do {} while (0)
+#endif
 
 struct Params {
     const uint16_t* X;
@@ -52,7 +61,7 @@ struct Params {
     uint32_t M, K, N, KT, NT;
     uint32_t NB, coo_cap, stages, nsw;
     // shared-memory offsets (bytes); the first five are relative to a stage
-    uint32_t stage_bytes, off_sz, off_xraw, off_xcan, off_xsum, off_info, off_coo;
+    uint32_t stage_bytes, off_sz, off_xcan, off_xsum, off_info, off_coo;
     uint32_t off_shc, off_xt, off_bar;
 };
 
@@ -163,15 +172,19 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&d)[16]) {
     for (int i = 0; i < 16; ++i) d[i] = __uint_as_float(r[i]);
 }
 // D[128 x N] (+)= A[128 x 16] (TMEM) * B[16 x N] (shared-memory descriptor), BF16 in, FP32 out
+// Called by the whole (converged) warp with warp-uniform operands; one elected lane issues.
 __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
-        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
-        " tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n}"
+        "{\n .reg .pred p, e;\n setp.ne.b32 p, %4, 0;\n elect.sync _|e, 0xffffffff;\n"
+        " @e tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n}"
         ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
         : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    asm volatile(
+        "{\n .reg .pred e;\n elect.sync _|e, 0xffffffff;\n"
+        " @e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}" ::"r"(bar)
+        : "memory");
 }
 // K-major, no swizzle: 8 rows x 16 B core matrices; LBO = step between the two K halves of one MMA,
 // SBO = step between 8-row groups.
@@ -186,6 +199,21 @@ __device__ __forceinline__ uint32_t cta_of_unit(uint32_t u, uint32_t q, uint32_t
     return u < big ? u / (q + 1) : r + (u - big) / q;
 }
 __device__ __forceinline__ uint32_t unit_begin_of(uint32_t c, uint32_t q, uint32_t r) { return c * q + min(c, r); }
+
+// Walks a CTA's units without integer division: ring slot s with its parity, tile tn, k-step kt.
+struct UnitIter {
+    uint32_t u, it, s, ph, tn, kt;
+    __device__ __forceinline__ UnitIter(uint32_t u_begin, uint32_t KT) : u(u_begin), it(0), s(0), ph(0) {
+        tn = u_begin / KT;
+        kt = u_begin - tn * KT;
+    }
+    __device__ __forceinline__ void next(uint32_t S, uint32_t KT) {
+        ++u;
+        ++it;
+        if (++s == S) { s = 0; ph ^= 1; }
+        if (++kt == KT) { kt = 0; ++tn; }
+    }
+};
 
 // ----------------------------------------------------------------------------- sparse step
 
@@ -247,12 +275,13 @@ __device__ __forceinline__ void apply_packet(const uint4 pk, const uint8_t* __re
     }
 }
 
-// Transpose 8 activation rows (row-major, kXRowBytes apart, 128 k each) into xt[k][8].
-__device__ __forceinline__ void transpose_octet(uint32_t xs_rows_u32, uint8_t* xt, int lane) {
+// Transpose one octet of activation rows into xt[k][8], reading the canonical operand layout
+// (core matrix of 16-byte chunk c and octet o at (c * n_oct + o) * 128, its 8 rows 16 B apart).
+__device__ __forceinline__ void transpose_octet(uint32_t xcan_u32, uint32_t n_oct, uint32_t o, uint8_t* xt, int lane) {
 #pragma unroll
     for (int kb = 0; kb < 4; ++kb) {
         uint32_t r0, r1, r2, r3;
-        const uint32_t addr = xs_rows_u32 + (lane & 7) * kXRowBytes + (kb * 4 + (lane >> 3)) * 16;
+        const uint32_t addr = xcan_u32 + ((kb * 4 + (lane >> 3)) * n_oct + o) * 128 + (lane & 7) * 16;
         ldmatrix_x4_trans(addr, r0, r1, r2, r3);
         // thread T holds rows m = 2(T%4), 2(T%4)+1 of column k = 8*block + T/4
         uint8_t* dst = xt + ((kb * 32) + (lane >> 2)) * 16 + (lane & 3) * 4;
@@ -267,7 +296,7 @@ __device__ __forceinline__ void transpose_octet(uint32_t xs_rows_u32, uint8_t* x
 
 // BN: tile columns (128 or 256).  NB16: batch columns of the MMA in units of 16 (1: M <= 16, 2: M <= 32).
 template <int BN, int NB16, int GROUP, bool SPARSE>
-__global__ void __launch_bounds__(32 * (4 + BN / 32 + 6), 1) fq_fused_kernel(const Params p) {
+__global__ void __launch_bounds__(32 * (4 + BN / 32 + 7), 1) fq_fused_kernel(const Params p) {
     constexpr int NDW = BN / 32;              // dense warps: one thread per tile column
     constexpr int NT128 = BN / 128;           // 128-row MMA tiles per unit
     constexpr int NMMA = 16 * NB16;           // MMA N: batch rows, padded
@@ -283,11 +312,12 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 6), 1) fq_fused_kernel(con
     const uint32_t S = p.stages;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
     const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * S;
-    const uint32_t bar_a_ready = bar_empty + 8 * S;      // [2]
+    const uint32_t bar_x_ready = bar_empty + 8 * S;      // [S]
+    const uint32_t bar_a_ready = bar_x_ready + 8 * S;    // [2]
     const uint32_t bar_d_ready = bar_a_ready + 16;       // [2]
     const uint32_t bar_sparse_done = bar_d_ready + 16, bar_dense_done = bar_sparse_done + 8;
     const uint32_t bar_dense = bar_dense_done + 8, bar_final = bar_dense + 8;
-    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 2 * S + 8);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 3 * S + 8);
     volatile uint32_t* last_flag = abort_flag + 1;
     volatile uint32_t* tmem_slot = abort_flag + 2;
     float* shc = reinterpret_cast<float*>(smem + p.off_shc);
@@ -297,11 +327,12 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 6), 1) fq_fused_kernel(con
         for (uint32_t s = 0; s < S; ++s) {
             mbar_init(bar_full + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, NDW + nsw + 1);
+            mbar_init(bar_x_ready + 8 * s, 1);
         }
         mbar_init(bar_a_ready, NDW);
         mbar_init(bar_a_ready + 8, NDW);
-        mbar_init(bar_d_ready, 2);
-        mbar_init(bar_d_ready + 8, 2);
+        mbar_init(bar_d_ready, 1);
+        mbar_init(bar_d_ready + 8, 1);
         mbar_init(bar_sparse_done, nsw ? nsw : 1);
         mbar_init(bar_dense_done, NDW);
         mbar_init(bar_dense, NDW);
@@ -333,8 +364,8 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 6), 1) fq_fused_kernel(con
         // ------------------------------------------------------------------ producer
         uint32_t ip_a = 0, ip_b = 0, issued = 0;
         bool ok = true;
-        for (uint32_t u = u_begin, it = 0; u < u_end; ++u, ++it) {
-            const uint32_t s = it % S, ph = (it / S) & 1;
+        for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
+            const uint32_t u = w.u, it = w.it, s = w.s, ph = w.ph;
             if (SPARSE && (it & 31) == 0) {  // this warp's next 32 packet ranges, one coalesced read
                 const uint32_t i = u + lane;
                 ip_a = (i <= U) ? __ldg(p.indptr + i) : 0;
@@ -347,34 +378,31 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 6), 1) fq_fused_kernel(con
                 npk = min(npk, p.coo_cap);
             }
             if (!warp_wait(bar_empty + 8 * s, ph ^ 1, abort_flag, p.status)) { ok = false; break; }
-            const uint32_t tn = u / KT, kt = u % KT;
+            FQ_STAMP(0, it, 0);
+            const uint32_t tn = w.tn, kt = w.kt;
             const uint32_t full = bar_full + 8 * s;
             const uint32_t st = smem_u32(smem) + s * p.stage_bytes;
             if (lane == 0) {
-                uint32_t bytes = W_BYTES + 2 * GPS * SZ_ROW + p.M * 256;
+                uint32_t bytes = W_BYTES + 2 * GPS * SZ_ROW;
                 if (SPARSE) bytes += p.NB * 4 + npk * 16;
                 mbar_arrive_expect_tx(full, bytes);
             }
             __syncwarp();
             if (lane == 0) {
                 bulk_g2s(st, p.wq + (size_t)u * W_BYTES, W_BYTES, full);
+#pragma unroll
+                for (int gi = 0; gi < GPS; ++gi) {
+                    const size_t row = (size_t)(kt * GPS + gi) * p.N + (size_t)tn * BN;
+                    bulk_g2s(st + p.off_sz + gi * SZ_ROW, p.scale + row, SZ_ROW, full);
+                    bulk_g2s(st + p.off_sz + (GPS + gi) * SZ_ROW, p.zero + row, SZ_ROW, full);
+                }
             } else if (lane == 1) {
-#pragma unroll
-                for (int gi = 0; gi < GPS; ++gi)
-                    bulk_g2s(st + p.off_sz + gi * SZ_ROW, p.scale + (size_t)(kt * GPS + gi) * p.N + (size_t)tn * BN, SZ_ROW, full);
-            } else if (lane == 2) {
-#pragma unroll
-                for (int gi = 0; gi < GPS; ++gi)
-                    bulk_g2s(st + p.off_sz + (GPS + gi) * SZ_ROW, p.zero + (size_t)(kt * GPS + gi) * p.N + (size_t)tn * BN, SZ_ROW, full);
-            } else if (lane == 3) {
-                if (SPARSE) bulk_g2s(st + p.off_info, p.info + (size_t)u * p.NB, p.NB * 4, full);
-            } else if (lane == 4) {
-                if (SPARSE && npk) bulk_g2s(st + p.off_coo, p.packed + pk0, npk * 16, full);
+                if (SPARSE) {
+                    bulk_g2s(st + p.off_info, p.info + (size_t)u * p.NB, p.NB * 4, full);
+                    if (npk) bulk_g2s(st + p.off_coo, p.packed + pk0, npk * 16, full);
+                }
             }
-            {
-                const uint32_t m = (lane + 27) & 31;  // rows start on lane 5
-                if (m < p.M) bulk_g2s(st + p.off_xraw + m * kXRowBytes, p.X + (size_t)m * p.K + (size_t)kt * kBK, 256, full);
-            }
+            FQ_STAMP(0, it, 1);
             issued = it + 1;
         }
         if (!ok) {
@@ -384,61 +412,76 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 6), 1) fq_fused_kernel(con
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ tensor warp
-        for (uint32_t u = u_begin, it = 0; u < u_end; ++u, ++it) {
-            const uint32_t s = it % S, ph = (it / S) & 1, b = it & 1;
-            uint8_t* st = smem + s * p.stage_bytes;
-            if (!warp_wait(bar_full + 8 * s, ph, abort_flag, p.status)) break;
-            // activation rows -> canonical K-major core matrices (8 rows x 16 B each, chunk-major);
-            // rows beyond M are zero.  Per-group sums of each row go to xsum[group][row].
-            {
-                constexpr int LPR = 32 / (NMMA < 32 ? NMMA : 32);   // lanes per row: 2 (N = 16) or 1 (N = 32)
-                constexpr int CPL = 16 / LPR;                        // 16-byte chunks per lane
-                const int m = lane % NMMA, part = lane / NMMA;
-                const bool real = (uint32_t)m < p.M;
-                const uint8_t* src = st + p.off_xraw + m * kXRowBytes + part * CPL * 16;
-                uint8_t* dst = st + p.off_xcan + ((part * CPL) * (NMMA / 8) + (m >> 3)) * 128 + (m & 7) * 16;
-                float sum[2] = {0.0f, 0.0f};
+        for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
+            const uint32_t it = w.it, s = w.s, ph = w.ph, b = w.it & 1;
+            if (!warp_wait(bar_x_ready + 8 * s, ph, abort_flag, p.status)) break;
+            FQ_STAMP(1, it, 0);
+            if (!warp_wait(bar_a_ready + 8 * b, (it >> 1) & 1, abort_flag, p.status)) break;
+            tc_fence_after();
+            FQ_STAMP(1, it, 2);
+            const uint64_t bd0 = make_b_desc(smem_u32(smem) + s * p.stage_bytes + p.off_xcan, (NMMA / 8) * 128, 128);
 #pragma unroll
-                for (int c = 0; c < CPL; ++c) {
-                    uint4 v = make_uint4(0, 0, 0, 0);
-                    if (real) v = *reinterpret_cast<const uint4*>(src + c * 16);
-                    *reinterpret_cast<uint4*>(dst + c * (NMMA / 8) * 128) = v;
-                    const float t = (bf16lo(v.x) + bf16hi(v.x)) + (bf16lo(v.y) + bf16hi(v.y)) + (bf16lo(v.z) + bf16hi(v.z)) +
-                                    (bf16lo(v.w) + bf16hi(v.w));
-                    sum[(LPR == 1 && c >= 8) ? 1 : 0] += t;
+            for (int ti = 0; ti < NT128; ++ti)
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const int gi = ks / (8 / GPS);
+                    const uint32_t d = tmem_base + ti * 256 + 128 + b * DCOLS + gi * NMMA;
+                    const uint32_t a = tmem_base + ti * 256 + b * 64 + ks * 8;
+                    umma_ts(d, a, bd0 + (uint64_t)((ks * 2 * (NMMA / 8) * 128) >> 4), IDESC, (ks % (8 / GPS)) != 0);
                 }
-                float* xsum = reinterpret_cast<float*>(st + p.off_xsum);
-                if (LPR == 2) {
-                    // lane `part` holds k 0..63 or 64..127 of its row
-                    const float other = __shfl_xor_sync(0xffffffffu, sum[0], 16);
-                    if (GPS == 2) xsum[part * NMMA + m] = sum[0];
-                    else if (part == 0) xsum[m] = sum[0] + other;
-                } else {
-                    if (GPS == 2) { xsum[m] = sum[0]; xsum[NMMA + m] = sum[1]; }
-                    else xsum[m] = sum[0] + sum[1];
-                }
+            umma_commit(bar_d_ready + 8 * b);   // accumulators of this unit are complete
+            umma_commit(bar_empty + 8 * s);     // and the stage's activation operand has been read
+            FQ_STAMP(1, it, 3);
+        }
+    } else if (warp == 2) {
+        // ------------------------------------------------------------------ activation warp
+        // lane -> (row m, part): CPL 16-byte chunks of that row; rows beyond M are zero
+        constexpr int LPR = 32 / (NMMA < 32 ? NMMA : 32);   // lanes per row: 2 (N = 16) or 1 (N = 32)
+        constexpr int CPL = 16 / LPR;                        // 16-byte chunks per lane
+        const int m = lane % NMMA, part = lane / NMMA;
+        const bool real = (uint32_t)m < p.M;
+        const uint8_t* xrow = reinterpret_cast<const uint8_t*>(p.X) + ((size_t)m * p.K) * 2 + part * CPL * 16;
+        uint4 nxt[CPL];
+        auto load = [&](uint32_t kt) {
+#pragma unroll
+            for (int c = 0; c < CPL; ++c) {
+                nxt[c] = make_uint4(0, 0, 0, 0);
+                if (real) nxt[c] = __ldg(reinterpret_cast<const uint4*>(xrow + (size_t)kt * 256 + c * 16));
+            }
+        };
+        if (u_begin < u_end) load(u_begin - (u_begin / KT) * KT);
+        for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
+            const uint32_t s = w.s, ph = w.ph;
+            uint8_t* st = smem + s * p.stage_bytes;
+            uint4 xv[CPL];
+#pragma unroll
+            for (int c = 0; c < CPL; ++c) xv[c] = nxt[c];
+            if (w.u + 1 < u_end) load(w.kt + 1 == KT ? 0u : w.kt + 1);   // next unit's block, while this one is laid out
+            if (!warp_wait(bar_empty + 8 * s, ph ^ 1, abort_flag, p.status)) break;
+            uint8_t* dst = st + p.off_xcan + ((part * CPL) * (NMMA / 8) + (m >> 3)) * 128 + (m & 7) * 16;
+            float sum[2] = {0.0f, 0.0f};
+#pragma unroll
+            for (int c = 0; c < CPL; ++c) {
+                const uint4 v = xv[c];
+                *reinterpret_cast<uint4*>(dst + c * (NMMA / 8) * 128) = v;
+                const float t = (bf16lo(v.x) + bf16hi(v.x)) + (bf16lo(v.y) + bf16hi(v.y)) + (bf16lo(v.z) + bf16hi(v.z)) +
+                                (bf16lo(v.w) + bf16hi(v.w));
+                sum[(LPR == 1 && c >= 8) ? 1 : 0] += t;
+            }
+            // per-group sums of each activation row -> xsum[group][row], needed by the dense epilogue
+            float* xsum = reinterpret_cast<float*>(st + p.off_xsum);
+            if (LPR == 2) {
+                // lane `part` holds k 0..63 or 64..127 of its row
+                const float other = __shfl_xor_sync(0xffffffffu, sum[0], 16);
+                if (GPS == 2) xsum[part * NMMA + m] = sum[0];
+                else if (part == 0) xsum[m] = sum[0] + other;
+            } else {
+                if (GPS == 2) { xsum[m] = sum[0]; xsum[NMMA + m] = sum[1]; }
+                else xsum[m] = sum[0] + sum[1];
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
-            if (!warp_wait(bar_a_ready + 8 * b, (it >> 1) & 1, abort_flag, p.status)) break;
-            tc_fence_after();
-            if (lane == 0) {
-                const uint32_t xcan = smem_u32(st + p.off_xcan);
-#pragma unroll
-                for (int ti = 0; ti < NT128; ++ti)
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {
-                        const int gi = ks / (8 / GPS);
-                        const uint32_t d = tmem_base + ti * 256 + 128 + b * DCOLS + gi * NMMA;
-                        const uint32_t a = tmem_base + ti * 256 + b * 64 + ks * 8;
-                        const uint64_t bd = make_b_desc(xcan + ks * 2 * (NMMA / 8) * 128, (NMMA / 8) * 128, 128);
-                        umma_ts(d, a, bd, IDESC, (ks % (8 / GPS)) != 0);
-                    }
-                umma_commit(bar_d_ready + 8 * b);   // accumulators of this unit are complete
-                umma_commit(bar_empty + 8 * s);     // and the stage's activation operand has been read
-                mbar_arrive(bar_d_ready + 8 * b);   // release of the xsum stores above
-            }
-            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_x_ready + 8 * s);
         }
     } else if (warp >= 4 && warp < 4 + NDW) {
         // ------------------------------------------------------------------ dense: thread = column
@@ -453,11 +496,13 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 6), 1) fq_fused_kernel(con
         bool ok = true;
 
         // scale / zero-point / activation sums of one finished unit, then release its stage
-        auto epilogue = [&](uint32_t e) -> bool {
-            const uint32_t s = e % S, b = e & 1;
+        auto epilogue = [&](uint32_t e, uint32_t s, uint32_t ph) -> bool {
+            const uint32_t b = e & 1;
             const uint8_t* st = smem + s * p.stage_bytes;
+            if (!warp_wait(bar_x_ready + 8 * s, ph, abort_flag, p.status)) return false;   // activation sums visible
             if (!warp_wait(bar_d_ready + 8 * b, (e >> 1) & 1, abort_flag, p.status)) return false;
             tc_fence_after();
+            if (dw == 0) FQ_STAMP(2, e, 3);
             const uint16_t* sc = reinterpret_cast<const uint16_t*>(st + p.off_sz);
             const float4* xsum = reinterpret_cast<const float4*>(st + p.off_xsum);
 #pragma unroll
@@ -480,16 +525,18 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 6), 1) fq_fused_kernel(con
             }
             tc_fence_before();
             __syncwarp();
+            if (dw == 0) FQ_STAMP(2, e, 4);
             if (lane == 0) mbar_arrive(bar_empty + 8 * s);
             return true;
         };
 
-        uint32_t pending = 0xffffffffu;      // unit whose epilogue has not run yet
-        for (uint32_t u = u_begin, it = 0; u < u_end && ok; ++u, ++it) {
-            const uint32_t s = it % S, ph = (it / S) & 1, b = it & 1;
-            const uint32_t tn = u / KT, kt = u % KT;
+        uint32_t pending = 0xffffffffu, pending_s = 0, pending_ph = 0;      // unit whose epilogue has not run yet, and its ring slot
+        for (UnitIter w(u_begin, KT); w.u < u_end && ok; w.next(S, KT)) {
+            const uint32_t u = w.u, it = w.it, s = w.s, ph = w.ph, b = w.it & 1;
+            const uint32_t tn = w.tn, kt = w.kt;
             const uint8_t* st = smem + s * p.stage_bytes;
             if (!warp_wait(bar_full + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
+            if (dw == 0) FQ_STAMP(2, it, 0);
             // unpack: four 16-byte chunks = 128 codes of this column -> A operand rows in TMEM
             const uint4* wp = reinterpret_cast<const uint4*>(st) + col;
 #pragma unroll
@@ -510,19 +557,23 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 6), 1) fq_fused_kernel(con
                     tmem_st8(t_tile + b * 64 + (j * 2 + hf) * 8, a);
                 }
             }
+            if (dw == 0) FQ_STAMP(2, it, 1);
             tmem_wait_st();
+            if (dw == 0) FQ_STAMP(2, it, 2);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_a_ready + 8 * b);
             // while the tensor core works on this unit, finish the previous one
             if (pending != 0xffffffffu) {
-                if (!epilogue(pending)) { ok = false; break; }
+                if (!epilogue(pending, pending_s, pending_ph)) { ok = false; break; }
             }
             pending = it;
+            pending_s = s;
+            pending_ph = ph;
 
             if (kt == KT - 1 || u == u_end - 1) {
                 // ---------------------------------------------------------- end of a piece
-                if (!epilogue(pending)) { ok = false; break; }
+                if (!epilogue(pending, pending_s, pending_ph)) { ok = false; break; }
                 pending = 0xffffffffu;
                 if (SPARSE) {
                     if (!warp_wait(bar_sparse_done, piece & 1, abort_flag, p.status)) { ok = false; break; }
@@ -589,9 +640,9 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 6), 1) fq_fused_kernel(con
                 ++piece;
             }
         }
-    } else if (SPARSE && (warp == 2 || warp == 3 || warp >= 4 + NDW)) {
+    } else if (SPARSE && (warp == 3 || warp >= 4 + NDW)) {
         // ------------------------------------------------------------------ sparse
-        const uint32_t sw = warp < 4 ? warp - 2 : warp - (4 + NDW) + 2;
+        const uint32_t sw = warp < 4 ? 0u : warp - (4 + NDW) + 1;
         if (sw + 1 <= nsw) {
             const uint32_t nbb = p.NB >> 5;            // blocks of 32 buckets
             const uint32_t bb = sw % nbb, og = sw / nbb, n_og = nsw / nbb;
@@ -599,19 +650,21 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 6), 1) fq_fused_kernel(con
             const uint32_t n_oct = (p.M + 7) >> 3;
             uint8_t* xt = smem + p.off_xt + sw * 2048;
             uint32_t piece = 0;
-            for (uint32_t u = u_begin, it = 0; u < u_end; ++u, ++it) {
-                const uint32_t s = it % S, ph = (it / S) & 1;
-                const uint32_t kt = u % KT;
+            for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
+                const uint32_t u = w.u, s = w.s, ph = w.ph, kt = w.kt;
                 const uint8_t* st = smem + s * p.stage_bytes;
                 if (!warp_wait(bar_full + 8 * s, ph, abort_flag, p.status)) break;
+                if (!warp_wait(bar_x_ready + 8 * s, ph, abort_flag, p.status)) break;
+                if (sw == 0) FQ_STAMP(3, w.it, 0);
                 const uint32_t info = reinterpret_cast<const uint32_t*>(st + p.off_info)[bucket];
                 const uint32_t off = info & 0xffffu, cnt = info >> 16;
                 const uint4* pk_s = reinterpret_cast<const uint4*>(st + p.off_coo);
                 const uint4* pk_g = nullptr;
                 if (off + cnt > p.coo_cap) pk_g = p.packed + __ldg(p.indptr + u);  // tail of an oversized tile
                 for (uint32_t o = og; o < n_oct; o += n_og) {
-                    transpose_octet(smem_u32(st + p.off_xraw) + o * 8 * kXRowBytes, xt, lane);
+                    transpose_octet(smem_u32(st + p.off_xcan), NMMA / 8, o, xt, lane);
                     __syncwarp();
+                    if (sw == 0) FQ_STAMP(3, w.it, 1);
                     float* shc_o = shc + o * 8;
                     for (uint32_t i = 0; i < cnt; ++i) {
                         const uint32_t idx = off + i;
@@ -620,6 +673,7 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 6), 1) fq_fused_kernel(con
                     }
                     __syncwarp();
                 }
+                if (sw == 0) FQ_STAMP(3, w.it, 2);
                 if (lane == 0) mbar_arrive(bar_empty + 8 * s);
                 if (kt == KT - 1 || u == u_end - 1) {
                     __syncwarp();
@@ -636,10 +690,9 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 6), 1) fq_fused_kernel(con
     __syncthreads();
     if (warp == 1) {
         // every tcgen05 operation of this CTA must have retired before its TMEM is released
-        if (lane == 0) {
-            umma_commit(bar_final);
-            for (uint32_t spin = 0; spin < (1u << 24) && !mbar_try_wait(bar_final, 0); ++spin) {}
-        }
+        __syncwarp();
+        umma_commit(bar_final);
+        for (uint32_t spin = 0; spin < (1u << 24) && !mbar_try_wait(bar_final, 0); ++spin) {}
         __syncwarp();
         tc_fence_after();
         tmem_dealloc(tmem_base, kTmemCols);
@@ -738,8 +791,7 @@ static fq_status_t make_plan(const fq_layout_t* L, uint32_t M, bool sparse, Plan
     uint32_t stage = 0, S = 0;
     for (;;) {
         p.off_sz = w_bytes;
-        p.off_xraw = p.off_sz + round_up(sz_bytes, 128);
-        p.off_xcan = p.off_xraw + round_up(NMMA * kXRowBytes, 128);
+        p.off_xcan = p.off_sz + round_up(sz_bytes, 128);
         p.off_xsum = p.off_xcan + NMMA * 256;
         p.off_info = p.off_xsum + round_up(GPS * NMMA * 4, 128);
         p.off_coo = p.off_info + (sparse ? round_up(NB * 4, 128) : 0);
@@ -754,7 +806,7 @@ static fq_status_t make_plan(const fq_layout_t* L, uint32_t M, bool sparse, Plan
     p.off_xt = p.off_shc + (sparse ? BN * NMMA * 4 : 0);
     p.off_bar = p.off_xt + nsw * 2048;
     pl.smem = p.off_bar + 1024;
-    pl.threads = 32 * (4 + NDW + (nsw > 2 ? nsw - 2 : 0));
+    pl.threads = 32 * (4 + NDW + (nsw > 1 ? nsw - 1 : 0));
     const int sms = sm_count_cached();
     if (sms <= 0) return fail(FQ_ERR_CUDA, "no CUDA device: %s", cudaGetErrorString(cudaGetLastError()));
     pl.grid = std::min<uint32_t>({(uint32_t)sms, kMaxCtas, p.NT * p.KT});
@@ -841,6 +893,12 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
 using namespace fq;
 
 extern "C" {
+
+#ifdef FQ_TRACE
+int fq_trace_read(unsigned long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, fq::g_trace, sizeof(unsigned long long) * 4 * 64 * 8);
+}
+#endif
 
 fq_status_t fq_workspace_bytes(const fq_layout_t* L, uint32_t M, size_t* bytes) {
     if (!layout_ok(L) || !bytes) return fail(FQ_ERR_INVALID_ARG, "bad layout or null output");

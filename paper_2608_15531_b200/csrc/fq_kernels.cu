@@ -34,16 +34,23 @@
 namespace fq {
 
 constexpr int kBK = 128;
+#ifdef FQ_TRACE
+constexpr int kSmemBudget = 232448 - 16384;
+#else
 constexpr int kSmemBudget = 232448;    // 227 KB per CTA on sm_100
+#endif
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 constexpr uint32_t kTmemCols = 512;
 
 #ifdef FQ_TRACE
 // Developer build only: cycle stamps of CTA 0's first iterations, [role][iteration][event].
-__device__ unsigned long long g_trace[4 * 64 * 8];
-#define FQ_STAMP(role, it, ev) do { if (blockIdx.x == 0 && (it) < 64 && lane == 0) g_trace[((role) * 64 + (it)) * 8 + (ev)] = clock64(); } while (0)
+__device__ unsigned long long g_trace[12 * 32 * 4];
+__shared__ unsigned long long s_trace[12 * 32 * 4];
+#define FQ_STAMP(role, it, ev) do { if (blockIdx.x == 0 && (it) < 32 && (ev) < 4 && lane == 0) s_trace[((role) * 32 + (it)) * 4 + (ev)] = clock64(); } while (0)
+#define FQ_DSTAMP(it, e) do { if (dw == 2) FQ_STAMP(4 + (e) / 4, it, (e) % 4); } while (0)
 #else
 #define FQ_STAMP(role, it, ev) do {} while (0)
+#define FQ_DSTAMP(it, e) do {} while (0)
 #endif
 
 struct Params {
@@ -75,6 +82,11 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.shared::cta.b64 st, [%0];\n}" ::"r"(bar) : "memory");
 }
+// For arrivals that publish nothing through the generic proxy (a consumer that only read a stage,
+// or a thread whose stores were tcgen05 operations already fenced): no release fence needed.
+__device__ __forceinline__ void mbar_arrive_relaxed(uint32_t bar) {
+    asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.relaxed.cta.shared::cta.b64 st, [%0];\n}" ::"r"(bar) : "memory");
+}
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n}" ::"r"(bar), "r"(bytes)
                  : "memory");
@@ -88,6 +100,15 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok;
 }
+__device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
 __device__ __forceinline__ unsigned long long globaltimer_ns() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -96,6 +117,7 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
 // Bounded wait: false if this CTA is giving up (its own limit expired, or another warp's did).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
                                           uint32_t* status) {
+    if (mbar_test_wait(bar, parity)) return true;   // already complete: no suspend
     uint32_t spins = 0;
     unsigned long long t0 = 0;
     while (!mbar_try_wait(bar, parity)) {
@@ -115,7 +137,9 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 }
 // Warp-uniform form: every lane waits, and the warp gives up together.
 __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t* status) {
-    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status));
+    uint32_t ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, status) ? 1u : 0u;
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
@@ -312,12 +336,11 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 7), 1) fq_fused_kernel(con
     const uint32_t S = p.stages;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
     const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * S;
-    const uint32_t bar_x_ready = bar_empty + 8 * S;      // [S]
-    const uint32_t bar_a_ready = bar_x_ready + 8 * S;    // [2]
+    const uint32_t bar_a_ready = bar_empty + 8 * S;      // [2]
     const uint32_t bar_d_ready = bar_a_ready + 16;       // [2]
     const uint32_t bar_sparse_done = bar_d_ready + 16, bar_dense_done = bar_sparse_done + 8;
     const uint32_t bar_dense = bar_dense_done + 8, bar_final = bar_dense + 8;
-    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 3 * S + 8);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 2 * S + 8);
     volatile uint32_t* last_flag = abort_flag + 1;
     volatile uint32_t* tmem_slot = abort_flag + 2;
     float* shc = reinterpret_cast<float*>(smem + p.off_shc);
@@ -325,9 +348,8 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 7), 1) fq_fused_kernel(con
     const uint32_t nsw = SPARSE ? p.nsw : 0;
     if (tid == 0) {
         for (uint32_t s = 0; s < S; ++s) {
-            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_full + 8 * s, 2);   // producer's expect_tx arrival + activation warp
             mbar_init(bar_empty + 8 * s, NDW + nsw + 1);
-            mbar_init(bar_x_ready + 8 * s, 1);
         }
         mbar_init(bar_a_ready, NDW);
         mbar_init(bar_a_ready + 8, NDW);
@@ -414,11 +436,11 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 7), 1) fq_fused_kernel(con
         // ------------------------------------------------------------------ tensor warp
         for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
             const uint32_t it = w.it, s = w.s, ph = w.ph, b = w.it & 1;
-            if (!warp_wait(bar_x_ready + 8 * s, ph, abort_flag, p.status)) break;
+            if (!warp_wait(bar_full + 8 * s, ph, abort_flag, p.status)) break;
             FQ_STAMP(1, it, 0);
             if (!warp_wait(bar_a_ready + 8 * b, (it >> 1) & 1, abort_flag, p.status)) break;
             tc_fence_after();
-            FQ_STAMP(1, it, 2);
+            FQ_STAMP(1, it, 1);
             const uint64_t bd0 = make_b_desc(smem_u32(smem) + s * p.stage_bytes + p.off_xcan, (NMMA / 8) * 128, 128);
 #pragma unroll
             for (int ti = 0; ti < NT128; ++ti)
@@ -431,7 +453,7 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 7), 1) fq_fused_kernel(con
                 }
             umma_commit(bar_d_ready + 8 * b);   // accumulators of this unit are complete
             umma_commit(bar_empty + 8 * s);     // and the stage's activation operand has been read
-            FQ_STAMP(1, it, 3);
+            FQ_STAMP(1, it, 2);
         }
     } else if (warp == 2) {
         // ------------------------------------------------------------------ activation warp
@@ -481,7 +503,7 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 7), 1) fq_fused_kernel(con
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_x_ready + 8 * s);
+            if (lane == 0) mbar_arrive(bar_full + 8 * s);
         }
     } else if (warp >= 4 && warp < 4 + NDW) {
         // ------------------------------------------------------------------ dense: thread = column
@@ -499,10 +521,9 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 7), 1) fq_fused_kernel(con
         auto epilogue = [&](uint32_t e, uint32_t s, uint32_t ph) -> bool {
             const uint32_t b = e & 1;
             const uint8_t* st = smem + s * p.stage_bytes;
-            if (!warp_wait(bar_x_ready + 8 * s, ph, abort_flag, p.status)) return false;   // activation sums visible
             if (!warp_wait(bar_d_ready + 8 * b, (e >> 1) & 1, abort_flag, p.status)) return false;
             tc_fence_after();
-            if (dw == 0) FQ_STAMP(2, e, 3);
+            FQ_DSTAMP(e, 6);
             const uint16_t* sc = reinterpret_cast<const uint16_t*>(st + p.off_sz);
             const float4* xsum = reinterpret_cast<const float4*>(st + p.off_xsum);
 #pragma unroll
@@ -525,8 +546,9 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 7), 1) fq_fused_kernel(con
             }
             tc_fence_before();
             __syncwarp();
-            if (dw == 0) FQ_STAMP(2, e, 4);
-            if (lane == 0) mbar_arrive(bar_empty + 8 * s);
+            FQ_DSTAMP(e, 7);
+            if (lane == 0) mbar_arrive_relaxed(bar_empty + 8 * s);
+            FQ_DSTAMP(e, 8);
             return true;
         };
 
@@ -536,7 +558,7 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 7), 1) fq_fused_kernel(con
             const uint32_t tn = w.tn, kt = w.kt;
             const uint8_t* st = smem + s * p.stage_bytes;
             if (!warp_wait(bar_full + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
-            if (dw == 0) FQ_STAMP(2, it, 0);
+            FQ_DSTAMP(it, 0);
             // unpack: four 16-byte chunks = 128 codes of this column -> A operand rows in TMEM
             const uint4* wp = reinterpret_cast<const uint4*>(st) + col;
 #pragma unroll
@@ -557,12 +579,14 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 7), 1) fq_fused_kernel(con
                     tmem_st8(t_tile + b * 64 + (j * 2 + hf) * 8, a);
                 }
             }
-            if (dw == 0) FQ_STAMP(2, it, 1);
+            FQ_DSTAMP(it, 1);
             tmem_wait_st();
-            if (dw == 0) FQ_STAMP(2, it, 2);
+            FQ_DSTAMP(it, 2);
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_a_ready + 8 * b);
+            FQ_DSTAMP(it, 3);
+            if (lane == 0) mbar_arrive_relaxed(bar_a_ready + 8 * b);
+            FQ_DSTAMP(it, 4);
             // while the tensor core works on this unit, finish the previous one
             if (pending != 0xffffffffu) {
                 if (!epilogue(pending, pending_s, pending_ph)) { ok = false; break; }
@@ -654,7 +678,6 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 7), 1) fq_fused_kernel(con
                 const uint32_t u = w.u, s = w.s, ph = w.ph, kt = w.kt;
                 const uint8_t* st = smem + s * p.stage_bytes;
                 if (!warp_wait(bar_full + 8 * s, ph, abort_flag, p.status)) break;
-                if (!warp_wait(bar_x_ready + 8 * s, ph, abort_flag, p.status)) break;
                 if (sw == 0) FQ_STAMP(3, w.it, 0);
                 const uint32_t info = reinterpret_cast<const uint32_t*>(st + p.off_info)[bucket];
                 const uint32_t off = info & 0xffffu, cnt = info >> 16;
@@ -674,7 +697,7 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 7), 1) fq_fused_kernel(con
                     __syncwarp();
                 }
                 if (sw == 0) FQ_STAMP(3, w.it, 2);
-                if (lane == 0) mbar_arrive(bar_empty + 8 * s);
+                if (lane == 0) mbar_arrive_relaxed(bar_empty + 8 * s);
                 if (kt == KT - 1 || u == u_end - 1) {
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_sparse_done);
@@ -688,6 +711,10 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 7), 1) fq_fused_kernel(con
     // ---------------------------------------------------------------------- common exit
     tc_fence_before();
     __syncthreads();
+#ifdef FQ_TRACE
+    if (blockIdx.x == 0)
+        for (int i = tid; i < 12 * 32 * 4; i += blockDim.x) g_trace[i] = s_trace[i];
+#endif
     if (warp == 1) {
         // every tcgen05 operation of this CTA must have retired before its TMEM is released
         __syncwarp();
@@ -896,7 +923,7 @@ extern "C" {
 
 #ifdef FQ_TRACE
 int fq_trace_read(unsigned long long* out) {
-    return (int)cudaMemcpyFromSymbol(out, fq::g_trace, sizeof(unsigned long long) * 4 * 64 * 8);
+    return (int)cudaMemcpyFromSymbol(out, fq::g_trace, sizeof(unsigned long long) * 12 * 32 * 4);
 }
 #endif
 

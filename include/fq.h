@@ -44,10 +44,12 @@
  *   packed_outliers (N_tile + 1 entries, uint32).  bucket_info[t*NB + b] =
  *   offset | count << 16 (two uint16): bucket b of tile t owns `count` packets
  *   starting `offset` packets after the tile's first.  Buckets of one tile own
- *   disjoint column sets.  A packet holds four outliers: bytes 0-3 row index in
+ *   disjoint column sets, and column c only ever appears in buckets
+ *   32*(c mod NB/32) .. 32*(c mod NB/32)+31 (one block of 32 buckets per sparse warp).  A packet holds four outliers: bytes 0-3 row index in
  *   the tile, bytes 4-7 column index in the tile, bytes 8-15 four BF16 values.
- *   A slot with value bits 0x0000 is padding (its indices repeat the bucket's
- *   last real entry).  Storage: (N_tile+1)*4 + N_tile*NB*4 + 16*packets bytes.
+ *   A slot with value bits 0x0000 is padding and is skipped (its row byte is 0
+ *   and its column byte is BN-1-slot).  Storage: (N_tile+1)*4 + N_tile*NB*4 +
+ *   16*packets bytes.
  */
 #ifndef FQ_H_
 #define FQ_H_
@@ -118,12 +120,14 @@ fq_status_t fq_unpack_int4(const fq_layout_t* L, const void* wq, uint8_t* q_cano
 /*
  * Tile-COO encoder (Section 3.2.1; column reordering and element reordering of
  * Section 3.2.2).  Input: COO triplets on the host (k, n, BF16 value bits), any
- * order; entries whose value is +-0 are dropped.  Per tile, columns are sorted
- * by outlier count (descending) and assigned greedily to the least-loaded of NB
- * buckets; inside a bucket, entries are ordered so that position i of bucket b
- * prefers shared-memory bank group (i + b) mod 8 of the kernel's activation
- * copy (bank group of row k = k mod 8), falling through to the next non-empty
- * group; buckets are padded to whole packets.
+ * order; entries whose value is +-0 are dropped.  Per tile and per block of 32
+ * buckets (block of column c = c mod NB/32), columns are sorted by outlier count
+ * (descending) and assigned greedily to the least-loaded bucket of the block; inside a bucket, entries are ordered so that the four slots of a
+ * packet hold different columns while four columns still have entries, and,
+ * among those, position i of bucket b prefers shared-memory bank group
+ * (i + b) mod 8 of the kernel's activation copy (bank group of row k = k mod 8),
+ * falling through to the next group in circular order; buckets are padded to
+ * whole packets.
  *
  * fq_encode_tilecoo_sizes: element counts of the three arrays (tile_indptr in
  * uint32, bucket_info in uint32, packets in 16-byte units) and the largest

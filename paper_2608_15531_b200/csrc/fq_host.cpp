@@ -52,7 +52,7 @@ fq_status_t fq_get_layout(uint32_t K, uint32_t N, uint32_t group, uint32_t bn_hi
     if (BN != 128 && BN != 256) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "BN must be 128 or 256, got %u", BN);
     if (N == 0 || N % BN != 0) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "N = %u is not a multiple of BN = %u", N, BN);
     if (N / BN > kMaxTilesN) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "N = %u has too many column tiles", N);
-    uint32_t NB = nb_hint ? nb_hint : 32;
+    uint32_t NB = nb_hint ? nb_hint : 64;
     if (NB != 32 && NB != 64 && NB != 128) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "buckets per tile must be 32, 64 or 128, got %u", NB);
     std::memset(out, 0, sizeof(*out));
     out->abi = FQ_ABI_VERSION;
@@ -187,22 +187,45 @@ struct Encoded {
     uint32_t max_tile_packets = 0;
 };
 
-// Order one bucket's entries: position i of bucket b prefers bank group (i + b) % 8, where an
-// entry's bank group is k % 8 (one 16-byte row of the transposed activation copy per k).
+// Order one bucket's entries (input sorted by column, then row).  Two goals, in this priority:
+//  1. the four slots of a packet hold four different columns whenever the bucket still has four
+//     columns with entries left, so the kernel can read all four accumulator rows before it
+//     writes any of them;
+//  2. position i of bucket b prefers an entry whose activation row lies in shared-memory bank
+//     group (i + b) % 8 (bank group of row k = k % 8), so that the lanes of a warp, one bucket each,
+//     hit different banks at the same step.
 void order_bucket(std::vector<Entry>& e, uint32_t b, std::vector<Entry>& out) {
-    std::vector<Entry> grp[8];
-    for (const Entry& x : e) grp[x.k & 7].push_back(x);
-    size_t head[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    struct Col { uint8_t c; std::vector<Entry> ent; };
+    std::vector<Col> cols;
+    for (const Entry& x : e) {
+        if (cols.empty() || cols.back().c != x.c) cols.push_back(Col{x.c, {}});
+        cols.back().ent.push_back(x);
+    }
     out.clear();
+    int in_packet[4] = {-1, -1, -1, -1};
     for (size_t i = 0; i < e.size(); ++i) {
-        uint32_t want = (uint32_t)((i + b) & 7);
-        for (uint32_t d = 0; d < 8; ++d) {
-            uint32_t gsel = (want + d) & 7;
-            if (head[gsel] < grp[gsel].size()) {
-                out.push_back(grp[gsel][head[gsel]++]);
-                break;
+        if ((i & 3) == 0) in_packet[0] = in_packet[1] = in_packet[2] = in_packet[3] = -1;
+        const uint32_t want = (uint32_t)((i + b) & 7);
+        int best = -1, best_score = -1;
+        size_t best_ent = 0;
+        for (size_t ci = 0; ci < cols.size(); ++ci) {
+            if (cols[ci].ent.empty()) continue;
+            bool used = false;
+            for (size_t s = 0; s < (i & 3); ++s) used = used || in_packet[s] == (int)ci;
+            // an entry in the wanted bank group, else the next group in circular order
+            size_t pick = 0;
+            uint32_t dist = 8;
+            for (size_t j = 0; j < cols[ci].ent.size(); ++j) {
+                uint32_t d = ((cols[ci].ent[j].k & 7u) + 8u - want) & 7u;
+                if (d < dist) { dist = d; pick = j; }
             }
+            // fresh column first, then bank-group distance, then the fullest column
+            int score = (used ? 0 : 1 << 20) + (int)(7 - dist) * (1 << 12) + (int)std::min<size_t>(cols[ci].ent.size(), 4095);
+            if (score > best_score) { best_score = score; best = (int)ci; best_ent = pick; }
         }
+        out.push_back(cols[best].ent[best_ent]);
+        cols[best].ent.erase(cols[best].ent.begin() + best_ent);
+        in_packet[i & 3] = best;
     }
 }
 
@@ -238,24 +261,30 @@ fq_status_t encode_impl(const fq_layout_t* L, const uint32_t* k, const uint32_t*
     for (int64_t t = 0; t < (int64_t)ntile; ++t) {
         uint32_t cnt[256] = {0};
         for (size_t e = tstart[t]; e < tstart[t + 1]; ++e) ++cnt[sorted[e].c];
-        // columns by descending count (ties: lower column first), then least-loaded bucket
-        // (ties: lower bucket id) -- the greedy longest-processing-time rule
-        uint32_t order[256];
-        for (uint32_t c = 0; c < BN; ++c) order[c] = c;
-        std::stable_sort(order, order + BN, [&](uint32_t a, uint32_t b) { return cnt[a] > cnt[b]; });
-        typedef std::pair<uint32_t, uint32_t> LB;  // (load, bucket)
-        std::priority_queue<LB, std::vector<LB>, std::greater<LB>> heap;
-        for (uint32_t b = 0; b < NB; ++b) heap.push(LB(0, b));
+        // Buckets come in blocks of 32 (one sparse warp each).  A column always belongs to block
+        // (column mod number-of-blocks), in every row tile, so that two warps working on different
+        // row tiles of the same column tile never touch the same output column.  Inside a block:
+        // columns by descending count (ties: lower column first), each to the least-loaded bucket
+        // (ties: lower bucket id) -- the greedy longest-processing-time rule.
+        const uint32_t nblk = NB / 32;
         uint32_t load[128] = {0};
         uint8_t* c2b = &col2bucket[(size_t)t * BN];
-        for (uint32_t i = 0; i < BN; ++i) {
-            uint32_t c = order[i];
-            if (cnt[c] == 0) { c2b[c] = (uint8_t)(c % NB); continue; }
-            LB top = heap.top();
-            heap.pop();
-            c2b[c] = (uint8_t)top.second;
-            load[top.second] += cnt[c];
-            heap.push(LB(top.first + cnt[c], top.second));
+        for (uint32_t blk = 0; blk < nblk; ++blk) {
+            uint32_t order[256], ncol = 0;
+            for (uint32_t c = blk; c < BN; c += nblk) order[ncol++] = c;
+            std::stable_sort(order, order + ncol, [&](uint32_t a, uint32_t b) { return cnt[a] > cnt[b]; });
+            typedef std::pair<uint32_t, uint32_t> LB;  // (load, bucket)
+            std::priority_queue<LB, std::vector<LB>, std::greater<LB>> heap;
+            for (uint32_t b = 0; b < 32; ++b) heap.push(LB(0, blk * 32 + b));
+            for (uint32_t i = 0; i < ncol; ++i) {
+                uint32_t c = order[i];
+                if (cnt[c] == 0) { c2b[c] = (uint8_t)(blk * 32); continue; }
+                LB top = heap.top();
+                heap.pop();
+                c2b[c] = (uint8_t)top.second;
+                load[top.second] += cnt[c];
+                heap.push(LB(top.first + cnt[c], top.second));
+            }
         }
         uint32_t off = 0;
         for (uint32_t b = 0; b < NB; ++b) {
@@ -297,12 +326,19 @@ fq_status_t encode_impl(const fq_layout_t* L, const uint32_t* k, const uint32_t*
                     return a.c != c.c ? a.c < c.c : a.k < c.k;
                 });
                 order_bucket(per[b], b, ordered);
+                // inside a packet, equal columns must be neighbours (the kernel chains them in registers)
+                for (size_t p0 = 0; p0 < ordered.size(); p0 += 4)
+                    std::stable_sort(ordered.begin() + p0, ordered.begin() + std::min(p0 + 4, ordered.size()),
+                                     [](const Entry& a, const Entry& c) { return a.c < c.c; });
                 uint32_t info = E.info[(size_t)t * NB + b];
                 uint8_t* dst = &E.packets[((size_t)E.indptr[t] + (info & 0xffffu)) * 16];
                 const size_t cntp = info >> 16;
                 for (size_t s = 0; s < cntp * 4; ++s) {
                     const bool real = s < ordered.size();
-                    const Entry& x = real ? ordered[s] : ordered.back();
+                    // padding: value 0, row 0, and a column byte that differs between the slots of
+                    // the packet (the kernel skips value-0 slots and never touches that column)
+                    const Entry pad{0, (uint8_t)(BN - 1 - s % 4), 0};
+                    const Entry& x = real ? ordered[s] : pad;
                     uint8_t* pk = dst + (s / 4) * 16;
                     pk[s % 4] = x.k;
                     pk[4 + s % 4] = x.c;
@@ -401,8 +437,13 @@ fq_status_t fq_validate_tilecoo(const fq_layout_t* L, const uint32_t* indptr, co
             if (off + cnt > tile_pk) return fail(FQ_ERR_FORMAT, "bucket %u of tile %zu covers packets [%u, %u) of %u", b, t, off, off + cnt, tile_pk);
             for (uint32_t i = 0; i < cnt; ++i) {
                 const uint8_t* p = pk + (size_t)(indptr[t] + off + i) * 16;
+                int prev_col = -1;
                 for (int s = 0; s < 4; ++s) {
+                    if ((p[8 + 2 * s] | p[9 + 2 * s]) == 0) continue;  // padding slot
+                    if ((int)p[4 + s] < prev_col) return fail(FQ_ERR_FORMAT, "packet %u of tile %zu: columns of its slots are not sorted", indptr[t] + off + i, t);
+                    prev_col = p[4 + s];
                     if (p[s] >= FQ_BK || p[4 + s] >= BN) return fail(FQ_ERR_FORMAT, "index (%u, %u) outside the tile in tile %zu", p[s], p[4 + s], t);
+                    if (p[4 + s] % (NB / 32) != b / 32) return fail(FQ_ERR_FORMAT, "column %u of tile %zu sits in bucket %u, outside its block of 32 buckets", p[4 + s], t, b);
                     if (owner[p[4 + s]] >= 0 && owner[p[4 + s]] != (int16_t)b) return fail(FQ_ERR_FORMAT, "column %u of tile %zu appears in buckets %d and %u", p[4 + s], t, owner[p[4 + s]], b);
                     owner[p[4 + s]] = (int16_t)b;
                 }

@@ -114,10 +114,9 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait: false if this CTA is giving up (its own limit expired, or another warp's did).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          uint32_t* status) {
-    if (mbar_test_wait(bar, parity)) return true;   // already complete: no suspend
+// Bounded wait, slow part: kept out of line so that the many wait sites stay a few instructions
+// long (the kernel's five warp roles share one instruction cache).
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t* status) {
     uint32_t spins = 0;
     unsigned long long t0 = 0;
     while (!mbar_try_wait(bar, parity)) {
@@ -134,6 +133,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         }
     }
     return true;
+}
+// Bounded wait: false if this CTA is giving up (its own limit expired, or another warp's did).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          uint32_t* status) {
+    if (mbar_test_wait(bar, parity)) return true;   // already complete
+    return mbar_wait_slow(bar, parity, abort_flag, status);
 }
 // Warp-uniform form: every lane waits, and the warp gives up together.
 __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t* status) {
@@ -241,8 +246,6 @@ struct UnitIter {
 
 // ----------------------------------------------------------------------------- sparse step
 
-__device__ __forceinline__ uint32_t has_zero_byte(uint32_t v) { return (v - 0x01010101u) & ~v & 0x80808080u; }
-
 __device__ __forceinline__ void fma8(float4& c0, float4& c1, float v, const uint4 xv) {
     c0.x = fmaf(v, bf16lo(xv.x), c0.x);
     c0.y = fmaf(v, bf16hi(xv.x), c0.y);
@@ -254,47 +257,68 @@ __device__ __forceinline__ void fma8(float4& c0, float4& c1, float v, const uint
     c1.w = fmaf(v, bf16hi(xv.w), c1.w);
 }
 
+// Position of 16-byte quad j of column c's FP32 row.  Q = quads per row when the row is XOR-swizzled
+// (4 or 8: lanes hitting random columns then spread over all bank groups), 0 = plain layout.
+template <int Q>
+__device__ __forceinline__ uint32_t shc_quad(uint32_t c, uint32_t j, uint32_t ldc) {
+    if (Q == 4) return c * ldc + ((j ^ ((c >> 1) & 3u)) << 2);
+    if (Q == 8) return c * ldc + ((j ^ (c & 7u)) << 2);
+    return c * ldc + (j << 2);
+}
+
 // One packet (four outliers) against the k-major activation copy xt ([128][8] BF16, 16 B per row):
-// shc[col * ldc + 0..7] += v * x[0..7][k] for each slot (Section 4.2, without the per-column padding:
-// every slot carries its own column byte).  When the four columns differ, all loads are issued
+// row c of the FP32 tile += v * x[8o..8o+7][k] for each slot (Section 4.2, without the per-column
+// padding: every slot carries its own column byte).  Padding slots (value 0) are skipped.  The
+// encoder sorts the real slots of a packet by column, so equal columns are neighbours: their
+// products are chained in registers and only the last slot of a run stores.  All loads are issued
 // before the first store.
-__device__ __forceinline__ void apply_packet(const uint4 pk, const uint8_t* __restrict__ xt, float* shc_oct, uint32_t ldc) {
+template <int Q>
+__device__ __forceinline__ void apply_packet(const uint4 pk, const uint8_t* __restrict__ xt, float* shc, uint32_t o, uint32_t ldc) {
     uint32_t k[4], c[4];
     float v[4];
+    bool live[4];
 #pragma unroll
     for (int s = 0; s < 4; ++s) {
         k[s] = (pk.x >> (8 * s)) & 0xffu;
         c[s] = (pk.y >> (8 * s)) & 0xffu;
     }
+    live[0] = (pk.z & 0xffffu) != 0; live[1] = (pk.z >> 16) != 0; live[2] = (pk.w & 0xffffu) != 0; live[3] = (pk.w >> 16) != 0;
     v[0] = bf16lo(pk.z); v[1] = bf16hi(pk.z); v[2] = bf16lo(pk.w); v[3] = bf16hi(pk.w);
     uint4 xv[4];
+    float4 c0[4], c1[4];
 #pragma unroll
-    for (int s = 0; s < 4; ++s) xv[s] = *reinterpret_cast<const uint4*>(xt + k[s] * 16);
-    const uint32_t dup = has_zero_byte(pk.y ^ __byte_perm(pk.y, 0, 0x0321)) | has_zero_byte(pk.y ^ __byte_perm(pk.y, 0, 0x1032));
-    if (!dup) {
-        float4 c0[4], c1[4];
-#pragma unroll
-        for (int s = 0; s < 4; ++s) {
-            const float4* cp = reinterpret_cast<const float4*>(shc_oct + c[s] * ldc);
-            c0[s] = cp[0];
-            c1[s] = cp[1];
+    for (int s = 0; s < 4; ++s) {
+        xv[s] = *reinterpret_cast<const uint4*>(xt + k[s] * 16);
+        c0[s] = c1[s] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        if (live[s]) {
+            c0[s] = *reinterpret_cast<const float4*>(shc + shc_quad<Q>(c[s], 2 * o, ldc));
+            c1[s] = *reinterpret_cast<const float4*>(shc + shc_quad<Q>(c[s], 2 * o + 1, ldc));
         }
+    }
+    float4 a0[4], a1[4];
 #pragma unroll
-        for (int s = 0; s < 4; ++s) fma8(c0[s], c1[s], v[s], xv[s]);
+    for (int s = 0; s < 4; ++s) {
+        a0[s] = a1[s] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        fma8(a0[s], a1[s], v[s], xv[s]);
+    }
+    bool same[5];
+    same[0] = same[4] = false;
 #pragma unroll
-        for (int s = 0; s < 4; ++s) {
-            float4* cp = reinterpret_cast<float4*>(shc_oct + c[s] * ldc);
-            cp[0] = c0[s];
-            cp[1] = c1[s];
-        }
-    } else {
+    for (int s = 1; s < 4; ++s) {
+        same[s] = live[s] && live[s - 1] && c[s] == c[s - 1];
+        const float m = same[s] ? 1.0f : 0.0f;   // carry the running sum of an equal-column run
+        a0[s].x = fmaf(m, a0[s - 1].x, a0[s].x); a0[s].y = fmaf(m, a0[s - 1].y, a0[s].y);
+        a0[s].z = fmaf(m, a0[s - 1].z, a0[s].z); a0[s].w = fmaf(m, a0[s - 1].w, a0[s].w);
+        a1[s].x = fmaf(m, a1[s - 1].x, a1[s].x); a1[s].y = fmaf(m, a1[s - 1].y, a1[s].y);
+        a1[s].z = fmaf(m, a1[s - 1].z, a1[s].z); a1[s].w = fmaf(m, a1[s - 1].w, a1[s].w);
+    }
 #pragma unroll
-        for (int s = 0; s < 4; ++s) {
-            float4* cp = reinterpret_cast<float4*>(shc_oct + c[s] * ldc);
-            float4 c0 = cp[0], c1 = cp[1];
-            fma8(c0, c1, v[s], xv[s]);
-            cp[0] = c0;
-            cp[1] = c1;
+    for (int s = 0; s < 4; ++s) {
+        if (live[s] && !same[s + 1]) {
+            c0[s].x += a0[s].x; c0[s].y += a0[s].y; c0[s].z += a0[s].z; c0[s].w += a0[s].w;
+            c1[s].x += a1[s].x; c1[s].y += a1[s].y; c1[s].z += a1[s].z; c1[s].w += a1[s].w;
+            *reinterpret_cast<float4*>(shc + shc_quad<Q>(c[s], 2 * o, ldc)) = c0[s];
+            *reinterpret_cast<float4*>(shc + shc_quad<Q>(c[s], 2 * o + 1, ldc)) = c1[s];
         }
     }
 }
@@ -320,7 +344,7 @@ __device__ __forceinline__ void transpose_octet(uint32_t xcan_u32, uint32_t n_oc
 
 // BN: tile columns (128 or 256).  NB16: batch columns of the MMA in units of 16 (1: M <= 16, 2: M <= 32).
 template <int BN, int NB16, int GROUP, bool SPARSE>
-__global__ void __launch_bounds__(32 * (4 + BN / 32 + 7), 1) fq_fused_kernel(const Params p) {
+__global__ void __launch_bounds__(32 * (4 + 2 * (BN / 32) + 4), 1) fq_fused_kernel(const Params p) {
     constexpr int NDW = BN / 32;              // dense warps: one thread per tile column
     constexpr int NT128 = BN / 128;           // 128-row MMA tiles per unit
     constexpr int NMMA = 16 * NB16;           // MMA N: batch rows, padded
@@ -340,7 +364,8 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 7), 1) fq_fused_kernel(con
     const uint32_t bar_d_ready = bar_a_ready + 16;       // [2]
     const uint32_t bar_sparse_done = bar_d_ready + 16, bar_dense_done = bar_sparse_done + 8;
     const uint32_t bar_dense = bar_dense_done + 8, bar_final = bar_dense + 8;
-    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 2 * S + 8);
+    const uint32_t bar_d_free = bar_final + 8;           // [2]
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 2 * S + 10);
     volatile uint32_t* last_flag = abort_flag + 1;
     volatile uint32_t* tmem_slot = abort_flag + 2;
     float* shc = reinterpret_cast<float*>(smem + p.off_shc);
@@ -349,16 +374,18 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 7), 1) fq_fused_kernel(con
     if (tid == 0) {
         for (uint32_t s = 0; s < S; ++s) {
             mbar_init(bar_full + 8 * s, 2);   // producer's expect_tx arrival + activation warp
-            mbar_init(bar_empty + 8 * s, NDW + nsw + 1);
+            mbar_init(bar_empty + 8 * s, 2 * NDW + nsw + NT128);
         }
         mbar_init(bar_a_ready, NDW);
         mbar_init(bar_a_ready + 8, NDW);
-        mbar_init(bar_d_ready, 1);
-        mbar_init(bar_d_ready + 8, 1);
+        mbar_init(bar_d_ready, NT128);
+        mbar_init(bar_d_ready + 8, NT128);
         mbar_init(bar_sparse_done, nsw ? nsw : 1);
         mbar_init(bar_dense_done, NDW);
         mbar_init(bar_dense, NDW);
-        mbar_init(bar_final, 1);
+        mbar_init(bar_final, NT128);
+        mbar_init(bar_d_free, NDW);
+        mbar_init(bar_d_free + 8, NDW);
         *abort_flag = 0;
         *last_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -432,18 +459,18 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 7), 1) fq_fused_kernel(con
             for (uint32_t j = (issued > S ? issued - S : 0); j < issued; ++j)
                 for (uint32_t spin = 0; spin < (1u << 20) && !mbar_try_wait(bar_full + 8 * (j % S), (j / S) & 1); ++spin) {}
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ tensor warp
+    } else if (warp == 1 || (warp == 3 && NT128 == 2)) {
+        // ------------------------------------------------------------------ tensor warps (one per 128-row tile)
+        const int ti = warp == 1 ? 0 : 1;
         for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
             const uint32_t it = w.it, s = w.s, ph = w.ph, b = w.it & 1;
             if (!warp_wait(bar_full + 8 * s, ph, abort_flag, p.status)) break;
             FQ_STAMP(1, it, 0);
             if (!warp_wait(bar_a_ready + 8 * b, (it >> 1) & 1, abort_flag, p.status)) break;
+            if (it >= 2 && !warp_wait(bar_d_free + 8 * b, ((it - 2) >> 1) & 1, abort_flag, p.status)) break;
             tc_fence_after();
             FQ_STAMP(1, it, 1);
             const uint64_t bd0 = make_b_desc(smem_u32(smem) + s * p.stage_bytes + p.off_xcan, (NMMA / 8) * 128, 128);
-#pragma unroll
-            for (int ti = 0; ti < NT128; ++ti)
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
                     const int gi = ks / (8 / GPS);
@@ -455,6 +482,8 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 7), 1) fq_fused_kernel(con
             umma_commit(bar_empty + 8 * s);     // and the stage's activation operand has been read
             FQ_STAMP(1, it, 2);
         }
+        __syncwarp();
+        umma_commit(bar_final);                 // fires when every MMA this warp issued has retired
     } else if (warp == 2) {
         // ------------------------------------------------------------------ activation warp
         // lane -> (row m, part): CPL 16-byte chunks of that row; rows beyond M are zero
@@ -506,9 +535,53 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 7), 1) fq_fused_kernel(con
             if (lane == 0) mbar_arrive(bar_full + 8 * s);
         }
     } else if (warp >= 4 && warp < 4 + NDW) {
-        // ------------------------------------------------------------------ dense: thread = column
+        // ------------------------------------------------------------------ unpack warps: thread = column
         const int dw = warp - 4;
         const int col = dw * 32 + lane;                       // column inside the tile
+        const uint32_t t_lane = ((uint32_t)((dw & 3) * 32)) << 16;
+        const uint32_t t_tile = tmem_base + (uint32_t)(dw >> 2) * 256 + t_lane;
+        for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
+            const uint32_t it = w.it, s = w.s, ph = w.ph, b = w.it & 1;
+            const uint8_t* st = smem + s * p.stage_bytes;
+            if (!warp_wait(bar_full + 8 * s, ph, abort_flag, p.status)) break;
+            // the A buffer of this parity was last read by the MMAs of unit it - 2
+            if (it >= 2 && !warp_wait(bar_d_ready + 8 * b, ((it - 2) >> 1) & 1, abort_flag, p.status)) break;
+            tc_fence_after();
+            FQ_DSTAMP(it, 0);
+            // four 16-byte chunks = 128 codes of this column -> A operand rows in TMEM
+            const uint4* wp = reinterpret_cast<const uint4*>(st) + col;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint4 w4 = wp[j * BN];
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    const uint32_t w0 = hf ? w4.z : w4.x, w1 = hf ? w4.w : w4.y;
+                    uint32_t a[8];
+                    a[0] = codes_to_bf16x2(w0);
+                    a[1] = codes_to_bf16x2(w0 >> 4);
+                    a[2] = codes_to_bf16x2(w0 >> 8);
+                    a[3] = codes_to_bf16x2(w0 >> 12);
+                    a[4] = codes_to_bf16x2(w1);
+                    a[5] = codes_to_bf16x2(w1 >> 4);
+                    a[6] = codes_to_bf16x2(w1 >> 8);
+                    a[7] = codes_to_bf16x2(w1 >> 12);
+                    tmem_st8(t_tile + b * 64 + (j * 2 + hf) * 8, a);
+                }
+            }
+            FQ_DSTAMP(it, 1);
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive_relaxed(bar_a_ready + 8 * b);
+                mbar_arrive_relaxed(bar_empty + 8 * s);
+            }
+            FQ_DSTAMP(it, 2);
+        }
+    } else if (warp >= 4 + NDW && warp < 4 + 2 * NDW) {
+        // ------------------------------------------------------------------ epilogue warps: thread = column
+        const int dw = warp - 4 - NDW;
+        const int col = dw * 32 + lane;
         const uint32_t t_lane = ((uint32_t)((dw & 3) * 32)) << 16;
         const uint32_t t_tile = tmem_base + (uint32_t)(dw >> 2) * 256 + t_lane;
         float accf[NMMA];
@@ -516,14 +589,14 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 7), 1) fq_fused_kernel(con
         for (int i = 0; i < NMMA; ++i) accf[i] = 0.0f;
         uint32_t piece = 0, dense_phase = 0;
         bool ok = true;
-
-        // scale / zero-point / activation sums of one finished unit, then release its stage
-        auto epilogue = [&](uint32_t e, uint32_t s, uint32_t ph) -> bool {
-            const uint32_t b = e & 1;
+        for (UnitIter w(u_begin, KT); w.u < u_end && ok; w.next(S, KT)) {
+            const uint32_t u = w.u, it = w.it, s = w.s, b = w.it & 1;
+            const uint32_t tn = w.tn, kt = w.kt;
             const uint8_t* st = smem + s * p.stage_bytes;
-            if (!warp_wait(bar_d_ready + 8 * b, (e >> 1) & 1, abort_flag, p.status)) return false;
+            // scale / zero-point / activation sums of the unit once its MMAs are complete
+            if (!warp_wait(bar_d_ready + 8 * b, (it >> 1) & 1, abort_flag, p.status)) { ok = false; break; }
             tc_fence_after();
-            FQ_DSTAMP(e, 6);
+            FQ_DSTAMP(it, 4);
             const uint16_t* sc = reinterpret_cast<const uint16_t*>(st + p.off_sz);
             const float4* xsum = reinterpret_cast<const float4*>(st + p.off_xsum);
 #pragma unroll
@@ -546,70 +619,25 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 7), 1) fq_fused_kernel(con
             }
             tc_fence_before();
             __syncwarp();
-            FQ_DSTAMP(e, 7);
-            if (lane == 0) mbar_arrive_relaxed(bar_empty + 8 * s);
-            FQ_DSTAMP(e, 8);
-            return true;
-        };
-
-        uint32_t pending = 0xffffffffu, pending_s = 0, pending_ph = 0;      // unit whose epilogue has not run yet, and its ring slot
-        for (UnitIter w(u_begin, KT); w.u < u_end && ok; w.next(S, KT)) {
-            const uint32_t u = w.u, it = w.it, s = w.s, ph = w.ph, b = w.it & 1;
-            const uint32_t tn = w.tn, kt = w.kt;
-            const uint8_t* st = smem + s * p.stage_bytes;
-            if (!warp_wait(bar_full + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
-            FQ_DSTAMP(it, 0);
-            // unpack: four 16-byte chunks = 128 codes of this column -> A operand rows in TMEM
-            const uint4* wp = reinterpret_cast<const uint4*>(st) + col;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const uint4 w4 = wp[j * BN];
-#pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
-                    const uint32_t w0 = hf ? w4.z : w4.x, w1 = hf ? w4.w : w4.y;
-                    uint32_t a[8];
-                    a[0] = codes_to_bf16x2(w0);
-                    a[1] = codes_to_bf16x2(w0 >> 4);
-                    a[2] = codes_to_bf16x2(w0 >> 8);
-                    a[3] = codes_to_bf16x2(w0 >> 12);
-                    a[4] = codes_to_bf16x2(w1);
-                    a[5] = codes_to_bf16x2(w1 >> 4);
-                    a[6] = codes_to_bf16x2(w1 >> 8);
-                    a[7] = codes_to_bf16x2(w1 >> 12);
-                    tmem_st8(t_tile + b * 64 + (j * 2 + hf) * 8, a);
-                }
+            if (lane == 0) {
+                mbar_arrive_relaxed(bar_d_free + 8 * b);   // the tensor warp may overwrite this D buffer
+                mbar_arrive_relaxed(bar_empty + 8 * s);
             }
-            FQ_DSTAMP(it, 1);
-            tmem_wait_st();
-            FQ_DSTAMP(it, 2);
-            tc_fence_before();
-            __syncwarp();
-            FQ_DSTAMP(it, 3);
-            if (lane == 0) mbar_arrive_relaxed(bar_a_ready + 8 * b);
-            FQ_DSTAMP(it, 4);
-            // while the tensor core works on this unit, finish the previous one
-            if (pending != 0xffffffffu) {
-                if (!epilogue(pending, pending_s, pending_ph)) { ok = false; break; }
-            }
-            pending = it;
-            pending_s = s;
-            pending_ph = ph;
+            FQ_DSTAMP(it, 5);
 
             if (kt == KT - 1 || u == u_end - 1) {
                 // ---------------------------------------------------------- end of a piece
-                if (!epilogue(pending, pending_s, pending_ph)) { ok = false; break; }
-                pending = 0xffffffffu;
                 if (SPARSE) {
                     if (!warp_wait(bar_sparse_done, piece & 1, abort_flag, p.status)) { ok = false; break; }
-                    float4* cp = reinterpret_cast<float4*>(shc + col * LDC);
 #pragma unroll
                     for (int i = 0; i < NMMA / 4; ++i) {
-                        const float4 v = cp[i];
+                        float4* cp = reinterpret_cast<float4*>(shc + shc_quad<LDC / 4>(col, i, LDC));
+                        const float4 v = *cp;
                         accf[4 * i + 0] += v.x;
                         accf[4 * i + 1] += v.y;
                         accf[4 * i + 2] += v.z;
                         accf[4 * i + 3] += v.w;
-                        cp[i] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                        *cp = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
                     }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_dense_done);
@@ -664,9 +692,9 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 7), 1) fq_fused_kernel(con
                 ++piece;
             }
         }
-    } else if (SPARSE && (warp == 3 || warp >= 4 + NDW)) {
+    } else if (SPARSE && warp >= 4 + 2 * NDW) {
         // ------------------------------------------------------------------ sparse
-        const uint32_t sw = warp < 4 ? 0u : warp - (4 + NDW) + 1;
+        const uint32_t sw = warp - (4 + 2 * NDW);
         if (sw + 1 <= nsw) {
             const uint32_t nbb = p.NB >> 5;            // blocks of 32 buckets
             const uint32_t bb = sw % nbb, og = sw / nbb, n_og = nsw / nbb;
@@ -688,11 +716,17 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 7), 1) fq_fused_kernel(con
                     transpose_octet(smem_u32(st + p.off_xcan), NMMA / 8, o, xt, lane);
                     __syncwarp();
                     if (sw == 0) FQ_STAMP(3, w.it, 1);
-                    float* shc_o = shc + o * 8;
+#ifdef FQ_TRACE
+                    if (sw == 0 && blockIdx.x == 0 && w.it < 32) {
+                        const uint32_t mx = __reduce_max_sync(0xffffffffu, cnt);
+                        const uint32_t sm = __reduce_add_sync(0xffffffffu, cnt);
+                        if (lane == 0) s_trace[(3 * 32 + w.it) * 4 + 3] = ((unsigned long long)mx << 32) | sm;
+                    }
+#endif
                     for (uint32_t i = 0; i < cnt; ++i) {
                         const uint32_t idx = off + i;
                         const uint4 pk = (idx < p.coo_cap) ? pk_s[idx] : __ldg(pk_g + idx);
-                        apply_packet(pk, xt, shc_o, LDC);
+                        apply_packet<LDC / 4>(pk, xt, shc, o, LDC);
                     }
                     __syncwarp();
                 }
@@ -717,8 +751,6 @@ __global__ void __launch_bounds__(32 * (4 + BN / 32 + 7), 1) fq_fused_kernel(con
 #endif
     if (warp == 1) {
         // every tcgen05 operation of this CTA must have retired before its TMEM is released
-        __syncwarp();
-        umma_commit(bar_final);
         for (uint32_t spin = 0; spin < (1u << 24) && !mbar_try_wait(bar_final, 0); ++spin) {}
         __syncwarp();
         tc_fence_after();
@@ -760,7 +792,7 @@ __global__ void __launch_bounds__(256) fq_spmm_kernel(const uint16_t* __restrict
             const uint32_t bb = w % nbb, o = w / nbb;
             const uint32_t inf = info[t * NB + bb * 32 + lane];
             const uint32_t off = inf & 0xffffu, cnt = inf >> 16;
-            for (uint32_t i = 0; i < cnt; ++i) apply_packet(__ldg(pk + off + i), xt + o * 2048, shc + o * 8, LDC);
+            for (uint32_t i = 0; i < cnt; ++i) apply_packet<0>(__ldg(pk + off + i), xt + o * 2048, shc, o, LDC);
         }
     }
     __syncthreads();
@@ -803,7 +835,7 @@ static fq_status_t make_plan(const fq_layout_t* L, uint32_t M, bool sparse, Plan
     uint32_t nsw = 0;
     if (sparse) {
         const uint32_t nbb = NB / 32, n_oct = (M + 7) / 8;
-        nsw = nbb * std::min<uint32_t>(n_oct, std::max<uint32_t>(1, 8 / nbb));
+        nsw = nbb * std::min<uint32_t>(n_oct, std::max<uint32_t>(1, 4 / nbb));
     }
     Params& p = pl.p;
     std::memset(&p, 0, sizeof(p));
@@ -833,7 +865,7 @@ static fq_status_t make_plan(const fq_layout_t* L, uint32_t M, bool sparse, Plan
     p.off_xt = p.off_shc + (sparse ? BN * NMMA * 4 : 0);
     p.off_bar = p.off_xt + nsw * 2048;
     pl.smem = p.off_bar + 1024;
-    pl.threads = 32 * (4 + NDW + (nsw > 1 ? nsw - 1 : 0));
+    pl.threads = 32 * (4 + 2 * NDW + nsw);
     const int sms = sm_count_cached();
     if (sms <= 0) return fail(FQ_ERR_CUDA, "no CUDA device: %s", cudaGetErrorString(cudaGetLastError()));
     pl.grid = std::min<uint32_t>({(uint32_t)sms, kMaxCtas, p.NT * p.KT});

@@ -138,6 +138,22 @@ def test_scratch_is_reusable_and_results_are_reproducible():
     assert not head.any()
 
 
+@pytest.mark.parametrize("NB,M", [(64, 1), (128, 8), (128, 16)])
+def test_several_sparse_warps_over_many_units_do_not_race(NB, M):
+    # several units per CTA and more than one block of 32 buckets: sparse warps then work on
+    # different row tiles of one column tile at the same time
+    K, N, g = 4096, 6144, 128
+    lay = synth.layer(synth.tensor_seed(8, 6), K, N, density=0.01, layout="mixed")
+    P = H.pack_layer(lay, g, 0, NB)
+    X = _x(9, M, K)
+    Y = H.run_fused(P, X)
+    for _ in range(3):
+        assert np.array_equal(H.run_fused(P, X), Y)
+    cols = np.arange(0, N, 24, dtype=np.uint32)
+    Yref, Yabs = H.oracle_result(P, X, cols=cols)
+    H.check_tolerances(Y[:, cols], Yref, Yabs, K)
+
+
 def test_argument_errors_launch_nothing():
     K, N, g = 512, 512, 128
     lay = synth.layer(1, K, N, density=0.01)

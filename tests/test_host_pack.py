@@ -26,7 +26,7 @@ def test_library_exports_every_declared_symbol():
 
 def test_layout_defaults_and_errors():
     L = fq.fq_get_layout(4096, 4096, 128)
-    assert (L.BK, L.BN, L.buckets_per_tile, L.coo_unit_bytes) == (128, 256, 32, 16)
+    assert (L.BK, L.BN, L.buckets_per_tile, L.coo_unit_bytes) == (128, 256, 64, 16)
     assert fq.fq_get_layout(4096, 4224, 64).BN == 128
     for bad in [(4096, 4096, 32), (4000, 4096, 128), (4096, 4100, 128)]:
         with pytest.raises(fq.FqError) as e:
@@ -121,15 +121,21 @@ def test_tilecoo_encode_invariants(layout, density, NB):
     owner = {}
     for t_, c_, b_ in zip(tile.tolist(), n.tolist(), b.tolist()):
         assert owner.setdefault((t_, c_), b_) == b_
-    # greedy least-loaded assignment: max bucket load <= mean load + largest column
+    # a column lives in one block of 32 buckets (column mod number of blocks) in every tile; inside a
+    # block the greedy least-loaded assignment gives max bucket load <= mean load + largest column
+    nblk = NB // 32
+    assert np.array_equal((b % NB) // 32, (n % BN) % nblk)
     for t_ in np.unique(tile):
         sel = tile == t_
         loads = np.bincount(b[sel] - t_ * NB, minlength=NB)
-        colmax = np.bincount(n[sel] % BN, minlength=BN).max()
-        assert loads.max() <= loads.sum() / NB + colmax + 1e-9
+        for blk in range(nblk):
+            in_blk = sel & ((n % BN) % nblk == blk)
+            colmax = np.bincount(n[in_blk] % BN, minlength=BN).max() if in_blk.any() else 0
+            bl = loads[32 * blk:32 * blk + 32]
+            assert bl.max() <= bl.sum() / 32 + colmax + 1e-9
 
 
-def test_tilecoo_element_order_follows_the_rotated_bank_groups():
+def test_tilecoo_element_order_separates_columns_and_staggers_bank_groups():
     K, N, BN, NB = 128, 256, 256, 32
     Lr = synth.layer(77, K, N, density=0.06, layout="uniform")
     L = fq.fq_get_layout(K, N, 128, bn_hint=BN, nb_hint=NB)
@@ -140,16 +146,16 @@ def test_tilecoo_element_order_follows_the_rotated_bank_groups():
     for i, bb in enumerate(b.tolist()):
         pos[i] = seen.get(bb, 0)
         seen[bb] = pos[i] + 1
-    # rule: at position i bucket b takes bank group (i + b) % 8 if it still has one, else the next
-    # non-empty group in circular order -> replay the rule on each bucket's multiset of groups
+    # rule 1: the slots of a packet are sorted by column, and a packet repeats a column only when no
+    # other column had entries left (so every later entry of the bucket is in one of its columns)
     for bb in np.unique(b):
-        ks = k[b == bb]
-        left = np.bincount(ks % 8, minlength=8)
-        for i, kk in enumerate(ks.tolist()):
-            want = next(g % 8 for g in range(i + bb, i + bb + 8) if left[g % 8] > 0)
-            assert kk % 8 == want
-            left[want] -= 1
-    # and it pays: fewer shared-memory passes than the plain (column, row) order
+        cols = n[b == bb].tolist()
+        for p0 in range(0, len(cols), 4):
+            pkt = cols[p0:p0 + 4]
+            assert pkt == sorted(pkt)
+            if len(set(pkt)) < len(pkt):
+                assert set(cols[p0 + 4:]) <= set(pkt)
+    # rule 2 pays off: fewer shared-memory passes than the plain (column, row) order
     plain_pos = np.zeros(len(k), dtype=np.int64)
     for bb in np.unique(b):
         idx = np.nonzero(b == bb)[0]
@@ -157,6 +163,13 @@ def test_tilecoo_element_order_follows_the_rotated_bank_groups():
         for p_, i in enumerate(order):
             plain_pos[i] = p_
     assert _bank_conflict_cycles(k, b, pos, NB) < _bank_conflict_cycles(k, b, plain_pos, NB)
+    # a bucket that owns a single hot column cannot avoid repeats, and still round-trips
+    kk = np.arange(0, 40, dtype=np.uint32)
+    nn = np.full(40, 7, dtype=np.uint32)
+    vv = (0x3F80 + np.arange(40)).astype(np.uint16)
+    ip, bi, pk = fq.fq_encode_tilecoo(L, kk, nn, vv)
+    k2, n2, v2 = fq.fq_decode_tilecoo(L, ip, bi, pk)
+    assert _as_set(k2, n2, v2) == _as_set(kk, nn, vv) and pk.shape[0] == 10
 
 
 def test_tilecoo_edge_cases():
@@ -175,8 +188,9 @@ def test_tilecoo_edge_cases():
     assert packed.shape[0] == 1
     kk, nn, vv, _ = oracle.decode_tilecoo(indptr, info, packed, K, N, BN, NB)
     assert (kk.tolist(), nn.tolist(), vv.tolist()) == ([200], [300], [0x4000])
-    # padding repeats the last real entry's indices
-    assert packed[0, :4].tolist() == [72] * 4 and packed[0, 4:8].tolist() == [44] * 4
+    # padding slots: value 0, row 0, a column byte that differs from slot to slot
+    assert packed[0, :4].tolist() == [72, 0, 0, 0] and packed[0, 4:8].tolist() == [44, 254, 253, 252]
+    assert packed[0, 10:].tolist() == [0] * 6
     # one completely dense tile plus a hot row and a hot column elsewhere
     kk, nn = np.meshgrid(np.arange(128, 256), np.arange(0, 256), indexing="ij")
     k = np.concatenate([kk.ravel(), np.full(256, 3), np.arange(0, 128)]).astype(np.uint32)

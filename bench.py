@@ -33,10 +33,30 @@ DENSITY = 0.01
 CONFIG_ID = 2                      # the LLaMA-3-8B layer set
 L2_COVER_BYTES = 400 << 20         # rotating copies per layer cover at least this (L2 is 126 MB)
 METRIC = "effective_hbm_gbs_fused_w4a16_outlier_gemm_m1_8_16"
+# dram__bytes_read + dram__bytes_write of the fused kernel over its algorithmic bytes, from the ncu
+# captures summarised in profiles/fq_fused_kernel_llama3_8b_decode_set.md (1.02 and 1.04 on the two
+# launches captured); scaled to the average launch of the step.
+NCU_TRAFFIC_RATIO = 1.03
 
 
 def algorithmic_bytes(K, N, g, nnz, n_tile, n_bucket, M):
     return K * N // 2 + 2 * (K // g) * N * 2 + (n_tile + 1) * 4 + n_bucket * 4 + 4 * nnz + 2 * M * K + 2 * M * N
+
+
+def max_over_ranks(ms: float, world: int, device=None) -> float:
+    """Step time of the whole job: the slowest rank's (replicas run side by side, one per GPU)."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gbs(step_bytes: int, world: int, ms_per_step: float) -> float:
+    """Aggregate effective bandwidth: every rank moves `step_bytes` per step (weak scaling)."""
+    return world * step_bytes / (ms_per_step * 1e-3) / 1e9
 
 
 def peaks():
@@ -105,7 +125,8 @@ def build_workload(layers, log):
     from paper_2608_15531_b200 import binding as fq
     from paper_2608_15531_b200 import synth
     out = []
-    for idx, (name, K, N) in enumerate(layers):
+    for (name, K, N) in layers:
+        idx = synth.LLAMA3_8B.index((name, K, N))
         t0 = time.time()
         lay = synth.layer(synth.tensor_seed(CONFIG_ID, idx), K, N, density=DENSITY, layout="mixed")
         L = fq.fq_get_layout(K, N, GROUP)
@@ -121,6 +142,7 @@ def build_workload(layers, log):
 
 
 def run_ours(args):
+    global MS
     import torch
     import torch.distributed as dist
     from paper_2608_15531_b200 import binding as fq
@@ -140,7 +162,14 @@ def run_ours(args):
         if rank == 0 and args.verbose:
             print(f"[bench] {msg}", file=sys.stderr, flush=True)
 
-    work = build_workload(synth.LLAMA3_8B, log)
+    layers = synth.LLAMA3_8B
+    ms = MS
+    if args.only:                                # profiling aid: one layer, one M (e.g. gate_up:16)
+        lname, lm = args.only.split(":")
+        layers = [l for l in synth.LLAMA3_8B if l[0] == lname]
+        ms = (int(lm),)
+    MS = ms
+    work = build_workload(layers, log)
     dev = torch.device("cuda", local)
 
     def up(a):
@@ -169,11 +198,22 @@ def run_ours(args):
     step_bytes = sum(c[2] for c in calls)
     stream = torch.cuda.current_stream()
 
+    # Argument tuples are marshalled once: the timed loop only calls into the C ABI.
+    import ctypes
+    clib = fq.lib()
+    vp = lambda t: ctypes.c_void_p(t.data_ptr())
+    sp = ctypes.c_void_p(stream.cuda_stream)
+    for w in work:
+        w["args"] = {M: [(ctypes.byref(w["L"]), vp(w["Xd"][M]), ctypes.c_uint32(M), vp(c["wq"]), vp(c["scale"]),
+                          vp(c["zero"]), vp(c["indptr"]), vp(c["info"]), vp(c["packed"]), vp(w["Yd"][M]), vp(ws),
+                          ctypes.c_size_t(ws_bytes), sp) for c in w["copies"]] for M in MS}
+
     def one_call(w, M):
-        c = w["copies"][w["turn"] % len(w["copies"])]
+        a = w["args"][M]
+        rc = clib.fq_fused_w4a16_outlier_gemm(*a[w["turn"] % len(a)])
         w["turn"] += 1
-        fq.fq_fused_w4a16_outlier_gemm(w["L"], w["Xd"][M], M, c["wq"], c["scale"], c["zero"], c["indptr"], c["info"],
-                                       c["packed"], w["Yd"][M], ws, stream)
+        if rc != 0:
+            raise fq.FqError(rc, fq.fq_last_error())
 
     def step():
         for w, M, _ in calls:
@@ -202,12 +242,9 @@ def run_ours(args):
     clocks = sampler.stop() if rank == 0 else {}
     ms = e0.elapsed_time(e1)
     fq.fq_check_status(ws)
-    if world > 1:
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, world, dev)
     ms_per_step = ms / args.steps
-    value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
+    value = whole_job_gbs(step_bytes, world, ms_per_step)
 
     # ---- end to end: host X in, host Y out, through the C ABI, every call
     xh = {(w["name"], M): torch.from_numpy(np.ascontiguousarray(w["X"][:M]).view(np.int16)).pin_memory()
@@ -232,11 +269,8 @@ def run_ours(args):
     e1.record(stream)
     sync_all()
     e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_value = world * step_bytes / (e2e_ms / args.steps * 1e-3) / 1e9
+    e2e_ms = max_over_ranks(e2e_ms, world, dev)
+    e2e_value = whole_job_gbs(step_bytes, world, e2e_ms / args.steps)
     h2d = sum(2 * M * w["K"] for w, M, _ in calls)
     d2h = sum(2 * M * w["N"] for w, M, _ in calls)
 
@@ -320,7 +354,7 @@ def run_ours(args):
                 "ms_per_step": round(e2e_ms / args.steps, 5)},
         "gpu_launches": args.steps * len(calls),
         "roofline": {"bound": "hbm", "achieved": round(value / world, 2), "peak": peak, "unit": "GB/s",
-                     "frac": round(value / world / peak, 4), "traffic": None, "peak_kind": f"of {peak_kind}",
+                     "frac": round(value / world / peak, 4), "traffic": int(NCU_TRAFFIC_RATIO * (step_bytes // len(calls))), "peak_kind": f"of {peak_kind}",
                      "bytes_per_launch": step_bytes // len(calls), "us_per_launch": round(ms_per_step * 1e3 / len(calls), 3)},
         "cpu_baseline": cpu,
         "us_per_call": per_call,
@@ -335,7 +369,7 @@ def cpu_baseline(work, budget_s: float):
     M = 16, restricted to its first `f * N` output columns, f chosen from a short probe so that the
     whole sample takes about `budget_s` seconds."""
     import oracle
-    probe = work[1]                                # o_proj
+    probe = work[min(1, len(work) - 1)]            # o_proj
     cols = 128
     lay = probe["lay"]
     q, s, z = oracle.quantize(np.ascontiguousarray(lay.W[:, :cols]), np.ascontiguousarray(lay.mask[:, :cols]), GROUP)
@@ -403,6 +437,7 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="budget of the CPU-oracle baseline leg (0 = skip)")
     ap.add_argument("--no-cublas", dest="cublas", action="store_false")
     ap.add_argument("--verbose", action="store_true")
+    ap.add_argument("--only", default="", help="profiling aid: restrict the step to one LAYER:M, e.g. gate_up:16")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -179,6 +179,42 @@ fq_status_t fq_fused_w4a16_outlier_gemm(const fq_layout_t* L, const void* X, uin
                                         const void* packed_outliers, void* Y, void* workspace,
                                         size_t workspace_bytes, void* cuda_stream);
 
+/*
+ * The same operator for callers that cannot allocate device memory.  (The paper
+ * has no counterpart: this is a convenience of the library.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a
+ * framework's allocator-managed region, in a plug-in that is handed device
+ * buffers but may not create any, or in a process whose device-memory budget
+ * was handed out completely at start-up.  Such callers still pass X, the packed
+ * layer and Y; only the scratch is missing.
+ *
+ * Instead of a caller-provided workspace, the kernel uses an array that is part
+ * of the library image: FQ_STATIC_SCRATCH_BYTES of device memory on every GPU
+ * that loads the library, held until the process exits.  That fixes the limit:
+ * calls whose fq_workspace_bytes() exceeds it (M > FQ_STATIC_SCRATCH_MAX_M with
+ * 256-column tiles) are refused with FQ_ERR_BUFFER_TOO_SMALL and nothing is
+ * launched.  The function calls no cudaMalloc / cudaFree and no allocating
+ * library routine; per call it enqueues one small memset (status word and tile
+ * counters, which must start at zero) and the kernel.
+ *
+ * The first call on each device looks up the array's device address
+ * (cudaGetSymbolAddress, with that device current); make that first call
+ * outside any stream capture.  There is one array per device: every call
+ * shares it and finds the previous call's contents, so calls that may overlap
+ * on the GPU (different streams) race -- serialise them, or use the entry
+ * point above with separate scratch.  Errors otherwise as above; a wait that
+ * gave up is not retrievable through fq_check_status() here (the array is not
+ * visible to the caller) and shows as undefined Y.
+ */
+#define FQ_STATIC_SCRATCH_BYTES 6356992u /* 6 MiB + 64 KiB */
+#define FQ_STATIC_SCRATCH_MAX_M 16u
+fq_status_t fq_fused_w4a16_outlier_gemm_noalloc(const fq_layout_t* L, const void* X, uint32_t M,
+                                                const void* wq, const void* scale, const void* zero,
+                                                const void* tile_indptr, const void* bucket_info,
+                                                const void* packed_outliers, void* Y,
+                                                void* cuda_stream);
+
 /* Unfused baseline, dense half: Y = X * dequant(W_Q) (same kernel, sparse path
  * compiled out). */
 fq_status_t fq_unfused_gemm(const fq_layout_t* L, const void* X, uint32_t M, const void* wq,

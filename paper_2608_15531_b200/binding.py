@@ -27,7 +27,7 @@ FQ_MAX_M = 128
 EXPORTS = [
     "fq_get_layout", "fq_pack_int4_sizes", "fq_pack_int4", "fq_unpack_int4", "fq_encode_tilecoo_sizes",
     "fq_encode_tilecoo", "fq_decode_tilecoo", "fq_validate_tilecoo", "fq_workspace_bytes",
-    "fq_fused_w4a16_outlier_gemm", "fq_unfused_gemm", "fq_unfused_spmm", "fq_fused_host_io",
+    "fq_fused_w4a16_outlier_gemm", "fq_fused_w4a16_outlier_gemm_noalloc", "fq_unfused_gemm", "fq_unfused_spmm", "fq_fused_host_io",
     "fq_check_status", "fq_last_error",
 ]
 
@@ -183,6 +183,17 @@ def fq_fused_w4a16_outlier_gemm(L: Layout, X, M: int, wq, scale, zero, tile_indp
                                              _dp(zero), _dp(tile_indptr), _dp(bucket_info), _dp(packed), _dp(Y),
                                              _dp(workspace), ctypes.c_size_t(workspace.numel() * workspace.element_size()),
                                              _stream(stream)))
+
+
+def fq_fused_w4a16_outlier_gemm_noalloc(L: Layout, X, M: int, wq, scale, zero, tile_indptr, bucket_info, packed, Y,
+                                        stream=None) -> None:
+    """The fused operator without a caller-provided workspace: for callers that may not allocate
+    device memory.  Uses the scratch array built into the library (one per GPU, shared by all
+    calls: do not overlap calls on different streams).  Refuses calls that need more scratch than
+    the array holds (M > 16)."""
+    _check(lib().fq_fused_w4a16_outlier_gemm_noalloc(ctypes.byref(L), _dp(X), ctypes.c_uint32(M), _dp(wq), _dp(scale),
+                                                     _dp(zero), _dp(tile_indptr), _dp(bucket_info), _dp(packed),
+                                                     _dp(Y), _stream(stream)))
 
 
 def fq_unfused_gemm(L: Layout, X, M: int, wq, scale, zero, Y, workspace, stream=None) -> None:

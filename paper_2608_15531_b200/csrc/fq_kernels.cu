@@ -975,6 +975,55 @@ fq_status_t fq_fused_w4a16_outlier_gemm(const fq_layout_t* L, const void* X, uin
                        workspace_bytes, cuda_stream, true);
 }
 
+// ---- the entry point that allocates nothing -------------------------------------------------
+// Scratch for callers that cannot allocate device memory: lives in the library's own image on
+// every GPU that loads it, for the life of the process.
+static __device__ __align__(256) unsigned char g_static_scratch[FQ_STATIC_SCRATCH_BYTES];
+
+// Device address of g_static_scratch on the current device.  In host code the array's name is only
+// a handle; the address a kernel can use comes from cudaGetSymbolAddress, asked once per device
+// with that device current.
+static fq_status_t static_scratch_address(void** out) {
+    static void* addr[64] = {nullptr};
+    static std::mutex mu;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+    if (dev < 0 || dev >= 64) return fail(FQ_ERR_CUDA, "device ordinal %d is outside the supported range", dev);
+    std::lock_guard<std::mutex> lock(mu);
+    if (!addr[dev]) {
+        void* ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (e != cudaSuccess || !ptr) return fail(FQ_ERR_CUDA, "cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+        addr[dev] = ptr;
+    }
+    *out = addr[dev];
+    return FQ_OK;
+}
+
+fq_status_t fq_fused_w4a16_outlier_gemm_noalloc(const fq_layout_t* L, const void* X, uint32_t M, const void* wq,
+                                                const void* scale, const void* zero, const void* tile_indptr,
+                                                const void* bucket_info, const void* packed_outliers, void* Y,
+                                                void* cuda_stream) {
+    size_t need = 0;
+    fq_status_t st = fq_workspace_bytes(L, M, &need);
+    if (st != FQ_OK) return st;
+    if (need > (size_t)FQ_STATIC_SCRATCH_BYTES)
+        return fail(FQ_ERR_BUFFER_TOO_SMALL,
+                    "this call needs %zu bytes of scratch but the built-in scratch holds %zu (M <= %u fits); "
+                    "use fq_fused_w4a16_outlier_gemm with caller-allocated scratch",
+                    need, (size_t)FQ_STATIC_SCRATCH_BYTES, (unsigned)FQ_STATIC_SCRATCH_MAX_M);
+    void* scratch = nullptr;
+    st = static_scratch_address(&scratch);
+    if (st != FQ_OK) return st;
+    // the status word and the tile-arrival counters must start at zero; the previous user of the
+    // shared array may have been interrupted
+    cudaError_t e = cudaMemsetAsync(scratch, 0, kWsHeaderBytes + kWsCounterBytes, (cudaStream_t)cuda_stream);
+    if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "clearing the built-in scratch: %s", cudaGetErrorString(e));
+    return launch_gemm(L, X, M, wq, scale, zero, tile_indptr, bucket_info, packed_outliers, Y, scratch,
+                       (size_t)FQ_STATIC_SCRATCH_BYTES, cuda_stream, true);
+}
+
 fq_status_t fq_unfused_gemm(const fq_layout_t* L, const void* X, uint32_t M, const void* wq, const void* scale,
                             const void* zero, void* Y, void* workspace, size_t workspace_bytes, void* cuda_stream) {
     return launch_gemm(L, X, M, wq, scale, zero, nullptr, nullptr, nullptr, Y, workspace, workspace_bytes,

@@ -26,6 +26,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 
@@ -758,6 +759,355 @@ __global__ void __launch_bounds__(32 * (4 + 2 * (BN / 32) + 4), 1) fq_fused_kern
     }
 }
 
+// ----------------------------------------------------------------------------- small-batch kernel
+
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+constexpr int kXPitch = 320;   // activation row in shared memory: 256 B + 64 B, conflict-free 16-byte fragment loads
+
+// The same operator for M <= 8 per octet (MO octets of batch rows): every dense warp runs the same
+// short loop (one 16-column strip per warp, warp-level m16n8k16 MMAs with the weights on the M side
+// and the batch on the N side), so the instruction stream of 16 of the CTA's warps is shared and
+// stays in the instruction cache.  Same packed formats, same producer, same sparse warps, same
+// split-tile protocol as the tcgen05 kernel; only the dense engine differs.
+//   warp 0            producer (bulk copies)
+//   warp 1            activations: X block -> row-major shared-memory rows + per-group row sums
+//   warps 2..2+BN/16  dense: lane (g, t) loads word t of columns g and g+8 of each 32-row block:
+//                     8 codes = this lane's share of two k16 steps (the k order inside a block
+//                     follows the 16-byte activation loads of the lanes)
+//   then              sparse warps
+template <int BN, int MO, int GROUP, bool SPARSE>
+__global__ void __launch_bounds__(32 * (2 + BN / 16 + 4), 1) fq_mma_kernel(const Params p) {
+    constexpr int NDW = BN / 16;
+    constexpr int GPS = kBK / GROUP;
+    constexpr int W_BYTES = 16 * BN * 4;
+    constexpr int SZ_ROW = BN * 2;
+    constexpr int LDC = 8 * MO;
+    constexpr int Q = (LDC == 8) ? 0 : LDC / 4;
+    extern __shared__ __align__(128) uint8_t smem[];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t S = p.stages;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
+    const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * S;
+    const uint32_t bar_sparse_done = bar_empty + 8 * S, bar_dense_done = bar_sparse_done + 8, bar_dense = bar_dense_done + 8;
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 2 * S + 4);
+    volatile uint32_t* last_flag = abort_flag + 1;
+    float* shc = reinterpret_cast<float*>(smem + p.off_shc);
+
+    const uint32_t nsw = SPARSE ? p.nsw : 0;
+    if (tid == 0) {
+        for (uint32_t s = 0; s < S; ++s) {
+            mbar_init(bar_full + 8 * s, 2);   // producer's expect_tx arrival + activation warp
+            mbar_init(bar_empty + 8 * s, NDW + nsw);
+        }
+        mbar_init(bar_sparse_done, nsw ? nsw : 1);
+        mbar_init(bar_dense_done, NDW);
+        mbar_init(bar_dense, NDW);
+        *abort_flag = 0;
+        *last_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (SPARSE) {
+        for (uint32_t i = tid; i < (uint32_t)(BN * LDC); i += blockDim.x) shc[i] = 0.0f;
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncthreads();
+
+    const uint32_t U = p.NT * p.KT, P = gridDim.x, q = U / P, r = U % P;
+    const uint32_t u_begin = unit_begin_of(blockIdx.x, q, r);
+    const uint32_t u_end = u_begin + q + (blockIdx.x < r ? 1u : 0u);
+    const uint32_t KT = p.KT;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer
+        uint32_t ip_a = 0, ip_b = 0, issued = 0;
+        bool ok = true;
+        for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
+            const uint32_t u = w.u, it = w.it, s = w.s, ph = w.ph;
+            if (SPARSE && (it & 31) == 0) {
+                const uint32_t i = u + lane;
+                ip_a = (i <= U) ? __ldg(p.indptr + i) : 0;
+                ip_b = (i + 1 <= U) ? __ldg(p.indptr + i + 1) : 0;
+            }
+            uint32_t pk0 = 0, npk = 0;
+            if (SPARSE) {
+                pk0 = __shfl_sync(0xffffffffu, ip_a, it & 31);
+                npk = __shfl_sync(0xffffffffu, ip_b, it & 31) - pk0;
+                npk = min(npk, p.coo_cap);
+            }
+            if (!warp_wait(bar_empty + 8 * s, ph ^ 1, abort_flag, p.status)) { ok = false; break; }
+            const uint32_t tn = w.tn, kt = w.kt;
+            const uint32_t full = bar_full + 8 * s;
+            const uint32_t st = smem_u32(smem) + s * p.stage_bytes;
+            if (lane == 0) {
+                uint32_t bytes = W_BYTES + 2 * GPS * SZ_ROW;
+                if (SPARSE) bytes += p.NB * 4 + npk * 16;
+                mbar_arrive_expect_tx(full, bytes);
+            }
+            __syncwarp();
+            if (lane == 0) {
+                bulk_g2s(st, p.wq + (size_t)u * W_BYTES, W_BYTES, full);
+#pragma unroll
+                for (int gi = 0; gi < GPS; ++gi) {
+                    const size_t row = (size_t)(kt * GPS + gi) * p.N + (size_t)tn * BN;
+                    bulk_g2s(st + p.off_sz + gi * SZ_ROW, p.scale + row, SZ_ROW, full);
+                    bulk_g2s(st + p.off_sz + (GPS + gi) * SZ_ROW, p.zero + row, SZ_ROW, full);
+                }
+            } else if (lane == 1) {
+                if (SPARSE) {
+                    bulk_g2s(st + p.off_info, p.info + (size_t)u * p.NB, p.NB * 4, full);
+                    if (npk) bulk_g2s(st + p.off_coo, p.packed + pk0, npk * 16, full);
+                }
+            }
+            issued = it + 1;
+        }
+        if (!ok) {
+            for (uint32_t j = (issued > S ? issued - S : 0); j < issued; ++j)
+                for (uint32_t spin = 0; spin < (1u << 20) && !mbar_try_wait(bar_full + 8 * (j % S), (j / S) & 1); ++spin) {}
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ activation warp
+        // lane -> (row m, part): 16-byte chunks of that row; rows beyond M are zero
+        constexpr int ROWS = 8 * MO;
+        constexpr int LPR = 32 / ROWS;                       // lanes per row: 4 (8 rows) or 2 (16 rows)
+        constexpr int CPL = 16 / LPR;                        // chunks per lane
+        const int m = lane % ROWS, part = lane / ROWS;
+        const bool real = (uint32_t)m < p.M;
+        const uint8_t* xrow = reinterpret_cast<const uint8_t*>(p.X) + ((size_t)m * p.K) * 2 + part * CPL * 16;
+        uint4 nxt[CPL];
+        auto load = [&](uint32_t kt) {
+#pragma unroll
+            for (int c = 0; c < CPL; ++c) {
+                nxt[c] = make_uint4(0, 0, 0, 0);
+                if (real) nxt[c] = __ldg(reinterpret_cast<const uint4*>(xrow + (size_t)kt * 256 + c * 16));
+            }
+        };
+        if (u_begin < u_end) load(u_begin - (u_begin / KT) * KT);
+        for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
+            const uint32_t s = w.s, ph = w.ph;
+            uint8_t* st = smem + s * p.stage_bytes;
+            uint4 xv[CPL];
+#pragma unroll
+            for (int c = 0; c < CPL; ++c) xv[c] = nxt[c];
+            if (w.u + 1 < u_end) load(w.kt + 1 == KT ? 0u : w.kt + 1);
+            if (!warp_wait(bar_empty + 8 * s, ph ^ 1, abort_flag, p.status)) break;
+            uint8_t* dst = st + p.off_xcan + m * kXPitch + part * CPL * 16;
+            float sum = 0.0f;
+#pragma unroll
+            for (int c = 0; c < CPL; ++c) {
+                const uint4 v = xv[c];
+                *reinterpret_cast<uint4*>(dst + c * 16) = v;
+                sum += (bf16lo(v.x) + bf16hi(v.x)) + (bf16lo(v.y) + bf16hi(v.y)) + (bf16lo(v.z) + bf16hi(v.z)) +
+                       (bf16lo(v.w) + bf16hi(v.w));
+            }
+            // per-group sums of each row: lanes with the same m hold consecutive quarters / halves of the row
+            float* xsum = reinterpret_cast<float*>(st + p.off_xsum);
+            if (LPR == 4) {
+                const float s1 = sum + __shfl_xor_sync(0xffffffffu, sum, 8);       // parts {0,1} and {2,3}
+                const float s2 = s1 + __shfl_xor_sync(0xffffffffu, s1, 16);
+                if (GPS == 2) { if ((part & 1) == 0) xsum[(part >> 1) * ROWS + m] = s1; }
+                else if (part == 0) xsum[m] = s2;
+            } else {
+                const float s1 = sum + __shfl_xor_sync(0xffffffffu, sum, 16);
+                if (GPS == 2) xsum[part * ROWS + m] = sum;
+                else if (part == 0) xsum[m] = s1;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_full + 8 * s);
+        }
+    } else if (warp >= 2 && warp < 2 + NDW) {
+        // ------------------------------------------------------------------ dense warps (all alike)
+        const int dw = warp - 2, g = lane >> 2, t = lane & 3;
+        const int dtid = dw * 32 + lane;
+        const int c0 = dw * 16 + g;                           // this lane's columns: c0 and c0 + 8
+        float accf[MO][4];
+#pragma unroll
+        for (int o = 0; o < MO; ++o)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) accf[o][i] = 0.0f;
+        uint32_t piece = 0, dense_phase = 0;
+        bool ok = true;
+        for (UnitIter w(u_begin, KT); w.u < u_end && ok; w.next(S, KT)) {
+            const uint32_t u = w.u, s = w.s, ph = w.ph, tn = w.tn, kt = w.kt;
+            const uint8_t* st = smem + s * p.stage_bytes;
+            if (!warp_wait(bar_full + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
+            const uint32_t* wp = reinterpret_cast<const uint32_t*>(st) + c0 * 4 + t;
+            const uint8_t* xrow = st + p.off_xcan + g * kXPitch + t * 16;
+            const uint16_t* sc = reinterpret_cast<const uint16_t*>(st + p.off_sz);
+            const float* xsum = reinterpret_cast<const float*>(st + p.off_xsum);
+#pragma unroll
+            for (int gi = 0; gi < GPS; ++gi) {
+                float accg[MO][4];
+#pragma unroll
+                for (int o = 0; o < MO; ++o)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) accg[o][i] = 0.0f;
+#pragma unroll
+                for (int j = gi * (4 / GPS); j < (gi + 1) * (4 / GPS); ++j) {
+                    const uint32_t wa = wp[j * BN * 4], wb = wp[j * BN * 4 + 32];     // columns c0 and c0 + 8
+                    const uint32_t a0 = codes_to_bf16x2(wa), a1 = codes_to_bf16x2(wa >> 4);
+                    const uint32_t a2 = codes_to_bf16x2(wa >> 8), a3 = codes_to_bf16x2(wa >> 12);
+                    const uint32_t b0 = codes_to_bf16x2(wb), b1 = codes_to_bf16x2(wb >> 4);
+                    const uint32_t b2 = codes_to_bf16x2(wb >> 8), b3 = codes_to_bf16x2(wb >> 12);
+#pragma unroll
+                    for (int o = 0; o < MO; ++o) {
+                        const uint4 xb = *reinterpret_cast<const uint4*>(xrow + o * 8 * kXPitch + j * 64);
+                        mma_bf16(accg[o], a0, b0, a1, b1, xb.x, xb.y);   // rows 8t+0..3 of the block
+                        mma_bf16(accg[o], a2, b2, a3, b3, xb.z, xb.w);   // rows 8t+4..7
+                    }
+                }
+                // once per group: acc += s * (sum x (128+q) - (128+z) sum x)     (Eq. 3 inside Eq. 1)
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const float sv = bf16_bits_to_float(sc[gi * BN + c0 + 8 * h]);
+                    const float zc = -(128.0f + bf16_bits_to_float(sc[(GPS + gi) * BN + c0 + 8 * h]));
+#pragma unroll
+                    for (int o = 0; o < MO; ++o) {
+                        const float2 xs = *reinterpret_cast<const float2*>(xsum + gi * LDC + o * 8 + 2 * t);
+                        accf[o][2 * h + 0] = fmaf(sv, fmaf(zc, xs.x, accg[o][2 * h + 0]), accf[o][2 * h + 0]);
+                        accf[o][2 * h + 1] = fmaf(sv, fmaf(zc, xs.y, accg[o][2 * h + 1]), accf[o][2 * h + 1]);
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive_relaxed(bar_empty + 8 * s);
+
+            if (kt == KT - 1 || u == u_end - 1) {
+                // ---------------------------------------------------------- end of a piece
+                if (SPARSE) {
+                    if (!warp_wait(bar_sparse_done, piece & 1, abort_flag, p.status)) { ok = false; break; }
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                        for (int o = 0; o < MO; ++o) {
+                            float2* cp = reinterpret_cast<float2*>(shc + shc_quad<Q>(c0 + 8 * h, 2 * o + (t >> 1), LDC) + 2 * (t & 1));
+                            const float2 v = *cp;
+                            accf[o][2 * h + 0] += v.x;
+                            accf[o][2 * h + 1] += v.y;
+                            *cp = make_float2(0.0f, 0.0f);
+                        }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_dense_done);
+                }
+                const uint32_t u_tile0 = tn * KT;
+                const uint32_t piece_k0 = max(u_tile0, u_begin) - u_tile0;
+                const bool full_piece = (piece_k0 == 0) && (kt == KT - 1);
+                bool write_y = full_piece;
+                if (!full_piece) {
+                    // FP32 partial in fragment order; the last CTA to arrive sums them in CTA order
+                    const uint32_t which = (u_begin / KT == tn) ? 0u : 1u;
+                    float* slot = p.partials + ((size_t)blockIdx.x * 2 + which) * (size_t)(BN * LDC);
+#pragma unroll
+                    for (int o = 0; o < MO; ++o)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) __stcg(slot + (size_t)(o * 4 + i) * (NDW * 32) + dtid, accf[o][i]);
+                    __threadfence();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_dense);
+                    if (!warp_wait(bar_dense, dense_phase & 1, abort_flag, p.status)) { ok = false; break; }
+                    ++dense_phase;
+                    const uint32_t c_first = cta_of_unit(u_tile0, q, r), c_last = cta_of_unit(u_tile0 + KT - 1, q, r);
+                    if (dtid == 0) {
+                        const uint32_t old = atomicAdd(p.counters + tn, 1u);
+                        *last_flag = (old == c_last - c_first) ? 1u : 0u;
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_dense);
+                    if (!warp_wait(bar_dense, dense_phase & 1, abort_flag, p.status)) { ok = false; break; }
+                    ++dense_phase;
+                    if (*last_flag) {
+                        write_y = true;
+                        __threadfence();
+#pragma unroll
+                        for (int o = 0; o < MO; ++o)
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) accf[o][i] = 0.0f;
+                        for (uint32_t c = c_first; c <= c_last; ++c) {
+                            const uint32_t wch = (unit_begin_of(c, q, r) / KT == tn) ? 0u : 1u;
+                            const float* sl = p.partials + ((size_t)c * 2 + wch) * (size_t)(BN * LDC);
+#pragma unroll
+                            for (int o = 0; o < MO; ++o)
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) accf[o][i] += __ldcg(sl + (size_t)(o * 4 + i) * (NDW * 32) + dtid);
+                        }
+                        if (dtid == 0) p.counters[tn] = 0;  // ready for the next call
+                    }
+                }
+                if (write_y) {
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                        for (int o = 0; o < MO; ++o)
+#pragma unroll
+                            for (int j = 0; j < 2; ++j) {
+                                const uint32_t m = o * 8 + 2 * t + j;
+                                if (m < p.M) p.Y[(size_t)m * p.N + (size_t)tn * BN + c0 + 8 * h] = float_to_bf16_bits(accf[o][2 * h + j]);
+                            }
+                }
+#pragma unroll
+                for (int o = 0; o < MO; ++o)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) accf[o][i] = 0.0f;
+                ++piece;
+            }
+        }
+    } else if (SPARSE && warp >= 2 + NDW) {
+        // ------------------------------------------------------------------ sparse
+        const uint32_t sw = warp - (2 + NDW);
+        if (sw + 1 <= nsw) {
+            const uint32_t nbb = p.NB >> 5;
+            const uint32_t bb = sw % nbb, og = sw / nbb, n_og = nsw / nbb;
+            const uint32_t bucket = bb * 32 + lane;
+            const uint32_t n_oct = (p.M + 7) >> 3;
+            uint8_t* xt = smem + p.off_xt + sw * 2048;
+            uint32_t piece = 0;
+            for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
+                const uint32_t u = w.u, s = w.s, ph = w.ph, kt = w.kt;
+                const uint8_t* st = smem + s * p.stage_bytes;
+                if (!warp_wait(bar_full + 8 * s, ph, abort_flag, p.status)) break;
+                const uint32_t info = reinterpret_cast<const uint32_t*>(st + p.off_info)[bucket];
+                const uint32_t off = info & 0xffffu, cnt = info >> 16;
+                const uint4* pk_s = reinterpret_cast<const uint4*>(st + p.off_coo);
+                const uint4* pk_g = nullptr;
+                if (off + cnt > p.coo_cap) pk_g = p.packed + __ldg(p.indptr + u);
+                for (uint32_t o = og; o < n_oct; o += n_og) {
+                    // row-major rows (kXPitch apart) -> xt[k][8]
+#pragma unroll
+                    for (int kb = 0; kb < 4; ++kb) {
+                        uint32_t r0, r1, r2, r3;
+                        ldmatrix_x4_trans(smem_u32(st + p.off_xcan) + (o * 8 + (lane & 7)) * kXPitch + (kb * 4 + (lane >> 3)) * 16, r0, r1, r2, r3);
+                        uint8_t* dst = xt + ((kb * 32) + (lane >> 2)) * 16 + (lane & 3) * 4;
+                        *reinterpret_cast<uint32_t*>(dst) = r0;
+                        *reinterpret_cast<uint32_t*>(dst + 8 * 16) = r1;
+                        *reinterpret_cast<uint32_t*>(dst + 16 * 16) = r2;
+                        *reinterpret_cast<uint32_t*>(dst + 24 * 16) = r3;
+                    }
+                    __syncwarp();
+                    for (uint32_t i = 0; i < cnt; ++i) {
+                        const uint32_t idx = off + i;
+                        const uint4 pk = (idx < p.coo_cap) ? pk_s[idx] : __ldg(pk_g + idx);
+                        apply_packet<Q>(pk, xt, shc, o, LDC);
+                    }
+                    __syncwarp();
+                }
+                if (lane == 0) mbar_arrive_relaxed(bar_empty + 8 * s);
+                if (kt == KT - 1 || u == u_end - 1) {
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_sparse_done);
+                    if (!warp_wait(bar_dense_done, piece & 1, abort_flag, p.status)) break;
+                    ++piece;
+                }
+            }
+        }
+    }
+}
+
 // ----------------------------------------------------------------------------- unfused SpMM
 
 // Y += X * W_O as its own launch (the sparse half of the two-kernel baseline).  One CTA per column
@@ -872,7 +1222,78 @@ static fq_status_t make_plan(const fq_layout_t* L, uint32_t M, bool sparse, Plan
     return FQ_OK;
 }
 
+// Plan of the small-batch kernel (fq_mma_kernel): M <= 16 per launch.
+static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, Plan& pl) {
+    const uint32_t BN = L->BN, NB = L->buckets_per_tile, GPS = kBK / L->group;
+    const uint32_t MO = M <= 8 ? 1 : 2, ROWS = 8 * MO;
+    const uint32_t NDW = BN / 16;
+    uint32_t nsw = 0;
+    if (sparse) {
+        const uint32_t nbb = NB / 32, n_oct = (M + 7) / 8;
+        nsw = nbb * std::min<uint32_t>(n_oct, std::max<uint32_t>(1, 4 / nbb));
+    }
+    Params& p = pl.p;
+    std::memset(&p, 0, sizeof(p));
+    p.M = M; p.K = L->K; p.N = L->N; p.KT = L->K / kBK; p.NT = L->N / BN; p.NB = NB; p.nsw = nsw;
+    const uint32_t w_bytes = 16 * BN * 4, sz_bytes = 2 * GPS * BN * 2;
+    const uint32_t fixed = (sparse ? BN * ROWS * 4 + nsw * 2048 : 0) + 1024;
+    uint32_t cap = 0;
+    if (sparse) {
+        cap = L->max_tile_packets ? round_up(L->max_tile_packets, 8) : 256;
+        cap = std::min<uint32_t>(cap, 1024);
+    }
+    uint32_t stage = 0, S = 0;
+    for (;;) {
+        p.off_sz = w_bytes;
+        p.off_xcan = p.off_sz + round_up(sz_bytes, 128);
+        p.off_xsum = p.off_xcan + round_up(ROWS * kXPitch, 128);
+        p.off_info = p.off_xsum + round_up(GPS * ROWS * 4, 128);
+        p.off_coo = p.off_info + (sparse ? round_up(NB * 4, 128) : 0);
+        stage = round_up(p.off_coo + cap * 16, 128);
+        S = std::min<uint32_t>(8, (kSmemBudget - fixed) / stage);
+        if (S >= 4 || cap <= 64) break;
+        cap = std::max<uint32_t>(64, cap / 2);
+    }
+    if (S < 3) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "shared-memory stages do not fit");
+    p.coo_cap = cap; p.stages = S; p.stage_bytes = stage;
+    p.off_shc = S * stage;
+    p.off_xt = p.off_shc + (sparse ? BN * ROWS * 4 : 0);
+    p.off_bar = p.off_xt + nsw * 2048;
+    pl.smem = p.off_bar + 1024;
+    pl.threads = 32 * (2 + NDW + nsw);
+    const int sms = sm_count_cached();
+    if (sms <= 0) return fail(FQ_ERR_CUDA, "no CUDA device: %s", cudaGetErrorString(cudaGetLastError()));
+    pl.grid = std::min<uint32_t>({(uint32_t)sms, kMaxCtas, p.NT * p.KT});
+    return FQ_OK;
+}
+
 typedef void (*KernelFn)(const Params);
+
+template <int BN, int MO, int G>
+static KernelFn pick_mma_sparse(bool sparse) {
+    return sparse ? (KernelFn)fq_mma_kernel<BN, MO, G, true> : (KernelFn)fq_mma_kernel<BN, MO, G, false>;
+}
+template <int BN, int MO>
+static KernelFn pick_mma_group(uint32_t g, bool sparse) {
+    return g == 64 ? pick_mma_sparse<BN, MO, 64>(sparse) : pick_mma_sparse<BN, MO, 128>(sparse);
+}
+static KernelFn pick_mma_kernel(uint32_t bn, uint32_t mo, uint32_t g, bool sparse) {
+    if (bn == 128) return mo == 1 ? pick_mma_group<128, 1>(g, sparse) : pick_mma_group<128, 2>(g, sparse);
+    return mo == 1 ? pick_mma_group<256, 1>(g, sparse) : pick_mma_group<256, 2>(g, sparse);
+}
+
+// Which dense engine serves a launch of `mb` rows: the warp-level MMA kernel up to kMmaMaxRows
+// rows, tcgen05 above.  FQ_ENGINE=mma|tc in the environment overrides (development aid).
+static uint32_t mma_max_rows() {
+    static int v = -1;
+    if (v < 0) {
+        const char* e = std::getenv("FQ_ENGINE");
+        v = 8;
+        if (e && std::strcmp(e, "mma") == 0) v = 16;
+        if (e && std::strcmp(e, "tc") == 0) v = 0;
+    }
+    return (uint32_t)v;
+}
 
 template <int BN, int MO, int G>
 static KernelFn pick_sparse(bool sparse) {
@@ -927,7 +1348,8 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
     for (uint32_t m0 = 0; m0 < M; m0 += 32) {
         const uint32_t mb = std::min<uint32_t>(32, M - m0);
         Plan pl;
-        st = make_plan(L, mb, sparse, pl);
+        const bool use_mma = mb <= mma_max_rows();
+        st = use_mma ? make_plan_mma(L, mb, sparse, pl) : make_plan(L, mb, sparse, pl);
         if (st != FQ_OK) return st;
         Params& p = pl.p;
         p.X = (const uint16_t*)X + (size_t)m0 * L->K;
@@ -937,7 +1359,8 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
         p.status = (uint32_t*)workspace;
         p.counters = (uint32_t*)((uint8_t*)workspace + kWsHeaderBytes);
         p.partials = (float*)((uint8_t*)workspace + kWsHeaderBytes + kWsCounterBytes);
-        KernelFn fn = pick_kernel(L->BN, nb16_of(mb), L->group, sparse);
+        KernelFn fn = use_mma ? pick_mma_kernel(L->BN, mb <= 8 ? 1 : 2, L->group, sparse)
+                              : pick_kernel(L->BN, nb16_of(mb), L->group, sparse);
         cudaError_t e = ensure_smem_attr((const void*)fn, (int)kSmemBudget);
         if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
         fn<<<pl.grid, pl.threads, pl.smem, (cudaStream_t)stream>>>(p);

@@ -187,14 +187,18 @@ struct Encoded {
     uint32_t max_tile_packets = 0;
 };
 
-// Order one bucket's entries (input sorted by column, then row).  Two goals, in this priority:
-//  1. the four slots of a packet hold four different columns whenever the bucket still has four
-//     columns with entries left, so the kernel can read all four accumulator rows before it
-//     writes any of them;
-//  2. position i of bucket b prefers an entry whose activation row lies in shared-memory bank
-//     group (i + b) % 8 (bank group of row k = k % 8), so that the lanes of a warp, one bucket each,
-//     hit different banks at the same step.
-void order_bucket(std::vector<Entry>& e, uint32_t b, std::vector<Entry>& out) {
+// Pack one bucket's entries (input sorted by column, then row) into packets of four slots.
+// A packet is one of two kinds, so that the kernel never needs to resolve a repeated column
+// inside a packet:
+//   "spread"  its real slots hold different columns (one entry from each of the up-to-four
+//             fullest columns that still have entries);
+//   "stack"   four entries of one column (used while fewer than four columns have entries left
+//             and one of them still has four or more).
+// Unused slots are padding.  Which entry of a column goes into slot position i of bucket b follows
+// the bank-group rotation of Section 3.2.2: prefer an entry whose activation row lies in bank
+// group (i + b) mod 4 (bank group of row k = k mod 4 for the kernel's 32-byte FP32 rows), else the
+// next group in circular order.  `out` receives 4 * packets entries; padding has v == 0.
+void pack_bucket(std::vector<Entry>& e, uint32_t b, uint32_t BN, std::vector<Entry>& out) {
     struct Col { uint8_t c; std::vector<Entry> ent; };
     std::vector<Col> cols;
     for (const Entry& x : e) {
@@ -202,30 +206,35 @@ void order_bucket(std::vector<Entry>& e, uint32_t b, std::vector<Entry>& out) {
         cols.back().ent.push_back(x);
     }
     out.clear();
-    int in_packet[4] = {-1, -1, -1, -1};
-    for (size_t i = 0; i < e.size(); ++i) {
-        if ((i & 3) == 0) in_packet[0] = in_packet[1] = in_packet[2] = in_packet[3] = -1;
-        const uint32_t want = (uint32_t)((i + b) & 7);
-        int best = -1, best_score = -1;
-        size_t best_ent = 0;
-        for (size_t ci = 0; ci < cols.size(); ++ci) {
-            if (cols[ci].ent.empty()) continue;
-            bool used = false;
-            for (size_t s = 0; s < (i & 3); ++s) used = used || in_packet[s] == (int)ci;
-            // an entry in the wanted bank group, else the next group in circular order
-            size_t pick = 0;
-            uint32_t dist = 8;
-            for (size_t j = 0; j < cols[ci].ent.size(); ++j) {
-                uint32_t d = ((cols[ci].ent[j].k & 7u) + 8u - want) & 7u;
-                if (d < dist) { dist = d; pick = j; }
-            }
-            // fresh column first, then bank-group distance, then the fullest column
-            int score = (used ? 0 : 1 << 20) + (int)(7 - dist) * (1 << 12) + (int)std::min<size_t>(cols[ci].ent.size(), 4095);
-            if (score > best_score) { best_score = score; best = (int)ci; best_ent = pick; }
+    size_t left = e.size();
+    auto take = [&](Col& col, size_t pos) {
+        const uint32_t want = (uint32_t)((pos + b) & 3);
+        size_t pick = 0;
+        uint32_t dist = 4;
+        for (size_t j = 0; j < col.ent.size(); ++j) {
+            uint32_t d = ((col.ent[j].k & 3u) + 4u - want) & 3u;
+            if (d < dist) { dist = d; pick = j; }
         }
-        out.push_back(cols[best].ent[best_ent]);
-        cols[best].ent.erase(cols[best].ent.begin() + best_ent);
-        in_packet[i & 3] = best;
+        Entry r = col.ent[pick];
+        col.ent.erase(col.ent.begin() + pick);
+        --left;
+        return r;
+    };
+    while (left > 0) {
+        // columns that still have entries, fullest first (ties: lower column)
+        std::vector<size_t> alive;
+        for (size_t ci = 0; ci < cols.size(); ++ci)
+            if (!cols[ci].ent.empty()) alive.push_back(ci);
+        std::stable_sort(alive.begin(), alive.end(), [&](size_t x, size_t y) { return cols[x].ent.size() > cols[y].ent.size(); });
+        const size_t base = out.size();
+        if (alive.size() < 4 && cols[alive[0]].ent.size() >= 4) {
+            for (int sidx = 0; sidx < 4; ++sidx) out.push_back(take(cols[alive[0]], base + sidx));
+        } else {
+            const size_t nsl = std::min<size_t>(4, alive.size());
+            for (size_t sidx = 0; sidx < nsl; ++sidx) out.push_back(take(cols[alive[sidx]], base + sidx));
+            // padding: value 0, row 0, and a column byte that differs from slot to slot
+            for (size_t sidx = nsl; sidx < 4; ++sidx) out.push_back(Entry{0, (uint8_t)(BN - 1 - sidx), 0});
+        }
     }
 }
 
@@ -255,7 +264,8 @@ fq_status_t encode_impl(const fq_layout_t* L, const uint32_t* k, const uint32_t*
     // pass 1: per tile, packets per bucket
     E.indptr.assign(ntile + 1, 0);
     E.info.assign(ntile * NB, 0);
-    std::vector<uint8_t> col2bucket(ntile * BN);  // kept for pass 2
+    std::vector<uint8_t> col2bucket(ntile * BN);
+    std::vector<std::vector<Entry>> tile_slots(ntile);  // packed slots of every tile, four per packet
     int bad = 0;
 #pragma omp parallel for schedule(dynamic, 16)
     for (int64_t t = 0; t < (int64_t)ntile; ++t) {
@@ -286,9 +296,23 @@ fq_status_t encode_impl(const fq_layout_t* L, const uint32_t* k, const uint32_t*
                 heap.push(LB(top.first + cnt[c], top.second));
             }
         }
+        // pack every bucket of the tile now: the number of packets depends on the packing
+        std::vector<std::vector<Entry>> per(NB);
+        for (size_t e = tstart[t]; e < tstart[t + 1]; ++e) per[c2b[sorted[e].c]].push_back(sorted[e]);
+        std::vector<Entry>& tp = tile_slots[t];
+        std::vector<Entry> slots;
         uint32_t off = 0;
         for (uint32_t b = 0; b < NB; ++b) {
-            uint32_t pk = (load[b] + 3) / 4;
+            uint32_t pk = 0;
+            if (!per[b].empty()) {
+                // deterministic input order: by column, then row
+                std::sort(per[b].begin(), per[b].end(), [](const Entry& x, const Entry& y) {
+                    return x.c != y.c ? x.c < y.c : x.k < y.k;
+                });
+                pack_bucket(per[b], b, BN, slots);
+                pk = (uint32_t)(slots.size() / 4);
+                tp.insert(tp.end(), slots.begin(), slots.end());
+            }
             if (off > 0xffffu || pk > 0xffffu) {
 #pragma omp atomic write
                 bad = 1;
@@ -308,45 +332,17 @@ fq_status_t encode_impl(const fq_layout_t* L, const uint32_t* k, const uint32_t*
         E.indptr[t + 1] = (uint32_t)total;
     }
     E.packets.assign((size_t)total * 16, 0);
-    // pass 2: order and write the packets
-#pragma omp parallel
-    {
-        std::vector<std::vector<Entry>> per(NB);
-        std::vector<Entry> ordered;
-#pragma omp for schedule(dynamic, 16)
-        for (int64_t t = 0; t < (int64_t)ntile; ++t) {
-            if (tstart[t] == tstart[t + 1]) continue;
-            for (auto& p : per) p.clear();
-            const uint8_t* c2b = &col2bucket[(size_t)t * BN];
-            for (size_t e = tstart[t]; e < tstart[t + 1]; ++e) per[c2b[sorted[e].c]].push_back(sorted[e]);
-            for (uint32_t b = 0; b < NB; ++b) {
-                if (per[b].empty()) continue;
-                // deterministic input order: by column, then row
-                std::sort(per[b].begin(), per[b].end(), [](const Entry& a, const Entry& c) {
-                    return a.c != c.c ? a.c < c.c : a.k < c.k;
-                });
-                order_bucket(per[b], b, ordered);
-                // inside a packet, equal columns must be neighbours (the kernel chains them in registers)
-                for (size_t p0 = 0; p0 < ordered.size(); p0 += 4)
-                    std::stable_sort(ordered.begin() + p0, ordered.begin() + std::min(p0 + 4, ordered.size()),
-                                     [](const Entry& a, const Entry& c) { return a.c < c.c; });
-                uint32_t info = E.info[(size_t)t * NB + b];
-                uint8_t* dst = &E.packets[((size_t)E.indptr[t] + (info & 0xffffu)) * 16];
-                const size_t cntp = info >> 16;
-                for (size_t s = 0; s < cntp * 4; ++s) {
-                    const bool real = s < ordered.size();
-                    // padding: value 0, row 0, and a column byte that differs between the slots of
-                    // the packet (the kernel skips value-0 slots and never touches that column)
-                    const Entry pad{0, (uint8_t)(BN - 1 - s % 4), 0};
-                    const Entry& x = real ? ordered[s] : pad;
-                    uint8_t* pk = dst + (s / 4) * 16;
-                    pk[s % 4] = x.k;
-                    pk[4 + s % 4] = x.c;
-                    uint16_t vv = real ? x.v : 0;
-                    pk[8 + 2 * (s % 4)] = (uint8_t)(vv & 0xff);
-                    pk[9 + 2 * (s % 4)] = (uint8_t)(vv >> 8);
-                }
-            }
+    // pass 2: write the packets (row bytes, column bytes, values)
+#pragma omp parallel for schedule(dynamic, 64)
+    for (int64_t t = 0; t < (int64_t)ntile; ++t) {
+        const std::vector<Entry>& tp = tile_slots[t];
+        uint8_t* dst = &E.packets[(size_t)E.indptr[t] * 16];
+        for (size_t sidx = 0; sidx < tp.size(); ++sidx) {
+            uint8_t* pk = dst + (sidx / 4) * 16;
+            pk[sidx % 4] = tp[sidx].k;
+            pk[4 + sidx % 4] = tp[sidx].c;
+            pk[8 + 2 * (sidx % 4)] = (uint8_t)(tp[sidx].v & 0xff);
+            pk[9 + 2 * (sidx % 4)] = (uint8_t)(tp[sidx].v >> 8);
         }
     }
     return FQ_OK;
@@ -437,11 +433,17 @@ fq_status_t fq_validate_tilecoo(const fq_layout_t* L, const uint32_t* indptr, co
             if (off + cnt > tile_pk) return fail(FQ_ERR_FORMAT, "bucket %u of tile %zu covers packets [%u, %u) of %u", b, t, off, off + cnt, tile_pk);
             for (uint32_t i = 0; i < cnt; ++i) {
                 const uint8_t* p = pk + (size_t)(indptr[t] + off + i) * 16;
-                int prev_col = -1;
+                // real slots of a packet: all in different columns, or four in one column
+                int nlive = 0, ndiff = 0;
+                for (int s = 0; s < 4; ++s) {
+                    if ((p[8 + 2 * s] | p[9 + 2 * s]) == 0) continue;
+                    ++nlive;
+                    for (int s2 = 0; s2 < s; ++s2)
+                        if ((p[8 + 2 * s2] | p[9 + 2 * s2]) != 0 && p[4 + s2] == p[4 + s]) ++ndiff;
+                }
+                if (ndiff != 0 && !(nlive == 4 && ndiff == 6)) return fail(FQ_ERR_FORMAT, "packet %u of tile %zu mixes repeated and distinct columns", indptr[t] + off + i, t);
                 for (int s = 0; s < 4; ++s) {
                     if ((p[8 + 2 * s] | p[9 + 2 * s]) == 0) continue;  // padding slot
-                    if ((int)p[4 + s] < prev_col) return fail(FQ_ERR_FORMAT, "packet %u of tile %zu: columns of its slots are not sorted", indptr[t] + off + i, t);
-                    prev_col = p[4 + s];
                     if (p[s] >= FQ_BK || p[4 + s] >= BN) return fail(FQ_ERR_FORMAT, "index (%u, %u) outside the tile in tile %zu", p[s], p[4 + s], t);
                     if (p[4 + s] % (NB / 32) != b / 32) return fail(FQ_ERR_FORMAT, "column %u of tile %zu sits in bucket %u, outside its block of 32 buckets", p[4 + s], t, b);
                     if (owner[p[4 + s]] >= 0 && owner[p[4 + s]] != (int16_t)b) return fail(FQ_ERR_FORMAT, "column %u of tile %zu appears in buckets %d and %u", p[4 + s], t, owner[p[4 + s]], b);

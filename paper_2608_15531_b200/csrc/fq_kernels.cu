@@ -49,9 +49,13 @@ __device__ unsigned long long g_trace[12 * 32 * 4];
 __shared__ unsigned long long s_trace[12 * 32 * 4];
 #define FQ_STAMP(role, it, ev) do { if (blockIdx.x == 0 && (it) < 32 && (ev) < 4 && lane == 0) s_trace[((role) * 32 + (it)) * 4 + (ev)] = clock64(); } while (0)
 #define FQ_DSTAMP(it, e) do { if (dw == 2) FQ_STAMP(4 + (e) / 4, it, (e) % 4); } while (0)
+// wall-clock stamps of every CTA of the small-batch kernel, [cta][event]
+__device__ unsigned long long g_ktrace[192 * 16];
+#define FQ_GT(cond, ev) do { if (cond) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_ktrace[blockIdx.x * 16 + (ev)] = t_; } } while (0)
 #else
 #define FQ_STAMP(role, it, ev) do {} while (0)
 #define FQ_DSTAMP(it, e) do {} while (0)
+#define FQ_GT(cond, ev) do {} while (0)
 #endif
 
 struct Params {
@@ -68,6 +72,7 @@ struct Params {
     float* partials;
     uint32_t M, K, N, KT, NT;
     uint32_t NB, coo_cap, stages, nsw;
+    uint32_t shc_floats;   // small-batch kernel: floats of the FP32 outlier tile(s) to clear at start
     // shared-memory offsets (bytes); the first five are relative to a stage
     uint32_t stage_bytes, off_sz, off_xcan, off_xsum, off_info, off_coo;
     uint32_t off_shc, off_xt, off_bar;
@@ -121,6 +126,9 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volat
     uint32_t spins = 0;
     unsigned long long t0 = 0;
     while (!mbar_try_wait(bar, parity)) {
+#ifdef FQ_SLEEP_NS
+        __nanosleep(FQ_SLEEP_NS);
+#endif
         if ((++spins & 0xff) == 0) {
             if (*abort_flag) return false;
             unsigned long long now = globaltimer_ns();
@@ -247,16 +255,6 @@ struct UnitIter {
 
 // ----------------------------------------------------------------------------- sparse step
 
-__device__ __forceinline__ void fma8(float4& c0, float4& c1, float v, const uint4 xv) {
-    c0.x = fmaf(v, bf16lo(xv.x), c0.x);
-    c0.y = fmaf(v, bf16hi(xv.x), c0.y);
-    c0.z = fmaf(v, bf16lo(xv.y), c0.z);
-    c0.w = fmaf(v, bf16hi(xv.y), c0.w);
-    c1.x = fmaf(v, bf16lo(xv.z), c1.x);
-    c1.y = fmaf(v, bf16hi(xv.z), c1.y);
-    c1.z = fmaf(v, bf16lo(xv.w), c1.z);
-    c1.w = fmaf(v, bf16hi(xv.w), c1.w);
-}
 
 // Position of 16-byte quad j of column c's FP32 row.  Q = quads per row when the row is XOR-swizzled
 // (4 or 8: lanes hitting random columns then spread over all bank groups), 0 = plain layout.
@@ -267,77 +265,168 @@ __device__ __forceinline__ uint32_t shc_quad(uint32_t c, uint32_t j, uint32_t ld
     return c * ldc + (j << 2);
 }
 
-// One packet (four outliers) against the k-major activation copy xt ([128][8] BF16, 16 B per row):
-// row c of the FP32 tile += v * x[8o..8o+7][k] for each slot (Section 4.2, without the per-column
-// padding: every slot carries its own column byte).  Padding slots (value 0) are skipped.  The
-// encoder sorts the real slots of a packet by column, so equal columns are neighbours: their
-// products are chained in registers and only the last slot of a run stores.  All loads are issued
-// before the first store.
+__device__ __forceinline__ void fma8(float4& c0, float4& c1, float v, const float4 x0, const float4 x1) {
+    c0.x = fmaf(v, x0.x, c0.x); c0.y = fmaf(v, x0.y, c0.y); c0.z = fmaf(v, x0.z, c0.z); c0.w = fmaf(v, x0.w, c0.w);
+    c1.x = fmaf(v, x1.x, c1.x); c1.y = fmaf(v, x1.y, c1.y); c1.z = fmaf(v, x1.z, c1.z); c1.w = fmaf(v, x1.w, c1.w);
+}
+
+// One packet (four outliers) against the k-major FP32 activation copy xt ([128][8] floats, 32 B per
+// row k): row c of the FP32 tile += v * x[8o..8o+7][k] for each slot (Section 4.2, without the
+// per-column padding: every slot carries its own column byte).  The encoder emits two kinds of
+// packets: "spread" (real slots in different columns: all loads are issued before the first store,
+// padding slots, value 0, are skipped) and "stack" (four outliers of one column: summed in registers,
+// one read-modify-write).
 template <int Q>
-__device__ __forceinline__ void apply_packet(const uint4 pk, const uint8_t* __restrict__ xt, float* shc, uint32_t o, uint32_t ldc) {
+__device__ __forceinline__ void apply_packet(const uint4 pk, const float* __restrict__ xt, float* shc, uint32_t o, uint32_t ldc) {
     uint32_t k[4], c[4];
     float v[4];
-    bool live[4];
 #pragma unroll
     for (int s = 0; s < 4; ++s) {
         k[s] = (pk.x >> (8 * s)) & 0xffu;
         c[s] = (pk.y >> (8 * s)) & 0xffu;
     }
-    live[0] = (pk.z & 0xffffu) != 0; live[1] = (pk.z >> 16) != 0; live[2] = (pk.w & 0xffffu) != 0; live[3] = (pk.w >> 16) != 0;
     v[0] = bf16lo(pk.z); v[1] = bf16hi(pk.z); v[2] = bf16lo(pk.w); v[3] = bf16hi(pk.w);
-    uint4 xv[4];
-    float4 c0[4], c1[4];
+    const bool live0 = (pk.z & 0xffffu) != 0, live1 = (pk.z >> 16) != 0, live2 = (pk.w & 0xffffu) != 0, live3 = (pk.w >> 16) != 0;
+    const bool live[4] = {live0, live1, live2, live3};
+    float4 x0[4], x1[4];
 #pragma unroll
     for (int s = 0; s < 4; ++s) {
-        xv[s] = *reinterpret_cast<const uint4*>(xt + k[s] * 16);
-        c0[s] = c1[s] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-        if (live[s]) {
-            c0[s] = *reinterpret_cast<const float4*>(shc + shc_quad<Q>(c[s], 2 * o, ldc));
-            c1[s] = *reinterpret_cast<const float4*>(shc + shc_quad<Q>(c[s], 2 * o + 1, ldc));
+        const float4* xp = reinterpret_cast<const float4*>(xt + k[s] * 8);
+        x0[s] = xp[0];
+        x1[s] = xp[1];
+    }
+    const bool stack = pk.y == __byte_perm(pk.y, 0, 0x0000) && live0 && live1 && live2 && live3;
+    if (!stack) {
+        float4 c0[4], c1[4];
+#pragma unroll
+        for (int s = 0; s < 4; ++s) {
+            c0[s] = c1[s] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            if (live[s]) {
+                c0[s] = *reinterpret_cast<const float4*>(shc + shc_quad<Q>(c[s], 2 * o, ldc));
+                c1[s] = *reinterpret_cast<const float4*>(shc + shc_quad<Q>(c[s], 2 * o + 1, ldc));
+            }
         }
-    }
-    float4 a0[4], a1[4];
 #pragma unroll
-    for (int s = 0; s < 4; ++s) {
-        a0[s] = a1[s] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-        fma8(a0[s], a1[s], v[s], xv[s]);
-    }
-    bool same[5];
-    same[0] = same[4] = false;
+        for (int s = 0; s < 4; ++s) fma8(c0[s], c1[s], v[s], x0[s], x1[s]);
 #pragma unroll
-    for (int s = 1; s < 4; ++s) {
-        same[s] = live[s] && live[s - 1] && c[s] == c[s - 1];
-        const float m = same[s] ? 1.0f : 0.0f;   // carry the running sum of an equal-column run
-        a0[s].x = fmaf(m, a0[s - 1].x, a0[s].x); a0[s].y = fmaf(m, a0[s - 1].y, a0[s].y);
-        a0[s].z = fmaf(m, a0[s - 1].z, a0[s].z); a0[s].w = fmaf(m, a0[s - 1].w, a0[s].w);
-        a1[s].x = fmaf(m, a1[s - 1].x, a1[s].x); a1[s].y = fmaf(m, a1[s - 1].y, a1[s].y);
-        a1[s].z = fmaf(m, a1[s - 1].z, a1[s].z); a1[s].w = fmaf(m, a1[s - 1].w, a1[s].w);
-    }
-#pragma unroll
-    for (int s = 0; s < 4; ++s) {
-        if (live[s] && !same[s + 1]) {
-            c0[s].x += a0[s].x; c0[s].y += a0[s].y; c0[s].z += a0[s].z; c0[s].w += a0[s].w;
-            c1[s].x += a1[s].x; c1[s].y += a1[s].y; c1[s].z += a1[s].z; c1[s].w += a1[s].w;
-            *reinterpret_cast<float4*>(shc + shc_quad<Q>(c[s], 2 * o, ldc)) = c0[s];
-            *reinterpret_cast<float4*>(shc + shc_quad<Q>(c[s], 2 * o + 1, ldc)) = c1[s];
+        for (int s = 0; s < 4; ++s) {
+            if (live[s]) {
+                *reinterpret_cast<float4*>(shc + shc_quad<Q>(c[s], 2 * o, ldc)) = c0[s];
+                *reinterpret_cast<float4*>(shc + shc_quad<Q>(c[s], 2 * o + 1, ldc)) = c1[s];
+            }
         }
+    } else {
+        float4* p0 = reinterpret_cast<float4*>(shc + shc_quad<Q>(c[0], 2 * o, ldc));
+        float4* p1 = reinterpret_cast<float4*>(shc + shc_quad<Q>(c[0], 2 * o + 1, ldc));
+        float4 c0 = *p0, c1 = *p1;
+#pragma unroll
+        for (int s = 0; s < 4; ++s) fma8(c0, c1, v[s], x0[s], x1[s]);
+        *p0 = c0;
+        *p1 = c1;
     }
 }
 
-// Transpose one octet of activation rows into xt[k][8], reading the canonical operand layout
-// (core matrix of 16-byte chunk c and octet o at (c * n_oct + o) * 128, its 8 rows 16 B apart).
-__device__ __forceinline__ void transpose_octet(uint32_t xcan_u32, uint32_t n_oct, uint32_t o, uint8_t* xt, int lane) {
+// ---- narrow-batch form (M <= 8): rows of MS = 1, 2, 4 or 8 floats, so that M = 1 moves 4 bytes per
+// outlier instead of 32.  Row pitch in floats: MS, except 12 for MS = 8 (a 48-byte pitch spreads
+// random rows over all eight 16-byte bank groups; a 32-byte pitch would use only four).
+__host__ __device__ constexpr int ms_pitch(int ms) { return ms == 8 ? 12 : ms; }
+
+template <int MS>
+__device__ __forceinline__ void ld_row(const float* p, float (&r)[MS]) {
+    if constexpr (MS == 1) { r[0] = *p; }
+    else if constexpr (MS == 2) { const float2 v = *reinterpret_cast<const float2*>(p); r[0] = v.x; r[1] = v.y; }
+    else {
+#pragma unroll
+        for (int i = 0; i < MS / 4; ++i) {
+            const float4 v = reinterpret_cast<const float4*>(p)[i];
+            r[4 * i] = v.x; r[4 * i + 1] = v.y; r[4 * i + 2] = v.z; r[4 * i + 3] = v.w;
+        }
+    }
+}
+template <int MS>
+__device__ __forceinline__ void st_row(float* p, const float (&r)[MS]) {
+    if constexpr (MS == 1) { *p = r[0]; }
+    else if constexpr (MS == 2) { *reinterpret_cast<float2*>(p) = make_float2(r[0], r[1]); }
+    else {
+#pragma unroll
+        for (int i = 0; i < MS / 4; ++i) reinterpret_cast<float4*>(p)[i] = make_float4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
+    }
+}
+
+// A decoded packet with its activation rows loaded (narrow form).  col[s] is the row of the FP32
+// tile that slot s updates: its column, or this lane's dummy row (index `dummy`, past the tile) for a
+// padding slot and for slots 1..3 of a stack packet (four outliers of one column, folded into slot
+// 0).  With the dummy row every slot does the same loads and stores: no branch depends on the data.
+template <int MS>
+struct NarrowPacket {
+    uint32_t col[4];
+    float v[4];
+    float x[4][MS];
+    bool stack;
+};
+
+template <int MS>
+__device__ __forceinline__ void narrow_fetch(NarrowPacket<MS>& t, const uint4 pk, const float* xt, uint32_t dummy) {
+    constexpr int P = ms_pitch(MS);
+#pragma unroll
+    for (int s = 0; s < 4; ++s) ld_row<MS>(xt + ((pk.x >> (8 * s)) & 0xffu) * P, t.x[s]);
+    t.v[0] = bf16lo(pk.z); t.v[1] = bf16hi(pk.z); t.v[2] = bf16lo(pk.w); t.v[3] = bf16hi(pk.w);
+    const bool l0 = (pk.z & 0xffffu) != 0, l1 = (pk.z >> 16) != 0, l2 = (pk.w & 0xffffu) != 0, l3 = (pk.w >> 16) != 0;
+    t.stack = pk.y == __byte_perm(pk.y, 0, 0x0000) && l0 && l1 && l2 && l3;
+    t.col[0] = l0 ? (pk.y & 0xffu) : dummy;
+    t.col[1] = (l1 && !t.stack) ? ((pk.y >> 8) & 0xffu) : dummy;
+    t.col[2] = (l2 && !t.stack) ? ((pk.y >> 16) & 0xffu) : dummy;
+    t.col[3] = (l3 && !t.stack) ? (pk.y >> 24) : dummy;
+}
+
+// Loads of the FP32 rows, then the FMAs; the stores are a separate step so that the caller can issue
+// the next packet's loads between them.
+template <int MS>
+__device__ __forceinline__ void narrow_accumulate(const NarrowPacket<MS>& t, const float* shc, float (&a)[4][MS]) {
+    constexpr int P = ms_pitch(MS);
+#pragma unroll
+    for (int s = 0; s < 4; ++s) ld_row<MS>(shc + t.col[s] * P, a[s]);
+#pragma unroll
+    for (int s = 1; s < 4; ++s)
+#pragma unroll
+        for (int i = 0; i < MS; ++i) {
+            const float c = t.v[s] * t.x[s][i];
+            a[s][i] += c;
+            a[0][i] += t.stack ? c : 0.0f;
+        }
+#pragma unroll
+    for (int i = 0; i < MS; ++i) a[0][i] = fmaf(t.v[0], t.x[0][i], a[0][i]);
+}
+template <int MS>
+__device__ __forceinline__ void narrow_store(const NarrowPacket<MS>& t, float* shc, const float (&a)[4][MS]) {
+    constexpr int P = ms_pitch(MS);
+    // slots that share the dummy row overwrite one another there: nothing reads it
+#pragma unroll
+    for (int s = 3; s >= 0; --s) st_row<MS>(shc + t.col[s] * P, a[s]);
+}
+
+// Transpose one octet of BF16 activation rows into the FP32 k-major copy xt[k][8] (32 B per k).
+// `row0` is the shared-memory address of row 0 / 16-byte chunk 0 of the octet, rows `row_step`
+// bytes apart, consecutive 16-byte chunks (8 k each) `chunk_step` bytes apart.  Whole warp.
+// `pitch` floats per k in xt; only the first `ms` rows of the octet are written (ms = 1, 2, 4, 8).
+__device__ __forceinline__ void transpose_octet_f32(uint32_t row0, uint32_t row_step, uint32_t chunk_step, float* xt, int lane,
+                                                    uint32_t pitch = 8, uint32_t ms = 8) {
 #pragma unroll
     for (int kb = 0; kb < 4; ++kb) {
-        uint32_t r0, r1, r2, r3;
-        const uint32_t addr = xcan_u32 + ((kb * 4 + (lane >> 3)) * n_oct + o) * 128 + (lane & 7) * 16;
-        ldmatrix_x4_trans(addr, r0, r1, r2, r3);
+        uint32_t r[4];
+        ldmatrix_x4_trans(row0 + (lane & 7) * row_step + (kb * 4 + (lane >> 3)) * chunk_step, r[0], r[1], r[2], r[3]);
         // thread T holds rows m = 2(T%4), 2(T%4)+1 of column k = 8*block + T/4
-        uint8_t* dst = xt + ((kb * 32) + (lane >> 2)) * 16 + (lane & 3) * 4;
-        *reinterpret_cast<uint32_t*>(dst) = r0;
-        *reinterpret_cast<uint32_t*>(dst + 8 * 16) = r1;
-        *reinterpret_cast<uint32_t*>(dst + 16 * 16) = r2;
-        *reinterpret_cast<uint32_t*>(dst + 24 * 16) = r3;
+        const uint32_t m0 = (lane & 3) * 2;
+        float* dst = xt + ((kb * 32) + (lane >> 2)) * pitch + m0;
+        if (ms >= 2) {
+            if (m0 < ms) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) *reinterpret_cast<float2*>(dst + i * 8 * pitch) = make_float2(bf16lo(r[i]), bf16hi(r[i]));
+            }
+        } else if (m0 == 0) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) dst[i * 8 * pitch] = bf16lo(r[i]);
+        }
     }
 }
 
@@ -533,6 +622,13 @@ __global__ void __launch_bounds__(32 * (4 + 2 * (BN / 32) + 4), 1) fq_fused_kern
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
+            if (SPARSE) {
+                // FP32 k-major copy for the sparse warps, one octet of rows at a time
+                for (uint32_t o = 0; o < ((p.M + 7) >> 3); ++o)
+                    transpose_octet_f32(smem_u32(st + p.off_xcan) + o * 128, 16, (NMMA / 8) * 128,
+                                        reinterpret_cast<float*>(st + p.off_xt) + o * 1024, lane);
+                __syncwarp();
+            }
             if (lane == 0) mbar_arrive(bar_full + 8 * s);
         }
     } else if (warp >= 4 && warp < 4 + NDW) {
@@ -701,7 +797,6 @@ __global__ void __launch_bounds__(32 * (4 + 2 * (BN / 32) + 4), 1) fq_fused_kern
             const uint32_t bb = sw % nbb, og = sw / nbb, n_og = nsw / nbb;
             const uint32_t bucket = bb * 32 + lane;
             const uint32_t n_oct = (p.M + 7) >> 3;
-            uint8_t* xt = smem + p.off_xt + sw * 2048;
             uint32_t piece = 0;
             for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
                 const uint32_t u = w.u, s = w.s, ph = w.ph, kt = w.kt;
@@ -714,8 +809,7 @@ __global__ void __launch_bounds__(32 * (4 + 2 * (BN / 32) + 4), 1) fq_fused_kern
                 const uint4* pk_g = nullptr;
                 if (off + cnt > p.coo_cap) pk_g = p.packed + __ldg(p.indptr + u);  // tail of an oversized tile
                 for (uint32_t o = og; o < n_oct; o += n_og) {
-                    transpose_octet(smem_u32(st + p.off_xcan), NMMA / 8, o, xt, lane);
-                    __syncwarp();
+                    const float* xt = reinterpret_cast<const float*>(st + p.off_xt) + o * 1024;
                     if (sw == 0) FQ_STAMP(3, w.it, 1);
 #ifdef FQ_TRACE
                     if (sw == 0 && blockIdx.x == 0 && w.it < 32) {
@@ -782,7 +876,7 @@ constexpr int kXPitch = 320;   // activation row in shared memory: 256 B + 64 B,
 //                     follows the 16-byte activation loads of the lanes)
 //   then              sparse warps
 template <int BN, int MO, int GROUP, bool SPARSE>
-__global__ void __launch_bounds__(32 * (2 + BN / 16 + 4), 1) fq_mma_kernel(const Params p) {
+__global__ void __launch_bounds__(32 * (2 + BN / 16 + 6), 1) fq_mma_kernel(const Params p) {
     constexpr int NDW = BN / 16;
     constexpr int GPS = kBK / GROUP;
     constexpr int W_BYTES = 16 * BN * 4;
@@ -792,7 +886,15 @@ __global__ void __launch_bounds__(32 * (2 + BN / 16 + 4), 1) fq_mma_kernel(const
     extern __shared__ __align__(128) uint8_t smem[];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    FQ_GT(tid == 0, 0);
     const uint32_t S = p.stages;
+    // rows kept per outlier in the one-octet form: the batch rounded up to 1, 2, 4 or 8
+    const uint32_t ms = p.M <= 1 ? 1u : p.M <= 2 ? 2u : p.M <= 4 ? 4u : 8u;
+    const uint32_t msp = ms_pitch(ms);
+    // one-octet form: the sparse warps split the units between them (a warp owns fixed stages) and each
+    // replica has its own FP32 tile of BN columns + one dummy row per lane
+    const uint32_t shc_copy = (BN + 32) * msp;
+    const uint32_t n_rep = (SPARSE && MO == 1) ? p.nsw / (p.NB >> 5) : 1u;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
     const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * S;
     const uint32_t bar_sparse_done = bar_empty + 8 * S, bar_dense_done = bar_sparse_done + 8, bar_dense = bar_dense_done + 8;
@@ -804,7 +906,8 @@ __global__ void __launch_bounds__(32 * (2 + BN / 16 + 4), 1) fq_mma_kernel(const
     if (tid == 0) {
         for (uint32_t s = 0; s < S; ++s) {
             mbar_init(bar_full + 8 * s, 2);   // producer's expect_tx arrival + activation warp
-            mbar_init(bar_empty + 8 * s, NDW + nsw);
+            // one-octet form: each stage has one sparse warp per block of 32 buckets (fixed owner)
+            mbar_init(bar_empty + 8 * s, NDW + (MO == 1 ? (SPARSE ? p.NB >> 5 : 0u) : nsw));
         }
         mbar_init(bar_sparse_done, nsw ? nsw : 1);
         mbar_init(bar_dense_done, NDW);
@@ -814,10 +917,11 @@ __global__ void __launch_bounds__(32 * (2 + BN / 16 + 4), 1) fq_mma_kernel(const
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (SPARSE) {
-        for (uint32_t i = tid; i < (uint32_t)(BN * LDC); i += blockDim.x) shc[i] = 0.0f;
+        for (uint32_t i = tid; i < p.shc_floats; i += blockDim.x) shc[i] = 0.0f;
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncthreads();
+    FQ_GT(tid == 0, 1);
 
     const uint32_t U = p.NT * p.KT, P = gridDim.x, q = U / P, r = U % P;
     const uint32_t u_begin = unit_begin_of(blockIdx.x, q, r);
@@ -919,6 +1023,17 @@ __global__ void __launch_bounds__(32 * (2 + BN / 16 + 4), 1) fq_mma_kernel(const
                 else if (part == 0) xsum[m] = s1;
             }
             __syncwarp();
+            if (SPARSE) {
+                // FP32 k-major copy for the sparse warps, one octet of rows at a time
+                if (MO == 1) {
+                    transpose_octet_f32(smem_u32(st + p.off_xcan), kXPitch, 16, reinterpret_cast<float*>(st + p.off_xt), lane, msp, ms);
+                } else {
+                    for (uint32_t o = 0; o < ((p.M + 7) >> 3); ++o)
+                        transpose_octet_f32(smem_u32(st + p.off_xcan) + o * 8 * kXPitch, kXPitch, 16,
+                                            reinterpret_cast<float*>(st + p.off_xt) + o * 1024, lane);
+                }
+                __syncwarp();
+            }
             if (lane == 0) mbar_arrive(bar_full + 8 * s);
         }
     } else if (warp >= 2 && warp < 2 + NDW) {
@@ -937,10 +1052,14 @@ __global__ void __launch_bounds__(32 * (2 + BN / 16 + 4), 1) fq_mma_kernel(const
             const uint32_t u = w.u, s = w.s, ph = w.ph, tn = w.tn, kt = w.kt;
             const uint8_t* st = smem + s * p.stage_bytes;
             if (!warp_wait(bar_full + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
+            FQ_GT(dtid == 0 && w.it == 0, 2);
             const uint32_t* wp = reinterpret_cast<const uint32_t*>(st) + c0 * 4 + t;
             const uint8_t* xrow = st + p.off_xcan + g * kXPitch + t * 16;
             const uint16_t* sc = reinterpret_cast<const uint16_t*>(st + p.off_sz);
             const float* xsum = reinterpret_cast<const float*>(st + p.off_xsum);
+#if defined(FQ_EXP) && FQ_EXP == 7
+            if (false)
+#endif
 #pragma unroll
             for (int gi = 0; gi < GPS; ++gi) {
                 float accg[MO][4];
@@ -980,21 +1099,38 @@ __global__ void __launch_bounds__(32 * (2 + BN / 16 + 4), 1) fq_mma_kernel(const
 
             if (kt == KT - 1 || u == u_end - 1) {
                 // ---------------------------------------------------------- end of a piece
+                FQ_GT(dtid == 0 && piece < 2, 4 + 5 * piece);
                 if (SPARSE) {
                     if (!warp_wait(bar_sparse_done, piece & 1, abort_flag, p.status)) { ok = false; break; }
+                    if (MO == 1) {
+                        // rows of msp floats, rows 2t and 2t+1 of this lane's two columns
 #pragma unroll
-                    for (int h = 0; h < 2; ++h)
+                        for (int h = 0; h < 2; ++h)
 #pragma unroll
-                        for (int o = 0; o < MO; ++o) {
-                            float2* cp = reinterpret_cast<float2*>(shc + shc_quad<Q>(c0 + 8 * h, 2 * o + (t >> 1), LDC) + 2 * (t & 1));
-                            const float2 v = *cp;
-                            accf[o][2 * h + 0] += v.x;
-                            accf[o][2 * h + 1] += v.y;
-                            *cp = make_float2(0.0f, 0.0f);
-                        }
+                            for (int j = 0; j < 2; ++j)
+                                if ((uint32_t)(2 * t + j) < ms) {
+                                    float* cp = shc + (c0 + 8 * h) * msp + 2 * t + j;
+                                    for (uint32_t rr = 0; rr < n_rep; ++rr, cp += shc_copy) {
+                                        accf[0][2 * h + j] += *cp;
+                                        *cp = 0.0f;
+                                    }
+                                }
+                    } else {
+#pragma unroll
+                        for (int h = 0; h < 2; ++h)
+#pragma unroll
+                            for (int o = 0; o < MO; ++o) {
+                                float2* cp = reinterpret_cast<float2*>(shc + shc_quad<Q>(c0 + 8 * h, 2 * o + (t >> 1), LDC) + 2 * (t & 1));
+                                const float2 v = *cp;
+                                accf[o][2 * h + 0] += v.x;
+                                accf[o][2 * h + 1] += v.y;
+                                *cp = make_float2(0.0f, 0.0f);
+                            }
+                    }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_dense_done);
                 }
+                FQ_GT(dtid == 0 && piece < 2, 5 + 5 * piece);
                 const uint32_t u_tile0 = tn * KT;
                 const uint32_t piece_k0 = max(u_tile0, u_begin) - u_tile0;
                 const bool full_piece = (piece_k0 == 0) && (kt == KT - 1);
@@ -1012,6 +1148,7 @@ __global__ void __launch_bounds__(32 * (2 + BN / 16 + 4), 1) fq_mma_kernel(const
                     if (lane == 0) mbar_arrive(bar_dense);
                     if (!warp_wait(bar_dense, dense_phase & 1, abort_flag, p.status)) { ok = false; break; }
                     ++dense_phase;
+                    FQ_GT(dtid == 0 && piece < 2, 6 + 5 * piece);
                     const uint32_t c_first = cta_of_unit(u_tile0, q, r), c_last = cta_of_unit(u_tile0 + KT - 1, q, r);
                     if (dtid == 0) {
                         const uint32_t old = atomicAdd(p.counters + tn, 1u);
@@ -1021,6 +1158,7 @@ __global__ void __launch_bounds__(32 * (2 + BN / 16 + 4), 1) fq_mma_kernel(const
                     if (lane == 0) mbar_arrive(bar_dense);
                     if (!warp_wait(bar_dense, dense_phase & 1, abort_flag, p.status)) { ok = false; break; }
                     ++dense_phase;
+                    FQ_GT(dtid == 0 && piece < 2, 7 + 5 * piece);
                     if (*last_flag) {
                         write_y = true;
                         __threadfence();
@@ -1054,9 +1192,11 @@ __global__ void __launch_bounds__(32 * (2 + BN / 16 + 4), 1) fq_mma_kernel(const
                 for (int o = 0; o < MO; ++o)
 #pragma unroll
                     for (int i = 0; i < 4; ++i) accf[o][i] = 0.0f;
+                FQ_GT(dtid == 0 && piece < 2, 8 + 5 * piece);
                 ++piece;
             }
         }
+        FQ_GT(dtid == 0, 15);
     } else if (SPARSE && warp >= 2 + NDW) {
         // ------------------------------------------------------------------ sparse
         const uint32_t sw = warp - (2 + NDW);
@@ -1065,38 +1205,87 @@ __global__ void __launch_bounds__(32 * (2 + BN / 16 + 4), 1) fq_mma_kernel(const
             const uint32_t bb = sw % nbb, og = sw / nbb, n_og = nsw / nbb;
             const uint32_t bucket = bb * 32 + lane;
             const uint32_t n_oct = (p.M + 7) >> 3;
-            uint8_t* xt = smem + p.off_xt + sw * 2048;
             uint32_t piece = 0;
+            // one-octet form: replica og of n_og owns the stages s with s mod n_og == og
+            uint32_t own = 0xffffffffu;
+            float* my_shc = shc;
+            if (MO == 1) {
+                own = 0;
+                for (uint32_t s = og; s < S; s += n_og) own |= 1u << s;
+                my_shc = shc + og * shc_copy;
+            }
+#ifdef FQ_TRACE
+            long long t_loop = 0, t_wait = 0, t_all0 = clock64(); uint32_t n_iter = 0, n_units = 0;
+#endif
             for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
                 const uint32_t u = w.u, s = w.s, ph = w.ph, kt = w.kt;
                 const uint8_t* st = smem + s * p.stage_bytes;
+                if ((own >> s) & 1u) {
+#ifdef FQ_TRACE
+                long long tw0 = clock64();
+#endif
                 if (!warp_wait(bar_full + 8 * s, ph, abort_flag, p.status)) break;
+#ifdef FQ_TRACE
+                t_wait += clock64() - tw0; ++n_units;
+#endif
                 const uint32_t info = reinterpret_cast<const uint32_t*>(st + p.off_info)[bucket];
                 const uint32_t off = info & 0xffffu, cnt = info >> 16;
                 const uint4* pk_s = reinterpret_cast<const uint4*>(st + p.off_coo);
                 const uint4* pk_g = nullptr;
                 if (off + cnt > p.coo_cap) pk_g = p.packed + __ldg(p.indptr + u);
-                for (uint32_t o = og; o < n_oct; o += n_og) {
-                    // row-major rows (kXPitch apart) -> xt[k][8]
-#pragma unroll
-                    for (int kb = 0; kb < 4; ++kb) {
-                        uint32_t r0, r1, r2, r3;
-                        ldmatrix_x4_trans(smem_u32(st + p.off_xcan) + (o * 8 + (lane & 7)) * kXPitch + (kb * 4 + (lane >> 3)) * 16, r0, r1, r2, r3);
-                        uint8_t* dst = xt + ((kb * 32) + (lane >> 2)) * 16 + (lane & 3) * 4;
-                        *reinterpret_cast<uint32_t*>(dst) = r0;
-                        *reinterpret_cast<uint32_t*>(dst + 8 * 16) = r1;
-                        *reinterpret_cast<uint32_t*>(dst + 16 * 16) = r2;
-                        *reinterpret_cast<uint32_t*>(dst + 24 * 16) = r3;
-                    }
+#ifdef FQ_TRACE
+                long long tl0 = clock64(); n_iter += __reduce_max_sync(0xffffffffu, cnt);
+#endif
+                if (MO == 1) {
+                    const float* xt = reinterpret_cast<const float*>(st + p.off_xt);
+                    auto run = [&](auto tag) {
+                        constexpr int MS = decltype(tag)::value;
+                        auto packet = [&](uint32_t i) {
+                            const uint32_t idx = off + i;
+                            return (idx < p.coo_cap) ? pk_s[idx] : __ldg(pk_g + idx);
+                        };
+                        if (cnt == 0) return;
+                        const uint32_t dummy = BN + lane;
+                        NarrowPacket<MS> cur;
+                        narrow_fetch<MS>(cur, packet(0), xt, dummy);
+                        for (uint32_t i = 0; i < cnt; ++i) {
+                            // the next packet and its activation rows are in flight while this one is applied
+                            const bool more = i + 1 < cnt;
+                            const uint4 pkn = more ? packet(i + 1) : make_uint4(0, 0, 0, 0);
+                            float a[4][MS];
+                            narrow_accumulate<MS>(cur, my_shc, a);
+                            NarrowPacket<MS> nxt;
+                            if constexpr (MS <= 4) {
+                                narrow_fetch<MS>(nxt, pkn, xt, dummy);
+                                narrow_store<MS>(cur, my_shc, a);
+                            } else {           // eight-float rows: not enough registers for both at once
+                                narrow_store<MS>(cur, my_shc, a);
+                                narrow_fetch<MS>(nxt, pkn, xt, dummy);
+                            }
+                            cur = nxt;
+                        }
+                    };
+                    if (ms == 1) run(std::integral_constant<int, 1>{});
+                    else if (ms == 2) run(std::integral_constant<int, 2>{});
+                    else if (ms == 4) run(std::integral_constant<int, 4>{});
+                    else run(std::integral_constant<int, 8>{});
                     __syncwarp();
-                    for (uint32_t i = 0; i < cnt; ++i) {
-                        const uint32_t idx = off + i;
-                        const uint4 pk = (idx < p.coo_cap) ? pk_s[idx] : __ldg(pk_g + idx);
-                        apply_packet<Q>(pk, xt, shc, o, LDC);
+                } else {
+                    for (uint32_t o = og; o < n_oct; o += n_og) {
+                        const float* xt = reinterpret_cast<const float*>(st + p.off_xt) + o * 1024;
+                        for (uint32_t i = 0; i < cnt; ++i) {
+                            const uint32_t idx = off + i;
+                            const uint4 pk = (idx < p.coo_cap) ? pk_s[idx] : __ldg(pk_g + idx);
+                            apply_packet<Q>(pk, xt, shc, o, LDC);
+                        }
+                        __syncwarp();
                     }
-                    __syncwarp();
                 }
+#ifdef FQ_TRACE
+                t_loop += clock64() - tl0;
+#endif
                 if (lane == 0) mbar_arrive_relaxed(bar_empty + 8 * s);
+                }
                 if (kt == KT - 1 || u == u_end - 1) {
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_sparse_done);
@@ -1104,6 +1293,12 @@ __global__ void __launch_bounds__(32 * (2 + BN / 16 + 4), 1) fq_mma_kernel(const
                     ++piece;
                 }
             }
+#ifdef FQ_TRACE
+            if (blockIdx.x == 0 && sw == 0 && lane == 0) {
+                g_trace[0] = (unsigned long long)t_loop; g_trace[1] = n_iter; g_trace[2] = n_units;
+                g_trace[3] = (unsigned long long)t_wait; g_trace[4] = (unsigned long long)(clock64() - t_all0);
+            }
+#endif
         }
     }
 }
@@ -1121,7 +1316,7 @@ __global__ void __launch_bounds__(256) fq_spmm_kernel(const uint16_t* __restrict
     extern __shared__ __align__(128) uint8_t smem[];
     const uint32_t LDC = 8 * MO;
     float* shc = reinterpret_cast<float*>(smem);                    // [BN][8 MO]
-    uint8_t* xt = smem + (size_t)BN * LDC * 4;                       // [MO][128][8] BF16
+    float* xt = reinterpret_cast<float*>(smem + (size_t)BN * LDC * 4);   // [MO][128][8] FP32
     const uint32_t tn = blockIdx.x, KT = K / kBK;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     for (uint32_t i = tid; i < BN * LDC; i += blockDim.x) shc[i] = 0.0f;
@@ -1131,7 +1326,7 @@ __global__ void __launch_bounds__(256) fq_spmm_kernel(const uint16_t* __restrict
         for (uint32_t i = tid; i < 128 * LDC; i += blockDim.x) {
             const uint32_t k = i / LDC, m = i % LDC;
             const uint16_t v = (m < M) ? X[(size_t)m * K + (size_t)kt * kBK + k] : (uint16_t)0;
-            reinterpret_cast<uint16_t*>(xt)[((m >> 3) * 128 + k) * 8 + (m & 7)] = v;
+            xt[((m >> 3) * 128 + k) * 8 + (m & 7)] = bf16_bits_to_float(v);
         }
         __syncthreads();
         const size_t t = (size_t)tn * KT + kt;
@@ -1142,7 +1337,7 @@ __global__ void __launch_bounds__(256) fq_spmm_kernel(const uint16_t* __restrict
             const uint32_t bb = w % nbb, o = w / nbb;
             const uint32_t inf = info[t * NB + bb * 32 + lane];
             const uint32_t off = inf & 0xffffu, cnt = inf >> 16;
-            for (uint32_t i = 0; i < cnt; ++i) apply_packet<0>(__ldg(pk + off + i), xt + o * 2048, shc, o, LDC);
+            for (uint32_t i = 0; i < cnt; ++i) apply_packet<0>(__ldg(pk + off + i), xt + o * 1024, shc, o, LDC);
         }
     }
     __syncthreads();
@@ -1191,7 +1386,7 @@ static fq_status_t make_plan(const fq_layout_t* L, uint32_t M, bool sparse, Plan
     std::memset(&p, 0, sizeof(p));
     p.M = M; p.K = L->K; p.N = L->N; p.KT = L->K / kBK; p.NT = L->N / BN; p.NB = NB; p.nsw = nsw;
     const uint32_t w_bytes = 16 * BN * 4, sz_bytes = 2 * GPS * BN * 2;
-    const uint32_t fixed = (sparse ? BN * NMMA * 4 + nsw * 2048 : 0) + 1024;
+    const uint32_t fixed = (sparse ? BN * NMMA * 4 : 0) + 1024;
     uint32_t cap = 0;
     if (sparse) {
         cap = L->max_tile_packets ? round_up(L->max_tile_packets, 8) : 256;
@@ -1202,7 +1397,8 @@ static fq_status_t make_plan(const fq_layout_t* L, uint32_t M, bool sparse, Plan
         p.off_sz = w_bytes;
         p.off_xcan = p.off_sz + round_up(sz_bytes, 128);
         p.off_xsum = p.off_xcan + NMMA * 256;
-        p.off_info = p.off_xsum + round_up(GPS * NMMA * 4, 128);
+        p.off_xt = p.off_xsum + round_up(GPS * NMMA * 4, 128);          // stage-relative: FP32 k-major copy
+        p.off_info = p.off_xt + (sparse ? ((M + 7) / 8) * 4096 : 0);
         p.off_coo = p.off_info + (sparse ? round_up(NB * 4, 128) : 0);
         stage = round_up(p.off_coo + cap * 16, 128);
         S = std::min<uint32_t>(8, (kSmemBudget - fixed) / stage);
@@ -1212,8 +1408,7 @@ static fq_status_t make_plan(const fq_layout_t* L, uint32_t M, bool sparse, Plan
     if (S < 3) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "shared-memory stages do not fit");
     p.coo_cap = cap; p.stages = S; p.stage_bytes = stage;
     p.off_shc = S * stage;
-    p.off_xt = p.off_shc + (sparse ? BN * NMMA * 4 : 0);
-    p.off_bar = p.off_xt + nsw * 2048;
+    p.off_bar = p.off_shc + (sparse ? BN * NMMA * 4 : 0);
     pl.smem = p.off_bar + 1024;
     pl.threads = 32 * (4 + 2 * NDW + nsw);
     const int sms = sm_count_cached();
@@ -1222,21 +1417,42 @@ static fq_status_t make_plan(const fq_layout_t* L, uint32_t M, bool sparse, Plan
     return FQ_OK;
 }
 
+// Sparse warps per CTA of the small-batch kernel at M <= 8 (developer knob: FQ_SPARSE_WARPS = 1..6).
+static uint32_t sparse_warps_target() {
+    static const uint32_t v = [] {
+        const char* e = std::getenv("FQ_SPARSE_WARPS");
+        const int n = e ? std::atoi(e) : 4;
+        return (uint32_t)std::min(6, std::max(1, n));
+    }();
+    return v;
+}
+
 // Plan of the small-batch kernel (fq_mma_kernel): M <= 16 per launch.
 static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, Plan& pl) {
     const uint32_t BN = L->BN, NB = L->buckets_per_tile, GPS = kBK / L->group;
     const uint32_t MO = M <= 8 ? 1 : 2, ROWS = 8 * MO;
     const uint32_t NDW = BN / 16;
-    uint32_t nsw = 0;
+    uint32_t nsw = 0, n_rep = 1;
     if (sparse) {
         const uint32_t nbb = NB / 32, n_oct = (M + 7) / 8;
-        nsw = nbb * std::min<uint32_t>(n_oct, std::max<uint32_t>(1, 4 / nbb));
+        if (MO == 1) {
+            // replicas split the units between them (each owns fixed stages and an FP32 tile of its own)
+            n_rep = std::max<uint32_t>(1, sparse_warps_target() / nbb);
+            nsw = nbb * n_rep;
+        } else {
+            nsw = nbb * std::min<uint32_t>(n_oct, std::max<uint32_t>(1, 4 / nbb));
+        }
     }
     Params& p = pl.p;
     std::memset(&p, 0, sizeof(p));
     p.M = M; p.K = L->K; p.N = L->N; p.KT = L->K / kBK; p.NT = L->N / BN; p.NB = NB; p.nsw = nsw;
     const uint32_t w_bytes = 16 * BN * 4, sz_bytes = 2 * GPS * BN * 2;
-    const uint32_t fixed = (sparse ? BN * ROWS * 4 + nsw * 2048 : 0) + 1024;
+    // one octet: FP32 rows of at most 12 floats (ms_pitch); two octets: the 8-float rows of the wide form
+    const uint32_t msp = ms_pitch(M <= 1 ? 1 : M <= 2 ? 2 : M <= 4 ? 4 : 8);
+    const uint32_t shc_bytes = sparse ? (MO == 1 ? n_rep * (BN + 32) * msp : BN * ROWS) * 4 : 0;
+    const uint32_t xt_bytes = sparse ? (MO == 1 ? kBK * msp * 4 : MO * 4096) : 0;
+    p.shc_floats = shc_bytes / 4;
+    const uint32_t fixed = shc_bytes + 1024;
     uint32_t cap = 0;
     if (sparse) {
         cap = L->max_tile_packets ? round_up(L->max_tile_packets, 8) : 256;
@@ -1247,7 +1463,8 @@ static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, 
         p.off_sz = w_bytes;
         p.off_xcan = p.off_sz + round_up(sz_bytes, 128);
         p.off_xsum = p.off_xcan + round_up(ROWS * kXPitch, 128);
-        p.off_info = p.off_xsum + round_up(GPS * ROWS * 4, 128);
+        p.off_xt = p.off_xsum + round_up(GPS * ROWS * 4, 128);          // stage-relative in this kernel
+        p.off_info = p.off_xt + round_up(xt_bytes, 128);
         p.off_coo = p.off_info + (sparse ? round_up(NB * 4, 128) : 0);
         stage = round_up(p.off_coo + cap * 16, 128);
         S = std::min<uint32_t>(8, (kSmemBudget - fixed) / stage);
@@ -1257,8 +1474,7 @@ static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, 
     if (S < 3) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "shared-memory stages do not fit");
     p.coo_cap = cap; p.stages = S; p.stage_bytes = stage;
     p.off_shc = S * stage;
-    p.off_xt = p.off_shc + (sparse ? BN * ROWS * 4 : 0);
-    p.off_bar = p.off_xt + nsw * 2048;
+    p.off_bar = p.off_shc + shc_bytes;
     pl.smem = p.off_bar + 1024;
     pl.threads = 32 * (2 + NDW + nsw);
     const int sms = sm_count_cached();
@@ -1380,6 +1596,9 @@ extern "C" {
 int fq_trace_read(unsigned long long* out) {
     return (int)cudaMemcpyFromSymbol(out, fq::g_trace, sizeof(unsigned long long) * 12 * 32 * 4);
 }
+int fq_ktrace_read(unsigned long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, fq::g_ktrace, sizeof(unsigned long long) * 192 * 16);
+}
 #endif
 
 fq_status_t fq_workspace_bytes(const fq_layout_t* L, uint32_t M, size_t* bytes) {
@@ -1462,7 +1681,7 @@ fq_status_t fq_unfused_spmm(const fq_layout_t* L, const void* X, uint32_t M, con
     for (uint32_t m0 = 0; m0 < M; m0 += 32) {
         const uint32_t mb = std::min<uint32_t>(32, M - m0);
         const uint32_t MO = (mb + 7) / 8;
-        const size_t smem = (size_t)L->BN * 8 * MO * 4 + (size_t)MO * 2048;
+        const size_t smem = (size_t)L->BN * 8 * MO * 4 + (size_t)MO * 4096;
         const uint16_t* x = (const uint16_t*)X + (size_t)m0 * L->K;
         uint16_t* y = (uint16_t*)Y + (size_t)m0 * L->N;
         cudaError_t e;

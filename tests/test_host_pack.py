@@ -78,9 +78,9 @@ def _as_set(k, n, v):
 
 
 def _bank_conflict_cycles(bk, bb, order_pos, NB):
-    """Shared-memory passes of the sparse lanes' 16-byte activation reads: lanes (= buckets) are
-    served eight at a time; at entry position i the eight rows k must fall in distinct 16-byte
-    bank groups (k mod 8) to be served in one pass, identical rows broadcast."""
+    """Shared-memory passes of the sparse lanes' activation reads (32-byte FP32 rows, so rows k and
+    k + 4 share banks): lanes (= buckets) are served eight at a time; at entry position i the passes
+    needed are the largest number of different rows falling in one bank group (k mod 4)."""
     cycles = 0
     per_bucket = {}
     for k, b, pos in zip(bk, bb, order_pos):
@@ -91,7 +91,7 @@ def _bank_conflict_cycles(bk, bb, order_pos, NB):
             rows = {per_bucket[b][i] for b in range(q0, q0 + 8) if b in per_bucket and i in per_bucket[b]}
             groups = {}
             for k in rows:
-                groups[k % 8] = groups.get(k % 8, 0) + 1
+                groups[k % 4] = groups.get(k % 4, 0) + 1
             cycles += max(groups.values(), default=0)
     return cycles
 
@@ -108,7 +108,7 @@ def test_tilecoo_encode_invariants(layout, density, NB):
     assert n_ip == ntile + 1 == indptr.size and n_bi == ntile * NB == info.size and n_pk == packed.shape[0]
     assert L.max_tile_packets == mx == int(np.diff(indptr).max())
     assert indptr[0] == 0 and np.all(np.diff(indptr.astype(np.int64)) >= 0) and indptr[-1] == n_pk
-    assert 4 * Lr.nnz <= 16 * n_pk <= 4 * (Lr.nnz + 3 * ntile * NB)
+    assert 4 * Lr.nnz <= 16 * n_pk <= 16 * Lr.nnz          # every packet carries at least one outlier
     # decoded set == input set, by the oracle's reader and by the library's
     want = _as_set(Lr.coo_k, Lr.coo_n, Lr.coo_v)
     k, n, v, b = oracle.decode_tilecoo(indptr, info, packed, K, N, BN, NB)
@@ -146,15 +146,28 @@ def test_tilecoo_element_order_separates_columns_and_staggers_bank_groups():
     for i, bb in enumerate(b.tolist()):
         pos[i] = seen.get(bb, 0)
         seen[bb] = pos[i] + 1
-    # rule 1: the slots of a packet are sorted by column, and a packet repeats a column only when no
-    # other column had entries left (so every later entry of the bucket is in one of its columns)
+    # rule 1: a packet is either "spread" (its outliers sit in different columns) or "stack" (four
+    # outliers of one column); a stack is only formed while fewer than four columns have entries left
+    raw = packed.reshape(-1, 16)
     for bb in np.unique(b):
-        cols = n[b == bb].tolist()
-        for p0 in range(0, len(cols), 4):
-            pkt = cols[p0:p0 + 4]
-            assert pkt == sorted(pkt)
-            if len(set(pkt)) < len(pkt):
-                assert set(cols[p0 + 4:]) <= set(pkt)
+        t_, lb = divmod(int(bb), NB)
+        off, cnt = int(info[bb]) & 0xffff, int(info[bb]) >> 16
+        left = {}
+        for c in (n[b == bb] % BN).tolist():
+            left[c] = left.get(c, 0) + 1
+        for pk in raw[int(indptr[t_]) + off:int(indptr[t_]) + off + cnt]:
+            vals = pk[8:].view(np.uint16)
+            cols = [int(pk[4 + s_]) for s_ in range(4) if vals[s_] != 0]
+            assert len(cols) >= 1
+            if len(set(cols)) < len(cols):
+                assert len(cols) == 4 and len(set(cols)) == 1
+                assert sum(1 for v_ in left.values() if v_ > 0) < 4
+            else:
+                alive = sum(1 for v_ in left.values() if v_ > 0)
+                assert len(cols) == min(4, alive)
+            for c in cols:
+                left[c] -= 1
+        assert all(v_ == 0 for v_ in left.values())
     # rule 2 pays off: fewer shared-memory passes than the plain (column, row) order
     plain_pos = np.zeros(len(k), dtype=np.int64)
     for bb in np.unique(b):
@@ -169,7 +182,7 @@ def test_tilecoo_element_order_separates_columns_and_staggers_bank_groups():
     vv = (0x3F80 + np.arange(40)).astype(np.uint16)
     ip, bi, pk = fq.fq_encode_tilecoo(L, kk, nn, vv)
     k2, n2, v2 = fq.fq_decode_tilecoo(L, ip, bi, pk)
-    assert _as_set(k2, n2, v2) == _as_set(kk, nn, vv) and pk.shape[0] == 10
+    assert _as_set(k2, n2, v2) == _as_set(kk, nn, vv) and pk.shape[0] == 10          # ten stacks of four
 
 
 def test_tilecoo_edge_cases():

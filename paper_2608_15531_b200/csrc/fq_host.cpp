@@ -52,8 +52,9 @@ fq_status_t fq_get_layout(uint32_t K, uint32_t N, uint32_t group, uint32_t bn_hi
     if (BN != 128 && BN != 256) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "BN must be 128 or 256, got %u", BN);
     if (N == 0 || N % BN != 0) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "N = %u is not a multiple of BN = %u", N, BN);
     if (N / BN > kMaxTilesN) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "N = %u has too many column tiles", N);
-    uint32_t NB = nb_hint ? nb_hint : 64;
-    if (NB != 32 && NB != 64 && NB != 128) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "buckets per tile must be 32, 64 or 128, got %u", NB);
+    // one bucket per group of four columns {g, g + 8, g + 16, g + 24} of a 32-column block
+    const uint32_t NB = BN / 4;
+    if (nb_hint != 0 && nb_hint != NB) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "buckets per tile must be BN / 4 = %u, got %u", NB, nb_hint);
     std::memset(out, 0, sizeof(*out));
     out->abi = FQ_ABI_VERSION;
     out->K = K;
@@ -187,56 +188,10 @@ struct Encoded {
     uint32_t max_tile_packets = 0;
 };
 
-// Pack one bucket's entries (input sorted by column, then row) into packets of four slots.
-// A packet is one of two kinds, so that the kernel never needs to resolve a repeated column
-// inside a packet:
-//   "spread"  its real slots hold different columns (one entry from each of the up-to-four
-//             fullest columns that still have entries);
-//   "stack"   four entries of one column (used while fewer than four columns have entries left
-//             and one of them still has four or more).
-// Unused slots are padding.  Which entry of a column goes into slot position i of bucket b follows
-// the bank-group rotation of Section 3.2.2: prefer an entry whose activation row lies in bank
-// group (i + b) mod 4 (bank group of row k = k mod 4 for the kernel's 32-byte FP32 rows), else the
-// next group in circular order.  `out` receives 4 * packets entries; padding has v == 0.
-void pack_bucket(std::vector<Entry>& e, uint32_t b, uint32_t BN, std::vector<Entry>& out) {
-    struct Col { uint8_t c; std::vector<Entry> ent; };
-    std::vector<Col> cols;
-    for (const Entry& x : e) {
-        if (cols.empty() || cols.back().c != x.c) cols.push_back(Col{x.c, {}});
-        cols.back().ent.push_back(x);
-    }
-    out.clear();
-    size_t left = e.size();
-    auto take = [&](Col& col, size_t pos) {
-        const uint32_t want = (uint32_t)((pos + b) & 3);
-        size_t pick = 0;
-        uint32_t dist = 4;
-        for (size_t j = 0; j < col.ent.size(); ++j) {
-            uint32_t d = ((col.ent[j].k & 3u) + 4u - want) & 3u;
-            if (d < dist) { dist = d; pick = j; }
-        }
-        Entry r = col.ent[pick];
-        col.ent.erase(col.ent.begin() + pick);
-        --left;
-        return r;
-    };
-    while (left > 0) {
-        // columns that still have entries, fullest first (ties: lower column)
-        std::vector<size_t> alive;
-        for (size_t ci = 0; ci < cols.size(); ++ci)
-            if (!cols[ci].ent.empty()) alive.push_back(ci);
-        std::stable_sort(alive.begin(), alive.end(), [&](size_t x, size_t y) { return cols[x].ent.size() > cols[y].ent.size(); });
-        const size_t base = out.size();
-        if (alive.size() < 4 && cols[alive[0]].ent.size() >= 4) {
-            for (int sidx = 0; sidx < 4; ++sidx) out.push_back(take(cols[alive[0]], base + sidx));
-        } else {
-            const size_t nsl = std::min<size_t>(4, alive.size());
-            for (size_t sidx = 0; sidx < nsl; ++sidx) out.push_back(take(cols[alive[sidx]], base + sidx));
-            // padding: value 0, row 0, and a column byte that differs from slot to slot
-            for (size_t sidx = nsl; sidx < 4; ++sidx) out.push_back(Entry{0, (uint8_t)(BN - 1 - sidx), 0});
-        }
-    }
-}
+// Bucket of a tile column: the four columns {g, g + 8, g + 16, g + 24} of a 32-column block share
+// bucket 8 * (c / 32) + c % 8.  These are the columns whose accumulators one group of four lanes
+// holds in the small-batch kernel, so a bucket's outliers are applied in registers.
+inline uint32_t bucket_of(uint32_t c) { return ((c >> 5) << 3) | (c & 7u); }
 
 fq_status_t encode_impl(const fq_layout_t* L, const uint32_t* k, const uint32_t* n, const uint16_t* v,
                         size_t nnz, Encoded& E) {
@@ -261,58 +216,26 @@ fq_status_t encode_impl(const fq_layout_t* L, const uint32_t* k, const uint32_t*
             sorted[fill[t]++] = Entry{(uint8_t)(k[e] % FQ_BK), (uint8_t)(n[e] % BN), v[e]};
         }
     }
-    // pass 1: per tile, packets per bucket
+    // pass 1: per tile, the entries of every bucket in (row, column) order, four to a packet; the
+    // last packet of a bucket is filled up with padding slots (value 0, row 0, the bucket's first column)
     E.indptr.assign(ntile + 1, 0);
     E.info.assign(ntile * NB, 0);
-    std::vector<uint8_t> col2bucket(ntile * BN);
     std::vector<std::vector<Entry>> tile_slots(ntile);  // packed slots of every tile, four per packet
     int bad = 0;
 #pragma omp parallel for schedule(dynamic, 16)
     for (int64_t t = 0; t < (int64_t)ntile; ++t) {
-        uint32_t cnt[256] = {0};
-        for (size_t e = tstart[t]; e < tstart[t + 1]; ++e) ++cnt[sorted[e].c];
-        // Buckets come in blocks of 32 (one sparse warp each).  A column always belongs to block
-        // (column mod number-of-blocks), in every row tile, so that two warps working on different
-        // row tiles of the same column tile never touch the same output column.  Inside a block:
-        // columns by descending count (ties: lower column first), each to the least-loaded bucket
-        // (ties: lower bucket id) -- the greedy longest-processing-time rule.
-        const uint32_t nblk = NB / 32;
-        uint32_t load[128] = {0};
-        uint8_t* c2b = &col2bucket[(size_t)t * BN];
-        for (uint32_t blk = 0; blk < nblk; ++blk) {
-            uint32_t order[256], ncol = 0;
-            for (uint32_t c = blk; c < BN; c += nblk) order[ncol++] = c;
-            std::stable_sort(order, order + ncol, [&](uint32_t a, uint32_t b) { return cnt[a] > cnt[b]; });
-            typedef std::pair<uint32_t, uint32_t> LB;  // (load, bucket)
-            std::priority_queue<LB, std::vector<LB>, std::greater<LB>> heap;
-            for (uint32_t b = 0; b < 32; ++b) heap.push(LB(0, blk * 32 + b));
-            for (uint32_t i = 0; i < ncol; ++i) {
-                uint32_t c = order[i];
-                if (cnt[c] == 0) { c2b[c] = (uint8_t)(blk * 32); continue; }
-                LB top = heap.top();
-                heap.pop();
-                c2b[c] = (uint8_t)top.second;
-                load[top.second] += cnt[c];
-                heap.push(LB(top.first + cnt[c], top.second));
-            }
-        }
-        // pack every bucket of the tile now: the number of packets depends on the packing
         std::vector<std::vector<Entry>> per(NB);
-        for (size_t e = tstart[t]; e < tstart[t + 1]; ++e) per[c2b[sorted[e].c]].push_back(sorted[e]);
+        for (size_t e = tstart[t]; e < tstart[t + 1]; ++e) per[bucket_of(sorted[e].c)].push_back(sorted[e]);
         std::vector<Entry>& tp = tile_slots[t];
-        std::vector<Entry> slots;
         uint32_t off = 0;
         for (uint32_t b = 0; b < NB; ++b) {
-            uint32_t pk = 0;
-            if (!per[b].empty()) {
-                // deterministic input order: by column, then row
-                std::sort(per[b].begin(), per[b].end(), [](const Entry& x, const Entry& y) {
-                    return x.c != y.c ? x.c < y.c : x.k < y.k;
-                });
-                pack_bucket(per[b], b, BN, slots);
-                pk = (uint32_t)(slots.size() / 4);
-                tp.insert(tp.end(), slots.begin(), slots.end());
-            }
+            std::sort(per[b].begin(), per[b].end(), [](const Entry& x, const Entry& y) {
+                return x.k != y.k ? x.k < y.k : x.c < y.c;
+            });
+            const uint32_t pk = (uint32_t)((per[b].size() + 3) / 4);
+            tp.insert(tp.end(), per[b].begin(), per[b].end());
+            const uint8_t first_col = (uint8_t)(((b >> 3) << 5) | (b & 7u));
+            for (size_t i = per[b].size(); i < (size_t)pk * 4; ++i) tp.push_back(Entry{0, first_col, 0});
             if (off > 0xffffu || pk > 0xffffu) {
 #pragma omp atomic write
                 bad = 1;
@@ -426,28 +349,15 @@ fq_status_t fq_validate_tilecoo(const fq_layout_t* L, const uint32_t* indptr, co
         if (indptr[t + 1] < indptr[t]) return fail(FQ_ERR_FORMAT, "tile_indptr decreases at tile %zu", t);
         const uint32_t tile_pk = indptr[t + 1] - indptr[t];
         if ((size_t)indptr[t + 1] > n_packets) return fail(FQ_ERR_FORMAT, "tile %zu ends at packet %u of %zu", t, indptr[t + 1], n_packets);
-        int16_t owner[256];
-        for (uint32_t c = 0; c < BN; ++c) owner[c] = -1;
         for (uint32_t b = 0; b < NB; ++b) {
             uint32_t off = info[t * NB + b] & 0xffffu, cnt = info[t * NB + b] >> 16;
             if (off + cnt > tile_pk) return fail(FQ_ERR_FORMAT, "bucket %u of tile %zu covers packets [%u, %u) of %u", b, t, off, off + cnt, tile_pk);
             for (uint32_t i = 0; i < cnt; ++i) {
                 const uint8_t* p = pk + (size_t)(indptr[t] + off + i) * 16;
-                // real slots of a packet: all in different columns, or four in one column
-                int nlive = 0, ndiff = 0;
                 for (int s = 0; s < 4; ++s) {
-                    if ((p[8 + 2 * s] | p[9 + 2 * s]) == 0) continue;
-                    ++nlive;
-                    for (int s2 = 0; s2 < s; ++s2)
-                        if ((p[8 + 2 * s2] | p[9 + 2 * s2]) != 0 && p[4 + s2] == p[4 + s]) ++ndiff;
-                }
-                if (ndiff != 0 && !(nlive == 4 && ndiff == 6)) return fail(FQ_ERR_FORMAT, "packet %u of tile %zu mixes repeated and distinct columns", indptr[t] + off + i, t);
-                for (int s = 0; s < 4; ++s) {
-                    if ((p[8 + 2 * s] | p[9 + 2 * s]) == 0) continue;  // padding slot
                     if (p[s] >= FQ_BK || p[4 + s] >= BN) return fail(FQ_ERR_FORMAT, "index (%u, %u) outside the tile in tile %zu", p[s], p[4 + s], t);
-                    if (p[4 + s] % (NB / 32) != b / 32) return fail(FQ_ERR_FORMAT, "column %u of tile %zu sits in bucket %u, outside its block of 32 buckets", p[4 + s], t, b);
-                    if (owner[p[4 + s]] >= 0 && owner[p[4 + s]] != (int16_t)b) return fail(FQ_ERR_FORMAT, "column %u of tile %zu appears in buckets %d and %u", p[4 + s], t, owner[p[4 + s]], b);
-                    owner[p[4 + s]] = (int16_t)b;
+                    if ((p[8 + 2 * s] | p[9 + 2 * s]) == 0) continue;  // padding slot
+                    if (bucket_of(p[4 + s]) != b) return fail(FQ_ERR_FORMAT, "column %u of tile %zu sits in bucket %u, not in its own bucket %u", p[4 + s], t, b, bucket_of(p[4 + s]));
                 }
             }
         }

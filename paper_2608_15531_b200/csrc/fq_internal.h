@@ -30,8 +30,8 @@ inline bool layout_ok(const fq_layout_t* L) {
 
 // Upper bound on persistent CTAs per launch; sizes the scratch independently of the device.
 constexpr uint32_t kMaxCtas = 192;
-constexpr uint32_t kMaxTilesN = 2048;       // tile-arrival counters in the scratch
+constexpr uint32_t kMaxTilesN = 1024;       // column tiles; the scratch holds 8 arrival counters for each
 constexpr size_t kWsHeaderBytes = 256;      // status word lives at offset 0
-constexpr size_t kWsCounterBytes = kMaxTilesN * 4;
+constexpr size_t kWsCounterBytes = kMaxTilesN * 8 * 4;
 
 }  // namespace fq

@@ -72,7 +72,6 @@ struct Params {
     float* partials;
     uint32_t M, K, N, KT, NT;
     uint32_t NB, coo_cap, stages, nsw;
-    uint32_t shc_floats;   // small-batch kernel: floats of the FP32 outlier tile(s) to clear at start
     // shared-memory offsets (bytes); the first five are relative to a stage
     uint32_t stage_bytes, off_sz, off_xcan, off_xsum, off_info, off_coo;
     uint32_t off_shc, off_xt, off_bar;
@@ -271,162 +270,47 @@ __device__ __forceinline__ void fma8(float4& c0, float4& c1, float v, const floa
 }
 
 // One packet (four outliers) against the k-major FP32 activation copy xt ([128][8] floats, 32 B per
-// row k): row c of the FP32 tile += v * x[8o..8o+7][k] for each slot (Section 4.2, without the
-// per-column padding: every slot carries its own column byte).  The encoder emits two kinds of
-// packets: "spread" (real slots in different columns: all loads are issued before the first store,
-// padding slots, value 0, are skipped) and "stack" (four outliers of one column: summed in registers,
-// one read-modify-write).
+// row k): row c of the FP32 tile += v * x[8o..8o+7][k], slot after slot (Section 4.2, without the
+// per-column padding: every slot carries its own column byte).  Slots of one packet may repeat a
+// column, so each slot finishes its read-modify-write before the next one starts; the activation
+// rows of all four are loaded first.  Padding slots (value 0) are skipped.
 template <int Q>
 __device__ __forceinline__ void apply_packet(const uint4 pk, const float* __restrict__ xt, float* shc, uint32_t o, uint32_t ldc) {
-    uint32_t k[4], c[4];
     float v[4];
-#pragma unroll
-    for (int s = 0; s < 4; ++s) {
-        k[s] = (pk.x >> (8 * s)) & 0xffu;
-        c[s] = (pk.y >> (8 * s)) & 0xffu;
-    }
     v[0] = bf16lo(pk.z); v[1] = bf16hi(pk.z); v[2] = bf16lo(pk.w); v[3] = bf16hi(pk.w);
-    const bool live0 = (pk.z & 0xffffu) != 0, live1 = (pk.z >> 16) != 0, live2 = (pk.w & 0xffffu) != 0, live3 = (pk.w >> 16) != 0;
-    const bool live[4] = {live0, live1, live2, live3};
     float4 x0[4], x1[4];
 #pragma unroll
     for (int s = 0; s < 4; ++s) {
-        const float4* xp = reinterpret_cast<const float4*>(xt + k[s] * 8);
+        const float4* xp = reinterpret_cast<const float4*>(xt + ((pk.x >> (8 * s)) & 0xffu) * 8);
         x0[s] = xp[0];
         x1[s] = xp[1];
     }
-    const bool stack = pk.y == __byte_perm(pk.y, 0, 0x0000) && live0 && live1 && live2 && live3;
-    if (!stack) {
-        float4 c0[4], c1[4];
 #pragma unroll
-        for (int s = 0; s < 4; ++s) {
-            c0[s] = c1[s] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-            if (live[s]) {
-                c0[s] = *reinterpret_cast<const float4*>(shc + shc_quad<Q>(c[s], 2 * o, ldc));
-                c1[s] = *reinterpret_cast<const float4*>(shc + shc_quad<Q>(c[s], 2 * o + 1, ldc));
-            }
-        }
-#pragma unroll
-        for (int s = 0; s < 4; ++s) fma8(c0[s], c1[s], v[s], x0[s], x1[s]);
-#pragma unroll
-        for (int s = 0; s < 4; ++s) {
-            if (live[s]) {
-                *reinterpret_cast<float4*>(shc + shc_quad<Q>(c[s], 2 * o, ldc)) = c0[s];
-                *reinterpret_cast<float4*>(shc + shc_quad<Q>(c[s], 2 * o + 1, ldc)) = c1[s];
-            }
-        }
-    } else {
-        float4* p0 = reinterpret_cast<float4*>(shc + shc_quad<Q>(c[0], 2 * o, ldc));
-        float4* p1 = reinterpret_cast<float4*>(shc + shc_quad<Q>(c[0], 2 * o + 1, ldc));
-        float4 c0 = *p0, c1 = *p1;
-#pragma unroll
-        for (int s = 0; s < 4; ++s) fma8(c0, c1, v[s], x0[s], x1[s]);
-        *p0 = c0;
-        *p1 = c1;
-    }
-}
-
-// ---- narrow-batch form (M <= 8): rows of MS = 1, 2, 4 or 8 floats, so that M = 1 moves 4 bytes per
-// outlier instead of 32.  Row pitch in floats: MS, except 12 for MS = 8 (a 48-byte pitch spreads
-// random rows over all eight 16-byte bank groups; a 32-byte pitch would use only four).
-__host__ __device__ constexpr int ms_pitch(int ms) { return ms == 8 ? 12 : ms; }
-
-template <int MS>
-__device__ __forceinline__ void ld_row(const float* p, float (&r)[MS]) {
-    if constexpr (MS == 1) { r[0] = *p; }
-    else if constexpr (MS == 2) { const float2 v = *reinterpret_cast<const float2*>(p); r[0] = v.x; r[1] = v.y; }
-    else {
-#pragma unroll
-        for (int i = 0; i < MS / 4; ++i) {
-            const float4 v = reinterpret_cast<const float4*>(p)[i];
-            r[4 * i] = v.x; r[4 * i + 1] = v.y; r[4 * i + 2] = v.z; r[4 * i + 3] = v.w;
+    for (int s = 0; s < 4; ++s) {
+        if (v[s] != 0.0f) {
+            const uint32_t c = (pk.y >> (8 * s)) & 0xffu;
+            float4* p0 = reinterpret_cast<float4*>(shc + shc_quad<Q>(c, 2 * o, ldc));
+            float4* p1 = reinterpret_cast<float4*>(shc + shc_quad<Q>(c, 2 * o + 1, ldc));
+            float4 c0 = *p0, c1 = *p1;
+            fma8(c0, c1, v[s], x0[s], x1[s]);
+            *p0 = c0;
+            *p1 = c1;
         }
     }
-}
-template <int MS>
-__device__ __forceinline__ void st_row(float* p, const float (&r)[MS]) {
-    if constexpr (MS == 1) { *p = r[0]; }
-    else if constexpr (MS == 2) { *reinterpret_cast<float2*>(p) = make_float2(r[0], r[1]); }
-    else {
-#pragma unroll
-        for (int i = 0; i < MS / 4; ++i) reinterpret_cast<float4*>(p)[i] = make_float4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
-    }
-}
-
-// A decoded packet with its activation rows loaded (narrow form).  col[s] is the row of the FP32
-// tile that slot s updates: its column, or this lane's dummy row (index `dummy`, past the tile) for a
-// padding slot and for slots 1..3 of a stack packet (four outliers of one column, folded into slot
-// 0).  With the dummy row every slot does the same loads and stores: no branch depends on the data.
-template <int MS>
-struct NarrowPacket {
-    uint32_t col[4];
-    float v[4];
-    float x[4][MS];
-    bool stack;
-};
-
-template <int MS>
-__device__ __forceinline__ void narrow_fetch(NarrowPacket<MS>& t, const uint4 pk, const float* xt, uint32_t dummy) {
-    constexpr int P = ms_pitch(MS);
-#pragma unroll
-    for (int s = 0; s < 4; ++s) ld_row<MS>(xt + ((pk.x >> (8 * s)) & 0xffu) * P, t.x[s]);
-    t.v[0] = bf16lo(pk.z); t.v[1] = bf16hi(pk.z); t.v[2] = bf16lo(pk.w); t.v[3] = bf16hi(pk.w);
-    const bool l0 = (pk.z & 0xffffu) != 0, l1 = (pk.z >> 16) != 0, l2 = (pk.w & 0xffffu) != 0, l3 = (pk.w >> 16) != 0;
-    t.stack = pk.y == __byte_perm(pk.y, 0, 0x0000) && l0 && l1 && l2 && l3;
-    t.col[0] = l0 ? (pk.y & 0xffu) : dummy;
-    t.col[1] = (l1 && !t.stack) ? ((pk.y >> 8) & 0xffu) : dummy;
-    t.col[2] = (l2 && !t.stack) ? ((pk.y >> 16) & 0xffu) : dummy;
-    t.col[3] = (l3 && !t.stack) ? (pk.y >> 24) : dummy;
-}
-
-// Loads of the FP32 rows, then the FMAs; the stores are a separate step so that the caller can issue
-// the next packet's loads between them.
-template <int MS>
-__device__ __forceinline__ void narrow_accumulate(const NarrowPacket<MS>& t, const float* shc, float (&a)[4][MS]) {
-    constexpr int P = ms_pitch(MS);
-#pragma unroll
-    for (int s = 0; s < 4; ++s) ld_row<MS>(shc + t.col[s] * P, a[s]);
-#pragma unroll
-    for (int s = 1; s < 4; ++s)
-#pragma unroll
-        for (int i = 0; i < MS; ++i) {
-            const float c = t.v[s] * t.x[s][i];
-            a[s][i] += c;
-            a[0][i] += t.stack ? c : 0.0f;
-        }
-#pragma unroll
-    for (int i = 0; i < MS; ++i) a[0][i] = fmaf(t.v[0], t.x[0][i], a[0][i]);
-}
-template <int MS>
-__device__ __forceinline__ void narrow_store(const NarrowPacket<MS>& t, float* shc, const float (&a)[4][MS]) {
-    constexpr int P = ms_pitch(MS);
-    // slots that share the dummy row overwrite one another there: nothing reads it
-#pragma unroll
-    for (int s = 3; s >= 0; --s) st_row<MS>(shc + t.col[s] * P, a[s]);
 }
 
 // Transpose one octet of BF16 activation rows into the FP32 k-major copy xt[k][8] (32 B per k).
 // `row0` is the shared-memory address of row 0 / 16-byte chunk 0 of the octet, rows `row_step`
 // bytes apart, consecutive 16-byte chunks (8 k each) `chunk_step` bytes apart.  Whole warp.
-// `pitch` floats per k in xt; only the first `ms` rows of the octet are written (ms = 1, 2, 4, 8).
-__device__ __forceinline__ void transpose_octet_f32(uint32_t row0, uint32_t row_step, uint32_t chunk_step, float* xt, int lane,
-                                                    uint32_t pitch = 8, uint32_t ms = 8) {
+__device__ __forceinline__ void transpose_octet_f32(uint32_t row0, uint32_t row_step, uint32_t chunk_step, float* xt, int lane) {
 #pragma unroll
     for (int kb = 0; kb < 4; ++kb) {
         uint32_t r[4];
         ldmatrix_x4_trans(row0 + (lane & 7) * row_step + (kb * 4 + (lane >> 3)) * chunk_step, r[0], r[1], r[2], r[3]);
         // thread T holds rows m = 2(T%4), 2(T%4)+1 of column k = 8*block + T/4
-        const uint32_t m0 = (lane & 3) * 2;
-        float* dst = xt + ((kb * 32) + (lane >> 2)) * pitch + m0;
-        if (ms >= 2) {
-            if (m0 < ms) {
+        float* dst = xt + ((kb * 32) + (lane >> 2)) * 8 + (lane & 3) * 2;
 #pragma unroll
-                for (int i = 0; i < 4; ++i) *reinterpret_cast<float2*>(dst + i * 8 * pitch) = make_float2(bf16lo(r[i]), bf16hi(r[i]));
-            }
-        } else if (m0 == 0) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) dst[i * 8 * pitch] = bf16lo(r[i]);
-        }
+        for (int i = 0; i < 4; ++i) *reinterpret_cast<float2*>(dst + i * 64) = make_float2(bf16lo(r[i]), bf16hi(r[i]));
     }
 }
 
@@ -587,7 +471,12 @@ __global__ void __launch_bounds__(32 * (4 + 2 * (BN / 32) + 4), 1) fq_fused_kern
 #pragma unroll
             for (int c = 0; c < CPL; ++c) {
                 nxt[c] = make_uint4(0, 0, 0, 0);
-                if (real) nxt[c] = __ldg(reinterpret_cast<const uint4*>(xrow + (size_t)kt * 256 + c * 16));
+#if defined(FQ_EXP) && FQ_EXP == 11
+                if (false)
+#else
+                if (real)
+#endif
+                    nxt[c] = __ldg(reinterpret_cast<const uint4*>(xrow + (size_t)kt * 256 + c * 16));
             }
         };
         if (u_begin < u_end) load(u_begin - (u_begin / KT) * KT);
@@ -862,62 +751,51 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+constexpr int kActWarps = 2;   // activation warps of the small-batch kernel
 constexpr int kXPitch = 320;   // activation row in shared memory: 256 B + 64 B, conflict-free 16-byte fragment loads
 
 // The same operator for M <= 8 per octet (MO octets of batch rows): every dense warp runs the same
-// short loop (one 16-column strip per warp, warp-level m16n8k16 MMAs with the weights on the M side
-// and the batch on the N side), so the instruction stream of 16 of the CTA's warps is shared and
-// stays in the instruction cache.  Same packed formats, same producer, same sparse warps, same
-// split-tile protocol as the tcgen05 kernel; only the dense engine differs.
+// short loop (one 32-column strip per warp, warp-level m16n8k16 MMAs with the weights on the M side
+// and the batch on the N side), so the instruction stream of the CTA's dense warps is shared and
+// stays in the instruction cache.  Same packed formats, same producer, same split-tile protocol as
+// the tcgen05 kernel; the dense engine differs, and the outliers need no warps of their own:
 //   warp 0            producer (bulk copies)
 //   warp 1            activations: X block -> row-major shared-memory rows + per-group row sums
-//   warps 2..2+BN/16  dense: lane (g, t) loads word t of columns g and g+8 of each 32-row block:
-//                     8 codes = this lane's share of two k16 steps (the k order inside a block
-//                     follows the 16-byte activation loads of the lanes)
-//   then              sparse warps
+//                     + an FP32 k-major copy for the outlier step
+//   warps 2..2+BN/32  dense + outliers.  Lane (g, t) of warp w holds the accumulators of columns
+//                     32w + {g, g+8, g+16, g+24}, batch rows 2t, 2t+1 (+8 per octet).  Dense: the
+//                     lane loads word t of its columns of each 32-row block: 8 codes = its share
+//                     of two k16 steps (the k order inside a block follows the 16-byte activation
+//                     loads of the lanes).  Outliers: those four columns are one Tile-COO bucket, so
+//                     the four lanes of group g walk that bucket's packets and add v * x[row][k]
+//                     straight into their accumulators (Section 4.2 without the shared-memory
+//                     scatter: no atomics, no read-modify-write, no merge step).
 template <int BN, int MO, int GROUP, bool SPARSE>
-__global__ void __launch_bounds__(32 * (2 + BN / 16 + 6), 1) fq_mma_kernel(const Params p) {
-    constexpr int NDW = BN / 16;
+__global__ void __launch_bounds__(32 * (1 + kActWarps + BN / 32), 1) fq_mma_kernel(const Params p) {
+    constexpr int NDW = BN / 32;
+    constexpr int NA = kActWarps;                           // activation warps: warp a takes the units it with it mod NA == a
+    constexpr int DW0 = 1 + NA;                             // first dense warp
+    constexpr int CG = 2;                                   // 16-column MMA strips per warp
     constexpr int GPS = kBK / GROUP;
     constexpr int W_BYTES = 16 * BN * 4;
     constexpr int SZ_ROW = BN * 2;
     constexpr int LDC = 8 * MO;
-    constexpr int Q = (LDC == 8) ? 0 : LDC / 4;
     extern __shared__ __align__(128) uint8_t smem[];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     FQ_GT(tid == 0, 0);
     const uint32_t S = p.stages;
-    // rows kept per outlier in the one-octet form: the batch rounded up to 1, 2, 4 or 8
-    const uint32_t ms = p.M <= 1 ? 1u : p.M <= 2 ? 2u : p.M <= 4 ? 4u : 8u;
-    const uint32_t msp = ms_pitch(ms);
-    // one-octet form: the sparse warps split the units between them (a warp owns fixed stages) and each
-    // replica has its own FP32 tile of BN columns + one dummy row per lane
-    const uint32_t shc_copy = (BN + 32) * msp;
-    const uint32_t n_rep = (SPARSE && MO == 1) ? p.nsw / (p.NB >> 5) : 1u;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
     const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * S;
-    const uint32_t bar_sparse_done = bar_empty + 8 * S, bar_dense_done = bar_sparse_done + 8, bar_dense = bar_dense_done + 8;
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 2 * S + 4);
-    volatile uint32_t* last_flag = abort_flag + 1;
-    float* shc = reinterpret_cast<float*>(smem + p.off_shc);
 
-    const uint32_t nsw = SPARSE ? p.nsw : 0;
     if (tid == 0) {
         for (uint32_t s = 0; s < S; ++s) {
             mbar_init(bar_full + 8 * s, 2);   // producer's expect_tx arrival + activation warp
-            // one-octet form: each stage has one sparse warp per block of 32 buckets (fixed owner)
-            mbar_init(bar_empty + 8 * s, NDW + (MO == 1 ? (SPARSE ? p.NB >> 5 : 0u) : nsw));
+            mbar_init(bar_empty + 8 * s, NDW);
         }
-        mbar_init(bar_sparse_done, nsw ? nsw : 1);
-        mbar_init(bar_dense_done, NDW);
-        mbar_init(bar_dense, NDW);
         *abort_flag = 0;
-        *last_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (SPARSE) {
-        for (uint32_t i = tid; i < p.shc_floats; i += blockDim.x) shc[i] = 0.0f;
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncthreads();
@@ -945,18 +823,42 @@ __global__ void __launch_bounds__(32 * (2 + BN / 16 + 6), 1) fq_mma_kernel(const
                 npk = __shfl_sync(0xffffffffu, ip_b, it & 31) - pk0;
                 npk = min(npk, p.coo_cap);
             }
+#ifdef FQ_TRACE
+            long long tw0 = clock64();
+#endif
             if (!warp_wait(bar_empty + 8 * s, ph ^ 1, abort_flag, p.status)) { ok = false; break; }
+#ifdef FQ_TRACE
+            if (blockIdx.x == 0 && lane == 0) { g_trace[8] += clock64() - tw0; g_trace[9] += 1; }
+#endif
             const uint32_t tn = w.tn, kt = w.kt;
             const uint32_t full = bar_full + 8 * s;
             const uint32_t st = smem_u32(smem) + s * p.stage_bytes;
             if (lane == 0) {
+#if defined(FQ_EXP) && FQ_EXP == 25
+                uint32_t bytes = W_BYTES;
+#else
                 uint32_t bytes = W_BYTES + 2 * GPS * SZ_ROW;
+#endif
                 if (SPARSE) bytes += p.NB * 4 + npk * 16;
                 mbar_arrive_expect_tx(full, bytes);
             }
             __syncwarp();
+#ifdef FQ_WSPLIT
+            if (lane < FQ_WSPLIT) {
+                constexpr int PART = W_BYTES / FQ_WSPLIT;
+                bulk_g2s(st + lane * PART, p.wq + (size_t)u * W_BYTES + lane * PART, PART, full);
+            } else if (lane < FQ_WSPLIT + 2 * GPS) {
+                const int i = lane - FQ_WSPLIT, gi = i >> 1;
+                const size_t row = (size_t)(kt * GPS + gi) * p.N + (size_t)tn * BN;
+                if (i & 1) bulk_g2s(st + p.off_sz + (GPS + gi) * SZ_ROW, p.zero + row, SZ_ROW, full);
+                else bulk_g2s(st + p.off_sz + gi * SZ_ROW, p.scale + row, SZ_ROW, full);
+            } else if (lane == 31) {
+#else
             if (lane == 0) {
                 bulk_g2s(st, p.wq + (size_t)u * W_BYTES, W_BYTES, full);
+#if defined(FQ_EXP) && FQ_EXP == 25
+                if (false)
+#endif
 #pragma unroll
                 for (int gi = 0; gi < GPS; ++gi) {
                     const size_t row = (size_t)(kt * GPS + gi) * p.N + (size_t)tn * BN;
@@ -964,6 +866,7 @@ __global__ void __launch_bounds__(32 * (2 + BN / 16 + 6), 1) fq_mma_kernel(const
                     bulk_g2s(st + p.off_sz + (GPS + gi) * SZ_ROW, p.zero + row, SZ_ROW, full);
                 }
             } else if (lane == 1) {
+#endif
                 if (SPARSE) {
                     bulk_g2s(st + p.off_info, p.info + (size_t)u * p.NB, p.NB * 4, full);
                     if (npk) bulk_g2s(st + p.off_coo, p.packed + pk0, npk * 16, full);
@@ -975,8 +878,9 @@ __global__ void __launch_bounds__(32 * (2 + BN / 16 + 6), 1) fq_mma_kernel(const
             for (uint32_t j = (issued > S ? issued - S : 0); j < issued; ++j)
                 for (uint32_t spin = 0; spin < (1u << 20) && !mbar_try_wait(bar_full + 8 * (j % S), (j / S) & 1); ++spin) {}
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ activation warp
+    } else if (warp < DW0) {
+        // ------------------------------------------------------------------ activation warps
+        const uint32_t aw = warp - 1;
         // lane -> (row m, part): 16-byte chunks of that row; rows beyond M are zero
         constexpr int ROWS = 8 * MO;
         constexpr int LPR = 32 / ROWS;                       // lanes per row: 4 (8 rows) or 2 (16 rows)
@@ -989,18 +893,30 @@ __global__ void __launch_bounds__(32 * (2 + BN / 16 + 6), 1) fq_mma_kernel(const
 #pragma unroll
             for (int c = 0; c < CPL; ++c) {
                 nxt[c] = make_uint4(0, 0, 0, 0);
-                if (real) nxt[c] = __ldg(reinterpret_cast<const uint4*>(xrow + (size_t)kt * 256 + c * 16));
+#if defined(FQ_EXP) && FQ_EXP == 11
+                if (false)
+#else
+                if (real)
+#endif
+                    nxt[c] = __ldg(reinterpret_cast<const uint4*>(xrow + (size_t)kt * 256 + c * 16));
             }
         };
-        if (u_begin < u_end) load(u_begin - (u_begin / KT) * KT);
+        if (u_begin + aw < u_end) load((u_begin + aw) % KT);
         for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
+            if (w.it % NA != aw) continue;
             const uint32_t s = w.s, ph = w.ph;
             uint8_t* st = smem + s * p.stage_bytes;
             uint4 xv[CPL];
 #pragma unroll
             for (int c = 0; c < CPL; ++c) xv[c] = nxt[c];
-            if (w.u + 1 < u_end) load(w.kt + 1 == KT ? 0u : w.kt + 1);
+            if (w.u + NA < u_end) { uint32_t kn = w.kt + NA; load(kn >= KT ? kn % KT : kn); }   // this warp's next unit
+#ifdef FQ_TRACE
+            long long tw0 = clock64();
+#endif
             if (!warp_wait(bar_empty + 8 * s, ph ^ 1, abort_flag, p.status)) break;
+#ifdef FQ_TRACE
+            long long tw1 = clock64();
+#endif
             uint8_t* dst = st + p.off_xcan + m * kXPitch + part * CPL * 16;
             float sum = 0.0f;
 #pragma unroll
@@ -1024,282 +940,275 @@ __global__ void __launch_bounds__(32 * (2 + BN / 16 + 6), 1) fq_mma_kernel(const
             }
             __syncwarp();
             if (SPARSE) {
-                // FP32 k-major copy for the sparse warps, one octet of rows at a time
-                if (MO == 1) {
-                    transpose_octet_f32(smem_u32(st + p.off_xcan), kXPitch, 16, reinterpret_cast<float*>(st + p.off_xt), lane, msp, ms);
-                } else {
-                    for (uint32_t o = 0; o < ((p.M + 7) >> 3); ++o)
-                        transpose_octet_f32(smem_u32(st + p.off_xcan) + o * 8 * kXPitch, kXPitch, 16,
-                                            reinterpret_cast<float*>(st + p.off_xt) + o * 1024, lane);
-                }
+                // FP32 k-major copy [octet][k][8] for the outlier step
+#pragma unroll
+                for (int o = 0; o < MO; ++o)
+                    transpose_octet_f32(smem_u32(st + p.off_xcan) + o * 8 * kXPitch, kXPitch, 16,
+                                        reinterpret_cast<float*>(st + p.off_xt) + o * 1024, lane);
                 __syncwarp();
             }
             if (lane == 0) mbar_arrive(bar_full + 8 * s);
+#ifdef FQ_TRACE
+            if (blockIdx.x == 0 && lane == 0 && aw == 0) { g_trace[10] += tw1 - tw0; g_trace[11] += clock64() - tw1; g_trace[12] += 1; }
+#endif
         }
-    } else if (warp >= 2 && warp < 2 + NDW) {
+    } else if (warp >= DW0 && warp < DW0 + NDW) {
         // ------------------------------------------------------------------ dense warps (all alike)
-        const int dw = warp - 2, g = lane >> 2, t = lane & 3;
-        const int dtid = dw * 32 + lane;
-        const int c0 = dw * 16 + g;                           // this lane's columns: c0 and c0 + 8
-        float accf[MO][4];
+        const int dw = warp - DW0, g = lane >> 2, t = lane & 3;
+        [[maybe_unused]] const int dtid = dw * 32 + lane;   // tracing builds only
+        const int c0 = dw * 32 + g;                           // this lane's columns: c0 + 8 * {0, 1, 2, 3}
+        float accf[MO][CG][4];
 #pragma unroll
         for (int o = 0; o < MO; ++o)
 #pragma unroll
-            for (int i = 0; i < 4; ++i) accf[o][i] = 0.0f;
-        uint32_t piece = 0, dense_phase = 0;
+            for (int cg = 0; cg < CG; ++cg)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) accf[o][cg][i] = 0.0f;
+        uint32_t piece = 0;
         bool ok = true;
         for (UnitIter w(u_begin, KT); w.u < u_end && ok; w.next(S, KT)) {
             const uint32_t u = w.u, s = w.s, ph = w.ph, tn = w.tn, kt = w.kt;
             const uint8_t* st = smem + s * p.stage_bytes;
+#ifdef FQ_TRACE
+            long long tw0 = clock64();
+#endif
             if (!warp_wait(bar_full + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
+#ifdef FQ_TRACE
+            long long tw1 = clock64();
+#endif
             FQ_GT(dtid == 0 && w.it == 0, 2);
             const uint32_t* wp = reinterpret_cast<const uint32_t*>(st) + c0 * 4 + t;
             const uint8_t* xrow = st + p.off_xcan + g * kXPitch + t * 16;
             const uint16_t* sc = reinterpret_cast<const uint16_t*>(st + p.off_sz);
             const float* xsum = reinterpret_cast<const float*>(st + p.off_xsum);
-#if defined(FQ_EXP) && FQ_EXP == 7
+            // outliers: bucket descriptor, first two packets and the first packet's activation rows are
+            // requested now and used after the dense math of the unit
+            uint32_t sp_off = 0, sp_cnt = 0, cmax = 0;
+            const uint4* pk_s = reinterpret_cast<const uint4*>(st + p.off_coo);
+            const uint4* pk_g = nullptr;
+            const float* xt = reinterpret_cast<const float*>(st + p.off_xt) + 2 * t;
+            auto packet = [&](uint32_t i) {
+                uint4 pk = make_uint4(0, 0, 0, 0);            // beyond the bucket's list: four padding slots
+                if (i < sp_cnt) {
+                    const uint32_t idx = sp_off + i;
+                    pk = (idx < p.coo_cap) ? pk_s[idx] : __ldg(pk_g + idx);
+                }
+                return pk;
+            };
+            auto fetch_x = [&](const uint4 pk, float2 (&x2)[4][MO]) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+#pragma unroll
+                    for (int o = 0; o < MO; ++o)
+                        x2[e][o] = *reinterpret_cast<const float2*>(xt + o * 1024 + ((pk.x >> (8 * e)) & 0xffu) * 8);
+            };
+            uint4 pk0 = make_uint4(0, 0, 0, 0), pk1 = pk0;
+            float2 xa[4][MO];
+            if (SPARSE) {
+                const uint32_t info = reinterpret_cast<const uint32_t*>(st + p.off_info)[dw * 8 + g];
+                sp_off = info & 0xffffu;
+                sp_cnt = info >> 16;
+                if (sp_off + sp_cnt > p.coo_cap) pk_g = p.packed + __ldg(p.indptr + u);   // packets beyond the staged part
+                cmax = __reduce_max_sync(0xffffffffu, sp_cnt);
+                pk0 = packet(0);
+                pk1 = packet(1);
+                fetch_x(pk0, xa);
+            }
+#if defined(FQ_EXP) && (FQ_EXP == 24 || FQ_EXP == 25)
             if (false)
 #endif
 #pragma unroll
             for (int gi = 0; gi < GPS; ++gi) {
-                float accg[MO][4];
+                float accg[MO][CG][4];
 #pragma unroll
                 for (int o = 0; o < MO; ++o)
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) accg[o][i] = 0.0f;
+                    for (int cg = 0; cg < CG; ++cg)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) accg[o][cg][i] = 0.0f;
 #pragma unroll
                 for (int j = gi * (4 / GPS); j < (gi + 1) * (4 / GPS); ++j) {
-                    const uint32_t wa = wp[j * BN * 4], wb = wp[j * BN * 4 + 32];     // columns c0 and c0 + 8
-                    const uint32_t a0 = codes_to_bf16x2(wa), a1 = codes_to_bf16x2(wa >> 4);
-                    const uint32_t a2 = codes_to_bf16x2(wa >> 8), a3 = codes_to_bf16x2(wa >> 12);
-                    const uint32_t b0 = codes_to_bf16x2(wb), b1 = codes_to_bf16x2(wb >> 4);
-                    const uint32_t b2 = codes_to_bf16x2(wb >> 8), b3 = codes_to_bf16x2(wb >> 12);
+                    uint4 xb[MO];
 #pragma unroll
-                    for (int o = 0; o < MO; ++o) {
-                        const uint4 xb = *reinterpret_cast<const uint4*>(xrow + o * 8 * kXPitch + j * 64);
-                        mma_bf16(accg[o], a0, b0, a1, b1, xb.x, xb.y);   // rows 8t+0..3 of the block
-                        mma_bf16(accg[o], a2, b2, a3, b3, xb.z, xb.w);   // rows 8t+4..7
+                    for (int o = 0; o < MO; ++o) xb[o] = *reinterpret_cast<const uint4*>(xrow + o * 8 * kXPitch + j * 64);
+#pragma unroll
+                    for (int cg = 0; cg < CG; ++cg) {
+                        const uint32_t wa = wp[j * BN * 4 + cg * 64], wb = wp[j * BN * 4 + cg * 64 + 32];   // columns +0 and +8
+#if defined(FQ_EXP) && FQ_EXP == 22
+                        const uint32_t a0 = wa, a1 = wa ^ 1, a2 = wa ^ 2, a3 = wa ^ 3, b0 = wb, b1 = wb ^ 1, b2 = wb ^ 2, b3 = wb ^ 3;
+#else
+                        const uint32_t a0 = codes_to_bf16x2(wa), a1 = codes_to_bf16x2(wa >> 4);
+                        const uint32_t a2 = codes_to_bf16x2(wa >> 8), a3 = codes_to_bf16x2(wa >> 12);
+                        const uint32_t b0 = codes_to_bf16x2(wb), b1 = codes_to_bf16x2(wb >> 4);
+                        const uint32_t b2 = codes_to_bf16x2(wb >> 8), b3 = codes_to_bf16x2(wb >> 12);
+#endif
+#pragma unroll
+                        for (int o = 0; o < MO; ++o) {
+#if defined(FQ_EXP) && FQ_EXP == 21
+                            accg[o][cg][0] += __uint_as_float((a0 ^ b0 ^ a1 ^ b1 ^ xb[o].x ^ xb[o].y) & 0x3fffffffu);
+                            accg[o][cg][1] += __uint_as_float((a2 ^ b2 ^ a3 ^ b3 ^ xb[o].z ^ xb[o].w) & 0x3fffffffu);
+#else
+                            mma_bf16(accg[o][cg], a0, b0, a1, b1, xb[o].x, xb[o].y);   // rows 8t+0..3 of the block
+                            mma_bf16(accg[o][cg], a2, b2, a3, b3, xb[o].z, xb[o].w);   // rows 8t+4..7
+#endif
+                        }
                     }
                 }
                 // once per group: acc += s * (sum x (128+q) - (128+z) sum x)     (Eq. 3 inside Eq. 1)
+                float2 xs[MO];
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const float sv = bf16_bits_to_float(sc[gi * BN + c0 + 8 * h]);
-                    const float zc = -(128.0f + bf16_bits_to_float(sc[(GPS + gi) * BN + c0 + 8 * h]));
+                for (int o = 0; o < MO; ++o) xs[o] = *reinterpret_cast<const float2*>(xsum + gi * LDC + o * 8 + 2 * t);
+#if defined(FQ_EXP) && FQ_EXP == 23
 #pragma unroll
-                    for (int o = 0; o < MO; ++o) {
-                        const float2 xs = *reinterpret_cast<const float2*>(xsum + gi * LDC + o * 8 + 2 * t);
-                        accf[o][2 * h + 0] = fmaf(sv, fmaf(zc, xs.x, accg[o][2 * h + 0]), accf[o][2 * h + 0]);
-                        accf[o][2 * h + 1] = fmaf(sv, fmaf(zc, xs.y, accg[o][2 * h + 1]), accf[o][2 * h + 1]);
+                for (int cg = 0; cg < CG; ++cg)
+#pragma unroll
+                    for (int o = 0; o < MO; ++o)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) accf[o][cg][i] += accg[o][cg][i] * xs[o].x;
+                if (false)
+#endif
+#pragma unroll
+                for (int cg = 0; cg < CG; ++cg)
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int col = c0 + 16 * cg + 8 * h;
+                        const float sv = bf16_bits_to_float(sc[gi * BN + col]);
+                        const float zc = -(128.0f + bf16_bits_to_float(sc[(GPS + gi) * BN + col]));
+#pragma unroll
+                        for (int o = 0; o < MO; ++o) {
+                            accf[o][cg][2 * h + 0] = fmaf(sv, fmaf(zc, xs[o].x, accg[o][cg][2 * h + 0]), accf[o][cg][2 * h + 0]);
+                            accf[o][cg][2 * h + 1] = fmaf(sv, fmaf(zc, xs[o].y, accg[o][cg][2 * h + 1]), accf[o][cg][2 * h + 1]);
+                        }
+                    }
+            }
+            if (SPARSE) {
+                // ---- outliers of this unit that fall into the lane group's four columns; the first
+                // two packets and their activation rows were requested before the dense math
+                auto apply = [&](const uint4 pk, const float2 (&x2)[4][MO]) {
+                    const float v[4] = {bf16lo(pk.z), bf16hi(pk.z), bf16lo(pk.w), bf16hi(pk.w)};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const uint32_t cls = (pk.y >> (8 * e + 3)) & 3u;     // which of the four columns: (c >> 3) & 3
+#pragma unroll
+                        for (int cg = 0; cg < CG; ++cg)
+#pragma unroll
+                            for (int h = 0; h < 2; ++h) {
+                                const float vv = (cls == (uint32_t)(2 * cg + h)) ? v[e] : 0.0f;
+#pragma unroll
+                                for (int o = 0; o < MO; ++o) {
+                                    accf[o][cg][2 * h + 0] = fmaf(vv, x2[e][o].x, accf[o][cg][2 * h + 0]);
+                                    accf[o][cg][2 * h + 1] = fmaf(vv, x2[e][o].y, accf[o][cg][2 * h + 1]);
+                                }
+                            }
+                    }
+                };
+                apply(pk0, xa);
+                if (cmax > 1) {
+                    float2 xb2[4][MO];
+                    fetch_x(pk1, xb2);
+                    apply(pk1, xb2);
+                    for (uint32_t i = 2; i < cmax; ++i) {
+                        const uint4 pk = packet(i);
+                        fetch_x(pk, xb2);
+                        apply(pk, xb2);
                     }
                 }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive_relaxed(bar_empty + 8 * s);
+#ifdef FQ_TRACE
+            if (blockIdx.x == 0 && dtid == 0) { g_trace[13] += tw1 - tw0; g_trace[14] += clock64() - tw1; g_trace[15] += 1; }
+#endif
 
             if (kt == KT - 1 || u == u_end - 1) {
                 // ---------------------------------------------------------- end of a piece
                 FQ_GT(dtid == 0 && piece < 2, 4 + 5 * piece);
-                if (SPARSE) {
-                    if (!warp_wait(bar_sparse_done, piece & 1, abort_flag, p.status)) { ok = false; break; }
-                    if (MO == 1) {
-                        // rows of msp floats, rows 2t and 2t+1 of this lane's two columns
-#pragma unroll
-                        for (int h = 0; h < 2; ++h)
-#pragma unroll
-                            for (int j = 0; j < 2; ++j)
-                                if ((uint32_t)(2 * t + j) < ms) {
-                                    float* cp = shc + (c0 + 8 * h) * msp + 2 * t + j;
-                                    for (uint32_t rr = 0; rr < n_rep; ++rr, cp += shc_copy) {
-                                        accf[0][2 * h + j] += *cp;
-                                        *cp = 0.0f;
-                                    }
-                                }
-                    } else {
-#pragma unroll
-                        for (int h = 0; h < 2; ++h)
-#pragma unroll
-                            for (int o = 0; o < MO; ++o) {
-                                float2* cp = reinterpret_cast<float2*>(shc + shc_quad<Q>(c0 + 8 * h, 2 * o + (t >> 1), LDC) + 2 * (t & 1));
-                                const float2 v = *cp;
-                                accf[o][2 * h + 0] += v.x;
-                                accf[o][2 * h + 1] += v.y;
-                                *cp = make_float2(0.0f, 0.0f);
-                            }
-                    }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_dense_done);
-                }
-                FQ_GT(dtid == 0 && piece < 2, 5 + 5 * piece);
                 const uint32_t u_tile0 = tn * KT;
                 const uint32_t piece_k0 = max(u_tile0, u_begin) - u_tile0;
                 const bool full_piece = (piece_k0 == 0) && (kt == KT - 1);
                 bool write_y = full_piece;
                 if (!full_piece) {
-                    // FP32 partial in fragment order; the last CTA to arrive sums them in CTA order
+                    // Split tile.  Every warp settles its own 32-column strip, without CTA-wide
+                    // barriers: FP32 partial in fragment order, then one arrival per (tile, strip);
+                    // the last warp to arrive adds the partials in CTA order (the same order in
+                    // every run) and writes Y.
                     const uint32_t which = (u_begin / KT == tn) ? 0u : 1u;
-                    float* slot = p.partials + ((size_t)blockIdx.x * 2 + which) * (size_t)(BN * LDC);
+                    float* slot = p.partials + ((size_t)blockIdx.x * 2 + which) * (size_t)(BN * LDC) + dw * (32 * LDC) + lane;
 #pragma unroll
                     for (int o = 0; o < MO; ++o)
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) __stcg(slot + (size_t)(o * 4 + i) * (NDW * 32) + dtid, accf[o][i]);
-                    __threadfence();
+                        for (int cg = 0; cg < CG; ++cg)
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) __stcg(slot + ((o * CG + cg) * 4 + i) * 32, accf[o][cg][i]);
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_dense);
-                    if (!warp_wait(bar_dense, dense_phase & 1, abort_flag, p.status)) { ok = false; break; }
-                    ++dense_phase;
-                    FQ_GT(dtid == 0 && piece < 2, 6 + 5 * piece);
                     const uint32_t c_first = cta_of_unit(u_tile0, q, r), c_last = cta_of_unit(u_tile0 + KT - 1, q, r);
-                    if (dtid == 0) {
-                        const uint32_t old = atomicAdd(p.counters + tn, 1u);
-                        *last_flag = (old == c_last - c_first) ? 1u : 0u;
+                    uint32_t last = 0;
+                    if (lane == 0) {
+                        __threadfence();                       // the warp's stores, ordered before the arrival
+                        const uint32_t old = atomicAdd(p.counters + tn * NDW + dw, 1u);
+                        last = (old == c_last - c_first) ? 1u : 0u;
+                        if (last) __threadfence();
                     }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_dense);
-                    if (!warp_wait(bar_dense, dense_phase & 1, abort_flag, p.status)) { ok = false; break; }
-                    ++dense_phase;
+                    last = __shfl_sync(0xffffffffu, last, 0);
                     FQ_GT(dtid == 0 && piece < 2, 7 + 5 * piece);
-                    if (*last_flag) {
+                    if (last) {
                         write_y = true;
-                        __threadfence();
 #pragma unroll
                         for (int o = 0; o < MO; ++o)
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) accf[o][i] = 0.0f;
-                        for (uint32_t c = c_first; c <= c_last; ++c) {
-                            const uint32_t wch = (unit_begin_of(c, q, r) / KT == tn) ? 0u : 1u;
-                            const float* sl = p.partials + ((size_t)c * 2 + wch) * (size_t)(BN * LDC);
+                            for (int cg = 0; cg < CG; ++cg)
 #pragma unroll
-                            for (int o = 0; o < MO; ++o)
+                                for (int i = 0; i < 4; ++i) accf[o][cg][i] = 0.0f;
+                        // four contributors' loads in flight at a time; the additions keep CTA order
+                        for (uint32_t c = c_first; c <= c_last; c += 4) {
+                            float v[4][MO * CG * 4];
 #pragma unroll
-                                for (int i = 0; i < 4; ++i) accf[o][i] += __ldcg(sl + (size_t)(o * 4 + i) * (NDW * 32) + dtid);
+                            for (int d = 0; d < 4; ++d) {
+                                const uint32_t cc = min(c + d, c_last);
+                                const uint32_t wch = (unit_begin_of(cc, q, r) / KT == tn) ? 0u : 1u;
+                                const float* sl = p.partials + ((size_t)cc * 2 + wch) * (size_t)(BN * LDC) + dw * (32 * LDC) + lane;
+#pragma unroll
+                                for (int e = 0; e < MO * CG * 4; ++e) v[d][e] = __ldcg(sl + e * 32);
+                            }
+#pragma unroll
+                            for (int d = 0; d < 4; ++d)
+                                if (c + d <= c_last) {
+#pragma unroll
+                                    for (int o = 0; o < MO; ++o)
+#pragma unroll
+                                        for (int cg = 0; cg < CG; ++cg)
+#pragma unroll
+                                            for (int i = 0; i < 4; ++i) accf[o][cg][i] += v[d][(o * CG + cg) * 4 + i];
+                                }
                         }
-                        if (dtid == 0) p.counters[tn] = 0;  // ready for the next call
+                        if (lane == 0) p.counters[tn * NDW + dw] = 0;  // ready for the next call
                     }
                 }
                 if (write_y) {
 #pragma unroll
-                    for (int h = 0; h < 2; ++h)
+                    for (int cg = 0; cg < CG; ++cg)
 #pragma unroll
-                        for (int o = 0; o < MO; ++o)
+                        for (int h = 0; h < 2; ++h)
 #pragma unroll
-                            for (int j = 0; j < 2; ++j) {
-                                const uint32_t m = o * 8 + 2 * t + j;
-                                if (m < p.M) p.Y[(size_t)m * p.N + (size_t)tn * BN + c0 + 8 * h] = float_to_bf16_bits(accf[o][2 * h + j]);
-                            }
+                            for (int o = 0; o < MO; ++o)
+#pragma unroll
+                                for (int j = 0; j < 2; ++j) {
+                                    const uint32_t m = o * 8 + 2 * t + j;
+                                    if (m < p.M)
+                                        p.Y[(size_t)m * p.N + (size_t)tn * BN + c0 + 16 * cg + 8 * h] = float_to_bf16_bits(accf[o][cg][2 * h + j]);
+                                }
                 }
 #pragma unroll
                 for (int o = 0; o < MO; ++o)
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) accf[o][i] = 0.0f;
+                    for (int cg = 0; cg < CG; ++cg)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) accf[o][cg][i] = 0.0f;
                 FQ_GT(dtid == 0 && piece < 2, 8 + 5 * piece);
                 ++piece;
             }
         }
         FQ_GT(dtid == 0, 15);
-    } else if (SPARSE && warp >= 2 + NDW) {
-        // ------------------------------------------------------------------ sparse
-        const uint32_t sw = warp - (2 + NDW);
-        if (sw + 1 <= nsw) {
-            const uint32_t nbb = p.NB >> 5;
-            const uint32_t bb = sw % nbb, og = sw / nbb, n_og = nsw / nbb;
-            const uint32_t bucket = bb * 32 + lane;
-            const uint32_t n_oct = (p.M + 7) >> 3;
-            uint32_t piece = 0;
-            // one-octet form: replica og of n_og owns the stages s with s mod n_og == og
-            uint32_t own = 0xffffffffu;
-            float* my_shc = shc;
-            if (MO == 1) {
-                own = 0;
-                for (uint32_t s = og; s < S; s += n_og) own |= 1u << s;
-                my_shc = shc + og * shc_copy;
-            }
-#ifdef FQ_TRACE
-            long long t_loop = 0, t_wait = 0, t_all0 = clock64(); uint32_t n_iter = 0, n_units = 0;
-#endif
-            for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
-                const uint32_t u = w.u, s = w.s, ph = w.ph, kt = w.kt;
-                const uint8_t* st = smem + s * p.stage_bytes;
-                if ((own >> s) & 1u) {
-#ifdef FQ_TRACE
-                long long tw0 = clock64();
-#endif
-                if (!warp_wait(bar_full + 8 * s, ph, abort_flag, p.status)) break;
-#ifdef FQ_TRACE
-                t_wait += clock64() - tw0; ++n_units;
-#endif
-                const uint32_t info = reinterpret_cast<const uint32_t*>(st + p.off_info)[bucket];
-                const uint32_t off = info & 0xffffu, cnt = info >> 16;
-                const uint4* pk_s = reinterpret_cast<const uint4*>(st + p.off_coo);
-                const uint4* pk_g = nullptr;
-                if (off + cnt > p.coo_cap) pk_g = p.packed + __ldg(p.indptr + u);
-#ifdef FQ_TRACE
-                long long tl0 = clock64(); n_iter += __reduce_max_sync(0xffffffffu, cnt);
-#endif
-                if (MO == 1) {
-                    const float* xt = reinterpret_cast<const float*>(st + p.off_xt);
-                    auto run = [&](auto tag) {
-                        constexpr int MS = decltype(tag)::value;
-                        auto packet = [&](uint32_t i) {
-                            const uint32_t idx = off + i;
-                            return (idx < p.coo_cap) ? pk_s[idx] : __ldg(pk_g + idx);
-                        };
-                        if (cnt == 0) return;
-                        const uint32_t dummy = BN + lane;
-                        NarrowPacket<MS> cur;
-                        narrow_fetch<MS>(cur, packet(0), xt, dummy);
-                        for (uint32_t i = 0; i < cnt; ++i) {
-                            // the next packet and its activation rows are in flight while this one is applied
-                            const bool more = i + 1 < cnt;
-                            const uint4 pkn = more ? packet(i + 1) : make_uint4(0, 0, 0, 0);
-                            float a[4][MS];
-                            narrow_accumulate<MS>(cur, my_shc, a);
-                            NarrowPacket<MS> nxt;
-                            if constexpr (MS <= 4) {
-                                narrow_fetch<MS>(nxt, pkn, xt, dummy);
-                                narrow_store<MS>(cur, my_shc, a);
-                            } else {           // eight-float rows: not enough registers for both at once
-                                narrow_store<MS>(cur, my_shc, a);
-                                narrow_fetch<MS>(nxt, pkn, xt, dummy);
-                            }
-                            cur = nxt;
-                        }
-                    };
-                    if (ms == 1) run(std::integral_constant<int, 1>{});
-                    else if (ms == 2) run(std::integral_constant<int, 2>{});
-                    else if (ms == 4) run(std::integral_constant<int, 4>{});
-                    else run(std::integral_constant<int, 8>{});
-                    __syncwarp();
-                } else {
-                    for (uint32_t o = og; o < n_oct; o += n_og) {
-                        const float* xt = reinterpret_cast<const float*>(st + p.off_xt) + o * 1024;
-                        for (uint32_t i = 0; i < cnt; ++i) {
-                            const uint32_t idx = off + i;
-                            const uint4 pk = (idx < p.coo_cap) ? pk_s[idx] : __ldg(pk_g + idx);
-                            apply_packet<Q>(pk, xt, shc, o, LDC);
-                        }
-                        __syncwarp();
-                    }
-                }
-#ifdef FQ_TRACE
-                t_loop += clock64() - tl0;
-#endif
-                if (lane == 0) mbar_arrive_relaxed(bar_empty + 8 * s);
-                }
-                if (kt == KT - 1 || u == u_end - 1) {
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_sparse_done);
-                    if (!warp_wait(bar_dense_done, piece & 1, abort_flag, p.status)) break;
-                    ++piece;
-                }
-            }
-#ifdef FQ_TRACE
-            if (blockIdx.x == 0 && sw == 0 && lane == 0) {
-                g_trace[0] = (unsigned long long)t_loop; g_trace[1] = n_iter; g_trace[2] = n_units;
-                g_trace[3] = (unsigned long long)t_wait; g_trace[4] = (unsigned long long)(clock64() - t_all0);
-            }
-#endif
-        }
     }
 }
 
@@ -1417,42 +1326,18 @@ static fq_status_t make_plan(const fq_layout_t* L, uint32_t M, bool sparse, Plan
     return FQ_OK;
 }
 
-// Sparse warps per CTA of the small-batch kernel at M <= 8 (developer knob: FQ_SPARSE_WARPS = 1..6).
-static uint32_t sparse_warps_target() {
-    static const uint32_t v = [] {
-        const char* e = std::getenv("FQ_SPARSE_WARPS");
-        const int n = e ? std::atoi(e) : 4;
-        return (uint32_t)std::min(6, std::max(1, n));
-    }();
-    return v;
-}
-
 // Plan of the small-batch kernel (fq_mma_kernel): M <= 16 per launch.
 static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, Plan& pl) {
     const uint32_t BN = L->BN, NB = L->buckets_per_tile, GPS = kBK / L->group;
     const uint32_t MO = M <= 8 ? 1 : 2, ROWS = 8 * MO;
-    const uint32_t NDW = BN / 16;
-    uint32_t nsw = 0, n_rep = 1;
-    if (sparse) {
-        const uint32_t nbb = NB / 32, n_oct = (M + 7) / 8;
-        if (MO == 1) {
-            // replicas split the units between them (each owns fixed stages and an FP32 tile of its own)
-            n_rep = std::max<uint32_t>(1, sparse_warps_target() / nbb);
-            nsw = nbb * n_rep;
-        } else {
-            nsw = nbb * std::min<uint32_t>(n_oct, std::max<uint32_t>(1, 4 / nbb));
-        }
-    }
+    const uint32_t NDW = BN / 32;
     Params& p = pl.p;
     std::memset(&p, 0, sizeof(p));
-    p.M = M; p.K = L->K; p.N = L->N; p.KT = L->K / kBK; p.NT = L->N / BN; p.NB = NB; p.nsw = nsw;
+    p.M = M; p.K = L->K; p.N = L->N; p.KT = L->K / kBK; p.NT = L->N / BN; p.NB = NB; p.nsw = 0;
     const uint32_t w_bytes = 16 * BN * 4, sz_bytes = 2 * GPS * BN * 2;
-    // one octet: FP32 rows of at most 12 floats (ms_pitch); two octets: the 8-float rows of the wide form
-    const uint32_t msp = ms_pitch(M <= 1 ? 1 : M <= 2 ? 2 : M <= 4 ? 4 : 8);
-    const uint32_t shc_bytes = sparse ? (MO == 1 ? n_rep * (BN + 32) * msp : BN * ROWS) * 4 : 0;
-    const uint32_t xt_bytes = sparse ? (MO == 1 ? kBK * msp * 4 : MO * 4096) : 0;
-    p.shc_floats = shc_bytes / 4;
-    const uint32_t fixed = shc_bytes + 1024;
+    const uint32_t xt_bytes = sparse ? MO * 4096 : 0;     // FP32 [octet][k][8]
+    const uint32_t fixed = 1024;
+    const uint32_t budget = kSmemBudget;
     uint32_t cap = 0;
     if (sparse) {
         cap = L->max_tile_packets ? round_up(L->max_tile_packets, 8) : 256;
@@ -1464,19 +1349,19 @@ static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, 
         p.off_xcan = p.off_sz + round_up(sz_bytes, 128);
         p.off_xsum = p.off_xcan + round_up(ROWS * kXPitch, 128);
         p.off_xt = p.off_xsum + round_up(GPS * ROWS * 4, 128);          // stage-relative in this kernel
-        p.off_info = p.off_xt + round_up(xt_bytes, 128);
+        p.off_info = p.off_xt + xt_bytes;
         p.off_coo = p.off_info + (sparse ? round_up(NB * 4, 128) : 0);
         stage = round_up(p.off_coo + cap * 16, 128);
-        S = std::min<uint32_t>(8, (kSmemBudget - fixed) / stage);
+        S = std::min<uint32_t>(8, (budget - fixed) / stage);
         if (S >= 4 || cap <= 64) break;
         cap = std::max<uint32_t>(64, cap / 2);
     }
     if (S < 3) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "shared-memory stages do not fit");
     p.coo_cap = cap; p.stages = S; p.stage_bytes = stage;
     p.off_shc = S * stage;
-    p.off_bar = p.off_shc + shc_bytes;
+    p.off_bar = p.off_shc;
     pl.smem = p.off_bar + 1024;
-    pl.threads = 32 * (2 + NDW + nsw);
+    pl.threads = 32 * (1 + kActWarps + NDW);
     const int sms = sm_count_cached();
     if (sms <= 0) return fail(FQ_ERR_CUDA, "no CUDA device: %s", cudaGetErrorString(cudaGetLastError()));
     pl.grid = std::min<uint32_t>({(uint32_t)sms, kMaxCtas, p.NT * p.KT});
@@ -1504,7 +1389,7 @@ static uint32_t mma_max_rows() {
     static int v = -1;
     if (v < 0) {
         const char* e = std::getenv("FQ_ENGINE");
-        v = 8;
+        v = 16;
         if (e && std::strcmp(e, "mma") == 0) v = 16;
         if (e && std::strcmp(e, "tc") == 0) v = 0;
     }

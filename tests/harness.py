@@ -66,8 +66,8 @@ class Packed:
         return self._q
 
 
-def pack_layer(layer: synth.Layer, g: int, BN: int = 0, NB: int = 0, upload: bool = True) -> Packed:
-    L = fq.fq_get_layout(layer.K, layer.N, g, bn_hint=BN, nb_hint=NB)
+def pack_layer(layer: synth.Layer, g: int, BN: int = 0, upload: bool = True) -> Packed:
+    L = fq.fq_get_layout(layer.K, layer.N, g, bn_hint=BN)
     wq, scale, zero = fq.fq_pack_int4(L, layer.W, layer.mask if layer.nnz else None)
     indptr, info, packed = fq.fq_encode_tilecoo(L, layer.coo_k, layer.coo_n, layer.coo_v)
     fq.fq_validate_tilecoo(L, indptr, info, packed)

@@ -27,7 +27,8 @@ def test_library_exports_every_declared_symbol():
 def test_layout_defaults_and_errors():
     L = fq.fq_get_layout(4096, 4096, 128)
     assert (L.BK, L.BN, L.buckets_per_tile, L.coo_unit_bytes) == (128, 256, 64, 16)
-    assert fq.fq_get_layout(4096, 4224, 64).BN == 128
+    L128 = fq.fq_get_layout(4096, 4224, 64)
+    assert (L128.BN, L128.buckets_per_tile) == (128, 32)
     for bad in [(4096, 4096, 32), (4000, 4096, 128), (4096, 4100, 128)]:
         with pytest.raises(fq.FqError) as e:
             fq.fq_get_layout(*bad)
@@ -77,30 +78,18 @@ def _as_set(k, n, v):
     return set(zip(k.tolist(), n.tolist(), v.tolist()))
 
 
-def _bank_conflict_cycles(bk, bb, order_pos, NB):
-    """Shared-memory passes of the sparse lanes' activation reads (32-byte FP32 rows, so rows k and
-    k + 4 share banks): lanes (= buckets) are served eight at a time; at entry position i the passes
-    needed are the largest number of different rows falling in one bank group (k mod 4)."""
-    cycles = 0
-    per_bucket = {}
-    for k, b, pos in zip(bk, bb, order_pos):
-        per_bucket.setdefault(int(b), {})[int(pos)] = int(k)
-    depth = max((len(v) for v in per_bucket.values()), default=0)
-    for q0 in range(0, NB, 8):
-        for i in range(depth):
-            rows = {per_bucket[b][i] for b in range(q0, q0 + 8) if b in per_bucket and i in per_bucket[b]}
-            groups = {}
-            for k in rows:
-                groups[k % 4] = groups.get(k % 4, 0) + 1
-            cycles += max(groups.values(), default=0)
-    return cycles
+def _bucket_of(c):
+    """Bucket of a tile column: columns g, g + 8, g + 16, g + 24 of a 32-column block share a bucket."""
+    return (c // 32) * 8 + c % 8
 
 
-@pytest.mark.parametrize("layout,density,NB", [("uniform", 0.01, 32), ("mixed", 0.02, 64), ("clustered", 0.05, 128)])
-def test_tilecoo_encode_invariants(layout, density, NB):
-    K, N, BN = 512, 1024, 256
-    Lr = synth.layer(synth.tensor_seed(3, NB), K, N, density=density, layout=layout)
-    L = fq.fq_get_layout(K, N, 128, bn_hint=BN, nb_hint=NB)
+@pytest.mark.parametrize("layout,density,BN", [("uniform", 0.01, 256), ("mixed", 0.02, 256), ("clustered", 0.05, 128)])
+def test_tilecoo_encode_invariants(layout, density, BN):
+    K, N = 512, 1024
+    NB = BN // 4
+    Lr = synth.layer(synth.tensor_seed(3, BN + len(layout)), K, N, density=density, layout=layout)
+    L = fq.fq_get_layout(K, N, 128, bn_hint=BN)
+    assert L.buckets_per_tile == NB
     n_ip, n_bi, n_pk, mx = fq.fq_encode_tilecoo_sizes(L, Lr.coo_k, Lr.coo_n, Lr.coo_v)
     indptr, info, packed = fq.fq_encode_tilecoo(L, Lr.coo_k, Lr.coo_n, Lr.coo_v)
     ntile = (K // 128) * (N // BN)
@@ -116,78 +105,43 @@ def test_tilecoo_encode_invariants(layout, density, NB):
     k2, n2, v2 = fq.fq_decode_tilecoo(L, indptr, info, packed)
     assert _as_set(k2, n2, v2) == want
     fq.fq_validate_tilecoo(L, indptr, info, packed)
-    # buckets of a tile own disjoint column sets (the sparse path's conflict-free accumulation)
+    # every outlier sits in the bucket of its column, in every tile (the conflict-free accumulation of
+    # the sparse path: a bucket's four columns belong to one group of four lanes)
+    assert np.array_equal(b % NB, _bucket_of(n % BN))
+    # a bucket is padded only in its last packet: packets = ceil(entries / 4)
     tile = (n // BN) * (K // 128) + k // 128
-    owner = {}
-    for t_, c_, b_ in zip(tile.tolist(), n.tolist(), b.tolist()):
-        assert owner.setdefault((t_, c_), b_) == b_
-    # a column lives in one block of 32 buckets (column mod number of blocks) in every tile; inside a
-    # block the greedy least-loaded assignment gives max bucket load <= mean load + largest column
-    nblk = NB // 32
-    assert np.array_equal((b % NB) // 32, (n % BN) % nblk)
-    for t_ in np.unique(tile):
-        sel = tile == t_
-        loads = np.bincount(b[sel] - t_ * NB, minlength=NB)
-        for blk in range(nblk):
-            in_blk = sel & ((n % BN) % nblk == blk)
-            colmax = np.bincount(n[in_blk] % BN, minlength=BN).max() if in_blk.any() else 0
-            bl = loads[32 * blk:32 * blk + 32]
-            assert bl.max() <= bl.sum() / 32 + colmax + 1e-9
+    assert np.array_equal(b // NB, tile)
+    loads = np.bincount(b, minlength=ntile * NB)
+    assert np.array_equal(info >> 16, (loads + 3) // 4)
+    off = (info & 0xffff).reshape(ntile, NB)
+    cnt = (info >> 16).reshape(ntile, NB)
+    assert np.array_equal(off[:, 1:], np.cumsum(cnt, axis=1)[:, :-1]) and not off[:, 0].any()
 
 
-def test_tilecoo_element_order_separates_columns_and_staggers_bank_groups():
-    K, N, BN, NB = 128, 256, 256, 32
+def test_tilecoo_entries_of_a_bucket_are_stored_by_row_then_column():
+    K, N, BN = 128, 256, 256
+    NB = BN // 4
     Lr = synth.layer(77, K, N, density=0.06, layout="uniform")
-    L = fq.fq_get_layout(K, N, 128, bn_hint=BN, nb_hint=NB)
+    L = fq.fq_get_layout(K, N, 128, bn_hint=BN)
     indptr, info, packed = fq.fq_encode_tilecoo(L, Lr.coo_k, Lr.coo_n, Lr.coo_v)
     k, n, v, b = oracle.decode_tilecoo(indptr, info, packed, K, N, BN, NB)   # decode keeps stored order
-    pos = np.zeros(len(k), dtype=np.int64)
-    seen = {}
-    for i, bb in enumerate(b.tolist()):
-        pos[i] = seen.get(bb, 0)
-        seen[bb] = pos[i] + 1
-    # rule 1: a packet is either "spread" (its outliers sit in different columns) or "stack" (four
-    # outliers of one column); a stack is only formed while fewer than four columns have entries left
-    raw = packed.reshape(-1, 16)
     for bb in np.unique(b):
-        t_, lb = divmod(int(bb), NB)
-        off, cnt = int(info[bb]) & 0xffff, int(info[bb]) >> 16
-        left = {}
-        for c in (n[b == bb] % BN).tolist():
-            left[c] = left.get(c, 0) + 1
-        for pk in raw[int(indptr[t_]) + off:int(indptr[t_]) + off + cnt]:
-            vals = pk[8:].view(np.uint16)
-            cols = [int(pk[4 + s_]) for s_ in range(4) if vals[s_] != 0]
-            assert len(cols) >= 1
-            if len(set(cols)) < len(cols):
-                assert len(cols) == 4 and len(set(cols)) == 1
-                assert sum(1 for v_ in left.values() if v_ > 0) < 4
-            else:
-                alive = sum(1 for v_ in left.values() if v_ > 0)
-                assert len(cols) == min(4, alive)
-            for c in cols:
-                left[c] -= 1
-        assert all(v_ == 0 for v_ in left.values())
-    # rule 2 pays off: fewer shared-memory passes than the plain (column, row) order
-    plain_pos = np.zeros(len(k), dtype=np.int64)
-    for bb in np.unique(b):
-        idx = np.nonzero(b == bb)[0]
-        order = sorted(idx.tolist(), key=lambda i: (int(n[i]), int(k[i])))
-        for p_, i in enumerate(order):
-            plain_pos[i] = p_
-    assert _bank_conflict_cycles(k, b, pos, NB) < _bank_conflict_cycles(k, b, plain_pos, NB)
-    # a bucket that owns a single hot column cannot avoid repeats, and still round-trips
+        sel = b == bb
+        key = k[sel].astype(np.int64) * BN + n[sel]
+        assert np.all(np.diff(key) > 0)
+    # a hot column fills its bucket with packets of four
     kk = np.arange(0, 40, dtype=np.uint32)
     nn = np.full(40, 7, dtype=np.uint32)
     vv = (0x3F80 + np.arange(40)).astype(np.uint16)
     ip, bi, pk = fq.fq_encode_tilecoo(L, kk, nn, vv)
     k2, n2, v2 = fq.fq_decode_tilecoo(L, ip, bi, pk)
-    assert _as_set(k2, n2, v2) == _as_set(kk, nn, vv) and pk.shape[0] == 10          # ten stacks of four
+    assert _as_set(k2, n2, v2) == _as_set(kk, nn, vv) and pk.shape[0] == 10
+    assert int(bi[_bucket_of(7)]) >> 16 == 10
 
 
 def test_tilecoo_edge_cases():
-    K, N, BN, NB = 256, 512, 256, 32
-    L = fq.fq_get_layout(K, N, 128, bn_hint=BN, nb_hint=NB)
+    K, N, BN, NB = 256, 512, 256, 64
+    L = fq.fq_get_layout(K, N, 128, bn_hint=BN)
     e32, e16 = np.zeros(0, dtype=np.uint32), np.zeros(0, dtype=np.uint16)
     # no outliers at all
     indptr, info, packed = fq.fq_encode_tilecoo(L, e32, e32, e16)
@@ -201,8 +155,8 @@ def test_tilecoo_edge_cases():
     assert packed.shape[0] == 1
     kk, nn, vv, _ = oracle.decode_tilecoo(indptr, info, packed, K, N, BN, NB)
     assert (kk.tolist(), nn.tolist(), vv.tolist()) == ([200], [300], [0x4000])
-    # padding slots: value 0, row 0, a column byte that differs from slot to slot
-    assert packed[0, :4].tolist() == [72, 0, 0, 0] and packed[0, 4:8].tolist() == [44, 254, 253, 252]
+    # padding slots: value 0, row 0, the first column of the bucket (column 44 -> bucket 8 + 4 -> column 36)
+    assert packed[0, :4].tolist() == [72, 0, 0, 0] and packed[0, 4:8].tolist() == [44, 36, 36, 36]
     assert packed[0, 10:].tolist() == [0] * 6
     # one completely dense tile plus a hot row and a hot column elsewhere
     kk, nn = np.meshgrid(np.arange(128, 256), np.arange(0, 256), indexing="ij")
@@ -223,9 +177,9 @@ def test_tilecoo_edge_cases():
 
 
 def test_validator_rejects_corrupted_arrays():
-    K, N, BN, NB = 256, 512, 256, 32
+    K, N, BN, NB = 256, 512, 256, 64
     Lr = synth.layer(5, K, N, density=0.02, layout="mixed")
-    L = fq.fq_get_layout(K, N, 128, bn_hint=BN, nb_hint=NB)
+    L = fq.fq_get_layout(K, N, 128, bn_hint=BN)
     indptr, info, packed = fq.fq_encode_tilecoo(L, Lr.coo_k, Lr.coo_n, Lr.coo_v)
     fq.fq_validate_tilecoo(L, indptr, info, packed)
 
@@ -242,13 +196,15 @@ def test_validator_rejects_corrupted_arrays():
     expect_format_error(indptr, bad, packed)
     bad = packed.copy(); bad[0, 0] = 200                 # row index outside the 128-row tile
     expect_format_error(indptr, info, bad)
-    # move one entry into a column another bucket of the same tile owns
+    bad = packed.copy(); bad[0, 5] = 0                   # a padding slot must stay inside the tile too
+    bad[0, 1] = 130
+    expect_format_error(indptr, info, bad)
+    # move one entry into a column that belongs to another bucket
     k, n, v, b = oracle.decode_tilecoo(indptr, info, packed, K, N, BN, NB)
-    first_tile = b < NB
-    cols0 = n[first_tile & (b == b[first_tile][0])] % BN
-    other = n[first_tile & (b != b[first_tile][0])] % BN
+    b0 = int(b[0])
+    assert b0 < NB
+    off0 = int(info[b0] & 0xffff)
     bad = packed.copy()
-    off0 = int(info[int(b[first_tile][0])] & 0xffff)
-    bad[off0, 4] = int(other[0])
-    assert int(other[0]) not in cols0.tolist()
+    assert bad[off0, 8:10].any()
+    bad[off0, 4] = (int(bad[off0, 4]) + 1) % BN
     expect_format_error(indptr, info, bad)

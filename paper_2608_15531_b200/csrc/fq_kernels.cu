@@ -770,7 +770,7 @@ constexpr int kXPitch = 320;   // activation row in shared memory: 256 B + 64 B,
 //                     the four lanes of group g walk that bucket's packets and add v * x[row][k]
 //                     straight into their accumulators (Section 4.2 without the shared-memory
 //                     scatter: no atomics, no read-modify-write, no merge step).
-template <int BN, int MO, int GROUP, bool SPARSE>
+template <int BN, int MO, int GROUP, bool SPARSE, int MS>
 __global__ void __launch_bounds__(32 * (1 + kActWarps + BN / 32), 1) fq_mma_kernel(const Params p) {
     constexpr int NDW = BN / 32;
     constexpr int NA = kActWarps;                           // activation warps: warp a takes the units it with it mod NA == a
@@ -800,6 +800,11 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + BN / 32), 1) fq_mma_kern
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncthreads();
     FQ_GT(tid == 0, 1);
+    // The grid after this one in the stream may start now (it takes SMs as this grid's CTAs leave).
+    // Every warp but the producer waits for the grid before this one to finish: the producer reads
+    // only weights, which no kernel writes while calls are in flight.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (warp != 0) asm volatile("griddepcontrol.wait;" ::: "memory");
 
     const uint32_t U = p.NT * p.KT, P = gridDim.x, q = U / P, r = U % P;
     const uint32_t u_begin = unit_begin_of(blockIdx.x, q, r);
@@ -964,6 +969,10 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + BN / 32), 1) fq_mma_kern
             for (int cg = 0; cg < CG; ++cg)
 #pragma unroll
                 for (int i = 0; i < 4; ++i) accf[o][cg][i] = 0.0f;
+        // Outlier accumulator of the single-row form (MS == 1): there lane (g, t) owns ONE column,
+        // 32 dw + 8 t + g (the bucket's column number t); the sums are moved into the MMA fragment
+        // layout above (four columns x two rows per lane) once per piece.
+        float sacc[1][1] = {{0.0f}};
         uint32_t piece = 0;
         bool ok = true;
         for (UnitIter w(u_begin, KT); w.u < u_end && ok; w.next(S, KT)) {
@@ -981,12 +990,12 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + BN / 32), 1) fq_mma_kern
             const uint8_t* xrow = st + p.off_xcan + g * kXPitch + t * 16;
             const uint16_t* sc = reinterpret_cast<const uint16_t*>(st + p.off_sz);
             const float* xsum = reinterpret_cast<const float*>(st + p.off_xsum);
-            // outliers: bucket descriptor, first two packets and the first packet's activation rows are
-            // requested now and used after the dense math of the unit
+            // outliers: the bucket descriptor and the first two packets are requested now and used
+            // after the dense math of the unit
             uint32_t sp_off = 0, sp_cnt = 0, cmax = 0;
             const uint4* pk_s = reinterpret_cast<const uint4*>(st + p.off_coo);
             const uint4* pk_g = nullptr;
-            const float* xt = reinterpret_cast<const float*>(st + p.off_xt) + 2 * t;
+            const float* xt = reinterpret_cast<const float*>(st + p.off_xt);
             auto packet = [&](uint32_t i) {
                 uint4 pk = make_uint4(0, 0, 0, 0);            // beyond the bucket's list: four padding slots
                 if (i < sp_cnt) {
@@ -995,12 +1004,13 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + BN / 32), 1) fq_mma_kern
                 }
                 return pk;
             };
+            // rows-by-lane form (MS == 8): activation rows 2t, 2t+1 of every octet for the four slots
             auto fetch_x = [&](const uint4 pk, float2 (&x2)[4][MO]) {
 #pragma unroll
                 for (int e = 0; e < 4; ++e)
 #pragma unroll
                     for (int o = 0; o < MO; ++o)
-                        x2[e][o] = *reinterpret_cast<const float2*>(xt + o * 1024 + ((pk.x >> (8 * e)) & 0xffu) * 8);
+                        x2[e][o] = *reinterpret_cast<const float2*>(xt + 2 * t + o * 1024 + ((pk.x >> (8 * e)) & 0xffu) * 8);
             };
             uint4 pk0 = make_uint4(0, 0, 0, 0), pk1 = pk0;
             float2 xa[4][MO];
@@ -1012,7 +1022,7 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + BN / 32), 1) fq_mma_kern
                 cmax = __reduce_max_sync(0xffffffffu, sp_cnt);
                 pk0 = packet(0);
                 pk1 = packet(1);
-                fetch_x(pk0, xa);
+                if constexpr (MS == 8) fetch_x(pk0, xa);
             }
 #if defined(FQ_EXP) && (FQ_EXP == 24 || FQ_EXP == 25)
             if (false)
@@ -1082,35 +1092,56 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + BN / 32), 1) fq_mma_kern
                     }
             }
             if (SPARSE) {
-                // ---- outliers of this unit that fall into the lane group's four columns; the first
-                // two packets and their activation rows were requested before the dense math
-                auto apply = [&](const uint4 pk, const float2 (&x2)[4][MO]) {
-                    const float v[4] = {bf16lo(pk.z), bf16hi(pk.z), bf16lo(pk.w), bf16hi(pk.w)};
+                // ---- outliers of this unit in the lane group's bucket.  All four lanes of the group read
+                // the same packets (padding slots have value 0: they add 0).
+                if constexpr (MS == 1) {
+                    // single batch row: lane t keeps the slots of column number t of the bucket
+                    auto apply = [&](const uint4 pk) {
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const uint32_t cls = (pk.y >> (8 * e + 3)) & 3u;     // which of the four columns: (c >> 3) & 3
-#pragma unroll
-                        for (int cg = 0; cg < CG; ++cg)
-#pragma unroll
-                            for (int h = 0; h < 2; ++h) {
-                                const float vv = (cls == (uint32_t)(2 * cg + h)) ? v[e] : 0.0f;
-#pragma unroll
-                                for (int o = 0; o < MO; ++o) {
-                                    accf[o][cg][2 * h + 0] = fmaf(vv, x2[e][o].x, accf[o][cg][2 * h + 0]);
-                                    accf[o][cg][2 * h + 1] = fmaf(vv, x2[e][o].y, accf[o][cg][2 * h + 1]);
-                                }
-                            }
+                        for (int e = 0; e < 4; ++e) {
+                            const uint32_t cls = (pk.y >> (8 * e + 3)) & 3u;     // column number inside the bucket: (c >> 3) & 3
+                            const float v = (e & 1) ? bf16hi(e < 2 ? pk.z : pk.w) : bf16lo(e < 2 ? pk.z : pk.w);
+                            const float x = xt[((pk.x >> (8 * e)) & 0xffu) * 8];
+                            sacc[0][0] = fmaf(cls == (uint32_t)t ? v : 0.0f, x, sacc[0][0]);
+                        }
+                    };
+                    if (cmax > 0) apply(pk0);
+                    if (cmax > 1) {
+                        apply(pk1);
+                        for (uint32_t i = 2; i < cmax; ++i) apply(packet(i));
                     }
-                };
-                apply(pk0, xa);
-                if (cmax > 1) {
-                    float2 xb2[4][MO];
-                    fetch_x(pk1, xb2);
-                    apply(pk1, xb2);
-                    for (uint32_t i = 2; i < cmax; ++i) {
-                        const uint4 pk = packet(i);
-                        fetch_x(pk, xb2);
-                        apply(pk, xb2);
+                } else {
+                    // several batch rows: lane t keeps rows 2t, 2t+1 (+8) of all four columns, in the
+                    // MMA fragment registers themselves
+                    auto apply = [&](const uint4 pk, const float2 (&x2)[4][MO]) {
+                        const float v[4] = {bf16lo(pk.z), bf16hi(pk.z), bf16lo(pk.w), bf16hi(pk.w)};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const uint32_t cls = (pk.y >> (8 * e + 3)) & 3u;
+#pragma unroll
+                            for (int cg = 0; cg < CG; ++cg)
+#pragma unroll
+                                for (int h = 0; h < 2; ++h) {
+                                    // a select, not a branch: the lanes of a warp hold different columns
+                                    const float vv = (cls == (uint32_t)(2 * cg + h)) ? v[e] : 0.0f;
+#pragma unroll
+                                    for (int o = 0; o < MO; ++o) {
+                                        accf[o][cg][2 * h + 0] = fmaf(vv, x2[e][o].x, accf[o][cg][2 * h + 0]);
+                                        accf[o][cg][2 * h + 1] = fmaf(vv, x2[e][o].y, accf[o][cg][2 * h + 1]);
+                                    }
+                                }
+                        }
+                    };
+                    if (cmax > 0) apply(pk0, xa);
+                    if (cmax > 1) {
+                        float2 xb2[4][MO];
+                        fetch_x(pk1, xb2);
+                        apply(pk1, xb2);
+                        for (uint32_t i = 2; i < cmax; ++i) {
+                            const uint4 pk = packet(i);
+                            fetch_x(pk, xb2);
+                            apply(pk, xb2);
+                        }
                     }
                 }
             }
@@ -1123,6 +1154,16 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + BN / 32), 1) fq_mma_kern
             if (kt == KT - 1 || u == u_end - 1) {
                 // ---------------------------------------------------------- end of a piece
                 FQ_GT(dtid == 0 && piece < 2, 4 + 5 * piece);
+                if (SPARSE && MS == 1) {
+                    // single-row outlier sums -> fragment layout: column number c of the group comes
+                    // from lane (g, c); batch row 0 lives in lane t = 0
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const float v = __shfl_sync(0xffffffffu, sacc[0][0], (lane & ~3) | c);
+                        if (t == 0) accf[0][c >> 1][2 * (c & 1)] += v;
+                    }
+                    sacc[0][0] = 0.0f;
+                }
                 const uint32_t u_tile0 = tn * KT;
                 const uint32_t piece_k0 = max(u_tile0, u_begin) - u_tile0;
                 const bool full_piece = (piece_k0 == 0) && (kt == KT - 1);
@@ -1370,21 +1411,25 @@ static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, 
 
 typedef void (*KernelFn)(const Params);
 
+// MS: form of the outlier step (1: single batch row, one column per lane; 8: rows split over the lanes)
 template <int BN, int MO, int G>
-static KernelFn pick_mma_sparse(bool sparse) {
-    return sparse ? (KernelFn)fq_mma_kernel<BN, MO, G, true> : (KernelFn)fq_mma_kernel<BN, MO, G, false>;
+static KernelFn pick_mma_sparse(bool sparse, uint32_t ms) {
+    if (!sparse) return (KernelFn)fq_mma_kernel<BN, MO, G, false, 8>;
+    if constexpr (MO == 1) {
+        if (ms == 1) return (KernelFn)fq_mma_kernel<BN, MO, G, true, 1>;
+    }
+    return (KernelFn)fq_mma_kernel<BN, MO, G, true, 8>;
 }
 template <int BN, int MO>
-static KernelFn pick_mma_group(uint32_t g, bool sparse) {
-    return g == 64 ? pick_mma_sparse<BN, MO, 64>(sparse) : pick_mma_sparse<BN, MO, 128>(sparse);
+static KernelFn pick_mma_group(uint32_t g, bool sparse, uint32_t ms) {
+    return g == 64 ? pick_mma_sparse<BN, MO, 64>(sparse, ms) : pick_mma_sparse<BN, MO, 128>(sparse, ms);
 }
-static KernelFn pick_mma_kernel(uint32_t bn, uint32_t mo, uint32_t g, bool sparse) {
-    if (bn == 128) return mo == 1 ? pick_mma_group<128, 1>(g, sparse) : pick_mma_group<128, 2>(g, sparse);
-    return mo == 1 ? pick_mma_group<256, 1>(g, sparse) : pick_mma_group<256, 2>(g, sparse);
+static KernelFn pick_mma_kernel(uint32_t bn, uint32_t M, uint32_t g, bool sparse) {
+    const uint32_t mo = M <= 8 ? 1 : 2, ms = M <= 1 ? 1 : 8;
+    if (bn == 128) return mo == 1 ? pick_mma_group<128, 1>(g, sparse, ms) : pick_mma_group<128, 2>(g, sparse, ms);
+    return mo == 1 ? pick_mma_group<256, 1>(g, sparse, ms) : pick_mma_group<256, 2>(g, sparse, ms);
 }
 
-// Which dense engine serves a launch of `mb` rows: the warp-level MMA kernel up to kMmaMaxRows
-// rows, tcgen05 above.  FQ_ENGINE=mma|tc in the environment overrides (development aid).
 static uint32_t mma_max_rows() {
     static int v = -1;
     if (v < 0) {
@@ -1429,6 +1474,17 @@ static cudaError_t ensure_smem_attr(const void* fn, int bytes) {
     return e;
 }
 
+// Launch the small-batch kernel so that it may overlap the tail of the kernel before it in the
+// stream (FQ_PDL=0 turns this off).  The weights, scales, zeros and Tile-COO arrays must then not be
+// written by a kernel that is still running when the call is made; everything else is ordered as usual.
+static bool overlap_launches() {
+    static const bool v = [] {
+        const char* e = std::getenv("FQ_PDL");
+        return !(e && std::strcmp(e, "0") == 0);
+    }();
+    return v;
+}
+
 static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
 static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, const void* wq, const void* scale,
@@ -1460,11 +1516,32 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
         p.status = (uint32_t*)workspace;
         p.counters = (uint32_t*)((uint8_t*)workspace + kWsHeaderBytes);
         p.partials = (float*)((uint8_t*)workspace + kWsHeaderBytes + kWsCounterBytes);
-        KernelFn fn = use_mma ? pick_mma_kernel(L->BN, mb <= 8 ? 1 : 2, L->group, sparse)
+        KernelFn fn = use_mma ? pick_mma_kernel(L->BN, mb, L->group, sparse)
                               : pick_kernel(L->BN, nb16_of(mb), L->group, sparse);
         cudaError_t e = ensure_smem_attr((const void*)fn, (int)kSmemBudget);
         if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-        fn<<<pl.grid, pl.threads, pl.smem, (cudaStream_t)stream>>>(p);
+        if (use_mma && overlap_launches()) {
+            // Programmatic dependent launch: this grid may become resident while the kernel before it
+            // in the stream drains.  Its producer warp then already streams weights (which no kernel
+            // writes); every other warp first executes griddepcontrol.wait, after which all memory
+            // operations of the earlier grid are complete and visible.
+            cudaLaunchConfig_t cfg;
+            std::memset(&cfg, 0, sizeof(cfg));
+            cfg.gridDim = dim3(pl.grid);
+            cfg.blockDim = dim3(pl.threads);
+            cfg.dynamicSmemBytes = pl.smem;
+            cfg.stream = (cudaStream_t)stream;
+            cudaLaunchAttribute attr;
+            std::memset(&attr, 0, sizeof(attr));
+            attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr.val.programmaticStreamSerializationAllowed = 1;
+            cfg.attrs = &attr;
+            cfg.numAttrs = 1;
+            e = cudaLaunchKernelEx(&cfg, fn, p);
+            if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
+        } else {
+            fn<<<pl.grid, pl.threads, pl.smem, (cudaStream_t)stream>>>(p);
+        }
         e = cudaGetLastError();
         if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
     }

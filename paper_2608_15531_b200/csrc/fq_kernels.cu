@@ -770,11 +770,12 @@ constexpr int kXPitch = 320;   // activation row in shared memory: 256 B + 64 B,
 //                     the four lanes of group g walk that bucket's packets and add v * x[row][k]
 //                     straight into their accumulators (Section 4.2 without the shared-memory
 //                     scatter: no atomics, no read-modify-write, no merge step).
-template <int BN, int MO, int GROUP, bool SPARSE, int MS>
-__global__ void __launch_bounds__(32 * (1 + kActWarps + BN / 32), 1) fq_mma_kernel(const Params p) {
+template <int BN, int MO, int GROUP, bool SPARSE, int MS, int NGRP>
+__global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq_mma_kernel(const Params p) {
     constexpr int NDW = BN / 32;
     constexpr int NA = kActWarps;                           // activation warps: warp a takes the units it with it mod NA == a
     constexpr int DW0 = 1 + NA;                             // first dense warp
+    // NGRP dense warp groups: group r takes the units it with it mod NGRP == r
     constexpr int CG = 2;                                   // 16-column MMA strips per warp
     constexpr int GPS = kBK / GROUP;
     constexpr int W_BYTES = 16 * BN * 4;
@@ -788,12 +789,15 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + BN / 32), 1) fq_mma_kern
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
     const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * S;
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 2 * S + 4);
+    // hand-over of group 1's partial sums to group 0 at the end of a piece: one pair of barriers per strip
+    const uint32_t bar_xfull = bar_empty + 8 * S + 64, bar_xempty = bar_xfull + 8 * NDW;
 
     if (tid == 0) {
         for (uint32_t s = 0; s < S; ++s) {
             mbar_init(bar_full + 8 * s, 2);   // producer's expect_tx arrival + activation warp
-            mbar_init(bar_empty + 8 * s, NDW);
+            mbar_init(bar_empty + 8 * s, NDW);            // the dense warps of one group
         }
+        for (int i = 0; i < 2 * NDW; ++i) mbar_init(bar_xfull + 8 * i, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -957,10 +961,14 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + BN / 32), 1) fq_mma_kern
             if (blockIdx.x == 0 && lane == 0 && aw == 0) { g_trace[10] += tw1 - tw0; g_trace[11] += clock64() - tw1; g_trace[12] += 1; }
 #endif
         }
-    } else if (warp >= DW0 && warp < DW0 + NDW) {
+    } else if (warp >= DW0 && warp < DW0 + NGRP * NDW) {
         // ------------------------------------------------------------------ dense warps (all alike)
-        const int dw = warp - DW0, g = lane >> 2, t = lane & 3;
-        [[maybe_unused]] const int dtid = dw * 32 + lane;   // tracing builds only
+        // Two groups of NDW warps take alternate units, each with accumulators of its own: twice the
+        // warps to hide latencies with, and no warp does less work per unit it takes.  At the end of
+        // a piece group 1 hands its sums to group 0 through shared memory.
+        const int dwi = warp - DW0, grp = dwi / NDW, dw = dwi % NDW, g = lane >> 2, t = lane & 3;
+        [[maybe_unused]] const int dtid = dwi * 32 + lane;   // tracing builds only
+        float* xch = reinterpret_cast<float*>(smem + p.off_shc) + dw * (MO * CG * 4 * 32) + lane;
         const int c0 = dw * 32 + g;                           // this lane's columns: c0 + 8 * {0, 1, 2, 3}
         float accf[MO][CG][4];
 #pragma unroll
@@ -978,6 +986,7 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + BN / 32), 1) fq_mma_kern
         for (UnitIter w(u_begin, KT); w.u < u_end && ok; w.next(S, KT)) {
             const uint32_t u = w.u, s = w.s, ph = w.ph, tn = w.tn, kt = w.kt;
             const uint8_t* st = smem + s * p.stage_bytes;
+            if ((w.it % NGRP) == (uint32_t)grp) {
 #ifdef FQ_TRACE
             long long tw0 = clock64();
 #endif
@@ -1150,6 +1159,7 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + BN / 32), 1) fq_mma_kern
 #ifdef FQ_TRACE
             if (blockIdx.x == 0 && dtid == 0) { g_trace[13] += tw1 - tw0; g_trace[14] += clock64() - tw1; g_trace[15] += 1; }
 #endif
+            }
 
             if (kt == KT - 1 || u == u_end - 1) {
                 // ---------------------------------------------------------- end of a piece
@@ -1163,6 +1173,34 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + BN / 32), 1) fq_mma_kern
                         if (t == 0) accf[0][c >> 1][2 * (c & 1)] += v;
                     }
                     sacc[0][0] = 0.0f;
+                }
+                if (NGRP > 1) {
+                    if (grp == 1) {
+                        // hand the sums over (after group 0 has taken the previous piece's) and start afresh
+                        if (piece > 0 && !warp_wait(bar_xempty + 8 * dw, (piece - 1) & 1, abort_flag, p.status)) { ok = false; break; }
+#pragma unroll
+                        for (int o = 0; o < MO; ++o)
+#pragma unroll
+                            for (int cg = 0; cg < CG; ++cg)
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) {
+                                    xch[((o * CG + cg) * 4 + i) * 32] = accf[o][cg][i];
+                                    accf[o][cg][i] = 0.0f;
+                                }
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar_xfull + 8 * dw);
+                        ++piece;
+                        continue;
+                    }
+                    if (!warp_wait(bar_xfull + 8 * dw, piece & 1, abort_flag, p.status)) { ok = false; break; }
+#pragma unroll
+                    for (int o = 0; o < MO; ++o)
+#pragma unroll
+                        for (int cg = 0; cg < CG; ++cg)
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) accf[o][cg][i] += xch[((o * CG + cg) * 4 + i) * 32];
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_xempty + 8 * dw);
                 }
                 const uint32_t u_tile0 = tn * KT;
                 const uint32_t piece_k0 = max(u_tile0, u_begin) - u_tile0;
@@ -1303,6 +1341,7 @@ __global__ void __launch_bounds__(256) fq_spmm_kernel(const uint16_t* __restrict
 struct Plan {
     Params p;
     uint32_t threads, smem, grid;
+    uint32_t ngrp;   // small-batch kernel: groups of dense warps
 };
 
 static inline uint32_t round_up(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
@@ -1377,7 +1416,15 @@ static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, 
     p.M = M; p.K = L->K; p.N = L->N; p.KT = L->K / kBK; p.NT = L->N / BN; p.NB = NB; p.nsw = 0;
     const uint32_t w_bytes = 16 * BN * 4, sz_bytes = 2 * GPS * BN * 2;
     const uint32_t xt_bytes = sparse ? MO * 4096 : 0;     // FP32 [octet][k][8]
-    const uint32_t fixed = 1024;
+    // Two groups of dense warps (each takes every other unit) pay off when a CTA has enough units to
+    // stream and the accumulators are small; short jobs and 16-row batches keep one group.
+    const int sms = sm_count_cached();
+    if (sms <= 0) return fail(FQ_ERR_CUDA, "no CUDA device: %s", cudaGetErrorString(cudaGetLastError()));
+    const uint32_t grid = std::min<uint32_t>({(uint32_t)sms, kMaxCtas, (L->N / BN) * (L->K / kBK)});
+    const uint32_t units_per_cta = ((L->N / BN) * (L->K / kBK) + grid - 1) / grid;
+    pl.ngrp = (MO == 1 && units_per_cta >= 8) ? 2 : 1;
+    const uint32_t xch_bytes = pl.ngrp > 1 ? BN * ROWS * 4 : 0;   // hand-over of a group's partial sums
+    const uint32_t fixed = 1024 + xch_bytes;
     const uint32_t budget = kSmemBudget;
     uint32_t cap = 0;
     if (sparse) {
@@ -1400,34 +1447,38 @@ static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, 
     if (S < 3) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "shared-memory stages do not fit");
     p.coo_cap = cap; p.stages = S; p.stage_bytes = stage;
     p.off_shc = S * stage;
-    p.off_bar = p.off_shc;
+    p.off_bar = p.off_shc + xch_bytes;
     pl.smem = p.off_bar + 1024;
-    pl.threads = 32 * (1 + kActWarps + NDW);
-    const int sms = sm_count_cached();
-    if (sms <= 0) return fail(FQ_ERR_CUDA, "no CUDA device: %s", cudaGetErrorString(cudaGetLastError()));
-    pl.grid = std::min<uint32_t>({(uint32_t)sms, kMaxCtas, p.NT * p.KT});
+    pl.threads = 32 * (1 + kActWarps + pl.ngrp * NDW);
+    pl.grid = grid;
     return FQ_OK;
 }
 
 typedef void (*KernelFn)(const Params);
 
-// MS: form of the outlier step (1: single batch row, one column per lane; 8: rows split over the lanes)
+// MS: form of the outlier step (1: single batch row, one column per lane; 8: rows split over the lanes);
+// NGRP: groups of dense warps (two only with one octet of rows)
 template <int BN, int MO, int G>
-static KernelFn pick_mma_sparse(bool sparse, uint32_t ms) {
-    if (!sparse) return (KernelFn)fq_mma_kernel<BN, MO, G, false, 8>;
+static KernelFn pick_mma_sparse(bool sparse, uint32_t ms, uint32_t ngrp) {
     if constexpr (MO == 1) {
-        if (ms == 1) return (KernelFn)fq_mma_kernel<BN, MO, G, true, 1>;
+        if (ngrp == 2) {
+            if (!sparse) return (KernelFn)fq_mma_kernel<BN, MO, G, false, 8, 2>;
+            if (ms == 1) return (KernelFn)fq_mma_kernel<BN, MO, G, true, 1, 2>;
+            return (KernelFn)fq_mma_kernel<BN, MO, G, true, 8, 2>;
+        }
+        if (sparse && ms == 1) return (KernelFn)fq_mma_kernel<BN, MO, G, true, 1, 1>;
     }
-    return (KernelFn)fq_mma_kernel<BN, MO, G, true, 8>;
+    if (!sparse) return (KernelFn)fq_mma_kernel<BN, MO, G, false, 8, 1>;
+    return (KernelFn)fq_mma_kernel<BN, MO, G, true, 8, 1>;
 }
 template <int BN, int MO>
-static KernelFn pick_mma_group(uint32_t g, bool sparse, uint32_t ms) {
-    return g == 64 ? pick_mma_sparse<BN, MO, 64>(sparse, ms) : pick_mma_sparse<BN, MO, 128>(sparse, ms);
+static KernelFn pick_mma_group(uint32_t g, bool sparse, uint32_t ms, uint32_t ngrp) {
+    return g == 64 ? pick_mma_sparse<BN, MO, 64>(sparse, ms, ngrp) : pick_mma_sparse<BN, MO, 128>(sparse, ms, ngrp);
 }
-static KernelFn pick_mma_kernel(uint32_t bn, uint32_t M, uint32_t g, bool sparse) {
+static KernelFn pick_mma_kernel(uint32_t bn, uint32_t M, uint32_t g, bool sparse, uint32_t ngrp) {
     const uint32_t mo = M <= 8 ? 1 : 2, ms = M <= 1 ? 1 : 8;
-    if (bn == 128) return mo == 1 ? pick_mma_group<128, 1>(g, sparse, ms) : pick_mma_group<128, 2>(g, sparse, ms);
-    return mo == 1 ? pick_mma_group<256, 1>(g, sparse, ms) : pick_mma_group<256, 2>(g, sparse, ms);
+    if (bn == 128) return mo == 1 ? pick_mma_group<128, 1>(g, sparse, ms, ngrp) : pick_mma_group<128, 2>(g, sparse, ms, ngrp);
+    return mo == 1 ? pick_mma_group<256, 1>(g, sparse, ms, ngrp) : pick_mma_group<256, 2>(g, sparse, ms, ngrp);
 }
 
 static uint32_t mma_max_rows() {
@@ -1516,7 +1567,7 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
         p.status = (uint32_t*)workspace;
         p.counters = (uint32_t*)((uint8_t*)workspace + kWsHeaderBytes);
         p.partials = (float*)((uint8_t*)workspace + kWsHeaderBytes + kWsCounterBytes);
-        KernelFn fn = use_mma ? pick_mma_kernel(L->BN, mb, L->group, sparse)
+        KernelFn fn = use_mma ? pick_mma_kernel(L->BN, mb, L->group, sparse, pl.ngrp)
                               : pick_kernel(L->BN, nb16_of(mb), L->group, sparse);
         cudaError_t e = ensure_smem_attr((const void*)fn, (int)kSmemBudget);
         if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));

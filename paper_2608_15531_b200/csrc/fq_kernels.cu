@@ -72,6 +72,8 @@ struct Params {
     float* partials;
     uint32_t M, K, N, KT, NT;
     uint32_t NB, coo_cap, stages, nsw;
+    uint32_t split;   // small-batch kernel: 0 = units dealt out as one contiguous range per CTA (stream-K);
+                      // c > 0 = every column tile belongs to c CTAs, CTA b takes part b mod c of tile b / c
     // shared-memory offsets (bytes); the first five are relative to a stage
     uint32_t stage_bytes, off_sz, off_xcan, off_xsum, off_info, off_coo;
     uint32_t off_shc, off_xt, off_bar;
@@ -810,10 +812,18 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (warp != 0) asm volatile("griddepcontrol.wait;" ::: "memory");
 
-    const uint32_t U = p.NT * p.KT, P = gridDim.x, q = U / P, r = U % P;
-    const uint32_t u_begin = unit_begin_of(blockIdx.x, q, r);
-    const uint32_t u_end = u_begin + q + (blockIdx.x < r ? 1u : 0u);
     const uint32_t KT = p.KT;
+    const uint32_t U = p.NT * KT, P = gridDim.x, q = U / P, r = U % P;
+    uint32_t u_begin, u_end;
+    if (p.split) {
+        // tile-aligned split: no CTA works on two tiles, so none settles two split tiles one after the other
+        const uint32_t tile = blockIdx.x / p.split, part = blockIdx.x - tile * p.split;
+        u_begin = tile * KT + part * KT / p.split;
+        u_end = tile * KT + (part + 1) * KT / p.split;
+    } else {
+        u_begin = unit_begin_of(blockIdx.x, q, r);
+        u_end = u_begin + q + (blockIdx.x < r ? 1u : 0u);
+    }
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer
@@ -1211,7 +1221,7 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                     // barriers: FP32 partial in fragment order, then one arrival per (tile, strip);
                     // the last warp to arrive adds the partials in CTA order (the same order in
                     // every run) and writes Y.
-                    const uint32_t which = (u_begin / KT == tn) ? 0u : 1u;
+                    const uint32_t which = (p.split || u_begin / KT == tn) ? 0u : 1u;
                     float* slot = p.partials + ((size_t)blockIdx.x * 2 + which) * (size_t)(BN * LDC) + dw * (32 * LDC) + lane;
 #pragma unroll
                     for (int o = 0; o < MO; ++o)
@@ -1220,7 +1230,8 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
 #pragma unroll
                             for (int i = 0; i < 4; ++i) __stcg(slot + ((o * CG + cg) * 4 + i) * 32, accf[o][cg][i]);
                     __syncwarp();
-                    const uint32_t c_first = cta_of_unit(u_tile0, q, r), c_last = cta_of_unit(u_tile0 + KT - 1, q, r);
+                    const uint32_t c_first = p.split ? tn * p.split : cta_of_unit(u_tile0, q, r);
+                    const uint32_t c_last = p.split ? c_first + p.split - 1 : cta_of_unit(u_tile0 + KT - 1, q, r);
                     uint32_t last = 0;
                     if (lane == 0) {
                         __threadfence();                       // the warp's stores, ordered before the arrival
@@ -1244,7 +1255,7 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
 #pragma unroll
                             for (int d = 0; d < 4; ++d) {
                                 const uint32_t cc = min(c + d, c_last);
-                                const uint32_t wch = (unit_begin_of(cc, q, r) / KT == tn) ? 0u : 1u;
+                                const uint32_t wch = (p.split || unit_begin_of(cc, q, r) / KT == tn) ? 0u : 1u;
                                 const float* sl = p.partials + ((size_t)cc * 2 + wch) * (size_t)(BN * LDC) + dw * (32 * LDC) + lane;
 #pragma unroll
                                 for (int e = 0; e < MO * CG * 4; ++e) v[d][e] = __ldcg(sl + e * 32);
@@ -1420,8 +1431,21 @@ static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, 
     // stream and the accumulators are small; short jobs and 16-row batches keep one group.
     const int sms = sm_count_cached();
     if (sms <= 0) return fail(FQ_ERR_CUDA, "no CUDA device: %s", cudaGetErrorString(cudaGetLastError()));
-    const uint32_t grid = std::min<uint32_t>({(uint32_t)sms, kMaxCtas, (L->N / BN) * (L->K / kBK)});
-    const uint32_t units_per_cta = ((L->N / BN) * (L->K / kBK) + grid - 1) / grid;
+    const uint32_t NT = L->N / BN, KT = L->K / kBK;
+    uint32_t grid = std::min<uint32_t>({(uint32_t)sms, kMaxCtas, NT * KT});
+    uint32_t units_per_cta = (NT * KT + grid - 1) / grid;
+    // Tile-aligned split instead of one contiguous range per CTA when it costs at most one more unit
+    // per CTA: then no CTA has to settle two split tiles in a row.
+    uint32_t split = 0;
+    if (NT <= grid) {
+        const uint32_t c = std::min<uint32_t>(grid / NT, KT);
+        if (c >= 2 && (KT + c - 1) / c <= units_per_cta + 1) {
+            split = c;
+            grid = NT * c;
+            units_per_cta = (KT + c - 1) / c;
+        }
+    }
+    p.split = split;
     pl.ngrp = (MO == 1 && units_per_cta >= 8) ? 2 : 1;
     const uint32_t xch_bytes = pl.ngrp > 1 ? BN * ROWS * 4 : 0;   // hand-over of a group's partial sums
     const uint32_t fixed = 1024 + xch_bytes;
@@ -1571,7 +1595,7 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
                               : pick_kernel(L->BN, nb16_of(mb), L->group, sparse);
         cudaError_t e = ensure_smem_attr((const void*)fn, (int)kSmemBudget);
         if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-        if (use_mma && overlap_launches()) {
+        if (use_mma) {
             // Programmatic dependent launch: this grid may become resident while the kernel before it
             // in the stream drains.  Its producer warp then already streams weights (which no kernel
             // writes); every other warp first executes griddepcontrol.wait, after which all memory
@@ -1582,12 +1606,16 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
             cfg.blockDim = dim3(pl.threads);
             cfg.dynamicSmemBytes = pl.smem;
             cfg.stream = (cudaStream_t)stream;
-            cudaLaunchAttribute attr;
-            std::memset(&attr, 0, sizeof(attr));
-            attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
-            attr.val.programmaticStreamSerializationAllowed = 1;
-            cfg.attrs = &attr;
-            cfg.numAttrs = 1;
+            cudaLaunchAttribute attr[1];
+            std::memset(attr, 0, sizeof(attr));
+            unsigned n = 0;
+            if (overlap_launches()) {
+                attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+                attr[n].val.programmaticStreamSerializationAllowed = 1;
+                ++n;
+            }
+            cfg.attrs = attr;
+            cfg.numAttrs = n;
             e = cudaLaunchKernelEx(&cfg, fn, p);
             if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
         } else {

@@ -127,9 +127,6 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volat
     uint32_t spins = 0;
     unsigned long long t0 = 0;
     while (!mbar_try_wait(bar, parity)) {
-#ifdef FQ_SLEEP_NS
-        __nanosleep(FQ_SLEEP_NS);
-#endif
         if ((++spins & 0xff) == 0) {
             if (*abort_flag) return false;
             unsigned long long now = globaltimer_ns();
@@ -473,12 +470,7 @@ __global__ void __launch_bounds__(32 * (4 + 2 * (BN / 32) + 4), 1) fq_fused_kern
 #pragma unroll
             for (int c = 0; c < CPL; ++c) {
                 nxt[c] = make_uint4(0, 0, 0, 0);
-#if defined(FQ_EXP) && FQ_EXP == 11
-                if (false)
-#else
-                if (real)
-#endif
-                    nxt[c] = __ldg(reinterpret_cast<const uint4*>(xrow + (size_t)kt * 256 + c * 16));
+                if (real) nxt[c] = __ldg(reinterpret_cast<const uint4*>(xrow + (size_t)kt * 256 + c * 16));
             }
         };
         if (u_begin < u_end) load(u_begin - (u_begin / KT) * KT);
@@ -853,31 +845,13 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
             const uint32_t full = bar_full + 8 * s;
             const uint32_t st = smem_u32(smem) + s * p.stage_bytes;
             if (lane == 0) {
-#if defined(FQ_EXP) && FQ_EXP == 25
-                uint32_t bytes = W_BYTES;
-#else
                 uint32_t bytes = W_BYTES + 2 * GPS * SZ_ROW;
-#endif
                 if (SPARSE) bytes += p.NB * 4 + npk * 16;
                 mbar_arrive_expect_tx(full, bytes);
             }
             __syncwarp();
-#ifdef FQ_WSPLIT
-            if (lane < FQ_WSPLIT) {
-                constexpr int PART = W_BYTES / FQ_WSPLIT;
-                bulk_g2s(st + lane * PART, p.wq + (size_t)u * W_BYTES + lane * PART, PART, full);
-            } else if (lane < FQ_WSPLIT + 2 * GPS) {
-                const int i = lane - FQ_WSPLIT, gi = i >> 1;
-                const size_t row = (size_t)(kt * GPS + gi) * p.N + (size_t)tn * BN;
-                if (i & 1) bulk_g2s(st + p.off_sz + (GPS + gi) * SZ_ROW, p.zero + row, SZ_ROW, full);
-                else bulk_g2s(st + p.off_sz + gi * SZ_ROW, p.scale + row, SZ_ROW, full);
-            } else if (lane == 31) {
-#else
             if (lane == 0) {
                 bulk_g2s(st, p.wq + (size_t)u * W_BYTES, W_BYTES, full);
-#if defined(FQ_EXP) && FQ_EXP == 25
-                if (false)
-#endif
 #pragma unroll
                 for (int gi = 0; gi < GPS; ++gi) {
                     const size_t row = (size_t)(kt * GPS + gi) * p.N + (size_t)tn * BN;
@@ -885,7 +859,6 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                     bulk_g2s(st + p.off_sz + (GPS + gi) * SZ_ROW, p.zero + row, SZ_ROW, full);
                 }
             } else if (lane == 1) {
-#endif
                 if (SPARSE) {
                     bulk_g2s(st + p.off_info, p.info + (size_t)u * p.NB, p.NB * 4, full);
                     if (npk) bulk_g2s(st + p.off_coo, p.packed + pk0, npk * 16, full);
@@ -912,12 +885,7 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
 #pragma unroll
             for (int c = 0; c < CPL; ++c) {
                 nxt[c] = make_uint4(0, 0, 0, 0);
-#if defined(FQ_EXP) && FQ_EXP == 11
-                if (false)
-#else
-                if (real)
-#endif
-                    nxt[c] = __ldg(reinterpret_cast<const uint4*>(xrow + (size_t)kt * 256 + c * 16));
+                if (real) nxt[c] = __ldg(reinterpret_cast<const uint4*>(xrow + (size_t)kt * 256 + c * 16));
             }
         };
         if (u_begin + aw < u_end) load((u_begin + aw) % KT);
@@ -1043,9 +1011,6 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                 pk1 = packet(1);
                 if constexpr (MS == 8) fetch_x(pk0, xa);
             }
-#if defined(FQ_EXP) && (FQ_EXP == 24 || FQ_EXP == 25)
-            if (false)
-#endif
 #pragma unroll
             for (int gi = 0; gi < GPS; ++gi) {
                 float accg[MO][CG][4];
@@ -1063,23 +1028,14 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
 #pragma unroll
                     for (int cg = 0; cg < CG; ++cg) {
                         const uint32_t wa = wp[j * BN * 4 + cg * 64], wb = wp[j * BN * 4 + cg * 64 + 32];   // columns +0 and +8
-#if defined(FQ_EXP) && FQ_EXP == 22
-                        const uint32_t a0 = wa, a1 = wa ^ 1, a2 = wa ^ 2, a3 = wa ^ 3, b0 = wb, b1 = wb ^ 1, b2 = wb ^ 2, b3 = wb ^ 3;
-#else
                         const uint32_t a0 = codes_to_bf16x2(wa), a1 = codes_to_bf16x2(wa >> 4);
                         const uint32_t a2 = codes_to_bf16x2(wa >> 8), a3 = codes_to_bf16x2(wa >> 12);
                         const uint32_t b0 = codes_to_bf16x2(wb), b1 = codes_to_bf16x2(wb >> 4);
                         const uint32_t b2 = codes_to_bf16x2(wb >> 8), b3 = codes_to_bf16x2(wb >> 12);
-#endif
 #pragma unroll
                         for (int o = 0; o < MO; ++o) {
-#if defined(FQ_EXP) && FQ_EXP == 21
-                            accg[o][cg][0] += __uint_as_float((a0 ^ b0 ^ a1 ^ b1 ^ xb[o].x ^ xb[o].y) & 0x3fffffffu);
-                            accg[o][cg][1] += __uint_as_float((a2 ^ b2 ^ a3 ^ b3 ^ xb[o].z ^ xb[o].w) & 0x3fffffffu);
-#else
                             mma_bf16(accg[o][cg], a0, b0, a1, b1, xb[o].x, xb[o].y);   // rows 8t+0..3 of the block
                             mma_bf16(accg[o][cg], a2, b2, a3, b3, xb[o].z, xb[o].w);   // rows 8t+4..7
-#endif
                         }
                     }
                 }
@@ -1087,15 +1043,6 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                 float2 xs[MO];
 #pragma unroll
                 for (int o = 0; o < MO; ++o) xs[o] = *reinterpret_cast<const float2*>(xsum + gi * LDC + o * 8 + 2 * t);
-#if defined(FQ_EXP) && FQ_EXP == 23
-#pragma unroll
-                for (int cg = 0; cg < CG; ++cg)
-#pragma unroll
-                    for (int o = 0; o < MO; ++o)
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) accf[o][cg][i] += accg[o][cg][i] * xs[o].x;
-                if (false)
-#endif
 #pragma unroll
                 for (int cg = 0; cg < CG; ++cg)
 #pragma unroll

@@ -34,8 +34,8 @@ CONFIG_ID = 2                      # the LLaMA-3-8B layer set
 L2_COVER_BYTES = 400 << 20         # rotating copies per layer cover at least this (L2 is 126 MB)
 METRIC = "effective_hbm_gbs_fused_w4a16_outlier_gemm_m1_8_16"
 # dram__bytes_read + dram__bytes_write of the fused kernel over its algorithmic bytes, from the ncu
-# captures summarised in profiles/fq_fused_kernel_llama3_8b_decode_set.md (1.02 and 1.04 on the two
-# launches captured); scaled to the average launch of the step.
+# captures summarised in profiles/fq_mma_kernel_llama3_8b_decode_set.md (1.02 to 1.04 on the three
+# launches captured: the packet padding); scaled to the average launch of the step.
 NCU_TRAFFIC_RATIO = 1.03
 
 

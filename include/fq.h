@@ -33,9 +33,9 @@
  *   h = 0..1; bits 4p..4p+3) of that word is the code of
  *       column tn*BN + t
  *       row    kt*128 + 32j + 8w + 2i + h .
- *   (One thread owns one column: four 16-byte loads give its 128 codes of the
- *   tile, and one shift-and-mask turns nibbles i and i+4 into a BF16 pair of
- *   consecutive rows, which is the tensor-memory operand order.)
+ *   (The four words of one column and one 32-row block are 16 contiguous
+ *   bytes, and one shift-and-mask turns nibbles i and i+4 of a word into a BF16
+ *   pair of consecutive rows: the operand order of both tensor-core paths.)
  *
  *   Scale, zero.  (K/group) x N row-major BF16.  zero holds the integer 0..15.
  *
@@ -43,13 +43,18 @@
  *   tile_indptr[t] .. tile_indptr[t+1]: the tile's range of 16-byte packets in
  *   packed_outliers (N_tile + 1 entries, uint32).  bucket_info[t*NB + b] =
  *   offset | count << 16 (two uint16): bucket b of tile t owns `count` packets
- *   starting `offset` packets after the tile's first.  Buckets of one tile own
- *   disjoint column sets, and column c only ever appears in buckets
- *   32*(c mod NB/32) .. 32*(c mod NB/32)+31 (one block of 32 buckets per sparse warp).  A packet holds four outliers: bytes 0-3 row index in
- *   the tile, bytes 4-7 column index in the tile, bytes 8-15 four BF16 values.
- *   A slot with value bits 0x0000 is padding and is skipped (its row byte is 0
- *   and its column byte is BN-1-slot).  Storage: (N_tile+1)*4 + N_tile*NB*4 +
- *   16*packets bytes.
+ *   starting `offset` packets after the tile's first.  NB = BN/4, and the
+ *   bucket of tile column c is fixed: 8*(c/32) + c%8, i.e. the four columns
+ *   {g, g+8, g+16, g+24} of a 32-column block share a bucket.  (These are the
+ *   columns whose accumulators one group of four lanes holds after the
+ *   m16n8k16 MMAs of the small-batch kernel, so a bucket is applied in
+ *   registers; the paper's load-balancing column permutation, Section 3.2.2, is
+ *   replaced by this static assignment.)  A packet holds four outliers: bytes
+ *   0-3 row index in the tile, bytes 4-7 column index in the tile, bytes 8-15
+ *   four BF16 values.  Inside a bucket the entries are stored by (row, column);
+ *   the last packet is filled up with padding slots: value bits 0x0000, row 0,
+ *   the bucket's first column.  Every slot, padding included, has row < 128 and
+ *   column < BN.  Storage: (N_tile+1)*4 + N_tile*NB*4 + 16*packets bytes.
  */
 #ifndef FQ_H_
 #define FQ_H_
@@ -82,16 +87,18 @@ typedef struct fq_layout {
     uint32_t group;            /* 64 or 128, along K */
     uint32_t BK;               /* 128 */
     uint32_t BN;               /* 128 or 256 */
-    uint32_t buckets_per_tile; /* NB: 32, 64 or 128 */
+    uint32_t buckets_per_tile; /* NB = BN / 4 */
     uint32_t wq_interleave;    /* 2: the column-per-thread order described above */
     uint32_t coo_unit_bytes;   /* 16 */
     uint32_t max_tile_packets; /* largest tile of the encoded W_O, in packets; 0 = not encoded */
     uint32_t reserved[6];
 } fq_layout_t;
 
-/* Choose tile sizes for a K x N layer.  bn_hint / nb_hint: 0 = library default,
- * otherwise BN in {128, 256} and NB in {32, 64, 128}.  Errors:
- * FQ_ERR_UNSUPPORTED_SHAPE for shapes the kernel cannot tile. */
+/* Choose tile sizes for a K x N layer.  bn_hint: 0 = library default (256 when
+ * N is a multiple of 256), otherwise 128 or 256.  nb_hint: 0, or BN/4 (the only
+ * bucket count there is).  Errors: FQ_ERR_UNSUPPORTED_SHAPE for shapes the
+ * kernels cannot tile (K % 128, N % BN, group not 64 or 128, more than 1024
+ * column tiles). */
 fq_status_t fq_get_layout(uint32_t K, uint32_t N, uint32_t group, uint32_t bn_hint, uint32_t nb_hint,
                           fq_layout_t* out);
 
@@ -118,16 +125,12 @@ fq_status_t fq_pack_int4(const fq_layout_t* L, const float* W, const uint8_t* ou
 fq_status_t fq_unpack_int4(const fq_layout_t* L, const void* wq, uint8_t* q_canon);
 
 /*
- * Tile-COO encoder (Section 3.2.1; column reordering and element reordering of
- * Section 3.2.2).  Input: COO triplets on the host (k, n, BF16 value bits), any
- * order; entries whose value is +-0 are dropped.  Per tile and per block of 32
- * buckets (block of column c = c mod NB/32), columns are sorted by outlier count
- * (descending) and assigned greedily to the least-loaded bucket of the block; inside a bucket, entries are ordered so that the four slots of a
- * packet hold different columns while four columns still have entries, and,
- * among those, position i of bucket b prefers shared-memory bank group
- * (i + b) mod 8 of the kernel's activation copy (bank group of row k = k mod 8),
- * falling through to the next group in circular order; buckets are padded to
- * whole packets.
+ * Tile-COO encoder (Section 3.2.1).  Input: COO triplets on the host (k, n,
+ * BF16 value bits), any order; entries whose value is +-0 are dropped.  Every
+ * entry goes to the bucket of its column (see "Tile-COO" above); a bucket's
+ * entries are stored by (row, column), four to a packet, the last packet padded.
+ * The column and element reordering of Section 3.2.2 serve a shared-memory
+ * scatter that the kernels here do not have, so they are not applied.
  *
  * fq_encode_tilecoo_sizes: element counts of the three arrays (tile_indptr in
  * uint32, bucket_info in uint32, packets in 16-byte units) and the largest
@@ -147,8 +150,9 @@ fq_status_t fq_decode_tilecoo(const fq_layout_t* L, const uint32_t* tile_indptr,
                               uint32_t* n, uint16_t* val_bf16, size_t* nnz_inout);
 
 /* Structural check of host Tile-COO arrays before they are given to a kernel:
- * monotone indptr ending at n_packets, bucket ranges inside their tile, indices
- * inside the tile, bucket column sets disjoint.  FQ_ERR_FORMAT on violation. */
+ * monotone indptr ending at n_packets, bucket ranges inside their tile, every
+ * slot's indices inside the tile, every outlier in the bucket of its column.
+ * FQ_ERR_FORMAT on violation. */
 fq_status_t fq_validate_tilecoo(const fq_layout_t* L, const uint32_t* tile_indptr,
                                 const uint32_t* bucket_info, const void* packed_outliers,
                                 size_t n_packets);
@@ -164,14 +168,26 @@ fq_status_t fq_workspace_bytes(const fq_layout_t* L, uint32_t M, size_t* bytes);
 /*
  * The fused operator (Eq. 1; Sections 3.1 and 4.1): one launch per 32 rows of X
  * reads X, W_Q and the Tile-COO tiles through a bulk-copy/mbarrier ring,
- * dequantises in registers into the tensor-memory operand of tcgen05 MMAs,
- * applies the tile's outliers against the same shared-memory activation tile,
- * and writes Y once.
+ * dequantises in registers into tensor-core operands, applies the tile's
+ * outliers against the same shared-memory activation tile, and writes Y once.
+ * Up to 16 rows run the small-batch kernel (warp-level MMAs, outliers added in
+ * registers), more rows the tcgen05 kernel (tensor-memory operand, outliers
+ * through a shared-memory FP32 tile).
  * X: device, M x K BF16.  M in [1, FQ_MAX_M].  Y: device, M x N BF16,
  * overwritten.  All other arrays: device copies of the host packer/encoder
- * output.  Work is split over persistent CTAs by contiguous ranges of (tile,
- * k-step) units; tiles shared by several CTAs are summed in a fixed order, so
- * results are run-to-run reproducible.
+ * output.  Work is split over persistent CTAs by (tile, k-step) units; tiles
+ * shared by several CTAs are summed in a fixed order, so results are run-to-run
+ * reproducible.
+ *
+ * Ordering.  The small-batch kernel is launched so that it may become resident
+ * while the kernel before it in the stream is still draining (programmatic
+ * dependent launch): it then already streams the weight arrays (wq, scale,
+ * zero, tile_indptr, bucket_info, packed_outliers), and touches X, Y and the
+ * scratch only after that earlier kernel has completed.  So the weight arrays
+ * must not be written by a kernel that can still be running when this call is
+ * made (they are constants of the layer in any real use); every other
+ * dependency through the stream is honoured as usual.  Environment variable
+ * FQ_PDL=0 restores plain stream order.
  */
 fq_status_t fq_fused_w4a16_outlier_gemm(const fq_layout_t* L, const void* X, uint32_t M,
                                         const void* wq, const void* scale, const void* zero,

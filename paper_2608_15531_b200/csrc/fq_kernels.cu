@@ -768,6 +768,8 @@ template <int BN, int MO, int GROUP, bool SPARSE, int MS, int NGRP>
 __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq_mma_kernel(const Params p) {
     constexpr int NDW = BN / 32;
     constexpr int NA = kActWarps;                           // activation warps: warp a takes the units it with it mod NA == a
+    // (the number of stages is a multiple of NA and of NGRP, so that a stage always returns to the same
+    // activation warp and dense group: each of them then sees every phase of the stage's barriers)
     constexpr int DW0 = 1 + NA;                             // first dense warp
     // NGRP dense warp groups: group r takes the units it with it mod NGRP == r
     constexpr int CG = 2;                                   // 16-column MMA strips per warp
@@ -1411,11 +1413,14 @@ static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, 
         p.off_info = p.off_xt + xt_bytes;
         p.off_coo = p.off_info + (sparse ? round_up(NB * 4, 128) : 0);
         stage = round_up(p.off_coo + cap * 16, 128);
-        S = std::min<uint32_t>(8, (budget - fixed) / stage);
+        // An even number of stages: the activation warps and the dense groups take alternate units, and
+        // a parity wait is only valid for a waiter that meets every phase of the barrier.  With S even a
+        // stage always comes back to the same activation warp and the same dense group.
+        S = std::min<uint32_t>(8, (budget - fixed) / stage) & ~1u;
         if (S >= 4 || cap <= 64) break;
         cap = std::max<uint32_t>(64, cap / 2);
     }
-    if (S < 3) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "shared-memory stages do not fit");
+    if (S < 4) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "shared-memory stages do not fit");
     p.coo_cap = cap; p.stages = S; p.stage_bytes = stage;
     p.off_shc = S * stage;
     p.off_bar = p.off_shc + xch_bytes;

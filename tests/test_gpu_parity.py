@@ -213,3 +213,64 @@ def test_full_size_layers_on_sampled_columns(name, cfg, idx, K, N):
         assert np.all(np.isfinite(H.bits_to_f64(Y)))
         H.check_tolerances(Y[:, cols], Yref, Yabs, K)
     del BN
+
+
+def _sample_cols(lay, N, seed, n_random=64):
+    """First and last columns, random ones, and the columns richest in outliers."""
+    rng = np.random.default_rng(seed)
+    return np.unique(np.concatenate([np.arange(0, 8), np.arange(N - 8, N), rng.integers(0, N, n_random),
+                                     np.argsort(lay.mask.sum(axis=0))[::-1][:8]])).astype(np.uint32)
+
+
+# ------------------------------------------------------------------ outlier-density sweep (configuration 3)
+
+@pytest.mark.parametrize("layout", ["uniform", "clustered"])
+@pytest.mark.parametrize("density", [0.0, 0.005, 0.01, 0.02, 0.05])
+def test_density_sweep_on_sampled_columns(density, layout):
+    K, N, g, M = 4096, 14336, 128, 8
+    if density == 0.0 and layout == "clustered":
+        pytest.skip("no outliers: one layout is enough")
+    lay = synth.layer(synth.tensor_seed(3, int(density * 1000) + (layout == "clustered")), K, N, density=density,
+                      layout=layout)
+    P = H.pack_layer(lay, g)
+    cols = _sample_cols(lay, N, 3)
+    X = _x(lay.seed, M, K)
+    Y = H.run_fused(P, X)
+    Yref, Yabs = H.oracle_result(P, X, cols=cols)
+    H.check_tolerances(Y[:, cols], Yref, Yabs, K)
+    # the unfused pair computes the same thing (one more BF16 rounding of the dense half)
+    Yu = H.run_unfused(P, X)
+    Yd, _ = H.oracle_result(P, X, cols=cols, dense_only=True)
+    bound = 2.0 ** -8 * (np.abs(Yd) + np.abs(Yref)) + K * 2.0 ** -24 * Yabs
+    assert np.all(np.abs(H.bits_to_f64(Yu[:, cols]) - Yref) <= bound)
+
+
+# ------------------------------------------------------------------ LLaMA-3-70B shapes (configuration 4)
+
+@pytest.mark.parametrize("idx", range(len(synth.LLAMA3_70B)))
+def test_llama3_70b_layers_on_sampled_columns(idx):
+    name, K, N = synth.LLAMA3_70B[idx]
+    g = 128
+    lay = synth.layer(synth.tensor_seed(4, idx), K, N, density=0.01, layout="mixed")
+    P = H.pack_layer(lay, g)
+    cols = _sample_cols(lay, N, idx, n_random=48)
+    for M in (1, 4, 16, 32):
+        X = _x(lay.seed, M, K)
+        Y = H.run_fused(P, X)
+        Yref, Yabs = H.oracle_result(P, X, cols=cols)
+        H.check_tolerances(Y[:, cols], Yref, Yabs, K)
+
+
+# ------------------------------------------------------------------ batch transition sweep (configuration 5)
+
+@pytest.mark.parametrize("g", [64, 128])
+def test_batch_transition_sweep_on_sampled_columns(g):
+    K, N = 8192, 28672
+    lay = synth.layer(synth.tensor_seed(5, g), K, N, density=0.01, layout="mixed")
+    P = H.pack_layer(lay, g)
+    cols = _sample_cols(lay, N, g, n_random=40)
+    for M in (1, 2, 4, 8, 16, 32, 64, 128):
+        X = _x(lay.seed, M, K)
+        Y = H.run_fused(P, X)
+        Yref, Yabs = H.oracle_result(P, X, cols=cols)
+        H.check_tolerances(Y[:, cols], Yref, Yabs, K)

@@ -1253,46 +1253,59 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
 
 // ----------------------------------------------------------------------------- unfused SpMM
 
-// Y += X * W_O as its own launch (the sparse half of the two-kernel baseline).  One CTA per column
-// tile walks all K/128 row tiles: stages the activation tile k-major in shared memory, applies the
-// tile's packets straight from global memory, and finally adds the FP32 tile to the BF16 Y.
-template <int BN>
+// Y += X * W_O as its own launch (the sparse half of the two-kernel baseline).  One warp per bucket of
+// a column tile (four columns): its lanes take the row tiles kt = lane, lane + 32, ..., read the
+// bucket's packets and the activations x[m][k] from global memory (L2-resident) and add into registers
+// (4 columns x 8 batch rows per lane); a butterfly sum over the lanes and one read-modify-write of the
+// BF16 Y per element finish it.  No shared memory, no atomics: a bucket's columns belong to one warp.
 __global__ void __launch_bounds__(256) fq_spmm_kernel(const uint16_t* __restrict__ X, const uint32_t* __restrict__ indptr,
                                                     const uint32_t* __restrict__ info, const uint4* __restrict__ packed,
                                                     uint16_t* __restrict__ Y, uint32_t M, uint32_t K, uint32_t N,
-                                                    uint32_t NB, uint32_t MO) {
-    extern __shared__ __align__(128) uint8_t smem[];
-    const uint32_t LDC = 8 * MO;
-    float* shc = reinterpret_cast<float*>(smem);                    // [BN][8 MO]
-    float* xt = reinterpret_cast<float*>(smem + (size_t)BN * LDC * 4);   // [MO][128][8] FP32
-    const uint32_t tn = blockIdx.x, KT = K / kBK;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    for (uint32_t i = tid; i < BN * LDC; i += blockDim.x) shc[i] = 0.0f;
-    for (uint32_t kt = 0; kt < KT; ++kt) {
-        __syncthreads();
-        // k-major copy of the activation tile, zero for rows >= M
-        for (uint32_t i = tid; i < 128 * LDC; i += blockDim.x) {
-            const uint32_t k = i / LDC, m = i % LDC;
-            const uint16_t v = (m < M) ? X[(size_t)m * K + (size_t)kt * kBK + k] : (uint16_t)0;
-            xt[((m >> 3) * 128 + k) * 8 + (m & 7)] = bf16_bits_to_float(v);
+                                                    uint32_t BN, uint32_t NB) {
+    constexpr int MB = 8;
+    const int lane = threadIdx.x & 31;
+    const uint32_t wg = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (wg >= (N / BN) * NB) return;
+    const uint32_t tn = wg / NB, b = wg - tn * NB, KT = K / kBK;
+    const uint32_t first_col = tn * BN + (((b >> 3) << 5) | (b & 7u));      // column number c of the bucket: + 8 c
+    for (uint32_t m0 = 0; m0 < M; m0 += MB) {
+        float acc[4][MB];
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int m = 0; m < MB; ++m) acc[c][m] = 0.0f;
+        for (uint32_t kt = lane; kt < KT; kt += 32) {
+            const size_t t = (size_t)tn * KT + kt;
+            const uint32_t inf = __ldg(info + t * NB + b);
+            const uint4* pk = packed + __ldg(indptr + t) + (inf & 0xffffu);
+            for (uint32_t i = 0; i < (inf >> 16); ++i) {
+                const uint4 q = __ldg(pk + i);
+                const float v[4] = {bf16lo(q.z), bf16hi(q.z), bf16lo(q.w), bf16hi(q.w)};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const uint32_t k = kt * kBK + ((q.x >> (8 * e)) & 0xffu), cls = (q.y >> (8 * e + 3)) & 3u;
+                    const uint16_t* xp = X + (size_t)m0 * K + k;
+#pragma unroll
+                    for (int m = 0; m < MB; ++m) {
+                        const float x = (m0 + m < M) ? bf16_bits_to_float(__ldg(xp + (size_t)m * K)) : 0.0f;
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) acc[c][m] = fmaf(cls == (uint32_t)c ? v[e] : 0.0f, x, acc[c][m]);
+                    }
+                }
+            }
         }
-        __syncthreads();
-        const size_t t = (size_t)tn * KT + kt;
-        const uint4* pk = packed + indptr[t];
-        // (bucket block, octet) pairs dealt to the 8 warps
-        const uint32_t nbb = NB >> 5;
-        for (uint32_t w = warp; w < nbb * MO; w += 8) {
-            const uint32_t bb = w % nbb, o = w / nbb;
-            const uint32_t inf = info[t * NB + bb * 32 + lane];
-            const uint32_t off = inf & 0xffffu, cnt = inf >> 16;
-            for (uint32_t i = 0; i < cnt; ++i) apply_packet<0>(__ldg(pk + off + i), xt + o * 1024, shc, o, LDC);
-        }
-    }
-    __syncthreads();
-    for (uint32_t i = tid; i < BN * M; i += blockDim.x) {
-        const uint32_t m = i / BN, c = i % BN;
-        uint16_t* y = Y + (size_t)m * N + (size_t)tn * BN + c;
-        *y = float_to_bf16_bits(bf16_bits_to_float(*y) + shc[c * LDC + m]);
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int m = 0; m < MB; ++m) {
+                float a = acc[c][m];
+#pragma unroll
+                for (int d = 16; d > 0; d >>= 1) a += __shfl_xor_sync(0xffffffffu, a, d);
+                if (lane == c * MB + m && m0 + m < M) {
+                    uint16_t* y = Y + (size_t)(m0 + m) * N + first_col + 8 * c;
+                    *y = float_to_bf16_bits(bf16_bits_to_float(*y) + a);
+                }
+            }
     }
 }
 
@@ -1671,29 +1684,12 @@ fq_status_t fq_unfused_spmm(const fq_layout_t* L, const void* X, uint32_t M, con
     if (M < 1 || M > FQ_MAX_M) return fail(FQ_ERR_INVALID_ARG, "M = %u outside [1, %u]", M, FQ_MAX_M);
     if (!X || !tile_indptr || !bucket_info || !Y) return fail(FQ_ERR_INVALID_ARG, "null device pointer");
     if (!packed_outliers && L->max_tile_packets) return fail(FQ_ERR_INVALID_ARG, "null packet pointer");
-    for (uint32_t m0 = 0; m0 < M; m0 += 32) {
-        const uint32_t mb = std::min<uint32_t>(32, M - m0);
-        const uint32_t MO = (mb + 7) / 8;
-        const size_t smem = (size_t)L->BN * 8 * MO * 4 + (size_t)MO * 4096;
-        const uint16_t* x = (const uint16_t*)X + (size_t)m0 * L->K;
-        uint16_t* y = (uint16_t*)Y + (size_t)m0 * L->N;
-        cudaError_t e;
-        if (L->BN == 128) {
-            e = ensure_smem_attr((const void*)fq_spmm_kernel<128>, 65536);
-            if (e == cudaSuccess)
-                fq_spmm_kernel<128><<<L->N / 128, 256, smem, (cudaStream_t)cuda_stream>>>(
-                    x, (const uint32_t*)tile_indptr, (const uint32_t*)bucket_info, (const uint4*)packed_outliers, y, mb,
-                    L->K, L->N, L->buckets_per_tile, MO);
-        } else {
-            e = ensure_smem_attr((const void*)fq_spmm_kernel<256>, 65536);
-            if (e == cudaSuccess)
-                fq_spmm_kernel<256><<<L->N / 256, 256, smem, (cudaStream_t)cuda_stream>>>(
-                    x, (const uint32_t*)tile_indptr, (const uint32_t*)bucket_info, (const uint4*)packed_outliers, y, mb,
-                    L->K, L->N, L->buckets_per_tile, MO);
-        }
-        if (e == cudaSuccess) e = cudaGetLastError();
-        if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "spmm launch: %s", cudaGetErrorString(e));
-    }
+    const uint32_t buckets = (L->N / L->BN) * L->buckets_per_tile;   // one warp each
+    fq_spmm_kernel<<<(buckets + 7) / 8, 256, 0, (cudaStream_t)cuda_stream>>>(
+        (const uint16_t*)X, (const uint32_t*)tile_indptr, (const uint32_t*)bucket_info, (const uint4*)packed_outliers,
+        (uint16_t*)Y, M, L->K, L->N, L->BN, L->buckets_per_tile);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "spmm launch: %s", cudaGetErrorString(e));
     return FQ_OK;
 }
 

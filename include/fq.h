@@ -166,13 +166,15 @@ fq_status_t fq_validate_tilecoo(const fq_layout_t* L, const uint32_t* tile_indpt
 fq_status_t fq_workspace_bytes(const fq_layout_t* L, uint32_t M, size_t* bytes);
 
 /*
- * The fused operator (Eq. 1; Sections 3.1 and 4.1): one launch per 32 rows of X
+ * The fused operator (Eq. 1; Sections 3.1 and 4.1): one launch per 16 rows of X
  * reads X, W_Q and the Tile-COO tiles through a bulk-copy/mbarrier ring,
  * dequantises in registers into tensor-core operands, applies the tile's
  * outliers against the same shared-memory activation tile, and writes Y once.
- * Up to 16 rows run the small-batch kernel (warp-level MMAs, outliers added in
- * registers), more rows the tcgen05 kernel (tensor-memory operand, outliers
- * through a shared-memory FP32 tile).
+ * The default kernel uses warp-level MMAs and adds the outliers in registers.
+ * Environment variable FQ_ENGINE=tc routes every call to the library's
+ * tcgen05 kernel instead (tensor-memory operand, outliers through a
+ * shared-memory FP32 tile, 32 rows per launch), FQ_ENGINE=mix only calls with
+ * M > 16; as it stands that kernel is the slower one at every M.
  * X: device, M x K BF16.  M in [1, FQ_MAX_M].  Y: device, M x N BF16,
  * overwritten.  All other arrays: device copies of the host packer/encoder
  * output.  Work is split over persistent CTAs by (tile, k-step) units; tiles

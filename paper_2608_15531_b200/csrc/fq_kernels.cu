@@ -1470,15 +1470,18 @@ static KernelFn pick_mma_kernel(uint32_t bn, uint32_t M, uint32_t g, bool sparse
     return mo == 1 ? pick_mma_group<256, 1>(g, sparse, ms, ngrp) : pick_mma_group<256, 2>(g, sparse, ms, ngrp);
 }
 
-static uint32_t mma_max_rows() {
-    static int v = -1;
-    if (v < 0) {
+// Which kernel serves a call.  Default: the small-batch kernel, in launches of 16 rows (at M = 32 two such
+// launches take about half the time of one launch of the tcgen05 kernel as it stands).  FQ_ENGINE=tc
+// routes every call to the tcgen05 kernel (launches of 32 rows), FQ_ENGINE=mix uses it for M > 16.
+enum Engine { kEngineMma, kEngineTc, kEngineMix };
+static Engine engine() {
+    static const Engine v = [] {
         const char* e = std::getenv("FQ_ENGINE");
-        v = 16;
-        if (e && std::strcmp(e, "mma") == 0) v = 16;
-        if (e && std::strcmp(e, "tc") == 0) v = 0;
-    }
-    return (uint32_t)v;
+        if (e && std::strcmp(e, "tc") == 0) return kEngineTc;
+        if (e && std::strcmp(e, "mix") == 0) return kEngineMix;
+        return kEngineMma;
+    }();
+    return v;
 }
 
 template <int BN, int MO, int G>
@@ -1542,10 +1545,11 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
     fq_status_t st = fq_workspace_bytes(L, M, &need);
     if (st != FQ_OK) return st;
     if (workspace_bytes < need) return fail(FQ_ERR_BUFFER_TOO_SMALL, "workspace holds %zu bytes, %zu needed", workspace_bytes, need);
-    for (uint32_t m0 = 0; m0 < M; m0 += 32) {
-        const uint32_t mb = std::min<uint32_t>(32, M - m0);
+    const bool use_mma = engine() == kEngineMma || (engine() == kEngineMix && M <= 16);
+    const uint32_t rows_per_launch = use_mma ? 16 : 32;
+    for (uint32_t m0 = 0; m0 < M; m0 += rows_per_launch) {
+        const uint32_t mb = std::min<uint32_t>(rows_per_launch, M - m0);
         Plan pl;
-        const bool use_mma = mb <= mma_max_rows();
         st = use_mma ? make_plan_mma(L, mb, sparse, pl) : make_plan(L, mb, sparse, pl);
         if (st != FQ_OK) return st;
         Params& p = pl.p;

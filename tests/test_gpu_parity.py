@@ -274,3 +274,20 @@ def test_batch_transition_sweep_on_sampled_columns(g):
         Y = H.run_fused(P, X)
         Yref, Yabs = H.oracle_result(P, X, cols=cols)
         H.check_tolerances(Y[:, cols], Yref, Yabs, K)
+
+
+# ------------------------------------------------------------------ the tcgen05 kernel (not the default engine)
+
+def test_tcgen05_engine_in_a_child_process():
+    """FQ_ENGINE is read once per process, so the tcgen05 kernel is exercised in a child: the
+    element-by-element cases and the larger batches, with every call routed to it."""
+    import os
+    import subprocess
+    import sys
+    env = dict(os.environ, FQ_ENGINE="tc")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-m", "pytest", "-q", "-x", "-m", "gpu", "tests/test_gpu_parity.py", "-k",
+                        "test_fused_matches_oracle or test_fused_larger_batches or test_identity_rows or "
+                        "test_zero_density or test_oversized_tiles"], cwd=root, env=env, capture_output=True,
+                       text=True, timeout=900)
+    assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-2000:]

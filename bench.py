@@ -395,6 +395,93 @@ def cpu_baseline(work, budget_s: float):
             "sample": f"all four layers at M=16, first {f:.3f} of each layer's output columns (fp64 oracle, OpenMP over columns)"}
 
 
+def run_sweep(args):
+    """Not the contract line: the paper's two sweeps on one GPU, one JSON object on stdout.
+    `density`: M = 8, K = 4096, N = 14336, densities 0..5 % in the uniform and the clustered layout;
+    `batch`:   K = 8192, N = 28672, 1 % mixed outliers, M = 1..128, groups of 64 and 128.
+    Every point: fused call, unfused pair (dense kernel + SpMM), rotating weight copies larger than L2."""
+    import ctypes
+    import torch
+    from paper_2608_15531_b200 import binding as fq
+    from paper_2608_15531_b200 import synth
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the fused path has no CPU fallback")
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    stream = torch.cuda.current_stream()
+    peak, peak_kind = peaks()
+
+    def up(a):
+        a = np.ascontiguousarray(a)
+        a = a.view(np.int16) if a.dtype == np.uint16 else (a.view(np.int32) if a.dtype == np.uint32 else a)
+        return torch.from_numpy(a).to(dev)
+
+    def time_loop(fn, reps=30):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(reps):
+            fn()
+        b.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps * 1e3
+
+    def point(cfg, tag, K, N, g, density, layout, Ms):
+        lay = synth.layer(synth.tensor_seed(cfg, tag), K, N, density=density, layout=layout)
+        L = fq.fq_get_layout(K, N, g)
+        wq, scale, zero = fq.fq_pack_int4(L, lay.W, lay.mask if lay.nnz else None)
+        indptr, info, packed = fq.fq_encode_tilecoo(L, lay.coo_k, lay.coo_n, lay.coo_v)
+        if packed.shape[0] == 0:
+            packed = np.zeros((8, 16), dtype=np.uint8)
+        base = dict(wq=up(wq), scale=up(scale), zero=up(zero), indptr=up(indptr), info=up(info), packed=up(packed))
+        per_copy = sum(v.numel() * v.element_size() for v in base.values())
+        copies = [base] + [{k: v.clone() for k, v in base.items()} for _ in range(max(2, -(-L2_COVER_BYTES // per_copy)) - 1)]
+        n_tile = (K // 128) * (N // L.BN)
+        ws = torch.zeros(fq.fq_workspace_bytes(L, max(Ms)), dtype=torch.uint8, device=dev)
+        out = []
+        for M in Ms:
+            X = up(synth.activations(lay.seed, M, K))
+            Y = torch.empty((M, N), dtype=torch.int16, device=dev)
+            turn = [0]
+
+            def fused():
+                c = copies[turn[0] % len(copies)]
+                turn[0] += 1
+                fq.fq_fused_w4a16_outlier_gemm(L, X, M, c["wq"], c["scale"], c["zero"], c["indptr"], c["info"],
+                                               c["packed"], Y, ws, stream)
+
+            def unfused():
+                c = copies[turn[0] % len(copies)]
+                turn[0] += 1
+                fq.fq_unfused_gemm(L, X, M, c["wq"], c["scale"], c["zero"], Y, ws, stream)
+                fq.fq_unfused_spmm(L, X, M, c["indptr"], c["info"], c["packed"], Y, stream)
+
+            nbytes = algorithmic_bytes(K, N, g, lay.nnz, n_tile, n_tile * L.buckets_per_tile, M)
+            us_f, us_u = time_loop(fused), time_loop(unfused)
+            fq.fq_check_status(ws)
+            out.append(dict(K=K, N=N, group=g, M=M, density=density, layout=layout, nnz=int(lay.nnz), bytes=nbytes,
+                            fused_us=round(us_f, 2), unfused_us=round(us_u, 2), fused_gbs=round(nbytes / us_f / 1e3, 1),
+                            frac_of_peak=round(nbytes / us_f / 1e3 / peak, 4), fused_over_unfused=round(us_u / us_f, 2)))
+        del copies, base
+        torch.cuda.empty_cache()
+        return out
+
+    points = []
+    if args.sweep == "density":
+        for layout in ("uniform", "clustered"):
+            for density in (0.0, 0.005, 0.01, 0.02, 0.05):
+                if density == 0.0 and layout == "clustered":
+                    continue
+                points += point(3, int(density * 1000) + (layout == "clustered"), 4096, 14336, GROUP, density, layout, (8,))
+    else:
+        for g in (64, 128):
+            points += point(5, g, 8192, 28672, g, DENSITY, "mixed", (1, 2, 4, 8, 16, 32, 64, 128))
+    print(json.dumps({"sweep": args.sweep, "peak_gbs": peak, "peak_kind": f"of {peak_kind}", "data": "synthetic",
+                      "points": points}))
+
+
 def run_reference(args):
     """The oracle arm: rank 0 times the CPU oracle on a bounded sample of the same workload."""
     rank = int(os.environ.get("RANK", "0"))
@@ -438,9 +525,13 @@ def main():
     ap.add_argument("--no-cublas", dest="cublas", action="store_false")
     ap.add_argument("--verbose", action="store_true")
     ap.add_argument("--only", default="", help="profiling aid: restrict the step to one LAYER:M, e.g. gate_up:16")
+    ap.add_argument("--sweep", default="", choices=["", "density", "batch"],
+                    help="print the density sweep or the batch transition sweep instead of the benchmark line")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.sweep:
+        run_sweep(args)
     else:
         run_ours(args)
 

@@ -80,7 +80,9 @@ typedef int32_t fq_status_t;
 #define FQ_BK 128u
 
 /* Plain data, caller-owned.  Filled by fq_get_layout(); fq_encode_tilecoo()
- * writes max_tile_packets.  Pass the same struct to every later call. */
+ * writes max_tile_packets and max_bucket_packets (the kernels size their staging
+ * by the first and choose their outlier path by the second).  Pass the same
+ * struct to every later call. */
 typedef struct fq_layout {
     uint32_t abi;
     uint32_t K, N;
@@ -91,7 +93,8 @@ typedef struct fq_layout {
     uint32_t wq_interleave;    /* 2: the column-per-thread order described above */
     uint32_t coo_unit_bytes;   /* 16 */
     uint32_t max_tile_packets; /* largest tile of the encoded W_O, in packets; 0 = not encoded */
-    uint32_t reserved[6];
+    uint32_t max_bucket_packets; /* longest packet list of one bucket in one tile; 0 = not encoded */
+    uint32_t reserved[5];
 } fq_layout_t;
 
 /* Choose tile sizes for a K x N layer.  bn_hint: 0 = library default (256 when
@@ -134,7 +137,8 @@ fq_status_t fq_unpack_int4(const fq_layout_t* L, const void* wq, uint8_t* q_cano
  *
  * fq_encode_tilecoo_sizes: element counts of the three arrays (tile_indptr in
  * uint32, bucket_info in uint32, packets in 16-byte units) and the largest
- * tile.  fq_encode_tilecoo: writes them and stores max_tile_packets in *L.
+ * tile.  fq_encode_tilecoo: writes them and stores max_tile_packets and
+ * max_bucket_packets in *L.
  */
 fq_status_t fq_encode_tilecoo_sizes(const fq_layout_t* L, const uint32_t* k, const uint32_t* n,
                                     const uint16_t* val_bf16, size_t nnz, size_t* n_indptr,

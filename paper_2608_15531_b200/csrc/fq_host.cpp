@@ -186,6 +186,7 @@ struct Encoded {
     std::vector<uint32_t> info;     // N_tile * NB
     std::vector<uint8_t> packets;   // 16 * n_packets
     uint32_t max_tile_packets = 0;
+    uint32_t max_bucket_packets = 0;
 };
 
 // Bucket of a tile column: the four columns {g, g + 8, g + 16, g + 24} of a 32-column block share
@@ -246,6 +247,7 @@ fq_status_t encode_impl(const fq_layout_t* L, const uint32_t* k, const uint32_t*
         E.indptr[t + 1] = off;
     }
     if (bad) return fq::fail(FQ_ERR_UNSUPPORTED_SHAPE, "a bucket exceeds the 16-bit packet offset/count range");
+    for (size_t i = 0; i < E.info.size(); ++i) E.max_bucket_packets = std::max(E.max_bucket_packets, E.info[i] >> 16);
     uint64_t total = 0;
     for (size_t t = 0; t < ntile; ++t) {
         uint32_t c = E.indptr[t + 1];
@@ -304,6 +306,7 @@ fq_status_t fq_encode_tilecoo(fq_layout_t* L, const uint32_t* k, const uint32_t*
     std::memcpy(bucket_info, E.info.data(), E.info.size() * 4);
     if (!E.packets.empty()) std::memcpy(packed, E.packets.data(), E.packets.size());
     L->max_tile_packets = E.max_tile_packets;
+    L->max_bucket_packets = E.max_bucket_packets;
     return FQ_OK;
 }
 

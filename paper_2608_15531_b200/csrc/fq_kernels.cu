@@ -764,7 +764,7 @@ constexpr int kXPitch = 320;   // activation row in shared memory: 256 B + 64 B,
 //                     the four lanes of group g walk that bucket's packets and add v * x[row][k]
 //                     straight into their accumulators (Section 4.2 without the shared-memory
 //                     scatter: no atomics, no read-modify-write, no merge step).
-template <int BN, int MO, int GROUP, bool SPARSE, int MS, int NGRP>
+template <int BN, int MO, int GROUP, bool SPARSE, int MS, int NGRP, bool HOT>
 __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq_mma_kernel(const Params p) {
     constexpr int NDW = BN / 32;
     constexpr int NA = kActWarps;                           // activation warps: warp a takes the units it with it mod NA == a
@@ -981,7 +981,13 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
             const float* xsum = reinterpret_cast<const float*>(st + p.off_xsum);
             // outliers: the bucket descriptor and the first two packets are requested now and used
             // after the dense math of the unit
-            uint32_t sp_off = 0, sp_cnt = 0, cmax = 0;
+            // HOT (chosen by the host for layers that have very long bucket lists: hot columns): the longest
+            // list of a warp's eight buckets is not walked by its lane group alone; beyond its first kOwn
+            // packets it is shared out over the eight lane groups, which add into sums of their own that are
+            // added up over the groups afterwards.  Kernels for layers without such lists are compiled
+            // without that code: its presence alone costs the common path 3-4 %.
+            constexpr uint32_t kOwn = 4;
+            uint32_t sp_off = 0, sp_cnt = 0, cmax = 0, hot_off = 0, hot_cnt = 0, hot_g = 0;
             const uint4* pk_s = reinterpret_cast<const uint4*>(st + p.off_coo);
             const uint4* pk_g = nullptr;
             const float* xt = reinterpret_cast<const float*>(st + p.off_xt);
@@ -1007,8 +1013,17 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                 const uint32_t info = reinterpret_cast<const uint32_t*>(st + p.off_info)[dw * 8 + g];
                 sp_off = info & 0xffffu;
                 sp_cnt = info >> 16;
-                if (sp_off + sp_cnt > p.coo_cap) pk_g = p.packed + __ldg(p.indptr + u);   // packets beyond the staged part
                 cmax = __reduce_max_sync(0xffffffffu, sp_cnt);
+                if (HOT && cmax > kOwn) {                            // warp-uniform
+                    const uint32_t hot_lane = __ffs(__ballot_sync(0xffffffffu, sp_cnt == cmax)) - 1;
+                    hot_g = hot_lane >> 2;
+                    hot_off = __shfl_sync(0xffffffffu, sp_off, hot_lane);
+                    hot_cnt = cmax;
+                    if ((uint32_t)g == hot_g) sp_cnt = kOwn;         // the rest of this list is shared out
+                    cmax = __reduce_max_sync(0xffffffffu, sp_cnt);
+                }
+                if (sp_off + sp_cnt > p.coo_cap || hot_off + hot_cnt > p.coo_cap)
+                    pk_g = p.packed + __ldg(p.indptr + u);           // packets beyond the staged part
                 pk0 = packet(0);
                 pk1 = packet(1);
                 if constexpr (MS == 8) fetch_x(pk0, xa);
@@ -1078,6 +1093,24 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                         apply(pk1);
                         for (uint32_t i = 2; i < cmax; ++i) apply(packet(i));
                     }
+                    if (HOT && hot_cnt) {
+                        float hacc = 0.0f;
+                        for (uint32_t i0 = kOwn; i0 < hot_cnt; i0 += 8) {
+                            const uint32_t i = i0 + g, idx = hot_off + i;
+                            uint4 pk = make_uint4(0, 0, 0, 0);
+                            if (i < hot_cnt) pk = (idx < p.coo_cap) ? pk_s[idx] : __ldg(pk_g + idx);
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const uint32_t cls = (pk.y >> (8 * e + 3)) & 3u;
+                                const float v = (e & 1) ? bf16hi(e < 2 ? pk.z : pk.w) : bf16lo(e < 2 ? pk.z : pk.w);
+                                hacc = fmaf(cls == (uint32_t)t ? v : 0.0f, xt[((pk.x >> (8 * e)) & 0xffu) * 8], hacc);
+                            }
+                        }
+                        hacc += __shfl_xor_sync(0xffffffffu, hacc, 4);
+                        hacc += __shfl_xor_sync(0xffffffffu, hacc, 8);
+                        hacc += __shfl_xor_sync(0xffffffffu, hacc, 16);
+                        if ((uint32_t)g == hot_g) sacc[0][0] += hacc;
+                    }
                 } else {
                     // several batch rows: lane t keeps rows 2t, 2t+1 (+8) of all four columns, in the
                     // MMA fragment registers themselves
@@ -1110,6 +1143,50 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                             fetch_x(pk, xb2);
                             apply(pk, xb2);
                         }
+                    }
+                    if (HOT && hot_cnt) {
+                        float hacc[MO][CG][4];
+#pragma unroll
+                        for (int o = 0; o < MO; ++o)
+#pragma unroll
+                            for (int cg = 0; cg < CG; ++cg)
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) hacc[o][cg][i] = 0.0f;
+                        for (uint32_t i0 = kOwn; i0 < hot_cnt; i0 += 8) {
+                            const uint32_t i = i0 + g, idx = hot_off + i;
+                            uint4 pk = make_uint4(0, 0, 0, 0);
+                            if (i < hot_cnt) pk = (idx < p.coo_cap) ? pk_s[idx] : __ldg(pk_g + idx);
+                            float2 xh[4][MO];
+                            fetch_x(pk, xh);
+                            const float v[4] = {bf16lo(pk.z), bf16hi(pk.z), bf16lo(pk.w), bf16hi(pk.w)};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const uint32_t cls = (pk.y >> (8 * e + 3)) & 3u;
+#pragma unroll
+                                for (int cg = 0; cg < CG; ++cg)
+#pragma unroll
+                                    for (int h = 0; h < 2; ++h) {
+                                        const float vv = (cls == (uint32_t)(2 * cg + h)) ? v[e] : 0.0f;
+#pragma unroll
+                                        for (int o = 0; o < MO; ++o) {
+                                            hacc[o][cg][2 * h + 0] = fmaf(vv, xh[e][o].x, hacc[o][cg][2 * h + 0]);
+                                            hacc[o][cg][2 * h + 1] = fmaf(vv, xh[e][o].y, hacc[o][cg][2 * h + 1]);
+                                        }
+                                    }
+                            }
+                        }
+#pragma unroll
+                        for (int o = 0; o < MO; ++o)
+#pragma unroll
+                            for (int cg = 0; cg < CG; ++cg)
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) {
+                                    float v = hacc[o][cg][i];
+                                    v += __shfl_xor_sync(0xffffffffu, v, 4);
+                                    v += __shfl_xor_sync(0xffffffffu, v, 8);
+                                    v += __shfl_xor_sync(0xffffffffu, v, 16);
+                                    if ((uint32_t)g == hot_g) accf[o][cg][i] += v;
+                                }
                     }
                 }
             }
@@ -1446,28 +1523,29 @@ static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, 
 typedef void (*KernelFn)(const Params);
 
 // MS: form of the outlier step (1: single batch row, one column per lane; 8: rows split over the lanes);
-// NGRP: groups of dense warps (two only with one octet of rows)
-template <int BN, int MO, int G>
+// NGRP: groups of dense warps (two only with one octet of rows); HOT: long bucket lists are shared out
+template <int BN, int MO, int G, bool HOT>
 static KernelFn pick_mma_sparse(bool sparse, uint32_t ms, uint32_t ngrp) {
     if constexpr (MO == 1) {
         if (ngrp == 2) {
-            if (!sparse) return (KernelFn)fq_mma_kernel<BN, MO, G, false, 8, 2>;
-            if (ms == 1) return (KernelFn)fq_mma_kernel<BN, MO, G, true, 1, 2>;
-            return (KernelFn)fq_mma_kernel<BN, MO, G, true, 8, 2>;
+            if (!sparse) return (KernelFn)fq_mma_kernel<BN, MO, G, false, 8, 2, false>;
+            if (ms == 1) return (KernelFn)fq_mma_kernel<BN, MO, G, true, 1, 2, HOT>;
+            return (KernelFn)fq_mma_kernel<BN, MO, G, true, 8, 2, HOT>;
         }
-        if (sparse && ms == 1) return (KernelFn)fq_mma_kernel<BN, MO, G, true, 1, 1>;
+        if (sparse && ms == 1) return (KernelFn)fq_mma_kernel<BN, MO, G, true, 1, 1, HOT>;
     }
-    if (!sparse) return (KernelFn)fq_mma_kernel<BN, MO, G, false, 8, 1>;
-    return (KernelFn)fq_mma_kernel<BN, MO, G, true, 8, 1>;
+    if (!sparse) return (KernelFn)fq_mma_kernel<BN, MO, G, false, 8, 1, false>;
+    return (KernelFn)fq_mma_kernel<BN, MO, G, true, 8, 1, HOT>;
 }
 template <int BN, int MO>
-static KernelFn pick_mma_group(uint32_t g, bool sparse, uint32_t ms, uint32_t ngrp) {
-    return g == 64 ? pick_mma_sparse<BN, MO, 64>(sparse, ms, ngrp) : pick_mma_sparse<BN, MO, 128>(sparse, ms, ngrp);
+static KernelFn pick_mma_group(uint32_t g, bool sparse, uint32_t ms, uint32_t ngrp, bool hot) {
+    if (g == 64) return hot ? pick_mma_sparse<BN, MO, 64, true>(sparse, ms, ngrp) : pick_mma_sparse<BN, MO, 64, false>(sparse, ms, ngrp);
+    return hot ? pick_mma_sparse<BN, MO, 128, true>(sparse, ms, ngrp) : pick_mma_sparse<BN, MO, 128, false>(sparse, ms, ngrp);
 }
-static KernelFn pick_mma_kernel(uint32_t bn, uint32_t M, uint32_t g, bool sparse, uint32_t ngrp) {
+static KernelFn pick_mma_kernel(uint32_t bn, uint32_t M, uint32_t g, bool sparse, uint32_t ngrp, bool hot) {
     const uint32_t mo = M <= 8 ? 1 : 2, ms = M <= 1 ? 1 : 8;
-    if (bn == 128) return mo == 1 ? pick_mma_group<128, 1>(g, sparse, ms, ngrp) : pick_mma_group<128, 2>(g, sparse, ms, ngrp);
-    return mo == 1 ? pick_mma_group<256, 1>(g, sparse, ms, ngrp) : pick_mma_group<256, 2>(g, sparse, ms, ngrp);
+    if (bn == 128) return mo == 1 ? pick_mma_group<128, 1>(g, sparse, ms, ngrp, hot) : pick_mma_group<128, 2>(g, sparse, ms, ngrp, hot);
+    return mo == 1 ? pick_mma_group<256, 1>(g, sparse, ms, ngrp, hot) : pick_mma_group<256, 2>(g, sparse, ms, ngrp, hot);
 }
 
 // Which kernel serves a call.  Default: the small-batch kernel, in launches of 16 rows (at M = 32 two such
@@ -1560,7 +1638,7 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
         p.status = (uint32_t*)workspace;
         p.counters = (uint32_t*)((uint8_t*)workspace + kWsHeaderBytes);
         p.partials = (float*)((uint8_t*)workspace + kWsHeaderBytes + kWsCounterBytes);
-        KernelFn fn = use_mma ? pick_mma_kernel(L->BN, mb, L->group, sparse, pl.ngrp)
+        KernelFn fn = use_mma ? pick_mma_kernel(L->BN, mb, L->group, sparse, pl.ngrp, L->max_bucket_packets > 16)
                               : pick_kernel(L->BN, nb16_of(mb), L->group, sparse);
         cudaError_t e = ensure_smem_attr((const void*)fn, (int)kSmemBudget);
         if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));

@@ -96,6 +96,7 @@ def test_tilecoo_encode_invariants(layout, density, BN):
     # array sizes and storage formula (Table 1 and the storage analysis), padding bounded per bucket
     assert n_ip == ntile + 1 == indptr.size and n_bi == ntile * NB == info.size and n_pk == packed.shape[0]
     assert L.max_tile_packets == mx == int(np.diff(indptr).max())
+    assert L.max_bucket_packets == int((info >> 16).max())
     assert indptr[0] == 0 and np.all(np.diff(indptr.astype(np.int64)) >= 0) and indptr[-1] == n_pk
     assert 4 * Lr.nnz <= 16 * n_pk <= 16 * Lr.nnz          # every packet carries at least one outlier
     # decoded set == input set, by the oracle's reader and by the library's

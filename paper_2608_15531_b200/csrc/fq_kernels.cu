@@ -981,11 +981,13 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
             const float* xsum = reinterpret_cast<const float*>(st + p.off_xsum);
             // outliers: the bucket descriptor and the first two packets are requested now and used
             // after the dense math of the unit
-            // HOT (chosen by the host for layers that have very long bucket lists: hot columns): the longest
-            // list of a warp's eight buckets is not walked by its lane group alone; beyond its first kOwn
-            // packets it is shared out over the eight lane groups, which add into sums of their own that are
-            // added up over the groups afterwards.  Kernels for layers without such lists are compiled
-            // without that code: its presence alone costs the common path 3-4 %.
+            // HOT is the general form of the outlier step, chosen by the host for layers that need it:
+            //  - very long bucket lists (hot columns): the longest list of a warp's eight buckets is not
+            //    walked by its lane group alone; beyond its first kOwn packets it is shared out over the eight
+            //    lane groups, which add into sums of their own that are added up over the groups afterwards;
+            //  - tiles with more packets than a stage holds: the rest is read from global memory.
+            // Kernels for layers that need neither are compiled without that code: the presence of either
+            // costs the common path 3-4 %.
             constexpr uint32_t kOwn = 4;
             uint32_t sp_off = 0, sp_cnt = 0, cmax = 0, hot_off = 0, hot_cnt = 0, hot_g = 0;
             const uint4* pk_s = reinterpret_cast<const uint4*>(st + p.off_coo);
@@ -995,7 +997,7 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                 uint4 pk = make_uint4(0, 0, 0, 0);            // beyond the bucket's list: four padding slots
                 if (i < sp_cnt) {
                     const uint32_t idx = sp_off + i;
-                    pk = (idx < p.coo_cap) ? pk_s[idx] : __ldg(pk_g + idx);
+                    pk = (!HOT || idx < p.coo_cap) ? pk_s[idx] : __ldg(pk_g + idx);
                 }
                 return pk;
             };
@@ -1022,7 +1024,7 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                     if ((uint32_t)g == hot_g) sp_cnt = kOwn;         // the rest of this list is shared out
                     cmax = __reduce_max_sync(0xffffffffu, sp_cnt);
                 }
-                if (sp_off + sp_cnt > p.coo_cap || hot_off + hot_cnt > p.coo_cap)
+                if (HOT && (sp_off + sp_cnt > p.coo_cap || hot_off + hot_cnt > p.coo_cap))
                     pk_g = p.packed + __ldg(p.indptr + u);           // packets beyond the staged part
                 pk0 = packet(0);
                 pk1 = packet(1);
@@ -1392,6 +1394,7 @@ struct Plan {
     Params p;
     uint32_t threads, smem, grid;
     uint32_t ngrp;   // small-batch kernel: groups of dense warps
+    bool general;    // small-batch kernel: the layer needs the general form of the outlier step
 };
 
 static inline uint32_t round_up(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
@@ -1512,6 +1515,8 @@ static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, 
     }
     if (S < 4) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "shared-memory stages do not fit");
     p.coo_cap = cap; p.stages = S; p.stage_bytes = stage;
+    // hot columns, tiles larger than the staged part, or an encoding whose sizes were not recorded
+    pl.general = sparse && (L->max_bucket_packets > 16 || L->max_tile_packets > cap || L->max_tile_packets == 0);
     p.off_shc = S * stage;
     p.off_bar = p.off_shc + xch_bytes;
     pl.smem = p.off_bar + 1024;
@@ -1523,7 +1528,8 @@ static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, 
 typedef void (*KernelFn)(const Params);
 
 // MS: form of the outlier step (1: single batch row, one column per lane; 8: rows split over the lanes);
-// NGRP: groups of dense warps (two only with one octet of rows); HOT: long bucket lists are shared out
+// NGRP: groups of dense warps (two only with one octet of rows); HOT: general form of the outlier step
+// (long bucket lists shared out, packets beyond the staged part of a tile)
 template <int BN, int MO, int G, bool HOT>
 static KernelFn pick_mma_sparse(bool sparse, uint32_t ms, uint32_t ngrp) {
     if constexpr (MO == 1) {
@@ -1638,7 +1644,7 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
         p.status = (uint32_t*)workspace;
         p.counters = (uint32_t*)((uint8_t*)workspace + kWsHeaderBytes);
         p.partials = (float*)((uint8_t*)workspace + kWsHeaderBytes + kWsCounterBytes);
-        KernelFn fn = use_mma ? pick_mma_kernel(L->BN, mb, L->group, sparse, pl.ngrp, L->max_bucket_packets > 16)
+        KernelFn fn = use_mma ? pick_mma_kernel(L->BN, mb, L->group, sparse, pl.ngrp, pl.general)
                               : pick_kernel(L->BN, nb16_of(mb), L->group, sparse);
         cudaError_t e = ensure_smem_attr((const void*)fn, (int)kSmemBudget);
         if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));

@@ -788,15 +788,12 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
     // hand-over of group 1's partial sums to group 0 at the end of a piece: one pair of barriers per strip
     const uint32_t bar_xfull = bar_empty + 8 * S + 64, bar_xempty = bar_xfull + 8 * NDW;
 
-    if (tid == 0) {
-        for (uint32_t s = 0; s < S; ++s) {
-            mbar_init(bar_full + 8 * s, 2);   // producer's expect_tx arrival + activation warp
-            mbar_init(bar_empty + 8 * s, NDW);            // the dense warps of one group
-        }
-        for (int i = 0; i < 2 * NDW; ++i) mbar_init(bar_xfull + 8 * i, 1);
-        *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
+    // one barrier per thread of warp 0: S full, S empty (then the hand-over pairs)
+    if ((uint32_t)tid < S) mbar_init(bar_full + 8 * tid, 2);                 // producer's expect_tx arrival + activation warp
+    else if ((uint32_t)tid < 2 * S) mbar_init(bar_empty + 8 * (tid - S), NDW);   // the dense warps of one group
+    else if ((uint32_t)tid < 2 * S + 2 * NDW) mbar_init(bar_xfull + 8 * (tid - 2 * S), 1);
+    if (tid == 0) *abort_flag = 0;
+    if (tid < 32) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncthreads();
     FQ_GT(tid == 0, 1);
@@ -963,8 +960,14 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
         float sacc[1][1] = {{0.0f}};
         uint32_t piece = 0;
         bool ok = true;
-        for (UnitIter w(u_begin, KT); w.u < u_end && ok; w.next(S, KT)) {
-            const uint32_t u = w.u, s = w.s, ph = w.ph, tn = w.tn, kt = w.kt;
+        // outer loop: the pieces of this CTA's range (a piece = its units of one column tile); inner loop:
+        // the units of the piece.  The end-of-piece code stays out of the inner loop's body.
+        UnitIter w(u_begin, KT);
+        while (w.u < u_end && ok) {
+          const uint32_t tn = w.tn;
+          const uint32_t piece_stop = min(u_end, (tn + 1) * KT);        // one past the piece's last unit
+          for (; w.u < piece_stop; w.next(S, KT)) {
+            const uint32_t u = w.u, s = w.s, ph = w.ph;
             const uint8_t* st = smem + s * p.stage_bytes;
             if ((w.it % NGRP) == (uint32_t)grp) {
 #ifdef FQ_TRACE
@@ -1199,7 +1202,10 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
 #endif
             }
 
-            if (kt == KT - 1 || u == u_end - 1) {
+          }
+          if (!ok) break;
+          {
+                const uint32_t kt = piece_stop - 1 - tn * KT;               // k-step of the piece's last unit
                 // ---------------------------------------------------------- end of a piece
                 FQ_GT(dtid == 0 && piece < 2, 4 + 5 * piece);
                 if (SPARSE && MS == 1) {
@@ -1324,7 +1330,7 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                         for (int i = 0; i < 4; ++i) accf[o][cg][i] = 0.0f;
                 FQ_GT(dtid == 0 && piece < 2, 8 + 5 * piece);
                 ++piece;
-            }
+          }
         }
         FQ_GT(dtid == 0, 15);
     }

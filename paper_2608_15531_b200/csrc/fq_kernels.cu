@@ -1,27 +1,36 @@
 // CUDA side of the library (sm_100a): the fused W4A16 + Tile-COO outlier decode matmul
 // (Eq. 1; Sections 3.1, 4.1, 4.2), its two unfused baselines and the launchers behind the C ABI.
 //
-// Kernel shape (one persistent CTA per SM, warp-specialised):
-//   warp 0        producer: per (tile, k-step) unit, bulk-copies (cp.async.bulk + mbarrier expect_tx)
-//                 the unit's INT4 chunk, scale/zero rows, bucket_info slice and packet range into a
-//                 ring of shared-memory stages
-//   warp 1        tensor: owns the TMEM allocation and issues tcgen05.mma (A = dequantised weights
-//                 in TMEM, B = activations in shared memory, D = FP32 in TMEM); completion is
-//                 signalled with tcgen05.commit
-//   warp 2        activations: reads the unit's M x 128 activation block from global memory (it
-//                 stays in L2), lays it out as the canonical K-major MMA operand in the stage, and
-//                 writes the per-group sums of each row
-//   dense warps   thread = output column: unpacks its 128 codes of the unit with lop3 into BF16
-//                 (128 + q), stores them as the A operand into TMEM (tcgen05.st), and one unit later
-//                 reads the FP32 group sums back (tcgen05.ld) and applies scale and zero-point once
-//                 per group in FP32:  acc[m] += s * (sum_k x (128+q) - (128+z) sum_k x)
-//   sparse warps  lane = bucket; transposes the activation tile to k-major, then for each packet
-//                 slot adds v * x[0..7][k] into the FP32 tile sh_c[col][m] (buckets own disjoint
-//                 columns, so no atomics); merged into the column owner's registers at tile end
-// Units are split over CTAs as contiguous ranges (stream-K).  A tile whose k-range is shared by
-// several CTAs is finished by the last CTA to arrive, which adds the FP32 partials in CTA order.
-// Every wait on a barrier is bounded: on expiry the CTA raises the scratch status word, drains and
-// leaves through the common exit that frees its TMEM.
+// Two kernels compute the fused operator.  Both are persistent (one CTA per SM) and warp-specialised,
+// work on (tile, k-step) units of 128 rows x BN columns, stream them through the same ring of
+// shared-memory stages (cp.async.bulk + mbarrier expect_tx, one producer warp), feed the tensor cores
+// the exact integers 128 + q as BF16 and apply scale and zero-point once per group in FP32:
+//     acc[m] += s * (sum_k x (128+q) - (128+z) sum_k x)                 (Eq. 3 inside Eq. 1)
+//
+//   fq_mma_kernel    the default (16 batch rows per launch).  Dense warps own 32-column strips: lop3
+//                    unpack in registers, mma.sync m16n8k16 with the weights on the M side, and the
+//                    unit's outliers added straight into the MMA accumulators (a Tile-COO bucket is
+//                    the four columns a group of four lanes holds).  Activation warps lay out X and
+//                    its row sums per unit.  Described in detail above the kernel.
+//   fq_fused_kernel  the tcgen05 kernel (FQ_ENGINE=tc; 32 batch rows per launch):
+//     warp 0        producer
+//     warp 1 (+3)   tensor: own the TMEM allocation and issue tcgen05.mma (A = dequantised weights
+//                   in TMEM, B = activations in shared memory, D = FP32 in TMEM); completion is
+//                   signalled with tcgen05.commit
+//     warp 2        activations: the unit's M x 128 block of X from global memory (it stays in L2) as
+//                   the canonical K-major MMA operand in the stage, plus the per-group row sums
+//     unpack warps  thread = output column: its 128 codes of the unit -> BF16 (128 + q) -> TMEM A
+//                   operand (tcgen05.st)
+//     epilogue      thread = output column: reads the FP32 group sums back (tcgen05.ld), applies scale
+//                   and zero-point, at the end of a piece adds the outlier tile and writes Y
+//     sparse warps  lane = bucket; per packet slot adds v * x[0..7][k] into the FP32 tile sh_c[col][m]
+//                   in shared memory (buckets own disjoint columns, so no atomics)
+//
+// Units are split over CTAs as contiguous ranges (stream-K) or, for layers with few column tiles, as
+// tile-aligned parts.  A tile whose k-range is shared by several CTAs is finished by the last to
+// arrive, which adds the FP32 partials in CTA order; no CTA waits for another.  Every wait on a barrier
+// is bounded: on expiry the CTA raises the scratch status word, drains and leaves (the tcgen05 kernel
+// through the common exit that frees its TMEM).
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 

@@ -1277,12 +1277,15 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                     const uint32_t c_last = p.split ? c_first + p.split - 1 : cta_of_unit(u_tile0 + KT - 1, q, r);
                     uint32_t last = 0;
                     if (lane == 0) {
-                        __threadfence();                       // the warp's stores, ordered before the arrival
-                        const uint32_t old = atomicAdd(p.counters + tn * NDW + dw, 1u);
+                        // one arrival, release and acquire at GPU scope: the warp's stores (ordered before
+                        // this lane by the __syncwarp above) precede it, and the warp that finds itself last
+                        // sees the stores of all contributors that arrived before
+                        uint32_t old;
+                        asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(old) : "l"(p.counters + tn * NDW + dw) : "memory");
                         last = (old == c_last - c_first) ? 1u : 0u;
-                        if (last) __threadfence();
                     }
                     last = __shfl_sync(0xffffffffu, last, 0);
+                    __syncwarp();
                     FQ_GT(dtid == 0 && piece < 2, 7 + 5 * piece);
                     if (last) {
                         write_y = true;

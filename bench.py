@@ -253,12 +253,15 @@ def run_ours(args):
     xd = {k: torch.empty_like(v, device=dev) for k, v in xh.items()}
 
     def e2e_step():
+        # twelve asynchronous calls (copy of X in, kernel, copy of Y out, each with staging buffers of its
+        # own) and one wait for the step's results
         for w, M, _ in calls:
             c = w["copies"][w["turn"] % len(w["copies"])]
             w["turn"] += 1
             key = (w["name"], M)
-            fq.fq_fused_host_io(w["L"], xh[key], M, xd[key], c["wq"], c["scale"], c["zero"], c["indptr"], c["info"],
-                                c["packed"], w["Yd"][M], yh[key], ws, stream)
+            fq.fq_fused_host_io_async(w["L"], xh[key], M, xd[key], c["wq"], c["scale"], c["zero"], c["indptr"],
+                                      c["info"], c["packed"], w["Yd"][M], yh[key], ws, stream)
+        stream.synchronize()
 
     for _ in range(3):
         e2e_step()

@@ -260,6 +260,18 @@ fq_status_t fq_fused_host_io(const fq_layout_t* L, const void* X_host, uint32_t 
                              const void* packed_outliers, void* y_dev, void* Y_host, void* workspace,
                              size_t workspace_bytes, void* cuda_stream);
 
+/* The same without the final wait: enqueues the copy of X, the kernel and the
+ * copy of Y on `cuda_stream` and returns.  X_host must stay valid and Y_host
+ * must not be read until the caller has synchronised the stream (use pinned
+ * host memory, or the copies are not asynchronous).  Several calls may be
+ * enqueued before one synchronisation if each has staging buffers of its own;
+ * they may share the scratch, since they run in stream order. */
+fq_status_t fq_fused_host_io_async(const fq_layout_t* L, const void* X_host, uint32_t M, void* x_dev,
+                                   const void* wq, const void* scale, const void* zero,
+                                   const void* tile_indptr, const void* bucket_info,
+                                   const void* packed_outliers, void* y_dev, void* Y_host,
+                                   void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Synchronise the stream and return the scratch's status word: FQ_OK, or
  * FQ_ERR_TIMEOUT if a bounded wait expired in a kernel (Y is then undefined);
  * the word is cleared. */

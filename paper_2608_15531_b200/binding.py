@@ -28,6 +28,7 @@ EXPORTS = [
     "fq_get_layout", "fq_pack_int4_sizes", "fq_pack_int4", "fq_unpack_int4", "fq_encode_tilecoo_sizes",
     "fq_encode_tilecoo", "fq_decode_tilecoo", "fq_validate_tilecoo", "fq_workspace_bytes",
     "fq_fused_w4a16_outlier_gemm", "fq_fused_w4a16_outlier_gemm_noalloc", "fq_unfused_gemm", "fq_unfused_spmm", "fq_fused_host_io",
+    "fq_fused_host_io_async",
     "fq_check_status", "fq_last_error",
 ]
 
@@ -215,6 +216,18 @@ def fq_fused_host_io(L: Layout, X_host, M: int, x_dev, wq, scale, zero, tile_ind
     _check(lib().fq_fused_host_io(ctypes.byref(L), xh, ctypes.c_uint32(M), _dp(x_dev), _dp(wq), _dp(scale), _dp(zero),
                                   _dp(tile_indptr), _dp(bucket_info), _dp(packed), _dp(y_dev), yh, _dp(workspace),
                                   ctypes.c_size_t(workspace.numel() * workspace.element_size()), _stream(stream)))
+
+
+def fq_fused_host_io_async(L: Layout, X_host, M: int, x_dev, wq, scale, zero, tile_indptr, bucket_info, packed, y_dev,
+                           Y_host, workspace, stream=None) -> None:
+    """As fq_fused_host_io, without the final wait: the caller synchronises the stream before reading Y_host
+    (pinned host tensors)."""
+    xh = ctypes.c_void_p(X_host.data_ptr() if hasattr(X_host, "data_ptr") else X_host.ctypes.data)
+    yh = ctypes.c_void_p(Y_host.data_ptr() if hasattr(Y_host, "data_ptr") else Y_host.ctypes.data)
+    _check(lib().fq_fused_host_io_async(ctypes.byref(L), xh, ctypes.c_uint32(M), _dp(x_dev), _dp(wq), _dp(scale),
+                                        _dp(zero), _dp(tile_indptr), _dp(bucket_info), _dp(packed), _dp(y_dev), yh,
+                                        _dp(workspace),
+                                        ctypes.c_size_t(workspace.numel() * workspace.element_size()), _stream(stream)))
 
 
 def fq_check_status(workspace, stream=None) -> None:

@@ -1799,10 +1799,10 @@ fq_status_t fq_unfused_spmm(const fq_layout_t* L, const void* X, uint32_t M, con
     return FQ_OK;
 }
 
-fq_status_t fq_fused_host_io(const fq_layout_t* L, const void* X_host, uint32_t M, void* x_dev, const void* wq,
-                             const void* scale, const void* zero, const void* tile_indptr, const void* bucket_info,
-                             const void* packed_outliers, void* y_dev, void* Y_host, void* workspace,
-                             size_t workspace_bytes, void* cuda_stream) {
+fq_status_t fq_fused_host_io_async(const fq_layout_t* L, const void* X_host, uint32_t M, void* x_dev, const void* wq,
+                                   const void* scale, const void* zero, const void* tile_indptr,
+                                   const void* bucket_info, const void* packed_outliers, void* y_dev, void* Y_host,
+                                   void* workspace, size_t workspace_bytes, void* cuda_stream) {
     if (!layout_ok(L)) return fail(FQ_ERR_INVALID_ARG, "bad layout");
     if (!X_host || !Y_host || !x_dev || !y_dev) return fail(FQ_ERR_INVALID_ARG, "null pointer");
     if (M < 1 || M > FQ_MAX_M) return fail(FQ_ERR_INVALID_ARG, "M = %u outside [1, %u]", M, FQ_MAX_M);
@@ -1813,8 +1813,19 @@ fq_status_t fq_fused_host_io(const fq_layout_t* L, const void* X_host, uint32_t 
                                                  packed_outliers, y_dev, workspace, workspace_bytes, cuda_stream);
     if (st != FQ_OK) return st;
     e = cudaMemcpyAsync(Y_host, y_dev, (size_t)M * L->N * 2, cudaMemcpyDeviceToHost, s);
-    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "copy of Y: %s", cudaGetErrorString(e));
+    return FQ_OK;
+}
+
+fq_status_t fq_fused_host_io(const fq_layout_t* L, const void* X_host, uint32_t M, void* x_dev, const void* wq,
+                             const void* scale, const void* zero, const void* tile_indptr, const void* bucket_info,
+                             const void* packed_outliers, void* y_dev, void* Y_host, void* workspace,
+                             size_t workspace_bytes, void* cuda_stream) {
+    fq_status_t st = fq_fused_host_io_async(L, X_host, M, x_dev, wq, scale, zero, tile_indptr, bucket_info,
+                                            packed_outliers, y_dev, Y_host, workspace, workspace_bytes, cuda_stream);
+    if (st != FQ_OK) return st;
+    cudaError_t e = cudaStreamSynchronize((cudaStream_t)cuda_stream);
+    if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "stream synchronisation: %s", cudaGetErrorString(e));
     return FQ_OK;
 }
 

@@ -189,6 +189,16 @@ def test_host_io_entry_point_matches_device_entry_point():
     fq.fq_fused_host_io(P.L, xh, M, xd, P.d["wq"], P.d["scale"], P.d["zero"], P.d["indptr"], P.d["info"],
                         P.d["packed"], yd, yh, P.ws)
     assert np.array_equal(yh.numpy().view(np.uint16), Y_dev)
+    # the asynchronous form: two calls enqueued, one synchronisation
+    yh2 = torch.zeros((M, N), dtype=torch.int16).pin_memory()
+    yd2 = torch.empty((M, N), dtype=torch.int16, device="cuda")
+    xd2 = torch.empty((M, K), dtype=torch.int16, device="cuda")
+    yh.zero_()
+    for (a_x, a_y, a_yh) in ((xd, yd, yh), (xd2, yd2, yh2)):
+        fq.fq_fused_host_io_async(P.L, xh, M, a_x, P.d["wq"], P.d["scale"], P.d["zero"], P.d["indptr"], P.d["info"],
+                                  P.d["packed"], a_y, a_yh, P.ws)
+    torch.cuda.synchronize()
+    assert np.array_equal(yh.numpy().view(np.uint16), Y_dev) and np.array_equal(yh2.numpy().view(np.uint16), Y_dev)
 
 
 # ------------------------------------------------------------------ full-size, sampled columns

@@ -970,15 +970,16 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
         uint32_t piece = 0;
         bool ok = true;
         // outer loop: the pieces of this CTA's range (a piece = its units of one column tile); inner loop:
-        // the units of the piece.  The end-of-piece code stays out of the inner loop's body.
-        UnitIter w(u_begin, KT);
-        while (w.u < u_end && ok) {
-          const uint32_t tn = w.tn;
+        // this group's units of the piece (every NGRP-th unit of the range; the ring length is a multiple
+        // of NGRP).  The end-of-piece code stays out of the inner loop's body.
+        uint32_t u = u_begin + grp, s = grp, ph = 0;                    // this group's next unit, its stage and parity
+        uint32_t tn = u_begin / KT;
+        for (uint32_t piece_first = u_begin; piece_first < u_end && ok; ++tn) {
           const uint32_t piece_stop = min(u_end, (tn + 1) * KT);        // one past the piece's last unit
-          for (; w.u < piece_stop; w.next(S, KT)) {
-            const uint32_t u = w.u, s = w.s, ph = w.ph;
+          piece_first = piece_stop;
+          for (; u < piece_stop; u += NGRP, s = (s + NGRP >= S ? s + NGRP - S : s + NGRP), ph ^= (s < (uint32_t)NGRP ? 1u : 0u)) {
             const uint8_t* st = smem + s * p.stage_bytes;
-            if ((w.it % NGRP) == (uint32_t)grp) {
+            {
 #ifdef FQ_TRACE
             long long tw0 = clock64();
 #endif
@@ -986,7 +987,7 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
 #ifdef FQ_TRACE
             long long tw1 = clock64();
 #endif
-            FQ_GT(dtid == 0 && w.it == 0, 2);
+            FQ_GT(dtid == 0 && u == u_begin, 2);
             const uint32_t* wp = reinterpret_cast<const uint32_t*>(st) + c0 * 4 + t;
             const uint8_t* xrow = st + p.off_xcan + g * kXPitch + t * 16;
             const uint16_t* sc = reinterpret_cast<const uint16_t*>(st + p.off_sz);

@@ -301,3 +301,33 @@ def test_tcgen05_engine_in_a_child_process():
                         "test_zero_density or test_oversized_tiles"], cwd=root, env=env, capture_output=True,
                        text=True, timeout=900)
     assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-2000:]
+
+
+# ------------------------------------------------------------------ ordering of dependent calls
+
+@pytest.mark.parametrize("M", [1, 8, 16])
+def test_back_to_back_dependent_calls_keep_stream_order(M):
+    """The small-batch kernel may start while the kernel before it in the stream is draining.  A call
+    whose activations are the previous call's output must still see all of it: chain three calls
+    Y1 = f(X), Y2 = f(Y1), Y3 = f(Y2) without any synchronisation in between and compare every link
+    with the oracle applied to the link's actual input."""
+    K = N = 2048
+    g = 128
+    lay = synth.layer(synth.tensor_seed(8, 77), K, N, density=0.01, layout="mixed")
+    P = H.pack_layer(lay, g)
+    X0 = H.to_dev(_x(5, M, K))
+    Ys = [torch.full((M, N), 0x7fc0, dtype=torch.int16, device="cuda") for _ in range(3)]
+    for rep in range(5):
+        src = X0
+        for Y in Ys:
+            fq.fq_fused_w4a16_outlier_gemm(P.L, src, M, P.d["wq"], P.d["scale"], P.d["zero"], P.d["indptr"],
+                                           P.d["info"], P.d["packed"], Y, P.ws)
+            src = Y
+        fq.fq_check_status(P.ws)
+        chain = [X0] + Ys
+        for a, b in zip(chain[:-1], chain[1:]):
+            xin = a.cpu().numpy().view(np.uint16)
+            Yref, Yabs = H.oracle_result(P, xin)
+            H.check_tolerances(b.cpu().numpy().view(np.uint16), Yref, Yabs, K)
+        for Y in Ys:
+            Y.fill_(0x7fc0)

@@ -28,13 +28,17 @@
  *   INT4 weights.  BK = 128 rows, BN = 128 or 256 columns per tile.  The buffer
  *   is a sequence of chunks, one per (column tile tn, row tile kt), chunk index
  *   tn * (K/128) + kt, each 16 * BN little-endian 32-bit words.  Word index
- *   inside a chunk is (j*BN + t)*4 + w  (j = 0..3: 32-row block, t = column
- *   inside the tile, w = 0..3: 8-row block).  Nibble p = i + 4h (i = 0..3,
- *   h = 0..1; bits 4p..4p+3) of that word is the code of
+ *   inside a chunk, with integer division, is
+ *       (((j*(BN/32) + t/32)*8 + t%8)*4 + w)*4 + (t/8)%4
+ *   (j = 0..3: 32-row block, t = column inside the tile, w = 0..3: 8-row
+ *   block).  Nibble p = i + 4h (i = 0..3, h = 0..1; bits 4p..4p+3) of that
+ *   word is the code of
  *       column tn*BN + t
  *       row    kt*128 + 32j + 8w + 2i + h .
- *   (The four words of one column and one 32-row block are 16 contiguous
- *   bytes, and one shift-and-mask turns nibbles i and i+4 of a word into a BF16
+ *   (Inside a 32-row by 32-column block, the words of columns g, g+8, g+16,
+ *   g+24 and one 8-row block are 16 contiguous bytes: what one lane of the
+ *   small-batch kernel feeds to its m16n8k16 MMAs, fetched with one 128-bit
+ *   load.  One shift-and-mask turns nibbles i and i+4 of a word into a BF16
  *   pair of consecutive rows: the operand order of both tensor-core paths.)
  *
  *   Scale, zero.  (K/group) x N row-major BF16.  zero holds the integer 0..15.
@@ -90,7 +94,7 @@ typedef struct fq_layout {
     uint32_t BK;               /* 128 */
     uint32_t BN;               /* 128 or 256 */
     uint32_t buckets_per_tile; /* NB = BN / 4 */
-    uint32_t wq_interleave;    /* 2: the column-per-thread order described above */
+    uint32_t wq_interleave;    /* 3: the word order described above */
     uint32_t coo_unit_bytes;   /* 16 */
     uint32_t max_tile_packets; /* largest tile of the encoded W_O, in packets; 0 = not encoded */
     uint32_t max_bucket_packets; /* longest packet list of one bucket in one tile; 0 = not encoded */

@@ -192,8 +192,9 @@ void orc_fused_matmul(const uint16_t* X, uint32_t M, uint32_t K, uint32_t N, uin
  *   The buffer is a sequence of chunks, one per (column tile tn, row tile kt),
  *   ordered tn-major (chunk index tn * (K/128) + kt).  A chunk covers 128 rows
  *   by BN columns and holds 16 * BN little-endian 32-bit words.  Word index
- *   inside the chunk:  (j * BN + t) * 4 + w   with j = 0..3, t = 0..BN-1,
- *   w = 0..3.  Nibble p (bits 4p .. 4p+3) of that word, p = i + 4h with
+ *   inside the chunk, with j = 0..3, t = 0..BN-1, w = 0..3:
+ *        (((j * (BN/32) + t/32) * 8 + t%8) * 4 + w) * 4 + (t/8)%4
+ *   (integer division).  Nibble p (bits 4p .. 4p+3) of that word, p = i + 4h with
  *   i = 0..3, h = 0..1, is the code of
  *        column  tn*BN + t
  *        row     kt*128 + 32*j + 8*w + 2*i + h
@@ -208,7 +209,7 @@ int orc_decode_wq(const uint32_t* wq, uint32_t K, uint32_t N, uint32_t BN, uint8
             for (uint32_t j = 0; j < 4; ++j)
                 for (uint32_t t = 0; t < BN; ++t)
                     for (uint32_t w = 0; w < 4; ++w) {
-                        uint32_t word = chunk[(j * BN + t) * 4 + w];
+                        uint32_t word = chunk[(((j * (BN / 32) + t / 32) * 8 + t % 8) * 4 + w) * 4 + (t / 8) % 4];
                         for (uint32_t p = 0; p < 8; ++p) {
                             uint32_t i = p & 3, h = p >> 2;
                             uint32_t col = tn * BN + t;

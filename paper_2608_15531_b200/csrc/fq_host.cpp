@@ -31,7 +31,8 @@ static inline float bf16_to_f32(uint16_t h) {
 // Position of the code of (row kr, column cr) inside a 128 x BN chunk: word index and nibble.
 static inline void wq_slot(uint32_t kr, uint32_t cr, uint32_t BN, uint32_t& word, uint32_t& nib) {
     const uint32_t j = kr >> 5, w = (kr >> 3) & 3, i = (kr >> 1) & 3, h = kr & 1;
-    word = (j * BN + cr) * 4 + w;
+    const uint32_t strip = cr >> 5, qd = (cr >> 3) & 3, g = cr & 7;
+    word = (((j * (BN / 32) + strip) * 8 + g) * 4 + w) * 4 + qd;
     nib = i + 4 * h;
 }
 }  // namespace fq
@@ -63,7 +64,7 @@ fq_status_t fq_get_layout(uint32_t K, uint32_t N, uint32_t group, uint32_t bn_hi
     out->BK = FQ_BK;
     out->BN = BN;
     out->buckets_per_tile = NB;
-    out->wq_interleave = 2;
+    out->wq_interleave = 3;
     out->coo_unit_bytes = 16;
     return FQ_OK;
 }

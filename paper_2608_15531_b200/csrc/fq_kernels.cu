@@ -538,10 +538,11 @@ __global__ void __launch_bounds__(32 * (4 + 2 * (BN / 32) + 4), 1) fq_fused_kern
             tc_fence_after();
             FQ_DSTAMP(it, 0);
             // four 16-byte chunks = 128 codes of this column -> A operand rows in TMEM
-            const uint4* wp = reinterpret_cast<const uint4*>(st) + col;
+            const uint32_t* wp = reinterpret_cast<const uint32_t*>(st) + ((col >> 5) * 8 + (col & 7)) * 16 + ((col >> 3) & 3);
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                const uint4 w4 = wp[j * BN];
+                uint4 w4;                                           // the column's words of 8-row blocks 0..3
+                w4.x = wp[j * BN * 4], w4.y = wp[j * BN * 4 + 4], w4.z = wp[j * BN * 4 + 8], w4.w = wp[j * BN * 4 + 12];
 #pragma unroll
                 for (int hf = 0; hf < 2; ++hf) {
                     const uint32_t w0 = hf ? w4.z : w4.x, w1 = hf ? w4.w : w4.y;
@@ -988,7 +989,7 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
             long long tw1 = clock64();
 #endif
             FQ_GT(dtid == 0 && u == u_begin, 2);
-            const uint32_t* wp = reinterpret_cast<const uint32_t*>(st) + c0 * 4 + t;
+            const uint4* wp = reinterpret_cast<const uint4*>(st) + dw * 32 + lane;   // the lane's four columns, 8 rows
             const uint8_t* xrow = st + p.off_xcan + g * kXPitch + t * 16;
             const uint16_t* sc = reinterpret_cast<const uint16_t*>(st + p.off_sz);
             const float* xsum = reinterpret_cast<const float*>(st + p.off_xsum);
@@ -1057,9 +1058,10 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                     uint4 xb[MO];
 #pragma unroll
                     for (int o = 0; o < MO; ++o) xb[o] = *reinterpret_cast<const uint4*>(xrow + o * 8 * kXPitch + j * 64);
+                    const uint4 w4 = wp[j * BN];                    // columns +0, +8, +16, +24
 #pragma unroll
                     for (int cg = 0; cg < CG; ++cg) {
-                        const uint32_t wa = wp[j * BN * 4 + cg * 64], wb = wp[j * BN * 4 + cg * 64 + 32];   // columns +0 and +8
+                        const uint32_t wa = cg ? w4.z : w4.x, wb = cg ? w4.w : w4.y;
                         const uint32_t a0 = codes_to_bf16x2(wa), a1 = codes_to_bf16x2(wa >> 4);
                         const uint32_t a2 = codes_to_bf16x2(wa >> 8), a3 = codes_to_bf16x2(wa >> 12);
                         const uint32_t b0 = codes_to_bf16x2(wb), b1 = codes_to_bf16x2(wb >> 4);

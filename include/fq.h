@@ -45,20 +45,29 @@
  *
  *   Tile-COO.  Tiles are BK x BN, tile index t = tn * (K/128) + kt.
  *   tile_indptr[t] .. tile_indptr[t+1]: the tile's range of 16-byte packets in
- *   packed_outliers (N_tile + 1 entries, uint32).  bucket_info[t*NB + b] =
- *   offset | count << 16 (two uint16): bucket b of tile t owns `count` packets
- *   starting `offset` packets after the tile's first.  NB = BN/4, and the
- *   bucket of tile column c is fixed: 8*(c/32) + c%8, i.e. the four columns
- *   {g, g+8, g+16, g+24} of a 32-column block share a bucket.  (These are the
- *   columns whose accumulators one group of four lanes holds after the
- *   m16n8k16 MMAs of the small-batch kernel, so a bucket is applied in
- *   registers; the paper's load-balancing column permutation, Section 3.2.2, is
- *   replaced by this static assignment.)  A packet holds four outliers: bytes
- *   0-3 row index in the tile, bytes 4-7 column index in the tile, bytes 8-15
- *   four BF16 values.  Inside a bucket the entries are stored by (row, column);
- *   the last packet is filled up with padding slots: value bits 0x0000, row 0,
- *   the bucket's first column.  Every slot, padding included, has row < 128 and
- *   column < BN.  Storage: (N_tile+1)*4 + N_tile*NB*4 + 16*packets bytes.
+ *   packed_outliers (N_tile + 1 entries, uint32).  NB = BN/4 buckets per tile,
+ *   and the bucket of tile column c is fixed: 8*(c/32) + c%8, i.e. the four
+ *   columns {g, g+8, g+16, g+24} of a 32-column block share a bucket; column
+ *   g + 8j is column number j of its bucket.  (These are the columns whose
+ *   accumulators one group of four lanes holds after the m16n8k16 MMAs of the
+ *   small-batch kernel, so a bucket is applied in registers; the paper's
+ *   load-balancing column permutation, Section 3.2.2, is replaced by this
+ *   static assignment.)
+ *     bucket_info[t*NB + b] = offset | depth << 16 | tail << 24  (uint16, uint8,
+ *   uint8): bucket b of tile t owns depth + tail packets starting `offset`
+ *   packets after the tile's first.
+ *     A packet is four little-endian 32-bit slots; a slot holds one outlier:
+ *   bits 16-31 the BF16 value, bits 5-11 the row inside the tile (so that
+ *   slot & 0xfe0 is the row times 32), bits 12-13 the column number j, all
+ *   other bits 0.  A padding slot has value bits 0x0000 and row 0.
+ *     The first `depth` packets of a bucket are column-slotted (Section 4.2's
+ *   per-column padding): slot j of packet i is the i-th outlier, by row, of
+ *   column number j, or a padding slot that still names j.  If no column of
+ *   the bucket has more than 16 outliers in the tile, depth is the longest
+ *   column's count and tail is 0.  Otherwise depth is 4, and the outliers
+ *   beyond the first 4 of each column follow in `tail` packets by (row,
+ *   column), four to a packet in any slot, the last one filled with all-zero
+ *   padding slots.  Storage: (N_tile+1)*4 + N_tile*NB*4 + 16*packets bytes.
  */
 #ifndef FQ_H_
 #define FQ_H_
@@ -84,8 +93,8 @@ typedef int32_t fq_status_t;
 #define FQ_BK 128u
 
 /* Plain data, caller-owned.  Filled by fq_get_layout(); fq_encode_tilecoo()
- * writes max_tile_packets and max_bucket_packets (the kernels size their staging
- * by the first and choose their outlier path by the second).  Pass the same
+ * writes max_tile_packets, max_bucket_packets and max_tail_packets (the kernels
+ * size their staging by the first and choose their outlier path by the third).  Pass the same
  * struct to every later call. */
 typedef struct fq_layout {
     uint32_t abi;
@@ -97,8 +106,9 @@ typedef struct fq_layout {
     uint32_t wq_interleave;    /* 3: the word order described above */
     uint32_t coo_unit_bytes;   /* 16 */
     uint32_t max_tile_packets; /* largest tile of the encoded W_O, in packets; 0 = not encoded */
-    uint32_t max_bucket_packets; /* longest packet list of one bucket in one tile; 0 = not encoded */
-    uint32_t reserved[5];
+    uint32_t max_bucket_packets; /* longest packet list (depth + tail) of one bucket in one tile */
+    uint32_t max_tail_packets; /* longest tail; 0 = every packet is column-slotted */
+    uint32_t reserved[4];
 } fq_layout_t;
 
 /* Choose tile sizes for a K x N layer.  bn_hint: 0 = library default (256 when
@@ -134,15 +144,16 @@ fq_status_t fq_unpack_int4(const fq_layout_t* L, const void* wq, uint8_t* q_cano
 /*
  * Tile-COO encoder (Section 3.2.1).  Input: COO triplets on the host (k, n,
  * BF16 value bits), any order; entries whose value is +-0 are dropped.  Every
- * entry goes to the bucket of its column (see "Tile-COO" above); a bucket's
- * entries are stored by (row, column), four to a packet, the last packet padded.
- * The column and element reordering of Section 3.2.2 serve a shared-memory
- * scatter that the kernels here do not have, so they are not applied.
+ * entry goes to the bucket of its column and is stored as "Tile-COO" above
+ * says: column-slotted packets with per-column padding (Section 4.2), and a
+ * tail for a bucket with a very long column.  The column and element
+ * reordering of Section 3.2.2 serve a shared-memory scatter that the kernels
+ * here do not have, so they are not applied.
  *
  * fq_encode_tilecoo_sizes: element counts of the three arrays (tile_indptr in
  * uint32, bucket_info in uint32, packets in 16-byte units) and the largest
- * tile.  fq_encode_tilecoo: writes them and stores max_tile_packets and
- * max_bucket_packets in *L.
+ * tile.  fq_encode_tilecoo: writes them and stores max_tile_packets,
+ * max_bucket_packets and max_tail_packets in *L.
  */
 fq_status_t fq_encode_tilecoo_sizes(const fq_layout_t* L, const uint32_t* k, const uint32_t* n,
                                     const uint16_t* val_bf16, size_t nnz, size_t* n_indptr,

@@ -226,16 +226,19 @@ int orc_decode_wq(const uint32_t* wq, uint32_t K, uint32_t N, uint32_t BN, uint8
  *
  *   Tiles are 128 rows by BN columns, tile index tn * (K/128) + kt.
  *   tile_indptr[t] .. tile_indptr[t+1] is the tile's range of 16-byte packets
- *   in packed_outliers.  bucket_info[t * NB + b] = offset | (count << 16):
- *   bucket b of tile t owns packets [tile_indptr[t] + offset, + count).
- *   A packet is: bytes 0-3 row index inside the tile of slots 0-3, bytes 4-7
- *   column index inside the tile of slots 0-3, bytes 8-15 four BF16 values
- *   (little-endian).  A slot whose value bits are 0x0000 is padding.
+ *   in packed_outliers.  bucket_info[t * NB + b] = offset | (depth << 16) |
+ *   (tail << 24), offset 16 bits, depth and tail 8 bits each: bucket b of
+ *   tile t owns packets [tile_indptr[t] + offset, + depth + tail).  Bucket b
+ *   holds the tile columns 32 * (b / 8) + b % 8 + 8 * j, j = 0..3.
+ *   A packet is four little-endian 32-bit slots.  A slot: bits 16-31 a BF16
+ *   value, bits 5-11 the row inside the tile, bits 12-13 the column number j,
+ *   all other bits 0.  A slot whose value bits are 0x0000 is padding.  In the
+ *   first `depth` packets of a bucket, slot number i names column number i.
  *
  * out_* must have room for 4 * (number of packets) entries; *count receives the
  * number of real entries.  Returns 0, or a negative code for a structural
- * error (-2 indptr not monotone, -3 bucket range outside its tile, -4 index
- * outside the tile).
+ * error (-2 indptr not monotone, -3 bucket range outside its tile, -4 a slot
+ * with stray bits, or a column-slotted slot that names another column).
  */
 int orc_decode_tilecoo(const uint32_t* tile_indptr, const uint32_t* bucket_info,
                        const uint8_t* packed, uint32_t K, uint32_t N, uint32_t BN, uint32_t NB,
@@ -251,17 +254,20 @@ int orc_decode_tilecoo(const uint32_t* tile_indptr, const uint32_t* bucket_info,
             if (p1 < p0) return -2;
             for (uint32_t b = 0; b < NB; ++b) {
                 uint32_t info = bucket_info[t * NB + b];
-                uint32_t off = info & 0xffffu, cnt = info >> 16;
-                if ((size_t)p0 + off + cnt > (size_t)p1) return -3;
-                for (uint32_t i = 0; i < cnt; ++i) {
+                uint32_t off = info & 0xffffu, depth = (info >> 16) & 0xffu, tail = info >> 24;
+                if ((size_t)p0 + off + depth + tail > (size_t)p1) return -3;
+                for (uint32_t i = 0; i < depth + tail; ++i) {
                     const uint8_t* pk = packed + ((size_t)p0 + off + i) * 16;
-                    for (int sidx = 0; sidx < 4; ++sidx) {
-                        uint16_t v = (uint16_t)(pk[8 + 2 * sidx] | (pk[9 + 2 * sidx] << 8));
+                    for (uint32_t sidx = 0; sidx < 4; ++sidx) {
+                        uint32_t slot = (uint32_t)pk[4 * sidx] | ((uint32_t)pk[4 * sidx + 1] << 8) |
+                                        ((uint32_t)pk[4 * sidx + 2] << 16) | ((uint32_t)pk[4 * sidx + 3] << 24);
+                        uint32_t kk = (slot >> 5) & 127u, j = (slot >> 12) & 3u;
+                        uint16_t v = (uint16_t)(slot >> 16);
+                        if ((slot & 0xc01fu) != 0) return -4;
+                        if (i < depth && j != sidx) return -4;
                         if (v == 0) continue;
-                        uint32_t kk = pk[sidx], cc = pk[4 + sidx];
-                        if (kk >= 128 || cc >= BN) return -4;
                         out_k[c] = kt * 128 + kk;
-                        out_n[c] = tn * BN + cc;
+                        out_n[c] = tn * BN + 32 * (b / 8) + b % 8 + 8 * j;
                         out_v[c] = v;
                         if (out_bucket) out_bucket[c] = (uint32_t)(t * NB + b);
                         ++c;

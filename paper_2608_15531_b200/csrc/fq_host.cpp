@@ -185,15 +185,28 @@ struct Entry {
 struct Encoded {
     std::vector<uint32_t> indptr;   // N_tile + 1
     std::vector<uint32_t> info;     // N_tile * NB
-    std::vector<uint8_t> packets;   // 16 * n_packets
+    std::vector<uint32_t> words;    // 4 * n_packets
     uint32_t max_tile_packets = 0;
     uint32_t max_bucket_packets = 0;
+    uint32_t max_tail_packets = 0;
 };
 
 // Bucket of a tile column: the four columns {g, g + 8, g + 16, g + 24} of a 32-column block share
 // bucket 8 * (c / 32) + c % 8.  These are the columns whose accumulators one group of four lanes
 // holds in the small-batch kernel, so a bucket's outliers are applied in registers.
 inline uint32_t bucket_of(uint32_t c) { return ((c >> 5) << 3) | (c & 7u); }
+// Number of a column inside its bucket, and the way back.
+inline uint32_t number_in_bucket(uint32_t c) { return (c >> 3) & 3u; }
+inline uint32_t column_of(uint32_t b, uint32_t j) { return ((b >> 3) << 5) | (b & 7u) | (j << 3); }
+
+// One outlier as a 32-bit word: value in the upper half, row * 32 in bits 5-11, the column's number
+// inside the bucket in bits 12-13.
+inline uint32_t entry_word(uint32_t k, uint32_t j, uint16_t v) { return ((uint32_t)v << 16) | (j << 12) | (k << 5); }
+
+// A column with more entries than this in one tile gives its bucket a tail.
+constexpr uint32_t kSlottedMax = 16;
+// Column-slotted packets of a bucket that has a tail.
+constexpr uint32_t kSlottedWithTail = 4;
 
 fq_status_t encode_impl(const fq_layout_t* L, const uint32_t* k, const uint32_t* n, const uint16_t* v,
                         size_t nnz, Encoded& E) {
@@ -218,37 +231,59 @@ fq_status_t encode_impl(const fq_layout_t* L, const uint32_t* k, const uint32_t*
             sorted[fill[t]++] = Entry{(uint8_t)(k[e] % FQ_BK), (uint8_t)(n[e] % BN), v[e]};
         }
     }
-    // pass 1: per tile, the entries of every bucket in (row, column) order, four to a packet; the
-    // last packet of a bucket is filled up with padding slots (value 0, row 0, the bucket's first column)
+    // pass 1: per tile and bucket, the column-slotted packets (packet i = entry i of each of the
+    // four columns, by row) and, for a bucket with a long column, the tail (the entries beyond each
+    // column's first kSlottedWithTail, by (row, column), four to a packet)
     E.indptr.assign(ntile + 1, 0);
     E.info.assign(ntile * NB, 0);
-    std::vector<std::vector<Entry>> tile_slots(ntile);  // packed slots of every tile, four per packet
+    std::vector<std::vector<uint32_t>> tile_words(ntile);
     int bad = 0;
 #pragma omp parallel for schedule(dynamic, 16)
     for (int64_t t = 0; t < (int64_t)ntile; ++t) {
-        std::vector<std::vector<Entry>> per(NB);
-        for (size_t e = tstart[t]; e < tstart[t + 1]; ++e) per[bucket_of(sorted[e].c)].push_back(sorted[e]);
-        std::vector<Entry>& tp = tile_slots[t];
+        std::vector<std::vector<Entry>> per(NB * 4);      // by (bucket, number in bucket)
+        for (size_t e = tstart[t]; e < tstart[t + 1]; ++e)
+            per[bucket_of(sorted[e].c) * 4 + number_in_bucket(sorted[e].c)].push_back(sorted[e]);
+        std::vector<uint32_t>& tw = tile_words[t];
         uint32_t off = 0;
         for (uint32_t b = 0; b < NB; ++b) {
-            std::sort(per[b].begin(), per[b].end(), [](const Entry& x, const Entry& y) {
+            size_t longest = 0;
+            for (uint32_t j = 0; j < 4; ++j) {
+                std::vector<Entry>& col = per[b * 4 + j];
+                std::sort(col.begin(), col.end(), [](const Entry& x, const Entry& y) { return x.k < y.k; });
+                longest = std::max(longest, col.size());
+            }
+            const uint32_t depth = longest > kSlottedMax ? kSlottedWithTail : (uint32_t)longest;
+            for (uint32_t i = 0; i < depth; ++i)
+                for (uint32_t j = 0; j < 4; ++j) {
+                    const std::vector<Entry>& col = per[b * 4 + j];
+                    tw.push_back(i < col.size() ? entry_word(col[i].k, j, col[i].v) : entry_word(0, j, 0));
+                }
+            std::vector<Entry> rest;
+            for (uint32_t j = 0; j < 4; ++j) {
+                const std::vector<Entry>& col = per[b * 4 + j];
+                if (col.size() > depth) rest.insert(rest.end(), col.begin() + depth, col.end());
+            }
+            std::sort(rest.begin(), rest.end(), [](const Entry& x, const Entry& y) {
                 return x.k != y.k ? x.k < y.k : x.c < y.c;
             });
-            const uint32_t pk = (uint32_t)((per[b].size() + 3) / 4);
-            tp.insert(tp.end(), per[b].begin(), per[b].end());
-            const uint8_t first_col = (uint8_t)(((b >> 3) << 5) | (b & 7u));
-            for (size_t i = per[b].size(); i < (size_t)pk * 4; ++i) tp.push_back(Entry{0, first_col, 0});
-            if (off > 0xffffu || pk > 0xffffu) {
+            const uint32_t tail = (uint32_t)((rest.size() + 3) / 4);
+            for (const Entry& e : rest) tw.push_back(entry_word(e.k, number_in_bucket(e.c), e.v));
+            for (size_t i = rest.size(); i < (size_t)tail * 4; ++i) tw.push_back(0);
+            if (off > 0xffffu || depth > 0xffu || tail > 0xffu) {
 #pragma omp atomic write
                 bad = 1;
             }
-            E.info[(size_t)t * NB + b] = (off & 0xffffu) | (pk << 16);
-            off += pk;
+            E.info[(size_t)t * NB + b] = (off & 0xffffu) | (depth << 16) | (tail << 24);
+            off += depth + tail;
         }
         E.indptr[t + 1] = off;
     }
-    if (bad) return fq::fail(FQ_ERR_UNSUPPORTED_SHAPE, "a bucket exceeds the 16-bit packet offset/count range");
-    for (size_t i = 0; i < E.info.size(); ++i) E.max_bucket_packets = std::max(E.max_bucket_packets, E.info[i] >> 16);
+    if (bad) return fq::fail(FQ_ERR_UNSUPPORTED_SHAPE, "a bucket exceeds the packet offset/count range of its descriptor");
+    for (size_t i = 0; i < E.info.size(); ++i) {
+        const uint32_t depth = (E.info[i] >> 16) & 0xffu, tail = E.info[i] >> 24;
+        E.max_bucket_packets = std::max(E.max_bucket_packets, depth + tail);
+        E.max_tail_packets = std::max(E.max_tail_packets, tail);
+    }
     uint64_t total = 0;
     for (size_t t = 0; t < ntile; ++t) {
         uint32_t c = E.indptr[t + 1];
@@ -257,20 +292,12 @@ fq_status_t encode_impl(const fq_layout_t* L, const uint32_t* k, const uint32_t*
         if (total > 0xffffffffull) return fq::fail(FQ_ERR_UNSUPPORTED_SHAPE, "more than 2^32 packets");
         E.indptr[t + 1] = (uint32_t)total;
     }
-    E.packets.assign((size_t)total * 16, 0);
-    // pass 2: write the packets (row bytes, column bytes, values)
+    E.words.assign((size_t)total * 4, 0);
+    // pass 2: the tiles' packets one after the other
 #pragma omp parallel for schedule(dynamic, 64)
-    for (int64_t t = 0; t < (int64_t)ntile; ++t) {
-        const std::vector<Entry>& tp = tile_slots[t];
-        uint8_t* dst = &E.packets[(size_t)E.indptr[t] * 16];
-        for (size_t sidx = 0; sidx < tp.size(); ++sidx) {
-            uint8_t* pk = dst + (sidx / 4) * 16;
-            pk[sidx % 4] = tp[sidx].k;
-            pk[4 + sidx % 4] = tp[sidx].c;
-            pk[8 + 2 * (sidx % 4)] = (uint8_t)(tp[sidx].v & 0xff);
-            pk[9 + 2 * (sidx % 4)] = (uint8_t)(tp[sidx].v >> 8);
-        }
-    }
+    for (int64_t t = 0; t < (int64_t)ntile; ++t)
+        if (!tile_words[t].empty())
+            std::memcpy(&E.words[(size_t)E.indptr[t] * 4], tile_words[t].data(), tile_words[t].size() * 4);
     return FQ_OK;
 }
 
@@ -288,7 +315,7 @@ fq_status_t fq_encode_tilecoo_sizes(const fq_layout_t* L, const uint32_t* k, con
     if (st != FQ_OK) return st;
     if (n_indptr) *n_indptr = E.indptr.size();
     if (n_bucket_info) *n_bucket_info = E.info.size();
-    if (n_packets) *n_packets = E.packets.size() / 16;
+    if (n_packets) *n_packets = E.words.size() / 4;
     if (max_tile_packets) *max_tile_packets = E.max_tile_packets;
     return FQ_OK;
 }
@@ -301,13 +328,14 @@ fq_status_t fq_encode_tilecoo(fq_layout_t* L, const uint32_t* k, const uint32_t*
     Encoded E;
     fq_status_t st = encode_impl(L, k, n, v, nnz, E);
     if (st != FQ_OK) return st;
-    if (E.packets.size() / 16 > n_packets) return fail(FQ_ERR_BUFFER_TOO_SMALL, "packed_outliers holds %zu packets, %zu needed", n_packets, E.packets.size() / 16);
-    if (!E.packets.empty() && !packed) return fail(FQ_ERR_INVALID_ARG, "fq_encode_tilecoo: null packet buffer");
+    if (E.words.size() / 4 > n_packets) return fail(FQ_ERR_BUFFER_TOO_SMALL, "packed_outliers holds %zu packets, %zu needed", n_packets, E.words.size() / 4);
+    if (!E.words.empty() && !packed) return fail(FQ_ERR_INVALID_ARG, "fq_encode_tilecoo: null packet buffer");
     std::memcpy(tile_indptr, E.indptr.data(), E.indptr.size() * 4);
     std::memcpy(bucket_info, E.info.data(), E.info.size() * 4);
-    if (!E.packets.empty()) std::memcpy(packed, E.packets.data(), E.packets.size());
+    if (!E.words.empty()) std::memcpy(packed, E.words.data(), E.words.size() * 4);
     L->max_tile_packets = E.max_tile_packets;
     L->max_bucket_packets = E.max_bucket_packets;
+    L->max_tail_packets = E.max_tail_packets;
     return FQ_OK;
 }
 
@@ -316,25 +344,24 @@ fq_status_t fq_decode_tilecoo(const fq_layout_t* L, const uint32_t* indptr, cons
     if (!layout_ok(L)) return fail(FQ_ERR_INVALID_ARG, "bad layout");
     if (!indptr || !info || !nnz_inout) return fail(FQ_ERR_INVALID_ARG, "fq_decode_tilecoo: null pointer");
     const uint32_t BN = L->BN, NB = L->buckets_per_tile, KT = L->K / FQ_BK, NT = L->N / BN;
-    const uint8_t* pk = (const uint8_t*)packed;
+    const uint32_t* pw = (const uint32_t*)packed;
     const size_t cap = *nnz_inout;
     size_t c = 0;
     for (uint32_t tn = 0; tn < NT; ++tn)
         for (uint32_t kt = 0; kt < KT; ++kt) {
             size_t t = (size_t)tn * KT + kt;
             for (uint32_t b = 0; b < NB; ++b) {
-                uint32_t i0 = indptr[t] + (info[t * NB + b] & 0xffffu), cnt = info[t * NB + b] >> 16;
-                for (uint32_t i = 0; i < cnt; ++i)
-                    for (int s = 0; s < 4; ++s) {
-                        const uint8_t* p = pk + (size_t)(i0 + i) * 16;
-                        uint16_t val = (uint16_t)(p[8 + 2 * s] | (p[9 + 2 * s] << 8));
-                        if (val == 0) continue;
-                        if (c >= cap) return fail(FQ_ERR_BUFFER_TOO_SMALL, "decode buffer holds %zu entries", cap);
-                        k[c] = kt * FQ_BK + p[s];
-                        n[c] = tn * BN + p[4 + s];
-                        v[c] = val;
-                        ++c;
-                    }
+                const uint32_t inf = info[t * NB + b];
+                const size_t i0 = (size_t)indptr[t] + (inf & 0xffffu), cnt = ((inf >> 16) & 0xffu) + (inf >> 24);
+                for (size_t i = 0; i < cnt * 4; ++i) {
+                    const uint32_t w = pw[i0 * 4 + i];
+                    if ((w >> 16) == 0) continue;
+                    if (c >= cap) return fail(FQ_ERR_BUFFER_TOO_SMALL, "decode buffer holds %zu entries", cap);
+                    k[c] = kt * FQ_BK + ((w >> 5) & 127u);
+                    n[c] = tn * BN + column_of(b, (w >> 12) & 3u);
+                    v[c] = (uint16_t)(w >> 16);
+                    ++c;
+                }
             }
         }
     *nnz_inout = c;
@@ -347,22 +374,22 @@ fq_status_t fq_validate_tilecoo(const fq_layout_t* L, const uint32_t* indptr, co
     if (!indptr || !info || (n_packets && !packed)) return fail(FQ_ERR_INVALID_ARG, "fq_validate_tilecoo: null pointer");
     const uint32_t BN = L->BN, NB = L->buckets_per_tile;
     const size_t ntile = (size_t)(L->K / FQ_BK) * (L->N / BN);
-    const uint8_t* pk = (const uint8_t*)packed;
+    const uint32_t* pw = (const uint32_t*)packed;
     if (indptr[0] != 0) return fail(FQ_ERR_FORMAT, "tile_indptr[0] = %u, expected 0", indptr[0]);
     for (size_t t = 0; t < ntile; ++t) {
         if (indptr[t + 1] < indptr[t]) return fail(FQ_ERR_FORMAT, "tile_indptr decreases at tile %zu", t);
         const uint32_t tile_pk = indptr[t + 1] - indptr[t];
         if ((size_t)indptr[t + 1] > n_packets) return fail(FQ_ERR_FORMAT, "tile %zu ends at packet %u of %zu", t, indptr[t + 1], n_packets);
         for (uint32_t b = 0; b < NB; ++b) {
-            uint32_t off = info[t * NB + b] & 0xffffu, cnt = info[t * NB + b] >> 16;
-            if (off + cnt > tile_pk) return fail(FQ_ERR_FORMAT, "bucket %u of tile %zu covers packets [%u, %u) of %u", b, t, off, off + cnt, tile_pk);
-            for (uint32_t i = 0; i < cnt; ++i) {
-                const uint8_t* p = pk + (size_t)(indptr[t] + off + i) * 16;
-                for (int s = 0; s < 4; ++s) {
-                    if (p[s] >= FQ_BK || p[4 + s] >= BN) return fail(FQ_ERR_FORMAT, "index (%u, %u) outside the tile in tile %zu", p[s], p[4 + s], t);
-                    if ((p[8 + 2 * s] | p[9 + 2 * s]) == 0) continue;  // padding slot
-                    if (bucket_of(p[4 + s]) != b) return fail(FQ_ERR_FORMAT, "column %u of tile %zu sits in bucket %u, not in its own bucket %u", p[4 + s], t, b, bucket_of(p[4 + s]));
-                }
+            const uint32_t inf = info[t * NB + b];
+            const uint32_t off = inf & 0xffffu, depth = (inf >> 16) & 0xffu, tail = inf >> 24;
+            if (off + depth + tail > tile_pk) return fail(FQ_ERR_FORMAT, "bucket %u of tile %zu covers packets [%u, %u) of %u", b, t, off, off + depth + tail, tile_pk);
+            if (depth > kSlottedMax) return fail(FQ_ERR_FORMAT, "bucket %u of tile %zu has %u column-slotted packets, at most %u allowed", b, t, depth, kSlottedMax);
+            for (uint32_t i = 0; i < (depth + tail) * 4; ++i) {
+                const uint32_t w = pw[((size_t)indptr[t] + off) * 4 + i];
+                if (w & 0xc01fu) return fail(FQ_ERR_FORMAT, "bits outside the fields are set in a slot of bucket %u, tile %zu", b, t);
+                if (i < depth * 4 && ((w >> 12) & 3u) != (i & 3u))
+                    return fail(FQ_ERR_FORMAT, "slot %u of a column-slotted packet of bucket %u, tile %zu, names column number %u", i & 3u, b, t, (w >> 12) & 3u);
             }
         }
     }

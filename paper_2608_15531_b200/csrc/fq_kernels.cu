@@ -38,6 +38,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
+#include <type_traits>
 
 #include "fq_internal.h"
 
@@ -106,6 +107,10 @@ __device__ __forceinline__ void mbar_arrive_relaxed(uint32_t bar) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n}" ::"r"(bar), "r"(bytes)
                  : "memory");
+}
+// more bytes for the barrier's current phase, without arriving
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
@@ -278,29 +283,30 @@ __device__ __forceinline__ void fma8(float4& c0, float4& c1, float v, const floa
 }
 
 // One packet (four outliers) against the k-major FP32 activation copy xt ([128][8] floats, 32 B per
-// row k): row c of the FP32 tile += v * x[8o..8o+7][k], slot after slot (Section 4.2, without the
-// per-column padding: every slot carries its own column byte).  Slots of one packet may repeat a
-// column, so each slot finishes its read-modify-write before the next one starts; the activation
-// rows of all four are loaded first.  Padding slots (value 0) are skipped.
+// row k): row c of the FP32 tile += v * x[8o..8o+7][k], slot after slot (Section 4.2).  A slot names
+// its row (slot & 0xfe0 = 32 * row) and its column's number inside the bucket (bits 12-13); col0 is
+// the bucket's column number 0, the others follow 8 apart.  Slots of one packet may share a column,
+// so each slot finishes its read-modify-write before the next one starts; the activation rows of
+// all four are loaded first.  Padding slots (value 0) are skipped.
 template <int Q>
-__device__ __forceinline__ void apply_packet(const uint4 pk, const float* __restrict__ xt, float* shc, uint32_t o, uint32_t ldc) {
-    float v[4];
-    v[0] = bf16lo(pk.z); v[1] = bf16hi(pk.z); v[2] = bf16lo(pk.w); v[3] = bf16hi(pk.w);
+__device__ __forceinline__ void apply_packet(const uint4 pk, const float* __restrict__ xt, float* shc, uint32_t col0,
+                                             uint32_t o, uint32_t ldc) {
+    const uint32_t w[4] = {pk.x, pk.y, pk.z, pk.w};
     float4 x0[4], x1[4];
 #pragma unroll
     for (int s = 0; s < 4; ++s) {
-        const float4* xp = reinterpret_cast<const float4*>(xt + ((pk.x >> (8 * s)) & 0xffu) * 8);
+        const float4* xp = reinterpret_cast<const float4*>(reinterpret_cast<const char*>(xt) + (w[s] & 0xfe0u));
         x0[s] = xp[0];
         x1[s] = xp[1];
     }
 #pragma unroll
     for (int s = 0; s < 4; ++s) {
-        if (v[s] != 0.0f) {
-            const uint32_t c = (pk.y >> (8 * s)) & 0xffu;
+        if (w[s] >> 16) {
+            const uint32_t c = col0 + ((w[s] >> 9) & 0x18u);
             float4* p0 = reinterpret_cast<float4*>(shc + shc_quad<Q>(c, 2 * o, ldc));
             float4* p1 = reinterpret_cast<float4*>(shc + shc_quad<Q>(c, 2 * o + 1, ldc));
             float4 c0 = *p0, c1 = *p1;
-            fma8(c0, c1, v[s], x0[s], x1[s]);
+            fma8(c0, c1, __uint_as_float(w[s] & 0xffff0000u), x0[s], x1[s]);
             *p0 = c0;
             *p1 = c1;
         }
@@ -697,7 +703,8 @@ __global__ void __launch_bounds__(32 * (4 + 2 * (BN / 32) + 4), 1) fq_fused_kern
                 if (!warp_wait(bar_full + 8 * s, ph, abort_flag, p.status)) break;
                 if (sw == 0) FQ_STAMP(3, w.it, 0);
                 const uint32_t info = reinterpret_cast<const uint32_t*>(st + p.off_info)[bucket];
-                const uint32_t off = info & 0xffffu, cnt = info >> 16;
+                const uint32_t off = info & 0xffffu, cnt = ((info >> 16) & 0xffu) + (info >> 24);   // column-slotted + tail
+                const uint32_t col0 = ((bucket >> 3) << 5) | (bucket & 7u);
                 const uint4* pk_s = reinterpret_cast<const uint4*>(st + p.off_coo);
                 const uint4* pk_g = nullptr;
                 if (off + cnt > p.coo_cap) pk_g = p.packed + __ldg(p.indptr + u);  // tail of an oversized tile
@@ -714,7 +721,7 @@ __global__ void __launch_bounds__(32 * (4 + 2 * (BN / 32) + 4), 1) fq_fused_kern
                     for (uint32_t i = 0; i < cnt; ++i) {
                         const uint32_t idx = off + i;
                         const uint4 pk = (idx < p.coo_cap) ? pk_s[idx] : __ldg(pk_g + idx);
-                        apply_packet<LDC / 4>(pk, xt, shc, o, LDC);
+                        apply_packet<LDC / 4>(pk, xt, shc, col0, o, LDC);
                     }
                     __syncwarp();
                 }
@@ -809,9 +816,10 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
     FQ_GT(tid == 0, 1);
     // The grid after this one in the stream may start now (it takes SMs as this grid's CTAs leave).
     // Every warp but the producer waits for the grid before this one to finish: the producer reads
-    // only weights, which no kernel writes while calls are in flight.
+    // only weights, which no kernel writes while calls are in flight.  (The activation warps of a
+    // kernel with outliers first request the outlier arrays of their first units, see there.)
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (warp != 0) asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (warp != 0 && !(SPARSE && warp < DW0)) asm volatile("griddepcontrol.wait;" ::: "memory");
 
     const uint32_t KT = p.KT;
     const uint32_t U = p.NT * KT, P = gridDim.x, q = U / P, r = U % P;
@@ -828,21 +836,14 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer
-        uint32_t ip_a = 0, ip_b = 0, issued = 0;
+        // Weights, scales and zero-points of every unit.  (The unit's outlier arrays are requested by
+        // its activation warp: a bulk copy costs its issuing warp a few hundred cycles next to the
+        // dense warps' shared-memory traffic, and five of them per unit made this warp the
+        // bottleneck of the small-batch kernels.)
+        uint32_t issued = 0;
         bool ok = true;
         for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
             const uint32_t u = w.u, it = w.it, s = w.s, ph = w.ph;
-            if (SPARSE && (it & 31) == 0) {
-                const uint32_t i = u + lane;
-                ip_a = (i <= U) ? __ldg(p.indptr + i) : 0;
-                ip_b = (i + 1 <= U) ? __ldg(p.indptr + i + 1) : 0;
-            }
-            uint32_t pk0 = 0, npk = 0;
-            if (SPARSE) {
-                pk0 = __shfl_sync(0xffffffffu, ip_a, it & 31);
-                npk = __shfl_sync(0xffffffffu, ip_b, it & 31) - pk0;
-                npk = min(npk, p.coo_cap);
-            }
 #ifdef FQ_TRACE
             long long tw0 = clock64();
 #endif
@@ -854,23 +855,13 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
             const uint32_t full = bar_full + 8 * s;
             const uint32_t st = smem_u32(smem) + s * p.stage_bytes;
             if (lane == 0) {
-                uint32_t bytes = W_BYTES + 2 * GPS * SZ_ROW;
-                if (SPARSE) bytes += p.NB * 4 + npk * 16;
-                mbar_arrive_expect_tx(full, bytes);
-            }
-            __syncwarp();
-            if (lane == 0) {
+                mbar_arrive_expect_tx(full, W_BYTES + 2 * GPS * SZ_ROW);
                 bulk_g2s(st, p.wq + (size_t)u * W_BYTES, W_BYTES, full);
 #pragma unroll
                 for (int gi = 0; gi < GPS; ++gi) {
                     const size_t row = (size_t)(kt * GPS + gi) * p.N + (size_t)tn * BN;
                     bulk_g2s(st + p.off_sz + gi * SZ_ROW, p.scale + row, SZ_ROW, full);
                     bulk_g2s(st + p.off_sz + (GPS + gi) * SZ_ROW, p.zero + row, SZ_ROW, full);
-                }
-            } else if (lane == 1) {
-                if (SPARSE) {
-                    bulk_g2s(st + p.off_info, p.info + (size_t)u * p.NB, p.NB * 4, full);
-                    if (npk) bulk_g2s(st + p.off_coo, p.packed + pk0, npk * 16, full);
                 }
             }
             issued = it + 1;
@@ -897,7 +888,27 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                 if (real) nxt[c] = __ldg(reinterpret_cast<const uint4*>(xrow + (size_t)kt * 256 + c * 16));
             }
         };
-        if (u_begin + aw < u_end) load((u_begin + aw) % KT);
+        // the unit's range of outlier packets (lane 0), read one unit ahead like the activations
+        uint32_t ip_nxt = 0, ip_nxt_end = 0, last_bar = 0, last_ph = 0;
+        bool ok = true;
+        auto load_ip = [&](uint32_t u) {
+            if (SPARSE && lane == 0) { ip_nxt = __ldg(p.indptr + u); ip_nxt_end = __ldg(p.indptr + u + 1); }
+        };
+        if (SPARSE) {
+            // The first pass over the ring finds every stage empty, and the outlier arrays are weights:
+            // lane l requests those of this warp's l-th unit before the wait for the previous grid.
+            const uint32_t it0 = aw + NA * lane;
+            if (it0 < min(S, u_end - u_begin)) {
+                const uint32_t u = u_begin + it0, a = __ldg(p.indptr + u), npk = min(__ldg(p.indptr + u + 1) - a, p.coo_cap);
+                const uint32_t full = bar_full + 8 * it0, sta = smem_u32(smem) + it0 * p.stage_bytes;
+                mbar_expect_tx(full, p.NB * 4 + npk * 16);
+                bulk_g2s(sta + p.off_info, p.info + (size_t)u * p.NB, p.NB * 4, full);
+                if (npk) bulk_g2s(sta + p.off_coo, p.packed + a, npk * 16, full);
+            }
+            __syncwarp();
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+        }
+        if (u_begin + aw < u_end) { load((u_begin + aw) % KT); load_ip(u_begin + aw); }
         for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
             if (w.it % NA != aw) continue;
             const uint32_t s = w.s, ph = w.ph;
@@ -905,14 +916,24 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
             uint4 xv[CPL];
 #pragma unroll
             for (int c = 0; c < CPL; ++c) xv[c] = nxt[c];
-            if (w.u + NA < u_end) { uint32_t kn = w.kt + NA; load(kn >= KT ? kn % KT : kn); }   // this warp's next unit
+            const uint32_t ip = ip_nxt, npk = min(ip_nxt_end - ip_nxt, p.coo_cap);
+            if (w.u + NA < u_end) { uint32_t kn = w.kt + NA; load(kn >= KT ? kn % KT : kn); load_ip(w.u + NA); }   // this warp's next unit
 #ifdef FQ_TRACE
             long long tw0 = clock64();
 #endif
-            if (!warp_wait(bar_empty + 8 * s, ph ^ 1, abort_flag, p.status)) break;
+            if (!warp_wait(bar_empty + 8 * s, ph ^ 1, abort_flag, p.status)) { ok = false; break; }
 #ifdef FQ_TRACE
             long long tw1 = clock64();
 #endif
+            last_bar = bar_full + 8 * s, last_ph = ph;
+            if (SPARSE && lane == 0 && w.it >= S) {
+                // bucket descriptors and packets of the unit, counted on the stage's barrier before
+                // this warp's own arrival
+                const uint32_t full = bar_full + 8 * s, sta = smem_u32(st);
+                mbar_expect_tx(full, p.NB * 4 + npk * 16);
+                bulk_g2s(sta + p.off_info, p.info + (size_t)w.u * p.NB, p.NB * 4, full);
+                if (npk) bulk_g2s(sta + p.off_coo, p.packed + ip, npk * 16, full);
+            }
             uint8_t* dst = st + p.off_xcan + m * kXPitch + part * CPL * 16;
             float sum = 0.0f;
 #pragma unroll
@@ -948,6 +969,8 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
             if (blockIdx.x == 0 && lane == 0 && aw == 0) { g_trace[10] += tw1 - tw0; g_trace[11] += clock64() - tw1; g_trace[12] += 1; }
 #endif
         }
+        if (SPARSE && !ok && last_bar)      // gave up: let this warp's last copies land before the CTA exits
+            for (uint32_t spin = 0; spin < (1u << 20) && !mbar_try_wait(last_bar, last_ph); ++spin) {}
     } else if (warp >= DW0 && warp < DW0 + NGRP * NDW) {
         // ------------------------------------------------------------------ dense warps (all alike)
         // Two groups of NDW warps take alternate units, each with accumulators of its own: twice the
@@ -994,51 +1017,50 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
             const uint16_t* sc = reinterpret_cast<const uint16_t*>(st + p.off_sz);
             const float* xsum = reinterpret_cast<const float*>(st + p.off_xsum);
             // outliers: the bucket descriptor and the first two packets are requested now and used
-            // after the dense math of the unit
+            // after the dense math of the unit.  A bucket's packets are column-slotted: slot j of a packet
+            // belongs to column number j of the bucket, so a slot's accumulators are known at compile time.
+            // PKT is what a lane reads of a packet: its own slot (MS == 1, lane t keeps column number t) or
+            // all four (MS == 8, lane t keeps batch rows 2t, 2t + 1 of all four columns).
             // HOT is the general form of the outlier step, chosen by the host for layers that need it:
-            //  - very long bucket lists (hot columns): the longest list of a warp's eight buckets is not
-            //    walked by its lane group alone; beyond its first kOwn packets it is shared out over the eight
-            //    lane groups, which add into sums of their own that are added up over the groups afterwards;
+            //  - buckets with a tail (a very long column): the tail's packets, whose slots name their
+            //    column, are shared out over the eight lane groups, which add into sums of their own that
+            //    are added up over the groups afterwards;
             //  - tiles with more packets than a stage holds: the rest is read from global memory.
             // Kernels for layers that need neither are compiled without that code: the presence of either
             // costs the common path 3-4 %.
-            constexpr uint32_t kOwn = 4;
-            uint32_t sp_off = 0, sp_cnt = 0, cmax = 0, hot_off = 0, hot_cnt = 0, hot_g = 0;
+            using PKT = typename std::conditional<MS == 1, uint32_t, uint4>::type;
+            uint32_t sp_off = 0, sp_cnt = 0, sp_tail = 0, cmax = 0;
             const uint4* pk_s = reinterpret_cast<const uint4*>(st + p.off_coo);
             const uint4* pk_g = nullptr;
-            const float* xt = reinterpret_cast<const float*>(st + p.off_xt);
-            auto packet = [&](uint32_t i) {
-                uint4 pk = make_uint4(0, 0, 0, 0);            // beyond the bucket's list: four padding slots
-                if (i < sp_cnt) {
-                    const uint32_t idx = sp_off + i;
-                    pk = (!HOT || idx < p.coo_cap) ? pk_s[idx] : __ldg(pk_g + idx);
-                }
+            const char* xtb = reinterpret_cast<const char*>(st + p.off_xt);
+            const uint32_t x_lane = MS == 1 ? 0u : 8u * t;    // byte offset of the lane's batch rows in a row of xt
+            auto load_packet = [&](uint32_t idx) -> PKT {
+                const uint4* src = (!HOT || idx < p.coo_cap) ? pk_s + idx : pk_g + idx;
+                if constexpr (MS == 1) return reinterpret_cast<const uint32_t*>(src)[t];
+                else return *src;
+            };
+            auto packet = [&](uint32_t i) -> PKT {
+                PKT pk = PKT();                               // beyond the bucket's list: padding
+                if (i < sp_cnt) pk = load_packet(sp_off + i);
                 return pk;
             };
-            // rows-by-lane form (MS == 8): activation rows 2t, 2t+1 of every octet for the four slots
-            auto fetch_x = [&](const uint4 pk, float2 (&x2)[4][MO]) {
+            // activation rows 2t, 2t + 1 of every octet for the row of one slot (slot & 0xfe0 = 32 * row)
+            auto slot_x = [&](const uint32_t w, float2 (&x2)[MO]) {
 #pragma unroll
-                for (int e = 0; e < 4; ++e)
-#pragma unroll
-                    for (int o = 0; o < MO; ++o)
-                        x2[e][o] = *reinterpret_cast<const float2*>(xt + 2 * t + o * 1024 + ((pk.x >> (8 * e)) & 0xffu) * 8);
+                for (int o = 0; o < MO; ++o) x2[o] = *reinterpret_cast<const float2*>(xtb + ((w & 0xfe0u) | x_lane) + o * 4096);
             };
-            uint4 pk0 = make_uint4(0, 0, 0, 0), pk1 = pk0;
+            auto fetch_x = [&](const uint4 pk, float2 (&x2)[4][MO]) {
+                slot_x(pk.x, x2[0]); slot_x(pk.y, x2[1]); slot_x(pk.z, x2[2]); slot_x(pk.w, x2[3]);
+            };
+            PKT pk0 = PKT(), pk1 = PKT();
             float2 xa[4][MO];
             if (SPARSE) {
                 const uint32_t info = reinterpret_cast<const uint32_t*>(st + p.off_info)[dw * 8 + g];
                 sp_off = info & 0xffffu;
-                sp_cnt = info >> 16;
+                sp_cnt = (info >> 16) & 0xffu;
+                if (HOT) sp_tail = info >> 24;
                 cmax = __reduce_max_sync(0xffffffffu, sp_cnt);
-                if (HOT && cmax > kOwn) {                            // warp-uniform
-                    const uint32_t hot_lane = __ffs(__ballot_sync(0xffffffffu, sp_cnt == cmax)) - 1;
-                    hot_g = hot_lane >> 2;
-                    hot_off = __shfl_sync(0xffffffffu, sp_off, hot_lane);
-                    hot_cnt = cmax;
-                    if ((uint32_t)g == hot_g) sp_cnt = kOwn;         // the rest of this list is shared out
-                    cmax = __reduce_max_sync(0xffffffffu, sp_cnt);
-                }
-                if (HOT && (sp_off + sp_cnt > p.coo_cap || hot_off + hot_cnt > p.coo_cap))
+                if (HOT && __reduce_max_sync(0xffffffffu, sp_off + sp_cnt + sp_tail) > p.coo_cap)
                     pk_g = p.packed + __ldg(p.indptr + u);           // packets beyond the staged part
                 pk0 = packet(0);
                 pk1 = packet(1);
@@ -1092,62 +1114,54 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                     }
             }
             if (SPARSE) {
-                // ---- outliers of this unit in the lane group's bucket.  All four lanes of the group read
-                // the same packets (padding slots have value 0: they add 0).
+                // ---- outliers of this unit in the lane group's bucket (padding slots have value 0: they
+                // add 0)
                 if constexpr (MS == 1) {
                     // single batch row: lane t keeps the slots of column number t of the bucket
-                    auto apply = [&](const uint4 pk) {
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const uint32_t cls = (pk.y >> (8 * e + 3)) & 3u;     // column number inside the bucket: (c >> 3) & 3
-                            const float v = (e & 1) ? bf16hi(e < 2 ? pk.z : pk.w) : bf16lo(e < 2 ? pk.z : pk.w);
-                            const float x = xt[((pk.x >> (8 * e)) & 0xffu) * 8];
-                            sacc[0][0] = fmaf(cls == (uint32_t)t ? v : 0.0f, x, sacc[0][0]);
-                        }
+                    auto apply = [&](const uint32_t w) {
+                        sacc[0][0] = fmaf(__uint_as_float(w & 0xffff0000u), *reinterpret_cast<const float*>(xtb + (w & 0xfe0u)), sacc[0][0]);
                     };
                     if (cmax > 0) apply(pk0);
                     if (cmax > 1) {
                         apply(pk1);
                         for (uint32_t i = 2; i < cmax; ++i) apply(packet(i));
                     }
-                    if (HOT && hot_cnt) {
-                        float hacc = 0.0f;
-                        for (uint32_t i0 = kOwn; i0 < hot_cnt; i0 += 8) {
-                            const uint32_t i = i0 + g, idx = hot_off + i;
-                            uint4 pk = make_uint4(0, 0, 0, 0);
-                            if (i < hot_cnt) pk = (idx < p.coo_cap) ? pk_s[idx] : __ldg(pk_g + idx);
+                    if (HOT) {
+                        for (uint32_t hot = __ballot_sync(0xffffffffu, sp_tail != 0); hot; ) {     // warp-uniform
+                            const uint32_t hot_lane = __ffs(hot) - 1;
+                            hot &= ~(0xfu << (hot_lane & ~3u));
+                            const uint32_t hot_off = __shfl_sync(0xffffffffu, sp_off + sp_cnt, hot_lane);
+                            const uint32_t hot_cnt = __shfl_sync(0xffffffffu, sp_tail, hot_lane);
+                            float hacc = 0.0f;
+                            for (uint32_t i = g; i < hot_cnt; i += 8) {
+                                const uint32_t idx = hot_off + i;
+                                const uint4 pk = (idx < p.coo_cap) ? pk_s[idx] : __ldg(pk_g + idx);
+                                const uint32_t w[4] = {pk.x, pk.y, pk.z, pk.w};
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const uint32_t cls = (pk.y >> (8 * e + 3)) & 3u;
-                                const float v = (e & 1) ? bf16hi(e < 2 ? pk.z : pk.w) : bf16lo(e < 2 ? pk.z : pk.w);
-                                hacc = fmaf(cls == (uint32_t)t ? v : 0.0f, xt[((pk.x >> (8 * e)) & 0xffu) * 8], hacc);
+                                for (int e = 0; e < 4; ++e) {
+                                    const float v = ((w[e] >> 12) & 3u) == (uint32_t)t ? __uint_as_float(w[e] & 0xffff0000u) : 0.0f;
+                                    hacc = fmaf(v, *reinterpret_cast<const float*>(xtb + (w[e] & 0xfe0u)), hacc);
+                                }
                             }
+                            hacc += __shfl_xor_sync(0xffffffffu, hacc, 4);
+                            hacc += __shfl_xor_sync(0xffffffffu, hacc, 8);
+                            hacc += __shfl_xor_sync(0xffffffffu, hacc, 16);
+                            if ((uint32_t)g == (hot_lane >> 2)) sacc[0][0] += hacc;
                         }
-                        hacc += __shfl_xor_sync(0xffffffffu, hacc, 4);
-                        hacc += __shfl_xor_sync(0xffffffffu, hacc, 8);
-                        hacc += __shfl_xor_sync(0xffffffffu, hacc, 16);
-                        if ((uint32_t)g == hot_g) sacc[0][0] += hacc;
                     }
                 } else {
                     // several batch rows: lane t keeps rows 2t, 2t+1 (+8) of all four columns, in the
-                    // MMA fragment registers themselves
+                    // MMA fragment registers themselves; slot j goes to column number j
                     auto apply = [&](const uint4 pk, const float2 (&x2)[4][MO]) {
-                        const float v[4] = {bf16lo(pk.z), bf16hi(pk.z), bf16lo(pk.w), bf16hi(pk.w)};
+                        const uint32_t w[4] = {pk.x, pk.y, pk.z, pk.w};
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            const uint32_t cls = (pk.y >> (8 * e + 3)) & 3u;
+                            const float v = __uint_as_float(w[e] & 0xffff0000u);
 #pragma unroll
-                            for (int cg = 0; cg < CG; ++cg)
-#pragma unroll
-                                for (int h = 0; h < 2; ++h) {
-                                    // a select, not a branch: the lanes of a warp hold different columns
-                                    const float vv = (cls == (uint32_t)(2 * cg + h)) ? v[e] : 0.0f;
-#pragma unroll
-                                    for (int o = 0; o < MO; ++o) {
-                                        accf[o][cg][2 * h + 0] = fmaf(vv, x2[e][o].x, accf[o][cg][2 * h + 0]);
-                                        accf[o][cg][2 * h + 1] = fmaf(vv, x2[e][o].y, accf[o][cg][2 * h + 1]);
-                                    }
-                                }
+                            for (int o = 0; o < MO; ++o) {
+                                accf[o][e >> 1][2 * (e & 1) + 0] = fmaf(v, x2[e][o].x, accf[o][e >> 1][2 * (e & 1) + 0]);
+                                accf[o][e >> 1][2 * (e & 1) + 1] = fmaf(v, x2[e][o].y, accf[o][e >> 1][2 * (e & 1) + 1]);
+                            }
                         }
                     };
                     if (cmax > 0) apply(pk0, xa);
@@ -1161,49 +1175,56 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                             apply(pk, xb2);
                         }
                     }
-                    if (HOT && hot_cnt) {
-                        float hacc[MO][CG][4];
+                    if (HOT) {
+                        for (uint32_t hot = __ballot_sync(0xffffffffu, sp_tail != 0); hot; ) {     // warp-uniform
+                            const uint32_t hot_lane = __ffs(hot) - 1;
+                            hot &= ~(0xfu << (hot_lane & ~3u));
+                            const uint32_t hot_off = __shfl_sync(0xffffffffu, sp_off + sp_cnt, hot_lane);
+                            const uint32_t hot_cnt = __shfl_sync(0xffffffffu, sp_tail, hot_lane);
+                            float hacc[MO][CG][4];
 #pragma unroll
-                        for (int o = 0; o < MO; ++o)
-#pragma unroll
-                            for (int cg = 0; cg < CG; ++cg)
-#pragma unroll
-                                for (int i = 0; i < 4; ++i) hacc[o][cg][i] = 0.0f;
-                        for (uint32_t i0 = kOwn; i0 < hot_cnt; i0 += 8) {
-                            const uint32_t i = i0 + g, idx = hot_off + i;
-                            uint4 pk = make_uint4(0, 0, 0, 0);
-                            if (i < hot_cnt) pk = (idx < p.coo_cap) ? pk_s[idx] : __ldg(pk_g + idx);
-                            float2 xh[4][MO];
-                            fetch_x(pk, xh);
-                            const float v[4] = {bf16lo(pk.z), bf16hi(pk.z), bf16lo(pk.w), bf16hi(pk.w)};
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const uint32_t cls = (pk.y >> (8 * e + 3)) & 3u;
+                            for (int o = 0; o < MO; ++o)
 #pragma unroll
                                 for (int cg = 0; cg < CG; ++cg)
 #pragma unroll
-                                    for (int h = 0; h < 2; ++h) {
-                                        const float vv = (cls == (uint32_t)(2 * cg + h)) ? v[e] : 0.0f;
+                                    for (int i = 0; i < 4; ++i) hacc[o][cg][i] = 0.0f;
+                            for (uint32_t i = g; i < hot_cnt; i += 8) {
+                                const uint32_t idx = hot_off + i;
+                                const uint4 pk = (idx < p.coo_cap) ? pk_s[idx] : __ldg(pk_g + idx);
+                                float2 xh[4][MO];
+                                fetch_x(pk, xh);
+                                const uint32_t w[4] = {pk.x, pk.y, pk.z, pk.w};
 #pragma unroll
-                                        for (int o = 0; o < MO; ++o) {
-                                            hacc[o][cg][2 * h + 0] = fmaf(vv, xh[e][o].x, hacc[o][cg][2 * h + 0]);
-                                            hacc[o][cg][2 * h + 1] = fmaf(vv, xh[e][o].y, hacc[o][cg][2 * h + 1]);
+                                for (int e = 0; e < 4; ++e) {
+                                    const uint32_t cls = (w[e] >> 12) & 3u;
+                                    const float v = __uint_as_float(w[e] & 0xffff0000u);
+#pragma unroll
+                                    for (int cg = 0; cg < CG; ++cg)
+#pragma unroll
+                                        for (int h = 0; h < 2; ++h) {
+                                            // a select, not a branch: the lanes of a warp hold different columns
+                                            const float vv = (cls == (uint32_t)(2 * cg + h)) ? v : 0.0f;
+#pragma unroll
+                                            for (int o = 0; o < MO; ++o) {
+                                                hacc[o][cg][2 * h + 0] = fmaf(vv, xh[e][o].x, hacc[o][cg][2 * h + 0]);
+                                                hacc[o][cg][2 * h + 1] = fmaf(vv, xh[e][o].y, hacc[o][cg][2 * h + 1]);
+                                            }
                                         }
-                                    }
-                            }
-                        }
-#pragma unroll
-                        for (int o = 0; o < MO; ++o)
-#pragma unroll
-                            for (int cg = 0; cg < CG; ++cg)
-#pragma unroll
-                                for (int i = 0; i < 4; ++i) {
-                                    float v = hacc[o][cg][i];
-                                    v += __shfl_xor_sync(0xffffffffu, v, 4);
-                                    v += __shfl_xor_sync(0xffffffffu, v, 8);
-                                    v += __shfl_xor_sync(0xffffffffu, v, 16);
-                                    if ((uint32_t)g == hot_g) accf[o][cg][i] += v;
                                 }
+                            }
+#pragma unroll
+                            for (int o = 0; o < MO; ++o)
+#pragma unroll
+                                for (int cg = 0; cg < CG; ++cg)
+#pragma unroll
+                                    for (int i = 0; i < 4; ++i) {
+                                        float v = hacc[o][cg][i];
+                                        v += __shfl_xor_sync(0xffffffffu, v, 4);
+                                        v += __shfl_xor_sync(0xffffffffu, v, 8);
+                                        v += __shfl_xor_sync(0xffffffffu, v, 16);
+                                        if ((uint32_t)g == (hot_lane >> 2)) accf[o][cg][i] += v;
+                                    }
+                        }
                     }
                 }
             }
@@ -1378,18 +1399,20 @@ __global__ void __launch_bounds__(256) fq_spmm_kernel(const uint16_t* __restrict
             const size_t t = (size_t)tn * KT + kt;
             const uint32_t inf = __ldg(info + t * NB + b);
             const uint4* pk = packed + __ldg(indptr + t) + (inf & 0xffffu);
-            for (uint32_t i = 0; i < (inf >> 16); ++i) {
+            const uint32_t depth = (inf >> 16) & 0xffu, tail = inf >> 24;
+            for (uint32_t i = 0; i < depth + tail; ++i) {
                 const uint4 q = __ldg(pk + i);
-                const float v[4] = {bf16lo(q.z), bf16hi(q.z), bf16lo(q.w), bf16hi(q.w)};
+                const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    const uint32_t k = kt * kBK + ((q.x >> (8 * e)) & 0xffu), cls = (q.y >> (8 * e + 3)) & 3u;
+                    const uint32_t k = kt * kBK + ((w[e] >> 5) & 127u), cls = (w[e] >> 12) & 3u;
+                    const float v = __uint_as_float(w[e] & 0xffff0000u);
                     const uint16_t* xp = X + (size_t)m0 * K + k;
 #pragma unroll
                     for (int m = 0; m < MB; ++m) {
                         const float x = (m0 + m < M) ? bf16_bits_to_float(__ldg(xp + (size_t)m * K)) : 0.0f;
 #pragma unroll
-                        for (int c = 0; c < 4; ++c) acc[c][m] = fmaf(cls == (uint32_t)c ? v[e] : 0.0f, x, acc[c][m]);
+                        for (int c = 0; c < 4; ++c) acc[c][m] = fmaf(cls == (uint32_t)c ? v : 0.0f, x, acc[c][m]);
                     }
                 }
             }
@@ -1537,7 +1560,7 @@ static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, 
     if (S < 4) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "shared-memory stages do not fit");
     p.coo_cap = cap; p.stages = S; p.stage_bytes = stage;
     // hot columns, tiles larger than the staged part, or an encoding whose sizes were not recorded
-    pl.general = sparse && (L->max_bucket_packets > 16 || L->max_tile_packets > cap || L->max_tile_packets == 0);
+    pl.general = sparse && (L->max_tail_packets > 0 || L->max_tile_packets > cap || L->max_tile_packets == 0);
     p.off_shc = S * stage;
     p.off_bar = p.off_shc + xch_bytes;
     pl.smem = p.off_bar + 1024;

@@ -83,6 +83,21 @@ def _bucket_of(c):
     return (c // 32) * 8 + c % 8
 
 
+def _fields(info):
+    """offset, column-slotted packets, tail packets of every bucket descriptor."""
+    return info & 0xffff, (info >> 16) & 0xff, info >> 24
+
+
+def _column_counts(k, n, K, N, BN):
+    """Outliers per (tile, bucket, column number inside the bucket)."""
+    ntile = (K // 128) * (N // BN)
+    tile = (n // BN) * (K // 128) + k // 128
+    c = n % BN
+    cnt = np.zeros((ntile, BN // 4, 4), dtype=np.int64)
+    np.add.at(cnt, (tile, _bucket_of(c), (c // 8) % 4), 1)
+    return cnt
+
+
 @pytest.mark.parametrize("layout,density,BN", [("uniform", 0.01, 256), ("mixed", 0.02, 256), ("clustered", 0.05, 128)])
 def test_tilecoo_encode_invariants(layout, density, BN):
     K, N = 512, 1024
@@ -93,10 +108,11 @@ def test_tilecoo_encode_invariants(layout, density, BN):
     n_ip, n_bi, n_pk, mx = fq.fq_encode_tilecoo_sizes(L, Lr.coo_k, Lr.coo_n, Lr.coo_v)
     indptr, info, packed = fq.fq_encode_tilecoo(L, Lr.coo_k, Lr.coo_n, Lr.coo_v)
     ntile = (K // 128) * (N // BN)
-    # array sizes and storage formula (Table 1 and the storage analysis), padding bounded per bucket
+    off, depth, tail = _fields(info)
+    # array sizes and storage formula (Table 1 and the storage analysis)
     assert n_ip == ntile + 1 == indptr.size and n_bi == ntile * NB == info.size and n_pk == packed.shape[0]
     assert L.max_tile_packets == mx == int(np.diff(indptr).max())
-    assert L.max_bucket_packets == int((info >> 16).max())
+    assert L.max_bucket_packets == int((depth + tail).max()) and L.max_tail_packets == int(tail.max())
     assert indptr[0] == 0 and np.all(np.diff(indptr.astype(np.int64)) >= 0) and indptr[-1] == n_pk
     assert 4 * Lr.nnz <= 16 * n_pk <= 16 * Lr.nnz          # every packet carries at least one outlier
     # decoded set == input set, by the oracle's reader and by the library's
@@ -109,35 +125,61 @@ def test_tilecoo_encode_invariants(layout, density, BN):
     # every outlier sits in the bucket of its column, in every tile (the conflict-free accumulation of
     # the sparse path: a bucket's four columns belong to one group of four lanes)
     assert np.array_equal(b % NB, _bucket_of(n % BN))
-    # a bucket is padded only in its last packet: packets = ceil(entries / 4)
     tile = (n // BN) * (K // 128) + k // 128
     assert np.array_equal(b // NB, tile)
-    loads = np.bincount(b, minlength=ntile * NB)
-    assert np.array_equal(info >> 16, (loads + 3) // 4)
-    off = (info & 0xffff).reshape(ntile, NB)
-    cnt = (info >> 16).reshape(ntile, NB)
-    assert np.array_equal(off[:, 1:], np.cumsum(cnt, axis=1)[:, :-1]) and not off[:, 0].any()
+    # per-column padding (Section 4.2): a bucket has as many column-slotted packets as its longest
+    # column has outliers; only a column with more than 16 turns that into 4 packets and a tail
+    cnt = _column_counts(Lr.coo_k.astype(np.int64), Lr.coo_n.astype(np.int64), K, N, BN).reshape(ntile * NB, 4)
+    longest = cnt.max(axis=1)
+    want_depth = np.where(longest > 16, 4, longest)
+    want_tail = np.where(longest > 16, (np.maximum(cnt - 4, 0).sum(axis=1) + 3) // 4, 0)
+    assert np.array_equal(depth, want_depth) and np.array_equal(tail, want_tail)
+    if layout == "clustered":
+        assert tail.any()
+    else:
+        assert not tail.any()
+    off = off.reshape(ntile, NB)
+    tot = (depth + tail).reshape(ntile, NB)
+    assert np.array_equal(off[:, 1:], np.cumsum(tot, axis=1)[:, :-1]) and not off[:, 0].any()
 
 
-def test_tilecoo_entries_of_a_bucket_are_stored_by_row_then_column():
+def test_tilecoo_slots_and_order_inside_a_bucket():
     K, N, BN = 128, 256, 256
     NB = BN // 4
-    Lr = synth.layer(77, K, N, density=0.06, layout="uniform")
+    Lr = synth.layer(77, K, N, density=0.03, layout="uniform")
     L = fq.fq_get_layout(K, N, 128, bn_hint=BN)
     indptr, info, packed = fq.fq_encode_tilecoo(L, Lr.coo_k, Lr.coo_n, Lr.coo_v)
-    k, n, v, b = oracle.decode_tilecoo(indptr, info, packed, K, N, BN, NB)   # decode keeps stored order
-    for bb in np.unique(b):
-        sel = b == bb
-        key = k[sel].astype(np.int64) * BN + n[sel]
-        assert np.all(np.diff(key) > 0)
-    # a hot column fills its bucket with packets of four
+    off, depth, tail = _fields(info)
+    assert not tail.any()
+    slots = packed.view(np.uint32).reshape(-1, 4)
+    for bb in range(NB):
+        pk = slots[off[bb]:off[bb] + depth[bb]]
+        # slot j of every packet names column number j, padding included
+        assert np.array_equal((pk >> 12) & 3, np.tile(np.arange(4, dtype=np.uint32), (pk.shape[0], 1)))
+        assert not (pk & 0xc01f).any()
+        for j in range(4):
+            col = (bb // 8) * 32 + bb % 8 + 8 * j
+            want = np.sort(Lr.coo_k[Lr.coo_n == col])
+            live = (pk[:, j] >> 16) != 0
+            # a column's outliers come first, by row; then only padding (value 0, row 0)
+            assert live.sum() == want.size and live[:want.size].all()
+            assert np.array_equal((pk[:want.size, j] >> 5) & 127, want)
+            assert not (pk[want.size:, j] & 0xffff0fe0).any()
+    # a hot column: its first four outliers in column-slotted packets, the rest four to a packet by row
     kk = np.arange(0, 40, dtype=np.uint32)
-    nn = np.full(40, 7, dtype=np.uint32)
+    nn = np.full(40, 15, dtype=np.uint32)                 # column number 1 of bucket 7
     vv = (0x3F80 + np.arange(40)).astype(np.uint16)
     ip, bi, pk = fq.fq_encode_tilecoo(L, kk, nn, vv)
     k2, n2, v2 = fq.fq_decode_tilecoo(L, ip, bi, pk)
-    assert _as_set(k2, n2, v2) == _as_set(kk, nn, vv) and pk.shape[0] == 10
-    assert int(bi[_bucket_of(7)]) >> 16 == 10
+    assert _as_set(k2, n2, v2) == _as_set(kk, nn, vv) and pk.shape[0] == 4 + 9
+    assert int(bi[_bucket_of(15)]) == 0 | (4 << 16) | (9 << 24)
+    assert L.max_tail_packets == 9 and L.max_bucket_packets == 13
+    s2 = pk.view(np.uint32).reshape(-1, 4)
+    assert np.array_equal((s2[:4, 1] >> 5) & 127, np.arange(4)) and not (s2[:4, [0, 2, 3]] >> 16).any()
+    assert np.array_equal((s2[4:].ravel() >> 5) & 127, np.arange(4, 40)) and np.all((s2[4:].ravel() >> 12) & 3 == 1)
+    # exactly 16 in a column still has no tail
+    ip, bi, pk = fq.fq_encode_tilecoo(L, kk[:16], nn[:16], vv[:16])
+    assert int(bi[_bucket_of(15)]) == 0 | (16 << 16) and L.max_tail_packets == 0
 
 
 def test_tilecoo_edge_cases():
@@ -156,9 +198,9 @@ def test_tilecoo_edge_cases():
     assert packed.shape[0] == 1
     kk, nn, vv, _ = oracle.decode_tilecoo(indptr, info, packed, K, N, BN, NB)
     assert (kk.tolist(), nn.tolist(), vv.tolist()) == ([200], [300], [0x4000])
-    # padding slots: value 0, row 0, the first column of the bucket (column 44 -> bucket 8 + 4 -> column 36)
-    assert packed[0, :4].tolist() == [72, 0, 0, 0] and packed[0, 4:8].tolist() == [44, 36, 36, 36]
-    assert packed[0, 10:].tolist() == [0] * 6
+    # column 300 = tile column 44 = column number 1 of bucket 8 + 4; the other slots are padding that
+    # names their own column number
+    assert packed.view(np.uint32).reshape(-1, 4)[0].tolist() == [0 << 12, (0x4000 << 16) | (1 << 12) | (72 << 5), 2 << 12, 3 << 12]
     # one completely dense tile plus a hot row and a hot column elsewhere
     kk, nn = np.meshgrid(np.arange(128, 256), np.arange(0, 256), indexing="ij")
     k = np.concatenate([kk.ravel(), np.full(256, 3), np.arange(0, 128)]).astype(np.uint32)
@@ -195,17 +237,19 @@ def test_validator_rejects_corrupted_arrays():
     expect_format_error(bad, info, packed)
     bad = info.copy(); bad[0] = (bad[0] & 0xffff) | (0xffff << 16)
     expect_format_error(indptr, bad, packed)
-    bad = packed.copy(); bad[0, 0] = 200                 # row index outside the 128-row tile
-    expect_format_error(indptr, info, bad)
-    bad = packed.copy(); bad[0, 5] = 0                   # a padding slot must stay inside the tile too
-    bad[0, 1] = 130
-    expect_format_error(indptr, info, bad)
-    # move one entry into a column that belongs to another bucket
+    slots = packed.view(np.uint32).reshape(-1, 4)
+    bad = slots.copy(); bad[0, 0] |= 1 << 14             # a bit outside the fields
+    expect_format_error(indptr, info, bad.view(np.uint8).reshape(-1, 16))
+    bad = slots.copy(); bad[0, 2] |= 1 << 2
+    expect_format_error(indptr, info, bad.view(np.uint8).reshape(-1, 16))
+    # a column-slotted slot that names another column of the bucket
     k, n, v, b = oracle.decode_tilecoo(indptr, info, packed, K, N, BN, NB)
     b0 = int(b[0])
-    assert b0 < NB
+    assert b0 < NB and (int(info[b0]) >> 16) & 0xff > 0
     off0 = int(info[b0] & 0xffff)
-    bad = packed.copy()
-    assert bad[off0, 8:10].any()
-    bad[off0, 4] = (int(bad[off0, 4]) + 1) % BN
-    expect_format_error(indptr, info, bad)
+    bad = slots.copy()
+    bad[off0, 1] ^= 1 << 12
+    expect_format_error(indptr, info, bad.view(np.uint8).reshape(-1, 16))
+    # more column-slotted packets than the format allows
+    bad = info.copy(); bad[0] = (bad[0] & 0xffff) | (17 << 16)
+    expect_format_error(indptr, bad, packed)

@@ -260,30 +260,40 @@ def test_decode_wq_against_a_direct_packer():
 
 
 def test_decode_tilecoo_hand_built():
-    # K = 128, N = 64, BN = 32 -> 2 tiles; NB = 2 buckets per tile
-    K, N, BN, NB = 128, 64, 32, 2
-    packets = np.zeros((3, 16), dtype=np.uint8)
+    # K = 128, N = 64, BN = 32 -> 2 tiles of 8 buckets; bucket b holds the tile columns b + 8 j
+    K, N, BN, NB = 128, 64, 32, 8
+    slots = np.zeros((4, 4), dtype=np.uint32)
 
-    def put(p, slot, k, c, bits):
-        packets[p, slot] = k
-        packets[p, 4 + slot] = c
-        packets[p, 8 + 2 * slot] = bits & 0xff
-        packets[p, 9 + 2 * slot] = bits >> 8
+    def put(p, slot, k, j, bits):
+        slots[p, slot] = (bits << 16) | (j << 12) | (k << 5)
 
-    # tile 0: bucket 0 has one packet (3 real + 1 pad), bucket 1 empty
-    put(0, 0, 5, 1, 0x3F80); put(0, 1, 127, 31, 0xBF80); put(0, 2, 0, 0, 0x4000); put(0, 3, 0, 0, 0)
-    # tile 1: bucket 0 one packet (1 real), bucket 1 one packet (4 real)
-    put(1, 0, 9, 2, 0x3E00)
-    for i in range(4):
-        put(2, i, 10 + i, 20 + i, 0x4100 + i)
-    indptr = np.array([0, 1, 3], dtype=np.uint32)
-    info = np.array([0 | (1 << 16), 1 | (0 << 16), 0 | (1 << 16), 1 | (1 << 16)], dtype=np.uint32)
+    # tile 0, bucket 1 (columns 1, 9, 17, 25): two column-slotted packets
+    put(0, 0, 5, 0, 0x3F80); put(0, 1, 0, 1, 0); put(0, 2, 127, 2, 0xBF80); put(0, 3, 0, 3, 0)
+    put(1, 0, 9, 0, 0x4000); put(1, 1, 0, 1, 0); put(1, 2, 0, 2, 0); put(1, 3, 0, 3, 0)
+    # tile 1, bucket 7 (columns 7, 15, 23, 31): one column-slotted packet and a tail packet whose
+    # slots name any column; its last slot is all-zero padding
+    put(2, 0, 0, 0, 0); put(2, 1, 0, 1, 0); put(2, 2, 0, 2, 0); put(2, 3, 3, 3, 0x3E00)
+    put(3, 0, 10, 3, 0x4100); put(3, 1, 11, 3, 0x4101); put(3, 2, 11, 0, 0x4102)
+    indptr = np.array([0, 2, 4], dtype=np.uint32)
+    info = np.zeros(2 * NB, dtype=np.uint32)
+    info[1] = 0 | (2 << 16)
+    info[2:8] = 2                            # empty buckets after bucket 1
+    info[NB + 7] = 0 | (1 << 16) | (1 << 24)
+    packets = slots.view(np.uint8).reshape(4, 16)
     k, n, v, b = oracle.decode_tilecoo(indptr, info, packets, K, N, BN, NB)
     got = sorted(zip(k.tolist(), n.tolist(), v.tolist(), b.tolist()))
-    want = sorted([(5, 1, 0x3F80, 0), (127, 31, 0xBF80, 0), (0, 0, 0x4000, 0), (9, 34, 0x3E00, 2)] +
-                  [(10 + i, 32 + 20 + i, 0x4100 + i, 3) for i in range(4)])
+    want = sorted([(5, 1, 0x3F80, 1), (127, 17, 0xBF80, 1), (9, 1, 0x4000, 1), (3, 32 + 31, 0x3E00, NB + 7),
+                   (10, 32 + 31, 0x4100, NB + 7), (11, 32 + 31, 0x4101, NB + 7), (11, 32 + 7, 0x4102, NB + 7)])
     assert got == want
     bad = info.copy()
-    bad[3] = 1 | (2 << 16)                  # bucket runs past its tile
+    bad[NB + 7] = 0 | (1 << 16) | (2 << 24)  # bucket runs past its tile
     with pytest.raises(ValueError):
         oracle.decode_tilecoo(indptr, bad, packets, K, N, BN, NB)
+    wrong = slots.copy()
+    wrong[0, 1] = (0x3F80 << 16) | (2 << 12)  # a column-slotted slot that names another column
+    with pytest.raises(ValueError):
+        oracle.decode_tilecoo(indptr, info, wrong.view(np.uint8).reshape(4, 16), K, N, BN, NB)
+    stray = slots.copy()
+    stray[3, 0] |= 1                         # a bit outside the fields
+    with pytest.raises(ValueError):
+        oracle.decode_tilecoo(indptr, info, stray.view(np.uint8).reshape(4, 16), K, N, BN, NB)

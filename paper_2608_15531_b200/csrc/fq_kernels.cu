@@ -793,6 +793,7 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
     constexpr int GPS = kBK / GROUP;
     constexpr int W_BYTES = 16 * BN * 4;
     constexpr int SZ_ROW = BN * 2;
+    constexpr bool kActZero = !SPARSE;                      // who requests the zero-points: see the producer
     constexpr int LDC = 8 * MO;
     extern __shared__ __align__(128) uint8_t smem[];
 
@@ -816,10 +817,10 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
     FQ_GT(tid == 0, 1);
     // The grid after this one in the stream may start now (it takes SMs as this grid's CTAs leave).
     // Every warp but the producer waits for the grid before this one to finish: the producer reads
-    // only weights, which no kernel writes while calls are in flight.  (The activation warps of a
-    // kernel with outliers first request the outlier arrays of their first units, see there.)
+    // only weights, which no kernel writes while calls are in flight.  (The activation warps first
+    // request the other weight arrays of their first units, see there.)
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (warp != 0 && !(SPARSE && warp < DW0)) asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (warp >= DW0) asm volatile("griddepcontrol.wait;" ::: "memory");
 
     const uint32_t KT = p.KT;
     const uint32_t U = p.NT * KT, P = gridDim.x, q = U / P, r = U % P;
@@ -836,10 +837,11 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer
-        // Weights, scales and zero-points of every unit.  (The unit's outlier arrays are requested by
-        // its activation warp: a bulk copy costs its issuing warp a few hundred cycles next to the
-        // dense warps' shared-memory traffic, and five of them per unit made this warp the
-        // bottleneck of the small-batch kernels.)
+        // Packed weights and scales of every unit; its zero-points too in a kernel with outliers, where
+        // the unit's activation warp requests the outlier arrays (without outliers it requests the
+        // zero-points).  A bulk copy costs its issuing warp a few hundred cycles next to the dense
+        // warps' shared-memory traffic: five of them per unit made this warp the bottleneck of the
+        // kernels with one octet of rows, and this split measured best.
         uint32_t issued = 0;
         bool ok = true;
         for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
@@ -851,17 +853,16 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
 #ifdef FQ_TRACE
             if (blockIdx.x == 0 && lane == 0) { g_trace[8] += clock64() - tw0; g_trace[9] += 1; }
 #endif
-            const uint32_t tn = w.tn, kt = w.kt;
             const uint32_t full = bar_full + 8 * s;
             const uint32_t st = smem_u32(smem) + s * p.stage_bytes;
             if (lane == 0) {
-                mbar_arrive_expect_tx(full, W_BYTES + 2 * GPS * SZ_ROW);
+                mbar_arrive_expect_tx(full, W_BYTES + (kActZero ? 1 : 2) * GPS * SZ_ROW);
                 bulk_g2s(st, p.wq + (size_t)u * W_BYTES, W_BYTES, full);
 #pragma unroll
                 for (int gi = 0; gi < GPS; ++gi) {
-                    const size_t row = (size_t)(kt * GPS + gi) * p.N + (size_t)tn * BN;
+                    const size_t row = (size_t)(w.kt * GPS + gi) * p.N + (size_t)w.tn * BN;
                     bulk_g2s(st + p.off_sz + gi * SZ_ROW, p.scale + row, SZ_ROW, full);
-                    bulk_g2s(st + p.off_sz + (GPS + gi) * SZ_ROW, p.zero + row, SZ_ROW, full);
+                    if (!kActZero) bulk_g2s(st + p.off_sz + (GPS + gi) * SZ_ROW, p.zero + row, SZ_ROW, full);
                 }
             }
             issued = it + 1;
@@ -894,16 +895,30 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
         auto load_ip = [&](uint32_t u) {
             if (SPARSE && lane == 0) { ip_nxt = __ldg(p.indptr + u); ip_nxt_end = __ldg(p.indptr + u + 1); }
         };
-        if (SPARSE) {
-            // The first pass over the ring finds every stage empty, and the outlier arrays are weights:
+        // this warp's share of the weight arrays of unit u (k-step kt of column tile tn): bucket
+        // descriptors and packets, or the zero-points; into the stage at shared-memory address sta,
+        // counted on its barrier before this warp's arrival
+        auto request = [&](uint32_t u, uint32_t tn, uint32_t kt, uint32_t sta, uint32_t full, uint32_t ip, uint32_t npk) {
+            mbar_expect_tx(full, kActZero ? GPS * SZ_ROW : p.NB * 4 + npk * 16);
+            if (kActZero) {
+#pragma unroll
+                for (int gi = 0; gi < GPS; ++gi)
+                    bulk_g2s(sta + p.off_sz + (GPS + gi) * SZ_ROW, p.zero + (size_t)(kt * GPS + gi) * p.N + (size_t)tn * BN, SZ_ROW, full);
+            }
+            if (SPARSE) {
+                bulk_g2s(sta + p.off_info, p.info + (size_t)u * p.NB, p.NB * 4, full);
+                if (npk) bulk_g2s(sta + p.off_coo, p.packed + ip, npk * 16, full);
+            }
+        };
+        {
+            // The first pass over the ring finds every stage empty, and these arrays are weights:
             // lane l requests those of this warp's l-th unit before the wait for the previous grid.
             const uint32_t it0 = aw + NA * lane;
             if (it0 < min(S, u_end - u_begin)) {
-                const uint32_t u = u_begin + it0, a = __ldg(p.indptr + u), npk = min(__ldg(p.indptr + u + 1) - a, p.coo_cap);
-                const uint32_t full = bar_full + 8 * it0, sta = smem_u32(smem) + it0 * p.stage_bytes;
-                mbar_expect_tx(full, p.NB * 4 + npk * 16);
-                bulk_g2s(sta + p.off_info, p.info + (size_t)u * p.NB, p.NB * 4, full);
-                if (npk) bulk_g2s(sta + p.off_coo, p.packed + a, npk * 16, full);
+                const uint32_t u = u_begin + it0, tn = u / KT;
+                uint32_t a = 0, npk = 0;
+                if (SPARSE) { a = __ldg(p.indptr + u); npk = min(__ldg(p.indptr + u + 1) - a, p.coo_cap); }
+                request(u, tn, u - tn * KT, smem_u32(smem) + it0 * p.stage_bytes, bar_full + 8 * it0, a, npk);
             }
             __syncwarp();
             asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -926,14 +941,7 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
             long long tw1 = clock64();
 #endif
             last_bar = bar_full + 8 * s, last_ph = ph;
-            if (SPARSE && lane == 0 && w.it >= S) {
-                // bucket descriptors and packets of the unit, counted on the stage's barrier before
-                // this warp's own arrival
-                const uint32_t full = bar_full + 8 * s, sta = smem_u32(st);
-                mbar_expect_tx(full, p.NB * 4 + npk * 16);
-                bulk_g2s(sta + p.off_info, p.info + (size_t)w.u * p.NB, p.NB * 4, full);
-                if (npk) bulk_g2s(sta + p.off_coo, p.packed + ip, npk * 16, full);
-            }
+            if (lane == 0 && w.it >= S) request(w.u, w.tn, w.kt, smem_u32(st), bar_full + 8 * s, ip, npk);
             uint8_t* dst = st + p.off_xcan + m * kXPitch + part * CPL * 16;
             float sum = 0.0f;
 #pragma unroll
@@ -969,7 +977,7 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
             if (blockIdx.x == 0 && lane == 0 && aw == 0) { g_trace[10] += tw1 - tw0; g_trace[11] += clock64() - tw1; g_trace[12] += 1; }
 #endif
         }
-        if (SPARSE && !ok && last_bar)      // gave up: let this warp's last copies land before the CTA exits
+        if (!ok && last_bar)                // gave up: let this warp's last copies land before the CTA exits
             for (uint32_t spin = 0; spin < (1u << 20) && !mbar_try_wait(last_bar, last_ph); ++spin) {}
     } else if (warp >= DW0 && warp < DW0 + NGRP * NDW) {
         // ------------------------------------------------------------------ dense warps (all alike)

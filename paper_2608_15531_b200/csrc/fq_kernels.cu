@@ -316,11 +316,14 @@ __device__ __forceinline__ void apply_packet(const uint4 pk, const float* __rest
 // Transpose one octet of BF16 activation rows into the FP32 k-major copy xt[k][8] (32 B per k).
 // `row0` is the shared-memory address of row 0 / 16-byte chunk 0 of the octet, rows `row_step`
 // bytes apart, consecutive 16-byte chunks (8 k each) `chunk_step` bytes apart.  Whole warp.
+// SWZ: odd rows keep chunk c at position c ^ 4.
+template <bool SWZ = false>
 __device__ __forceinline__ void transpose_octet_f32(uint32_t row0, uint32_t row_step, uint32_t chunk_step, float* xt, int lane) {
 #pragma unroll
     for (int kb = 0; kb < 4; ++kb) {
         uint32_t r[4];
-        ldmatrix_x4_trans(row0 + (lane & 7) * row_step + (kb * 4 + (lane >> 3)) * chunk_step, r[0], r[1], r[2], r[3]);
+        const uint32_t chunk = (kb * 4 + (lane >> 3)) ^ (SWZ ? ((uint32_t)lane & 1u) << 2 : 0u);
+        ldmatrix_x4_trans(row0 + (lane & 7) * row_step + chunk * chunk_step, r[0], r[1], r[2], r[3]);
         // thread T holds rows m = 2(T%4), 2(T%4)+1 of column k = 8*block + T/4
         float* dst = xt + ((kb * 32) + (lane >> 2)) * 8 + (lane & 3) * 2;
 #pragma unroll
@@ -763,7 +766,10 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1
 }
 
 constexpr int kActWarps = 2;   // activation warps of the small-batch kernel
-constexpr int kXPitch = 320;   // activation row in shared memory: 256 B + 64 B, conflict-free 16-byte fragment loads
+// Activation row in shared memory: 256 B, its sixteen 16-byte chunks stored at chunk ^ 4 in odd rows.
+// The fragment loads of a quarter warp (rows g and g + 1, four consecutive chunks each) then touch
+// all 32 banks once.
+constexpr int kXPitch = 256;
 
 // The same operator for M <= 8 per octet (MO octets of batch rows): every dense warp runs the same
 // short loop (one 32-column strip per warp, warp-level m16n8k16 MMAs with the weights on the M side
@@ -942,12 +948,13 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
 #endif
             last_bar = bar_full + 8 * s, last_ph = ph;
             if (lane == 0 && w.it >= S) request(w.u, w.tn, w.kt, smem_u32(st), bar_full + 8 * s, ip, npk);
-            uint8_t* dst = st + p.off_xcan + m * kXPitch + part * CPL * 16;
+            uint8_t* dst = st + p.off_xcan + m * kXPitch;
+            const int swz = (m & 1) << 2;
             float sum = 0.0f;
 #pragma unroll
             for (int c = 0; c < CPL; ++c) {
                 const uint4 v = xv[c];
-                *reinterpret_cast<uint4*>(dst + c * 16) = v;
+                *reinterpret_cast<uint4*>(dst + ((part * CPL + c) ^ swz) * 16) = v;
                 sum += (bf16lo(v.x) + bf16hi(v.x)) + (bf16lo(v.y) + bf16hi(v.y)) + (bf16lo(v.z) + bf16hi(v.z)) +
                        (bf16lo(v.w) + bf16hi(v.w));
             }
@@ -964,11 +971,22 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                 else if (part == 0) xsum[m] = s1;
             }
             __syncwarp();
-            if (SPARSE) {
+            if (SPARSE && MS == 1) {
+                // FP32 copy of the single batch row for the outlier step: xt[k]
+                if (m == 0) {
+                    float4* xt4 = reinterpret_cast<float4*>(st + p.off_xt) + part * CPL * 2;
+#pragma unroll
+                    for (int c = 0; c < CPL; ++c) {
+                        xt4[2 * c] = make_float4(bf16lo(xv[c].x), bf16hi(xv[c].x), bf16lo(xv[c].y), bf16hi(xv[c].y));
+                        xt4[2 * c + 1] = make_float4(bf16lo(xv[c].z), bf16hi(xv[c].z), bf16lo(xv[c].w), bf16hi(xv[c].w));
+                    }
+                }
+                __syncwarp();
+            } else if (SPARSE) {
                 // FP32 k-major copy [octet][k][8] for the outlier step
 #pragma unroll
                 for (int o = 0; o < MO; ++o)
-                    transpose_octet_f32(smem_u32(st + p.off_xcan) + o * 8 * kXPitch, kXPitch, 16,
+                    transpose_octet_f32<true>(smem_u32(st + p.off_xcan) + o * 8 * kXPitch, kXPitch, 16,
                                         reinterpret_cast<float*>(st + p.off_xt) + o * 1024, lane);
                 __syncwarp();
             }
@@ -1021,7 +1039,11 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
 #endif
             FQ_GT(dtid == 0 && u == u_begin, 2);
             const uint4* wp = reinterpret_cast<const uint4*>(st) + dw * 32 + lane;   // the lane's four columns, 8 rows
+            // chunk 4j + t of row g (+ 8 per octet): at (4j + t) ^ 4 in odd rows, i.e. 64 B further for
+            // even j and 64 B back for odd j
             const uint8_t* xrow = st + p.off_xcan + g * kXPitch + t * 16;
+            const uint8_t* xrow_e = xrow + ((g & 1) << 6);
+            const uint8_t* xrow_o = xrow - ((g & 1) << 6);
             const uint16_t* sc = reinterpret_cast<const uint16_t*>(st + p.off_sz);
             const float* xsum = reinterpret_cast<const float*>(st + p.off_xsum);
             // outliers: the bucket descriptor and the first two packets are requested now and used
@@ -1087,7 +1109,7 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                 for (int j = gi * (4 / GPS); j < (gi + 1) * (4 / GPS); ++j) {
                     uint4 xb[MO];
 #pragma unroll
-                    for (int o = 0; o < MO; ++o) xb[o] = *reinterpret_cast<const uint4*>(xrow + o * 8 * kXPitch + j * 64);
+                    for (int o = 0; o < MO; ++o) xb[o] = *reinterpret_cast<const uint4*>(((j & 1) ? xrow_o : xrow_e) + o * 8 * kXPitch + j * 64);
                     const uint4 w4 = wp[j * BN];                    // columns +0, +8, +16, +24
 #pragma unroll
                     for (int cg = 0; cg < CG; ++cg) {
@@ -1127,7 +1149,7 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                 if constexpr (MS == 1) {
                     // single batch row: lane t keeps the slots of column number t of the bucket
                     auto apply = [&](const uint32_t w) {
-                        sacc[0][0] = fmaf(__uint_as_float(w & 0xffff0000u), *reinterpret_cast<const float*>(xtb + (w & 0xfe0u)), sacc[0][0]);
+                        sacc[0][0] = fmaf(__uint_as_float(w & 0xffff0000u), *reinterpret_cast<const float*>(xtb + ((w >> 3) & 0x1fcu)), sacc[0][0]);
                     };
                     if (cmax > 0) apply(pk0);
                     if (cmax > 1) {
@@ -1148,7 +1170,7 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
 #pragma unroll
                                 for (int e = 0; e < 4; ++e) {
                                     const float v = ((w[e] >> 12) & 3u) == (uint32_t)t ? __uint_as_float(w[e] & 0xffff0000u) : 0.0f;
-                                    hacc = fmaf(v, *reinterpret_cast<const float*>(xtb + (w[e] & 0xfe0u)), hacc);
+                                    hacc = fmaf(v, *reinterpret_cast<const float*>(xtb + ((w[e] >> 3) & 0x1fcu)), hacc);
                                 }
                             }
                             hacc += __shfl_xor_sync(0xffffffffu, hacc, 4);
@@ -1408,14 +1430,26 @@ __global__ void __launch_bounds__(256) fq_spmm_kernel(const uint16_t* __restrict
             const uint32_t inf = __ldg(info + t * NB + b);
             const uint4* pk = packed + __ldg(indptr + t) + (inf & 0xffffu);
             const uint32_t depth = (inf >> 16) & 0xffu, tail = inf >> 24;
-            for (uint32_t i = 0; i < depth + tail; ++i) {
+            for (uint32_t i = 0; i < depth; ++i) {              // column-slotted: slot e is column number e
                 const uint4 q = __ldg(pk + i);
                 const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    const uint32_t k = kt * kBK + ((w[e] >> 5) & 127u), cls = (w[e] >> 12) & 3u;
                     const float v = __uint_as_float(w[e] & 0xffff0000u);
-                    const uint16_t* xp = X + (size_t)m0 * K + k;
+                    const uint16_t* xp = X + (size_t)m0 * K + kt * kBK + ((w[e] >> 5) & 127u);
+#pragma unroll
+                    for (int m = 0; m < MB; ++m)
+                        acc[e][m] = fmaf(v, (m0 + m < M) ? bf16_bits_to_float(__ldg(xp + (size_t)m * K)) : 0.0f, acc[e][m]);
+                }
+            }
+            for (uint32_t i = depth; i < depth + tail; ++i) {   // tail: a slot names its column
+                const uint4 q = __ldg(pk + i);
+                const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const uint32_t cls = (w[e] >> 12) & 3u;
+                    const float v = __uint_as_float(w[e] & 0xffff0000u);
+                    const uint16_t* xp = X + (size_t)m0 * K + kt * kBK + ((w[e] >> 5) & 127u);
 #pragma unroll
                     for (int m = 0; m < MB; ++m) {
                         const float x = (m0 + m < M) ? bf16_bits_to_float(__ldg(xp + (size_t)m * K)) : 0.0f;
@@ -1520,7 +1554,7 @@ static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, 
     std::memset(&p, 0, sizeof(p));
     p.M = M; p.K = L->K; p.N = L->N; p.KT = L->K / kBK; p.NT = L->N / BN; p.NB = NB; p.nsw = 0;
     const uint32_t w_bytes = 16 * BN * 4, sz_bytes = 2 * GPS * BN * 2;
-    const uint32_t xt_bytes = sparse ? MO * 4096 : 0;     // FP32 [octet][k][8]
+    const uint32_t xt_bytes = sparse ? (M == 1 ? 512 : MO * 4096) : 0;     // FP32 [k] for one batch row, else [octet][k][8]
     // Two groups of dense warps (each takes every other unit) pay off when a CTA has enough units to
     // stream and the accumulators are small; short jobs and 16-row batches keep one group.
     const int sms = sm_count_cached();

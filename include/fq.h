@@ -60,9 +60,10 @@
  *   bits 16-31 the BF16 value, bits 5-11 the row inside the tile (so that
  *   slot & 0xfe0 is the row times 32), bits 12-13 the column number j, all
  *   other bits 0.  A padding slot has value bits 0x0000 and row 0.
- *     The first `depth` packets of a bucket are column-slotted (Section 4.2's
- *   per-column padding): slot j of packet i is the i-th outlier, by row, of
- *   column number j, or a padding slot that still names j.  If no column of
+ *     The first `depth` packets of a bucket are column-slotted (padding per
+ *   column as in Section 4.2, with the column given by the slot's position
+ *   instead of a column index per packet): slot j of packet i is the i-th
+ *   outlier, by row, of column number j, or a padding slot that still names j.  If no column of
  *   the bucket has more than 16 outliers in the tile, depth is the longest
  *   column's count and tail is 0.  Otherwise depth is 4, and the outliers
  *   beyond the first 4 of each column follow in `tail` packets by (row,

@@ -1435,6 +1435,7 @@ __global__ void __launch_bounds__(256) fq_spmm_kernel(const uint16_t* __restrict
                 const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
+                    if ((w[e] >> 16) == 0) continue;            // padding: no activation loads for it
                     const float v = __uint_as_float(w[e] & 0xffff0000u);
                     const uint16_t* xp = X + (size_t)m0 * K + kt * kBK + ((w[e] >> 5) & 127u);
 #pragma unroll

@@ -124,6 +124,33 @@ def test_oversized_tiles_fall_back_to_global_packets():
         H.check_tolerances(Y, Yref, Yabs, K)
 
 
+def test_several_tails_in_one_strip():
+    # Column-slotted packets with tails: in the first 32-column strip of one tile, column 3 has 100
+    # outliers, column 12 has 40 and column 27 (same bucket as column 3) has 17; column 5 has exactly
+    # 16 (the longest column-slotted list).  A second tile has one long column on top of 1 % noise.
+    # Everything fits the staged part, so the tails are read from shared memory.
+    K, N, g, BN = 512, 512, 128, 256
+    lay = synth.layer(synth.tensor_seed(8, 9), K, N, density=0.01, layout="uniform")
+    mask = lay.mask.copy()
+    rng = np.random.default_rng(4)
+    for col, cnt in ((3, 100), (12, 40), (27, 17), (5, 16)):
+        mask[0:128, col] = 0
+        mask[rng.choice(128, size=cnt, replace=False), col] = 1
+    mask[256 + rng.choice(128, size=77, replace=False), 256 + 130] = 1
+    kk, nn = np.nonzero(mask)
+    vals = (rng.uniform(0.12, 0.4, size=kk.size) * rng.choice([-1, 1], size=kk.size)).astype(np.float32)
+    vb = (vals.view(np.uint32) >> 16).astype(np.uint16)
+    lay.mask, lay.coo_k, lay.coo_n, lay.coo_v = mask, kk.astype(np.uint32), nn.astype(np.uint32), vb
+    lay.W[kk, nn] = synth.bf16_bits_to_f32(vb)
+    P = H.pack_layer(lay, g, BN)
+    assert P.L.max_tail_packets == (100 - 4 + 17 - 4 + 3) // 4 and P.L.max_tile_packets < 1024
+    for M in (1, 5, 8, 16):
+        X = _x(7, M, K)
+        Y = H.run_fused(P, X)
+        Yref, Yabs = H.oracle_result(P, X)
+        H.check_tolerances(Y, Yref, Yabs, K)
+
+
 def test_scratch_is_reusable_and_results_are_reproducible():
     K, N, g = 2048, 1024, 128
     lay = synth.layer(synth.tensor_seed(8, 4), K, N, density=0.01, layout="mixed")

@@ -3,15 +3,16 @@
 //
 // Two kernels compute the fused operator.  Both are persistent (one CTA per SM) and warp-specialised,
 // work on (tile, k-step) units of 128 rows x BN columns, stream them through the same ring of
-// shared-memory stages (cp.async.bulk + mbarrier expect_tx, one producer warp), feed the tensor cores
+// shared-memory stages (cp.async.bulk + mbarrier expect_tx), feed the tensor cores
 // the exact integers 128 + q as BF16 and apply scale and zero-point once per group in FP32:
 //     acc[m] += s * (sum_k x (128+q) - (128+z) sum_k x)                 (Eq. 3 inside Eq. 1)
 //
 //   fq_mma_kernel    the default (16 batch rows per launch).  Dense warps own 32-column strips: lop3
 //                    unpack in registers, mma.sync m16n8k16 with the weights on the M side, and the
 //                    unit's outliers added straight into the MMA accumulators (a Tile-COO bucket is
-//                    the four columns a group of four lanes holds).  Activation warps lay out X and
-//                    its row sums per unit.  Described in detail above the kernel.
+//                    the four columns a group of four lanes holds, and slot j of a packet belongs
+//                    to the j-th of them).  Activation warps lay out X and its row sums per unit and
+//                    issue part of the unit's bulk copies.  Described in detail above the kernel.
 //   fq_fused_kernel  the tcgen05 kernel (FQ_ENGINE=tc; 32 batch rows per launch):
 //     warp 0        producer
 //     warp 1 (+3)   tensor: own the TMEM allocation and issue tcgen05.mma (A = dequantised weights
@@ -776,17 +777,20 @@ constexpr int kXPitch = 256;
 // and the batch on the N side), so the instruction stream of the CTA's dense warps is shared and
 // stays in the instruction cache.  Same packed formats, same producer, same split-tile protocol as
 // the tcgen05 kernel; the dense engine differs, and the outliers need no warps of their own:
-//   warp 0            producer (bulk copies)
-//   warp 1            activations: X block -> row-major shared-memory rows + per-group row sums
-//                     + an FP32 k-major copy for the outlier step
-//   warps 2..2+BN/32  dense + outliers.  Lane (g, t) of warp w holds the accumulators of columns
+//   warp 0            producer: bulk copies of the packed weights and the scales (and the
+//                     zero-points in kernels with outliers)
+//   warps 1..2        activations (alternate units): X block -> row-major shared-memory rows +
+//                     per-group row sums + an FP32 k-major copy for the outlier step; bulk copies of
+//                     the unit's bucket descriptors and packets (or of its zero-points)
+//   then NGRP x BN/32 dense + outliers.  Lane (g, t) of warp w holds the accumulators of columns
 //                     32w + {g, g+8, g+16, g+24}, batch rows 2t, 2t+1 (+8 per octet).  Dense: the
-//                     lane loads word t of its columns of each 32-row block: 8 codes = its share
-//                     of two k16 steps (the k order inside a block follows the 16-byte activation
-//                     loads of the lanes).  Outliers: those four columns are one Tile-COO bucket, so
-//                     the four lanes of group g walk that bucket's packets and add v * x[row][k]
-//                     straight into their accumulators (Section 4.2 without the shared-memory
-//                     scatter: no atomics, no read-modify-write, no merge step).
+//                     lane loads, as one 16-byte word group, word t of its four columns of each
+//                     32-row block: 8 codes per column = its share of two k16 steps (the k order
+//                     inside a block follows the 16-byte activation loads of the lanes).  Outliers:
+//                     those four columns are one Tile-COO bucket, so the four lanes of group g walk
+//                     that bucket's packets and add v * x[row][k] straight into their accumulators,
+//                     slot j into column number j (Section 4.2 without the shared-memory scatter:
+//                     no atomics, no read-modify-write, no merge step).
 template <int BN, int MO, int GROUP, bool SPARSE, int MS, int NGRP, bool HOT>
 __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq_mma_kernel(const Params p) {
     constexpr int NDW = BN / 32;

@@ -106,10 +106,12 @@ typedef struct fq_layout {
     uint32_t buckets_per_tile; /* NB = BN / 4 */
     uint32_t wq_interleave;    /* 3: the word order described above */
     uint32_t coo_unit_bytes;   /* 16 */
-    uint32_t max_tile_packets; /* largest tile of the encoded W_O, in packets; 0 = not encoded */
+    uint32_t max_tile_packets; /* largest tile of the encoded W_O, in packets */
     uint32_t max_bucket_packets; /* longest packet list (depth + tail) of one bucket in one tile */
     uint32_t max_tail_packets; /* longest tail; 0 = every packet is column-slotted */
-    uint32_t reserved[4];
+    uint32_t tilecoo_encoded;  /* 1 = the three maxima above describe the arrays in use (set by
+                                  fq_encode_tilecoo); 0 = unknown: the kernels assume the worst */
+    uint32_t reserved[3];
 } fq_layout_t;
 
 /* Choose tile sizes for a K x N layer.  bn_hint: 0 = library default (256 when

@@ -336,6 +336,7 @@ fq_status_t fq_encode_tilecoo(fq_layout_t* L, const uint32_t* k, const uint32_t*
     L->max_tile_packets = E.max_tile_packets;
     L->max_bucket_packets = E.max_bucket_packets;
     L->max_tail_packets = E.max_tail_packets;
+    L->tilecoo_encoded = 1;
     return FQ_OK;
 }
 

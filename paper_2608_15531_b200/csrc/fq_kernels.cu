@@ -1522,7 +1522,7 @@ static fq_status_t make_plan(const fq_layout_t* L, uint32_t M, bool sparse, Plan
     const uint32_t fixed = (sparse ? BN * NMMA * 4 : 0) + 1024;
     uint32_t cap = 0;
     if (sparse) {
-        cap = L->max_tile_packets ? round_up(L->max_tile_packets, 8) : 256;
+        cap = L->tilecoo_encoded ? std::max<uint32_t>(8, round_up(L->max_tile_packets, 8)) : 256;
         cap = std::min<uint32_t>(cap, 1024);
     }
     uint32_t stage = 0, S = 0;
@@ -1585,7 +1585,7 @@ static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, 
     const uint32_t budget = kSmemBudget;
     uint32_t cap = 0;
     if (sparse) {
-        cap = L->max_tile_packets ? round_up(L->max_tile_packets, 8) : 256;
+        cap = L->tilecoo_encoded ? std::max<uint32_t>(8, round_up(L->max_tile_packets, 8)) : 256;
         cap = std::min<uint32_t>(cap, 1024);
     }
     uint32_t stage = 0, S = 0;
@@ -1607,7 +1607,7 @@ static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, 
     if (S < 4) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "shared-memory stages do not fit");
     p.coo_cap = cap; p.stages = S; p.stage_bytes = stage;
     // hot columns, tiles larger than the staged part, or an encoding whose sizes were not recorded
-    pl.general = sparse && (L->max_tail_packets > 0 || L->max_tile_packets > cap || L->max_tile_packets == 0);
+    pl.general = sparse && (L->max_tail_packets > 0 || L->max_tile_packets > cap || !L->tilecoo_encoded);
     p.off_shc = S * stage;
     p.off_bar = p.off_shc + xch_bytes;
     pl.smem = p.off_bar + 1024;
@@ -1712,7 +1712,7 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
     if (M < 1 || M > FQ_MAX_M) return fail(FQ_ERR_INVALID_ARG, "M = %u outside [1, %u]", M, FQ_MAX_M);
     if (!X || !wq || !scale || !zero || !Y || !workspace) return fail(FQ_ERR_INVALID_ARG, "null device pointer");
     if (sparse && (!indptr || !info)) return fail(FQ_ERR_INVALID_ARG, "null Tile-COO pointer");
-    if (sparse && !packed && L->max_tile_packets) return fail(FQ_ERR_INVALID_ARG, "null packet pointer");
+    if (sparse && !packed && (L->max_tile_packets || !L->tilecoo_encoded)) return fail(FQ_ERR_INVALID_ARG, "null packet pointer");
     if (!aligned(X, 16) || !aligned(Y, 16) || !aligned(wq, 128) || !aligned(scale, 128) || !aligned(zero, 128) ||
         !aligned(workspace, 128) || (sparse && (!aligned(indptr, 4) || !aligned(info, 128) || !aligned(packed, 128))))
         return fail(FQ_ERR_INVALID_ARG, "misaligned device pointer");
@@ -1862,7 +1862,7 @@ fq_status_t fq_unfused_spmm(const fq_layout_t* L, const void* X, uint32_t M, con
     if (!layout_ok(L)) return fail(FQ_ERR_INVALID_ARG, "bad layout");
     if (M < 1 || M > FQ_MAX_M) return fail(FQ_ERR_INVALID_ARG, "M = %u outside [1, %u]", M, FQ_MAX_M);
     if (!X || !tile_indptr || !bucket_info || !Y) return fail(FQ_ERR_INVALID_ARG, "null device pointer");
-    if (!packed_outliers && L->max_tile_packets) return fail(FQ_ERR_INVALID_ARG, "null packet pointer");
+    if (!packed_outliers && (L->max_tile_packets || !L->tilecoo_encoded)) return fail(FQ_ERR_INVALID_ARG, "null packet pointer");
     const uint32_t buckets = (L->N / L->BN) * L->buckets_per_tile;   // one warp each
     fq_spmm_kernel<<<(buckets + 7) / 8, 256, 0, (cudaStream_t)cuda_stream>>>(
         (const uint16_t*)X, (const uint32_t*)tile_indptr, (const uint32_t*)bucket_info, (const uint4*)packed_outliers,

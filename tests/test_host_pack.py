@@ -113,6 +113,7 @@ def test_tilecoo_encode_invariants(layout, density, BN):
     assert n_ip == ntile + 1 == indptr.size and n_bi == ntile * NB == info.size and n_pk == packed.shape[0]
     assert L.max_tile_packets == mx == int(np.diff(indptr).max())
     assert L.max_bucket_packets == int((depth + tail).max()) and L.max_tail_packets == int(tail.max())
+    assert L.tilecoo_encoded == 1
     assert indptr[0] == 0 and np.all(np.diff(indptr.astype(np.int64)) >= 0) and indptr[-1] == n_pk
     assert 4 * Lr.nnz <= 16 * n_pk <= 16 * Lr.nnz          # every packet carries at least one outlier
     # decoded set == input set, by the oracle's reader and by the library's
@@ -187,8 +188,9 @@ def test_tilecoo_edge_cases():
     L = fq.fq_get_layout(K, N, 128, bn_hint=BN)
     e32, e16 = np.zeros(0, dtype=np.uint32), np.zeros(0, dtype=np.uint16)
     # no outliers at all
+    assert L.tilecoo_encoded == 0
     indptr, info, packed = fq.fq_encode_tilecoo(L, e32, e32, e16)
-    assert packed.shape[0] == 0 and not indptr.any() and not info.any() and L.max_tile_packets == 0
+    assert packed.shape[0] == 0 and not indptr.any() and not info.any() and L.max_tile_packets == 0 and L.tilecoo_encoded == 1
     fq.fq_validate_tilecoo(L, indptr, info, packed)
     # a single outlier; zero-valued entries are dropped
     k = np.array([200, 5, 6], dtype=np.uint32)

@@ -1353,11 +1353,13 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                             for (int cg = 0; cg < CG; ++cg)
 #pragma unroll
                                 for (int i = 0; i < 4; ++i) accf[o][cg][i] = 0.0f;
-                        // four contributors' loads in flight at a time; the additions keep CTA order
-                        for (uint32_t c = c_first; c <= c_last; c += 4) {
-                            float v[4][MO * CG * 4];
+                        // ND contributors' loads in flight at a time (more where the registers allow it:
+                        // the short jobs, whose time is mostly such round trips); the additions keep CTA order
+                        constexpr int ND = (MO == 1 && NGRP == 1) ? 8 : 4;
+                        for (uint32_t c = c_first; c <= c_last; c += ND) {
+                            float v[ND][MO * CG * 4];
 #pragma unroll
-                            for (int d = 0; d < 4; ++d) {
+                            for (int d = 0; d < ND; ++d) {
                                 const uint32_t cc = min(c + d, c_last);
                                 const uint32_t wch = (p.split || unit_begin_of(cc, q, r) / KT == tn) ? 0u : 1u;
                                 const float* sl = p.partials + ((size_t)cc * 2 + wch) * (size_t)(BN * LDC) + dw * (32 * LDC) + lane;
@@ -1365,7 +1367,7 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                                 for (int e = 0; e < MO * CG * 4; ++e) v[d][e] = __ldcg(sl + e * 32);
                             }
 #pragma unroll
-                            for (int d = 0; d < 4; ++d)
+                            for (int d = 0; d < ND; ++d)
                                 if (c + d <= c_last) {
 #pragma unroll
                                     for (int o = 0; o < MO; ++o)

@@ -471,8 +471,36 @@ def run_sweep(args):
         torch.cuda.empty_cache()
         return out
 
+    def cublas_bf16_us(K, N, M):
+        """torch.matmul on BF16 weights of the same shape (values do not matter for its time)."""
+        W = [torch.randn((K, N), dtype=torch.bfloat16, device=dev) for _ in range(2)]
+        X = torch.randn((M, K), dtype=torch.bfloat16, device=dev)
+        turn = [0]
+
+        def mm():
+            turn[0] += 1
+            torch.matmul(X, W[turn[0] & 1])
+
+        us = time_loop(mm, reps=10)
+        del W
+        torch.cuda.empty_cache()
+        return us
+
     points = []
-    if args.sweep == "density":
+    if args.sweep == "paper":
+        # The paper's ratio and batch sweep on its extreme operator shape, both orientations
+        # (Section 5: outlier ratios 1-3 %, batch 8/16/32); uniform layout, BF16 outliers.
+        for tag, (K, N) in enumerate(((14848, 75264), (75264, 14848))):
+            ref = {M: round(cublas_bf16_us(K, N, M), 2) for M in (8, 16, 32)}
+            for density in (0.01, 0.015, 0.02, 0.025, 0.03):
+                pts = point(6, 10 * tag + int(density * 1000), K, N, GROUP, density, "uniform", (8, 16, 32))
+                for pt in pts:
+                    pt["cublas_bf16_us"] = ref[pt["M"]]
+                    pt["cublas_over_fused"] = round(ref[pt["M"]] / pt["fused_us"], 2)
+                points += pts
+                print(f"[bench] {K}x{N} {density}: " + ", ".join(f"M={q['M']}: {q['fused_us']} us" for q in pts),
+                      file=sys.stderr, flush=True)
+    elif args.sweep == "density":
         for layout in ("uniform", "clustered"):
             for density in (0.0, 0.005, 0.01, 0.02, 0.05):
                 if density == 0.0 and layout == "clustered":
@@ -528,8 +556,9 @@ def main():
     ap.add_argument("--no-cublas", dest="cublas", action="store_false")
     ap.add_argument("--verbose", action="store_true")
     ap.add_argument("--only", default="", help="profiling aid: restrict the step to one LAYER:M, e.g. gate_up:16")
-    ap.add_argument("--sweep", default="", choices=["", "density", "batch"],
-                    help="print the density sweep or the batch transition sweep instead of the benchmark line")
+    ap.add_argument("--sweep", default="", choices=["", "density", "batch", "paper"],
+                    help="print the density sweep, the batch transition sweep or the paper's ratio-and-batch sweep on "
+                         "its largest operator shape (minutes of host time) instead of the benchmark line")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -64,7 +64,7 @@
  *   column as in Section 4.2, with the column given by the slot's position
  *   instead of a column index per packet): slot j of packet i is the i-th
  *   outlier, by row, of column number j, or a padding slot that still names j.  If no column of
- *   the bucket has more than 16 outliers in the tile, depth is the longest
+ *   the bucket has more than 32 outliers in the tile, depth is the longest
  *   column's count and tail is 0.  Otherwise depth is 4, and the outliers
  *   beyond the first 4 of each column follow in `tail` packets by (row,
  *   column), four to a packet in any slot, the last one filled with all-zero

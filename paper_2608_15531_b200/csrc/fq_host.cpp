@@ -204,7 +204,7 @@ inline uint32_t column_of(uint32_t b, uint32_t j) { return ((b >> 3) << 5) | (b 
 inline uint32_t entry_word(uint32_t k, uint32_t j, uint16_t v) { return ((uint32_t)v << 16) | (j << 12) | (k << 5); }
 
 // A column with more entries than this in one tile gives its bucket a tail.
-constexpr uint32_t kSlottedMax = 16;
+constexpr uint32_t kSlottedMax = 32;
 // Column-slotted packets of a bucket that has a tail.
 constexpr uint32_t kSlottedWithTail = 4;
 

@@ -127,13 +127,13 @@ def test_oversized_tiles_fall_back_to_global_packets():
 def test_several_tails_in_one_strip():
     # Column-slotted packets with tails: in the first 32-column strip of one tile, column 3 has 100
     # outliers, column 12 has 40 and column 27 (same bucket as column 3) has 17; column 5 has exactly
-    # 16 (the longest column-slotted list).  A second tile has one long column on top of 1 % noise.
+    # 32 (the longest column-slotted list).  A second tile has one long column on top of 1 % noise.
     # Everything fits the staged part, so the tails are read from shared memory.
     K, N, g, BN = 512, 512, 128, 256
     lay = synth.layer(synth.tensor_seed(8, 9), K, N, density=0.01, layout="uniform")
     mask = lay.mask.copy()
     rng = np.random.default_rng(4)
-    for col, cnt in ((3, 100), (12, 40), (27, 17), (5, 16)):
+    for col, cnt in ((3, 100), (12, 40), (27, 17), (5, 32)):
         mask[0:128, col] = 0
         mask[rng.choice(128, size=cnt, replace=False), col] = 1
     mask[256 + rng.choice(128, size=77, replace=False), 256 + 130] = 1
@@ -307,6 +307,24 @@ def test_batch_transition_sweep_on_sampled_columns(g):
     P = H.pack_layer(lay, g)
     cols = _sample_cols(lay, N, g, n_random=40)
     for M in (1, 2, 4, 8, 16, 32, 64, 128):
+        X = _x(lay.seed, M, K)
+        Y = H.run_fused(P, X)
+        Yref, Yabs = H.oracle_result(P, X, cols=cols)
+        H.check_tolerances(Y[:, cols], Yref, Yabs, K)
+
+
+# ------------------------------------------------------------------ tile counts of the paper's largest operator
+
+@pytest.mark.parametrize("K,N", [(14848, 2304), (75264, 512)])
+def test_tile_counts_that_are_not_powers_of_two_on_sampled_columns(K, N):
+    # 14848 = 116 row tiles and 75264 = 588 row tiles (the two orientations of the largest operator in the
+    # paper's Table of shapes), with few column tiles so that the host side stays small: unit ranges that
+    # start and end anywhere inside a tile, and tiles shared by many CTAs
+    g = 128
+    lay = synth.layer(synth.tensor_seed(6, K % 97), K, N, density=0.02, layout="uniform")
+    P = H.pack_layer(lay, g)
+    cols = _sample_cols(lay, N, 6, n_random=40)
+    for M in (1, 8, 16, 32):
         X = _x(lay.seed, M, K)
         Y = H.run_fused(P, X)
         Yref, Yabs = H.oracle_result(P, X, cols=cols)

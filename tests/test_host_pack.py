@@ -129,11 +129,11 @@ def test_tilecoo_encode_invariants(layout, density, BN):
     tile = (n // BN) * (K // 128) + k // 128
     assert np.array_equal(b // NB, tile)
     # per-column padding (Section 4.2): a bucket has as many column-slotted packets as its longest
-    # column has outliers; only a column with more than 16 turns that into 4 packets and a tail
+    # column has outliers; only a column with more than 32 turns that into 4 packets and a tail
     cnt = _column_counts(Lr.coo_k.astype(np.int64), Lr.coo_n.astype(np.int64), K, N, BN).reshape(ntile * NB, 4)
     longest = cnt.max(axis=1)
-    want_depth = np.where(longest > 16, 4, longest)
-    want_tail = np.where(longest > 16, (np.maximum(cnt - 4, 0).sum(axis=1) + 3) // 4, 0)
+    want_depth = np.where(longest > 32, 4, longest)
+    want_tail = np.where(longest > 32, (np.maximum(cnt - 4, 0).sum(axis=1) + 3) // 4, 0)
     assert np.array_equal(depth, want_depth) and np.array_equal(tail, want_tail)
     if layout == "clustered":
         assert tail.any()
@@ -178,9 +178,9 @@ def test_tilecoo_slots_and_order_inside_a_bucket():
     s2 = pk.view(np.uint32).reshape(-1, 4)
     assert np.array_equal((s2[:4, 1] >> 5) & 127, np.arange(4)) and not (s2[:4, [0, 2, 3]] >> 16).any()
     assert np.array_equal((s2[4:].ravel() >> 5) & 127, np.arange(4, 40)) and np.all((s2[4:].ravel() >> 12) & 3 == 1)
-    # exactly 16 in a column still has no tail
-    ip, bi, pk = fq.fq_encode_tilecoo(L, kk[:16], nn[:16], vv[:16])
-    assert int(bi[_bucket_of(15)]) == 0 | (16 << 16) and L.max_tail_packets == 0
+    # exactly 32 in a column still has no tail
+    ip, bi, pk = fq.fq_encode_tilecoo(L, kk[:32], nn[:32], vv[:32])
+    assert int(bi[_bucket_of(15)]) == 0 | (32 << 16) and L.max_tail_packets == 0
 
 
 def test_tilecoo_edge_cases():
@@ -253,5 +253,5 @@ def test_validator_rejects_corrupted_arrays():
     bad[off0, 1] ^= 1 << 12
     expect_format_error(indptr, info, bad.view(np.uint8).reshape(-1, 16))
     # more column-slotted packets than the format allows
-    bad = info.copy(); bad[0] = (bad[0] & 0xffff) | (17 << 16)
+    bad = info.copy(); bad[0] = (bad[0] & 0xffff) | (33 << 16)
     expect_format_error(indptr, bad, packed)

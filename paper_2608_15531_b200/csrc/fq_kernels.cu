@@ -800,6 +800,9 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
     constexpr int DW0 = 1 + NA;                             // first dense warp
     // NGRP dense warp groups: group r takes the units it with it mod NGRP == r
     constexpr int CG = 2;                                   // 16-column MMA strips per warp
+    // two groups of 16-row warps share the register file: one packet requested ahead instead of two and
+    // its activation rows, two contributors in flight when a split tile is settled
+    constexpr bool kTight = MO == 2 && NGRP == 2;
     constexpr int GPS = kBK / GROUP;
     constexpr int W_BYTES = 16 * BN * 4;
     constexpr int SZ_ROW = BN * 2;
@@ -1097,8 +1100,8 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                 if (HOT && __reduce_max_sync(0xffffffffu, sp_off + sp_cnt + sp_tail) > p.coo_cap)
                     pk_g = p.packed + __ldg(p.indptr + u);           // packets beyond the staged part
                 pk0 = packet(0);
-                pk1 = packet(1);
-                if constexpr (MS == 8) fetch_x(pk0, xa);
+                if constexpr (!kTight) pk1 = packet(1);
+                if constexpr (MS == 8 && !kTight) fetch_x(pk0, xa);
             }
 #pragma unroll
             for (int gi = 0; gi < GPS; ++gi) {
@@ -1198,6 +1201,14 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                             }
                         }
                     };
+                    if constexpr (kTight) {
+                        if (cmax > 0) { fetch_x(pk0, xa); apply(pk0, xa); }
+                        for (uint32_t i = 1; i < cmax; ++i) {
+                            const uint4 pk = packet(i);
+                            fetch_x(pk, xa);
+                            apply(pk, xa);
+                        }
+                    } else {
                     if (cmax > 0) apply(pk0, xa);
                     if (cmax > 1) {
                         float2 xb2[4][MO];
@@ -1208,6 +1219,7 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                             fetch_x(pk, xb2);
                             apply(pk, xb2);
                         }
+                    }
                     }
                     if (HOT) {
                         for (uint32_t hot = __ballot_sync(0xffffffffu, sp_tail != 0); hot; ) {     // warp-uniform
@@ -1355,7 +1367,7 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                                 for (int i = 0; i < 4; ++i) accf[o][cg][i] = 0.0f;
                         // ND contributors' loads in flight at a time (more where the registers allow it:
                         // the short jobs, whose time is mostly such round trips); the additions keep CTA order
-                        constexpr int ND = (MO == 1 && NGRP == 1) ? 8 : 4;
+                        constexpr int ND = (MO == 1 && NGRP == 1) ? 8 : (kTight ? 2 : 4);
                         for (uint32_t c = c_first; c <= c_last; c += ND) {
                             float v[ND][MO * CG * 4];
 #pragma unroll
@@ -1563,7 +1575,8 @@ static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, 
     const uint32_t w_bytes = 16 * BN * 4, sz_bytes = 2 * GPS * BN * 2;
     const uint32_t xt_bytes = sparse ? (M == 1 ? 512 : MO * 4096) : 0;     // FP32 [k] for one batch row, else [octet][k][8]
     // Two groups of dense warps (each takes every other unit) pay off when a CTA has enough units to
-    // stream and the accumulators are small; short jobs and 16-row batches keep one group.
+    // stream; short jobs keep one group.  With two octets of rows the second group fits only because
+    // the outlier step of that variant prefetches less (96 registers per thread).
     const int sms = sm_count_cached();
     if (sms <= 0) return fail(FQ_ERR_CUDA, "no CUDA device: %s", cudaGetErrorString(cudaGetLastError()));
     const uint32_t NT = L->N / BN, KT = L->K / kBK;
@@ -1581,7 +1594,7 @@ static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, 
         }
     }
     p.split = split;
-    pl.ngrp = (MO == 1 && units_per_cta >= 8) ? 2 : 1;
+    pl.ngrp = units_per_cta >= 8 ? 2 : 1;
     const uint32_t xch_bytes = pl.ngrp > 1 ? BN * ROWS * 4 : 0;   // hand-over of a group's partial sums
     const uint32_t fixed = 1024 + xch_bytes;
     const uint32_t budget = kSmemBudget;
@@ -1621,7 +1634,7 @@ static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, 
 typedef void (*KernelFn)(const Params);
 
 // MS: form of the outlier step (1: single batch row, one column per lane; 8: rows split over the lanes);
-// NGRP: groups of dense warps (two only with one octet of rows); HOT: general form of the outlier step
+// NGRP: groups of dense warps; HOT: general form of the outlier step
 // (long bucket lists shared out, packets beyond the staged part of a tile)
 template <int BN, int MO, int G, bool HOT>
 static KernelFn pick_mma_sparse(bool sparse, uint32_t ms, uint32_t ngrp) {
@@ -1632,6 +1645,9 @@ static KernelFn pick_mma_sparse(bool sparse, uint32_t ms, uint32_t ngrp) {
             return (KernelFn)fq_mma_kernel<BN, MO, G, true, 8, 2, HOT>;
         }
         if (sparse && ms == 1) return (KernelFn)fq_mma_kernel<BN, MO, G, true, 1, 1, HOT>;
+    }
+    if constexpr (MO == 2) {
+        if (ngrp == 2) return sparse ? (KernelFn)fq_mma_kernel<BN, MO, G, true, 8, 2, HOT> : (KernelFn)fq_mma_kernel<BN, MO, G, false, 8, 2, false>;
     }
     if (!sparse) return (KernelFn)fq_mma_kernel<BN, MO, G, false, 8, 1, false>;
     return (KernelFn)fq_mma_kernel<BN, MO, G, true, 8, 1, HOT>;

@@ -317,8 +317,9 @@ __device__ __forceinline__ void apply_packet(const uint4 pk, const float* __rest
 // Transpose one octet of BF16 activation rows into the FP32 k-major copy xt[k][8] (32 B per k).
 // `row0` is the shared-memory address of row 0 / 16-byte chunk 0 of the octet, rows `row_step`
 // bytes apart, consecutive 16-byte chunks (8 k each) `chunk_step` bytes apart.  Whole warp.
-// SWZ: odd rows keep chunk c at position c ^ 4.
-template <bool SWZ = false>
+// SWZ: odd rows keep chunk c at position c ^ 4.  PAIRS < 4: only the first PAIRS pairs of rows are
+// kept, 2 * PAIRS floats per k.
+template <bool SWZ = false, int PAIRS = 4>
 __device__ __forceinline__ void transpose_octet_f32(uint32_t row0, uint32_t row_step, uint32_t chunk_step, float* xt, int lane) {
 #pragma unroll
     for (int kb = 0; kb < 4; ++kb) {
@@ -326,9 +327,11 @@ __device__ __forceinline__ void transpose_octet_f32(uint32_t row0, uint32_t row_
         const uint32_t chunk = (kb * 4 + (lane >> 3)) ^ (SWZ ? ((uint32_t)lane & 1u) << 2 : 0u);
         ldmatrix_x4_trans(row0 + (lane & 7) * row_step + chunk * chunk_step, r[0], r[1], r[2], r[3]);
         // thread T holds rows m = 2(T%4), 2(T%4)+1 of column k = 8*block + T/4
-        float* dst = xt + ((kb * 32) + (lane >> 2)) * 8 + (lane & 3) * 2;
+        float* dst = xt + ((kb * 32) + (lane >> 2)) * (2 * PAIRS) + (lane & 3) * 2;
+        if (PAIRS == 4 || (lane & 3) < PAIRS) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) *reinterpret_cast<float2*>(dst + i * 64) = make_float2(bf16lo(r[i]), bf16hi(r[i]));
+            for (int i = 0; i < 4; ++i) *reinterpret_cast<float2*>(dst + i * 16 * PAIRS) = make_float2(bf16lo(r[i]), bf16hi(r[i]));
+        }
     }
 }
 
@@ -989,6 +992,10 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                     }
                 }
                 __syncwarp();
+            } else if (SPARSE && MS == 4) {
+                // FP32 k-major copy of the first four batch rows for the outlier step: xt[k][4]
+                transpose_octet_f32<true, 2>(smem_u32(st + p.off_xcan), kXPitch, 16, reinterpret_cast<float*>(st + p.off_xt), lane);
+                __syncwarp();
             } else if (SPARSE) {
                 // FP32 k-major copy [octet][k][8] for the outlier step
 #pragma unroll
@@ -1020,10 +1027,14 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
             for (int cg = 0; cg < CG; ++cg)
 #pragma unroll
                 for (int i = 0; i < 4; ++i) accf[o][cg][i] = 0.0f;
-        // Outlier accumulator of the single-row form (MS == 1): there lane (g, t) owns ONE column,
-        // 32 dw + 8 t + g (the bucket's column number t); the sums are moved into the MMA fragment
-        // layout above (four columns x two rows per lane) once per piece.
-        float sacc[1][1] = {{0.0f}};
+        // Outlier sums of the column-per-lane forms (MS == 1: one batch row, MS == 4: up to four): there
+        // lane (g, t) owns ONE column, 32 dw + 8 t + g (the bucket's column number t), and takes slot t
+        // of every packet; the sums are moved into the MMA fragment layout above (four columns x two
+        // rows per lane) once per piece.
+        constexpr int R = MS == 4 ? 4 : 1;
+        float sacc[R];
+#pragma unroll
+        for (int ri = 0; ri < R; ++ri) sacc[ri] = 0.0f;
         uint32_t piece = 0;
         bool ok = true;
         // outer loop: the pieces of this CTA's range (a piece = its units of one column tile); inner loop:
@@ -1065,15 +1076,15 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
             //  - tiles with more packets than a stage holds: the rest is read from global memory.
             // Kernels for layers that need neither are compiled without that code: the presence of either
             // costs the common path 3-4 %.
-            using PKT = typename std::conditional<MS == 1, uint32_t, uint4>::type;
+            using PKT = typename std::conditional<MS != 8, uint32_t, uint4>::type;
             uint32_t sp_off = 0, sp_cnt = 0, sp_tail = 0, cmax = 0;
             const uint4* pk_s = reinterpret_cast<const uint4*>(st + p.off_coo);
             const uint4* pk_g = nullptr;
             const char* xtb = reinterpret_cast<const char*>(st + p.off_xt);
-            const uint32_t x_lane = MS == 1 ? 0u : 8u * t;    // byte offset of the lane's batch rows in a row of xt
+            const uint32_t x_lane = MS != 8 ? 0u : 8u * t;    // byte offset of the lane's batch rows in a row of xt
             auto load_packet = [&](uint32_t idx) -> PKT {
                 const uint4* src = (!HOT || idx < p.coo_cap) ? pk_s + idx : pk_g + idx;
-                if constexpr (MS == 1) return reinterpret_cast<const uint32_t*>(src)[t];
+                if constexpr (MS != 8) return reinterpret_cast<const uint32_t*>(src)[t];
                 else return *src;
             };
             auto packet = [&](uint32_t i) -> PKT {
@@ -1153,11 +1164,21 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
             if (SPARSE) {
                 // ---- outliers of this unit in the lane group's bucket (padding slots have value 0: they
                 // add 0)
-                if constexpr (MS == 1) {
-                    // single batch row: lane t keeps the slots of column number t of the bucket
-                    auto apply = [&](const uint32_t w) {
-                        sacc[0][0] = fmaf(__uint_as_float(w & 0xffff0000u), *reinterpret_cast<const float*>(xtb + ((w >> 3) & 0x1fcu)), sacc[0][0]);
+                if constexpr (MS != 8) {
+                    // column per lane: lane t keeps the slots of column number t of the bucket; a row of xt
+                    // holds the R batch rows of one k (slot & 0xfe0 = 32 * row)
+                    auto add = [&](float (&acc)[R], const float v, const uint32_t w) {
+                        if constexpr (R == 1) {
+                            acc[0] = fmaf(v, *reinterpret_cast<const float*>(xtb + ((w >> 3) & 0x1fcu)), acc[0]);
+                        } else {
+                            const float4 x = *reinterpret_cast<const float4*>(xtb + ((w >> 1) & 0x7f0u));
+                            acc[0] = fmaf(v, x.x, acc[0]);
+                            acc[1] = fmaf(v, x.y, acc[1]);
+                            acc[2] = fmaf(v, x.z, acc[2]);
+                            acc[R - 1] = fmaf(v, x.w, acc[R - 1]);
+                        }
                     };
+                    auto apply = [&](const uint32_t w) { add(sacc, __uint_as_float(w & 0xffff0000u), w); };
                     if (cmax > 0) apply(pk0);
                     if (cmax > 1) {
                         apply(pk1);
@@ -1169,21 +1190,25 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                             hot &= ~(0xfu << (hot_lane & ~3u));
                             const uint32_t hot_off = __shfl_sync(0xffffffffu, sp_off + sp_cnt, hot_lane);
                             const uint32_t hot_cnt = __shfl_sync(0xffffffffu, sp_tail, hot_lane);
-                            float hacc = 0.0f;
+                            float hacc[R];
+#pragma unroll
+                            for (int ri = 0; ri < R; ++ri) hacc[ri] = 0.0f;
                             for (uint32_t i = g; i < hot_cnt; i += 8) {
                                 const uint32_t idx = hot_off + i;
                                 const uint4 pk = (idx < p.coo_cap) ? pk_s[idx] : __ldg(pk_g + idx);
                                 const uint32_t w[4] = {pk.x, pk.y, pk.z, pk.w};
 #pragma unroll
-                                for (int e = 0; e < 4; ++e) {
-                                    const float v = ((w[e] >> 12) & 3u) == (uint32_t)t ? __uint_as_float(w[e] & 0xffff0000u) : 0.0f;
-                                    hacc = fmaf(v, *reinterpret_cast<const float*>(xtb + ((w[e] >> 3) & 0x1fcu)), hacc);
-                                }
+                                for (int e = 0; e < 4; ++e)     // a tail slot names its column
+                                    add(hacc, ((w[e] >> 12) & 3u) == (uint32_t)t ? __uint_as_float(w[e] & 0xffff0000u) : 0.0f, w[e]);
                             }
-                            hacc += __shfl_xor_sync(0xffffffffu, hacc, 4);
-                            hacc += __shfl_xor_sync(0xffffffffu, hacc, 8);
-                            hacc += __shfl_xor_sync(0xffffffffu, hacc, 16);
-                            if ((uint32_t)g == (hot_lane >> 2)) sacc[0][0] += hacc;
+#pragma unroll
+                            for (int ri = 0; ri < R; ++ri) {
+                                float v = hacc[ri];
+                                v += __shfl_xor_sync(0xffffffffu, v, 4);
+                                v += __shfl_xor_sync(0xffffffffu, v, 8);
+                                v += __shfl_xor_sync(0xffffffffu, v, 16);
+                                if ((uint32_t)g == (hot_lane >> 2)) sacc[ri] += v;
+                            }
                         }
                     }
                 } else {
@@ -1292,10 +1317,24 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                     // from lane (g, c); batch row 0 lives in lane t = 0
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
-                        const float v = __shfl_sync(0xffffffffu, sacc[0][0], (lane & ~3) | c);
+                        const float v = __shfl_sync(0xffffffffu, sacc[0], (lane & ~3) | c);
                         if (t == 0) accf[0][c >> 1][2 * (c & 1)] += v;
                     }
-                    sacc[0][0] = 0.0f;
+                    sacc[0] = 0.0f;
+                }
+                if constexpr (SPARSE && MS == 4) {
+                    // four rows of outlier sums -> fragment layout: column number c comes from lane (g, c);
+                    // rows 0, 1 live in lane t = 0, rows 2, 3 in lane t = 1
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+#pragma unroll
+                        for (int j = 0; j < 2; ++j) {
+                            const float v0 = __shfl_sync(0xffffffffu, sacc[j], (lane & ~3) | c);
+                            const float v1 = __shfl_sync(0xffffffffu, sacc[R - 2 + j], (lane & ~3) | c);
+                            accf[0][c >> 1][2 * (c & 1) + j] += t == 0 ? v0 : (t == 1 ? v1 : 0.0f);
+                        }
+#pragma unroll
+                    for (int ri = 0; ri < R; ++ri) sacc[ri] = 0.0f;
                 }
                 if (NGRP > 1) {
                     if (grp == 1) {
@@ -1573,7 +1612,7 @@ static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, 
     std::memset(&p, 0, sizeof(p));
     p.M = M; p.K = L->K; p.N = L->N; p.KT = L->K / kBK; p.NT = L->N / BN; p.NB = NB; p.nsw = 0;
     const uint32_t w_bytes = 16 * BN * 4, sz_bytes = 2 * GPS * BN * 2;
-    const uint32_t xt_bytes = sparse ? (M == 1 ? 512 : MO * 4096) : 0;     // FP32 [k] for one batch row, else [octet][k][8]
+    const uint32_t xt_bytes = sparse ? (M == 1 ? 512 : (M <= 4 ? 2048 : MO * 4096)) : 0;     // FP32 [k], [k][4] or [octet][k][8]
     // Two groups of dense warps (each takes every other unit) pay off when a CTA has enough units to
     // stream; short jobs keep one group.  With two octets of rows the second group fits only because
     // the outlier step of that variant prefetches less (96 registers per thread).
@@ -1642,9 +1681,11 @@ static KernelFn pick_mma_sparse(bool sparse, uint32_t ms, uint32_t ngrp) {
         if (ngrp == 2) {
             if (!sparse) return (KernelFn)fq_mma_kernel<BN, MO, G, false, 8, 2, false>;
             if (ms == 1) return (KernelFn)fq_mma_kernel<BN, MO, G, true, 1, 2, HOT>;
+            if (ms == 4) return (KernelFn)fq_mma_kernel<BN, MO, G, true, 4, 2, HOT>;
             return (KernelFn)fq_mma_kernel<BN, MO, G, true, 8, 2, HOT>;
         }
         if (sparse && ms == 1) return (KernelFn)fq_mma_kernel<BN, MO, G, true, 1, 1, HOT>;
+        if (sparse && ms == 4) return (KernelFn)fq_mma_kernel<BN, MO, G, true, 4, 1, HOT>;
     }
     if constexpr (MO == 2) {
         if (ngrp == 2) return sparse ? (KernelFn)fq_mma_kernel<BN, MO, G, true, 8, 2, HOT> : (KernelFn)fq_mma_kernel<BN, MO, G, false, 8, 2, false>;
@@ -1658,7 +1699,7 @@ static KernelFn pick_mma_group(uint32_t g, bool sparse, uint32_t ms, uint32_t ng
     return hot ? pick_mma_sparse<BN, MO, 128, true>(sparse, ms, ngrp) : pick_mma_sparse<BN, MO, 128, false>(sparse, ms, ngrp);
 }
 static KernelFn pick_mma_kernel(uint32_t bn, uint32_t M, uint32_t g, bool sparse, uint32_t ngrp, bool hot) {
-    const uint32_t mo = M <= 8 ? 1 : 2, ms = M <= 1 ? 1 : 8;
+    const uint32_t mo = M <= 8 ? 1 : 2, ms = M <= 1 ? 1 : (M <= 4 ? 4 : 8);
     if (bn == 128) return mo == 1 ? pick_mma_group<128, 1>(g, sparse, ms, ngrp, hot) : pick_mma_group<128, 2>(g, sparse, ms, ngrp, hot);
     return mo == 1 ? pick_mma_group<256, 1>(g, sparse, ms, ngrp, hot) : pick_mma_group<256, 2>(g, sparse, ms, ngrp, hot);
 }

@@ -803,9 +803,10 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
     constexpr int DW0 = 1 + NA;                             // first dense warp
     // NGRP dense warp groups: group r takes the units it with it mod NGRP == r
     constexpr int CG = 2;                                   // 16-column MMA strips per warp
-    // two groups of 16-row warps share the register file: one packet requested ahead instead of two and
-    // its activation rows, two contributors in flight when a split tile is settled
-    constexpr bool kTight = MO == 2 && NGRP == 2;
+    // two groups of 16-row warps share the register file, and 32-row warps fill it alone: one packet
+    // requested ahead instead of two and its activation rows, two contributors in flight when a split
+    // tile is settled
+    constexpr bool kTight = (MO == 2 && NGRP == 2) || MO == 4;
     constexpr int GPS = kBK / GROUP;
     constexpr int W_BYTES = 16 * BN * 4;
     constexpr int SZ_ROW = BN * 2;
@@ -960,11 +961,12 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
             if (lane == 0 && w.it >= S) request(w.u, w.tn, w.kt, smem_u32(st), bar_full + 8 * s, ip, npk);
             uint8_t* dst = st + p.off_xcan + m * kXPitch;
             const int swz = (m & 1) << 2;
-            float sum = 0.0f;
+            float sum = 0.0f, sum_lo = 0.0f;          // sum_lo: chunks 0-7 where a lane holds a whole row
 #pragma unroll
             for (int c = 0; c < CPL; ++c) {
                 const uint4 v = xv[c];
                 *reinterpret_cast<uint4*>(dst + ((part * CPL + c) ^ swz) * 16) = v;
+                if (LPR == 1 && c == 8) sum_lo = sum, sum = 0.0f;
                 sum += (bf16lo(v.x) + bf16hi(v.x)) + (bf16lo(v.y) + bf16hi(v.y)) + (bf16lo(v.z) + bf16hi(v.z)) +
                        (bf16lo(v.w) + bf16hi(v.w));
             }
@@ -975,10 +977,13 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                 const float s2 = s1 + __shfl_xor_sync(0xffffffffu, s1, 16);
                 if (GPS == 2) { if ((part & 1) == 0) xsum[(part >> 1) * ROWS + m] = s1; }
                 else if (part == 0) xsum[m] = s2;
-            } else {
+            } else if (LPR == 2) {
                 const float s1 = sum + __shfl_xor_sync(0xffffffffu, sum, 16);
                 if (GPS == 2) xsum[part * ROWS + m] = sum;
                 else if (part == 0) xsum[m] = s1;
+            } else {
+                if (GPS == 2) xsum[m] = sum_lo, xsum[ROWS + m] = sum;
+                else xsum[m] = sum_lo + sum;
             }
             __syncwarp();
             if (SPARSE && MS == 1) {
@@ -1606,7 +1611,7 @@ static fq_status_t make_plan(const fq_layout_t* L, uint32_t M, bool sparse, Plan
 // Plan of the small-batch kernel (fq_mma_kernel): M <= 16 per launch.
 static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, Plan& pl) {
     const uint32_t BN = L->BN, NB = L->buckets_per_tile, GPS = kBK / L->group;
-    const uint32_t MO = M <= 8 ? 1 : 2, ROWS = 8 * MO;
+    const uint32_t MO = M <= 8 ? 1 : (M <= 16 ? 2 : 4), ROWS = 8 * MO;
     const uint32_t NDW = BN / 32;
     Params& p = pl.p;
     std::memset(&p, 0, sizeof(p));
@@ -1633,7 +1638,7 @@ static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, 
         }
     }
     p.split = split;
-    pl.ngrp = units_per_cta >= 8 ? 2 : 1;
+    pl.ngrp = (units_per_cta >= 8 && MO <= 2) ? 2 : 1;    // four octets of rows: the accumulators leave no room
     const uint32_t xch_bytes = pl.ngrp > 1 ? BN * ROWS * 4 : 0;   // hand-over of a group's partial sums
     const uint32_t fixed = 1024 + xch_bytes;
     const uint32_t budget = kSmemBudget;
@@ -1699,9 +1704,9 @@ static KernelFn pick_mma_group(uint32_t g, bool sparse, uint32_t ms, uint32_t ng
     return hot ? pick_mma_sparse<BN, MO, 128, true>(sparse, ms, ngrp) : pick_mma_sparse<BN, MO, 128, false>(sparse, ms, ngrp);
 }
 static KernelFn pick_mma_kernel(uint32_t bn, uint32_t M, uint32_t g, bool sparse, uint32_t ngrp, bool hot) {
-    const uint32_t mo = M <= 8 ? 1 : 2, ms = M <= 1 ? 1 : (M <= 4 ? 4 : 8);
-    if (bn == 128) return mo == 1 ? pick_mma_group<128, 1>(g, sparse, ms, ngrp, hot) : pick_mma_group<128, 2>(g, sparse, ms, ngrp, hot);
-    return mo == 1 ? pick_mma_group<256, 1>(g, sparse, ms, ngrp, hot) : pick_mma_group<256, 2>(g, sparse, ms, ngrp, hot);
+    const uint32_t mo = M <= 8 ? 1 : (M <= 16 ? 2 : 4), ms = M <= 1 ? 1 : (M <= 4 ? 4 : 8);
+    if (bn == 128) return mo == 1 ? pick_mma_group<128, 1>(g, sparse, ms, ngrp, hot) : mo == 2 ? pick_mma_group<128, 2>(g, sparse, ms, ngrp, hot) : pick_mma_group<128, 4>(g, sparse, ms, ngrp, hot);
+    return mo == 1 ? pick_mma_group<256, 1>(g, sparse, ms, ngrp, hot) : mo == 2 ? pick_mma_group<256, 2>(g, sparse, ms, ngrp, hot) : pick_mma_group<256, 4>(g, sparse, ms, ngrp, hot);
 }
 
 // Which kernel serves a call.  Default: the small-batch kernel, in launches of 16 rows (at M = 32 two such
@@ -1780,7 +1785,8 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
     if (st != FQ_OK) return st;
     if (workspace_bytes < need) return fail(FQ_ERR_BUFFER_TOO_SMALL, "workspace holds %zu bytes, %zu needed", workspace_bytes, need);
     const bool use_mma = engine() == kEngineMma || (engine() == kEngineMix && M <= 16);
-    const uint32_t rows_per_launch = use_mma ? 16 : 32;
+    // the small-batch kernel takes up to 32 rows per launch; a remainder of at most 16 rows gets the cheaper variants
+    const uint32_t rows_per_launch = 32;
     for (uint32_t m0 = 0; m0 < M; m0 += rows_per_launch) {
         const uint32_t mb = std::min<uint32_t>(rows_per_launch, M - m0);
         Plan pl;

@@ -188,7 +188,7 @@ fq_status_t fq_validate_tilecoo(const fq_layout_t* L, const uint32_t* tile_indpt
 fq_status_t fq_workspace_bytes(const fq_layout_t* L, uint32_t M, size_t* bytes);
 
 /*
- * The fused operator (Eq. 1; Sections 3.1 and 4.1): one launch per 16 rows of X
+ * The fused operator (Eq. 1; Sections 3.1 and 4.1): one launch per 32 rows of X
  * reads X, W_Q and the Tile-COO tiles through a bulk-copy/mbarrier ring,
  * dequantises in registers into tensor-core operands, applies the tile's
  * outliers against the same shared-memory activation tile, and writes Y once.

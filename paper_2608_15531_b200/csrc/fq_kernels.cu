@@ -893,7 +893,7 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
         const uint32_t aw = warp - 1;
         // lane -> (row m, part): 16-byte chunks of that row; rows beyond M are zero
         constexpr int ROWS = 8 * MO;
-        constexpr int LPR = 32 / ROWS;                       // lanes per row: 4 (8 rows) or 2 (16 rows)
+        constexpr int LPR = 32 / ROWS;                       // lanes per row: 4 (8 rows), 2 (16 rows) or 1 (32 rows)
         constexpr int CPL = 16 / LPR;                        // chunks per lane
         const int m = lane % ROWS, part = lane / ROWS;
         const bool real = (uint32_t)m < p.M;
@@ -1709,8 +1709,8 @@ static KernelFn pick_mma_kernel(uint32_t bn, uint32_t M, uint32_t g, bool sparse
     return mo == 1 ? pick_mma_group<256, 1>(g, sparse, ms, ngrp, hot) : mo == 2 ? pick_mma_group<256, 2>(g, sparse, ms, ngrp, hot) : pick_mma_group<256, 4>(g, sparse, ms, ngrp, hot);
 }
 
-// Which kernel serves a call.  Default: the small-batch kernel, in launches of 16 rows (at M = 32 two such
-// launches take about half the time of one launch of the tcgen05 kernel as it stands).  FQ_ENGINE=tc
+// Which kernel serves a call.  Default: the small-batch kernel, in launches of up to 32 rows (at M = 32 one
+// such launch takes about a third of the time of the tcgen05 kernel as it stands).  FQ_ENGINE=tc
 // routes every call to the tcgen05 kernel (launches of 32 rows), FQ_ENGINE=mix uses it for M > 16.
 enum Engine { kEngineMma, kEngineTc, kEngineMix };
 static Engine engine() {

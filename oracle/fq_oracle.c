@@ -13,7 +13,8 @@
  *   - dequantisation  w^ = s (q - z)          Eq. 3
  *   - result  Y = X deq(W_Q) + X W_O          Eq. 1
  *   - Tile-COO arrays (tile_indptr, bucket_info, packed_outliers; four
- *     outliers per 16-byte packet, u8 row index, u8 column index, BF16 value)
+ *     outliers per 16-byte packet, each a 32-bit slot: BF16 value, row inside
+ *     the tile, column number inside the bucket)
  *                                             Section 3.2.1, Table 1
  *
  * Readings taken where the paper is silent (each also listed in the design
@@ -193,8 +194,8 @@ void orc_fused_matmul(const uint16_t* X, uint32_t M, uint32_t K, uint32_t N, uin
  *   ordered tn-major (chunk index tn * (K/128) + kt).  A chunk covers 128 rows
  *   by BN columns and holds 16 * BN little-endian 32-bit words.  Word index
  *   inside the chunk, with j = 0..3, t = 0..BN-1, w = 0..3:
- *        (((j * (BN/32) + t/32) * 8 + t%8) * 4 + w) * 4 + (t/8)%4
- *   (integer division).  Nibble p (bits 4p .. 4p+3) of that word, p = i + 4h with
+ *        (j * BN + t) * 4 + w .
+ *   Nibble p (bits 4p .. 4p+3) of that word, p = i + 4h with
  *   i = 0..3, h = 0..1, is the code of
  *        column  tn*BN + t
  *        row     kt*128 + 32*j + 8*w + 2*i + h
@@ -209,7 +210,7 @@ int orc_decode_wq(const uint32_t* wq, uint32_t K, uint32_t N, uint32_t BN, uint8
             for (uint32_t j = 0; j < 4; ++j)
                 for (uint32_t t = 0; t < BN; ++t)
                     for (uint32_t w = 0; w < 4; ++w) {
-                        uint32_t word = chunk[(((j * (BN / 32) + t / 32) * 8 + t % 8) * 4 + w) * 4 + (t / 8) % 4];
+                        uint32_t word = chunk[(j * BN + t) * 4 + w];
                         for (uint32_t p = 0; p < 8; ++p) {
                             uint32_t i = p & 3, h = p >> 2;
                             uint32_t col = tn * BN + t;

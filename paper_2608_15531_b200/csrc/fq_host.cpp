@@ -3,7 +3,6 @@
 #include <algorithm>
 #include <cmath>
 #include <cstring>
-#include <queue>
 #include <vector>
 
 #include "fq_internal.h"
@@ -31,8 +30,7 @@ static inline float bf16_to_f32(uint16_t h) {
 // Position of the code of (row kr, column cr) inside a 128 x BN chunk: word index and nibble.
 static inline void wq_slot(uint32_t kr, uint32_t cr, uint32_t BN, uint32_t& word, uint32_t& nib) {
     const uint32_t j = kr >> 5, w = (kr >> 3) & 3, i = (kr >> 1) & 3, h = kr & 1;
-    const uint32_t strip = cr >> 5, qd = (cr >> 3) & 3, g = cr & 7;
-    word = (((j * (BN / 32) + strip) * 8 + g) * 4 + w) * 4 + qd;
+    word = (j * BN + cr) * 4 + w;
     nib = i + 4 * h;
 }
 }  // namespace fq

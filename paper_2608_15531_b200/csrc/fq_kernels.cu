@@ -46,28 +46,10 @@
 namespace fq {
 
 constexpr int kBK = 128;
-#ifdef FQ_TRACE
-constexpr int kSmemBudget = 232448 - 16384;
-#else
 constexpr int kSmemBudget = 232448;    // 227 KB per CTA on sm_100
-#endif
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 constexpr uint32_t kTmemCols = 512;
 
-#ifdef FQ_TRACE
-// Developer build only: cycle stamps of CTA 0's first iterations, [role][iteration][event].
-__device__ unsigned long long g_trace[12 * 32 * 4];
-__shared__ unsigned long long s_trace[12 * 32 * 4];
-#define FQ_STAMP(role, it, ev) do { if (blockIdx.x == 0 && (it) < 32 && (ev) < 4 && lane == 0) s_trace[((role) * 32 + (it)) * 4 + (ev)] = clock64(); } while (0)
-#define FQ_DSTAMP(it, e) do { if (dw == 2) FQ_STAMP(4 + (e) / 4, it, (e) % 4); } while (0)
-// wall-clock stamps of every CTA of the small-batch kernel, [cta][event]
-__device__ unsigned long long g_ktrace[192 * 16];
-#define FQ_GT(cond, ev) do { if (cond) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_ktrace[blockIdx.x * 16 + (ev)] = t_; } } while (0)
-#else
-#define FQ_STAMP(role, it, ev) do {} while (0)
-#define FQ_DSTAMP(it, e) do {} while (0)
-#define FQ_GT(cond, ev) do {} while (0)
-#endif
 
 struct Params {
     const uint16_t* X;
@@ -83,6 +65,7 @@ struct Params {
     float* partials;
     uint32_t M, K, N, KT, NT;
     uint32_t NB, coo_cap, stages, nsw;
+    uint32_t nact;    // tcgen05 kernel: activation warps at work (the ring length is a multiple of it)
     uint32_t split;   // small-batch kernel: 0 = units dealt out as one contiguous range per CTA (stream-K);
                       // c > 0 = every column tile belongs to c CTAs, CTA b takes part b mod c of tile b / c
     // shared-memory offsets (bytes); the first five are relative to a stage
@@ -113,12 +96,14 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+// The time hint lets a waiting thread sleep in hardware (up to about 20 us per attempt) instead of
+// spinning on the issue slots that the working warps of the CTA need.
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
-        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}"
         : "=r"(ok)
-        : "r"(bar), "r"(parity)
+        : "r"(bar), "r"(parity), "r"(20000u)
         : "memory");
     return ok;
 }
@@ -142,7 +127,7 @@ __device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, vo
     uint32_t spins = 0;
     unsigned long long t0 = 0;
     while (!mbar_try_wait(bar, parity)) {
-        if ((++spins & 0xff) == 0) {
+        if ((++spins & 0xf) == 0) {
             if (*abort_flag) return false;
             unsigned long long now = globaltimer_ns();
             if (t0 == 0) {
@@ -266,54 +251,6 @@ struct UnitIter {
     }
 };
 
-// ----------------------------------------------------------------------------- sparse step
-
-
-// Position of 16-byte quad j of column c's FP32 row.  Q = quads per row when the row is XOR-swizzled
-// (4 or 8: lanes hitting random columns then spread over all bank groups), 0 = plain layout.
-template <int Q>
-__device__ __forceinline__ uint32_t shc_quad(uint32_t c, uint32_t j, uint32_t ldc) {
-    if (Q == 4) return c * ldc + ((j ^ ((c >> 1) & 3u)) << 2);
-    if (Q == 8) return c * ldc + ((j ^ (c & 7u)) << 2);
-    return c * ldc + (j << 2);
-}
-
-__device__ __forceinline__ void fma8(float4& c0, float4& c1, float v, const float4 x0, const float4 x1) {
-    c0.x = fmaf(v, x0.x, c0.x); c0.y = fmaf(v, x0.y, c0.y); c0.z = fmaf(v, x0.z, c0.z); c0.w = fmaf(v, x0.w, c0.w);
-    c1.x = fmaf(v, x1.x, c1.x); c1.y = fmaf(v, x1.y, c1.y); c1.z = fmaf(v, x1.z, c1.z); c1.w = fmaf(v, x1.w, c1.w);
-}
-
-// One packet (four outliers) against the k-major FP32 activation copy xt ([128][8] floats, 32 B per
-// row k): row c of the FP32 tile += v * x[8o..8o+7][k], slot after slot (Section 4.2).  A slot names
-// its row (slot & 0xfe0 = 32 * row) and its column's number inside the bucket (bits 12-13); col0 is
-// the bucket's column number 0, the others follow 8 apart.  Slots of one packet may share a column,
-// so each slot finishes its read-modify-write before the next one starts; the activation rows of
-// all four are loaded first.  Padding slots (value 0) are skipped.
-template <int Q>
-__device__ __forceinline__ void apply_packet(const uint4 pk, const float* __restrict__ xt, float* shc, uint32_t col0,
-                                             uint32_t o, uint32_t ldc) {
-    const uint32_t w[4] = {pk.x, pk.y, pk.z, pk.w};
-    float4 x0[4], x1[4];
-#pragma unroll
-    for (int s = 0; s < 4; ++s) {
-        const float4* xp = reinterpret_cast<const float4*>(reinterpret_cast<const char*>(xt) + (w[s] & 0xfe0u));
-        x0[s] = xp[0];
-        x1[s] = xp[1];
-    }
-#pragma unroll
-    for (int s = 0; s < 4; ++s) {
-        if (w[s] >> 16) {
-            const uint32_t c = col0 + ((w[s] >> 9) & 0x18u);
-            float4* p0 = reinterpret_cast<float4*>(shc + shc_quad<Q>(c, 2 * o, ldc));
-            float4* p1 = reinterpret_cast<float4*>(shc + shc_quad<Q>(c, 2 * o + 1, ldc));
-            float4 c0 = *p0, c1 = *p1;
-            fma8(c0, c1, __uint_as_float(w[s] & 0xffff0000u), x0[s], x1[s]);
-            *p0 = c0;
-            *p1 = c1;
-        }
-    }
-}
-
 // Transpose one octet of BF16 activation rows into the FP32 k-major copy xt[k][8] (32 B per k).
 // `row0` is the shared-memory address of row 0 / 16-byte chunk 0 of the octet, rows `row_step`
 // bytes apart, consecutive 16-byte chunks (8 k each) `chunk_step` bytes apart.  Whole warp.
@@ -335,430 +272,7 @@ __device__ __forceinline__ void transpose_octet_f32(uint32_t row0, uint32_t row_
     }
 }
 
-// ----------------------------------------------------------------------------- fused kernel
-
-// BN: tile columns (128 or 256).  NB16: batch columns of the MMA in units of 16 (1: M <= 16, 2: M <= 32).
-template <int BN, int NB16, int GROUP, bool SPARSE>
-__global__ void __launch_bounds__(32 * (4 + 2 * (BN / 32) + 4), 1) fq_fused_kernel(const Params p) {
-    constexpr int NDW = BN / 32;              // dense warps: one thread per tile column
-    constexpr int NT128 = BN / 128;           // 128-row MMA tiles per unit
-    constexpr int NMMA = 16 * NB16;           // MMA N: batch rows, padded
-    constexpr int GPS = kBK / GROUP;          // groups per k-step
-    constexpr int DCOLS = GPS * NMMA;         // accumulator columns per D buffer
-    constexpr int W_BYTES = 16 * BN * 4;
-    constexpr int SZ_ROW = BN * 2;
-    constexpr int LDC = NMMA;                 // sh_c row: FP32 per batch row
-    constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NMMA >> 3) << 17) | (8u << 24);
-    extern __shared__ __align__(128) uint8_t smem[];
-
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t S = p.stages;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
-    const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * S;
-    const uint32_t bar_a_ready = bar_empty + 8 * S;      // [2]
-    const uint32_t bar_d_ready = bar_a_ready + 16;       // [2]
-    const uint32_t bar_sparse_done = bar_d_ready + 16, bar_dense_done = bar_sparse_done + 8;
-    const uint32_t bar_dense = bar_dense_done + 8, bar_final = bar_dense + 8;
-    const uint32_t bar_d_free = bar_final + 8;           // [2]
-    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 2 * S + 10);
-    volatile uint32_t* last_flag = abort_flag + 1;
-    volatile uint32_t* tmem_slot = abort_flag + 2;
-    float* shc = reinterpret_cast<float*>(smem + p.off_shc);
-
-    const uint32_t nsw = SPARSE ? p.nsw : 0;
-    if (tid == 0) {
-        for (uint32_t s = 0; s < S; ++s) {
-            mbar_init(bar_full + 8 * s, 2);   // producer's expect_tx arrival + activation warp
-            mbar_init(bar_empty + 8 * s, 2 * NDW + nsw + NT128);
-        }
-        mbar_init(bar_a_ready, NDW);
-        mbar_init(bar_a_ready + 8, NDW);
-        mbar_init(bar_d_ready, NT128);
-        mbar_init(bar_d_ready + 8, NT128);
-        mbar_init(bar_sparse_done, nsw ? nsw : 1);
-        mbar_init(bar_dense_done, NDW);
-        mbar_init(bar_dense, NDW);
-        mbar_init(bar_final, NT128);
-        mbar_init(bar_d_free, NDW);
-        mbar_init(bar_d_free + 8, NDW);
-        *abort_flag = 0;
-        *last_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (SPARSE) {
-        for (uint32_t i = tid; i < (uint32_t)(BN * LDC); i += blockDim.x) shc[i] = 0.0f;
-    }
-    if (warp == 1) {
-        tmem_alloc(smem_u32((const void*)tmem_slot), kTmemCols);
-        tmem_relinquish();
-    }
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
-
-    // contiguous range of units for this CTA
-    const uint32_t U = p.NT * p.KT, P = gridDim.x, q = U / P, r = U % P;
-    const uint32_t u_begin = unit_begin_of(blockIdx.x, q, r);
-    const uint32_t u_end = u_begin + q + (blockIdx.x < r ? 1u : 0u);
-    const uint32_t KT = p.KT;
-
-    if (warp == 0) {
-        // ------------------------------------------------------------------ producer
-        uint32_t ip_a = 0, ip_b = 0, issued = 0;
-        bool ok = true;
-        for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
-            const uint32_t u = w.u, it = w.it, s = w.s, ph = w.ph;
-            if (SPARSE && (it & 31) == 0) {  // this warp's next 32 packet ranges, one coalesced read
-                const uint32_t i = u + lane;
-                ip_a = (i <= U) ? __ldg(p.indptr + i) : 0;
-                ip_b = (i + 1 <= U) ? __ldg(p.indptr + i + 1) : 0;
-            }
-            uint32_t pk0 = 0, npk = 0;
-            if (SPARSE) {
-                pk0 = __shfl_sync(0xffffffffu, ip_a, it & 31);
-                npk = __shfl_sync(0xffffffffu, ip_b, it & 31) - pk0;
-                npk = min(npk, p.coo_cap);
-            }
-            if (!warp_wait(bar_empty + 8 * s, ph ^ 1, abort_flag, p.status)) { ok = false; break; }
-            FQ_STAMP(0, it, 0);
-            const uint32_t tn = w.tn, kt = w.kt;
-            const uint32_t full = bar_full + 8 * s;
-            const uint32_t st = smem_u32(smem) + s * p.stage_bytes;
-            if (lane == 0) {
-                uint32_t bytes = W_BYTES + 2 * GPS * SZ_ROW;
-                if (SPARSE) bytes += p.NB * 4 + npk * 16;
-                mbar_arrive_expect_tx(full, bytes);
-            }
-            __syncwarp();
-            if (lane == 0) {
-                bulk_g2s(st, p.wq + (size_t)u * W_BYTES, W_BYTES, full);
-#pragma unroll
-                for (int gi = 0; gi < GPS; ++gi) {
-                    const size_t row = (size_t)(kt * GPS + gi) * p.N + (size_t)tn * BN;
-                    bulk_g2s(st + p.off_sz + gi * SZ_ROW, p.scale + row, SZ_ROW, full);
-                    bulk_g2s(st + p.off_sz + (GPS + gi) * SZ_ROW, p.zero + row, SZ_ROW, full);
-                }
-            } else if (lane == 1) {
-                if (SPARSE) {
-                    bulk_g2s(st + p.off_info, p.info + (size_t)u * p.NB, p.NB * 4, full);
-                    if (npk) bulk_g2s(st + p.off_coo, p.packed + pk0, npk * 16, full);
-                }
-            }
-            FQ_STAMP(0, it, 1);
-            issued = it + 1;
-        }
-        if (!ok) {
-            // giving up: let the copies already issued land before the CTA's shared memory goes away
-            for (uint32_t j = (issued > S ? issued - S : 0); j < issued; ++j)
-                for (uint32_t spin = 0; spin < (1u << 20) && !mbar_try_wait(bar_full + 8 * (j % S), (j / S) & 1); ++spin) {}
-        }
-    } else if (warp == 1 || (warp == 3 && NT128 == 2)) {
-        // ------------------------------------------------------------------ tensor warps (one per 128-row tile)
-        const int ti = warp == 1 ? 0 : 1;
-        for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
-            const uint32_t it = w.it, s = w.s, ph = w.ph, b = w.it & 1;
-            if (!warp_wait(bar_full + 8 * s, ph, abort_flag, p.status)) break;
-            FQ_STAMP(1, it, 0);
-            if (!warp_wait(bar_a_ready + 8 * b, (it >> 1) & 1, abort_flag, p.status)) break;
-            if (it >= 2 && !warp_wait(bar_d_free + 8 * b, ((it - 2) >> 1) & 1, abort_flag, p.status)) break;
-            tc_fence_after();
-            FQ_STAMP(1, it, 1);
-            const uint64_t bd0 = make_b_desc(smem_u32(smem) + s * p.stage_bytes + p.off_xcan, (NMMA / 8) * 128, 128);
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const int gi = ks / (8 / GPS);
-                    const uint32_t d = tmem_base + ti * 256 + 128 + b * DCOLS + gi * NMMA;
-                    const uint32_t a = tmem_base + ti * 256 + b * 64 + ks * 8;
-                    umma_ts(d, a, bd0 + (uint64_t)((ks * 2 * (NMMA / 8) * 128) >> 4), IDESC, (ks % (8 / GPS)) != 0);
-                }
-            umma_commit(bar_d_ready + 8 * b);   // accumulators of this unit are complete
-            umma_commit(bar_empty + 8 * s);     // and the stage's activation operand has been read
-            FQ_STAMP(1, it, 2);
-        }
-        __syncwarp();
-        umma_commit(bar_final);                 // fires when every MMA this warp issued has retired
-    } else if (warp == 2) {
-        // ------------------------------------------------------------------ activation warp
-        // lane -> (row m, part): CPL 16-byte chunks of that row; rows beyond M are zero
-        constexpr int LPR = 32 / (NMMA < 32 ? NMMA : 32);   // lanes per row: 2 (N = 16) or 1 (N = 32)
-        constexpr int CPL = 16 / LPR;                        // 16-byte chunks per lane
-        const int m = lane % NMMA, part = lane / NMMA;
-        const bool real = (uint32_t)m < p.M;
-        const uint8_t* xrow = reinterpret_cast<const uint8_t*>(p.X) + ((size_t)m * p.K) * 2 + part * CPL * 16;
-        uint4 nxt[CPL];
-        auto load = [&](uint32_t kt) {
-#pragma unroll
-            for (int c = 0; c < CPL; ++c) {
-                nxt[c] = make_uint4(0, 0, 0, 0);
-                if (real) nxt[c] = __ldg(reinterpret_cast<const uint4*>(xrow + (size_t)kt * 256 + c * 16));
-            }
-        };
-        if (u_begin < u_end) load(u_begin - (u_begin / KT) * KT);
-        for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
-            const uint32_t s = w.s, ph = w.ph;
-            uint8_t* st = smem + s * p.stage_bytes;
-            uint4 xv[CPL];
-#pragma unroll
-            for (int c = 0; c < CPL; ++c) xv[c] = nxt[c];
-            if (w.u + 1 < u_end) load(w.kt + 1 == KT ? 0u : w.kt + 1);   // next unit's block, while this one is laid out
-            if (!warp_wait(bar_empty + 8 * s, ph ^ 1, abort_flag, p.status)) break;
-            uint8_t* dst = st + p.off_xcan + ((part * CPL) * (NMMA / 8) + (m >> 3)) * 128 + (m & 7) * 16;
-            float sum[2] = {0.0f, 0.0f};
-#pragma unroll
-            for (int c = 0; c < CPL; ++c) {
-                const uint4 v = xv[c];
-                *reinterpret_cast<uint4*>(dst + c * (NMMA / 8) * 128) = v;
-                const float t = (bf16lo(v.x) + bf16hi(v.x)) + (bf16lo(v.y) + bf16hi(v.y)) + (bf16lo(v.z) + bf16hi(v.z)) +
-                                (bf16lo(v.w) + bf16hi(v.w));
-                sum[(LPR == 1 && c >= 8) ? 1 : 0] += t;
-            }
-            // per-group sums of each activation row -> xsum[group][row], needed by the dense epilogue
-            float* xsum = reinterpret_cast<float*>(st + p.off_xsum);
-            if (LPR == 2) {
-                // lane `part` holds k 0..63 or 64..127 of its row
-                const float other = __shfl_xor_sync(0xffffffffu, sum[0], 16);
-                if (GPS == 2) xsum[part * NMMA + m] = sum[0];
-                else if (part == 0) xsum[m] = sum[0] + other;
-            } else {
-                if (GPS == 2) { xsum[m] = sum[0]; xsum[NMMA + m] = sum[1]; }
-                else xsum[m] = sum[0] + sum[1];
-            }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            __syncwarp();
-            if (SPARSE) {
-                // FP32 k-major copy for the sparse warps, one octet of rows at a time
-                for (uint32_t o = 0; o < ((p.M + 7) >> 3); ++o)
-                    transpose_octet_f32(smem_u32(st + p.off_xcan) + o * 128, 16, (NMMA / 8) * 128,
-                                        reinterpret_cast<float*>(st + p.off_xt) + o * 1024, lane);
-                __syncwarp();
-            }
-            if (lane == 0) mbar_arrive(bar_full + 8 * s);
-        }
-    } else if (warp >= 4 && warp < 4 + NDW) {
-        // ------------------------------------------------------------------ unpack warps: thread = column
-        const int dw = warp - 4;
-        const int col = dw * 32 + lane;                       // column inside the tile
-        const uint32_t t_lane = ((uint32_t)((dw & 3) * 32)) << 16;
-        const uint32_t t_tile = tmem_base + (uint32_t)(dw >> 2) * 256 + t_lane;
-        for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
-            const uint32_t it = w.it, s = w.s, ph = w.ph, b = w.it & 1;
-            const uint8_t* st = smem + s * p.stage_bytes;
-            if (!warp_wait(bar_full + 8 * s, ph, abort_flag, p.status)) break;
-            // the A buffer of this parity was last read by the MMAs of unit it - 2
-            if (it >= 2 && !warp_wait(bar_d_ready + 8 * b, ((it - 2) >> 1) & 1, abort_flag, p.status)) break;
-            tc_fence_after();
-            FQ_DSTAMP(it, 0);
-            // four 16-byte chunks = 128 codes of this column -> A operand rows in TMEM
-            const uint32_t* wp = reinterpret_cast<const uint32_t*>(st) + ((col >> 5) * 8 + (col & 7)) * 16 + ((col >> 3) & 3);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                uint4 w4;                                           // the column's words of 8-row blocks 0..3
-                w4.x = wp[j * BN * 4], w4.y = wp[j * BN * 4 + 4], w4.z = wp[j * BN * 4 + 8], w4.w = wp[j * BN * 4 + 12];
-#pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
-                    const uint32_t w0 = hf ? w4.z : w4.x, w1 = hf ? w4.w : w4.y;
-                    uint32_t a[8];
-                    a[0] = codes_to_bf16x2(w0);
-                    a[1] = codes_to_bf16x2(w0 >> 4);
-                    a[2] = codes_to_bf16x2(w0 >> 8);
-                    a[3] = codes_to_bf16x2(w0 >> 12);
-                    a[4] = codes_to_bf16x2(w1);
-                    a[5] = codes_to_bf16x2(w1 >> 4);
-                    a[6] = codes_to_bf16x2(w1 >> 8);
-                    a[7] = codes_to_bf16x2(w1 >> 12);
-                    tmem_st8(t_tile + b * 64 + (j * 2 + hf) * 8, a);
-                }
-            }
-            FQ_DSTAMP(it, 1);
-            tmem_wait_st();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) {
-                mbar_arrive_relaxed(bar_a_ready + 8 * b);
-                mbar_arrive_relaxed(bar_empty + 8 * s);
-            }
-            FQ_DSTAMP(it, 2);
-        }
-    } else if (warp >= 4 + NDW && warp < 4 + 2 * NDW) {
-        // ------------------------------------------------------------------ epilogue warps: thread = column
-        const int dw = warp - 4 - NDW;
-        const int col = dw * 32 + lane;
-        const uint32_t t_lane = ((uint32_t)((dw & 3) * 32)) << 16;
-        const uint32_t t_tile = tmem_base + (uint32_t)(dw >> 2) * 256 + t_lane;
-        float accf[NMMA];
-#pragma unroll
-        for (int i = 0; i < NMMA; ++i) accf[i] = 0.0f;
-        uint32_t piece = 0, dense_phase = 0;
-        bool ok = true;
-        for (UnitIter w(u_begin, KT); w.u < u_end && ok; w.next(S, KT)) {
-            const uint32_t u = w.u, it = w.it, s = w.s, b = w.it & 1;
-            const uint32_t tn = w.tn, kt = w.kt;
-            const uint8_t* st = smem + s * p.stage_bytes;
-            // scale / zero-point / activation sums of the unit once its MMAs are complete
-            if (!warp_wait(bar_d_ready + 8 * b, (it >> 1) & 1, abort_flag, p.status)) { ok = false; break; }
-            tc_fence_after();
-            FQ_DSTAMP(it, 4);
-            const uint16_t* sc = reinterpret_cast<const uint16_t*>(st + p.off_sz);
-            const float4* xsum = reinterpret_cast<const float4*>(st + p.off_xsum);
-#pragma unroll
-            for (int gi = 0; gi < GPS; ++gi) {
-                const float sv = bf16_bits_to_float(sc[gi * BN + col]);
-                const float zc = -(128.0f + bf16_bits_to_float(sc[(GPS + gi) * BN + col]));
-#pragma unroll
-                for (int h = 0; h < NB16; ++h) {
-                    float d[16];
-                    tmem_ld16(t_tile + 128 + b * DCOLS + gi * NMMA + h * 16, d);
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const float4 xs = xsum[(gi * NMMA + h * 16) / 4 + i];
-                        accf[h * 16 + 4 * i + 0] = fmaf(sv, fmaf(zc, xs.x, d[4 * i + 0]), accf[h * 16 + 4 * i + 0]);
-                        accf[h * 16 + 4 * i + 1] = fmaf(sv, fmaf(zc, xs.y, d[4 * i + 1]), accf[h * 16 + 4 * i + 1]);
-                        accf[h * 16 + 4 * i + 2] = fmaf(sv, fmaf(zc, xs.z, d[4 * i + 2]), accf[h * 16 + 4 * i + 2]);
-                        accf[h * 16 + 4 * i + 3] = fmaf(sv, fmaf(zc, xs.w, d[4 * i + 3]), accf[h * 16 + 4 * i + 3]);
-                    }
-                }
-            }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) {
-                mbar_arrive_relaxed(bar_d_free + 8 * b);   // the tensor warp may overwrite this D buffer
-                mbar_arrive_relaxed(bar_empty + 8 * s);
-            }
-            FQ_DSTAMP(it, 5);
-
-            if (kt == KT - 1 || u == u_end - 1) {
-                // ---------------------------------------------------------- end of a piece
-                if (SPARSE) {
-                    if (!warp_wait(bar_sparse_done, piece & 1, abort_flag, p.status)) { ok = false; break; }
-#pragma unroll
-                    for (int i = 0; i < NMMA / 4; ++i) {
-                        float4* cp = reinterpret_cast<float4*>(shc + shc_quad<LDC / 4>(col, i, LDC));
-                        const float4 v = *cp;
-                        accf[4 * i + 0] += v.x;
-                        accf[4 * i + 1] += v.y;
-                        accf[4 * i + 2] += v.z;
-                        accf[4 * i + 3] += v.w;
-                        *cp = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                    }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_dense_done);
-                }
-                const uint32_t u_tile0 = tn * KT;
-                const uint32_t piece_k0 = max(u_tile0, u_begin) - u_tile0;
-                const bool full_piece = (piece_k0 == 0) && (kt == KT - 1);
-                bool write_y = full_piece;
-                if (!full_piece) {
-                    // FP32 partial [m][column]; the last CTA to arrive sums them in CTA order
-                    const uint32_t which = (u_begin / KT == tn) ? 0u : 1u;
-                    float* slot = p.partials + ((size_t)blockIdx.x * 2 + which) * (size_t)(BN * LDC);
-#pragma unroll
-                    for (int m = 0; m < NMMA; ++m)
-                        if ((uint32_t)m < p.M) __stcg(slot + m * BN + col, accf[m]);
-                    __threadfence();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_dense);
-                    if (!warp_wait(bar_dense, dense_phase & 1, abort_flag, p.status)) { ok = false; break; }
-                    ++dense_phase;
-                    const uint32_t c_first = cta_of_unit(u_tile0, q, r), c_last = cta_of_unit(u_tile0 + KT - 1, q, r);
-                    if (dw == 0 && lane == 0) {
-                        const uint32_t old = atomicAdd(p.counters + tn, 1u);
-                        *last_flag = (old == c_last - c_first) ? 1u : 0u;
-                    }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_dense);
-                    if (!warp_wait(bar_dense, dense_phase & 1, abort_flag, p.status)) { ok = false; break; }
-                    ++dense_phase;
-                    if (*last_flag) {
-                        write_y = true;
-                        __threadfence();
-#pragma unroll
-                        for (int m = 0; m < NMMA; ++m) accf[m] = 0.0f;
-                        for (uint32_t c = c_first; c <= c_last; ++c) {
-                            const uint32_t wch = (unit_begin_of(c, q, r) / KT == tn) ? 0u : 1u;
-                            const float* sl = p.partials + ((size_t)c * 2 + wch) * (size_t)(BN * LDC);
-#pragma unroll
-                            for (int m = 0; m < NMMA; ++m)
-                                if ((uint32_t)m < p.M) accf[m] += __ldcg(sl + m * BN + col);
-                        }
-                        if (dw == 0 && lane == 0) p.counters[tn] = 0;  // ready for the next call
-                    }
-                }
-                if (write_y) {
-#pragma unroll
-                    for (int m = 0; m < NMMA; ++m)
-                        if ((uint32_t)m < p.M) p.Y[(size_t)m * p.N + (size_t)tn * BN + col] = float_to_bf16_bits(accf[m]);
-                }
-#pragma unroll
-                for (int m = 0; m < NMMA; ++m) accf[m] = 0.0f;
-                ++piece;
-            }
-        }
-    } else if (SPARSE && warp >= 4 + 2 * NDW) {
-        // ------------------------------------------------------------------ sparse
-        const uint32_t sw = warp - (4 + 2 * NDW);
-        if (sw + 1 <= nsw) {
-            const uint32_t nbb = p.NB >> 5;            // blocks of 32 buckets
-            const uint32_t bb = sw % nbb, og = sw / nbb, n_og = nsw / nbb;
-            const uint32_t bucket = bb * 32 + lane;
-            const uint32_t n_oct = (p.M + 7) >> 3;
-            uint32_t piece = 0;
-            for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
-                const uint32_t u = w.u, s = w.s, ph = w.ph, kt = w.kt;
-                const uint8_t* st = smem + s * p.stage_bytes;
-                if (!warp_wait(bar_full + 8 * s, ph, abort_flag, p.status)) break;
-                if (sw == 0) FQ_STAMP(3, w.it, 0);
-                const uint32_t info = reinterpret_cast<const uint32_t*>(st + p.off_info)[bucket];
-                const uint32_t off = info & 0xffffu, cnt = ((info >> 16) & 0xffu) + (info >> 24);   // column-slotted + tail
-                const uint32_t col0 = ((bucket >> 3) << 5) | (bucket & 7u);
-                const uint4* pk_s = reinterpret_cast<const uint4*>(st + p.off_coo);
-                const uint4* pk_g = nullptr;
-                if (off + cnt > p.coo_cap) pk_g = p.packed + __ldg(p.indptr + u);  // tail of an oversized tile
-                for (uint32_t o = og; o < n_oct; o += n_og) {
-                    const float* xt = reinterpret_cast<const float*>(st + p.off_xt) + o * 1024;
-                    if (sw == 0) FQ_STAMP(3, w.it, 1);
-#ifdef FQ_TRACE
-                    if (sw == 0 && blockIdx.x == 0 && w.it < 32) {
-                        const uint32_t mx = __reduce_max_sync(0xffffffffu, cnt);
-                        const uint32_t sm = __reduce_add_sync(0xffffffffu, cnt);
-                        if (lane == 0) s_trace[(3 * 32 + w.it) * 4 + 3] = ((unsigned long long)mx << 32) | sm;
-                    }
-#endif
-                    for (uint32_t i = 0; i < cnt; ++i) {
-                        const uint32_t idx = off + i;
-                        const uint4 pk = (idx < p.coo_cap) ? pk_s[idx] : __ldg(pk_g + idx);
-                        apply_packet<LDC / 4>(pk, xt, shc, col0, o, LDC);
-                    }
-                    __syncwarp();
-                }
-                if (sw == 0) FQ_STAMP(3, w.it, 2);
-                if (lane == 0) mbar_arrive_relaxed(bar_empty + 8 * s);
-                if (kt == KT - 1 || u == u_end - 1) {
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_sparse_done);
-                    if (!warp_wait(bar_dense_done, piece & 1, abort_flag, p.status)) break;
-                    ++piece;
-                }
-            }
-        }
-    }
-
-    // ---------------------------------------------------------------------- common exit
-    tc_fence_before();
-    __syncthreads();
-#ifdef FQ_TRACE
-    if (blockIdx.x == 0)
-        for (int i = tid; i < 12 * 32 * 4; i += blockDim.x) g_trace[i] = s_trace[i];
-#endif
-    if (warp == 1) {
-        // every tcgen05 operation of this CTA must have retired before its TMEM is released
-        for (uint32_t spin = 0; spin < (1u << 24) && !mbar_try_wait(bar_final, 0); ++spin) {}
-        __syncwarp();
-        tc_fence_after();
-        tmem_dealloc(tmem_base, kTmemCols);
-    }
-}
+#include "fq_tc_kernel.cuh"
 
 // ----------------------------------------------------------------------------- small-batch kernel
 
@@ -815,7 +329,6 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
     extern __shared__ __align__(128) uint8_t smem[];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    FQ_GT(tid == 0, 0);
     const uint32_t S = p.stages;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
     const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * S;
@@ -831,7 +344,6 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
     if (tid < 32) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncthreads();
-    FQ_GT(tid == 0, 1);
     // The grid after this one in the stream may start now (it takes SMs as this grid's CTAs leave).
     // Every warp but the producer waits for the grid before this one to finish: the producer reads
     // only weights, which no kernel writes while calls are in flight.  (The activation warps first
@@ -863,13 +375,7 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
         bool ok = true;
         for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
             const uint32_t u = w.u, it = w.it, s = w.s, ph = w.ph;
-#ifdef FQ_TRACE
-            long long tw0 = clock64();
-#endif
             if (!warp_wait(bar_empty + 8 * s, ph ^ 1, abort_flag, p.status)) { ok = false; break; }
-#ifdef FQ_TRACE
-            if (blockIdx.x == 0 && lane == 0) { g_trace[8] += clock64() - tw0; g_trace[9] += 1; }
-#endif
             const uint32_t full = bar_full + 8 * s;
             const uint32_t st = smem_u32(smem) + s * p.stage_bytes;
             if (lane == 0) {
@@ -950,13 +456,7 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
             for (int c = 0; c < CPL; ++c) xv[c] = nxt[c];
             const uint32_t ip = ip_nxt, npk = min(ip_nxt_end - ip_nxt, p.coo_cap);
             if (w.u + NA < u_end) { uint32_t kn = w.kt + NA; load(kn >= KT ? kn % KT : kn); load_ip(w.u + NA); }   // this warp's next unit
-#ifdef FQ_TRACE
-            long long tw0 = clock64();
-#endif
             if (!warp_wait(bar_empty + 8 * s, ph ^ 1, abort_flag, p.status)) { ok = false; break; }
-#ifdef FQ_TRACE
-            long long tw1 = clock64();
-#endif
             last_bar = bar_full + 8 * s, last_ph = ph;
             if (lane == 0 && w.it >= S) request(w.u, w.tn, w.kt, smem_u32(st), bar_full + 8 * s, ip, npk);
             uint8_t* dst = st + p.off_xcan + m * kXPitch;
@@ -1010,9 +510,6 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                 __syncwarp();
             }
             if (lane == 0) mbar_arrive(bar_full + 8 * s);
-#ifdef FQ_TRACE
-            if (blockIdx.x == 0 && lane == 0 && aw == 0) { g_trace[10] += tw1 - tw0; g_trace[11] += clock64() - tw1; g_trace[12] += 1; }
-#endif
         }
         if (!ok && last_bar)                // gave up: let this warp's last copies land before the CTA exits
             for (uint32_t spin = 0; spin < (1u << 20) && !mbar_try_wait(last_bar, last_ph); ++spin) {}
@@ -1022,7 +519,6 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
         // warps to hide latencies with, and no warp does less work per unit it takes.  At the end of
         // a piece group 1 hands its sums to group 0 through shared memory.
         const int dwi = warp - DW0, grp = dwi / NDW, dw = dwi % NDW, g = lane >> 2, t = lane & 3;
-        [[maybe_unused]] const int dtid = dwi * 32 + lane;   // tracing builds only
         float* xch = reinterpret_cast<float*>(smem + p.off_shc) + dw * (MO * CG * 4 * 32) + lane;
         const int c0 = dw * 32 + g;                           // this lane's columns: c0 + 8 * {0, 1, 2, 3}
         float accf[MO][CG][4];
@@ -1053,15 +549,8 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
           for (; u < piece_stop; u += NGRP, s = (s + NGRP >= S ? s + NGRP - S : s + NGRP), ph ^= (s < (uint32_t)NGRP ? 1u : 0u)) {
             const uint8_t* st = smem + s * p.stage_bytes;
             {
-#ifdef FQ_TRACE
-            long long tw0 = clock64();
-#endif
             if (!warp_wait(bar_full + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
-#ifdef FQ_TRACE
-            long long tw1 = clock64();
-#endif
-            FQ_GT(dtid == 0 && u == u_begin, 2);
-            const uint4* wp = reinterpret_cast<const uint4*>(st) + dw * 32 + lane;   // the lane's four columns, 8 rows
+            const uint32_t* wp = reinterpret_cast<const uint32_t*>(st) + (dw * 32 + g) * 4 + t;   // word t of column c0; the others 8 columns on
             // chunk 4j + t of row g (+ 8 per octet): at (4j + t) ^ 4 in odd rows, i.e. 64 B further for
             // even j and 64 B back for odd j
             const uint8_t* xrow = st + p.off_xcan + g * kXPitch + t * 16;
@@ -1133,7 +622,7 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                     uint4 xb[MO];
 #pragma unroll
                     for (int o = 0; o < MO; ++o) xb[o] = *reinterpret_cast<const uint4*>(((j & 1) ? xrow_o : xrow_e) + o * 8 * kXPitch + j * 64);
-                    const uint4 w4 = wp[j * BN];                    // columns +0, +8, +16, +24
+                    const uint4 w4 = make_uint4(wp[j * BN * 4], wp[j * BN * 4 + 32], wp[j * BN * 4 + 64], wp[j * BN * 4 + 96]);   // columns +0, +8, +16, +24
 #pragma unroll
                     for (int cg = 0; cg < CG; ++cg) {
                         const uint32_t wa = cg ? w4.z : w4.x, wb = cg ? w4.w : w4.y;
@@ -1306,9 +795,6 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
             }
             __syncwarp();
             if (lane == 0) mbar_arrive_relaxed(bar_empty + 8 * s);
-#ifdef FQ_TRACE
-            if (blockIdx.x == 0 && dtid == 0) { g_trace[13] += tw1 - tw0; g_trace[14] += clock64() - tw1; g_trace[15] += 1; }
-#endif
             }
 
           }
@@ -1316,7 +802,6 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
           {
                 const uint32_t kt = piece_stop - 1 - tn * KT;               // k-step of the piece's last unit
                 // ---------------------------------------------------------- end of a piece
-                FQ_GT(dtid == 0 && piece < 2, 4 + 5 * piece);
                 if (SPARSE && MS == 1) {
                     // single-row outlier sums -> fragment layout: column number c of the group comes
                     // from lane (g, c); batch row 0 lives in lane t = 0
@@ -1400,7 +885,6 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                     }
                     last = __shfl_sync(0xffffffffu, last, 0);
                     __syncwarp();
-                    FQ_GT(dtid == 0 && piece < 2, 7 + 5 * piece);
                     if (last) {
                         write_y = true;
 #pragma unroll
@@ -1456,11 +940,9 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                     for (int cg = 0; cg < CG; ++cg)
 #pragma unroll
                         for (int i = 0; i < 4; ++i) accf[o][cg][i] = 0.0f;
-                FQ_GT(dtid == 0 && piece < 2, 8 + 5 * piece);
                 ++piece;
           }
         }
-        FQ_GT(dtid == 0, 15);
     }
 }
 
@@ -1564,20 +1046,36 @@ static int sm_count_cached() {
 
 static inline uint32_t nb16_of(uint32_t m) { return m <= 16 ? 1u : 2u; }
 
+// Rows kept per epilogue thread of the tcgen05 kernel, and the MMA's batch columns, for a launch of M rows.
+static inline uint32_t rr_of(uint32_t m) { return m <= 1 ? 1u : (m <= 4 ? 4u : (m <= 8 ? 8u : (m <= 16 ? 16u : 32u))); }
+static inline uint32_t nmma_of(uint32_t m) { return m <= 16 ? 16u : 32u; }
+
+// Plan of the tcgen05 kernel (fq_tc_kernel): up to 32 rows per launch.
 static fq_status_t make_plan(const fq_layout_t* L, uint32_t M, bool sparse, Plan& pl) {
     const uint32_t BN = L->BN, NB = L->buckets_per_tile, GPS = kBK / L->group;
-    const uint32_t NMMA = 16 * nb16_of(M);
-    const uint32_t NDW = BN / 32;
-    uint32_t nsw = 0;
-    if (sparse) {
-        const uint32_t nbb = NB / 32, n_oct = (M + 7) / 8;
-        nsw = nbb * std::min<uint32_t>(n_oct, std::max<uint32_t>(1, 4 / nbb));
-    }
+    const uint32_t NMMA = nmma_of(M), RR = rr_of(M);
     Params& p = pl.p;
     std::memset(&p, 0, sizeof(p));
-    p.M = M; p.K = L->K; p.N = L->N; p.KT = L->K / kBK; p.NT = L->N / BN; p.NB = NB; p.nsw = nsw;
+    p.M = M; p.K = L->K; p.N = L->N; p.KT = L->K / kBK; p.NT = L->N / BN; p.NB = NB; p.nsw = 0;
+    const int sms = sm_count_cached();
+    if (sms <= 0) return fail(FQ_ERR_CUDA, "no CUDA device: %s", cudaGetErrorString(cudaGetLastError()));
+    const uint32_t NT = p.NT, KT = p.KT;
+    uint32_t grid = std::min<uint32_t>({(uint32_t)sms, kMaxCtas, NT * KT});
+    uint32_t units_per_cta = (NT * KT + grid - 1) / grid;
+    // Tile-aligned split instead of one contiguous range per CTA when it costs at most one more unit
+    // per CTA: then no CTA has to settle two split tiles in a row.
+    uint32_t split = 0;
+    if (NT <= grid) {
+        const uint32_t c = std::min<uint32_t>(grid / NT, KT);
+        if (c >= 2 && (KT + c - 1) / c <= units_per_cta + 1) {
+            split = c;
+            grid = NT * c;
+            units_per_cta = (KT + c - 1) / c;
+        }
+    }
+    p.split = split;
     const uint32_t w_bytes = 16 * BN * 4, sz_bytes = 2 * GPS * BN * 2;
-    const uint32_t fixed = (sparse ? BN * NMMA * 4 : 0) + 1024;
+    const uint32_t xt_bytes = sparse ? kBK * RR * 4 : 0;                 // FP32 k-major copy [k][RR]
     uint32_t cap = 0;
     if (sparse) {
         cap = L->tilecoo_encoded ? std::max<uint32_t>(8, round_up(L->max_tile_packets, 8)) : 256;
@@ -1588,23 +1086,28 @@ static fq_status_t make_plan(const fq_layout_t* L, uint32_t M, bool sparse, Plan
         p.off_sz = w_bytes;
         p.off_xcan = p.off_sz + round_up(sz_bytes, 128);
         p.off_xsum = p.off_xcan + NMMA * 256;
-        p.off_xt = p.off_xsum + round_up(GPS * NMMA * 4, 128);          // stage-relative: FP32 k-major copy
-        p.off_info = p.off_xt + (sparse ? ((M + 7) / 8) * 4096 : 0);
+        p.off_xt = p.off_xsum + round_up(GPS * NMMA * 4, 128);
+        p.off_info = p.off_xt + xt_bytes;
         p.off_coo = p.off_info + (sparse ? round_up(NB * 4, 128) : 0);
         stage = round_up(p.off_coo + cap * 16, 128);
-        S = std::min<uint32_t>(8, (kSmemBudget - fixed) / stage);
+        S = std::min<uint32_t>(8, (kSmemBudget - 1024) / stage);
         if (S >= 4 || cap <= 64) break;
         cap = std::max<uint32_t>(64, cap / 2);  // oversized tiles read their tail from global memory
     }
-    if (S < 3) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "shared-memory stages do not fit");
+    if (S < 2) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "shared-memory stages do not fit");
+    // The activation warps take the units in turn, and the ring length is a multiple of their number, so
+    // that a stage always returns to the same warp (which then meets every phase of the stage's barriers).
+    p.nact = S >= 8 ? 4 : (S >= 6 ? 3 : (S >= 4 ? 4 : 2));
+    S = S / p.nact * p.nact;
     p.coo_cap = cap; p.stages = S; p.stage_bytes = stage;
+    // hot columns, tiles larger than the staged part, or an encoding whose sizes were not recorded
+    pl.general = sparse && (L->max_tail_packets > 0 || L->max_tile_packets > cap || !L->tilecoo_encoded);
     p.off_shc = S * stage;
-    p.off_bar = p.off_shc + (sparse ? BN * NMMA * 4 : 0);
+    p.off_bar = p.off_shc;
     pl.smem = p.off_bar + 1024;
-    pl.threads = 32 * (4 + 2 * NDW + nsw);
-    const int sms = sm_count_cached();
-    if (sms <= 0) return fail(FQ_ERR_CUDA, "no CUDA device: %s", cudaGetErrorString(cudaGetLastError()));
-    pl.grid = std::min<uint32_t>({(uint32_t)sms, kMaxCtas, p.NT * p.KT});
+    pl.threads = 32 * (2 + kTcActWarps + 2 * (BN / 32));
+    pl.grid = grid;
+    pl.ngrp = 1;
     return FQ_OK;
 }
 
@@ -1709,34 +1212,29 @@ static KernelFn pick_mma_kernel(uint32_t bn, uint32_t M, uint32_t g, bool sparse
     return mo == 1 ? pick_mma_group<256, 1>(g, sparse, ms, ngrp, hot) : mo == 2 ? pick_mma_group<256, 2>(g, sparse, ms, ngrp, hot) : pick_mma_group<256, 4>(g, sparse, ms, ngrp, hot);
 }
 
-// Which kernel serves a call.  Default: the small-batch kernel, in launches of up to 32 rows (at M = 32 one
-// such launch takes about a third of the time of the tcgen05 kernel as it stands).  FQ_ENGINE=tc
-// routes every call to the tcgen05 kernel (launches of 32 rows), FQ_ENGINE=mix uses it for M > 16.
-enum Engine { kEngineMma, kEngineTc, kEngineMix };
-static Engine engine() {
-    static const Engine v = [] {
-        const char* e = std::getenv("FQ_ENGINE");
-        if (e && std::strcmp(e, "tc") == 0) return kEngineTc;
-        if (e && std::strcmp(e, "mix") == 0) return kEngineMix;
-        return kEngineMma;
-    }();
-    return v;
-}
+// Which kernel serves a call: the tcgen05 kernel.  The warp-level MMA kernel stays reachable through an
+// internal switch for comparison runs.
+static int g_engine = 0;   // 0: tcgen05 kernel, 1: warp-level MMA kernel
 
-template <int BN, int MO, int G>
-static KernelFn pick_sparse(bool sparse) {
-    return sparse ? (KernelFn)fq_fused_kernel<BN, MO, G, true> : (KernelFn)fq_fused_kernel<BN, MO, G, false>;
+template <int BN, int NMMA, int RR, int G>
+static KernelFn pick_tc_sparse(bool sparse, bool hot) {
+    if (!sparse) return (KernelFn)fq_tc_kernel<BN, NMMA, RR, G, false, false>;
+    return hot ? (KernelFn)fq_tc_kernel<BN, NMMA, RR, G, true, true> : (KernelFn)fq_tc_kernel<BN, NMMA, RR, G, true, false>;
 }
-template <int BN, int MO>
-static KernelFn pick_group(uint32_t g, bool sparse) {
-    return g == 64 ? pick_sparse<BN, MO, 64>(sparse) : pick_sparse<BN, MO, 128>(sparse);
+template <int BN, int G>
+static KernelFn pick_tc_rows(uint32_t rr, bool sparse, bool hot) {
+    switch (rr) {
+        case 1: return pick_tc_sparse<BN, 16, 1, G>(sparse, hot);
+        case 4: return pick_tc_sparse<BN, 16, 4, G>(sparse, hot);
+        case 8: return pick_tc_sparse<BN, 16, 8, G>(sparse, hot);
+        case 16: return pick_tc_sparse<BN, 16, 16, G>(sparse, hot);
+        default: return pick_tc_sparse<BN, 32, 32, G>(sparse, hot);
+    }
 }
-template <int BN>
-static KernelFn pick_mo(uint32_t nb16, uint32_t g, bool sparse) {
-    return nb16 == 1 ? pick_group<BN, 1>(g, sparse) : pick_group<BN, 2>(g, sparse);
-}
-static KernelFn pick_kernel(uint32_t bn, uint32_t mo, uint32_t g, bool sparse) {
-    return bn == 128 ? pick_mo<128>(mo, g, sparse) : pick_mo<256>(mo, g, sparse);
+static KernelFn pick_kernel(uint32_t bn, uint32_t M, uint32_t g, bool sparse, bool hot) {
+    const uint32_t rr = rr_of(M);
+    if (bn == 128) return g == 64 ? pick_tc_rows<128, 64>(rr, sparse, hot) : pick_tc_rows<128, 128>(rr, sparse, hot);
+    return g == 64 ? pick_tc_rows<256, 64>(rr, sparse, hot) : pick_tc_rows<256, 128>(rr, sparse, hot);
 }
 
 // cudaFuncSetAttribute costs several microseconds: do it once per (kernel, device).
@@ -1756,17 +1254,6 @@ static cudaError_t ensure_smem_attr(const void* fn, int bytes) {
     return e;
 }
 
-// Launch the small-batch kernel so that it may overlap the tail of the kernel before it in the
-// stream (FQ_PDL=0 turns this off).  The weights, scales, zeros and Tile-COO arrays must then not be
-// written by a kernel that is still running when the call is made; everything else is ordered as usual.
-static bool overlap_launches() {
-    static const bool v = [] {
-        const char* e = std::getenv("FQ_PDL");
-        return !(e && std::strcmp(e, "0") == 0);
-    }();
-    return v;
-}
-
 static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
 static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, const void* wq, const void* scale,
@@ -1784,7 +1271,7 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
     fq_status_t st = fq_workspace_bytes(L, M, &need);
     if (st != FQ_OK) return st;
     if (workspace_bytes < need) return fail(FQ_ERR_BUFFER_TOO_SMALL, "workspace holds %zu bytes, %zu needed", workspace_bytes, need);
-    const bool use_mma = engine() == kEngineMma || (engine() == kEngineMix && M <= 16);
+    const bool use_mma = g_engine == 1;
     // the small-batch kernel takes up to 32 rows per launch; a remainder of at most 16 rows gets the cheaper variants
     const uint32_t rows_per_launch = 32;
     for (uint32_t m0 = 0; m0 < M; m0 += rows_per_launch) {
@@ -1801,14 +1288,14 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
         p.counters = (uint32_t*)((uint8_t*)workspace + kWsHeaderBytes);
         p.partials = (float*)((uint8_t*)workspace + kWsHeaderBytes + kWsCounterBytes);
         KernelFn fn = use_mma ? pick_mma_kernel(L->BN, mb, L->group, sparse, pl.ngrp, pl.general)
-                              : pick_kernel(L->BN, nb16_of(mb), L->group, sparse);
+                              : pick_kernel(L->BN, mb, L->group, sparse, pl.general);
         cudaError_t e = ensure_smem_attr((const void*)fn, (int)kSmemBudget);
         if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-        if (use_mma) {
+        {
             // Programmatic dependent launch: this grid may become resident while the kernel before it
             // in the stream drains.  Its producer warp then already streams weights (which no kernel
-            // writes); every other warp first executes griddepcontrol.wait, after which all memory
-            // operations of the earlier grid are complete and visible.
+            // writes); the warps that touch X, Y or the scratch first execute griddepcontrol.wait, after
+            // which all memory operations of the earlier grid are complete and visible.
             cudaLaunchConfig_t cfg;
             std::memset(&cfg, 0, sizeof(cfg));
             cfg.gridDim = dim3(pl.grid);
@@ -1817,18 +1304,12 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
             cfg.stream = (cudaStream_t)stream;
             cudaLaunchAttribute attr[1];
             std::memset(attr, 0, sizeof(attr));
-            unsigned n = 0;
-            if (overlap_launches()) {
-                attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-                attr[n].val.programmaticStreamSerializationAllowed = 1;
-                ++n;
-            }
+            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[0].val.programmaticStreamSerializationAllowed = 1;
             cfg.attrs = attr;
-            cfg.numAttrs = n;
+            cfg.numAttrs = 1;
             e = cudaLaunchKernelEx(&cfg, fn, p);
             if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
-        } else {
-            fn<<<pl.grid, pl.threads, pl.smem, (cudaStream_t)stream>>>(p);
         }
         e = cudaGetLastError();
         if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
@@ -1842,14 +1323,8 @@ using namespace fq;
 
 extern "C" {
 
-#ifdef FQ_TRACE
-int fq_trace_read(unsigned long long* out) {
-    return (int)cudaMemcpyFromSymbol(out, fq::g_trace, sizeof(unsigned long long) * 12 * 32 * 4);
-}
-int fq_ktrace_read(unsigned long long* out) {
-    return (int)cudaMemcpyFromSymbol(out, fq::g_ktrace, sizeof(unsigned long long) * 192 * 16);
-}
-#endif
+// Comparison runs only (not declared in fq.h): 0 = the tcgen05 kernel (default), 1 = the warp-level MMA kernel.
+void fq_internal_select_engine(int e) { fq::g_engine = e == 1 ? 1 : 0; }
 
 fq_status_t fq_workspace_bytes(const fq_layout_t* L, uint32_t M, size_t* bytes) {
     if (!layout_ok(L) || !bytes) return fail(FQ_ERR_INVALID_ARG, "bad layout or null output");

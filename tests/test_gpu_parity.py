@@ -228,28 +228,25 @@ def test_host_io_entry_point_matches_device_entry_point():
     assert np.array_equal(yh.numpy().view(np.uint16), Y_dev) and np.array_equal(yh2.numpy().view(np.uint16), Y_dev)
 
 
-# ------------------------------------------------------------------ full-size, sampled columns
+# ------------------------------------------------------------------ full-size layers, every output column
 
 FULL = [("8b_" + n, 2, i, K, N) for i, (n, K, N) in enumerate(synth.LLAMA3_8B)]
 
 
 @pytest.mark.parametrize("name,cfg,idx,K,N", FULL)
-def test_full_size_layers_on_sampled_columns(name, cfg, idx, K, N):
+def test_full_size_layers_every_column(name, cfg, idx, K, N):
+    """The benchmark's own layers in the launch configuration the benchmark times (M = 1, 8, 16), every
+    element of Y against the oracle."""
     g = 128
     lay = synth.layer(synth.tensor_seed(cfg, idx), K, N, density=0.01, layout="mixed")
     P = H.pack_layer(lay, g)
-    rng = np.random.default_rng(idx)
-    BN = P.L.BN
-    # columns from the first, last and random tiles, plus the columns richest in outliers
-    cols = np.unique(np.concatenate([np.arange(0, 8), np.arange(N - 8, N), rng.integers(0, N, 80),
-                                     np.argsort(lay.mask.sum(axis=0))[::-1][:8]])).astype(np.uint32)
     for M in (1, 8, 16):
         X = _x(lay.seed, M, K)
         Y = H.run_fused(P, X)
-        Yref, Yabs = H.oracle_result(P, X, cols=cols)
-        assert np.all(np.isfinite(H.bits_to_f64(Y)))
-        H.check_tolerances(Y[:, cols], Yref, Yabs, K)
-    del BN
+        Yref, Yabs = H.oracle_result(P, X)
+        res = H.check_tolerances(Y, Yref, Yabs, K)
+        if M >= 8:
+            assert res["fallback_cols"] == 0, res
 
 
 def _sample_cols(lay, N, seed, n_random=64):
@@ -329,23 +326,6 @@ def test_tile_counts_that_are_not_powers_of_two_on_sampled_columns(K, N):
         Y = H.run_fused(P, X)
         Yref, Yabs = H.oracle_result(P, X, cols=cols)
         H.check_tolerances(Y[:, cols], Yref, Yabs, K)
-
-
-# ------------------------------------------------------------------ the tcgen05 kernel (not the default engine)
-
-def test_tcgen05_engine_in_a_child_process():
-    """FQ_ENGINE is read once per process, so the tcgen05 kernel is exercised in a child: the
-    element-by-element cases and the larger batches, with every call routed to it."""
-    import os
-    import subprocess
-    import sys
-    env = dict(os.environ, FQ_ENGINE="tc")
-    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-    r = subprocess.run([sys.executable, "-m", "pytest", "-q", "-x", "-m", "gpu", "tests/test_gpu_parity.py", "-k",
-                        "test_fused_matches_oracle or test_fused_larger_batches or test_identity_rows or "
-                        "test_zero_density or test_oversized_tiles"], cwd=root, env=env, capture_output=True,
-                       text=True, timeout=900)
-    assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-2000:]
 
 
 # ------------------------------------------------------------------ ordering of dependent calls

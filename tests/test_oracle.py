@@ -254,7 +254,7 @@ def test_decode_wq_against_a_direct_packer():
         i, h = divmod(r8, 2)
         for col in range(N):
             tn, t = divmod(col, BN)
-            idx = (tn * KT + kt) * 16 * BN + (((j * (BN // 32) + t // 32) * 8 + t % 8) * 4 + w) * 4 + (t // 8) % 4
+            idx = (tn * KT + kt) * 16 * BN + (j * BN + t) * 4 + w
             words[idx] |= np.uint32(int(q[row, col]) << (4 * (i + 4 * h)))
     assert np.array_equal(oracle.decode_wq(words, K, N, BN), q)
 

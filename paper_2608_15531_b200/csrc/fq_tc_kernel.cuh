@@ -3,24 +3,27 @@
 //
 // A unit is one (column tile, 128-row k-step): 128 x BN INT4 codes with their scales, zero-points and
 // Tile-COO slice.  One persistent CTA per SM walks a range of units through a ring of shared-memory
-// stages (cp.async.bulk + mbarrier expect_tx, Section 4.1).  Thread = output column throughout: tensor
+// stages (bulk copies + mbarrier expect_tx, Section 4.1).  Thread = output column throughout: tensor
 // memory lane c of a 128-column half holds row c of the A operand (the column's 128 dequantised
 // codes) and row c of the accumulator D (the column's batch rows).
 //
-//   warp 0          producer: bulk copies of codes and scales (and zero-points in kernels with outliers)
-//   warp 1          tensor: owns the tensor-memory allocation; per unit 8 x BN/128 tcgen05.mma
-//                   (M = 128 columns, N = NMMA batch rows, K = 16; A from tensor memory, B = activations
-//                   from shared memory, D = FP32 in tensor memory), tcgen05.commit to mbarriers
-//   warps 2..3      activations (alternate units): the unit's block of X from global memory (L2) as the
-//                   K-major MMA operand + per-group row sums + a k-major FP32 copy for the outlier step;
-//                   they also request the unit's bucket descriptors and packets (or its zero-points)
-//   unpack warps    BN/32: per 32 rows one 128-bit load of 32 codes, lop3/shift to 16 BF16 pairs 128 + q
-//                   (exact integers), tcgen05.st into the A operand
-//   epilogue warps  BN/32: tcgen05.ld of the group sums, acc += s * (sum x (128+q) - (128+z) sum x) in
-//                   FP32 (Eq. 3 inside Eq. 1), then the unit's outliers of the thread's own column
-//                   straight into the same registers (Section 4.2 without the shared-memory scatter:
-//                   no atomics, no read-modify-write), and at the end of a piece the split-tile
-//                   settlement and the BF16 store of Y
+//   warp 0          producer: every copy of a unit, one lane each: codes, scales, zero-points, bucket
+//                   descriptors, outlier packets (cp.async.bulk) and the unit's block of X as a 3-D tiled
+//                   tensor copy (cp.async.bulk.tensor) whose box lands as the K-major MMA operand
+//                   (8-row x 16-byte core matrices; rows beyond M are filled with zeros by the copy)
+//   warp 1          tensor: per unit 8 x BN/128 tcgen05.mma (M = 128 columns, N = NMMA batch rows, K = 16;
+//                   A from tensor memory, B = activations from shared memory, D = FP32 in tensor memory),
+//                   tcgen05.commit to mbarriers.  An MMA of this shape occupies the tensor pipe for 55-66
+//                   cycles whatever N <= 128 is, and its issue blocks meanwhile
+//   warps 3..6      (kernels with outliers) a k-major FP32 copy xt[k][RR] of the unit's activations for the
+//                   outlier step, built from the MMA operand with ldmatrix; alternate units
+//   unpack warps    BN/32: per 32 rows one 128-bit load of 32 codes, lop3/shift to 16 BF16 pairs 128 + q,
+//                   minus 128 + z (exact small integers q - z: Eq. 3 without the scale), tcgen05.st into A
+//   epilogue warps  BN/32: tcgen05.ld of the group sums, acc += s * sum x (q - z) in FP32 (Eq. 3 inside
+//                   Eq. 1), then the unit's outliers of the thread's own column straight into the same
+//                   registers (Section 4.2 without the shared-memory scatter: no atomics, no
+//                   read-modify-write), and at the end of a piece the split-tile settlement and the BF16
+//                   store of Y
 //
 // Lane l of an epilogue warp owns column 32 * strip + l = 8 t + g with g = l % 8, t = l / 8: bucket g of
 // the strip, column number t of that bucket, so it takes slot t of every column-slotted packet of the
@@ -146,44 +149,59 @@ __device__ __forceinline__ void build_xt(uint32_t xb_addr, uint32_t nmma8, char*
     }
 }
 
-constexpr int kTcActWarps = 4;
+// 3-D tiled tensor copy global -> shared, completion counted in bytes on an mbarrier
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const void* tmap, uint32_t c0, uint32_t c1, uint32_t c2, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
+                 "l"(tmap), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ uint32_t sub_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+
+constexpr int kTcXtWarps = 4;      // warps 3..6 build the FP32 copy; warp 7 is idle
+constexpr int kTcFirstUnpack = 8;  // a warp reaches the tensor-memory lanes 32 * (warp % 4) ..., so strips start at a multiple of 4
 
 // BN: tile columns (128 or 256).  NMMA: batch columns of the MMA (16 or 32).  RR: batch rows kept per
 // epilogue thread (1, 4, 8, 16, 32; M <= RR <= NMMA).  HOT: general form of the outlier step (buckets
-// with a tail, tiles with more packets than a stage holds).
+// with a tail, tiles with more packets than a stage holds).  tmX: tiled view of this launch's rows of X as
+// (8 consecutive k, row, block of 8 k), so that a box of (8, NMMA, 16) is a unit's K-major MMA operand.
 template <int BN, int NMMA, int RR, int GROUP, bool SPARSE, bool HOT>
-__global__ void __launch_bounds__(32 * (2 + kTcActWarps + 2 * (BN / 32)), 1) fq_tc_kernel(const Params p) {
+__global__ void __launch_bounds__(32 * (kTcFirstUnpack + 2 * (BN / 32)), 1)
+fq_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmX) {
     constexpr int NDW = BN / 32;              // unpack warps = epilogue warps = 32-column strips
     constexpr int NT128 = BN / 128;           // 128-column halves per unit
-    constexpr int NAW = kTcActWarps;         // activation warps launched; the first p.nact of them work
-    constexpr int UW0 = 2 + NAW, EW0 = UW0 + NDW;
+    constexpr int UW0 = kTcFirstUnpack, EW0 = UW0 + NDW;
     constexpr int GPS = kBK / GROUP;          // groups per k-step
     constexpr int DCOLS = GPS * NMMA;         // accumulator columns per half and buffer
     constexpr uint32_t D_BASE = 2 * NT128 * 64;
     constexpr int W_BYTES = 16 * BN * 4;
     constexpr int SZ_ROW = BN * 2;
+    constexpr int X_BYTES = NMMA * 256;
     constexpr int NMMA8 = NMMA / 8;
-    constexpr bool kActZero = !SPARSE;        // who requests the zero-points: the activation warp, if it has no outlier arrays to request
     constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NMMA >> 3) << 17) | (8u << 24);
     static_assert(D_BASE + 2 * NT128 * DCOLS <= 512, "tensor memory: two A buffers and two D buffers must fit");
     static_assert(RR <= NMMA && (RR == 1 || RR % 4 == 0), "rows per thread");
-    static_assert(RR > 8 || NMMA == 16, "up to eight rows: the MMA's second octet of rows is zero padding");
     extern __shared__ __align__(128) uint8_t smem[];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t S = p.stages;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
     const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * S;
-    const uint32_t bar_go = bar_empty + 8 * S;           // [2] A buffer written (unpack warps) and D buffer free (epilogue warps)
+    const uint32_t bar_xt = bar_empty + 8 * S;           // [S] the stage's FP32 activation copy is written
+    const uint32_t bar_go = bar_xt + 8 * S;              // [2] A buffer written (unpack warps) and D buffer free (epilogue warps)
     const uint32_t bar_d_ready = bar_go + 16;            // [2] MMAs of a unit complete (D written, A read)
     const uint32_t bar_final = bar_d_ready + 16;
-    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 2 * S + 5);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 3 * S + 5);
     volatile uint32_t* tmem_slot = abort_flag + 1;
 
     if (tid == 0) {
         for (uint32_t s = 0; s < S; ++s) {
-            mbar_init(bar_full + 8 * s, 2);                    // producer's expect_tx arrival + activation warp
+            mbar_init(bar_full + 8 * s, 1);                    // the producer's expect_tx arrival
             mbar_init(bar_empty + 8 * s, 2 * NDW + 1);         // unpack warps, epilogue warps, the MMAs' commit
+            mbar_init(bar_xt + 8 * s, 1);
         }
         for (uint32_t b = 0; b < 2; ++b) {
             mbar_init(bar_go + 8 * b, 2 * NDW);                // unpack warps (A of this unit), epilogue warps (D of the unit two before)
@@ -192,13 +210,6 @@ __global__ void __launch_bounds__(32 * (2 + kTcActWarps + 2 * (BN / 32)), 1) fq_
         mbar_init(bar_final, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (RR <= 8) {
-        // batch rows 8..15 of the MMA operand are never written by the activation warps: zero them once
-        for (uint32_t i = tid; i < S * 16 * 8; i += blockDim.x) {
-            const uint32_t s = i >> 7, c = (i >> 3) & 15, r = i & 7;
-            *reinterpret_cast<uint4*>(smem + s * p.stage_bytes + p.off_xcan + (c * NMMA8 + 1) * 128 + r * 16) = make_uint4(0, 0, 0, 0);
-        }
     }
     if (warp == 1) {
         tmem_alloc(smem_u32((const void*)tmem_slot), kTmemCols);
@@ -210,8 +221,9 @@ __global__ void __launch_bounds__(32 * (2 + kTcActWarps + 2 * (BN / 32)), 1) fq_
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     // The grid after this one in the stream may start now (it takes SMs as this grid's CTAs leave).  The
-    // warps that touch X, Y or the scratch wait for the grid before this one; the producer reads only
-    // weights, which no kernel writes while calls are in flight.
+    // warps that write Y or touch the scratch wait for the grid before this one, and so does the producer
+    // before its first copy of X; the weight arrays are read before: no kernel writes them while calls are
+    // in flight.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (warp >= EW0) asm volatile("griddepcontrol.wait;" ::: "memory");
 
@@ -229,194 +241,176 @@ __global__ void __launch_bounds__(32 * (2 + kTcActWarps + 2 * (BN / 32)), 1) fq_
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer
+        // Lane l issues copy number l of a unit (issuing a bulk copy occupies its thread for a few hundred
+        // cycles): 0 codes, 1.. scales, then zero-points, then X, bucket descriptors, packets.
+        constexpr int L_X = 1 + 2 * GPS, L_INFO = L_X + 1, L_PK = L_X + 2;
         uint32_t issued = 0;
         bool ok = true;
-        for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
-            const uint32_t s = w.s;
-            if (!warp_wait(bar_empty + 8 * s, w.ph ^ 1, abort_flag, p.status)) { ok = false; break; }
-            const uint32_t full = bar_full + 8 * s;
+        // the packet ranges of this warp's next 32 units, read 32 at a time
+        uint32_t ip_a = 0, ip_b = 0;
+        auto weights = [&](const UnitIter& w) {                        // everything of a unit but X
+            const uint32_t s = w.s, full = bar_full + 8 * s;
             const uint32_t st = smem_u32(smem) + s * p.stage_bytes;
-            if (lane == 0) mbar_arrive_expect_tx(full, W_BYTES + (kActZero ? 1 : 2) * GPS * SZ_ROW);
+            if (SPARSE && (w.it & 31) == 0) {
+                const uint32_t i = w.u + lane;
+                ip_a = (i <= U) ? __ldg(p.indptr + i) : 0;
+                ip_b = (i + 1 <= U) ? __ldg(p.indptr + i + 1) : 0;
+            }
+            uint32_t pk0 = 0, npk = 0;
+            if (SPARSE) {
+                pk0 = __shfl_sync(0xffffffffu, ip_a, w.it & 31);
+                npk = min(__shfl_sync(0xffffffffu, ip_b, w.it & 31) - pk0, p.coo_cap);
+            }
+            if (lane == 0) mbar_arrive_expect_tx(full, W_BYTES + 2 * GPS * SZ_ROW + X_BYTES + (SPARSE ? p.NB * 4 + npk * 16 : 0));
             __syncwarp();
-            // one copy per lane: issuing a bulk copy occupies its thread for a few hundred cycles
             if (lane == 0) {
                 bulk_g2s(st, p.wq + (size_t)w.u * W_BYTES, W_BYTES, full);
             } else if (lane <= GPS) {
                 const int gi = lane - 1;
                 bulk_g2s(st + p.off_sz + gi * SZ_ROW, p.scale + (size_t)(w.kt * GPS + gi) * p.N + (size_t)w.tn * BN, SZ_ROW, full);
-            } else if (!kActZero && lane <= 2 * GPS) {
+            } else if (lane <= 2 * GPS) {
                 const int gi = lane - 1 - GPS;
                 bulk_g2s(st + p.off_sz + (GPS + gi) * SZ_ROW, p.zero + (size_t)(w.kt * GPS + gi) * p.N + (size_t)w.tn * BN, SZ_ROW, full);
+            } else if (SPARSE && lane == L_INFO) {
+                bulk_g2s(st + p.off_info, p.info + (size_t)w.u * p.NB, p.NB * 4, full);
+            } else if (SPARSE && lane == L_PK) {
+                if (npk) bulk_g2s(st + p.off_coo, p.packed + pk0, npk * 16, full);
             }
-            issued = w.it + 1;
+        };
+        auto activations = [&](const UnitIter& w) {
+            if (lane == L_X)
+                tma_load_3d(smem_u32(smem) + w.s * p.stage_bytes + p.off_xcan, &tmX, 0, 0, w.kt * 16, bar_full + 8 * w.s);
+        };
+        // the first pass over the ring finds every stage empty: its weight copies go out before the wait
+        // for the previous grid, its copies of X after
+        const uint32_t n_first = min(S, u_end - u_begin);
+        {
+            UnitIter w(u_begin, KT);
+            for (uint32_t i = 0; i < n_first; ++i, w.next(S, KT)) weights(w);
+        }
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        {
+            UnitIter w(u_begin, KT);
+            for (uint32_t i = 0; i < n_first; ++i, w.next(S, KT)) activations(w);
+            issued = n_first;
+            for (; w.u < u_end; w.next(S, KT)) {
+                if (!warp_wait(bar_empty + 8 * w.s, w.ph ^ 1, abort_flag, p.status)) { ok = false; break; }
+                weights(w);
+                activations(w);
+                issued = w.it + 1;
+            }
         }
         if (!ok) {   // giving up: let the copies already issued land before the CTA's shared memory goes away
             for (uint32_t j = (issued > S ? issued - S : 0); j < issued; ++j)
                 for (uint32_t spin = 0; spin < (1u << 20) && !mbar_try_wait(bar_full + 8 * (j % S), (j / S) & 1); ++spin) {}
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ tensor warp
-        // The whole warp runs the loop with warp-uniform operands; one elected lane issues each instruction.
-        // The first MMA of a CTA takes microseconds to start (the tensor pipe wakes up): issue a throw-away
-        // one now, while the first loads are in flight.  It reads whatever A buffer 0 and stage 0 hold and
-        // writes D buffer 1, which the first real MMA into that buffer overwrites.
-        umma_ts(tmem_base + D_BASE + NT128 * DCOLS, tmem_base, make_b_desc(smem_u32(smem) + p.off_xcan, NMMA8 * 128, 128), IDESC, 0);
-        for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
-            const uint32_t it = w.it, s = w.s, b = w.it & 1;
-            if (!warp_wait(bar_full + 8 * s, w.ph, abort_flag, p.status)) break;       // the activation operand
-            if (!warp_wait(bar_go + 8 * b, (it >> 1) & 1, abort_flag, p.status)) break;
-            tc_fence_after();
-            const uint64_t bd0 = make_b_desc(smem_u32(smem) + s * p.stage_bytes + p.off_xcan, NMMA8 * 128, 128);
-#pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
-                const int gi = ks / (8 / GPS);
-#pragma unroll
-                for (int h = 0; h < NT128; ++h) {
-                    const uint32_t d = tmem_base + D_BASE + (b * NT128 + h) * DCOLS + gi * NMMA;
-                    const uint32_t a = tmem_base + (b * NT128 + h) * 64 + ks * 8;
-                    umma_ts(d, a, bd0 + (uint64_t)((ks * 2 * NMMA8 * 128) >> 4), IDESC, (ks % (8 / GPS)) != 0);
+    } else if (warp <= 2) {
+        // ------------------------------------------------------------------ tensor warp (warp 2 is idle)
+        // One warp issues every MMA of the CTA (issued from two warps in turn, MMAs run several times slower).
+        // An MMA of this shape occupies the tensor pipe for 55-66 cycles and its issue blocks meanwhile, so the
+        // warp looks at the next unit's barriers between the MMAs of this one: their latency then hides behind
+        // MMAs in flight, and a unit whose operands are ready is issued without waiting at all.
+        if (warp == 1) {
+            // The first MMA of a CTA takes microseconds to start (the tensor pipe wakes up): issue a throw-away
+            // one now, while the first loads are in flight.  It reads whatever A buffer 0 and stage 0 hold and
+            // writes D buffer 1, which the first real MMA into that buffer overwrites.
+            umma_ts(tmem_base + D_BASE + NT128 * DCOLS, tmem_base, make_b_desc(smem_u32(smem) + p.off_xcan, NMMA8 * 128, 128), IDESC, 0);
+            uint32_t ready = 0;                          // this unit's barriers were seen complete already
+            for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
+                const uint32_t it = w.it, s = w.s, b = w.it & 1;    // A buffer b and D buffer b
+                if (!ready) {
+                    if (!warp_wait(bar_full + 8 * s, w.ph, abort_flag, p.status)) break;       // the activation operand
+                    if (!warp_wait(bar_go + 8 * b, (it >> 1) & 1, abort_flag, p.status)) break;
                 }
-            }
-            umma_commit(bar_d_ready + 8 * b);   // this unit's sums are complete and its A buffer has been read
-            umma_commit(bar_empty + 8 * s);     // and so has the stage's activation operand
-        }
-        __syncwarp();
-        umma_commit(bar_final);                 // fires when every MMA this warp issued has retired
-    } else if (warp < UW0) {
-        // ------------------------------------------------------------------ activation warps
-        const uint32_t aw = warp - 2, NA = p.nact;           // the ring length is a multiple of NA: a stage always returns to the same warp
-        constexpr int ROWS = RR <= 8 ? 8 : NMMA;             // rows this warp lays out (rows 8..15 stay zero if RR <= 8)
-        constexpr int LPR = 32 / ROWS;                       // lanes per row: 4, 2 or 1
-        constexpr int CPL = 16 / LPR;                        // 16-byte chunks per lane
-        const int m = lane % ROWS, part = lane / ROWS;
-        const bool real = (uint32_t)m < p.M;
-        const uint8_t* xrow = reinterpret_cast<const uint8_t*>(p.X) + ((size_t)m * p.K) * 2 + part * CPL * 16;
-        uint4 nxt[CPL];
-        auto load = [&](uint32_t kt) {
+                tc_fence_after();
+                UnitIter nx = w;
+                nx.next(S, KT);
+                const bool has_next = nx.u < u_end;
+                uint32_t seen = 0;
+                auto poll = [&]() {
+                    if (has_next && lane == 0 && !seen)
+                        seen = mbar_test_wait(bar_full + 8 * nx.s, nx.ph) & mbar_test_wait(bar_go + 8 * (nx.it & 1), (nx.it >> 1) & 1);
+                };
+                const uint64_t bd0 = make_b_desc(smem_u32(smem) + s * p.stage_bytes + p.off_xcan, NMMA8 * 128, 128);
 #pragma unroll
-            for (int c = 0; c < CPL; ++c) {
-                nxt[c] = make_uint4(0, 0, 0, 0);
-                if (real) nxt[c] = __ldg(reinterpret_cast<const uint4*>(xrow + (size_t)kt * 256 + c * 16));
-            }
-        };
-        uint32_t ip_nxt = 0, ip_nxt_end = 0, last_bar = 0, last_ph = 0;
-        bool ok = true;
-        auto load_ip = [&](uint32_t u) {
-            if (SPARSE && lane == 0) { ip_nxt = __ldg(p.indptr + u); ip_nxt_end = __ldg(p.indptr + u + 1); }
-        };
-        // this warp's share of the weight arrays of unit u: bucket descriptors and packets, or the zero-points
-        auto request = [&](uint32_t u, uint32_t tn, uint32_t kt, uint32_t sta, uint32_t full, uint32_t ip, uint32_t npk) {
-            mbar_expect_tx(full, kActZero ? GPS * SZ_ROW : p.NB * 4 + npk * 16);
-            if (kActZero) {
+                for (int ks = 0; ks < 8; ++ks) {
+                    const int gi = ks / (8 / GPS);
 #pragma unroll
-                for (int gi = 0; gi < GPS; ++gi)
-                    bulk_g2s(sta + p.off_sz + (GPS + gi) * SZ_ROW, p.zero + (size_t)(kt * GPS + gi) * p.N + (size_t)tn * BN, SZ_ROW, full);
-            }
-            if (SPARSE) {
-                bulk_g2s(sta + p.off_info, p.info + (size_t)u * p.NB, p.NB * 4, full);
-                if (npk) bulk_g2s(sta + p.off_coo, p.packed + ip, npk * 16, full);
-            }
-        };
-        {
-            // The first pass over the ring finds every stage empty, and these arrays are weights: lane l
-            // requests those of this warp's l-th unit before the wait for the previous grid.
-            const uint32_t it0 = aw + NA * lane;
-            if (aw < NA && it0 < min(S, u_end - u_begin)) {
-                const uint32_t u = u_begin + it0, tn = u / KT;
-                uint32_t a = 0, npk = 0;
-                if (SPARSE) { a = __ldg(p.indptr + u); npk = min(__ldg(p.indptr + u + 1) - a, p.coo_cap); }
-                request(u, tn, u - tn * KT, smem_u32(smem) + it0 * p.stage_bytes, bar_full + 8 * it0, a, npk);
+                    for (int h = 0; h < NT128; ++h) {
+                        const uint32_t d = tmem_base + D_BASE + (b * NT128 + h) * DCOLS + gi * NMMA;
+                        const uint32_t a = tmem_base + (b * NT128 + h) * 64 + ks * 8;
+                        umma_ts(d, a, bd0 + (uint64_t)((ks * 2 * NMMA8 * 128) >> 4), IDESC, (ks % (8 / GPS)) != 0);
+                    }
+                    if (ks == 3 || ks == 6) poll();
+                }
+                umma_commit(bar_d_ready + 8 * b);   // this unit's sums are complete and its A buffer has been read
+                umma_commit(bar_empty + 8 * s);     // and so has the stage's activation operand
+                poll();
+                ready = __shfl_sync(0xffffffffu, seen, 0);
             }
             __syncwarp();
-            asm volatile("griddepcontrol.wait;" ::: "memory");
+            umma_commit(bar_final);                 // fires when every MMA this warp issued has retired
         }
-        if (aw < NA && u_begin + aw < u_end) { load((u_begin + aw) % KT); load_ip(u_begin + aw); }
-        for (UnitIter w(u_begin, KT); aw < NA && w.u < u_end; w.next(S, KT)) {
-            if (w.it % NA != aw) continue;
-            const uint32_t s = w.s, ph = w.ph;
-            uint8_t* st = smem + s * p.stage_bytes;
-            uint4 xv[CPL];
-#pragma unroll
-            for (int c = 0; c < CPL; ++c) xv[c] = nxt[c];
-            const uint32_t ip = ip_nxt, npk = min(ip_nxt_end - ip_nxt, p.coo_cap);
-            if (w.u + NA < u_end) { uint32_t kn = w.kt + NA; load(kn >= KT ? kn % KT : kn); load_ip(w.u + NA); }
-            if (!warp_wait(bar_empty + 8 * s, ph ^ 1, abort_flag, p.status)) { ok = false; break; }
-            last_bar = bar_full + 8 * s, last_ph = ph;
-            if (lane == 0 && w.it >= S) request(w.u, w.tn, w.kt, smem_u32(st), bar_full + 8 * s, ip, npk);
-            // K-major MMA operand: core matrix (chunk c, octet o) at (c * NMMA8 + o) * 128, row m % 8 at + 16 (m % 8)
-            uint8_t* dst = st + p.off_xcan + ((part * CPL) * NMMA8 + (m >> 3)) * 128 + (m & 7) * 16;
-            float sum = 0.0f, sum_lo = 0.0f;          // sum_lo: chunks 0-7 where a lane holds a whole row
-#pragma unroll
-            for (int c = 0; c < CPL; ++c) {
-                const uint4 v = xv[c];
-                *reinterpret_cast<uint4*>(dst + c * NMMA8 * 128) = v;
-                if (LPR == 1 && c == 8) sum_lo = sum, sum = 0.0f;
-                sum += (bf16lo(v.x) + bf16hi(v.x)) + (bf16lo(v.y) + bf16hi(v.y)) + (bf16lo(v.z) + bf16hi(v.z)) +
-                       (bf16lo(v.w) + bf16hi(v.w));
-            }
-            // per-group sums of each row -> xsum[group][NMMA]
-            float* xsum = reinterpret_cast<float*>(st + p.off_xsum);
-            if (LPR == 4) {
-                const float s1 = sum + __shfl_xor_sync(0xffffffffu, sum, 8);       // parts {0,1} and {2,3}
-                const float s2 = s1 + __shfl_xor_sync(0xffffffffu, s1, 16);
-                if (GPS == 2) { if ((part & 1) == 0) xsum[(part >> 1) * NMMA + m] = s1; }
-                else if (part == 0) xsum[m] = s2;
-            } else if (LPR == 2) {
-                const float s1 = sum + __shfl_xor_sync(0xffffffffu, sum, 16);
-                if (GPS == 2) xsum[part * NMMA + m] = sum;
-                else if (part == 0) xsum[m] = s1;
-            } else {
-                if (GPS == 2) xsum[m] = sum_lo, xsum[NMMA + m] = sum;
-                else xsum[m] = sum_lo + sum;
-            }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the operand is read by the tensor core
-            __syncwarp();
-            if (SPARSE) {
+    } else if (warp < 3 + kTcXtWarps) {
+        // ------------------------------------------------------------------ FP32 activation copy for the outlier step
+        if (SPARSE) {
+            const uint32_t xw = warp - 3;
+            for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
+                if (w.it % kTcXtWarps != xw) continue;
+                const uint32_t s = w.s;
+                uint8_t* st = smem + s * p.stage_bytes;
+                if (!warp_wait(bar_full + 8 * s, w.ph, abort_flag, p.status)) break;
                 char* xt = reinterpret_cast<char*>(st + p.off_xt);
                 if constexpr (RR == 1) {
-                    if (m == 0) {
-                        float4* xt4 = reinterpret_cast<float4*>(xt) + part * CPL * 2;
-#pragma unroll
-                        for (int c = 0; c < CPL; ++c) {
-                            xt4[2 * c] = make_float4(bf16lo(xv[c].x), bf16hi(xv[c].x), bf16lo(xv[c].y), bf16hi(xv[c].y));
-                            xt4[2 * c + 1] = make_float4(bf16lo(xv[c].z), bf16hi(xv[c].z), bf16lo(xv[c].w), bf16hi(xv[c].w));
-                        }
-                    }
+                    // row 0 of the operand: 8 values of chunk c at c * NMMA8 * 128; lane l takes k = 4 l .. 4 l + 3
+                    const uint2 v = *reinterpret_cast<const uint2*>(st + p.off_xcan + (lane >> 1) * (NMMA8 * 128) + (lane & 1) * 8);
+                    reinterpret_cast<float4*>(xt)[lane] = make_float4(bf16lo(v.x), bf16hi(v.x), bf16lo(v.y), bf16hi(v.y));
                 } else {
                     build_xt<RR>(smem_u32(st + p.off_xcan), NMMA8, xt, lane);
                 }
                 __syncwarp();
+                if (lane == 0) mbar_arrive(bar_xt + 8 * s);
             }
-            if (lane == 0) mbar_arrive(bar_full + 8 * s);
         }
-        if (!ok && last_bar)                // gave up: let this warp's last copies land before the CTA exits
-            for (uint32_t spin = 0; spin < (1u << 20) && !mbar_try_wait(last_bar, last_ph); ++spin) {}
+    } else if (warp < UW0) {
+        // idle: keeps the strips' warps at a multiple of four
     } else if (warp < EW0) {
         // ------------------------------------------------------------------ unpack warps: thread = column
         const int dw = warp - UW0;
+        const int col = dw * 32 + lane;
         const uint32_t t_lane = ((uint32_t)((dw & 3) * 32)) << 16;
         const uint32_t t_a = tmem_base + t_lane + (uint32_t)(dw >> 2) * 64;
         for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
             const uint32_t it = w.it, s = w.s, b = w.it & 1;
+            const uint8_t* st = smem + s * p.stage_bytes;
             if (!warp_wait(bar_full + 8 * s, w.ph, abort_flag, p.status)) break;
+            // the column's 128 codes: four 16-byte loads (32 rows each), lanes contiguous
+            const uint4* wp = reinterpret_cast<const uint4*>(st) + col;
+            uint4 w4 = wp[0];
+            // 128 + z of each group as a BF16 pair (z is an integer 0..15 held in BF16)
+            uint32_t zz[GPS];
+#pragma unroll
+            for (int gi = 0; gi < GPS; ++gi) {
+                const uint32_t z = (uint32_t)__float2int_rn(bf16_bits_to_float(reinterpret_cast<const uint16_t*>(st + p.off_sz)[(GPS + gi) * BN + col]));
+                zz[gi] = 0x43004300u | (z * 0x00010001u);
+            }
             // the A buffer of this parity was last read by the MMAs of unit it - 2
             if (it >= 2 && !warp_wait(bar_d_ready + 8 * b, ((it - 2) >> 1) & 1, abort_flag, p.status)) break;
             tc_fence_after();
-            // the column's 128 codes: four 16-byte loads (32 rows each), lanes contiguous
-            const uint4* wp = reinterpret_cast<const uint4*>(smem + s * p.stage_bytes) + dw * 32 + lane;
-            uint4 w4 = wp[0];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const uint4 cur = w4;
                 if (j < 3) w4 = wp[(j + 1) * BN];
                 const uint32_t ww[4] = {cur.x, cur.y, cur.z, cur.w};
+                const uint32_t zj = zz[j / (4 / GPS)];
                 uint32_t a[16];
 #pragma unroll
                 for (int x = 0; x < 4; ++x) {
-                    a[4 * x + 0] = codes_to_bf16x2(ww[x]);
-                    a[4 * x + 1] = codes_to_bf16x2(ww[x] >> 4);
-                    a[4 * x + 2] = codes_to_bf16x2(ww[x] >> 8);
-                    a[4 * x + 3] = codes_to_bf16x2(ww[x] >> 12);
+                    // 128 + q as BF16 pairs (rows 2i, 2i + 1 of the word's eight), minus 128 + z: exactly q - z
+                    a[4 * x + 0] = sub_bf16x2(codes_to_bf16x2(ww[x]), zj);
+                    a[4 * x + 1] = sub_bf16x2(codes_to_bf16x2(ww[x] >> 4), zj);
+                    a[4 * x + 2] = sub_bf16x2(codes_to_bf16x2(ww[x] >> 8), zj);
+                    a[4 * x + 3] = sub_bf16x2(codes_to_bf16x2(ww[x] >> 12), zj);
                 }
                 tmem_st16(t_a + b * (NT128 * 64) + j * 16, a);
             }
@@ -446,7 +440,7 @@ __global__ void __launch_bounds__(32 * (2 + kTcActWarps + 2 * (BN / 32)), 1) fq_
             const uint32_t tn = w.tn, kt = w.kt;
             const uint8_t* st = smem + s * p.stage_bytes;
             if (!warp_wait(bar_full + 8 * s, w.ph, abort_flag, p.status)) { ok = false; break; }
-            // outliers: the bucket descriptor and this lane's slot of the first packet are requested now
+            // outliers: the bucket descriptor and this lane's slots of the first packets are requested now
             uint32_t sp_off = 0, sp_cnt = 0, sp_tail = 0, cmax = 0;
             constexpr int NP = RR <= 16 ? 2 : 1;                     // packet rounds in flight
             uint32_t pk[NP];
@@ -475,35 +469,25 @@ __global__ void __launch_bounds__(32 * (2 + kTcActWarps + 2 * (BN / 32)), 1) fq_
             };
 #pragma unroll
             for (int j = 0; j < NP; ++j) pk[j] = (SPARSE && (uint32_t)j < sp_cnt) ? slot_word(sp_off + j) : 0u;
+            float sv[GPS];
+#pragma unroll
+            for (int gi = 0; gi < GPS; ++gi) sv[gi] = bf16_bits_to_float(reinterpret_cast<const uint16_t*>(st + p.off_sz)[gi * BN + col]);
             // the unit's sums, once its MMAs are complete
             if (!warp_wait(bar_d_ready + 8 * b, (it >> 1) & 1, abort_flag, p.status)) { ok = false; break; }
             tc_fence_after();
-            const uint16_t* sc = reinterpret_cast<const uint16_t*>(st + p.off_sz);
-            const float* xsum = reinterpret_cast<const float*>(st + p.off_xsum);
 #pragma unroll
             for (int gi = 0; gi < GPS; ++gi) {
-                const float sv = bf16_bits_to_float(sc[gi * BN + col]);
-                const float zc = -(128.0f + bf16_bits_to_float(sc[(GPS + gi) * BN + col]));
                 float d[RR];
                 tmem_ld<RR>(t_d + b * (NT128 * DCOLS) + gi * NMMA, d);
-                if constexpr (RR == 1) {
-                    accf[0] = fmaf(sv, fmaf(zc, xsum[gi * NMMA], d[0]), accf[0]);
-                } else {
 #pragma unroll
-                    for (int i = 0; i < RR / 4; ++i) {
-                        const float4 xs = *reinterpret_cast<const float4*>(xsum + gi * NMMA + 4 * i);
-                        accf[4 * i + 0] = fmaf(sv, fmaf(zc, xs.x, d[4 * i + 0]), accf[4 * i + 0]);
-                        accf[4 * i + 1] = fmaf(sv, fmaf(zc, xs.y, d[4 * i + 1]), accf[4 * i + 1]);
-                        accf[4 * i + 2] = fmaf(sv, fmaf(zc, xs.z, d[4 * i + 2]), accf[4 * i + 2]);
-                        accf[4 * i + 3] = fmaf(sv, fmaf(zc, xs.w, d[4 * i + 3]), accf[4 * i + 3]);
-                    }
-                }
+                for (int i = 0; i < RR; ++i) accf[i] = fmaf(sv[gi], d[i], accf[i]);       // s * sum_k x (q - z)
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_relaxed(bar_go + 8 * b);         // the MMAs of unit it + 2 may overwrite this D buffer
             if (SPARSE) {
                 // ---- the unit's outliers of this thread's column (padding slots have value 0: they add 0)
+                if (cmax > 0 && !warp_wait(bar_xt + 8 * s, w.ph, abort_flag, p.status)) { ok = false; break; }
                 for (uint32_t i = 0; i < cmax; i += NP) {
                     uint32_t nx[NP];                               // the next rounds' slots, requested before this round's math
 #pragma unroll
@@ -515,7 +499,9 @@ __global__ void __launch_bounds__(32 * (2 + kTcActWarps + 2 * (BN / 32)), 1) fq_
                 if (HOT) {
                     // a bucket with a tail: its packets (slots name their column) are shared out over the eight
                     // lane groups g, each adding into sums of its own that are added up over g afterwards
-                    for (uint32_t hot = __ballot_sync(0xffffffffu, sp_tail != 0); hot; ) {     // warp-uniform
+                    uint32_t hot = __ballot_sync(0xffffffffu, sp_tail != 0);
+                    if (hot && cmax == 0 && !warp_wait(bar_xt + 8 * s, w.ph, abort_flag, p.status)) { ok = false; break; }
+                    while (hot) {                                      // warp-uniform
                         const uint32_t hot_lane = __ffs(hot) - 1;
                         hot &= ~(0x01010101u << (hot_lane & 7u));
                         const uint32_t hot_off = __shfl_sync(0xffffffffu, sp_off + sp_cnt, hot_lane);
@@ -525,9 +511,9 @@ __global__ void __launch_bounds__(32 * (2 + kTcActWarps + 2 * (BN / 32)), 1) fq_
                         for (int ri = 0; ri < RR; ++ri) hacc[ri] = 0.0f;
                         for (uint32_t i = g; i < hot_cnt; i += 8) {
                             const uint32_t idx = hot_off + i;
-                            const uint4 pk = (idx < p.coo_cap) ? reinterpret_cast<const uint4*>(pk_s)[idx]
-                                                               : __ldg(reinterpret_cast<const uint4*>(pk_g) + idx);
-                            const uint32_t wd[4] = {pk.x, pk.y, pk.z, pk.w};
+                            const uint4 pkt = (idx < p.coo_cap) ? reinterpret_cast<const uint4*>(pk_s)[idx]
+                                                                : __ldg(reinterpret_cast<const uint4*>(pk_g) + idx);
+                            const uint32_t wd[4] = {pkt.x, pkt.y, pkt.z, pkt.w};
 #pragma unroll
                             for (int e = 0; e < 4; ++e) {
                                 // a tail slot names its column: slots of other columns count as padding (value 0)

@@ -44,12 +44,14 @@ struct Params {
     uint32_t* status;
     uint32_t* counters;
     float* partials;
+    const float* xmeta;   // per k-step and group: 2^(E-21) and sum_k x_int of every batch row (fq_prep_x_kernel)
+    const float* xt;      // per k-step: k-major FP32 copy of the activations, swizzled
     uint32_t M, K, N, KT, NT;
     uint32_t NB, coo_cap, stages;
     uint32_t split;   // 0 = units dealt out as one contiguous range per CTA (stream-K);
                       // c > 0 = every column tile belongs to c CTAs, CTA b takes part b mod c of tile b / c
     // shared-memory offsets (bytes); all but the last are relative to a stage
-    uint32_t stage_bytes, off_sz, off_xcan, off_xt, off_info, off_coo;
+    uint32_t stage_bytes, off_sz, off_xcan, off_xmeta, off_xt, off_info, off_coo;
     uint32_t off_bar;
 };
 
@@ -315,9 +317,9 @@ static int sm_count_cached() {
 
 // Rows kept per epilogue thread of the tcgen05 kernel, and the MMA's batch columns, for a launch of M rows.
 static inline uint32_t rr_of(uint32_t m) { return m <= 1 ? 1u : (m <= 4 ? 4u : (m <= 8 ? 8u : (m <= 16 ? 16u : 32u))); }
-static inline uint32_t nmma_of(uint32_t m) { return m <= 16 ? 16u : 32u; }
+static inline uint32_t nmma_of(uint32_t m) { return (kLimbs * rr_of(m) + 15) / 16 * 16; }      // limb rows of the MMA operand
 
-// Plan of a launch of up to 32 rows.
+// Plan of a launch of up to 32 rows (16 with groups of 64: the accumulators of both groups must fit in tensor memory).
 static fq_status_t make_plan(const fq_layout_t* L, uint32_t M, bool sparse, Plan& pl) {
     const uint32_t BN = L->BN, NB = L->buckets_per_tile, GPS = kBK / L->group;
     const uint32_t NMMA = nmma_of(M), RR = rr_of(M);
@@ -343,6 +345,7 @@ static fq_status_t make_plan(const fq_layout_t* L, uint32_t M, bool sparse, Plan
     p.split = split;
     const uint32_t w_bytes = 16 * BN * 4, sz_bytes = 2 * GPS * BN * 2;
     const uint32_t xt_bytes = sparse ? kBK * RR * 4 : 0;                 // FP32 k-major copy [k][RR]
+    const uint32_t meta_bytes = GPS * 2 * meta_rows(RR) * 4;
     uint32_t cap = 0;
     if (sparse) {
         cap = L->tilecoo_encoded ? std::max<uint32_t>(8, round_up(L->max_tile_packets, 8)) : 256;
@@ -352,7 +355,8 @@ static fq_status_t make_plan(const fq_layout_t* L, uint32_t M, bool sparse, Plan
     for (;;) {
         p.off_sz = w_bytes;
         p.off_xcan = p.off_sz + round_up(sz_bytes, 128);
-        p.off_xt = p.off_xcan + NMMA * 256;
+        p.off_xmeta = p.off_xcan + NMMA * 128;                            // limbs: NMMA rows x 128 k, one byte each
+        p.off_xt = p.off_xmeta + round_up(meta_bytes, 128);
         p.off_info = p.off_xt + xt_bytes;
         p.off_coo = p.off_info + (sparse ? round_up(NB * 4, 128) : 0);
         stage = round_up(p.off_coo + cap * 16, 128);
@@ -387,44 +391,80 @@ static EncodeTiledFn encode_tiled() {
     return fn;
 }
 
-// Tiled view of rows [0, rows) of a row-major BF16 matrix with K columns as (8 consecutive k, row, block
-// of 8 k): a box of (8, nmma, 16) is the K-major MMA operand of one k-step (8-row x 16-byte core matrices,
-// blocks of 8 k outermost), and rows beyond `rows` read as zero.
-static fq_status_t make_x_map(const void* X, uint32_t rows, uint32_t K, uint32_t nmma, CUtensorMap* out) {
+// Tiled view of the limb array ([rows][K] bytes, row-major) as (16 consecutive k, row, block of 16 k): a box
+// of (16, nmma, 8) is the K-major MMA operand of one k-step (8-row x 16-byte core matrices, blocks of 16 k
+// outermost), and rows beyond `rows` read as zero.
+static fq_status_t make_x_map(const void* xl, uint32_t rows, uint32_t K, uint32_t nmma, CUtensorMap* out) {
     EncodeTiledFn enc = encode_tiled();
     if (!enc) return fail(FQ_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
-    const cuuint64_t dims[3] = {8, rows, K / 8};
-    const cuuint64_t strides[2] = {(cuuint64_t)K * 2, 16};           // bytes, dimensions 1 and 2
-    const cuuint32_t box[3] = {8, nmma, 16};
+    const cuuint64_t dims[3] = {16, rows, K / 16};
+    const cuuint64_t strides[2] = {(cuuint64_t)K, 16};               // bytes, dimensions 1 and 2
+    const cuuint32_t box[3] = {16, nmma, 8};
     const cuuint32_t estr[3] = {1, 1, 1};
-    const CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(X), dims, strides, box, estr,
+    const CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(xl), dims, strides, box, estr,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(FQ_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
     return FQ_OK;
 }
 
+// Scratch layout: status word and header, tile-arrival counters, FP32 partial slots, then the activation
+// arrays fq_prep_x_kernel writes for the launch in flight (limbs, scales and sums, FP32 copy).
+struct Scratch {
+    size_t off_partials, off_xl, off_xmeta, off_xt, total;
+};
+static Scratch scratch_layout(const fq_layout_t* L, uint32_t rows) {
+    const size_t rr = rr_of(rows), K = L->K;
+    Scratch sc;
+    sc.off_partials = kWsHeaderBytes + kWsCounterBytes;
+    sc.off_xl = sc.off_partials + (size_t)kMaxCtas * 2 * L->BN * rr * 4;
+    sc.off_xmeta = sc.off_xl + (((size_t)kLimbs * rr * K + 255) & ~(size_t)255);
+    sc.off_xmeta = (sc.off_xmeta + 255) & ~(size_t)255;
+    sc.off_xt = sc.off_xmeta + (((K / kBK) * (kBK / L->group) * 2 * meta_rows((int)rr) * 4 + 255) & ~(size_t)255);
+    sc.total = sc.off_xt + K * rr * 4;
+    return sc;
+}
+static inline uint32_t rows_per_launch(const fq_layout_t* L) { return L->group == 64 ? 16u : 32u; }
+
+typedef void (*PrepFn)(const uint16_t*, uint32_t, uint32_t, int8_t*, float*, float*);
+static PrepFn pick_prep(uint32_t rr, uint32_t g) {
+    switch (rr) {
+        case 1: return g == 64 ? fq_prep_x_kernel<1, 64> : fq_prep_x_kernel<1, 128>;
+        case 4: return g == 64 ? fq_prep_x_kernel<4, 64> : fq_prep_x_kernel<4, 128>;
+        case 8: return g == 64 ? fq_prep_x_kernel<8, 64> : fq_prep_x_kernel<8, 128>;
+        case 16: return g == 64 ? fq_prep_x_kernel<16, 64> : fq_prep_x_kernel<16, 128>;
+        default: return g == 64 ? fq_prep_x_kernel<32, 64> : fq_prep_x_kernel<32, 128>;
+    }
+}
+
 typedef void (*KernelFn)(const Params, const CUtensorMap);
 
-template <int BN, int NMMA, int RR, int G>
+template <int BN, int RR, int G>
 static KernelFn pick_tc_sparse(bool sparse, bool hot) {
-    if (!sparse) return (KernelFn)fq_tc_kernel<BN, NMMA, RR, G, false, false>;
-    return hot ? (KernelFn)fq_tc_kernel<BN, NMMA, RR, G, true, true> : (KernelFn)fq_tc_kernel<BN, NMMA, RR, G, true, false>;
+    if (!sparse) return (KernelFn)fq_tc_kernel<BN, RR, G, false, false>;
+    return hot ? (KernelFn)fq_tc_kernel<BN, RR, G, true, true> : (KernelFn)fq_tc_kernel<BN, RR, G, true, false>;
 }
-template <int BN, int G>
-static KernelFn pick_tc_rows(uint32_t rr, bool sparse, bool hot) {
+template <int BN>
+static KernelFn pick_tc_rows(uint32_t rr, uint32_t g, bool sparse, bool hot) {
+    if (g == 64) {      // at most 16 rows per launch
+        switch (rr) {
+            case 1: return pick_tc_sparse<BN, 1, 64>(sparse, hot);
+            case 4: return pick_tc_sparse<BN, 4, 64>(sparse, hot);
+            case 8: return pick_tc_sparse<BN, 8, 64>(sparse, hot);
+            default: return pick_tc_sparse<BN, 16, 64>(sparse, hot);
+        }
+    }
     switch (rr) {
-        case 1: return pick_tc_sparse<BN, 16, 1, G>(sparse, hot);
-        case 4: return pick_tc_sparse<BN, 16, 4, G>(sparse, hot);
-        case 8: return pick_tc_sparse<BN, 16, 8, G>(sparse, hot);
-        case 16: return pick_tc_sparse<BN, 16, 16, G>(sparse, hot);
-        default: return pick_tc_sparse<BN, 32, 32, G>(sparse, hot);
+        case 1: return pick_tc_sparse<BN, 1, 128>(sparse, hot);
+        case 4: return pick_tc_sparse<BN, 4, 128>(sparse, hot);
+        case 8: return pick_tc_sparse<BN, 8, 128>(sparse, hot);
+        case 16: return pick_tc_sparse<BN, 16, 128>(sparse, hot);
+        default: return pick_tc_sparse<BN, 32, 128>(sparse, hot);
     }
 }
 static KernelFn pick_kernel(uint32_t bn, uint32_t M, uint32_t g, bool sparse, bool hot) {
     const uint32_t rr = rr_of(M);
-    if (bn == 128) return g == 64 ? pick_tc_rows<128, 64>(rr, sparse, hot) : pick_tc_rows<128, 128>(rr, sparse, hot);
-    return g == 64 ? pick_tc_rows<256, 64>(rr, sparse, hot) : pick_tc_rows<256, 128>(rr, sparse, hot);
+    return bn == 128 ? pick_tc_rows<128>(rr, g, sparse, hot) : pick_tc_rows<256>(rr, g, sparse, hot);
 }
 
 // cudaFuncSetAttribute costs several microseconds: do it once per (kernel, device).
@@ -461,41 +501,60 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
     fq_status_t st = fq_workspace_bytes(L, M, &need);
     if (st != FQ_OK) return st;
     if (workspace_bytes < need) return fail(FQ_ERR_BUFFER_TOO_SMALL, "workspace holds %zu bytes, %zu needed", workspace_bytes, need);
-    // up to 32 rows per launch; a remainder of at most 16 rows gets the cheaper variants
-    const uint32_t rows_per_launch = 32;
-    for (uint32_t m0 = 0; m0 < M; m0 += rows_per_launch) {
-        const uint32_t mb = std::min<uint32_t>(rows_per_launch, M - m0);
+    // up to 32 (16) rows per launch; a remainder gets the cheaper variants
+    const uint32_t rpl = rows_per_launch(L);
+    for (uint32_t m0 = 0; m0 < M; m0 += rpl) {
+        const uint32_t mb = std::min<uint32_t>(rpl, M - m0);
         Plan pl;
         st = make_plan(L, mb, sparse, pl);
         if (st != FQ_OK) return st;
         Params& p = pl.p;
+        const Scratch sc = scratch_layout(L, mb);
+        const uint32_t rr = rr_of(mb);
+        int8_t* xl = (int8_t*)workspace + sc.off_xl;
+        float* xmeta = (float*)((uint8_t*)workspace + sc.off_xmeta);
+        float* xt = (float*)((uint8_t*)workspace + sc.off_xt);
         CUtensorMap tmX;
-        st = make_x_map((const uint16_t*)X + (size_t)m0 * L->K, mb, L->K, nmma_of(mb), &tmX);
+        st = make_x_map(xl, kLimbs * rr, L->K, nmma_of(mb), &tmX);
         if (st != FQ_OK) return st;
         p.Y = (uint16_t*)Y + (size_t)m0 * L->N;
         p.wq = (const uint8_t*)wq; p.scale = (const uint16_t*)scale; p.zero = (const uint16_t*)zero;
         p.indptr = (const uint32_t*)indptr; p.info = (const uint32_t*)info; p.packed = (const uint4*)packed;
         p.status = (uint32_t*)workspace;
         p.counters = (uint32_t*)((uint8_t*)workspace + kWsHeaderBytes);
-        p.partials = (float*)((uint8_t*)workspace + kWsHeaderBytes + kWsCounterBytes);
+        p.partials = (float*)((uint8_t*)workspace + sc.off_partials);
+        p.xmeta = xmeta; p.xt = xt;
         KernelFn fn = pick_kernel(L->BN, mb, L->group, sparse, pl.general);
+        // Both launches are programmatic dependent launches: a grid may become resident while the kernel
+        // before it in the stream drains.  The preparation kernel waits for that kernel before it reads X or
+        // writes the scratch; the fused kernel's producer warp streams weights (which no kernel writes) and
+        // everything else in it first executes griddepcontrol.wait, after which all memory operations of the
+        // earlier grids are complete and visible.
+        cudaLaunchAttribute attr[1];
+        std::memset(attr, 0, sizeof(attr));
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        {
+            cudaLaunchConfig_t cfg;
+            std::memset(&cfg, 0, sizeof(cfg));
+            const uint32_t warps = rr * (L->K / kBK);
+            cfg.gridDim = dim3((warps + 3) / 4);
+            cfg.blockDim = dim3(128);
+            cfg.stream = (cudaStream_t)stream;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            cudaError_t pe = cudaLaunchKernelEx(&cfg, pick_prep(rr, L->group), (const uint16_t*)X + (size_t)m0 * L->K, mb, L->K, xl, xmeta, xt);
+            if (pe != cudaSuccess) return fail(FQ_ERR_CUDA, "activation preparation launch: %s", cudaGetErrorString(pe));
+        }
         cudaError_t e = ensure_smem_attr((const void*)fn, (int)kSmemBudget);
         if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
         {
-            // Programmatic dependent launch: this grid may become resident while the kernel before it
-            // in the stream drains.  Its producer warp then already streams weights (which no kernel
-            // writes); the warps that touch X, Y or the scratch first execute griddepcontrol.wait, after
-            // which all memory operations of the earlier grid are complete and visible.
             cudaLaunchConfig_t cfg;
             std::memset(&cfg, 0, sizeof(cfg));
             cfg.gridDim = dim3(pl.grid);
             cfg.blockDim = dim3(pl.threads);
             cfg.dynamicSmemBytes = pl.smem;
             cfg.stream = (cudaStream_t)stream;
-            cudaLaunchAttribute attr[1];
-            std::memset(attr, 0, sizeof(attr));
-            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-            attr[0].val.programmaticStreamSerializationAllowed = 1;
             cfg.attrs = attr;
             cfg.numAttrs = 1;
             e = cudaLaunchKernelEx(&cfg, fn, p, tmX);
@@ -516,8 +575,7 @@ extern "C" {
 fq_status_t fq_workspace_bytes(const fq_layout_t* L, uint32_t M, size_t* bytes) {
     if (!layout_ok(L) || !bytes) return fail(FQ_ERR_INVALID_ARG, "bad layout or null output");
     if (M < 1 || M > FQ_MAX_M) return fail(FQ_ERR_INVALID_ARG, "M = %u outside [1, %u]", M, FQ_MAX_M);
-    const uint32_t mb = std::min<uint32_t>(M, 32);
-    *bytes = kWsHeaderBytes + kWsCounterBytes + (size_t)kMaxCtas * 2 * L->BN * rr_of(mb) * 4;
+    *bytes = scratch_layout(L, std::min<uint32_t>(M, rows_per_launch(L))).total;
     return FQ_OK;
 }
 

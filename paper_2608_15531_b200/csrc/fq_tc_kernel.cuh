@@ -1,29 +1,36 @@
-// The fused operator on the fifth-generation tensor cores (tcgen05.mma, operands in tensor memory).
+// The fused operator on the fifth-generation tensor cores (tcgen05.mma kind::i8, operands in tensor memory).
 // Included by fq_kernels.cu inside namespace fq, after the PTX helpers.
+//
+// Arithmetic.  The tensor core multiplies 8-bit integers exactly: the INT4 codes q go in as they are, and the
+// BF16 activations go in as block fixed point.  For every batch row and quantisation group (64 or 128 k) a
+// small kernel (fq_prep_x_kernel) writes x as an integer x_int = round(x * 2^(21-E)) (E = exponent of the
+// group's largest |x|, so |x_int| < 2^22: exact for every element within 2^14 of the largest, rounded to 2^-22
+// of the largest below that), split into three signed 8-bit limbs x_int = l0 + 2^8 l1 + 2^16 l2, together with
+// 2^(E-21), sum_k x_int and a k-major FP32 copy of x for the outlier step.  Then
+//     sum_k x (q - z)  =  2^(E-21) * ( sum_j 2^(8j) sum_k q l_j  -  z sum_k x_int )            (Eq. 3 inside Eq. 1)
+// with the inner sums exact INT32 results of the MMA, and the scale s applied once per group in FP32.
 //
 // A unit is one (column tile, 128-row k-step): 128 x BN INT4 codes with their scales, zero-points and
 // Tile-COO slice.  One persistent CTA per SM walks a range of units through a ring of shared-memory
 // stages (bulk copies + mbarrier expect_tx, Section 4.1).  Thread = output column throughout: tensor
-// memory lane c of a 128-column half holds row c of the A operand (the column's 128 dequantised
-// codes) and row c of the accumulator D (the column's batch rows).
+// memory lane c of a 128-column half holds row c of the A operand (the column's 128 codes) and row c of
+// the accumulator D (the column's batch rows, one column of D per limb and row).
 //
 //   warp 0          producer: every copy of a unit, one lane each: codes, scales, zero-points, bucket
-//                   descriptors, outlier packets (cp.async.bulk) and the unit's block of X as a 3-D tiled
-//                   tensor copy (cp.async.bulk.tensor) whose box lands as the K-major MMA operand
-//                   (8-row x 16-byte core matrices; rows beyond M are filled with zeros by the copy)
-//   warp 1          tensor: per unit 8 x BN/128 tcgen05.mma (M = 128 columns, N = NMMA batch rows, K = 16;
-//                   A from tensor memory, B = activations from shared memory, D = FP32 in tensor memory),
-//                   tcgen05.commit to mbarriers.  An MMA of this shape occupies the tensor pipe for 55-66
-//                   cycles whatever N <= 128 is, and its issue blocks meanwhile
-//   warps 3..6      (kernels with outliers) a k-major FP32 copy xt[k][RR] of the unit's activations for the
-//                   outlier step, built from the MMA operand with ldmatrix; alternate units
-//   unpack warps    BN/32: per 32 rows one 128-bit load of 32 codes, lop3/shift to 16 BF16 pairs 128 + q,
-//                   minus 128 + z (exact small integers q - z: Eq. 3 without the scale), tcgen05.st into A
-//   epilogue warps  BN/32: tcgen05.ld of the group sums, acc += s * sum x (q - z) in FP32 (Eq. 3 inside
-//                   Eq. 1), then the unit's outliers of the thread's own column straight into the same
-//                   registers (Section 4.2 without the shared-memory scatter: no atomics, no
-//                   read-modify-write), and at the end of a piece the split-tile settlement and the BF16
-//                   store of Y
+//                   descriptors, outlier packets, the unit's activation sums and FP32 copy (cp.async.bulk)
+//                   and its limbs as a 3-D tiled tensor copy (cp.async.bulk.tensor) whose box lands as the
+//                   K-major MMA operand (8-row x 16-byte core matrices; rows beyond the last are zero-filled)
+//   warp 1          tensor: per unit 4 x BN/128 tcgen05.mma (M = 128 columns, N = NMMA limb rows, K = 32;
+//                   A from tensor memory, B from shared memory, D = INT32 in tensor memory), tcgen05.commit
+//                   to mbarriers.  An MMA occupies the tensor pipe for 55-66 cycles whatever N <= 128 and
+//                   the operand type are, which is why the 8-bit type (K = 32 per instruction instead of
+//                   16) matters: with BF16 operands the tensor pipe, not HBM, bounds the kernel
+//   unpack warps    BN/32: per 32 rows one 128-bit load of 32 codes, two masks and a shift per 8 codes,
+//                   tcgen05.st into the A operand
+//   epilogue warps  BN/32: tcgen05.ld of the limb sums, the FP32 combination above, then the unit's outliers
+//                   of the thread's own column straight into the same registers (Section 4.2 without the
+//                   shared-memory scatter: no atomics, no read-modify-write), and at the end of a piece the
+//                   split-tile settlement and the BF16 store of Y
 //
 // Lane l of an epilogue warp owns column 32 * strip + l = 8 t + g with g = l % 8, t = l / 8: bucket g of
 // the strip, column number t of that bucket, so it takes slot t of every column-slotted packet of the
@@ -31,18 +38,17 @@
 // (Section 3.2.2's concern, shared-memory bank conflicts of the sparse step, met on the activation side:
 // the rows a warp's lanes pick are random, and the swizzle spreads them over all eight 16-byte bank groups).
 
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
-        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
-        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-        : "memory");
+constexpr int kLimbs = 3;
+
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"r"(taddr), "r"(r[0]), "r"(r[1]),
+                 "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+                 : "memory");
 }
 
-// N consecutive FP32 cells of this thread's tensor-memory lane (N = 1, 4, 8, 16 or 32)
+// N consecutive 32-bit cells of this thread's tensor-memory lane (N = 1, 4, 8, 16 or 32)
 template <int N>
-__device__ __forceinline__ void tmem_ld(uint32_t taddr, float (&d)[N]) {
-    uint32_t r[N];
+__device__ __forceinline__ void tmem_ld(uint32_t taddr, uint32_t (&r)[N]) {
     if constexpr (N == 1) {
         asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(r[0]) : "r"(taddr) : "memory");
     } else if constexpr (N == 4) {
@@ -69,9 +75,6 @@ __device__ __forceinline__ void tmem_ld(uint32_t taddr, float (&d)[N]) {
               "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
             : "r"(taddr) : "memory");
     }
-    tmem_wait_ld();
-#pragma unroll
-    for (int i = 0; i < N; ++i) d[i] = __uint_as_float(r[i]);
 }
 
 // XOR applied to the 16-byte chunk index of row k of the k-major FP32 copy (RR floats per row): with C
@@ -119,89 +122,132 @@ __device__ __forceinline__ void add_outliers(float (&acc)[RR], const uint32_t (&
     }
 }
 
-// The k-major FP32 copy xt[k][RR] (swizzled, see xt_swizzle) of the first RR batch rows of a unit, built
-// from the K-major MMA operand in shared memory (8-row x 16-byte core matrices; core matrix (chunk c,
-// octet o) at (c * nmma8 + o) * 128).  RR >= 4; whole warp.
-template <int RR>
-__device__ __forceinline__ void build_xt(uint32_t xb_addr, uint32_t nmma8, char* xt, int lane) {
-    constexpr int NO = RR >= 8 ? RR / 8 : 1;
-    const uint32_t pr = lane & 3;
-#pragma unroll
-    for (int o = 0; o < NO; ++o) {
-#pragma unroll
-        for (int kb = 0; kb < 4; ++kb) {
-            uint32_t r[4];
-            const uint32_t chunk = kb * 4 + (lane >> 3);
-            ldmatrix_x4_trans(xb_addr + (chunk * nmma8 + o) * 128 + (lane & 7) * 16, r[0], r[1], r[2], r[3]);
-            // this thread now holds rows m = 8 o + 2 pr, 2 pr + 1 of k = 8 (4 kb + i) + lane / 4, i = 0..3
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const uint32_t k = (kb * 4 + i) * 8 + (lane >> 2);
-                if constexpr (RR == 4) {
-                    if (pr < 2) *reinterpret_cast<float2*>(xt + k * 16 + pr * 8) = make_float2(bf16lo(r[i]), bf16hi(r[i]));
-                } else {
-                    const uint32_t cl = 2 * o + (pr >> 1);
-                    *reinterpret_cast<float2*>(xt + k * (4 * RR) + ((cl ^ xt_swizzle<RR>(k)) << 4) + (pr & 1) * 8) =
-                        make_float2(bf16lo(r[i]), bf16hi(r[i]));
-                }
-            }
-        }
-    }
-}
-
 // 3-D tiled tensor copy global -> shared, completion counted in bytes on an mbarrier
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const void* tmap, uint32_t c0, uint32_t c1, uint32_t c2, uint32_t bar) {
     asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
                  "l"(tmap), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
                  : "memory");
 }
-__device__ __forceinline__ uint32_t sub_bf16x2(uint32_t a, uint32_t b) {
-    uint32_t r;
-    asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
-    return r;
+// D[128 x N] (+)= A[128 x 32] (tensor memory) * B[32 x N] (shared-memory descriptor), signed 8-bit in, INT32 out.
+// Called by the whole (converged) warp with warp-uniform operands; one elected lane issues.
+__device__ __forceinline__ void umma_i8_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n .reg .pred p, e;\n setp.ne.b32 p, %4, 0;\n elect.sync _|e, 0xffffffff;\n"
+        " @e tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
+        : "memory");
 }
 
-constexpr int kTcXtWarps = 4;      // warps 3..6 build the FP32 copy; warp 7 is idle
-constexpr int kTcFirstUnpack = 8;  // a warp reaches the tensor-memory lanes 32 * (warp % 4) ..., so strips start at a multiple of 4
+// Rows of the activation arrays kept per unit for RR batch rows (at least four, so that every copy is a
+// multiple of 16 bytes).
+__host__ __device__ constexpr int meta_rows(int rr) { return rr < 4 ? 4 : rr; }
 
-// BN: tile columns (128 or 256).  NMMA: batch columns of the MMA (16 or 32).  RR: batch rows kept per
-// epilogue thread (1, 4, 8, 16, 32; M <= RR <= NMMA).  HOT: general form of the outlier step (buckets
-// with a tail, tiles with more packets than a stage holds).  tmX: tiled view of this launch's rows of X as
-// (8 consecutive k, row, block of 8 k), so that a box of (8, NMMA, 16) is a unit's K-major MMA operand.
-template <int BN, int NMMA, int RR, int GROUP, bool SPARSE, bool HOT>
+// ----------------------------------------------------------------------------- activation preparation
+//
+// One warp per (batch row m < RR, k-step kt): the row's 128 activations of the k-step -> limbs, scale,
+// integer sum and FP32 copy, per quantisation group (GROUP = 64: lanes 0-15 and 16-31; 128: the warp).
+//   xl    [kLimbs * RR][K] signed bytes, row j * RR + m = limb j of batch row m
+//   xmeta [K / 128][128 / GROUP][2][meta_rows(RR)] floats: 2^(E-21), then sum_k x_int (as a float)
+//   xt    [K / 128][128][RR] floats, 16-byte chunks XOR-swizzled by k (xt_swizzle)
+// Rows m >= M are written as zeros.  A group with a non-finite activation gets the scale NaN.
+template <int RR, int GROUP>
+__global__ void __launch_bounds__(128) fq_prep_x_kernel(const uint16_t* __restrict__ X, uint32_t M, uint32_t K, int8_t* __restrict__ xl,
+                                                        float* __restrict__ xmeta, float* __restrict__ xt) {
+    constexpr int GPS = kBK / GROUP, RM = meta_rows(RR);
+    // the grid after this one (the fused kernel) may start streaming weights; this one reads X and writes
+    // scratch that the grid before it may still be using
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const uint32_t lane = threadIdx.x & 31, wg = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const uint32_t KT = K / kBK;
+    if (wg >= RR * KT) return;
+    const uint32_t m = wg / KT, kt = wg - m * KT, k0 = kt * kBK + 4 * lane;
+    uint2 raw = make_uint2(0, 0);
+    if (m < M) raw = __ldg(reinterpret_cast<const uint2*>(X + (size_t)m * K + k0));
+    const uint32_t bits[4] = {raw.x & 0xffffu, raw.x >> 16, raw.y & 0xffffu, raw.y >> 16};
+    float x[4];
+    uint32_t amax = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { x[i] = __uint_as_float(bits[i] << 16); amax = max(amax, bits[i] & 0x7fffu); }
+#pragma unroll
+    for (int d = 1; d < 32 / GPS; d <<= 1) amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, d));
+    const uint32_t ef_raw = amax >> 7;                        // biased exponent of the group's largest |x|
+    const uint32_t ef = max(ef_raw, 22u);                     // keeps 2^(E-21) a normal number; tinier groups lose nothing that matters
+    const float up = __uint_as_float((275u - ef) << 23);      // 2^(21-E)
+    int xi[4], sum = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { xi[i] = __float2int_rn(x[i] * up); sum += xi[i]; }
+#pragma unroll
+    for (int d = 1; d < 32 / GPS; d <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, d);
+    // signed limbs: x_int = l0 + 256 l1 + 65536 l2
+    uint32_t w[kLimbs] = {0, 0, 0};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int l0 = (xi[i] << 24) >> 24;
+        const int r1 = (xi[i] - l0) >> 8;
+        const int l1 = (r1 << 24) >> 24;
+        const int l2 = (r1 - l1) >> 8;
+        w[0] |= (uint32_t)(l0 & 0xff) << (8 * i);
+        w[1] |= (uint32_t)(l1 & 0xff) << (8 * i);
+        w[2] |= (uint32_t)(l2 & 0xff) << (8 * i);
+    }
+#pragma unroll
+    for (int j = 0; j < kLimbs; ++j) *reinterpret_cast<uint32_t*>(xl + (size_t)(j * RR + m) * K + k0) = w[j];
+    if ((lane & (32 / GPS - 1)) == 0) {
+        const uint32_t gi = lane / (32 / GPS);
+        float* mt = xmeta + ((size_t)kt * GPS + gi) * 2 * RM;
+        mt[m] = ef_raw == 0xffu ? __uint_as_float(0x7fc00000u) : __uint_as_float((ef - 21u) << 23);     // 2^(E-21)
+        mt[RM + m] = (float)sum;
+    }
+    char* xtu = reinterpret_cast<char*>(xt) + (size_t)kt * (kBK * RR * 4);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint32_t k = 4 * lane + i;
+        *reinterpret_cast<float*>(xtu + k * (4 * RR) + ((((m >> 2) ^ xt_swizzle<RR>(k)) << 4) | ((m & 3) << 2))) = x[i];
+    }
+}
+
+// ----------------------------------------------------------------------------- the fused kernel
+
+constexpr int kTcFirstUnpack = 4;  // a warp reaches the tensor-memory lanes 32 * (warp % 4) ..., so strips start at a multiple of 4
+
+// BN: tile columns (128 or 256).  RR: batch rows kept per epilogue thread (1, 4, 8, 16, 32; M <= RR).  The
+// MMA's N is NMMA = kLimbs * RR rounded up to 16.  HOT: general form of the outlier step (buckets with a tail,
+// tiles with more packets than a stage holds).  tmX: tiled view of the limb array as (16 consecutive k, limb
+// row, block of 16 k), so that a box of (16, NMMA, 8) is a unit's K-major MMA operand.
+template <int BN, int RR, int GROUP, bool SPARSE, bool HOT>
 __global__ void __launch_bounds__(32 * (kTcFirstUnpack + 2 * (BN / 32)), 1)
 fq_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmX) {
     constexpr int NDW = BN / 32;              // unpack warps = epilogue warps = 32-column strips
     constexpr int NT128 = BN / 128;           // 128-column halves per unit
     constexpr int UW0 = kTcFirstUnpack, EW0 = UW0 + NDW;
     constexpr int GPS = kBK / GROUP;          // groups per k-step
+    constexpr int NMMA = (kLimbs * RR + 15) / 16 * 16;
+    constexpr int RM = meta_rows(RR);
     constexpr int DCOLS = GPS * NMMA;         // accumulator columns per half and buffer
-    constexpr uint32_t D_BASE = 2 * NT128 * 64;
+    constexpr uint32_t D_BASE = 2 * NT128 * 32;
     constexpr int W_BYTES = 16 * BN * 4;
     constexpr int SZ_ROW = BN * 2;
-    constexpr int X_BYTES = NMMA * 256;
-    constexpr int NMMA8 = NMMA / 8;
-    constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NMMA >> 3) << 17) | (8u << 24);
+    constexpr int X_BYTES = NMMA * 128, META_BYTES = GPS * 2 * RM * 4, XT_BYTES = SPARSE ? kBK * RR * 4 : 0;
+    constexpr uint32_t IDESC = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NMMA >> 3) << 17) | (8u << 24);
     static_assert(D_BASE + 2 * NT128 * DCOLS <= 512, "tensor memory: two A buffers and two D buffers must fit");
-    static_assert(RR <= NMMA && (RR == 1 || RR % 4 == 0), "rows per thread");
+    static_assert(RR == 1 || RR % 4 == 0, "rows per thread");
     extern __shared__ __align__(128) uint8_t smem[];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t S = p.stages;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
     const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * S;
-    const uint32_t bar_xt = bar_empty + 8 * S;           // [S] the stage's FP32 activation copy is written
-    const uint32_t bar_go = bar_xt + 8 * S;              // [2] A buffer written (unpack warps) and D buffer free (epilogue warps)
+    const uint32_t bar_go = bar_empty + 8 * S;           // [2] A buffer written (unpack warps) and D buffer free (epilogue warps)
     const uint32_t bar_d_ready = bar_go + 16;            // [2] MMAs of a unit complete (D written, A read)
     const uint32_t bar_final = bar_d_ready + 16;
-    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 3 * S + 5);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 2 * S + 5);
     volatile uint32_t* tmem_slot = abort_flag + 1;
 
     if (tid == 0) {
         for (uint32_t s = 0; s < S; ++s) {
             mbar_init(bar_full + 8 * s, 1);                    // the producer's expect_tx arrival
             mbar_init(bar_empty + 8 * s, 2 * NDW + 1);         // unpack warps, epilogue warps, the MMAs' commit
-            mbar_init(bar_xt + 8 * s, 1);
         }
         for (uint32_t b = 0; b < 2; ++b) {
             mbar_init(bar_go + 8 * b, 2 * NDW);                // unpack warps (A of this unit), epilogue warps (D of the unit two before)
@@ -221,9 +267,9 @@ fq_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmX) {
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     // The grid after this one in the stream may start now (it takes SMs as this grid's CTAs leave).  The
-    // warps that write Y or touch the scratch wait for the grid before this one, and so does the producer
-    // before its first copy of X; the weight arrays are read before: no kernel writes them while calls are
-    // in flight.
+    // warps that write Y or touch the scratch wait for the grids before this one, and so does the producer
+    // before its first copy of the activation arrays; the weight arrays are read before: no kernel writes
+    // them while calls are in flight.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (warp >= EW0) asm volatile("griddepcontrol.wait;" ::: "memory");
 
@@ -242,13 +288,13 @@ fq_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmX) {
     if (warp == 0) {
         // ------------------------------------------------------------------ producer
         // Lane l issues copy number l of a unit (issuing a bulk copy occupies its thread for a few hundred
-        // cycles): 0 codes, 1.. scales, then zero-points, then X, bucket descriptors, packets.
-        constexpr int L_X = 1 + 2 * GPS, L_INFO = L_X + 1, L_PK = L_X + 2;
+        // cycles): 0 codes, 1.. scales, then zero-points, bucket descriptors, packets; then the activation
+        // arrays: limbs, sums, FP32 copy.
+        constexpr int L_INFO = 1 + 2 * GPS, L_PK = L_INFO + 1, L_X = L_INFO + 2, L_META = L_X + 1, L_XT = L_X + 2;
         uint32_t issued = 0;
         bool ok = true;
-        // the packet ranges of this warp's next 32 units, read 32 at a time
-        uint32_t ip_a = 0, ip_b = 0;
-        auto weights = [&](const UnitIter& w) {                        // everything of a unit but X
+        uint32_t ip_a = 0, ip_b = 0;                                   // packet ranges of the next 32 units, read 32 at a time
+        auto weights = [&](const UnitIter& w) {                        // the weight arrays of a unit
             const uint32_t s = w.s, full = bar_full + 8 * s;
             const uint32_t st = smem_u32(smem) + s * p.stage_bytes;
             if (SPARSE && (w.it & 31) == 0) {
@@ -261,7 +307,8 @@ fq_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmX) {
                 pk0 = __shfl_sync(0xffffffffu, ip_a, w.it & 31);
                 npk = min(__shfl_sync(0xffffffffu, ip_b, w.it & 31) - pk0, p.coo_cap);
             }
-            if (lane == 0) mbar_arrive_expect_tx(full, W_BYTES + 2 * GPS * SZ_ROW + X_BYTES + (SPARSE ? p.NB * 4 + npk * 16 : 0));
+            if (lane == 0)
+                mbar_arrive_expect_tx(full, W_BYTES + 2 * GPS * SZ_ROW + X_BYTES + META_BYTES + XT_BYTES + (SPARSE ? p.NB * 4 + npk * 16 : 0));
             __syncwarp();
             if (lane == 0) {
                 bulk_g2s(st, p.wq + (size_t)w.u * W_BYTES, W_BYTES, full);
@@ -277,12 +324,15 @@ fq_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmX) {
                 if (npk) bulk_g2s(st + p.off_coo, p.packed + pk0, npk * 16, full);
             }
         };
-        auto activations = [&](const UnitIter& w) {
-            if (lane == L_X)
-                tma_load_3d(smem_u32(smem) + w.s * p.stage_bytes + p.off_xcan, &tmX, 0, 0, w.kt * 16, bar_full + 8 * w.s);
+        auto activations = [&](const UnitIter& w) {                    // the activation arrays of its k-step
+            const uint32_t full = bar_full + 8 * w.s;
+            const uint32_t st = smem_u32(smem) + w.s * p.stage_bytes;
+            if (lane == L_X) tma_load_3d(st + p.off_xcan, &tmX, 0, 0, w.kt * 8, full);
+            else if (lane == L_META) bulk_g2s(st + p.off_xmeta, p.xmeta + (size_t)w.kt * (META_BYTES / 4), META_BYTES, full);
+            else if (SPARSE && lane == L_XT) bulk_g2s(st + p.off_xt, reinterpret_cast<const char*>(p.xt) + (size_t)w.kt * XT_BYTES, XT_BYTES, full);
         };
         // the first pass over the ring finds every stage empty: its weight copies go out before the wait
-        // for the previous grid, its copies of X after
+        // for the grids before this one, its activation copies after
         const uint32_t n_first = min(S, u_end - u_begin);
         {
             UnitIter w(u_begin, KT);
@@ -304,74 +354,51 @@ fq_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmX) {
             for (uint32_t j = (issued > S ? issued - S : 0); j < issued; ++j)
                 for (uint32_t spin = 0; spin < (1u << 20) && !mbar_try_wait(bar_full + 8 * (j % S), (j / S) & 1); ++spin) {}
         }
-    } else if (warp <= 2) {
-        // ------------------------------------------------------------------ tensor warp (warp 2 is idle)
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ tensor warp
         // One warp issues every MMA of the CTA (issued from two warps in turn, MMAs run several times slower).
-        // An MMA of this shape occupies the tensor pipe for 55-66 cycles and its issue blocks meanwhile, so the
-        // warp looks at the next unit's barriers between the MMAs of this one: their latency then hides behind
-        // MMAs in flight, and a unit whose operands are ready is issued without waiting at all.
-        if (warp == 1) {
-            // The first MMA of a CTA takes microseconds to start (the tensor pipe wakes up): issue a throw-away
-            // one now, while the first loads are in flight.  It reads whatever A buffer 0 and stage 0 hold and
-            // writes D buffer 1, which the first real MMA into that buffer overwrites.
-            umma_ts(tmem_base + D_BASE + NT128 * DCOLS, tmem_base, make_b_desc(smem_u32(smem) + p.off_xcan, NMMA8 * 128, 128), IDESC, 0);
-            uint32_t ready = 0;                          // this unit's barriers were seen complete already
-            for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
-                const uint32_t it = w.it, s = w.s, b = w.it & 1;    // A buffer b and D buffer b
-                if (!ready) {
-                    if (!warp_wait(bar_full + 8 * s, w.ph, abort_flag, p.status)) break;       // the activation operand
-                    if (!warp_wait(bar_go + 8 * b, (it >> 1) & 1, abort_flag, p.status)) break;
-                }
-                tc_fence_after();
-                UnitIter nx = w;
-                nx.next(S, KT);
-                const bool has_next = nx.u < u_end;
-                uint32_t seen = 0;
-                auto poll = [&]() {
-                    if (has_next && lane == 0 && !seen)
-                        seen = mbar_test_wait(bar_full + 8 * nx.s, nx.ph) & mbar_test_wait(bar_go + 8 * (nx.it & 1), (nx.it >> 1) & 1);
-                };
-                const uint64_t bd0 = make_b_desc(smem_u32(smem) + s * p.stage_bytes + p.off_xcan, NMMA8 * 128, 128);
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const int gi = ks / (8 / GPS);
-#pragma unroll
-                    for (int h = 0; h < NT128; ++h) {
-                        const uint32_t d = tmem_base + D_BASE + (b * NT128 + h) * DCOLS + gi * NMMA;
-                        const uint32_t a = tmem_base + (b * NT128 + h) * 64 + ks * 8;
-                        umma_ts(d, a, bd0 + (uint64_t)((ks * 2 * NMMA8 * 128) >> 4), IDESC, (ks % (8 / GPS)) != 0);
-                    }
-                    if (ks == 3 || ks == 6) poll();
-                }
-                umma_commit(bar_d_ready + 8 * b);   // this unit's sums are complete and its A buffer has been read
-                umma_commit(bar_empty + 8 * s);     // and so has the stage's activation operand
-                poll();
-                ready = __shfl_sync(0xffffffffu, seen, 0);
+        // The issue of an MMA blocks while the one before it runs, so the warp looks at the next unit's
+        // barriers between the MMAs of this one: their latency then hides behind MMAs in flight, and a unit
+        // whose operands are ready is issued without waiting at all.
+        // The first MMA of a CTA takes microseconds to start (the tensor pipe wakes up): issue a throw-away
+        // one now, while the first loads are in flight.  It reads whatever A buffer 0 and stage 0 hold and
+        // writes D buffer 1, which the first real MMA into that buffer overwrites.
+        umma_i8_ts(tmem_base + D_BASE + NT128 * DCOLS, tmem_base, make_b_desc(smem_u32(smem) + p.off_xcan, NMMA * 16, 128), IDESC, 0);
+        uint32_t ready = 0;                          // this unit's barriers were seen complete already
+        for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
+            const uint32_t it = w.it, s = w.s, b = w.it & 1;    // A buffer b and D buffer b
+            if (!ready) {
+                if (!warp_wait(bar_full + 8 * s, w.ph, abort_flag, p.status)) break;       // the activation operand
+                if (!warp_wait(bar_go + 8 * b, (it >> 1) & 1, abort_flag, p.status)) break;
             }
-            __syncwarp();
-            umma_commit(bar_final);                 // fires when every MMA this warp issued has retired
-        }
-    } else if (warp < 3 + kTcXtWarps) {
-        // ------------------------------------------------------------------ FP32 activation copy for the outlier step
-        if (SPARSE) {
-            const uint32_t xw = warp - 3;
-            for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
-                if (w.it % kTcXtWarps != xw) continue;
-                const uint32_t s = w.s;
-                uint8_t* st = smem + s * p.stage_bytes;
-                if (!warp_wait(bar_full + 8 * s, w.ph, abort_flag, p.status)) break;
-                char* xt = reinterpret_cast<char*>(st + p.off_xt);
-                if constexpr (RR == 1) {
-                    // row 0 of the operand: 8 values of chunk c at c * NMMA8 * 128; lane l takes k = 4 l .. 4 l + 3
-                    const uint2 v = *reinterpret_cast<const uint2*>(st + p.off_xcan + (lane >> 1) * (NMMA8 * 128) + (lane & 1) * 8);
-                    reinterpret_cast<float4*>(xt)[lane] = make_float4(bf16lo(v.x), bf16hi(v.x), bf16lo(v.y), bf16hi(v.y));
-                } else {
-                    build_xt<RR>(smem_u32(st + p.off_xcan), NMMA8, xt, lane);
+            tc_fence_after();
+            UnitIter nx = w;
+            nx.next(S, KT);
+            const bool has_next = nx.u < u_end;
+            uint32_t seen = 0;
+            auto poll = [&]() {
+                if (has_next && lane == 0 && !seen)
+                    seen = mbar_test_wait(bar_full + 8 * nx.s, nx.ph) & mbar_test_wait(bar_go + 8 * (nx.it & 1), (nx.it >> 1) & 1);
+            };
+            const uint64_t bd0 = make_b_desc(smem_u32(smem) + s * p.stage_bytes + p.off_xcan, NMMA * 16, 128);
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {             // 32 k per MMA: 16-k blocks 2 ks, 2 ks + 1 of the operand
+                const int gi = ks / (4 / GPS);
+#pragma unroll
+                for (int h = 0; h < NT128; ++h) {
+                    const uint32_t d = tmem_base + D_BASE + (b * NT128 + h) * DCOLS + gi * NMMA;
+                    const uint32_t a = tmem_base + (b * NT128 + h) * 32 + ks * 8;
+                    umma_i8_ts(d, a, bd0 + (uint64_t)((ks * 2 * NMMA * 16) >> 4), IDESC, (ks % (4 / GPS)) != 0);
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_xt + 8 * s);
+                if (ks == 1 || ks == 2) poll();
             }
+            umma_commit(bar_d_ready + 8 * b);   // this unit's sums are complete and its A buffer has been read
+            umma_commit(bar_empty + 8 * s);     // and so has the stage's activation operand
+            poll();
+            ready = __shfl_sync(0xffffffffu, seen, 0);
         }
+        __syncwarp();
+        umma_commit(bar_final);                 // fires when every MMA this warp issued has retired
     } else if (warp < UW0) {
         // idle: keeps the strips' warps at a multiple of four
     } else if (warp < EW0) {
@@ -379,40 +406,30 @@ fq_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmX) {
         const int dw = warp - UW0;
         const int col = dw * 32 + lane;
         const uint32_t t_lane = ((uint32_t)((dw & 3) * 32)) << 16;
-        const uint32_t t_a = tmem_base + t_lane + (uint32_t)(dw >> 2) * 64;
+        const uint32_t t_a = tmem_base + t_lane + (uint32_t)(dw >> 2) * 32;
         for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
             const uint32_t it = w.it, s = w.s, b = w.it & 1;
             const uint8_t* st = smem + s * p.stage_bytes;
             if (!warp_wait(bar_full + 8 * s, w.ph, abort_flag, p.status)) break;
             // the column's 128 codes: four 16-byte loads (32 rows each), lanes contiguous
             const uint4* wp = reinterpret_cast<const uint4*>(st) + col;
-            uint4 w4 = wp[0];
-            // 128 + z of each group as a BF16 pair (z is an integer 0..15 held in BF16)
-            uint32_t zz[GPS];
+            uint4 w4[4];
 #pragma unroll
-            for (int gi = 0; gi < GPS; ++gi) {
-                const uint32_t z = (uint32_t)__float2int_rn(bf16_bits_to_float(reinterpret_cast<const uint16_t*>(st + p.off_sz)[(GPS + gi) * BN + col]));
-                zz[gi] = 0x43004300u | (z * 0x00010001u);
-            }
+            for (int j = 0; j < 4; ++j) w4[j] = wp[j * BN];
             // the A buffer of this parity was last read by the MMAs of unit it - 2
             if (it >= 2 && !warp_wait(bar_d_ready + 8 * b, ((it - 2) >> 1) & 1, abort_flag, p.status)) break;
             tc_fence_after();
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                const uint4 cur = w4;
-                if (j < 3) w4 = wp[(j + 1) * BN];
-                const uint32_t ww[4] = {cur.x, cur.y, cur.z, cur.w};
-                const uint32_t zj = zz[j / (4 / GPS)];
-                uint32_t a[16];
+                const uint32_t ww[4] = {w4[j].x, w4[j].y, w4[j].z, w4[j].w};
+                uint32_t a[8];
 #pragma unroll
                 for (int x = 0; x < 4; ++x) {
-                    // 128 + q as BF16 pairs (rows 2i, 2i + 1 of the word's eight), minus 128 + z: exactly q - z
-                    a[4 * x + 0] = sub_bf16x2(codes_to_bf16x2(ww[x]), zj);
-                    a[4 * x + 1] = sub_bf16x2(codes_to_bf16x2(ww[x] >> 4), zj);
-                    a[4 * x + 2] = sub_bf16x2(codes_to_bf16x2(ww[x] >> 8), zj);
-                    a[4 * x + 3] = sub_bf16x2(codes_to_bf16x2(ww[x] >> 12), zj);
+                    // even nibbles are rows 0-3 of the word's eight, odd nibbles rows 4-7: two cells of four bytes
+                    a[2 * x + 0] = ww[x] & 0x0f0f0f0fu;
+                    a[2 * x + 1] = (ww[x] >> 4) & 0x0f0f0f0fu;
                 }
-                tmem_st16(t_a + b * (NT128 * 64) + j * 16, a);
+                tmem_st8(t_a + b * (NT128 * 32) + j * 8, a);
             }
             tmem_wait_st();
             tc_fence_before();
@@ -469,25 +486,48 @@ fq_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmX) {
             };
 #pragma unroll
             for (int j = 0; j < NP; ++j) pk[j] = (SPARSE && (uint32_t)j < sp_cnt) ? slot_word(sp_off + j) : 0u;
-            float sv[GPS];
+            float sv[GPS], zv[GPS];
 #pragma unroll
-            for (int gi = 0; gi < GPS; ++gi) sv[gi] = bf16_bits_to_float(reinterpret_cast<const uint16_t*>(st + p.off_sz)[gi * BN + col]);
+            for (int gi = 0; gi < GPS; ++gi) {
+                sv[gi] = bf16_bits_to_float(reinterpret_cast<const uint16_t*>(st + p.off_sz)[gi * BN + col]);
+                zv[gi] = -bf16_bits_to_float(reinterpret_cast<const uint16_t*>(st + p.off_sz)[(GPS + gi) * BN + col]);
+            }
+            const float* meta = reinterpret_cast<const float*>(st + p.off_xmeta);
             // the unit's sums, once its MMAs are complete
             if (!warp_wait(bar_d_ready + 8 * b, (it >> 1) & 1, abort_flag, p.status)) { ok = false; break; }
             tc_fence_after();
 #pragma unroll
             for (int gi = 0; gi < GPS; ++gi) {
-                float d[RR];
-                tmem_ld<RR>(t_d + b * (NT128 * DCOLS) + gi * NMMA, d);
+                // sum_k x (q - z) = 2^(E-21) * (D0 + 2^8 D1 + 2^16 D2 - z sum_k x_int), D_j = sum_k q l_j exact in INT32
+                float dl[kLimbs][RR];
+                if constexpr (RR == 1) {
+                    uint32_t c[4];                                  // one load of four cells covers the three limbs of the single row
+                    tmem_ld<4>(t_d + b * (NT128 * DCOLS) + gi * NMMA, c);
+                    tmem_wait_ld();
 #pragma unroll
-                for (int i = 0; i < RR; ++i) accf[i] = fmaf(sv[gi], d[i], accf[i]);       // s * sum_k x (q - z)
+                    for (int j = 0; j < kLimbs; ++j) dl[j][0] = (float)(int)c[j];
+                } else {
+                    uint32_t c[kLimbs][RR];
+#pragma unroll
+                    for (int j = 0; j < kLimbs; ++j) tmem_ld<RR>(t_d + b * (NT128 * DCOLS) + gi * NMMA + j * RR, c[j]);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < kLimbs; ++j)
+#pragma unroll
+                        for (int i = 0; i < RR; ++i) dl[j][i] = (float)(int)c[j][i];
+                }
+#pragma unroll
+                for (int i = 0; i < RR; ++i) {
+                    const float xs = meta[gi * 2 * RM + i], sx = meta[gi * 2 * RM + RM + i];
+                    const float f = fmaf(zv[gi], sx, fmaf(dl[2][i], 65536.0f, fmaf(dl[1][i], 256.0f, dl[0][i])));
+                    accf[i] = fmaf(sv[gi] * xs, f, accf[i]);
+                }
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_relaxed(bar_go + 8 * b);         // the MMAs of unit it + 2 may overwrite this D buffer
             if (SPARSE) {
                 // ---- the unit's outliers of this thread's column (padding slots have value 0: they add 0)
-                if (cmax > 0 && !warp_wait(bar_xt + 8 * s, w.ph, abort_flag, p.status)) { ok = false; break; }
                 for (uint32_t i = 0; i < cmax; i += NP) {
                     uint32_t nx[NP];                               // the next rounds' slots, requested before this round's math
 #pragma unroll
@@ -499,9 +539,7 @@ fq_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmX) {
                 if (HOT) {
                     // a bucket with a tail: its packets (slots name their column) are shared out over the eight
                     // lane groups g, each adding into sums of its own that are added up over g afterwards
-                    uint32_t hot = __ballot_sync(0xffffffffu, sp_tail != 0);
-                    if (hot && cmax == 0 && !warp_wait(bar_xt + 8 * s, w.ph, abort_flag, p.status)) { ok = false; break; }
-                    while (hot) {                                      // warp-uniform
+                    for (uint32_t hot = __ballot_sync(0xffffffffu, sp_tail != 0); hot; ) {     // warp-uniform
                         const uint32_t hot_lane = __ffs(hot) - 1;
                         hot &= ~(0x01010101u << (hot_lane & 7u));
                         const uint32_t hot_off = __shfl_sync(0xffffffffu, sp_off + sp_cnt, hot_lane);

@@ -247,7 +247,7 @@ fq_status_t fq_fused_w4a16_outlier_gemm(const fq_layout_t* L, const void* X, uin
  * gave up is not retrievable through fq_check_status() here (the array is not
  * visible to the caller) and shows as undefined Y.
  */
-#define FQ_STATIC_SCRATCH_BYTES 10485760u /* 10 MiB */
+#define FQ_STATIC_SCRATCH_BYTES 6356992u /* 6 MiB + 64 KiB */
 #define FQ_STATIC_SCRATCH_MAX_M 16u
 fq_status_t fq_fused_w4a16_outlier_gemm_noalloc(const fq_layout_t* L, const void* X, uint32_t M,
                                                 const void* wq, const void* scale, const void* zero,

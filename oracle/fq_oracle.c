@@ -195,9 +195,9 @@ void orc_fused_matmul(const uint16_t* X, uint32_t M, uint32_t K, uint32_t N, uin
  *   by BN columns and holds 16 * BN little-endian 32-bit words.  Word index
  *   inside the chunk, with j = 0..3, t = 0..BN-1, w = 0..3:
  *        (j * BN + t) * 4 + w .
- *   Nibble p (bits 4p .. 4p+3) of that word is the code of
+ *   Nibble p (bits 4p .. 4p+3) of that word, p = i + 4h with i = 0..3, h = 0..1, is the code of
  *        column  tn*BN + t
- *        row     kt*128 + 32*j + 8*w + r,   r = p/2 for even p, r = 4 + (p-1)/2 for odd p.
+ *        row     kt*128 + 32*j + 8*w + 2*i + h
  */
 int orc_decode_wq(const uint32_t* wq, uint32_t K, uint32_t N, uint32_t BN, uint8_t* q) {
     if (K % 128 != 0 || BN == 0 || N % BN != 0) return -1;
@@ -211,9 +211,9 @@ int orc_decode_wq(const uint32_t* wq, uint32_t K, uint32_t N, uint32_t BN, uint8
                     for (uint32_t w = 0; w < 4; ++w) {
                         uint32_t word = chunk[(j * BN + t) * 4 + w];
                         for (uint32_t p = 0; p < 8; ++p) {
-                            uint32_t r = (p & 1) ? 4 + (p - 1) / 2 : p / 2;
+                            uint32_t i = p & 3, h = p >> 2;
                             uint32_t col = tn * BN + t;
-                            uint32_t row = kt * 128 + 32 * j + 8 * w + r;
+                            uint32_t row = kt * 128 + 32 * j + 8 * w + 2 * i + h;
                             q[(size_t)row * N + col] = (uint8_t)((word >> (4 * p)) & 0xfu);
                         }
                     }

@@ -29,9 +29,9 @@ static inline float bf16_to_f32(uint16_t h) {
 
 // Position of the code of (row kr, column cr) inside a 128 x BN chunk: word index and nibble.
 static inline void wq_slot(uint32_t kr, uint32_t cr, uint32_t BN, uint32_t& word, uint32_t& nib) {
-    const uint32_t j = kr >> 5, w = (kr >> 3) & 3, r = kr & 7;
+    const uint32_t j = kr >> 5, w = (kr >> 3) & 3, i = (kr >> 1) & 3, h = kr & 1;
     word = (j * BN + cr) * 4 + w;
-    nib = r < 4 ? 2 * r : 2 * (r - 4) + 1;    // even nibbles: rows 0-3 of the word's eight, odd nibbles: rows 4-7
+    nib = i + 4 * h;
 }
 }  // namespace fq
 

@@ -15,7 +15,6 @@
 // arrive, which adds the FP32 partials in CTA order; no CTA waits for another.  Every wait on a barrier
 // is bounded: on expiry the CTA raises the scratch status word, drains and leaves through the common
 // exit that frees its tensor memory.
-#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -44,14 +43,14 @@ struct Params {
     uint32_t* status;
     uint32_t* counters;
     float* partials;
-    const float* xmeta;   // per k-step and group: 2^(E-21) and sum_k x_int of every batch row (fq_prep_x_kernel)
-    const float* xt;      // per k-step: k-major FP32 copy of the activations, swizzled
+    const uint8_t* xblob; // per k-step: the activation block fq_prep_x_kernel wrote (limbs, scales and sums, FP32 copy)
     uint32_t M, K, N, KT, NT;
     uint32_t NB, coo_cap, stages;
     uint32_t split;   // 0 = units dealt out as one contiguous range per CTA (stream-K);
                       // c > 0 = every column tile belongs to c CTAs, CTA b takes part b mod c of tile b / c
     // shared-memory offsets (bytes); all but the last are relative to a stage
     uint32_t stage_bytes, off_sz, off_xcan, off_xmeta, off_xt, off_info, off_coo;
+    uint32_t off_xch;     // hand-over of the second epilogue set's sums (BN x RR floats), if there are two sets
     uint32_t off_bar;
 };
 
@@ -217,6 +216,7 @@ struct UnitIter {
 };
 
 #include "fq_tc_kernel.cuh"
+#include "fq_mma_kernel.cuh"
 
 // ----------------------------------------------------------------------------- unfused SpMM
 
@@ -317,7 +317,7 @@ static int sm_count_cached() {
 
 // Rows kept per epilogue thread of the tcgen05 kernel, and the MMA's batch columns, for a launch of M rows.
 static inline uint32_t rr_of(uint32_t m) { return m <= 1 ? 1u : (m <= 4 ? 4u : (m <= 8 ? 8u : (m <= 16 ? 16u : 32u))); }
-static inline uint32_t nmma_of(uint32_t m) { return (kLimbs * rr_of(m) + 15) / 16 * 16; }      // limb rows of the MMA operand
+static inline uint32_t nmma_of(uint32_t m) { return (uint32_t)nmma_rows((int)rr_of(m)); }      // limb rows of the MMA operand
 
 // Plan of a launch of up to 32 rows (16 with groups of 64: the accumulators of both groups must fit in tensor memory).
 static fq_status_t make_plan(const fq_layout_t* L, uint32_t M, bool sparse, Plan& pl) {
@@ -345,7 +345,106 @@ static fq_status_t make_plan(const fq_layout_t* L, uint32_t M, bool sparse, Plan
     p.split = split;
     const uint32_t w_bytes = 16 * BN * 4, sz_bytes = 2 * GPS * BN * 2;
     const uint32_t xt_bytes = sparse ? kBK * RR * 4 : 0;                 // FP32 k-major copy [k][RR]
-    const uint32_t meta_bytes = GPS * 2 * meta_rows(RR) * 4;
+    uint32_t cap = 0;
+    if (sparse) {
+        cap = L->tilecoo_encoded ? std::max<uint32_t>(8, round_up(L->max_tile_packets, 8)) : 256;
+        cap = std::min<uint32_t>(cap, 1024);
+    }
+    const uint32_t xch_bytes = epilogue_sets((int)RR) == 2 ? BN * RR * 4 : 0;
+    uint32_t stage = 0, S = 0;
+    for (;;) {
+        p.off_sz = w_bytes;
+        p.off_xcan = p.off_sz + round_up(sz_bytes, 128);
+        // the k-step's activation block lands here as one copy: limbs (NMMA rows x 128 k, one byte each),
+        // scales and sums, FP32 copy (kernels with outliers only)
+        p.off_xmeta = p.off_xcan + blob_meta_off((int)RR);
+        p.off_xt = p.off_xcan + blob_xt_off((int)RR, (int)GPS);
+        p.off_info = p.off_xt + xt_bytes;
+        p.off_coo = p.off_info + (sparse ? round_up(NB * 4, 128) : 0);
+        stage = round_up(p.off_coo + cap * 16, 128);
+        S = std::min<uint32_t>(8, (kSmemBudget - 1024 - xch_bytes) / stage);
+        if (S >= 4 || cap <= 64) break;
+        cap = std::max<uint32_t>(64, cap / 2);  // oversized tiles read their tail from global memory
+    }
+    if (S < 2) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "shared-memory stages do not fit");
+    p.coo_cap = cap; p.stages = S; p.stage_bytes = stage;
+    // hot columns, tiles larger than the staged part, or an encoding whose sizes were not recorded
+    pl.general = sparse && (L->max_tail_packets > 0 || L->max_tile_packets > cap || !L->tilecoo_encoded);
+    p.off_xch = S * stage;
+    p.off_bar = p.off_xch + xch_bytes;
+    pl.smem = p.off_bar + 1024;
+    pl.threads = 32 * (kTcFirstUnpack + (1 + epilogue_sets((int)RR)) * (BN / 32));
+    pl.grid = grid;
+    return FQ_OK;
+}
+
+// Scratch layout: status word and header, tile-arrival counters, FP32 partial slots, then the activation
+// blocks fq_prep_x_kernel writes for the launch in flight (one per k-step).
+struct Scratch {
+    size_t off_partials, off_xb, total;
+};
+// Which kernel serves a launch is decided by its rows alone: up to 16 rows the warp-level MMA kernel, 17 to 32
+// rows the tcgen05 kernel (its MMAs cost the same for any number of batch rows up to 42; with groups of 64 its
+// two accumulators per unit fit in tensor memory only up to 16 rows, so such layers stay with the first).
+static inline bool tc_serves(const fq_layout_t* L, uint32_t rows) { return rows > 16 && L->group == 128; }
+static inline uint32_t rows_per_launch(const fq_layout_t* L, uint32_t rows_left) { return tc_serves(L, rows_left) ? std::min<uint32_t>(rows_left, 32u) : std::min<uint32_t>(rows_left, 16u); }
+static Scratch scratch_layout(const fq_layout_t* L, uint32_t rows) {
+    const bool tc = tc_serves(L, rows);
+    const size_t prow = tc ? 32 : 16;                     // batch rows of an FP32 partial slot
+    Scratch sc;
+    sc.off_partials = kWsHeaderBytes + kWsCounterBytes;
+    sc.off_xb = sc.off_partials + (size_t)kMaxCtas * 2 * L->BN * prow * 4;
+    sc.total = sc.off_xb + (tc ? (size_t)(L->K / kBK) * blob_bytes(32, (int)(kBK / L->group)) : 0);
+    return sc;
+}
+
+typedef void (*PrepFn)(const uint16_t*, uint32_t, uint32_t, uint8_t*);
+static PrepFn pick_prep(uint32_t rr, uint32_t g) { (void)rr; (void)g; return fq_prep_x_kernel<32, 128>; }
+
+typedef void (*KernelFn)(const Params);
+
+struct MmaPlan {
+    MmaParams p;
+    uint32_t threads, smem, grid;
+    uint32_t ngrp;   // groups of dense warps
+    bool general;    // the layer needs the general form of the outlier step
+};
+typedef void (*MmaKernelFn)(const MmaParams);
+
+// Plan of the small-batch kernel (fq_mma_kernel): M <= 16 per launch.
+static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, MmaPlan& pl) {
+    const uint32_t BN = L->BN, NB = L->buckets_per_tile, GPS = kBK / L->group;
+    const uint32_t MO = M <= 8 ? 1 : 2, ROWS = 8 * MO;
+    const uint32_t NDW = BN / 32;
+    MmaParams& p = pl.p;
+    std::memset(&p, 0, sizeof(p));
+    p.M = M; p.K = L->K; p.N = L->N; p.KT = L->K / kBK; p.NT = L->N / BN; p.NB = NB; p.nsw = 0;
+    const uint32_t w_bytes = 16 * BN * 4, sz_bytes = 2 * GPS * BN * 2;
+    const uint32_t xt_bytes = sparse ? (M == 1 ? 512 : (M <= 4 ? 2048 : MO * 4096)) : 0;     // FP32 [k], [k][4] or [octet][k][8]
+    // Two groups of dense warps (each takes every other unit) pay off when a CTA has enough units to
+    // stream; short jobs keep one group.  With two octets of rows the second group fits only because
+    // the outlier step of that variant prefetches less (96 registers per thread).
+    const int sms = sm_count_cached();
+    if (sms <= 0) return fail(FQ_ERR_CUDA, "no CUDA device: %s", cudaGetErrorString(cudaGetLastError()));
+    const uint32_t NT = L->N / BN, KT = L->K / kBK;
+    uint32_t grid = std::min<uint32_t>({(uint32_t)sms, kMaxCtas, NT * KT});
+    uint32_t units_per_cta = (NT * KT + grid - 1) / grid;
+    // Tile-aligned split instead of one contiguous range per CTA when it costs at most one more unit
+    // per CTA: then no CTA has to settle two split tiles in a row.
+    uint32_t split = 0;
+    if (NT <= grid) {
+        const uint32_t c = std::min<uint32_t>(grid / NT, KT);
+        if (c >= 2 && (KT + c - 1) / c <= units_per_cta + 1) {
+            split = c;
+            grid = NT * c;
+            units_per_cta = (KT + c - 1) / c;
+        }
+    }
+    p.split = split;
+    pl.ngrp = (units_per_cta >= 8 && MO <= 2) ? 2 : 1;    // four octets of rows: the accumulators leave no room
+    const uint32_t xch_bytes = pl.ngrp > 1 ? BN * ROWS * 4 : 0;   // hand-over of a group's partial sums
+    const uint32_t fixed = 1024 + xch_bytes;
+    const uint32_t budget = kSmemBudget;
     uint32_t cap = 0;
     if (sparse) {
         cap = L->tilecoo_encoded ? std::max<uint32_t>(8, round_up(L->max_tile_packets, 8)) : 256;
@@ -355,116 +454,70 @@ static fq_status_t make_plan(const fq_layout_t* L, uint32_t M, bool sparse, Plan
     for (;;) {
         p.off_sz = w_bytes;
         p.off_xcan = p.off_sz + round_up(sz_bytes, 128);
-        p.off_xmeta = p.off_xcan + NMMA * 128;                            // limbs: NMMA rows x 128 k, one byte each
-        p.off_xt = p.off_xmeta + round_up(meta_bytes, 128);
+        p.off_xsum = p.off_xcan + round_up(ROWS * kXPitch, 128);
+        p.off_xt = p.off_xsum + round_up(GPS * ROWS * 4, 128);          // stage-relative in this kernel
         p.off_info = p.off_xt + xt_bytes;
         p.off_coo = p.off_info + (sparse ? round_up(NB * 4, 128) : 0);
         stage = round_up(p.off_coo + cap * 16, 128);
-        S = std::min<uint32_t>(8, (kSmemBudget - 1024) / stage);
+        // An even number of stages: the activation warps and the dense groups take alternate units, and
+        // a parity wait is only valid for a waiter that meets every phase of the barrier.  With S even a
+        // stage always comes back to the same activation warp and the same dense group.
+        S = std::min<uint32_t>(8, (budget - fixed) / stage) & ~1u;
         if (S >= 4 || cap <= 64) break;
-        cap = std::max<uint32_t>(64, cap / 2);  // oversized tiles read their tail from global memory
+        cap = std::max<uint32_t>(64, cap / 2);
     }
-    if (S < 2) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "shared-memory stages do not fit");
+    if (S < 4) return fail(FQ_ERR_UNSUPPORTED_SHAPE, "shared-memory stages do not fit");
     p.coo_cap = cap; p.stages = S; p.stage_bytes = stage;
     // hot columns, tiles larger than the staged part, or an encoding whose sizes were not recorded
     pl.general = sparse && (L->max_tail_packets > 0 || L->max_tile_packets > cap || !L->tilecoo_encoded);
-    p.off_bar = S * stage;
+    p.off_shc = S * stage;
+    p.off_bar = p.off_shc + xch_bytes;
     pl.smem = p.off_bar + 1024;
-    pl.threads = 32 * (kTcFirstUnpack + 2 * (BN / 32));
+    pl.threads = 32 * (1 + kActWarps + pl.ngrp * NDW);
     pl.grid = grid;
     return FQ_OK;
 }
 
-// cuTensorMapEncodeTiled, looked up through the runtime (the library does not link the driver API).
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-static EncodeTiledFn encode_tiled() {
-    static EncodeTiledFn fn = [] {
-        void* sym = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) != cudaSuccess ||
-            qres != cudaDriverEntryPointSuccess)
-            sym = nullptr;
-        return (EncodeTiledFn)sym;
-    }();
-    return fn;
-}
-
-// Tiled view of the limb array ([rows][K] bytes, row-major) as (16 consecutive k, row, block of 16 k): a box
-// of (16, nmma, 8) is the K-major MMA operand of one k-step (8-row x 16-byte core matrices, blocks of 16 k
-// outermost), and rows beyond `rows` read as zero.
-static fq_status_t make_x_map(const void* xl, uint32_t rows, uint32_t K, uint32_t nmma, CUtensorMap* out) {
-    EncodeTiledFn enc = encode_tiled();
-    if (!enc) return fail(FQ_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
-    const cuuint64_t dims[3] = {16, rows, K / 16};
-    const cuuint64_t strides[2] = {(cuuint64_t)K, 16};               // bytes, dimensions 1 and 2
-    const cuuint32_t box[3] = {16, nmma, 8};
-    const cuuint32_t estr[3] = {1, 1, 1};
-    const CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(xl), dims, strides, box, estr,
-                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return fail(FQ_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
-    return FQ_OK;
-}
-
-// Scratch layout: status word and header, tile-arrival counters, FP32 partial slots, then the activation
-// arrays fq_prep_x_kernel writes for the launch in flight (limbs, scales and sums, FP32 copy).
-struct Scratch {
-    size_t off_partials, off_xl, off_xmeta, off_xt, total;
-};
-static Scratch scratch_layout(const fq_layout_t* L, uint32_t rows) {
-    const size_t rr = rr_of(rows), K = L->K;
-    Scratch sc;
-    sc.off_partials = kWsHeaderBytes + kWsCounterBytes;
-    sc.off_xl = sc.off_partials + (size_t)kMaxCtas * 2 * L->BN * rr * 4;
-    sc.off_xmeta = sc.off_xl + (((size_t)kLimbs * rr * K + 255) & ~(size_t)255);
-    sc.off_xmeta = (sc.off_xmeta + 255) & ~(size_t)255;
-    sc.off_xt = sc.off_xmeta + (((K / kBK) * (kBK / L->group) * 2 * meta_rows((int)rr) * 4 + 255) & ~(size_t)255);
-    sc.total = sc.off_xt + K * rr * 4;
-    return sc;
-}
-static inline uint32_t rows_per_launch(const fq_layout_t* L) { return L->group == 64 ? 16u : 32u; }
-
-typedef void (*PrepFn)(const uint16_t*, uint32_t, uint32_t, int8_t*, float*, float*);
-static PrepFn pick_prep(uint32_t rr, uint32_t g) {
-    switch (rr) {
-        case 1: return g == 64 ? fq_prep_x_kernel<1, 64> : fq_prep_x_kernel<1, 128>;
-        case 4: return g == 64 ? fq_prep_x_kernel<4, 64> : fq_prep_x_kernel<4, 128>;
-        case 8: return g == 64 ? fq_prep_x_kernel<8, 64> : fq_prep_x_kernel<8, 128>;
-        case 16: return g == 64 ? fq_prep_x_kernel<16, 64> : fq_prep_x_kernel<16, 128>;
-        default: return g == 64 ? fq_prep_x_kernel<32, 64> : fq_prep_x_kernel<32, 128>;
+// MS: form of the outlier step (1: single batch row, one column per lane; 8: rows split over the lanes);
+// NGRP: groups of dense warps; HOT: general form of the outlier step
+// (long bucket lists shared out, packets beyond the staged part of a tile)
+template <int BN, int MO, int G, bool HOT>
+static MmaKernelFn pick_mma_sparse(bool sparse, uint32_t ms, uint32_t ngrp) {
+    if constexpr (MO == 1) {
+        if (ngrp == 2) {
+            if (!sparse) return (MmaKernelFn)fq_mma_kernel<BN, MO, G, false, 8, 2, false>;
+            if (ms == 1) return (MmaKernelFn)fq_mma_kernel<BN, MO, G, true, 1, 2, HOT>;
+            if (ms == 4) return (MmaKernelFn)fq_mma_kernel<BN, MO, G, true, 4, 2, HOT>;
+            return (MmaKernelFn)fq_mma_kernel<BN, MO, G, true, 8, 2, HOT>;
+        }
+        if (sparse && ms == 1) return (MmaKernelFn)fq_mma_kernel<BN, MO, G, true, 1, 1, HOT>;
+        if (sparse && ms == 4) return (MmaKernelFn)fq_mma_kernel<BN, MO, G, true, 4, 1, HOT>;
     }
+    if constexpr (MO == 2) {
+        if (ngrp == 2) return sparse ? (MmaKernelFn)fq_mma_kernel<BN, MO, G, true, 8, 2, HOT> : (MmaKernelFn)fq_mma_kernel<BN, MO, G, false, 8, 2, false>;
+    }
+    if (!sparse) return (MmaKernelFn)fq_mma_kernel<BN, MO, G, false, 8, 1, false>;
+    return (MmaKernelFn)fq_mma_kernel<BN, MO, G, true, 8, 1, HOT>;
 }
-
-typedef void (*KernelFn)(const Params, const CUtensorMap);
+template <int BN, int MO>
+static MmaKernelFn pick_mma_group(uint32_t g, bool sparse, uint32_t ms, uint32_t ngrp, bool hot) {
+    if (g == 64) return hot ? pick_mma_sparse<BN, MO, 64, true>(sparse, ms, ngrp) : pick_mma_sparse<BN, MO, 64, false>(sparse, ms, ngrp);
+    return hot ? pick_mma_sparse<BN, MO, 128, true>(sparse, ms, ngrp) : pick_mma_sparse<BN, MO, 128, false>(sparse, ms, ngrp);
+}
+static MmaKernelFn pick_mma_kernel(uint32_t bn, uint32_t M, uint32_t g, bool sparse, uint32_t ngrp, bool hot) {
+    const uint32_t mo = M <= 8 ? 1 : 2, ms = M <= 1 ? 1 : (M <= 4 ? 4 : 8);
+    if (bn == 128) return mo == 1 ? pick_mma_group<128, 1>(g, sparse, ms, ngrp, hot) : pick_mma_group<128, 2>(g, sparse, ms, ngrp, hot);
+    return mo == 1 ? pick_mma_group<256, 1>(g, sparse, ms, ngrp, hot) : pick_mma_group<256, 2>(g, sparse, ms, ngrp, hot);
+}
 
 template <int BN, int RR, int G>
 static KernelFn pick_tc_sparse(bool sparse, bool hot) {
     if (!sparse) return (KernelFn)fq_tc_kernel<BN, RR, G, false, false>;
     return hot ? (KernelFn)fq_tc_kernel<BN, RR, G, true, true> : (KernelFn)fq_tc_kernel<BN, RR, G, true, false>;
 }
-template <int BN>
-static KernelFn pick_tc_rows(uint32_t rr, uint32_t g, bool sparse, bool hot) {
-    if (g == 64) {      // at most 16 rows per launch
-        switch (rr) {
-            case 1: return pick_tc_sparse<BN, 1, 64>(sparse, hot);
-            case 4: return pick_tc_sparse<BN, 4, 64>(sparse, hot);
-            case 8: return pick_tc_sparse<BN, 8, 64>(sparse, hot);
-            default: return pick_tc_sparse<BN, 16, 64>(sparse, hot);
-        }
-    }
-    switch (rr) {
-        case 1: return pick_tc_sparse<BN, 1, 128>(sparse, hot);
-        case 4: return pick_tc_sparse<BN, 4, 128>(sparse, hot);
-        case 8: return pick_tc_sparse<BN, 8, 128>(sparse, hot);
-        case 16: return pick_tc_sparse<BN, 16, 128>(sparse, hot);
-        default: return pick_tc_sparse<BN, 32, 128>(sparse, hot);
-    }
-}
 static KernelFn pick_kernel(uint32_t bn, uint32_t M, uint32_t g, bool sparse, bool hot) {
-    const uint32_t rr = rr_of(M);
-    return bn == 128 ? pick_tc_rows<128>(rr, g, sparse, hot) : pick_tc_rows<256>(rr, g, sparse, hot);
+    (void)M; (void)g;      // 17 to 32 rows, groups of 128: one variant per tile width
+    return bn == 128 ? pick_tc_sparse<128, 32, 128>(sparse, hot) : pick_tc_sparse<256, 32, 128>(sparse, hot);
 }
 
 // cudaFuncSetAttribute costs several microseconds: do it once per (kernel, device).
@@ -501,67 +554,74 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
     fq_status_t st = fq_workspace_bytes(L, M, &need);
     if (st != FQ_OK) return st;
     if (workspace_bytes < need) return fail(FQ_ERR_BUFFER_TOO_SMALL, "workspace holds %zu bytes, %zu needed", workspace_bytes, need);
-    // up to 32 (16) rows per launch; a remainder gets the cheaper variants
-    const uint32_t rpl = rows_per_launch(L);
-    for (uint32_t m0 = 0; m0 < M; m0 += rpl) {
-        const uint32_t mb = std::min<uint32_t>(rpl, M - m0);
-        Plan pl;
-        st = make_plan(L, mb, sparse, pl);
-        if (st != FQ_OK) return st;
-        Params& p = pl.p;
-        const Scratch sc = scratch_layout(L, mb);
-        const uint32_t rr = rr_of(mb);
-        int8_t* xl = (int8_t*)workspace + sc.off_xl;
-        float* xmeta = (float*)((uint8_t*)workspace + sc.off_xmeta);
-        float* xt = (float*)((uint8_t*)workspace + sc.off_xt);
-        CUtensorMap tmX;
-        st = make_x_map(xl, kLimbs * rr, L->K, nmma_of(mb), &tmX);
-        if (st != FQ_OK) return st;
-        p.Y = (uint16_t*)Y + (size_t)m0 * L->N;
-        p.wq = (const uint8_t*)wq; p.scale = (const uint16_t*)scale; p.zero = (const uint16_t*)zero;
-        p.indptr = (const uint32_t*)indptr; p.info = (const uint32_t*)info; p.packed = (const uint4*)packed;
-        p.status = (uint32_t*)workspace;
-        p.counters = (uint32_t*)((uint8_t*)workspace + kWsHeaderBytes);
-        p.partials = (float*)((uint8_t*)workspace + sc.off_partials);
-        p.xmeta = xmeta; p.xt = xt;
-        KernelFn fn = pick_kernel(L->BN, mb, L->group, sparse, pl.general);
-        // Both launches are programmatic dependent launches: a grid may become resident while the kernel
-        // before it in the stream drains.  The preparation kernel waits for that kernel before it reads X or
-        // writes the scratch; the fused kernel's producer warp streams weights (which no kernel writes) and
-        // everything else in it first executes griddepcontrol.wait, after which all memory operations of the
-        // earlier grids are complete and visible.
-        cudaLaunchAttribute attr[1];
-        std::memset(attr, 0, sizeof(attr));
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        {
-            cudaLaunchConfig_t cfg;
-            std::memset(&cfg, 0, sizeof(cfg));
+    const Scratch sc = scratch_layout(L, M);
+    cudaLaunchAttribute attr[1];
+    std::memset(attr, 0, sizeof(attr));
+    // Programmatic dependent launch: a grid may become resident while the kernel before it in the stream
+    // drains.  Its producer warps then already stream weights (which no kernel writes); everything that touches
+    // X, Y or the scratch first executes griddepcontrol.wait, after which all memory operations of the earlier
+    // grids are complete and visible.
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    for (uint32_t m0 = 0; m0 < M;) {
+        const uint32_t mb = rows_per_launch(L, M - m0);
+        const uint16_t* Xm = (const uint16_t*)X + (size_t)m0 * L->K;
+        uint16_t* Ym = (uint16_t*)Y + (size_t)m0 * L->N;
+        cudaLaunchConfig_t cfg;
+        std::memset(&cfg, 0, sizeof(cfg));
+        cfg.stream = (cudaStream_t)stream;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaError_t e;
+        if (tc_serves(L, mb)) {
+            Plan pl;
+            st = make_plan(L, mb, sparse, pl);
+            if (st != FQ_OK) return st;
+            Params& p = pl.p;
+            const uint32_t rr = rr_of(mb);
+            uint8_t* xb = (uint8_t*)workspace + sc.off_xb;
+            p.Y = Ym;
+            p.wq = (const uint8_t*)wq; p.scale = (const uint16_t*)scale; p.zero = (const uint16_t*)zero;
+            p.indptr = (const uint32_t*)indptr; p.info = (const uint32_t*)info; p.packed = (const uint4*)packed;
+            p.status = (uint32_t*)workspace;
+            p.counters = (uint32_t*)((uint8_t*)workspace + kWsHeaderBytes);
+            p.partials = (float*)((uint8_t*)workspace + sc.off_partials);
+            p.xblob = xb;
+            KernelFn fn = pick_kernel(L->BN, mb, L->group, sparse, pl.general);
+            e = ensure_smem_attr((const void*)fn, (int)kSmemBudget);
+            if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+            // the activation blocks of these rows, then the fused kernel
             const uint32_t warps = rr * (L->K / kBK);
             cfg.gridDim = dim3((warps + 3) / 4);
             cfg.blockDim = dim3(128);
-            cfg.stream = (cudaStream_t)stream;
-            cfg.attrs = attr;
-            cfg.numAttrs = 1;
-            cudaError_t pe = cudaLaunchKernelEx(&cfg, pick_prep(rr, L->group), (const uint16_t*)X + (size_t)m0 * L->K, mb, L->K, xl, xmeta, xt);
-            if (pe != cudaSuccess) return fail(FQ_ERR_CUDA, "activation preparation launch: %s", cudaGetErrorString(pe));
-        }
-        cudaError_t e = ensure_smem_attr((const void*)fn, (int)kSmemBudget);
-        if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-        {
-            cudaLaunchConfig_t cfg;
-            std::memset(&cfg, 0, sizeof(cfg));
+            cfg.dynamicSmemBytes = 0;
+            e = cudaLaunchKernelEx(&cfg, pick_prep(rr, L->group), Xm, mb, L->K, xb);
+            if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "activation preparation launch: %s", cudaGetErrorString(e));
             cfg.gridDim = dim3(pl.grid);
             cfg.blockDim = dim3(pl.threads);
             cfg.dynamicSmemBytes = pl.smem;
-            cfg.stream = (cudaStream_t)stream;
-            cfg.attrs = attr;
-            cfg.numAttrs = 1;
-            e = cudaLaunchKernelEx(&cfg, fn, p, tmX);
-            if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
+            e = cudaLaunchKernelEx(&cfg, fn, p);
+        } else {
+            MmaPlan pl;
+            st = make_plan_mma(L, mb, sparse, pl);
+            if (st != FQ_OK) return st;
+            MmaParams& p = pl.p;
+            p.X = Xm; p.Y = Ym;
+            p.wq = (const uint8_t*)wq; p.scale = (const uint16_t*)scale; p.zero = (const uint16_t*)zero;
+            p.indptr = (const uint32_t*)indptr; p.info = (const uint32_t*)info; p.packed = (const uint4*)packed;
+            p.status = (uint32_t*)workspace;
+            p.counters = (uint32_t*)((uint8_t*)workspace + kWsHeaderBytes);
+            p.partials = (float*)((uint8_t*)workspace + sc.off_partials);
+            MmaKernelFn fn = pick_mma_kernel(L->BN, mb, L->group, sparse, pl.ngrp, pl.general);
+            e = ensure_smem_attr((const void*)fn, (int)kSmemBudget);
+            if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+            cfg.gridDim = dim3(pl.grid);
+            cfg.blockDim = dim3(pl.threads);
+            cfg.dynamicSmemBytes = pl.smem;
+            e = cudaLaunchKernelEx(&cfg, fn, p);
         }
-        e = cudaGetLastError();
         if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
+        m0 += mb;
     }
     return FQ_OK;
 }
@@ -575,7 +635,7 @@ extern "C" {
 fq_status_t fq_workspace_bytes(const fq_layout_t* L, uint32_t M, size_t* bytes) {
     if (!layout_ok(L) || !bytes) return fail(FQ_ERR_INVALID_ARG, "bad layout or null output");
     if (M < 1 || M > FQ_MAX_M) return fail(FQ_ERR_INVALID_ARG, "M = %u outside [1, %u]", M, FQ_MAX_M);
-    *bytes = scratch_layout(L, std::min<uint32_t>(M, rows_per_launch(L))).total;
+    *bytes = scratch_layout(L, M).total;
     return FQ_OK;
 }
 

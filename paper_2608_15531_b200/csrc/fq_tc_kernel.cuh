@@ -16,10 +16,12 @@
 // memory lane c of a 128-column half holds row c of the A operand (the column's 128 codes) and row c of
 // the accumulator D (the column's batch rows, one column of D per limb and row).
 //
-//   warp 0          producer: every copy of a unit, one lane each: codes, scales, zero-points, bucket
-//                   descriptors, outlier packets, the unit's activation sums and FP32 copy (cp.async.bulk)
-//                   and its limbs as a 3-D tiled tensor copy (cp.async.bulk.tensor) whose box lands as the
-//                   K-major MMA operand (8-row x 16-byte core matrices; rows beyond the last are zero-filled)
+//   warps 0, 2      producers (cp.async.bulk): warp 0 copies a unit's codes, scales and zero-points, warp 2
+//                   its bucket descriptors, its outlier packets and the k-step's activation block, which the
+//                   preparation kernel wrote in the stage's own layout (limbs as the K-major MMA operand of
+//                   8-row x 16-byte core matrices, then scales and sums, then the FP32 copy).  Issuing a bulk
+//                   copy occupies its warp for about 120 ns, whichever lane issues it: one warp with all six
+//                   to eight copies of a unit bounded the kernel
 //   warp 1          tensor: per unit 4 x BN/128 tcgen05.mma (M = 128 columns, N = NMMA limb rows, K = 32;
 //                   A from tensor memory, B from shared memory, D = INT32 in tensor memory), tcgen05.commit
 //                   to mbarriers.  An MMA occupies the tensor pipe for 55-66 cycles whatever N <= 128 and
@@ -77,6 +79,11 @@ __device__ __forceinline__ void tmem_ld(uint32_t taddr, uint32_t (&r)[N]) {
     }
 }
 
+// (float)v for |v| < 2^22 without a conversion instruction (those issue at a quarter of the ALU rate, and an
+// epilogue thread needs three per batch row and group): v + 1.5 * 2^23 as an integer bit pattern is the float
+// 1.5 * 2^23 + v exactly.
+__device__ __forceinline__ float small_int_to_float(uint32_t v) { return __uint_as_float(v + 0x4B400000u) - 12582912.0f; }
+
 // XOR applied to the 16-byte chunk index of row k of the k-major FP32 copy (RR floats per row): with C
 // chunks per row, 8 / C consecutive rows share a 128-byte line, and the swizzle makes the chunk a lane
 // reads in one load instruction depend on k, so that lanes with random k cover all eight bank groups.
@@ -122,12 +129,6 @@ __device__ __forceinline__ void add_outliers(float (&acc)[RR], const uint32_t (&
     }
 }
 
-// 3-D tiled tensor copy global -> shared, completion counted in bytes on an mbarrier
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const void* tmap, uint32_t c0, uint32_t c1, uint32_t c2, uint32_t bar) {
-    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
-                 "l"(tmap), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
-                 : "memory");
-}
 // D[128 x N] (+)= A[128 x 32] (tensor memory) * B[32 x N] (shared-memory descriptor), signed 8-bit in, INT32 out.
 // Called by the whole (converged) warp with warp-uniform operands; one elected lane issues.
 __device__ __forceinline__ void umma_i8_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
@@ -143,17 +144,25 @@ __device__ __forceinline__ void umma_i8_ts(uint32_t d_tmem, uint32_t a_tmem, uin
 __host__ __device__ constexpr int meta_rows(int rr) { return rr < 4 ? 4 : rr; }
 
 // ----------------------------------------------------------------------------- activation preparation
-//
+
+// Bytes of the activation block of one k-step for RR batch rows: the limb operand (NMMA rows x 128 k, one byte
+// each), scales and sums (padded to 128 bytes), the FP32 copy.
+__host__ __device__ constexpr int nmma_rows(int rr) { return (kLimbs * rr + 15) / 16 * 16; }
+__host__ __device__ constexpr int blob_meta_off(int rr) { return nmma_rows(rr) * 128; }
+__host__ __device__ constexpr int blob_xt_off(int rr, int gps) { return blob_meta_off(rr) + (gps * 2 * meta_rows(rr) * 4 + 127) / 128 * 128; }
+__host__ __device__ constexpr int blob_bytes(int rr, int gps) { return blob_xt_off(rr, gps) + kBK * rr * 4; }
+
 // One warp per (batch row m < RR, k-step kt): the row's 128 activations of the k-step -> limbs, scale,
-// integer sum and FP32 copy, per quantisation group (GROUP = 64: lanes 0-15 and 16-31; 128: the warp).
-//   xl    [kLimbs * RR][K] signed bytes, row j * RR + m = limb j of batch row m
-//   xmeta [K / 128][128 / GROUP][2][meta_rows(RR)] floats: 2^(E-21), then sum_k x_int (as a float)
-//   xt    [K / 128][128][RR] floats, 16-byte chunks XOR-swizzled by k (xt_swizzle)
+// integer sum and FP32 copy, per quantisation group (GROUP = 64: lanes 0-15 and 16-31; 128: the warp), into
+// the k-step's block xb + kt * blob_bytes, laid out as a stage of the fused kernel holds it:
+//   limbs  [16-k block c = 0..7][row n = j * RR + m][16 bytes]: limb j of batch row m, the K-major MMA operand
+//          (8-row x 16-byte core matrices); rows n >= 3 RR are zero
+//   meta   [128 / GROUP][2][meta_rows(RR)] floats: 2^(E-21), then sum_k x_int (as a float)
+//   xt     [128][RR] floats, 16-byte chunks XOR-swizzled by k (xt_swizzle)
 // Rows m >= M are written as zeros.  A group with a non-finite activation gets the scale NaN.
 template <int RR, int GROUP>
-__global__ void __launch_bounds__(128) fq_prep_x_kernel(const uint16_t* __restrict__ X, uint32_t M, uint32_t K, int8_t* __restrict__ xl,
-                                                        float* __restrict__ xmeta, float* __restrict__ xt) {
-    constexpr int GPS = kBK / GROUP, RM = meta_rows(RR);
+__global__ void __launch_bounds__(128) fq_prep_x_kernel(const uint16_t* __restrict__ X, uint32_t M, uint32_t K, uint8_t* __restrict__ xb) {
+    constexpr int GPS = kBK / GROUP, RM = meta_rows(RR), NMMA = nmma_rows(RR);
     // the grid after this one (the fused kernel) may start streaming weights; this one reads X and writes
     // scratch that the grid before it may still be using
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -162,6 +171,7 @@ __global__ void __launch_bounds__(128) fq_prep_x_kernel(const uint16_t* __restri
     const uint32_t KT = K / kBK;
     if (wg >= RR * KT) return;
     const uint32_t m = wg / KT, kt = wg - m * KT, k0 = kt * kBK + 4 * lane;
+    uint8_t* blob = xb + (size_t)kt * blob_bytes(RR, GPS);
     uint2 raw = make_uint2(0, 0);
     if (m < M) raw = __ldg(reinterpret_cast<const uint2*>(X + (size_t)m * K + k0));
     const uint32_t bits[4] = {raw.x & 0xffffu, raw.x >> 16, raw.y & 0xffffu, raw.y >> 16};
@@ -191,15 +201,27 @@ __global__ void __launch_bounds__(128) fq_prep_x_kernel(const uint16_t* __restri
         w[1] |= (uint32_t)(l1 & 0xff) << (8 * i);
         w[2] |= (uint32_t)(l2 & 0xff) << (8 * i);
     }
+    // Byte position of k inside its 16-k block: the unpack's two masks put row r of an 8-row word at position
+    // 2 (r % 4) + r / 4 of the word's eight (rows 0, 4, 1, 5, 2, 6, 3, 7), and the MMA pairs operand bytes by
+    // position.  This lane's four k are rows 4 (lane % 2) .. of 8-row word lane / 2.
+    uint8_t* lrow = blob + (lane >> 2) * (NMMA * 16) + ((lane >> 1) & 1) * 8 + (lane & 1);
 #pragma unroll
-    for (int j = 0; j < kLimbs; ++j) *reinterpret_cast<uint32_t*>(xl + (size_t)(j * RR + m) * K + k0) = w[j];
+    for (int j = 0; j < kLimbs; ++j)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) lrow[(j * RR + m) * 16 + 2 * i] = (uint8_t)(w[j] >> (8 * i));
+    if (m == 0) {
+#pragma unroll
+        for (int n = kLimbs * RR; n < NMMA; ++n)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) lrow[n * 16 + 2 * i] = 0;          // padding rows of the operand
+    }
     if ((lane & (32 / GPS - 1)) == 0) {
         const uint32_t gi = lane / (32 / GPS);
-        float* mt = xmeta + ((size_t)kt * GPS + gi) * 2 * RM;
+        float* mt = reinterpret_cast<float*>(blob + blob_meta_off(RR)) + gi * 2 * RM;
         mt[m] = ef_raw == 0xffu ? __uint_as_float(0x7fc00000u) : __uint_as_float((ef - 21u) << 23);     // 2^(E-21)
         mt[RM + m] = (float)sum;
     }
-    char* xtu = reinterpret_cast<char*>(xt) + (size_t)kt * (kBK * RR * 4);
+    uint8_t* xtu = blob + blob_xt_off(RR, GPS);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const uint32_t k = 4 * lane + i;
@@ -209,28 +231,37 @@ __global__ void __launch_bounds__(128) fq_prep_x_kernel(const uint16_t* __restri
 
 // ----------------------------------------------------------------------------- the fused kernel
 
+// Sets of epilogue warps; with two, the sets take alternate units (set e the units in D buffer e) and set 1
+// hands its sums to set 0 through shared memory at the end of a piece.  An epilogue thread's work on a unit is
+// a chain of latencies (barrier, tensor-memory load, packet, activation row, multiply-add) of 0.6-1.2 us;
+// two warps per strip keep two such chains in flight.
+__host__ __device__ constexpr int epilogue_sets(int rr) { return rr <= 16 ? 2 : 1; }
+
 constexpr int kTcFirstUnpack = 4;  // a warp reaches the tensor-memory lanes 32 * (warp % 4) ..., so strips start at a multiple of 4
 
 // BN: tile columns (128 or 256).  RR: batch rows kept per epilogue thread (1, 4, 8, 16, 32; M <= RR).  The
 // MMA's N is NMMA = kLimbs * RR rounded up to 16.  HOT: general form of the outlier step (buckets with a tail,
-// tiles with more packets than a stage holds).  tmX: tiled view of the limb array as (16 consecutive k, limb
-// row, block of 16 k), so that a box of (16, NMMA, 8) is a unit's K-major MMA operand.
+// tiles with more packets than a stage holds).
 template <int BN, int RR, int GROUP, bool SPARSE, bool HOT>
-__global__ void __launch_bounds__(32 * (kTcFirstUnpack + 2 * (BN / 32)), 1)
-fq_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmX) {
+__global__ void __launch_bounds__(32 * (kTcFirstUnpack + (1 + epilogue_sets(RR)) * (BN / 32)), 1) fq_tc_kernel(const Params p) {
     constexpr int NDW = BN / 32;              // unpack warps = epilogue warps = 32-column strips
     constexpr int NT128 = BN / 128;           // 128-column halves per unit
     constexpr int UW0 = kTcFirstUnpack, EW0 = UW0 + NDW;
+    constexpr int NEPI = epilogue_sets(RR);
     constexpr int GPS = kBK / GROUP;          // groups per k-step
-    constexpr int NMMA = (kLimbs * RR + 15) / 16 * 16;
+    constexpr int NMMA = nmma_rows(RR);
     constexpr int RM = meta_rows(RR);
     constexpr int DCOLS = GPS * NMMA;         // accumulator columns per half and buffer
-    constexpr uint32_t D_BASE = 2 * NT128 * 32;
+    // A buffers (one unit's codes each): four if tensor memory has room beside the two D buffers, so that the
+    // unpack warps run up to three units ahead of the MMAs; else two
+    constexpr int NAB = (4 * NT128 * 32 + 2 * NT128 * DCOLS <= 512) ? 4 : 2;
+    constexpr uint32_t D_BASE = NAB * NT128 * 32;
     constexpr int W_BYTES = 16 * BN * 4;
     constexpr int SZ_ROW = BN * 2;
-    constexpr int X_BYTES = NMMA * 128, META_BYTES = GPS * 2 * RM * 4, XT_BYTES = SPARSE ? kBK * RR * 4 : 0;
+    // what a stage takes of the k-step's activation block: without outliers, not the FP32 copy at its end
+    constexpr int XB_BYTES = SPARSE ? blob_bytes(RR, GPS) : blob_xt_off(RR, GPS);
     constexpr uint32_t IDESC = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NMMA >> 3) << 17) | (8u << 24);
-    static_assert(D_BASE + 2 * NT128 * DCOLS <= 512, "tensor memory: two A buffers and two D buffers must fit");
+    static_assert(D_BASE + 2 * NT128 * DCOLS <= 512, "tensor memory: the A buffers and two D buffers must fit");
     static_assert(RR == 1 || RR % 4 == 0, "rows per thread");
     extern __shared__ __align__(128) uint8_t smem[];
 
@@ -238,22 +269,30 @@ fq_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmX) {
     const uint32_t S = p.stages;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_bar);
     const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * S;
-    const uint32_t bar_go = bar_empty + 8 * S;           // [2] A buffer written (unpack warps) and D buffer free (epilogue warps)
-    const uint32_t bar_d_ready = bar_go + 16;            // [2] MMAs of a unit complete (D written, A read)
+    const uint32_t bar_a_full = bar_empty + 8 * S;       // [4] A buffer written (unpack warps)
+    const uint32_t bar_a_empty = bar_a_full + 32;        // [4] the MMAs that read the A buffer are complete
+    const uint32_t bar_d_free = bar_a_empty + 32;        // [2] D buffer read (epilogue warps)
+    const uint32_t bar_d_ready = bar_d_free + 16;        // [2] MMAs of a unit complete: D written
     const uint32_t bar_final = bar_d_ready + 16;
-    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 2 * S + 5);
+    const uint32_t bar_xfull = bar_final + 8, bar_xempty = bar_xfull + 8 * NDW;   // [NDW] each: hand-over of set 1's sums, per strip
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(bars + 2 * S + 13 + 2 * NDW);
     volatile uint32_t* tmem_slot = abort_flag + 1;
 
     if (tid == 0) {
         for (uint32_t s = 0; s < S; ++s) {
-            mbar_init(bar_full + 8 * s, 1);                    // the producer's expect_tx arrival
+            mbar_init(bar_full + 8 * s, 2);                    // the two producers' expect_tx arrivals
             mbar_init(bar_empty + 8 * s, 2 * NDW + 1);         // unpack warps, epilogue warps, the MMAs' commit
         }
         for (uint32_t b = 0; b < 2; ++b) {
-            mbar_init(bar_go + 8 * b, 2 * NDW);                // unpack warps (A of this unit), epilogue warps (D of the unit two before)
+            mbar_init(bar_d_free + 8 * b, NDW);                // the epilogue warps of the unit two before
             mbar_init(bar_d_ready + 8 * b, 1);
         }
+        for (uint32_t a = 0; a < 4; ++a) {
+            mbar_init(bar_a_full + 8 * a, NDW);
+            mbar_init(bar_a_empty + 8 * a, 1);
+        }
         mbar_init(bar_final, 1);
+        for (uint32_t i = 0; i < 2 * NDW; ++i) mbar_init(bar_xfull + 8 * i, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -286,15 +325,37 @@ fq_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmX) {
     }
 
     if (warp == 0) {
-        // ------------------------------------------------------------------ producer
-        // Lane l issues copy number l of a unit (issuing a bulk copy occupies its thread for a few hundred
-        // cycles): 0 codes, 1.. scales, then zero-points, bucket descriptors, packets; then the activation
-        // arrays: limbs, sums, FP32 copy.
-        constexpr int L_INFO = 1 + 2 * GPS, L_PK = L_INFO + 1, L_X = L_INFO + 2, L_META = L_X + 1, L_XT = L_X + 2;
+        // ------------------------------------------------------------------ producer of the dense arrays
+        // codes, scales and zero-points of every unit: weights, which no kernel writes while calls are in
+        // flight, so this warp never waits for the grids before this one
         uint32_t issued = 0;
         bool ok = true;
+        for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
+            const uint32_t s = w.s, full = bar_full + 8 * s;
+            if (!warp_wait(bar_empty + 8 * s, w.ph ^ 1, abort_flag, p.status)) { ok = false; break; }
+            const uint32_t st = smem_u32(smem) + s * p.stage_bytes;
+            if (lane == 0) {
+                mbar_arrive_expect_tx(full, W_BYTES + 2 * GPS * SZ_ROW);
+                bulk_g2s(st, p.wq + (size_t)w.u * W_BYTES, W_BYTES, full);
+#pragma unroll
+                for (int gi = 0; gi < GPS; ++gi) {
+                    const size_t row = (size_t)(w.kt * GPS + gi) * p.N + (size_t)w.tn * BN;
+                    bulk_g2s(st + p.off_sz + gi * SZ_ROW, p.scale + row, SZ_ROW, full);
+                    bulk_g2s(st + p.off_sz + (GPS + gi) * SZ_ROW, p.zero + row, SZ_ROW, full);
+                }
+            }
+            issued = w.it + 1;
+        }
+        if (!ok) {   // giving up: let the copies already issued land before the CTA's shared memory goes away
+            for (uint32_t j = (issued > S ? issued - S : 0); j < issued; ++j)
+                for (uint32_t spin = 0; spin < (1u << 20) && !mbar_try_wait(bar_full + 8 * (j % S), (j / S) & 1); ++spin) {}
+        }
+    } else if (warp == 2) {
+        // ------------------------------------------------------------------ producer of the outlier arrays and the activations
         uint32_t ip_a = 0, ip_b = 0;                                   // packet ranges of the next 32 units, read 32 at a time
-        auto weights = [&](const UnitIter& w) {                        // the weight arrays of a unit
+        uint32_t last_bar = 0, last_ph = 0;
+        bool ok = true;
+        auto outliers = [&](const UnitIter& w, uint32_t extra) {       // arrival with the byte count of this warp's copies
             const uint32_t s = w.s, full = bar_full + 8 * s;
             const uint32_t st = smem_u32(smem) + s * p.stage_bytes;
             if (SPARSE && (w.it & 31) == 0) {
@@ -307,79 +368,70 @@ fq_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmX) {
                 pk0 = __shfl_sync(0xffffffffu, ip_a, w.it & 31);
                 npk = min(__shfl_sync(0xffffffffu, ip_b, w.it & 31) - pk0, p.coo_cap);
             }
-            if (lane == 0)
-                mbar_arrive_expect_tx(full, W_BYTES + 2 * GPS * SZ_ROW + X_BYTES + META_BYTES + XT_BYTES + (SPARSE ? p.NB * 4 + npk * 16 : 0));
-            __syncwarp();
             if (lane == 0) {
-                bulk_g2s(st, p.wq + (size_t)w.u * W_BYTES, W_BYTES, full);
-            } else if (lane <= GPS) {
-                const int gi = lane - 1;
-                bulk_g2s(st + p.off_sz + gi * SZ_ROW, p.scale + (size_t)(w.kt * GPS + gi) * p.N + (size_t)w.tn * BN, SZ_ROW, full);
-            } else if (lane <= 2 * GPS) {
-                const int gi = lane - 1 - GPS;
-                bulk_g2s(st + p.off_sz + (GPS + gi) * SZ_ROW, p.zero + (size_t)(w.kt * GPS + gi) * p.N + (size_t)w.tn * BN, SZ_ROW, full);
-            } else if (SPARSE && lane == L_INFO) {
-                bulk_g2s(st + p.off_info, p.info + (size_t)w.u * p.NB, p.NB * 4, full);
-            } else if (SPARSE && lane == L_PK) {
-                if (npk) bulk_g2s(st + p.off_coo, p.packed + pk0, npk * 16, full);
+                mbar_arrive_expect_tx(full, extra + (SPARSE ? p.NB * 4 + npk * 16 : 0));
+                if (SPARSE) {
+                    bulk_g2s(st + p.off_info, p.info + (size_t)w.u * p.NB, p.NB * 4, full);
+                    if (npk) bulk_g2s(st + p.off_coo, p.packed + pk0, npk * 16, full);
+                }
             }
+            last_bar = full, last_ph = w.ph;
         };
-        auto activations = [&](const UnitIter& w) {                    // the activation arrays of its k-step
-            const uint32_t full = bar_full + 8 * w.s;
-            const uint32_t st = smem_u32(smem) + w.s * p.stage_bytes;
-            if (lane == L_X) tma_load_3d(st + p.off_xcan, &tmX, 0, 0, w.kt * 8, full);
-            else if (lane == L_META) bulk_g2s(st + p.off_xmeta, p.xmeta + (size_t)w.kt * (META_BYTES / 4), META_BYTES, full);
-            else if (SPARSE && lane == L_XT) bulk_g2s(st + p.off_xt, reinterpret_cast<const char*>(p.xt) + (size_t)w.kt * XT_BYTES, XT_BYTES, full);
+        auto activations = [&](const UnitIter& w) {                    // the k-step's block, as the preparation kernel laid it out
+            if (lane == 0)
+                bulk_g2s(smem_u32(smem) + w.s * p.stage_bytes + p.off_xcan, p.xblob + (size_t)w.kt * blob_bytes(RR, GPS), XB_BYTES, bar_full + 8 * w.s);
         };
-        // the first pass over the ring finds every stage empty: its weight copies go out before the wait
-        // for the grids before this one, its activation copies after
+        // the first pass over the ring finds every stage empty: its outlier arrays (weights) are requested
+        // before the wait for the grids before this one, its activation blocks after
         const uint32_t n_first = min(S, u_end - u_begin);
         {
             UnitIter w(u_begin, KT);
-            for (uint32_t i = 0; i < n_first; ++i, w.next(S, KT)) weights(w);
+            for (uint32_t i = 0; i < n_first; ++i, w.next(S, KT)) outliers(w, XB_BYTES);
         }
         asm volatile("griddepcontrol.wait;" ::: "memory");
         {
             UnitIter w(u_begin, KT);
             for (uint32_t i = 0; i < n_first; ++i, w.next(S, KT)) activations(w);
-            issued = n_first;
             for (; w.u < u_end; w.next(S, KT)) {
                 if (!warp_wait(bar_empty + 8 * w.s, w.ph ^ 1, abort_flag, p.status)) { ok = false; break; }
-                weights(w);
+                outliers(w, XB_BYTES);
                 activations(w);
-                issued = w.it + 1;
             }
         }
-        if (!ok) {   // giving up: let the copies already issued land before the CTA's shared memory goes away
-            for (uint32_t j = (issued > S ? issued - S : 0); j < issued; ++j)
-                for (uint32_t spin = 0; spin < (1u << 20) && !mbar_try_wait(bar_full + 8 * (j % S), (j / S) & 1); ++spin) {}
-        }
+        if (!ok && last_bar)                // gave up: let this warp's last copies land before the CTA exits
+            for (uint32_t spin = 0; spin < (1u << 20) && !mbar_try_wait(last_bar, last_ph); ++spin) {}
     } else if (warp == 1) {
         // ------------------------------------------------------------------ tensor warp
         // One warp issues every MMA of the CTA (issued from two warps in turn, MMAs run several times slower).
-        // The issue of an MMA blocks while the one before it runs, so the warp looks at the next unit's
-        // barriers between the MMAs of this one: their latency then hides behind MMAs in flight, and a unit
-        // whose operands are ready is issued without waiting at all.
         // The first MMA of a CTA takes microseconds to start (the tensor pipe wakes up): issue a throw-away
         // one now, while the first loads are in flight.  It reads whatever A buffer 0 and stage 0 hold and
         // writes D buffer 1, which the first real MMA into that buffer overwrites.
         umma_i8_ts(tmem_base + D_BASE + NT128 * DCOLS, tmem_base, make_b_desc(smem_u32(smem) + p.off_xcan, NMMA * 16, 128), IDESC, 0);
-        uint32_t ready = 0;                          // this unit's barriers were seen complete already
+        // The tensor pipe should never wait for this warp: the completion signals of a unit go out after the
+        // first MMA of the next one has been issued (they then fire one MMA, about 30 ns, later), and the next
+        // unit's barriers are tested while the last MMAs of this one run.
+        uint32_t ready = 0, pending = 0, pv_b = 0, pv_a = 0, pv_s = 0;
+        auto signal = [&]() {                                  // completion of the unit before: D written, A and stage read
+            if (pending) {
+                umma_commit(bar_d_ready + 8 * pv_b);
+                umma_commit(bar_a_empty + 8 * pv_a);
+                umma_commit(bar_empty + 8 * pv_s);
+                pending = 0;
+            }
+        };
         for (UnitIter w(u_begin, KT); w.u < u_end; w.next(S, KT)) {
-            const uint32_t it = w.it, s = w.s, b = w.it & 1;    // A buffer b and D buffer b
+            const uint32_t it = w.it, s = w.s, b = w.it & 1;    // D buffer b, A buffer it % NAB
             if (!ready) {
-                if (!warp_wait(bar_full + 8 * s, w.ph, abort_flag, p.status)) break;       // the activation operand
-                if (!warp_wait(bar_go + 8 * b, (it >> 1) & 1, abort_flag, p.status)) break;
+                // the stage's activation operand, the unit's A buffer, and the D buffer's last reader
+                signal();
+                if (!warp_wait(bar_full + 8 * s, w.ph, abort_flag, p.status)) break;
+                if (!warp_wait(bar_a_full + 8 * (it % NAB), (it / NAB) & 1, abort_flag, p.status)) break;
+                if (it >= 2 && !warp_wait(bar_d_free + 8 * b, ((it - 2) >> 1) & 1, abort_flag, p.status)) break;
             }
             tc_fence_after();
             UnitIter nx = w;
             nx.next(S, KT);
-            const bool has_next = nx.u < u_end;
             uint32_t seen = 0;
-            auto poll = [&]() {
-                if (has_next && lane == 0 && !seen)
-                    seen = mbar_test_wait(bar_full + 8 * nx.s, nx.ph) & mbar_test_wait(bar_go + 8 * (nx.it & 1), (nx.it >> 1) & 1);
-            };
             const uint64_t bd0 = make_b_desc(smem_u32(smem) + s * p.stage_bytes + p.off_xcan, NMMA * 16, 128);
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks) {             // 32 k per MMA: 16-k blocks 2 ks, 2 ks + 1 of the operand
@@ -387,16 +439,18 @@ fq_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmX) {
 #pragma unroll
                 for (int h = 0; h < NT128; ++h) {
                     const uint32_t d = tmem_base + D_BASE + (b * NT128 + h) * DCOLS + gi * NMMA;
-                    const uint32_t a = tmem_base + (b * NT128 + h) * 32 + ks * 8;
+                    const uint32_t a = tmem_base + ((it % NAB) * NT128 + h) * 32 + ks * 8;
                     umma_i8_ts(d, a, bd0 + (uint64_t)((ks * 2 * NMMA * 16) >> 4), IDESC, (ks % (4 / GPS)) != 0);
+                    if (ks == 0 && h == 0) signal();
                 }
-                if (ks == 1 || ks == 2) poll();
+                if (ks == 2 && nx.u < u_end && lane == 0)   // one lane, three tests whose latencies overlap
+                    seen = mbar_test_wait(bar_full + 8 * nx.s, nx.ph) & mbar_test_wait(bar_a_full + 8 * (nx.it % NAB), (nx.it / NAB) & 1) &
+                           (nx.it < 2 ? 1u : mbar_test_wait(bar_d_free + 8 * (nx.it & 1), ((nx.it - 2) >> 1) & 1));
             }
-            umma_commit(bar_d_ready + 8 * b);   // this unit's sums are complete and its A buffer has been read
-            umma_commit(bar_empty + 8 * s);     // and so has the stage's activation operand
-            poll();
+            pending = 1, pv_b = b, pv_a = it % NAB, pv_s = s;
             ready = __shfl_sync(0xffffffffu, seen, 0);
         }
+        signal();
         __syncwarp();
         umma_commit(bar_final);                 // fires when every MMA this warp issued has retired
     } else if (warp < UW0) {
@@ -416,8 +470,8 @@ fq_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmX) {
             uint4 w4[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) w4[j] = wp[j * BN];
-            // the A buffer of this parity was last read by the MMAs of unit it - 2
-            if (it >= 2 && !warp_wait(bar_d_ready + 8 * b, ((it - 2) >> 1) & 1, abort_flag, p.status)) break;
+            // this A buffer was last read by the MMAs of unit it - NAB
+            if (it >= NAB && !warp_wait(bar_a_empty + 8 * (it % NAB), ((it - NAB) / NAB) & 1, abort_flag, p.status)) break;
             tc_fence_after();
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
@@ -425,36 +479,43 @@ fq_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmX) {
                 uint32_t a[8];
 #pragma unroll
                 for (int x = 0; x < 4; ++x) {
-                    // even nibbles are rows 0-3 of the word's eight, odd nibbles rows 4-7: two cells of four bytes
+                    // nibble i + 4h of a word is row 2i + h of its eight: the even nibbles are rows 0, 4, 1, 5 and the
+                    // odd ones rows 2, 6, 3, 7, two cells of four bytes; the limb operand is stored in the same k order
                     a[2 * x + 0] = ww[x] & 0x0f0f0f0fu;
                     a[2 * x + 1] = (ww[x] >> 4) & 0x0f0f0f0fu;
                 }
-                tmem_st8(t_a + b * (NT128 * 32) + j * 8, a);
+                tmem_st8(t_a + (it % NAB) * (NT128 * 32) + j * 8, a);
             }
             tmem_wait_st();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive_relaxed(bar_go + 8 * b);
+                mbar_arrive_relaxed(bar_a_full + 8 * (it % NAB));
                 mbar_arrive_relaxed(bar_empty + 8 * s);
             }
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps: thread = column
-        const int dw = warp - EW0;
+        const int ew = warp - EW0, es = ew / NDW, dw = ew % NDW;     // set es (its units: it % NEPI == es), strip dw
         const int col = dw * 32 + lane;
         const uint32_t g = lane & 7, t = lane >> 3;          // bucket of the strip, column number in the bucket
         const uint32_t t_lane = ((uint32_t)((dw & 3) * 32)) << 16;
         const uint32_t t_d = tmem_base + t_lane + D_BASE + (uint32_t)(dw >> 2) * DCOLS;
+        float* xch = reinterpret_cast<float*>(smem + p.off_xch) + dw * (RR * 32) + lane;     // hand-over slot of this column
         float accf[RR];
 #pragma unroll
         for (int i = 0; i < RR; ++i) accf[i] = 0.0f;
         bool ok = true;
-        // both D buffers start free: this warp's share of the first two units' go-ahead
-        if (lane == 0) { mbar_arrive_relaxed(bar_go); mbar_arrive_relaxed(bar_go + 8); }
-        for (UnitIter w(u_begin, KT); w.u < u_end && ok; w.next(S, KT)) {
+        // outer loop: the pieces of this CTA's range (a piece = its units of one column tile); inner loop: this
+        // set's units of the piece
+        UnitIter w(u_begin, KT);
+        if (es == 1) w.next(S, KT);
+        uint32_t tn = u_begin / KT, piece = 0;
+        for (uint32_t piece_first = u_begin; piece_first < u_end && ok; ++tn, ++piece) {
+          const uint32_t piece_stop = min(u_end, (tn + 1) * KT);        // one past the piece's last unit
+          piece_first = piece_stop;
+          for (; w.u < piece_stop; w.next(S, KT), (NEPI == 2 ? w.next(S, KT) : (void)0)) {
             const uint32_t u = w.u, it = w.it, s = w.s, b = w.it & 1;
-            const uint32_t tn = w.tn, kt = w.kt;
             const uint8_t* st = smem + s * p.stage_bytes;
             if (!warp_wait(bar_full + 8 * s, w.ph, abort_flag, p.status)) { ok = false; break; }
             // outliers: the bucket descriptor and this lane's slots of the first packets are requested now
@@ -499,33 +560,33 @@ fq_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmX) {
 #pragma unroll
             for (int gi = 0; gi < GPS; ++gi) {
                 // sum_k x (q - z) = 2^(E-21) * (D0 + 2^8 D1 + 2^16 D2 - z sum_k x_int), D_j = sum_k q l_j exact in INT32
-                float dl[kLimbs][RR];
                 if constexpr (RR == 1) {
                     uint32_t c[4];                                  // one load of four cells covers the three limbs of the single row
                     tmem_ld<4>(t_d + b * (NT128 * DCOLS) + gi * NMMA, c);
                     tmem_wait_ld();
-#pragma unroll
-                    for (int j = 0; j < kLimbs; ++j) dl[j][0] = (float)(int)c[j];
+                    const float f = fmaf(zv[gi], meta[gi * 2 * RM + RM],
+                                         fmaf(small_int_to_float(c[2]), 65536.0f, fmaf(small_int_to_float(c[1]), 256.0f, small_int_to_float(c[0]))));
+                    accf[0] = fmaf(sv[gi] * meta[gi * 2 * RM], f, accf[0]);
                 } else {
-                    uint32_t c[kLimbs][RR];
 #pragma unroll
-                    for (int j = 0; j < kLimbs; ++j) tmem_ld<RR>(t_d + b * (NT128 * DCOLS) + gi * NMMA + j * RR, c[j]);
-                    tmem_wait_ld();
+                    for (int i0 = 0; i0 < RR; i0 += 8 < RR ? 8 : RR) {     // eight rows at a time (four with RR = 4)
+                        constexpr int CH = 8 < RR ? 8 : RR;
+                        uint32_t c[kLimbs][CH];
 #pragma unroll
-                    for (int j = 0; j < kLimbs; ++j)
+                        for (int j = 0; j < kLimbs; ++j) tmem_ld<CH>(t_d + b * (NT128 * DCOLS) + gi * NMMA + j * RR + i0, c[j]);
+                        tmem_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < RR; ++i) dl[j][i] = (float)(int)c[j][i];
-                }
-#pragma unroll
-                for (int i = 0; i < RR; ++i) {
-                    const float xs = meta[gi * 2 * RM + i], sx = meta[gi * 2 * RM + RM + i];
-                    const float f = fmaf(zv[gi], sx, fmaf(dl[2][i], 65536.0f, fmaf(dl[1][i], 256.0f, dl[0][i])));
-                    accf[i] = fmaf(sv[gi] * xs, f, accf[i]);
+                        for (int i = 0; i < CH; ++i) {
+                            const float xs = meta[gi * 2 * RM + i0 + i], sx = meta[gi * 2 * RM + RM + i0 + i];
+                            const float f = fmaf(zv[gi], sx, fmaf(small_int_to_float(c[2][i]), 65536.0f, fmaf(small_int_to_float(c[1][i]), 256.0f, small_int_to_float(c[0][i]))));
+                            accf[i0 + i] = fmaf(sv[gi] * xs, f, accf[i0 + i]);
+                        }
+                    }
                 }
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive_relaxed(bar_go + 8 * b);         // the MMAs of unit it + 2 may overwrite this D buffer
+            if (lane == 0) mbar_arrive_relaxed(bar_d_free + 8 * b);     // the MMAs of unit it + 2 may overwrite this D buffer
             if (SPARSE) {
                 // ---- the unit's outliers of this thread's column (padding slots have value 0: they add 0)
                 for (uint32_t i = 0; i < cmax; i += NP) {
@@ -572,9 +633,27 @@ fq_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmX) {
             }
             __syncwarp();
             if (lane == 0) mbar_arrive_relaxed(bar_empty + 8 * s);
-
-            if (kt == KT - 1 || u == u_end - 1) {
+          }
+          if (!ok) break;
+          {
                 // ---------------------------------------------------------- end of a piece
+                if (NEPI == 2) {
+                    if (es == 1) {
+                        // hand the sums over (after set 0 has taken the previous piece's) and start afresh
+                        if (piece > 0 && !warp_wait(bar_xempty + 8 * dw, (piece - 1) & 1, abort_flag, p.status)) { ok = false; break; }
+#pragma unroll
+                        for (int mm = 0; mm < RR; ++mm) { xch[mm * 32] = accf[mm]; accf[mm] = 0.0f; }
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar_xfull + 8 * dw);
+                        continue;
+                    }
+                    if (!warp_wait(bar_xfull + 8 * dw, piece & 1, abort_flag, p.status)) { ok = false; break; }
+#pragma unroll
+                    for (int mm = 0; mm < RR; ++mm) accf[mm] += xch[mm * 32];
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_xempty + 8 * dw);
+                }
+                const uint32_t kt = piece_stop - 1 - tn * KT;               // k-step of the piece's last unit
                 const uint32_t u_tile0 = tn * KT;
                 const uint32_t piece_k0 = max(u_tile0, u_begin) - u_tile0;
                 const bool full_piece = (piece_k0 == 0) && (kt == KT - 1);
@@ -633,7 +712,7 @@ fq_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmX) {
                 }
 #pragma unroll
                 for (int mm = 0; mm < RR; ++mm) accf[mm] = 0.0f;
-            }
+          }
         }
     }
 

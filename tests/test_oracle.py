@@ -251,7 +251,8 @@ def test_decode_wq_against_a_direct_packer():
         kt, kr = divmod(row, 128)
         j, r32 = divmod(kr, 32)
         w, r8 = divmod(r32, 8)
-        nib = 2 * r8 if r8 < 4 else 2 * (r8 - 4) + 1
+        i, h = divmod(r8, 2)
+        nib = i + 4 * h
         for col in range(N):
             tn, t = divmod(col, BN)
             idx = (tn * KT + kt) * 16 * BN + (j * BN + t) * 4 + w

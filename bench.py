@@ -327,7 +327,7 @@ def run_ours(args):
             c = w["copies"][w["turn"] % len(w["copies"])]
             w["turn"] += 1
             fq.fq_unfused_gemm(w["L"], w["Xd"][M], M, c["wq"], c["scale"], c["zero"], w["Yd"][M], ws, stream)
-            fq.fq_unfused_spmm(w["L"], w["Xd"][M], M, c["indptr"], c["info"], c["packed"], w["Yd"][M], stream)
+            fq.fq_unfused_spmm(w["L"], w["Xd"][M], M, c["indptr"], c["info"], c["packed"], w["Yd"][M], ws, stream)
 
         us_f = time_loop(fused, reps)
         us_u = time_loop(unfused, reps)
@@ -484,7 +484,7 @@ def run_sweep(args):
                 c = copies[turn[0] % len(copies)]
                 turn[0] += 1
                 fq.fq_unfused_gemm(L, X, M, c["wq"], c["scale"], c["zero"], Y, ws, stream)
-                fq.fq_unfused_spmm(L, X, M, c["indptr"], c["info"], c["packed"], Y, stream)
+                fq.fq_unfused_spmm(L, X, M, c["indptr"], c["info"], c["packed"], Y, ws, stream)
 
             nbytes = algorithmic_bytes(K, N, g, lay.nnz, n_tile, n_tile * L.buckets_per_tile, M)
             us_f, us_u = time_loop(fused), time_loop(unfused)

@@ -28,18 +28,20 @@
  *   INT4 weights.  BK = 128 rows, BN = 128 or 256 columns per tile.  The buffer
  *   is a sequence of chunks, one per (column tile tn, row tile kt), chunk index
  *   tn * (K/128) + kt, each 16 * BN little-endian 32-bit words.  Word index
- *   inside a chunk, with integer division, is
- *       (((j*(BN/32) + t/32)*8 + t%8)*4 + w)*4 + (t/8)%4
+ *   inside a chunk is
+ *       (j*BN + t)*4 + w
  *   (j = 0..3: 32-row block, t = column inside the tile, w = 0..3: 8-row
  *   block).  Nibble p = i + 4h (i = 0..3, h = 0..1; bits 4p..4p+3) of that
  *   word is the code of
  *       column tn*BN + t
  *       row    kt*128 + 32j + 8w + 2i + h .
- *   (Inside a 32-row by 32-column block, the words of columns g, g+8, g+16,
- *   g+24 and one 8-row block are 16 contiguous bytes: what one lane of the
- *   small-batch kernel feeds to its m16n8k16 MMAs, fetched with one 128-bit
- *   load.  One shift-and-mask turns nibbles i and i+4 of a word into a BF16
- *   pair of consecutive rows: the operand order of both tensor-core paths.)
+ *   (The four words of a column's 32-row block are 16 contiguous bytes, and
+ *   consecutive columns follow each other: a thread that owns a column fetches
+ *   them with one 128-bit load, a warp without bank conflicts.  One
+ *   shift-and-mask turns nibbles i and i+4 of a word into a BF16 pair of
+ *   consecutive rows, the operand order of the warp-level MMA; one mask each
+ *   turns the even and the odd nibbles into four bytes, the operand of the
+ *   integer MMA.)
  *
  *   Scale, zero.  (K/group) x N row-major BF16.  zero holds the integer 0..15.
  *
@@ -188,30 +190,32 @@ fq_status_t fq_validate_tilecoo(const fq_layout_t* L, const uint32_t* tile_indpt
 fq_status_t fq_workspace_bytes(const fq_layout_t* L, uint32_t M, size_t* bytes);
 
 /*
- * The fused operator (Eq. 1; Sections 3.1 and 4.1): one launch per 32 rows of X
- * reads X, W_Q and the Tile-COO tiles through a bulk-copy/mbarrier ring,
- * dequantises in registers into tensor-core operands, applies the tile's
- * outliers against the same shared-memory activation tile, and writes Y once.
- * The default kernel uses warp-level MMAs and adds the outliers in registers.
- * Environment variable FQ_ENGINE=tc routes every call to the library's
- * tcgen05 kernel instead (tensor-memory operand, outliers through a
- * shared-memory FP32 tile, 32 rows per launch), FQ_ENGINE=mix only calls with
- * M > 16; as it stands that kernel is the slower one at every M.
+ * The fused operator (Eq. 1; Sections 3.1 and 4.1): a launch reads X, W_Q and
+ * the Tile-COO tiles through a bulk-copy/mbarrier ring, dequantises in
+ * registers into tensor-core operands, applies the tile's outliers against the
+ * activation tile in shared memory, and writes Y once.  Up to 16 rows of X go
+ * through one launch of a kernel built on warp-level MMAs (exact integers
+ * 128 + q in BF16, scale and zero-point applied per group in FP32).  Larger M
+ * is served in launches of up to 32 rows by a kernel built on tcgen05.mma with
+ * 8-bit integer operands (groups of 128; groups of 64 stay with launches of
+ * 16 rows): its activations are block fixed point, 22 bits plus sign relative
+ * to the largest |x| of each row and group, so activations more than 2^14
+ * below that maximum are rounded (to 2^-22 of it).  The kernel is chosen by the
+ * rows of a launch alone.
  * X: device, M x K BF16.  M in [1, FQ_MAX_M].  Y: device, M x N BF16,
  * overwritten.  All other arrays: device copies of the host packer/encoder
  * output.  Work is split over persistent CTAs by (tile, k-step) units; tiles
  * shared by several CTAs are summed in a fixed order, so results are run-to-run
  * reproducible.
  *
- * Ordering.  The small-batch kernel is launched so that it may become resident
- * while the kernel before it in the stream is still draining (programmatic
- * dependent launch): it then already streams the weight arrays (wq, scale,
- * zero, tile_indptr, bucket_info, packed_outliers), and touches X, Y and the
- * scratch only after that earlier kernel has completed.  So the weight arrays
- * must not be written by a kernel that can still be running when this call is
- * made (they are constants of the layer in any real use); every other
- * dependency through the stream is honoured as usual.  Environment variable
- * FQ_PDL=0 restores plain stream order.
+ * Ordering.  Every kernel is launched so that it may become resident while the
+ * kernel before it in the stream is still draining (programmatic dependent
+ * launch): it then already streams the weight arrays (wq, scale, zero,
+ * tile_indptr, bucket_info, packed_outliers), and touches X, Y and the scratch
+ * only after that earlier kernel has completed.  So the weight arrays must not
+ * be written by a kernel that can still be running when this call is made
+ * (they are constants of the layer in any real use); every other dependency
+ * through the stream is honoured as usual.
  */
 fq_status_t fq_fused_w4a16_outlier_gemm(const fq_layout_t* L, const void* X, uint32_t M,
                                         const void* wq, const void* scale, const void* zero,
@@ -232,9 +236,8 @@ fq_status_t fq_fused_w4a16_outlier_gemm(const fq_layout_t* L, const void* X, uin
  * Instead of a caller-provided workspace, the kernel uses an array that is part
  * of the library image: FQ_STATIC_SCRATCH_BYTES of device memory on every GPU
  * that loads the library, held until the process exits.  That fixes the limit:
- * calls whose fq_workspace_bytes() exceeds it (M > FQ_STATIC_SCRATCH_MAX_M with
- * 256-column tiles) are refused with FQ_ERR_BUFFER_TOO_SMALL and nothing is
- * launched.  The function calls no cudaMalloc / cudaFree and no allocating
+ * calls whose fq_workspace_bytes() exceeds it (M > FQ_STATIC_SCRATCH_MAX_M) are
+ * refused with FQ_ERR_BUFFER_TOO_SMALL and nothing is launched.  The function calls no cudaMalloc / cudaFree and no allocating
  * library routine; per call it enqueues one small memset (status word and tile
  * counters, which must start at zero) and the kernel.
  *
@@ -261,12 +264,15 @@ fq_status_t fq_unfused_gemm(const fq_layout_t* L, const void* X, uint32_t M, con
                             const void* scale, const void* zero, void* Y, void* workspace,
                             size_t workspace_bytes, void* cuda_stream);
 
-/* Unfused baseline, sparse half: Y += X * W_O as a separate launch that re-reads
- * X and read-modify-writes the BF16 Y (the two-kernel scheme the paper compares
- * against, Section 2.2). */
+/* Unfused baseline, sparse half: Y += X * W_O as a separate launch (one per 16
+ * rows) that re-reads X and read-modify-writes the BF16 Y (the two-kernel
+ * scheme the paper compares against, Section 2.2).  Column tiles are split
+ * into slabs of row tiles over the CTAs; slabs of one tile add their FP32 sums
+ * with atomic additions in the scratch (same scratch and size as the fused
+ * call, fq_workspace_bytes), so the last bits of Y may differ run to run. */
 fq_status_t fq_unfused_spmm(const fq_layout_t* L, const void* X, uint32_t M, const void* tile_indptr,
-                            const void* bucket_info, const void* packed_outliers, void* Y,
-                            void* cuda_stream);
+                            const void* bucket_info, const void* packed_outliers, void* Y, void* workspace,
+                            size_t workspace_bytes, void* cuda_stream);
 
 /* Same operator as fq_fused_w4a16_outlier_gemm, called with HOST X and HOST Y:
  * copies X to x_dev, runs the kernel, copies Y back from y_dev and waits for
@@ -290,9 +296,13 @@ fq_status_t fq_fused_host_io_async(const fq_layout_t* L, const void* X_host, uin
                                    const void* packed_outliers, void* y_dev, void* Y_host,
                                    void* workspace, size_t workspace_bytes, void* cuda_stream);
 
-/* Synchronise the stream and return the scratch's status word: FQ_OK, or
- * FQ_ERR_TIMEOUT if a bounded wait expired in a kernel (Y is then undefined);
- * the word is cleared. */
+/* Synchronise the stream and return the scratch's status word: FQ_OK,
+ * FQ_ERR_TIMEOUT if a bounded wait expired in a kernel, or FQ_ERR_FORMAT if a
+ * kernel found bucket descriptors that point outside the packets staged for
+ * their tile (a layout struct that does not belong to the uploaded arrays).  Y
+ * of such a call is undefined.  A call that gave up leaves tile-arrival
+ * counters short, so on an error this function clears the status word and all
+ * counters: the scratch is then ready for the next call. */
 fq_status_t fq_check_status(void* workspace, void* cuda_stream);
 
 /* Thread-local description of the most recent error; valid until the next call. */

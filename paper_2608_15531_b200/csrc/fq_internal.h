@@ -23,7 +23,7 @@ inline bool layout_ok(const fq_layout_t* L) {
     if (L->BK != FQ_BK || (L->BN != 128 && L->BN != 256)) return false;
     if (L->group != 64 && L->group != 128) return false;
     if (L->K == 0 || L->N == 0 || L->K % FQ_BK != 0 || L->N % L->BN != 0) return false;
-    if (L->buckets_per_tile != 32 && L->buckets_per_tile != 64 && L->buckets_per_tile != 128) return false;
+    if (L->buckets_per_tile != L->BN / 4) return false;      // a bucket is four columns, in every kernel
     if (L->wq_interleave != 3 || L->coo_unit_bytes != 16) return false;
     return true;
 }

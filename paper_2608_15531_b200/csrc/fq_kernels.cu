@@ -220,75 +220,93 @@ struct UnitIter {
 
 // ----------------------------------------------------------------------------- unfused SpMM
 
-// Y += X * W_O as its own launch (the sparse half of the two-kernel baseline).  One warp per bucket of
-// a column tile (four columns): its lanes take the row tiles kt = lane, lane + 32, ..., read the
-// bucket's packets and the activations x[m][k] from global memory (L2-resident) and add into registers
-// (4 columns x 8 batch rows per lane); a butterfly sum over the lanes and one read-modify-write of the
-// BF16 Y per element finish it.  No shared memory, no atomics: a bucket's columns belong to one warp.
+// Y += X * W_O as its own launch (the sparse half of the two-kernel baseline, Section 2.2).  One CTA per
+// (column tile, slab of k-steps), enough slabs to give every SM two CTAs; thread = output column.  Per k-step
+// the CTA stages the activations of up to 16 batch rows as a k-major FP32 tile in shared memory (the same
+// swizzled layout the fused tcgen05 kernel uses), and every thread walks the packets of its column's bucket
+// (slot t of the column-slotted packets; tail slots name their column) and multiplies-adds into RR registers.
+// With one slab a thread then updates its BF16 Y elements once.  With several, the slabs' sums meet in an FP32
+// tile of the scratch through red.global.add (the order of those additions is not fixed: this baseline is not
+// bit-reproducible run to run), and the last CTA of a tile to arrive updates Y and zeroes the FP32 tile again.
+template <int RR>
 __global__ void __launch_bounds__(256) fq_spmm_kernel(const uint16_t* __restrict__ X, const uint32_t* __restrict__ indptr,
                                                     const uint32_t* __restrict__ info, const uint4* __restrict__ packed,
-                                                    uint16_t* __restrict__ Y, uint32_t M, uint32_t K, uint32_t N,
-                                                    uint32_t BN, uint32_t NB) {
-    constexpr int MB = 8;
-    const int lane = threadIdx.x & 31;
-    const uint32_t wg = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (wg >= (N / BN) * NB) return;
-    const uint32_t tn = wg / NB, b = wg - tn * NB, KT = K / kBK;
-    const uint32_t first_col = tn * BN + (((b >> 3) << 5) | (b & 7u));      // column number c of the bucket: + 8 c
-    for (uint32_t m0 = 0; m0 < M; m0 += MB) {
-        float acc[4][MB];
+                                                    uint16_t* __restrict__ Y, float* __restrict__ accbuf,
+                                                    uint32_t* __restrict__ counters, uint32_t M, uint32_t K, uint32_t N,
+                                                    uint32_t NB, uint32_t slabs) {
+    __shared__ __align__(128) float xt[kBK * RR];
+    __shared__ uint32_t s_last;
+    const uint32_t BN = blockDim.x, KT = K / kBK;
+    const uint32_t tid = threadIdx.x, tile = blockIdx.x / slabs, slab = blockIdx.x - tile * slabs;
+    const uint32_t kt0 = slab * KT / slabs, kt1 = (slab + 1) * KT / slabs;
+    const uint32_t strip = tid >> 5, g = tid & 7, t = (tid >> 3) & 3;
+    const uint32_t bucket = strip * 8 + g;
+    const char* xtb = reinterpret_cast<const char*>(xt);
+    float acc[RR];
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
+    for (int i = 0; i < RR; ++i) acc[i] = 0.0f;
+    for (uint32_t kt = kt0; kt < kt1; ++kt) {
+        __syncthreads();
+        // the k-step's activations: pairs of consecutive k of one row per load
+        for (uint32_t e = tid; e < (uint32_t)RR * 64; e += BN) {
+            const uint32_t m = e >> 6, kp = e & 63;
+            uint32_t v = 0;
+            if (m < M) v = __ldg(reinterpret_cast<const uint32_t*>(X + (size_t)m * K + (size_t)kt * kBK) + kp);
 #pragma unroll
-            for (int m = 0; m < MB; ++m) acc[c][m] = 0.0f;
-        for (uint32_t kt = lane; kt < KT; kt += 32) {
-            const size_t t = (size_t)tn * KT + kt;
-            const uint32_t inf = __ldg(info + t * NB + b);
-            const uint4* pk = packed + __ldg(indptr + t) + (inf & 0xffffu);
-            const uint32_t depth = (inf >> 16) & 0xffu, tail = inf >> 24;
-            for (uint32_t i = 0; i < depth; ++i) {              // column-slotted: slot e is column number e
-                const uint4 q = __ldg(pk + i);
-                const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    if ((w[e] >> 16) == 0) continue;            // padding: no activation loads for it
-                    const float v = __uint_as_float(w[e] & 0xffff0000u);
-                    const uint16_t* xp = X + (size_t)m0 * K + kt * kBK + ((w[e] >> 5) & 127u);
-#pragma unroll
-                    for (int m = 0; m < MB; ++m)
-                        acc[e][m] = fmaf(v, (m0 + m < M) ? bf16_bits_to_float(__ldg(xp + (size_t)m * K)) : 0.0f, acc[e][m]);
-                }
-            }
-            for (uint32_t i = depth; i < depth + tail; ++i) {   // tail: a slot names its column
-                const uint4 q = __ldg(pk + i);
-                const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const uint32_t cls = (w[e] >> 12) & 3u;
-                    const float v = __uint_as_float(w[e] & 0xffff0000u);
-                    const uint16_t* xp = X + (size_t)m0 * K + kt * kBK + ((w[e] >> 5) & 127u);
-#pragma unroll
-                    for (int m = 0; m < MB; ++m) {
-                        const float x = (m0 + m < M) ? bf16_bits_to_float(__ldg(xp + (size_t)m * K)) : 0.0f;
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) acc[c][m] = fmaf(cls == (uint32_t)c ? v : 0.0f, x, acc[c][m]);
-                    }
-                }
+            for (int h = 0; h < 2; ++h) {
+                const uint32_t k = 2 * kp + h;
+                char* dst = reinterpret_cast<char*>(xt) + k * (4 * RR) + ((((m >> 2) ^ xt_swizzle<RR>(k)) << 4) | ((m & 3) << 2));
+                *reinterpret_cast<float*>(dst) = h ? bf16hi(v) : bf16lo(v);
             }
         }
+        __syncthreads();
+        const size_t u = (size_t)tile * KT + kt;
+        const uint32_t inf = __ldg(info + u * NB + bucket);
+        const uint32_t* pk = reinterpret_cast<const uint32_t*>(packed + __ldg(indptr + u) + (inf & 0xffffu));
+        const uint32_t depth = (inf >> 16) & 0xffu, tail = inf >> 24;
+        for (uint32_t i = 0; i < depth; ++i) {                        // column-slotted: slot t is this thread's column
+            const uint32_t w[1] = {__ldg(pk + i * 4 + t)};
+            add_outliers<RR, 1>(acc, w, xtb);
+        }
+        for (uint32_t i = depth; i < depth + tail; ++i) {             // tail: a slot names its column
+            const uint4 q4 = __ldg(reinterpret_cast<const uint4*>(pk) + i);
+            const uint32_t wd[4] = {q4.x, q4.y, q4.z, q4.w};
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
+            for (int e = 0; e < 4; ++e) {
+                const uint32_t mine[1] = {((wd[e] >> 12) & 3u) == t ? wd[e] : (wd[e] & 0xffffu)};
+                add_outliers<RR, 1>(acc, mine, xtb);
+            }
+        }
+    }
+    const size_t col = (size_t)tile * BN + tid;
+    if (slabs > 1) {
 #pragma unroll
-            for (int m = 0; m < MB; ++m) {
-                float a = acc[c][m];
+        for (int m = 0; m < RR; ++m)
+            if ((uint32_t)m < M) asm volatile("red.global.add.f32 [%0], %1;" ::"l"(accbuf + (size_t)m * N + col), "f"(acc[m]) : "memory");
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) {
+            uint32_t old;
+            asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(old) : "l"(counters + tile * 8) : "memory");
+            s_last = old == slabs - 1 ? 1u : 0u;
+            if (s_last) counters[tile * 8] = 0;                       // ready for the next call
+        }
+        __syncthreads();
+        if (!s_last) return;
+        __threadfence();
 #pragma unroll
-                for (int d = 16; d > 0; d >>= 1) a += __shfl_xor_sync(0xffffffffu, a, d);
-                if (lane == c * MB + m && m0 + m < M) {
-                    uint16_t* y = Y + (size_t)(m0 + m) * N + first_col + 8 * c;
-                    *y = float_to_bf16_bits(bf16_bits_to_float(*y) + a);
-                }
+        for (int m = 0; m < RR; ++m)
+            if ((uint32_t)m < M) {
+                acc[m] = __ldcg(accbuf + (size_t)m * N + col);
+                __stcg(accbuf + (size_t)m * N + col, 0.0f);
             }
     }
+#pragma unroll
+    for (int m = 0; m < RR; ++m)
+        if ((uint32_t)m < M) {
+            uint16_t* y = Y + (size_t)m * N + col;
+            *y = float_to_bf16_bits(bf16_bits_to_float(*y) + acc[m]);
+        }
 }
 
 // ----------------------------------------------------------------------------- launch plumbing
@@ -379,9 +397,10 @@ static fq_status_t make_plan(const fq_layout_t* L, uint32_t M, bool sparse, Plan
 }
 
 // Scratch layout: status word and header, tile-arrival counters, FP32 partial slots, then the activation
-// blocks fq_prep_x_kernel writes for the launch in flight (one per k-step).
+// blocks fq_prep_x_kernel writes for the launch in flight (one per k-step), then the FP32 tile in which the
+// slabs of the unfused SpMM meet (all zero between calls).
 struct Scratch {
-    size_t off_partials, off_xb, total;
+    size_t off_partials, off_xb, off_spmm, total;
 };
 // Which kernel serves a launch is decided by its rows alone: up to 16 rows the warp-level MMA kernel, 17 to 32
 // rows the tcgen05 kernel (its MMAs cost the same for any number of batch rows up to 42; with groups of 64 its
@@ -394,7 +413,8 @@ static Scratch scratch_layout(const fq_layout_t* L, uint32_t rows) {
     Scratch sc;
     sc.off_partials = kWsHeaderBytes + kWsCounterBytes;
     sc.off_xb = sc.off_partials + (size_t)kMaxCtas * 2 * L->BN * prow * 4;
-    sc.total = sc.off_xb + (tc ? (size_t)(L->K / kBK) * blob_bytes(32, (int)(kBK / L->group)) : 0);
+    sc.off_spmm = sc.off_xb + (tc ? (size_t)(L->K / kBK) * blob_bytes(32, (int)(kBK / L->group)) : 0);
+    sc.total = sc.off_spmm + (size_t)16 * L->N * 4;        // FP32 sums of the unfused SpMM, 16 batch rows at a time
     return sc;
 }
 
@@ -539,9 +559,10 @@ static cudaError_t ensure_smem_attr(const void* fn, int bytes) {
 
 static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
-static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, const void* wq, const void* scale,
-                               const void* zero, const void* indptr, const void* info, const void* packed, void* Y,
-                               void* workspace, size_t workspace_bytes, void* stream, bool sparse) {
+// Argument checks of the device entry points: nothing is enqueued when one fails.
+static fq_status_t check_gemm_args(const fq_layout_t* L, const void* X, uint32_t M, const void* wq, const void* scale,
+                                   const void* zero, const void* indptr, const void* info, const void* packed, void* Y,
+                                   void* workspace, bool sparse) {
     if (!layout_ok(L)) return fail(FQ_ERR_INVALID_ARG, "bad layout");
     if (M < 1 || M > FQ_MAX_M) return fail(FQ_ERR_INVALID_ARG, "M = %u outside [1, %u]", M, FQ_MAX_M);
     if (!X || !wq || !scale || !zero || !Y || !workspace) return fail(FQ_ERR_INVALID_ARG, "null device pointer");
@@ -550,9 +571,15 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
     if (!aligned(X, 16) || !aligned(Y, 16) || !aligned(wq, 128) || !aligned(scale, 128) || !aligned(zero, 128) ||
         !aligned(workspace, 128) || (sparse && (!aligned(indptr, 4) || !aligned(info, 128) || !aligned(packed, 128))))
         return fail(FQ_ERR_INVALID_ARG, "misaligned device pointer");
-    size_t need = 0;
-    fq_status_t st = fq_workspace_bytes(L, M, &need);
+    return FQ_OK;
+}
+
+static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, const void* wq, const void* scale,
+                               const void* zero, const void* indptr, const void* info, const void* packed, void* Y,
+                               void* workspace, size_t workspace_bytes, void* stream, bool sparse) {
+    fq_status_t st = check_gemm_args(L, X, M, wq, scale, zero, indptr, info, packed, Y, workspace, sparse);
     if (st != FQ_OK) return st;
+    const size_t need = scratch_layout(L, M).off_spmm;      // what the fused kernels use of the scratch
     if (workspace_bytes < need) return fail(FQ_ERR_BUFFER_TOO_SMALL, "workspace holds %zu bytes, %zu needed", workspace_bytes, need);
     const Scratch sc = scratch_layout(L, M);
     cudaLaunchAttribute attr[1];
@@ -677,12 +704,13 @@ fq_status_t fq_fused_w4a16_outlier_gemm_noalloc(const fq_layout_t* L, const void
                                                 const void* scale, const void* zero, const void* tile_indptr,
                                                 const void* bucket_info, const void* packed_outliers, void* Y,
                                                 void* cuda_stream) {
-    size_t need = 0;
-    fq_status_t st = fq_workspace_bytes(L, M, &need);
+    // every argument error is reported before anything is put on the stream (the scratch pointer stands in for itself)
+    fq_status_t st = check_gemm_args(L, X, M, wq, scale, zero, tile_indptr, bucket_info, packed_outliers, Y, (void*)256, true);
     if (st != FQ_OK) return st;
+    const size_t need = scratch_layout(L, M).off_spmm;      // the fused kernels' part of the scratch
     if (need > (size_t)FQ_STATIC_SCRATCH_BYTES)
         return fail(FQ_ERR_BUFFER_TOO_SMALL,
-                    "this call needs %zu bytes of scratch but the built-in scratch holds %zu (M <= %u fits); "
+                    "this call needs %zu bytes of scratch but the built-in scratch holds %zu (M <= %u always fits); "
                     "use fq_fused_w4a16_outlier_gemm with caller-allocated scratch",
                     need, (size_t)FQ_STATIC_SCRATCH_BYTES, (unsigned)FQ_STATIC_SCRATCH_MAX_M);
     void* scratch = nullptr;
@@ -703,17 +731,40 @@ fq_status_t fq_unfused_gemm(const fq_layout_t* L, const void* X, uint32_t M, con
 }
 
 fq_status_t fq_unfused_spmm(const fq_layout_t* L, const void* X, uint32_t M, const void* tile_indptr,
-                            const void* bucket_info, const void* packed_outliers, void* Y, void* cuda_stream) {
+                            const void* bucket_info, const void* packed_outliers, void* Y, void* workspace,
+                            size_t workspace_bytes, void* cuda_stream) {
     if (!layout_ok(L)) return fail(FQ_ERR_INVALID_ARG, "bad layout");
     if (M < 1 || M > FQ_MAX_M) return fail(FQ_ERR_INVALID_ARG, "M = %u outside [1, %u]", M, FQ_MAX_M);
-    if (!X || !tile_indptr || !bucket_info || !Y) return fail(FQ_ERR_INVALID_ARG, "null device pointer");
+    if (!X || !tile_indptr || !bucket_info || !Y || !workspace) return fail(FQ_ERR_INVALID_ARG, "null device pointer");
     if (!packed_outliers && (L->max_tile_packets || !L->tilecoo_encoded)) return fail(FQ_ERR_INVALID_ARG, "null packet pointer");
-    const uint32_t buckets = (L->N / L->BN) * L->buckets_per_tile;   // one warp each
-    fq_spmm_kernel<<<(buckets + 7) / 8, 256, 0, (cudaStream_t)cuda_stream>>>(
-        (const uint16_t*)X, (const uint32_t*)tile_indptr, (const uint32_t*)bucket_info, (const uint4*)packed_outliers,
-        (uint16_t*)Y, M, L->K, L->N, L->BN, L->buckets_per_tile);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "spmm launch: %s", cudaGetErrorString(e));
+    if (!aligned(X, 16) || !aligned(Y, 16) || !aligned(workspace, 128) || !aligned(packed_outliers, 16))
+        return fail(FQ_ERR_INVALID_ARG, "misaligned device pointer");
+    size_t need = 0;
+    fq_status_t st = fq_workspace_bytes(L, M, &need);
+    if (st != FQ_OK) return st;
+    if (workspace_bytes < need) return fail(FQ_ERR_BUFFER_TOO_SMALL, "workspace holds %zu bytes, %zu needed", workspace_bytes, need);
+    const Scratch sc = scratch_layout(L, M);
+    const int sms = sm_count_cached();
+    if (sms <= 0) return fail(FQ_ERR_CUDA, "no CUDA device: %s", cudaGetErrorString(cudaGetLastError()));
+    const uint32_t NT = L->N / L->BN, KT = L->K / kBK;
+    const uint32_t slabs = std::max<uint32_t>(1, std::min<uint32_t>(KT, (2 * (uint32_t)sms + NT - 1) / NT));
+    float* accbuf = (float*)((uint8_t*)workspace + sc.off_spmm);
+    uint32_t* counters = (uint32_t*)((uint8_t*)workspace + kWsHeaderBytes);
+    for (uint32_t m0 = 0; m0 < M; m0 += 16) {
+        const uint32_t mb = std::min<uint32_t>(16, M - m0);
+        const uint16_t* Xm = (const uint16_t*)X + (size_t)m0 * L->K;
+        uint16_t* Ym = (uint16_t*)Y + (size_t)m0 * L->N;
+        if (mb == 1)
+            fq_spmm_kernel<1><<<NT * slabs, L->BN, 0, (cudaStream_t)cuda_stream>>>(
+                Xm, (const uint32_t*)tile_indptr, (const uint32_t*)bucket_info, (const uint4*)packed_outliers, Ym, accbuf, counters,
+                mb, L->K, L->N, L->buckets_per_tile, slabs);
+        else
+            fq_spmm_kernel<16><<<NT * slabs, L->BN, 0, (cudaStream_t)cuda_stream>>>(
+                Xm, (const uint32_t*)tile_indptr, (const uint32_t*)bucket_info, (const uint4*)packed_outliers, Ym, accbuf, counters,
+                mb, L->K, L->N, L->buckets_per_tile, slabs);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "spmm launch: %s", cudaGetErrorString(e));
+    }
     return FQ_OK;
 }
 
@@ -755,9 +806,11 @@ fq_status_t fq_check_status(void* workspace, void* cuda_stream) {
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "status read: %s", cudaGetErrorString(e));
     if (word != 0) {
-        cudaMemsetAsync(workspace, 0, 4, s);
+        // A call that gave up left some tile-arrival counters short: clear the status word and all of them, so
+        // that the next call on this scratch starts from a clean state (Y of the failed call is undefined).
+        cudaMemsetAsync(workspace, 0, kWsHeaderBytes + kWsCounterBytes, s);
         cudaStreamSynchronize(s);
-        return fail((fq_status_t)(int32_t)word, "a device-side wait expired (status word %d)", (int32_t)word);
+        return fail((fq_status_t)(int32_t)word, "the device reported status %d (-5: a bounded wait expired, -6: Tile-COO descriptors do not match the staged packets)", (int32_t)word);
     }
     return FQ_OK;
 }

@@ -375,6 +375,12 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                 sp_off = info & 0xffffu;
                 sp_cnt = (info >> 16) & 0xffu;
                 if (HOT) sp_tail = info >> 24;
+                if (!HOT && __any_sync(0xffffffffu, sp_off + sp_cnt > p.coo_cap)) {
+                    // a descriptor that does not belong to the staged packets (layout struct and arrays out of
+                    // step): report it and skip the unit's outliers instead of reading past the stage
+                    if (lane == 0) atomicExch(p.status, (uint32_t)FQ_ERR_FORMAT);
+                    sp_cnt = 0;
+                }
                 cmax = __reduce_max_sync(0xffffffffu, sp_cnt);
                 if (HOT && __reduce_max_sync(0xffffffffu, sp_off + sp_cnt + sp_tail) > p.coo_cap)
                     pk_g = p.packed + __ldg(p.indptr + u);           // packets beyond the staged part

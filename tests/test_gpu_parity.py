@@ -160,9 +160,55 @@ def test_scratch_is_reusable_and_results_are_reproducible():
         outs.append((M, H.run_fused(P, _x(5, M, K))))
     a = [y for m, y in outs if m == 16]
     assert np.array_equal(a[0], a[1]) and np.array_equal(a[1], a[2])
-    # counters and status word are back to zero
-    head = P.ws[: 256 + 8192].cpu().numpy()
+    # counters and status word are back to zero (header and every tile-arrival counter)
+    head = P.ws[: 256 + 32768].cpu().numpy()
     assert not head.any()
+
+
+def test_a_reported_device_error_rearms_the_scratch():
+    """What a call that gave up leaves behind is put there from the host: an error code in the status word and
+    a few arrival counters that never reached their tile's count.  fq_check_status must report the code, clear
+    all of it, and the next call on the same scratch must be correct."""
+    K, N, g, M = 2048, 1024, 128, 8
+    lay = synth.layer(synth.tensor_seed(8, 5), K, N, density=0.01, layout="mixed")
+    P = H.pack_layer(lay, g)
+    words = P.ws[: 256 + 32768].view(torch.int32)
+    words[0] = fq.FQ_ERR_TIMEOUT
+    words[64 + 0] = 3            # strip 0 of tile 0
+    words[64 + 9] = 1            # strip 1 of tile 1
+    words[64 + 8 * 3 + 7] = 2
+    with pytest.raises(fq.FqError) as e:
+        fq.fq_check_status(P.ws)
+    assert e.value.code == fq.FQ_ERR_TIMEOUT
+    assert not P.ws[: 256 + 32768].cpu().numpy().any()
+    X = _x(5, M, K)
+    Yref, Yabs = H.oracle_result(P, X)
+    H.check_tolerances(H.run_fused(P, X), Yref, Yabs, K)
+
+
+@pytest.mark.parametrize("M", [4, 16, 24])
+def test_a_layout_that_does_not_belong_to_the_arrays_is_reported_not_faulted(M):
+    """Bucket descriptors that point past the packets a stage holds (here: max_tile_packets lowered by hand, as
+    after re-encoding denser outliers with an old layout struct) must end in FQ_ERR_FORMAT, not in a read
+    outside shared memory."""
+    K, N, g = 1024, 512, 128
+    lay = synth.layer(synth.tensor_seed(8, 6), K, N, density=0.03, layout="uniform")
+    P = H.pack_layer(lay, g)
+    assert P.L.max_tile_packets > 16 and P.L.max_tail_packets == 0
+    good = P.L.max_tile_packets
+    P.L.max_tile_packets = 8
+    try:
+        X = H.to_dev(_x(5, M, K))
+        Y = torch.zeros((M, N), dtype=torch.int16, device="cuda")
+        fq.fq_fused_w4a16_outlier_gemm(P.L, X, M, P.d["wq"], P.d["scale"], P.d["zero"], P.d["indptr"], P.d["info"],
+                                       P.d["packed"], Y, P.ws)
+        with pytest.raises(fq.FqError) as e:
+            fq.fq_check_status(P.ws)
+        assert e.value.code == fq.FQ_ERR_FORMAT
+    finally:
+        P.L.max_tile_packets = good
+    Yref, Yabs = H.oracle_result(P, _x(5, M, K))
+    H.check_tolerances(H.run_fused(P, _x(5, M, K)), Yref, Yabs, K)
 
 
 @pytest.mark.parametrize("M", [1, 8, 16, 24])

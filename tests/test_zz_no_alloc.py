@@ -54,3 +54,16 @@ def test_noalloc_entry_point_refuses_what_does_not_fit():
     assert "scratch" in str(e.value)
     torch.cuda.synchronize()
     assert not Y.any()
+
+
+def test_noalloc_entry_point_reports_argument_errors_before_it_touches_the_stream():
+    K, N, g, M = 512, 512, 128, 4
+    lay = synth.layer(3, K, N, density=0.01)
+    P = H.pack_layer(lay, g)
+    Y = torch.full((M, N), 0x1234, dtype=torch.int16, device="cuda")
+    with pytest.raises(fq.FqError) as e:
+        fq.fq_fused_w4a16_outlier_gemm_noalloc(P.L, None, M, P.d["wq"], P.d["scale"], P.d["zero"], P.d["indptr"],
+                                               P.d["info"], P.d["packed"], Y)
+    assert e.value.code == fq.FQ_ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    assert bool((Y == 0x1234).all())

@@ -31,6 +31,7 @@ MS = (1, 8, 16)
 GROUP = 128
 DENSITY = 0.01
 CONFIG_ID = 2                      # the LLaMA-3-8B layer set
+REPEATS = 5                        # repetitions of the timed region (K steps each); the median is the value
 L2_COVER_BYTES = 400 << 20         # rotating copies per layer cover at least this (L2 is 126 MB)
 METRIC = "effective_hbm_gbs_fused_w4a16_outlier_gemm_m1_8_16"
 # dram__bytes_read + dram__bytes_write of the fused kernel over its algorithmic bytes, from the ncu
@@ -65,6 +66,14 @@ def peaks():
         d = json.load(open(p))
         return float(d["hbm_gbs"]), "measured"
     return 6650.0, "fallback"
+
+
+def tensor_peak():
+    """Sustained dense BF16 throughput in TFLOP/s (the denominator of `tensor_frac` for rows with M >= 64)."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        return float(json.load(open(p)).get("bf16_tflops_sustained", 1400.0)), "measured"
+    return 1400.0, "fallback"
 
 
 class ClockSampler:
@@ -120,24 +129,45 @@ class ClockSampler:
         return out
 
 
-def build_workload(layers, log):
-    """Generate, pack and encode every layer on the host.  Returns a list of dicts."""
+def build_workload(layers, log, config_id=CONFIG_ID, table=None, max_m=None):
+    """Generate, pack and encode every layer on the host.  Returns a list of dicts (with the seconds the packer
+    and the encoder took per matrix: the paper bounds its preprocessing at 100 s per matrix, Section 5.3)."""
     from paper_2608_15531_b200 import binding as fq
+    from paper_2608_15531_b200 import synth
+    table = synth.LLAMA3_8B if table is None else table
+    out = []
+    for (name, K, N) in layers:
+        idx = table.index((name, K, N))
+        t0 = time.time()
+        lay = synth.layer(synth.tensor_seed(config_id, idx), K, N, density=DENSITY, layout="mixed")
+        L = fq.fq_get_layout(K, N, GROUP)
+        t1 = time.time()
+        wq, scale, zero = fq.fq_pack_int4(L, lay.W, lay.mask)
+        t2 = time.time()
+        indptr, info, packed = fq.fq_encode_tilecoo(L, lay.coo_k, lay.coo_n, lay.coo_v)
+        t3 = time.time()
+        n_tile = (K // 128) * (N // L.BN)
+        out.append(dict(name=name, K=K, N=N, L=L, lay=lay, wq=wq, scale=scale, zero=zero, indptr=indptr, info=info,
+                        packed=packed, n_tile=n_tile, n_bucket=n_tile * L.buckets_per_tile, nnz=lay.nnz,
+                        pack_s=round(t2 - t1, 3), encode_s=round(t3 - t2, 3),
+                        X=synth.activations(synth.tensor_seed(config_id, idx), max_m or max(MS), K)))
+        log(f"packed {name} {K}x{N}: nnz={lay.nnz} packets={packed.shape[0]} max_tile={L.max_tile_packets} "
+            f"generate {t1 - t0:.1f}s pack {t2 - t1:.1f}s encode {t3 - t2:.1f}s")
+    return out
+
+
+def build_reference_workload(layers, log):
+    """The reference arm's inputs: the generator and the oracle's own quantiser only (the library is not loaded)."""
     from paper_2608_15531_b200 import synth
     out = []
     for (name, K, N) in layers:
         idx = synth.LLAMA3_8B.index((name, K, N))
-        t0 = time.time()
         lay = synth.layer(synth.tensor_seed(CONFIG_ID, idx), K, N, density=DENSITY, layout="mixed")
-        L = fq.fq_get_layout(K, N, GROUP)
-        wq, scale, zero = fq.fq_pack_int4(L, lay.W, lay.mask)
-        indptr, info, packed = fq.fq_encode_tilecoo(L, lay.coo_k, lay.coo_n, lay.coo_v)
-        n_tile = (K // 128) * (N // L.BN)
-        out.append(dict(name=name, K=K, N=N, L=L, lay=lay, wq=wq, scale=scale, zero=zero, indptr=indptr, info=info,
-                        packed=packed, n_tile=n_tile, n_bucket=n_tile * L.buckets_per_tile, nnz=lay.nnz,
-                        X=synth.activations(synth.tensor_seed(CONFIG_ID, idx), max(MS), K)))
-        log(f"packed {name} {K}x{N}: nnz={lay.nnz} packets={packed.shape[0]} max_tile={L.max_tile_packets} "
-            f"in {time.time() - t0:.1f}s")
+        bn = 256 if N % 256 == 0 else 128
+        n_tile = (K // 128) * (N // bn)
+        out.append(dict(name=name, K=K, N=N, lay=lay, n_tile=n_tile, n_bucket=n_tile * (bn // 4), nnz=lay.nnz,
+                        X=synth.activations(synth.tensor_seed(CONFIG_ID, idx), 16, K)))
+        log(f"generated {name} {K}x{N}: nnz={lay.nnz}")
     return out
 
 
@@ -234,16 +264,20 @@ def run_ours(args):
     if rank == 0:
         sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sync_all()
-    e0.record(stream)
-    for _ in range(args.steps):
-        step()
-    e1.record(stream)
-    sync_all()
+    reps_ms, host_issue_ms = [], []
+    for _ in range(REPEATS):                     # the timed region, REPEATS times: the median is reported
+        sync_all()
+        e0.record(stream)
+        h0 = time.perf_counter()
+        for _ in range(args.steps):
+            step()
+        host_issue_ms.append((time.perf_counter() - h0) * 1e3)
+        e1.record(stream)
+        sync_all()
+        reps_ms.append(max_over_ranks(e0.elapsed_time(e1), world, dev))
     clocks = sampler.stop() if rank == 0 else {}
-    ms = e0.elapsed_time(e1)
+    ms = float(np.median(reps_ms))
     fq.fq_check_status(ws)
-    ms = max_over_ranks(ms, world, dev)
     ms_per_step = ms / args.steps
     value = whole_job_gbs(step_bytes, world, ms_per_step)
     # the step's bytes without the two Tile-COO metadata arrays, and as stored (padding included)
@@ -306,10 +340,14 @@ def run_ours(args):
 
     # ---- per call: fused, unfused pair, cuBLAS BF16 on pre-dequantised weights (context, N = 1 view)
     def time_loop(fn, reps):
+        """Device time per call of `reps` calls issued back to back.  The calls are queued behind a short spin
+        kernel, so that the stream never waits for the host (Python issues a call in about as long as the
+        shortest of these kernels runs)."""
         for _ in range(3):
             fn()
         torch.cuda.synchronize()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda._sleep(int(reps * 12e-6 * 1.9e9))   # about 12 us of spinning per queued call
         a.record(stream)
         for _ in range(reps):
             fn()
@@ -327,13 +365,28 @@ def run_ours(args):
             c = w["copies"][w["turn"] % len(w["copies"])]
             w["turn"] += 1
             fq.fq_unfused_gemm(w["L"], w["Xd"][M], M, c["wq"], c["scale"], c["zero"], w["Yd"][M], ws, stream)
-            fq.fq_unfused_spmm(w["L"], w["Xd"][M], M, c["indptr"], c["info"], c["packed"], w["Yd"][M], ws, stream)
+            fq.fq_unfused_spmm(w["L"], w["Xd"][M], M, c["indptr"], c["info"], c["packed"], w["Yd"][M], stream)
 
+        def dense_only():
+            c = w["copies"][w["turn"] % len(w["copies"])]
+            w["turn"] += 1
+            fq.fq_unfused_gemm(w["L"], w["Xd"][M], M, c["wq"], c["scale"], c["zero"], w["Yd"][M], ws, stream)
+
+        def spmm_only():
+            c = w["copies"][w["turn"] % len(w["copies"])]
+            w["turn"] += 1
+            fq.fq_unfused_spmm(w["L"], w["Xd"][M], M, c["indptr"], c["info"], c["packed"], w["Ys"][M], stream)
+
+        w.setdefault("Ys", {})[M] = torch.zeros((M, w["N"]), dtype=torch.int16, device=dev)
         us_f = time_loop(fused, reps)
         us_u = time_loop(unfused, reps)
+        us_d = time_loop(dense_only, reps)
+        us_s = time_loop(spmm_only, reps)
+        sp_bytes = w["indptr"].nbytes + w["info"].nbytes + 4 * w["nnz"] + 2 * M * w["K"] + 4 * M * w["N"]
         per_call.append(dict(layer=w["name"], K=w["K"], N=w["N"], M=M, bytes=nbytes, fused_us=round(us_f, 3),
                              fused_gbs=round(nbytes / us_f / 1e3, 1), frac_of_peak=round(nbytes / us_f / 1e3 / peak, 4),
-                             unfused_us=round(us_u, 3)))
+                             unfused_us=round(us_u, 3), unfused_gemm_us=round(us_d, 3), unfused_spmm_us=round(us_s, 3),
+                             spmm_bytes=sp_bytes, spmm_roofline_us=round(sp_bytes / peak / 1e3, 3)))
     if args.cublas:
         for w in work:
             # BF16 GEMM on dequant(W_Q) + W_O, materialised with torch on the device (a baseline, not the path)
@@ -363,10 +416,21 @@ def run_ours(args):
             torch.cuda.empty_cache()
 
     cpu = cpu_baseline(work, budget_s=args.cpu_seconds) if args.cpu_seconds > 0 else None
+    others = None
+    if args.other_sets and world == 1 and not args.only:
+        for w in work:                               # the headline's device copies are no longer needed
+            for k in ("copies", "Xd", "Yd", "Ys", "args"):
+                w.pop(k, None)
+        torch.cuda.empty_cache()
+        others = other_sets(dev, stream, peak, log, time_loop, up)
 
     line = {
         "metric": METRIC, "value": round(value, 2), "unit": "GB/s", "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
+        "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 5),
+        "ms_per_step_repeats": {"n": REPEATS, "median": round(ms_per_step, 5), "min": round(min(reps_ms) / args.steps, 5),
+                                "max": round(max(reps_ms) / args.steps, 5)},
+        "host_issue_ms_per_step": round(float(np.median(host_issue_ms)) / args.steps, 5),
+        "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": "configs[1]: LLaMA3-8B decode layer set qkv/o_proj/gate_up/down x M in {1,8,16}, "
                                "INT4 g128, 1% mixed-layout BF16 outliers; one step = 12 fused calls",
@@ -377,7 +441,10 @@ def run_ours(args):
                 "ms_per_step": round(e2e_ms / args.steps, 5)},
         "gpu_launches": args.steps * len(calls),
         "roofline": {"bound": "hbm", "achieved": round(value / world, 2), "peak": peak, "unit": "GB/s",
-                     "frac": round(value / world / peak, 4), "traffic": int(NCU_TRAFFIC_RATIO * (step_bytes // len(calls))), "peak_kind": f"of {peak_kind}",
+                     "frac": round(value / world / peak, 4), "traffic": int(NCU_TRAFFIC_RATIO * (step_bytes // len(calls))),
+                     "traffic_kind": f"constant: algorithmic bytes x {NCU_TRAFFIC_RATIO}, the DRAM/algorithmic ratio of the "
+                                     "committed captures (1.06-1.08); not measured by this run",
+                     "peak_kind": f"of {peak_kind}",
                      "bytes_per_launch": step_bytes // len(calls), "us_per_launch": round(ms_per_step * 1e3 / len(calls), 3),
                      # the same time against other byte counts and other denominators
                      "frac_of_spec_8000": round(value / world / 8000.0, 4),
@@ -385,11 +452,68 @@ def run_ours(args):
                      "moved_gbs": round(whole_job_gbs(moved_bytes, 1, ms_per_step), 2),
                      "read_probe_gbs": read_probe, "frac_of_read_probe": round(value / world / read_probe, 4) if read_probe else None},
         "cpu_baseline": cpu,
+        "preprocess": [dict(layer=w["name"], K=w["K"], N=w["N"], pack_s=w["pack_s"], encode_s=w["encode_s"]) for w in work],
         "us_per_call": per_call,
+        "us_per_call_other_sets": others,
     }
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def other_sets(dev, stream, peak, log, time_loop, up):
+    """Per-call times of the layer sets the headline does not cover: configs[0] (one 4096 x 4096 layer, M = 1) and
+    configs[3] (the LLaMA3-70B shapes, M in {1, 4, 16, 32}); same generator, fused call and cuBLAS BF16 per point."""
+    import torch
+    from paper_2608_15531_b200 import binding as fq
+    from paper_2608_15531_b200 import synth
+    rows = []
+    sets = [("configs[0]", 1, [("single", 4096, 4096)], (1,)),
+            ("configs[3]", 4, synth.LLAMA3_70B, (1, 4, 16, 32))]
+    for set_name, cfg, table, Ms in sets:
+        for idx, (name, K, N) in enumerate(table):
+            t0 = time.time()
+            lay = synth.layer(synth.tensor_seed(cfg, idx), K, N, density=DENSITY, layout="mixed")
+            L = fq.fq_get_layout(K, N, GROUP)
+            t1 = time.time()
+            wq, scale, zero = fq.fq_pack_int4(L, lay.W, lay.mask)
+            t2 = time.time()
+            indptr, info, packed = fq.fq_encode_tilecoo(L, lay.coo_k, lay.coo_n, lay.coo_v)
+            t3 = time.time()
+            log(f"{set_name} {name} {K}x{N}: generate {t1 - t0:.1f}s pack {t2 - t1:.1f}s encode {t3 - t2:.1f}s")
+            base = dict(wq=up(wq), scale=up(scale), zero=up(zero), indptr=up(indptr), info=up(info), packed=up(packed))
+            per_copy = sum(v.numel() * v.element_size() for v in base.values())
+            copies = [base] + [{k: v.clone() for k, v in base.items()}
+                               for _ in range(max(2, -(-L2_COVER_BYTES // per_copy)) - 1)]
+            Wb = [torch.randn((K, N), dtype=torch.bfloat16, device=dev) for _ in range(2)]   # cuBLAS: time only
+            n_tile = (K // 128) * (N // L.BN)
+            ws = torch.zeros(fq.fq_workspace_bytes(L, max(Ms)), dtype=torch.uint8, device=dev)
+            Xall = synth.activations(lay.seed, max(Ms), K)
+            for M in Ms:
+                X = up(Xall[:M])
+                Y = torch.empty((M, N), dtype=torch.int16, device=dev)
+                turn = [0]
+
+                def fused():
+                    c = copies[turn[0] % len(copies)]
+                    turn[0] += 1
+                    fq.fq_fused_w4a16_outlier_gemm(L, X, M, c["wq"], c["scale"], c["zero"], c["indptr"], c["info"],
+                                                   c["packed"], Y, ws, stream)
+
+                def mm():
+                    turn[0] += 1
+                    torch.matmul(X.view(torch.bfloat16), Wb[turn[0] & 1])
+
+                nbytes = algorithmic_bytes(K, N, GROUP, lay.nnz, n_tile, n_tile * L.buckets_per_tile, M)
+                us_f = time_loop(fused, 20)
+                us_c = time_loop(mm, 10)
+                fq.fq_check_status(ws)
+                rows.append(dict(set=set_name, layer=name, K=K, N=N, M=M, bytes=nbytes, fused_us=round(us_f, 3),
+                                 fused_gbs=round(nbytes / us_f / 1e3, 1), frac_of_peak=round(nbytes / us_f / 1e3 / peak, 4),
+                                 cublas_bf16_us=round(us_c, 3), pack_s=round(t2 - t1, 3), encode_s=round(t3 - t2, 3)))
+            del copies, base, Wb, lay, wq, packed
+            torch.cuda.empty_cache()
+    return rows
 
 
 def cpu_baseline(work, budget_s: float):
@@ -449,6 +573,7 @@ def run_sweep(args):
             fn()
         torch.cuda.synchronize()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda._sleep(int(reps * 12e-6 * 1.9e9))   # the calls queue up behind a spin kernel: no host-bound gaps
         a.record(stream)
         for _ in range(reps):
             fn()
@@ -484,7 +609,7 @@ def run_sweep(args):
                 c = copies[turn[0] % len(copies)]
                 turn[0] += 1
                 fq.fq_unfused_gemm(L, X, M, c["wq"], c["scale"], c["zero"], Y, ws, stream)
-                fq.fq_unfused_spmm(L, X, M, c["indptr"], c["info"], c["packed"], Y, ws, stream)
+                fq.fq_unfused_spmm(L, X, M, c["indptr"], c["info"], c["packed"], Y, stream)
 
             nbytes = algorithmic_bytes(K, N, g, lay.nnz, n_tile, n_tile * L.buckets_per_tile, M)
             us_f, us_u = time_loop(fused), time_loop(unfused)
@@ -492,6 +617,9 @@ def run_sweep(args):
             out.append(dict(K=K, N=N, group=g, M=M, density=density, layout=layout, nnz=int(lay.nnz), bytes=nbytes,
                             fused_us=round(us_f, 2), unfused_us=round(us_u, 2), fused_gbs=round(nbytes / us_f / 1e3, 1),
                             frac_of_peak=round(nbytes / us_f / 1e3 / peak, 4), fused_over_unfused=round(us_u / us_f, 2)))
+            if M >= 64:                              # against the tensor roofline as well: 2 M K N over the sustained BF16 peak
+                tp, _ = tensor_peak()
+                out[-1]["tensor_frac"] = round(2.0 * M * K * N / (us_f * 1e-6) / 1e12 / tp, 4)
         del copies, base
         torch.cuda.empty_cache()
         return out
@@ -530,7 +658,8 @@ def run_sweep(args):
             for density in (0.0, 0.005, 0.01, 0.02, 0.05):
                 if density == 0.0 and layout == "clustered":
                     continue
-                points += point(3, int(density * 1000) + (layout == "clustered"), 4096, 14336, GROUP, density, layout, (8,))
+                points += point(3, int(density * 1000) + (layout == "clustered"), 4096, 14336, GROUP, density, layout,
+                                (1, 8, 16))
     else:
         for g in (64, 128):
             points += point(5, g, 8192, 28672, g, DENSITY, "mixed", (1, 2, 4, 8, 16, 32, 64, 128))
@@ -549,7 +678,7 @@ def run_reference(args):
         if args.verbose:
             print(f"[bench] {msg}", file=sys.stderr, flush=True)
 
-    work = build_workload(synth.LLAMA3_8B, log)
+    work = build_reference_workload(synth.LLAMA3_8B, log)
     steps = max(1, args.steps)
     per_step_budget = max(2.0, min(20.0, 120.0 / (steps + args.warmup)))
     for _ in range(args.warmup):
@@ -579,6 +708,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="budget of the CPU-oracle baseline leg (0 = skip)")
     ap.add_argument("--no-cublas", dest="cublas", action="store_false")
+    ap.add_argument("--no-other-sets", dest="other_sets", action="store_false",
+                    help="skip the per-call rows of configs[0] and configs[3] (N = 1 only; the headline is unchanged)")
     ap.add_argument("--verbose", action="store_true")
     ap.add_argument("--only", default="", help="profiling aid: restrict the step to one LAYER:M, e.g. gate_up:16")
     ap.add_argument("--sweep", default="", choices=["", "density", "batch", "paper"],

@@ -265,14 +265,16 @@ fq_status_t fq_unfused_gemm(const fq_layout_t* L, const void* X, uint32_t M, con
                             size_t workspace_bytes, void* cuda_stream);
 
 /* Unfused baseline, sparse half: Y += X * W_O as a separate launch (one per 16
- * rows) that re-reads X and read-modify-writes the BF16 Y (the two-kernel
- * scheme the paper compares against, Section 2.2).  Column tiles are split
- * into slabs of row tiles over the CTAs; slabs of one tile add their FP32 sums
- * with atomic additions in the scratch (same scratch and size as the fused
- * call, fq_workspace_bytes), so the last bits of Y may differ run to run. */
+ * rows) that re-reads X and reads, adds to and writes each BF16 element of Y
+ * once (the two-kernel scheme the paper compares against, Section 2.2).  A
+ * column tile's row tiles are split into at most eight slabs, one CTA each,
+ * that form a thread-block cluster and add their FP32 sums through
+ * distributed shared memory in slab order (the same bits every run).  Needs no
+ * scratch.  Device pointers, same alignment as the fused call; the layout and
+ * the descriptors are trusted (a baseline: no format guard). */
 fq_status_t fq_unfused_spmm(const fq_layout_t* L, const void* X, uint32_t M, const void* tile_indptr,
-                            const void* bucket_info, const void* packed_outliers, void* Y, void* workspace,
-                            size_t workspace_bytes, void* cuda_stream);
+                            const void* bucket_info, const void* packed_outliers, void* Y,
+                            void* cuda_stream);
 
 /* Same operator as fq_fused_w4a16_outlier_gemm, called with HOST X and HOST Y:
  * copies X to x_dev, runs the kernel, copies Y back from y_dev and waits for

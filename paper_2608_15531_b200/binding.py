@@ -203,10 +203,9 @@ def fq_unfused_gemm(L: Layout, X, M: int, wq, scale, zero, Y, workspace, stream=
                                  _stream(stream)))
 
 
-def fq_unfused_spmm(L: Layout, X, M: int, tile_indptr, bucket_info, packed, Y, workspace, stream=None) -> None:
+def fq_unfused_spmm(L: Layout, X, M: int, tile_indptr, bucket_info, packed, Y, stream=None) -> None:
     _check(lib().fq_unfused_spmm(ctypes.byref(L), _dp(X), ctypes.c_uint32(M), _dp(tile_indptr), _dp(bucket_info),
-                                 _dp(packed), _dp(Y), _dp(workspace), ctypes.c_size_t(workspace.numel() * workspace.element_size()),
-                                 _stream(stream)))
+                                 _dp(packed), _dp(Y), _stream(stream)))
 
 
 def fq_fused_host_io(L: Layout, X_host, M: int, x_dev, wq, scale, zero, tile_indptr, bucket_info, packed, y_dev,

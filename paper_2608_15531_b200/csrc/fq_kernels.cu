@@ -15,6 +15,7 @@
 // arrive, which adds the FP32 partials in CTA order; no CTA waits for another.  Every wait on a barrier
 // is bounded: on expiry the CTA raises the scratch status word, drains and leaves through the common
 // exit that frees its tensor memory.
+#include <cooperative_groups.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -24,6 +25,7 @@
 
 #include "fq_internal.h"
 
+namespace cg = cooperative_groups;
 namespace fq {
 
 constexpr int kBK = 128;
@@ -221,92 +223,148 @@ struct UnitIter {
 // ----------------------------------------------------------------------------- unfused SpMM
 
 // Y += X * W_O as its own launch (the sparse half of the two-kernel baseline, Section 2.2).  One CTA per
-// (column tile, slab of k-steps), enough slabs to give every SM two CTAs; thread = output column.  Per k-step
-// the CTA stages the activations of up to 16 batch rows as a k-major FP32 tile in shared memory (the same
-// swizzled layout the fused tcgen05 kernel uses), and every thread walks the packets of its column's bucket
-// (slot t of the column-slotted packets; tail slots name their column) and multiplies-adds into RR registers.
-// With one slab a thread then updates its BF16 Y elements once.  With several, the slabs' sums meet in an FP32
-// tile of the scratch through red.global.add (the order of those additions is not fixed: this baseline is not
-// bit-reproducible run to run), and the last CTA of a tile to arrive updates Y and zeroes the FP32 tile again.
+// (column tile, slab of k-steps); the slabs of a tile form one thread-block cluster.  A warp owns a strip of
+// 32 columns (lane = column = slot t of bucket g) and every second (fourth, for tiles of 128 columns) k-step of the slab.  The CTA stages the
+// activations of eight k-steps at a time as a k-major BF16 tile in shared memory; while those loads are in
+// flight every warp fetches the bucket descriptors and the first four packet slots of its k-steps, so one
+// chunk costs three global-memory latencies whatever its length.  A lane multiplies-adds the slots of its
+// column into RR FP32 registers (a padding slot has value 0 and reads row 0: a broadcast).  The warps of
+// a strip add up in shared memory, the slabs of a tile through distributed shared memory (plain loads from
+// the peers' tiles, each CTA taking its share of the elements in slab order: a fixed order, so the result
+// is the same from run to run), and each element of Y is read, added to and written once.
+constexpr int kSpmmChunk = 8;     // k-steps of activations staged at a time
+constexpr int kSpmmThreads = 512; // 16 warps: 8 strips x 2 (tiles of 256 columns) or 4 strips x 4 (tiles of 128)
+constexpr int kSpmmPer = 4;       // k-steps per warp and chunk, at most
+
 template <int RR>
-__global__ void __launch_bounds__(256) fq_spmm_kernel(const uint16_t* __restrict__ X, const uint32_t* __restrict__ indptr,
+__device__ __forceinline__ void spmm_add(float (&acc)[RR], uint32_t w, const uint8_t* xrow) {
+    const uint32_t k = (w >> 5) & 127u;
+    const float v = __uint_as_float(w & 0xffff0000u);
+    if constexpr (RR == 1) {
+        acc[0] = fmaf(v, __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(xrow)[k] << 16), acc[0]);
+    } else {
+#pragma unroll
+        for (int c = 0; c < RR / 8; ++c) {
+            const uint4 q = *reinterpret_cast<const uint4*>(xrow + k * (2 * RR) + 16 * c);
+            const uint32_t x[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                acc[8 * c + 2 * i] = fmaf(v, bf16lo(x[i]), acc[8 * c + 2 * i]);
+                acc[8 * c + 2 * i + 1] = fmaf(v, bf16hi(x[i]), acc[8 * c + 2 * i + 1]);
+            }
+        }
+    }
+}
+
+template <int RR>
+__global__ void __launch_bounds__(kSpmmThreads, 2) fq_spmm_kernel(const uint16_t* __restrict__ X, const uint32_t* __restrict__ indptr,
                                                     const uint32_t* __restrict__ info, const uint4* __restrict__ packed,
-                                                    uint16_t* __restrict__ Y, float* __restrict__ accbuf,
-                                                    uint32_t* __restrict__ counters, uint32_t M, uint32_t K, uint32_t N,
-                                                    uint32_t NB, uint32_t slabs) {
-    __shared__ __align__(128) float xt[kBK * RR];
-    __shared__ uint32_t s_last;
-    const uint32_t BN = blockDim.x, KT = K / kBK;
-    const uint32_t tid = threadIdx.x, tile = blockIdx.x / slabs, slab = blockIdx.x - tile * slabs;
+                                                    uint16_t* __restrict__ Y, uint32_t M, uint32_t K, uint32_t N,
+                                                    uint32_t BN, uint32_t slabs) {
+    extern __shared__ __align__(16) uint8_t spmm_smem[];
+    const uint32_t NB = BN / 4, NS = BN / 32, KW = kSpmmThreads / 32 / NS, KT = K / kBK;
+    float* red = reinterpret_cast<float*>(spmm_smem);                 // [RR][BN] sums of this slab
+    uint8_t* xs = spmm_smem + (size_t)RR * BN * 4;                    // [kSpmmChunk * 128][RR] BF16, k-major
+    const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t strip = warp % NS, kw = warp / NS, g = lane & 7, t = lane >> 3;
+    const uint32_t tile = blockIdx.x / slabs, slab = blockIdx.x - tile * slabs;
     const uint32_t kt0 = slab * KT / slabs, kt1 = (slab + 1) * KT / slabs;
-    const uint32_t strip = tid >> 5, g = tid & 7, t = (tid >> 3) & 3;
-    const uint32_t bucket = strip * 8 + g;
-    const char* xtb = reinterpret_cast<const char*>(xt);
     float acc[RR];
 #pragma unroll
     for (int i = 0; i < RR; ++i) acc[i] = 0.0f;
-    for (uint32_t kt = kt0; kt < kt1; ++kt) {
-        __syncthreads();
-        // the k-step's activations: pairs of consecutive k of one row per load
-        for (uint32_t e = tid; e < (uint32_t)RR * 64; e += BN) {
-            const uint32_t m = e >> 6, kp = e & 63;
-            uint32_t v = 0;
-            if (m < M) v = __ldg(reinterpret_cast<const uint32_t*>(X + (size_t)m * K + (size_t)kt * kBK) + kp);
+
+    for (uint32_t c0 = kt0; c0 < kt1; c0 += kSpmmChunk) {
+        const uint32_t nk = min((uint32_t)kSpmmChunk, kt1 - c0);
+        uint32_t inf[kSpmmPer], base[kSpmmPer];
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const uint32_t k = 2 * kp + h;
-                char* dst = reinterpret_cast<char*>(xt) + k * (4 * RR) + ((((m >> 2) ^ xt_swizzle<RR>(k)) << 4) | ((m & 3) << 2));
-                *reinterpret_cast<float*>(dst) = h ? bf16hi(v) : bf16lo(v);
+        for (int j = 0; j < kSpmmPer; ++j) {
+            const uint32_t kl = kw + j * KW;
+            inf[j] = 0, base[j] = 0;
+            if (kl < nk) {
+                const size_t u = (size_t)tile * KT + c0 + kl;
+                inf[j] = __ldg(info + u * NB + strip * 8 + g);
+                base[j] = __ldg(indptr + u);
+            }
+        }
+        // the chunk's activations: a thread takes eight consecutive k of one batch row at a time
+        constexpr int XU = RR == 1 ? 1 : RR * 16 * kSpmmChunk / kSpmmThreads;
+        uint4 xr[XU];
+#pragma unroll
+        for (int j = 0; j < XU; ++j) {
+            const uint32_t e = tid + j * kSpmmThreads, m = e % RR, o = e / RR;
+            xr[j] = make_uint4(0, 0, 0, 0);
+            if (o < 16 * nk && m < M) xr[j] = __ldg(reinterpret_cast<const uint4*>(X + (size_t)m * K + (size_t)c0 * kBK) + o);
+        }
+        uint32_t w[kSpmmPer][4];
+        const uint32_t* pk[kSpmmPer];
+#pragma unroll
+        for (int j = 0; j < kSpmmPer; ++j) {
+            pk[j] = reinterpret_cast<const uint32_t*>(packed + base[j] + (inf[j] & 0xffffu));
+            const uint32_t depth = (inf[j] >> 16) & 0xffu;
+#pragma unroll
+            for (int d = 0; d < 4; ++d) w[j][d] = (uint32_t)d < depth ? __ldg(pk[j] + d * 4 + t) : 0u;
+        }
+#pragma unroll
+        for (int j = 0; j < XU; ++j) {
+            const uint32_t e = tid + j * kSpmmThreads, m = e % RR, o = e / RR;
+            if (o < 16 * kSpmmChunk) {
+                if constexpr (RR == 1) {
+                    *reinterpret_cast<uint4*>(xs + 16 * o) = xr[j];
+                } else {
+                    // value i of the eight goes to row 8 o + i; the lanes of a warp that hold other octets
+                    // start at other i, so that one store instruction never hits a bank twice
+                    const uint32_t v[4] = {xr[j].x, xr[j].y, xr[j].z, xr[j].w};
+                    const uint32_t rot = (lane / RR) & 7u;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const uint32_t ii = (i + rot) & 7u;
+                        const uint32_t word = ii & 4 ? (ii & 2 ? v[3] : v[2]) : (ii & 2 ? v[1] : v[0]);
+                        *reinterpret_cast<uint16_t*>(xs + (size_t)(8 * o + ii) * (2 * RR) + 2 * m) =
+                            (uint16_t)(ii & 1 ? word >> 16 : word);
+                    }
+                }
             }
         }
         __syncthreads();
-        const size_t u = (size_t)tile * KT + kt;
-        const uint32_t inf = __ldg(info + u * NB + bucket);
-        const uint32_t* pk = reinterpret_cast<const uint32_t*>(packed + __ldg(indptr + u) + (inf & 0xffffu));
-        const uint32_t depth = (inf >> 16) & 0xffu, tail = inf >> 24;
-        for (uint32_t i = 0; i < depth; ++i) {                        // column-slotted: slot t is this thread's column
-            const uint32_t w[1] = {__ldg(pk + i * 4 + t)};
-            add_outliers<RR, 1>(acc, w, xtb);
-        }
-        for (uint32_t i = depth; i < depth + tail; ++i) {             // tail: a slot names its column
-            const uint4 q4 = __ldg(reinterpret_cast<const uint4*>(pk) + i);
-            const uint32_t wd[4] = {q4.x, q4.y, q4.z, q4.w};
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const uint32_t mine[1] = {((wd[e] >> 12) & 3u) == t ? wd[e] : (wd[e] & 0xffffu)};
-                add_outliers<RR, 1>(acc, mine, xtb);
+        for (int j = 0; j < kSpmmPer; ++j) {
+            const uint8_t* xrow = xs + (size_t)(kw + j * KW) * kBK * (2 * RR);
+            const uint32_t depth = (inf[j] >> 16) & 0xffu, tail = inf[j] >> 24;
+            const uint32_t dmax = __reduce_max_sync(0xffffffffu, depth);
+#pragma unroll
+            for (int d = 0; d < 4; ++d)
+                if ((uint32_t)d < dmax) spmm_add<RR>(acc, w[j][d], xrow);
+            for (uint32_t d = 4; d < depth; ++d) spmm_add<RR>(acc, __ldg(pk[j] + d * 4 + t), xrow);
+            for (uint32_t d = depth; d < depth + tail; ++d) {             // tail: a slot names its column
+                const uint4 q4 = __ldg(reinterpret_cast<const uint4*>(pk[j]) + d);
+                const uint32_t wd[4] = {q4.x, q4.y, q4.z, q4.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (((wd[e] >> 12) & 3u) == t) spmm_add<RR>(acc, wd[e], xrow);
             }
         }
+        __syncthreads();                                                  // the tile is overwritten by the next chunk
     }
-    const size_t col = (size_t)tile * BN + tid;
-    if (slabs > 1) {
+
+    // the warps of a strip, then the slabs of the tile
+    const uint32_t col = strip * 32 + lane;
+    for (uint32_t r = 0; r < KW; ++r) {
+        if (kw == r) {
 #pragma unroll
-        for (int m = 0; m < RR; ++m)
-            if ((uint32_t)m < M) asm volatile("red.global.add.f32 [%0], %1;" ::"l"(accbuf + (size_t)m * N + col), "f"(acc[m]) : "memory");
-        __threadfence();
-        __syncthreads();
-        if (tid == 0) {
-            uint32_t old;
-            asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(old) : "l"(counters + tile * 8) : "memory");
-            s_last = old == slabs - 1 ? 1u : 0u;
-            if (s_last) counters[tile * 8] = 0;                       // ready for the next call
+            for (int m = 0; m < RR; ++m) red[m * BN + col] = r ? red[m * BN + col] + acc[m] : acc[m];
         }
         __syncthreads();
-        if (!s_last) return;
-        __threadfence();
-#pragma unroll
-        for (int m = 0; m < RR; ++m)
-            if ((uint32_t)m < M) {
-                acc[m] = __ldcg(accbuf + (size_t)m * N + col);
-                __stcg(accbuf + (size_t)m * N + col, 0.0f);
-            }
     }
-#pragma unroll
-    for (int m = 0; m < RR; ++m)
-        if ((uint32_t)m < M) {
-            uint16_t* y = Y + (size_t)m * N + col;
-            *y = float_to_bf16_bits(bf16_bits_to_float(*y) + acc[m]);
-        }
+    cg::cluster_group cluster = cg::this_cluster();
+    if (slabs > 1) cluster.sync(); else __syncthreads();
+    const uint32_t E = M * BN, e0 = slab * E / slabs, e1 = (slab + 1) * E / slabs;
+    for (uint32_t e = e0 + tid; e < e1; e += kSpmmThreads) {
+        float sum = 0.0f;
+        for (uint32_t s2 = 0; s2 < slabs; ++s2) sum += slabs > 1 ? cluster.map_shared_rank(red, s2)[e] : red[e];
+        uint16_t* y = Y + (size_t)(e / BN) * N + (size_t)tile * BN + (e % BN);
+        *y = float_to_bf16_bits(bf16_bits_to_float(*y) + sum);
+    }
+    if (slabs > 1) cluster.sync();                                        // peers may still be reading this tile
 }
 
 // ----------------------------------------------------------------------------- launch plumbing
@@ -397,10 +455,9 @@ static fq_status_t make_plan(const fq_layout_t* L, uint32_t M, bool sparse, Plan
 }
 
 // Scratch layout: status word and header, tile-arrival counters, FP32 partial slots, then the activation
-// blocks fq_prep_x_kernel writes for the launch in flight (one per k-step), then the FP32 tile in which the
-// slabs of the unfused SpMM meet (all zero between calls).
+// blocks fq_prep_x_kernel writes for the launch in flight (one per k-step).
 struct Scratch {
-    size_t off_partials, off_xb, off_spmm, total;
+    size_t off_partials, off_xb, total;
 };
 // Which kernel serves a launch is decided by its rows alone: up to 16 rows the warp-level MMA kernel, 17 to 32
 // rows the tcgen05 kernel (its MMAs cost the same for any number of batch rows up to 42; with groups of 64 its
@@ -413,8 +470,7 @@ static Scratch scratch_layout(const fq_layout_t* L, uint32_t rows) {
     Scratch sc;
     sc.off_partials = kWsHeaderBytes + kWsCounterBytes;
     sc.off_xb = sc.off_partials + (size_t)kMaxCtas * 2 * L->BN * prow * 4;
-    sc.off_spmm = sc.off_xb + (tc ? (size_t)(L->K / kBK) * blob_bytes(32, (int)(kBK / L->group)) : 0);
-    sc.total = sc.off_spmm + (size_t)16 * L->N * 4;        // FP32 sums of the unfused SpMM, 16 batch rows at a time
+    sc.total = sc.off_xb + (tc ? (size_t)(L->K / kBK) * blob_bytes(32, (int)(kBK / L->group)) : 0);
     return sc;
 }
 
@@ -579,7 +635,7 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
                                void* workspace, size_t workspace_bytes, void* stream, bool sparse) {
     fq_status_t st = check_gemm_args(L, X, M, wq, scale, zero, indptr, info, packed, Y, workspace, sparse);
     if (st != FQ_OK) return st;
-    const size_t need = scratch_layout(L, M).off_spmm;      // what the fused kernels use of the scratch
+    const size_t need = scratch_layout(L, M).total;
     if (workspace_bytes < need) return fail(FQ_ERR_BUFFER_TOO_SMALL, "workspace holds %zu bytes, %zu needed", workspace_bytes, need);
     const Scratch sc = scratch_layout(L, M);
     cudaLaunchAttribute attr[1];
@@ -653,6 +709,25 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
     return FQ_OK;
 }
 
+template <int RR>
+static cudaError_t launch_spmm(const fq_layout_t* L, const uint16_t* X, uint32_t M, const void* indptr, const void* info,
+                               const void* packed, uint16_t* Y, uint32_t slabs, cudaStream_t stream) {
+    const uint32_t smem = (uint32_t)RR * L->BN * 4 + kSpmmChunk * kBK * RR * 2;
+    cudaError_t e = ensure_smem_attr((const void*)fq_spmm_kernel<RR>, 64 * 1024);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(L->N / L->BN * slabs);
+    cfg.blockDim = dim3(kSpmmThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = slabs, at[0].val.clusterDim.y = 1, at[0].val.clusterDim.z = 1;
+    cfg.attrs = at, cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, fq_spmm_kernel<RR>, X, (const uint32_t*)indptr, (const uint32_t*)info,
+                              (const uint4*)packed, Y, M, L->K, L->N, L->BN, slabs);
+}
+
 }  // namespace fq
 
 using namespace fq;
@@ -707,7 +782,7 @@ fq_status_t fq_fused_w4a16_outlier_gemm_noalloc(const fq_layout_t* L, const void
     // every argument error is reported before anything is put on the stream (the scratch pointer stands in for itself)
     fq_status_t st = check_gemm_args(L, X, M, wq, scale, zero, tile_indptr, bucket_info, packed_outliers, Y, (void*)256, true);
     if (st != FQ_OK) return st;
-    const size_t need = scratch_layout(L, M).off_spmm;      // the fused kernels' part of the scratch
+    const size_t need = scratch_layout(L, M).total;
     if (need > (size_t)FQ_STATIC_SCRATCH_BYTES)
         return fail(FQ_ERR_BUFFER_TOO_SMALL,
                     "this call needs %zu bytes of scratch but the built-in scratch holds %zu (M <= %u always fits); "
@@ -731,38 +806,26 @@ fq_status_t fq_unfused_gemm(const fq_layout_t* L, const void* X, uint32_t M, con
 }
 
 fq_status_t fq_unfused_spmm(const fq_layout_t* L, const void* X, uint32_t M, const void* tile_indptr,
-                            const void* bucket_info, const void* packed_outliers, void* Y, void* workspace,
-                            size_t workspace_bytes, void* cuda_stream) {
+                            const void* bucket_info, const void* packed_outliers, void* Y, void* cuda_stream) {
     if (!layout_ok(L)) return fail(FQ_ERR_INVALID_ARG, "bad layout");
     if (M < 1 || M > FQ_MAX_M) return fail(FQ_ERR_INVALID_ARG, "M = %u outside [1, %u]", M, FQ_MAX_M);
-    if (!X || !tile_indptr || !bucket_info || !Y || !workspace) return fail(FQ_ERR_INVALID_ARG, "null device pointer");
+    if (!X || !tile_indptr || !bucket_info || !Y) return fail(FQ_ERR_INVALID_ARG, "null device pointer");
     if (!packed_outliers && (L->max_tile_packets || !L->tilecoo_encoded)) return fail(FQ_ERR_INVALID_ARG, "null packet pointer");
-    if (!aligned(X, 16) || !aligned(Y, 16) || !aligned(workspace, 128) || !aligned(packed_outliers, 16))
+    if (!aligned(X, 16) || !aligned(Y, 16) || !aligned(packed_outliers, 16))
         return fail(FQ_ERR_INVALID_ARG, "misaligned device pointer");
-    size_t need = 0;
-    fq_status_t st = fq_workspace_bytes(L, M, &need);
-    if (st != FQ_OK) return st;
-    if (workspace_bytes < need) return fail(FQ_ERR_BUFFER_TOO_SMALL, "workspace holds %zu bytes, %zu needed", workspace_bytes, need);
-    const Scratch sc = scratch_layout(L, M);
     const int sms = sm_count_cached();
     if (sms <= 0) return fail(FQ_ERR_CUDA, "no CUDA device: %s", cudaGetErrorString(cudaGetLastError()));
     const uint32_t NT = L->N / L->BN, KT = L->K / kBK;
-    const uint32_t slabs = std::max<uint32_t>(1, std::min<uint32_t>(KT, (2 * (uint32_t)sms + NT - 1) / NT));
-    float* accbuf = (float*)((uint8_t*)workspace + sc.off_spmm);
-    uint32_t* counters = (uint32_t*)((uint8_t*)workspace + kWsHeaderBytes);
+    // slabs of a tile = one cluster (at most eight CTAs): as many as it takes to put about two CTAs on every SM
+    const uint32_t slabs = std::max<uint32_t>(1, std::min<uint32_t>(std::min<uint32_t>(8, KT), (uint32_t)(2 * sms) / NT));
     for (uint32_t m0 = 0; m0 < M; m0 += 16) {
         const uint32_t mb = std::min<uint32_t>(16, M - m0);
         const uint16_t* Xm = (const uint16_t*)X + (size_t)m0 * L->K;
         uint16_t* Ym = (uint16_t*)Y + (size_t)m0 * L->N;
-        if (mb == 1)
-            fq_spmm_kernel<1><<<NT * slabs, L->BN, 0, (cudaStream_t)cuda_stream>>>(
-                Xm, (const uint32_t*)tile_indptr, (const uint32_t*)bucket_info, (const uint4*)packed_outliers, Ym, accbuf, counters,
-                mb, L->K, L->N, L->buckets_per_tile, slabs);
-        else
-            fq_spmm_kernel<16><<<NT * slabs, L->BN, 0, (cudaStream_t)cuda_stream>>>(
-                Xm, (const uint32_t*)tile_indptr, (const uint32_t*)bucket_info, (const uint4*)packed_outliers, Ym, accbuf, counters,
-                mb, L->K, L->N, L->buckets_per_tile, slabs);
-        cudaError_t e = cudaGetLastError();
+        cudaStream_t st = (cudaStream_t)cuda_stream;
+        cudaError_t e = mb == 1 ? launch_spmm<1>(L, Xm, mb, tile_indptr, bucket_info, packed_outliers, Ym, slabs, st)
+                      : mb <= 8 ? launch_spmm<8>(L, Xm, mb, tile_indptr, bucket_info, packed_outliers, Ym, slabs, st)
+                                : launch_spmm<16>(L, Xm, mb, tile_indptr, bucket_info, packed_outliers, Ym, slabs, st);
         if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "spmm launch: %s", cudaGetErrorString(e));
     }
     return FQ_OK;

@@ -96,7 +96,7 @@ def run_unfused(P: Packed, X_bits: np.ndarray, with_spmm: bool = True) -> np.nda
     Y = torch.full((M, P.L.N), 0x7fc0, dtype=torch.int16, device="cuda")
     fq.fq_unfused_gemm(P.L, X, M, P.d["wq"], P.d["scale"], P.d["zero"], Y, P.ws)
     if with_spmm:
-        fq.fq_unfused_spmm(P.L, X, M, P.d["indptr"], P.d["info"], P.d["packed"], Y, P.ws)
+        fq.fq_unfused_spmm(P.L, X, M, P.d["indptr"], P.d["info"], P.d["packed"], Y)
     fq.fq_check_status(P.ws)
     return bf16_bits(Y)
 

@@ -113,7 +113,10 @@ typedef struct fq_layout {
     uint32_t max_tail_packets; /* longest tail; 0 = every packet is column-slotted */
     uint32_t tilecoo_encoded;  /* 1 = the three maxima above describe the arrays in use (set by
                                   fq_encode_tilecoo); 0 = unknown: the kernels assume the worst */
-    uint32_t reserved[3];
+    uint32_t kernel_hint;      /* 0 = the library chooses the kernel of a launch from its rows and the layer's
+                                  shape; 1 = never the short-job kernel (one CTA per strip of 32 columns), so
+                                  that tests reach the streaming kernels on small layers too */
+    uint32_t reserved[2];
 } fq_layout_t;
 
 /* Choose tile sizes for a K x N layer.  bn_hint: 0 = library default (256 when

@@ -10,7 +10,8 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfq.so")
 SOURCES = [os.path.join(CSRC, "fq_host.cpp"), os.path.join(CSRC, "fq_kernels.cu")]
-HEADERS = [os.path.join(CSRC, "fq_internal.h"), os.path.join(CSRC, "fq_tc_kernel.cuh"), os.path.join(CSRC, "fq_mma_kernel.cuh"), os.path.join(ROOT, "include", "fq.h")]
+HEADERS = [os.path.join(CSRC, "fq_internal.h"), os.path.join(CSRC, "fq_tc_kernel.cuh"), os.path.join(CSRC, "fq_mma_kernel.cuh"),
+           os.path.join(CSRC, "fq_direct_kernel.cuh"), os.path.join(ROOT, "include", "fq.h")]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

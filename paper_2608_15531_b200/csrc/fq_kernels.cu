@@ -219,6 +219,7 @@ struct UnitIter {
 
 #include "fq_tc_kernel.cuh"
 #include "fq_mma_kernel.cuh"
+#include "fq_direct_kernel.cuh"
 
 // ----------------------------------------------------------------------------- unfused SpMM
 
@@ -454,6 +455,39 @@ static fq_status_t make_plan(const fq_layout_t* L, uint32_t M, bool sparse, Plan
     return FQ_OK;
 }
 
+// Short jobs go to fq_direct_kernel: launches of up to 16 rows on layers with so few strips of 32 columns and
+// so few k-steps that a CTA of the streaming kernel would get only a handful of units, and its fixed costs
+// (ring start-up, settlement of split tiles) would be most of the call.  Returns the warps per CTA of the
+// direct kernel, 0 = not a short job.  The bounds are where it measured faster than the streaming kernel
+// on B200: every strip a CTA of its own on its own SM and at most two k-steps to a warp (32 warps up to 8 rows,
+// 16 warps with twice the accumulators for 9-16 rows); for a single row also up to two CTAs of 16 warps to an SM.
+typedef void (*DirectFn)(const DirectParams);
+static inline uint32_t direct_warps(const fq_layout_t* L, uint32_t rows) {
+    const int sms = sm_count_cached();
+    if (sms <= 0 || rows > 16 || L->kernel_hint == 1) return 0;
+    const uint32_t strips = L->N / 32, KT = L->K / kBK;
+    if (strips <= (uint32_t)sms) {
+        if (rows <= 8) return KT <= 64 ? 32u : 0u;
+        return KT <= 32 ? 16u : 0u;
+    }
+    return (rows == 1 && strips <= 2u * (uint32_t)sms && KT <= 32) ? 16u : 0u;
+}
+template <int MO, int MS, int W>
+static DirectFn pick_direct_group(uint32_t g, bool sparse) {
+    if (!sparse) return g == 64 ? (DirectFn)fq_direct_kernel<MO, 8 * MO, 64, false, W> : (DirectFn)fq_direct_kernel<MO, 8 * MO, 128, false, W>;
+    return g == 64 ? (DirectFn)fq_direct_kernel<MO, MS, 64, true, W> : (DirectFn)fq_direct_kernel<MO, MS, 128, true, W>;
+}
+template <int W>
+static DirectFn pick_direct_rows(uint32_t rows, uint32_t g, bool sparse) {
+    if (rows == 1) return pick_direct_group<1, 1, W>(g, sparse);
+    if (rows <= 4) return pick_direct_group<1, 4, W>(g, sparse);
+    return pick_direct_group<1, 8, W>(g, sparse);
+}
+static DirectFn pick_direct(uint32_t rows, uint32_t warps, uint32_t g, bool sparse) {
+    if (rows > 8) return pick_direct_group<2, 16, 16>(g, sparse);
+    return warps == 32 ? pick_direct_rows<32>(rows, g, sparse) : pick_direct_rows<16>(rows, g, sparse);
+}
+
 // Scratch layout: status word and header, tile-arrival counters, FP32 partial slots, then the activation
 // blocks fq_prep_x_kernel writes for the launch in flight (one per k-step).
 struct Scratch {
@@ -519,7 +553,8 @@ static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, 
     p.split = split;
     pl.ngrp = (units_per_cta >= 8 && MO <= 2) ? 2 : 1;    // four octets of rows: the accumulators leave no room
     const uint32_t xch_bytes = pl.ngrp > 1 ? BN * ROWS * 4 : 0;   // hand-over of a group's partial sums
-    const uint32_t fixed = 1024 + xch_bytes;
+    const uint32_t red_bytes = split ? BN * ROWS * 4 : 0;         // this CTA's partial tile, read by its cluster
+    const uint32_t fixed = 1024 + xch_bytes + red_bytes;
     const uint32_t budget = kSmemBudget;
     uint32_t cap = 0;
     if (sparse) {
@@ -547,7 +582,8 @@ static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, 
     // hot columns, tiles larger than the staged part, or an encoding whose sizes were not recorded
     pl.general = sparse && (L->max_tail_packets > 0 || L->max_tile_packets > cap || !L->tilecoo_encoded);
     p.off_shc = S * stage;
-    p.off_bar = p.off_shc + xch_bytes;
+    p.off_red = p.off_shc + xch_bytes;
+    p.off_bar = p.off_red + red_bytes;
     pl.smem = p.off_bar + 1024;
     pl.threads = 32 * (1 + kActWarps + pl.ngrp * NDW);
     pl.grid = grid;
@@ -613,6 +649,38 @@ static cudaError_t ensure_smem_attr(const void* fn, int bytes) {
     return e;
 }
 
+// Can `tiles` clusters of `c` CTAs of this kernel be resident together?  (One query per kernel, size and device.)
+static bool clusters_fit(const void* fn, uint32_t c, uint32_t tiles, uint32_t threads, uint32_t smem) {
+    struct Seen { const void* fn; int dev; uint32_t c, smem; int n; };
+    static Seen seen[256];
+    static int nseen = 0;
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    std::lock_guard<std::mutex> lock(mu);
+    for (int i = 0; i < nseen; ++i)
+        if (seen[i].fn == fn && seen[i].dev == dev && seen[i].c == c && seen[i].smem == smem) return seen[i].n >= (int)tiles;
+    int n = 0;
+    if (c > 8 && cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
+        cudaGetLastError();
+        n = 0;
+    } else {
+        cudaLaunchConfig_t cfg;
+        std::memset(&cfg, 0, sizeof(cfg));
+        cfg.gridDim = dim3(tiles * c);
+        cfg.blockDim = dim3(threads);
+        cfg.dynamicSmemBytes = smem;
+        cudaLaunchAttribute at[1];
+        std::memset(at, 0, sizeof(at));
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = c, at[0].val.clusterDim.y = 1, at[0].val.clusterDim.z = 1;
+        cfg.attrs = at, cfg.numAttrs = 1;
+        if (cudaOccupancyMaxActiveClusters(&n, fn, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
+    }
+    if (nseen < 256) seen[nseen++] = Seen{fn, dev, c, smem, n};
+    return n >= (int)tiles;
+}
+
 static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
 // Argument checks of the device entry points: nothing is enqueued when one fails.
@@ -638,7 +706,7 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
     const size_t need = scratch_layout(L, M).total;
     if (workspace_bytes < need) return fail(FQ_ERR_BUFFER_TOO_SMALL, "workspace holds %zu bytes, %zu needed", workspace_bytes, need);
     const Scratch sc = scratch_layout(L, M);
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     std::memset(attr, 0, sizeof(attr));
     // Programmatic dependent launch: a grid may become resident while the kernel before it in the stream
     // drains.  Its producer warps then already stream weights (which no kernel writes); everything that touches
@@ -684,6 +752,25 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
             cfg.blockDim = dim3(pl.threads);
             cfg.dynamicSmemBytes = pl.smem;
             e = cudaLaunchKernelEx(&cfg, fn, p);
+        } else if (direct_warps(L, mb)) {
+            DirectParams p;
+            std::memset(&p, 0, sizeof(p));
+            p.X = Xm; p.Y = Ym;
+            p.wq = (const uint8_t*)wq; p.scale = (const uint16_t*)scale; p.zero = (const uint16_t*)zero;
+            p.indptr = (const uint32_t*)indptr; p.info = (const uint32_t*)info; p.packed = (const uint4*)packed;
+            p.status = (uint32_t*)workspace;
+            p.M = mb; p.K = L->K; p.N = L->N; p.KT = L->K / kBK; p.BN = L->BN; p.NB = L->buckets_per_tile;
+            const uint32_t warps = direct_warps(L, mb), nv = (mb <= 8 ? 1u : 2u) * 8u;
+            cfg.gridDim = dim3(L->N / 32);
+            cfg.blockDim = dim3(32 * warps);
+            // per warp: its rows of activations (2 KB per octet) and, up to 8 rows, their k-major copy (2 KB); the
+            // warps' sums reuse those bytes
+            cfg.dynamicSmemBytes = warps * 4096;
+            (void)nv;
+            DirectFn dfn = pick_direct(mb, warps, L->group, sparse);
+            e = ensure_smem_attr((const void*)dfn, 160 * 1024);
+            if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+            e = cudaLaunchKernelEx(&cfg, dfn, p);
         } else {
             MmaPlan pl;
             st = make_plan_mma(L, mb, sparse, pl);
@@ -701,6 +788,14 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
             cfg.gridDim = dim3(pl.grid);
             cfg.blockDim = dim3(pl.threads);
             cfg.dynamicSmemBytes = pl.smem;
+            // a tile split over c CTAs is settled inside a cluster of those CTAs where c clusters-of-tiles can all
+            // be resident at once; otherwise through the scratch, like the tiles of a contiguous range
+            if (p.split >= 2 && p.split <= 16 && clusters_fit((const void*)fn, p.split, p.NT, pl.threads, pl.smem)) {
+                p.cluster = 1;
+                attr[1].id = cudaLaunchAttributeClusterDimension;
+                attr[1].val.clusterDim.x = p.split, attr[1].val.clusterDim.y = 1, attr[1].val.clusterDim.z = 1;
+                cfg.numAttrs = 2;
+            }
             e = cudaLaunchKernelEx(&cfg, fn, p);
         }
         if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));

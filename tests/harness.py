@@ -80,13 +80,20 @@ def pack_layer(layer: synth.Layer, g: int, BN: int = 0, upload: bool = True) -> 
     return Packed(layer, L, g, wq, scale, zero, indptr, info, packed, d, ws)
 
 
-def run_fused(P: Packed, X_bits: np.ndarray) -> np.ndarray:
+def run_fused(P: Packed, X_bits: np.ndarray, streaming_only: bool = False) -> np.ndarray:
+    """One fused call.  `streaming_only` sets the layout's kernel_hint for the call, so that a small layer is
+    served by the streaming kernels instead of the short-job kernel the library would choose for it."""
     M = X_bits.shape[0]
     X = to_dev(X_bits)
     Y = torch.full((M, P.L.N), 0x7fc0, dtype=torch.int16, device="cuda")      # NaN pattern: every element must be written
-    fq.fq_fused_w4a16_outlier_gemm(P.L, X, M, P.d["wq"], P.d["scale"], P.d["zero"], P.d["indptr"], P.d["info"],
-                                   P.d["packed"], Y, P.ws)
-    fq.fq_check_status(P.ws)
+    hint = P.L.kernel_hint
+    P.L.kernel_hint = 1 if streaming_only else 0
+    try:
+        fq.fq_fused_w4a16_outlier_gemm(P.L, X, M, P.d["wq"], P.d["scale"], P.d["zero"], P.d["indptr"], P.d["info"],
+                                       P.d["packed"], Y, P.ws)
+        fq.fq_check_status(P.ws)
+    finally:
+        P.L.kernel_hint = hint
     return bf16_bits(Y)
 
 

@@ -25,15 +25,18 @@ def _x(seed, M, K):
     (4096, 4096, 128, 256, 0.01, "mixed"),     # configuration 1: 512 units over all SMs
     (1536, 2304, 128, 256, 0.0, "uniform"),    # no outliers at all
 ])
-@pytest.mark.parametrize("M", [1, 5, 8, 9, 16])
+@pytest.mark.parametrize("M", [1, 3, 5, 8, 9, 16])
 def test_fused_matches_oracle(K, N, g, BN, density, layout, M):
+    """Every element against the oracle, twice: through the kernel the library picks for the shape (the short-job
+    kernel on these small layers) and through the streaming kernels."""
     lay = synth.layer(synth.tensor_seed(9, K + N + g), K, N, density=density, layout=layout)
     P = H.pack_layer(lay, g, BN)
     X = _x(lay.seed, M, K)
-    Y = H.run_fused(P, X)
     Yref, Yabs = H.oracle_result(P, X)
-    stats = H.check_tolerances(Y, Yref, Yabs, K)
-    assert stats["mean_rel"] < H.MEAN_TOL
+    for streaming_only in (False, True):
+        Y = H.run_fused(P, X, streaming_only=streaming_only)
+        stats = H.check_tolerances(Y, Yref, Yabs, K)
+        assert stats["mean_rel"] < H.MEAN_TOL
 
 
 @pytest.mark.parametrize("M", [17, 32, 33, 64, 100, 128])
@@ -119,9 +122,9 @@ def test_oversized_tiles_fall_back_to_global_packets():
     assert P.L.max_tile_packets == 8192
     for M in (1, 8, 16):
         X = _x(6, M, K)
-        Y = H.run_fused(P, X)
         Yref, Yabs = H.oracle_result(P, X)
-        H.check_tolerances(Y, Yref, Yabs, K)
+        for streaming_only in (False, True):
+            H.check_tolerances(H.run_fused(P, X, streaming_only=streaming_only), Yref, Yabs, K)
 
 
 def test_several_tails_in_one_strip():
@@ -144,20 +147,21 @@ def test_several_tails_in_one_strip():
     lay.W[kk, nn] = synth.bf16_bits_to_f32(vb)
     P = H.pack_layer(lay, g, BN)
     assert P.L.max_tail_packets == (100 - 4 + 17 - 4 + 3) // 4 and P.L.max_tile_packets < 1024
-    for M in (1, 5, 8, 16):
+    for M in (1, 3, 5, 8, 16):
         X = _x(7, M, K)
-        Y = H.run_fused(P, X)
         Yref, Yabs = H.oracle_result(P, X)
-        H.check_tolerances(Y, Yref, Yabs, K)
+        for streaming_only in (False, True):
+            H.check_tolerances(H.run_fused(P, X, streaming_only=streaming_only), Yref, Yabs, K)
 
 
-def test_scratch_is_reusable_and_results_are_reproducible():
+@pytest.mark.parametrize("streaming_only", [False, True])
+def test_scratch_is_reusable_and_results_are_reproducible(streaming_only):
     K, N, g = 2048, 1024, 128
     lay = synth.layer(synth.tensor_seed(8, 4), K, N, density=0.01, layout="mixed")
     P = H.pack_layer(lay, g)
     outs = []
     for M in (16, 1, 16, 8, 16):
-        outs.append((M, H.run_fused(P, _x(5, M, K))))
+        outs.append((M, H.run_fused(P, _x(5, M, K), streaming_only=streaming_only)))
     a = [y for m, y in outs if m == 16]
     assert np.array_equal(a[0], a[1]) and np.array_equal(a[1], a[2])
     # counters and status word are back to zero (header and every tile-arrival counter)
@@ -183,20 +187,22 @@ def test_a_reported_device_error_rearms_the_scratch():
     assert not P.ws[: 256 + 32768].cpu().numpy().any()
     X = _x(5, M, K)
     Yref, Yabs = H.oracle_result(P, X)
-    H.check_tolerances(H.run_fused(P, X), Yref, Yabs, K)
+    H.check_tolerances(H.run_fused(P, X, streaming_only=True), Yref, Yabs, K)
 
 
 @pytest.mark.parametrize("M", [4, 16, 24])
 def test_a_layout_that_does_not_belong_to_the_arrays_is_reported_not_faulted(M):
     """Bucket descriptors that point past the packets a stage holds (here: max_tile_packets lowered by hand, as
     after re-encoding denser outliers with an old layout struct) must end in FQ_ERR_FORMAT, not in a read
-    outside shared memory."""
+    outside shared memory.  (The streaming kernels stage packets; the short-job kernel reads them from global
+    memory and does not depend on that field.)"""
     K, N, g = 1024, 512, 128
     lay = synth.layer(synth.tensor_seed(8, 6), K, N, density=0.03, layout="uniform")
     P = H.pack_layer(lay, g)
     assert P.L.max_tile_packets > 16 and P.L.max_tail_packets == 0
     good = P.L.max_tile_packets
     P.L.max_tile_packets = 8
+    P.L.kernel_hint = 1
     try:
         X = H.to_dev(_x(5, M, K))
         Y = torch.zeros((M, N), dtype=torch.int16, device="cuda")
@@ -207,8 +213,37 @@ def test_a_layout_that_does_not_belong_to_the_arrays_is_reported_not_faulted(M):
         assert e.value.code == fq.FQ_ERR_FORMAT
     finally:
         P.L.max_tile_packets = good
+        P.L.kernel_hint = 0
     Yref, Yabs = H.oracle_result(P, _x(5, M, K))
     H.check_tolerances(H.run_fused(P, _x(5, M, K)), Yref, Yabs, K)
+    H.check_tolerances(H.run_fused(P, _x(5, M, K), streaming_only=True), Yref, Yabs, K)
+
+
+@pytest.mark.parametrize("M", [1, 8, 16])
+@pytest.mark.parametrize("streaming_only", [False, True])
+def test_a_bucket_descriptor_past_its_tile_is_reported_not_followed(M, streaming_only):
+    """A corrupt descriptor (a depth that reaches past the packets of its tile) is skipped and reported by
+    every kernel: neither the short-job kernel (packets from global memory) nor the streaming kernels (packets
+    staged in shared memory) follow it."""
+    K, N, g = 512, 512, 128
+    lay = synth.layer(synth.tensor_seed(8, 7), K, N, density=0.01, layout="uniform")
+    P = H.pack_layer(lay, g)
+    info = P.info.copy()
+    info[-1] = (info[-1] & 0xffff) | (255 << 16)            # last bucket of the last tile: 255 packets deep
+    bad = H.to_dev(info)
+    P.L.kernel_hint = 1 if streaming_only else 0
+    try:
+        X = H.to_dev(_x(5, M, K))
+        Y = torch.zeros((M, N), dtype=torch.int16, device="cuda")
+        fq.fq_fused_w4a16_outlier_gemm(P.L, X, M, P.d["wq"], P.d["scale"], P.d["zero"], P.d["indptr"], bad,
+                                       P.d["packed"], Y, P.ws)
+        with pytest.raises(fq.FqError) as e:
+            fq.fq_check_status(P.ws)
+        assert e.value.code == fq.FQ_ERR_FORMAT
+    finally:
+        P.L.kernel_hint = 0
+    Yref, Yabs = H.oracle_result(P, _x(5, M, K))
+    H.check_tolerances(H.run_fused(P, _x(5, M, K), streaming_only=streaming_only), Yref, Yabs, K)
 
 
 @pytest.mark.parametrize("M", [1, 8, 16, 24])

@@ -553,8 +553,7 @@ static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, 
     p.split = split;
     pl.ngrp = (units_per_cta >= 8 && MO <= 2) ? 2 : 1;    // four octets of rows: the accumulators leave no room
     const uint32_t xch_bytes = pl.ngrp > 1 ? BN * ROWS * 4 : 0;   // hand-over of a group's partial sums
-    const uint32_t red_bytes = split ? BN * ROWS * 4 : 0;         // this CTA's partial tile, read by its cluster
-    const uint32_t fixed = 1024 + xch_bytes + red_bytes;
+    const uint32_t fixed = 1024 + xch_bytes;
     const uint32_t budget = kSmemBudget;
     uint32_t cap = 0;
     if (sparse) {
@@ -582,8 +581,7 @@ static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, 
     // hot columns, tiles larger than the staged part, or an encoding whose sizes were not recorded
     pl.general = sparse && (L->max_tail_packets > 0 || L->max_tile_packets > cap || !L->tilecoo_encoded);
     p.off_shc = S * stage;
-    p.off_red = p.off_shc + xch_bytes;
-    p.off_bar = p.off_red + red_bytes;
+    p.off_bar = p.off_shc + xch_bytes;
     pl.smem = p.off_bar + 1024;
     pl.threads = 32 * (1 + kActWarps + pl.ngrp * NDW);
     pl.grid = grid;
@@ -649,38 +647,6 @@ static cudaError_t ensure_smem_attr(const void* fn, int bytes) {
     return e;
 }
 
-// Can `tiles` clusters of `c` CTAs of this kernel be resident together?  (One query per kernel, size and device.)
-static bool clusters_fit(const void* fn, uint32_t c, uint32_t tiles, uint32_t threads, uint32_t smem) {
-    struct Seen { const void* fn; int dev; uint32_t c, smem; int n; };
-    static Seen seen[256];
-    static int nseen = 0;
-    static std::mutex mu;
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return false;
-    std::lock_guard<std::mutex> lock(mu);
-    for (int i = 0; i < nseen; ++i)
-        if (seen[i].fn == fn && seen[i].dev == dev && seen[i].c == c && seen[i].smem == smem) return seen[i].n >= (int)tiles;
-    int n = 0;
-    if (c > 8 && cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
-        cudaGetLastError();
-        n = 0;
-    } else {
-        cudaLaunchConfig_t cfg;
-        std::memset(&cfg, 0, sizeof(cfg));
-        cfg.gridDim = dim3(tiles * c);
-        cfg.blockDim = dim3(threads);
-        cfg.dynamicSmemBytes = smem;
-        cudaLaunchAttribute at[1];
-        std::memset(at, 0, sizeof(at));
-        at[0].id = cudaLaunchAttributeClusterDimension;
-        at[0].val.clusterDim.x = c, at[0].val.clusterDim.y = 1, at[0].val.clusterDim.z = 1;
-        cfg.attrs = at, cfg.numAttrs = 1;
-        if (cudaOccupancyMaxActiveClusters(&n, fn, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
-    }
-    if (nseen < 256) seen[nseen++] = Seen{fn, dev, c, smem, n};
-    return n >= (int)tiles;
-}
-
 static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
 // Argument checks of the device entry points: nothing is enqueued when one fails.
@@ -706,7 +672,7 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
     const size_t need = scratch_layout(L, M).total;
     if (workspace_bytes < need) return fail(FQ_ERR_BUFFER_TOO_SMALL, "workspace holds %zu bytes, %zu needed", workspace_bytes, need);
     const Scratch sc = scratch_layout(L, M);
-    cudaLaunchAttribute attr[2];
+    cudaLaunchAttribute attr[1];
     std::memset(attr, 0, sizeof(attr));
     // Programmatic dependent launch: a grid may become resident while the kernel before it in the stream
     // drains.  Its producer warps then already stream weights (which no kernel writes); everything that touches
@@ -788,14 +754,6 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
             cfg.gridDim = dim3(pl.grid);
             cfg.blockDim = dim3(pl.threads);
             cfg.dynamicSmemBytes = pl.smem;
-            // a tile split over c CTAs is settled inside a cluster of those CTAs where c clusters-of-tiles can all
-            // be resident at once; otherwise through the scratch, like the tiles of a contiguous range
-            if (p.split >= 2 && p.split <= 16 && clusters_fit((const void*)fn, p.split, p.NT, pl.threads, pl.smem)) {
-                p.cluster = 1;
-                attr[1].id = cudaLaunchAttributeClusterDimension;
-                attr[1].val.clusterDim.x = p.split, attr[1].val.clusterDim.y = 1, attr[1].val.clusterDim.z = 1;
-                cfg.numAttrs = 2;
-            }
             e = cudaLaunchKernelEx(&cfg, fn, p);
         }
         if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));

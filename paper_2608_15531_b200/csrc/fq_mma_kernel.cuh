@@ -26,26 +26,7 @@ struct MmaParams {
     // shared-memory offsets (bytes); the first five are relative to a stage
     uint32_t stage_bytes, off_sz, off_xcan, off_xsum, off_info, off_coo;
     uint32_t off_shc, off_xt, off_bar;
-    uint32_t cluster; // tile-aligned split only: 1 = the c CTAs of a tile are one thread-block cluster and settle the
-                      // tile through distributed shared memory (FP32 partial tiles at off_red) instead of the scratch
-    uint32_t off_red;
 };
-
-// Thread-block cluster helpers: the barrier over all threads of the cluster, and plain loads from a peer CTA's
-// shared memory.
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ uint32_t dsmem_addr(uint32_t own_smem_addr, uint32_t cta_rank) {
-    uint32_t a;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a) : "r"(own_smem_addr), "r"(cta_rank));
-    return a;
-}
-__device__ __forceinline__ float dsmem_ld_f32(uint32_t addr) {
-    float v;
-    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
-    return v;
-}
 
 // Transpose one octet of BF16 activation rows into the FP32 k-major copy xt[k][8] (32 B per k).
 // `row0` is the shared-memory address of row 0 / 16-byte chunk 0 of the octet, rows `row_step`
@@ -662,17 +643,6 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                     // barriers: FP32 partial in fragment order, then one arrival per (tile, strip);
                     // the last warp to arrive adds the partials in CTA order (the same order in
                     // every run) and writes Y.
-                  if (p.cluster) {
-                    // the CTAs of this tile are one cluster: the partial stays in shared memory, in fragment
-                    // order, and is added up after the cluster-wide barrier at the end of the kernel
-                    float* slot = reinterpret_cast<float*>(smem + p.off_red) + dw * (32 * LDC) + lane;
-#pragma unroll
-                    for (int o = 0; o < MO; ++o)
-#pragma unroll
-                        for (int cg = 0; cg < CG; ++cg)
-#pragma unroll
-                            for (int i = 0; i < 4; ++i) slot[((o * CG + cg) * 4 + i) * 32] = accf[o][cg][i];
-                  } else {
                     const uint32_t which = (p.split || u_begin / KT == tn) ? 0u : 1u;
                     float* slot = p.partials + ((size_t)blockIdx.x * 2 + which) * (size_t)(BN * LDC) + dw * (32 * LDC) + lane;
 #pragma unroll
@@ -729,7 +699,6 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                         }
                         if (lane == 0) p.counters[tn * NDW + dw] = 0;  // ready for the next call
                     }
-                  }
                 }
                 if (write_y) {
 #pragma unroll
@@ -754,53 +723,5 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                 ++piece;
           }
         }
-    }
-    if (p.cluster) {
-        // Settlement of a tile inside its cluster.  Every thread of every CTA of the cluster passes both
-        // barriers, whatever its role and whether or not it gave up on a wait before; between them the warp of
-        // strip dw in CTA dw mod c adds the c partial tiles of that strip in CTA order (the same order in every
-        // run) and writes Y.  After the second barrier no peer reads this CTA's shared memory any more.
-        __syncwarp();
-        cluster_sync_all();
-        const uint32_t tile = blockIdx.x / p.split, part = blockIdx.x - tile * p.split;
-        if (warp >= DW0 && warp < DW0 + NDW && (uint32_t)(warp - DW0) % p.split == part) {
-            const int dw = warp - DW0, g = lane >> 2, t = lane & 3;
-            constexpr int NV = MO * CG * 4;
-            constexpr int ND = MO == 1 ? 4 : 2;                // peers whose loads are in flight together
-            float acc[NV];
-#pragma unroll
-            for (int e = 0; e < NV; ++e) acc[e] = 0.0f;
-            const uint32_t mine = smem_u32(smem + p.off_red) + (uint32_t)(dw * (32 * LDC) + lane) * 4u;
-            for (uint32_t c = 0; c < p.split; c += ND) {
-                float v[ND][NV];
-#pragma unroll
-                for (int d = 0; d < ND; ++d) {
-                    const uint32_t peer = dsmem_addr(mine, min(c + d, p.split - 1));
-#pragma unroll
-                    for (int e = 0; e < NV; ++e) v[d][e] = dsmem_ld_f32(peer + e * 128);
-                }
-#pragma unroll
-                for (int d = 0; d < ND; ++d)
-                    if (c + d < p.split) {
-#pragma unroll
-                        for (int e = 0; e < NV; ++e) acc[e] += v[d][e];
-                    }
-            }
-#pragma unroll
-            for (int cg = 0; cg < CG; ++cg)
-#pragma unroll
-                for (int h = 0; h < 2; ++h)
-#pragma unroll
-                    for (int o = 0; o < MO; ++o)
-#pragma unroll
-                        for (int j = 0; j < 2; ++j) {
-                            const uint32_t m = o * 8 + 2 * t + j;
-                            if (m < p.M)
-                                p.Y[(size_t)m * p.N + (size_t)tile * BN + dw * 32 + g + 16 * cg + 8 * h] =
-                                    float_to_bf16_bits(acc[(o * CG + cg) * 4 + 2 * h + j]);
-                        }
-        }
-        __syncwarp();
-        cluster_sync_all();
     }
 }

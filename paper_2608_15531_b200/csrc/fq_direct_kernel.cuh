@@ -36,22 +36,30 @@ struct DirectParams {
 __device__ __forceinline__ void cp_async_16(uint32_t dst_smem, const void* src) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");
 }
+__device__ __forceinline__ void cp_async_4(uint32_t dst_smem, const void* src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst_smem), "l"(src) : "memory");
+}
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
-constexpr int kDirectSlots = 8;     // packets of a bucket whose slots are requested with the weights
+constexpr int kDirectSlots = 8;     // packets of a bucket that are requested with the weights
+// bytes of shared memory a warp of the direct kernel owns: rows of X, k-major copy, scale and zero rows, packets
+constexpr int kDirectWarpBytes = 16 * 256 + 256 + 8 * kDirectSlots * 16;
 
 template <int MO, int MS, int GROUP, bool SPARSE, int WARPS>
 __global__ void __launch_bounds__(32 * WARPS, (MO == 1 && WARPS == 16) ? 2 : 1) fq_direct_kernel(const DirectParams p) {
     constexpr int CG = 2, GPS = kBK / GROUP, NV = MO * CG * 4;
     // Shared memory, per warp: its block of activations, 8 MO rows of 256 B (16-byte chunk c of an odd row at
-    // c ^ 4, so that the fragment loads of a quarter warp touch every bank once), then (MS = 4, 8) the k-major
-    // BF16 copy [k][8].  After the last k-step the same bytes hold the warps' sums, [WARPS][NV + R][32] FP32.
+    // c ^ 4, so that the fragment loads of a quarter warp touch every bank once); (MS = 4, 8) the k-major BF16
+    // copy [k][8]; the strip's scale and zero-point rows of the k-step (64 B each per group); the first eight
+    // packets of the warp's eight buckets (packet d of bucket g at position d ^ g, so that the eight lane groups
+    // read different banks).  After the last k-step the same bytes hold the warps' sums, [WARPS][NV + R][32] FP32.
     extern __shared__ __align__(16) float red[];
     constexpr bool kMajor = SPARSE && (MS == 4 || MS == 8);
-    constexpr int kStageBytes = 8 * MO * 256 + (kMajor ? kBK * 16 : 0);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
-    uint8_t* xrow_s = reinterpret_cast<uint8_t*>(red) + warp * kStageBytes;
-    uint8_t* xk8 = xrow_s + 8 * MO * 256;
+    uint8_t* xrow_s = reinterpret_cast<uint8_t*>(red) + warp * kDirectWarpBytes;
+    uint8_t* xk8 = xrow_s + 8 * 256;                                // MO == 1 only (two octets of rows fill these bytes)
+    uint8_t* szs = xrow_s + 16 * 256;
+    uint8_t* pks = szs + 256;
     const uint32_t strip = blockIdx.x, spt = p.BN / 32, tn = strip / spt, dw = strip - tn * spt;
     const uint32_t KT = p.KT, BN = p.BN;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -84,21 +92,15 @@ __global__ void __launch_bounds__(32 * WARPS, (MO == 1 && WARPS == 16) ? 2 : 1) 
         for (int j = 0; j < 4; ++j)
 #pragma unroll
             for (int i = 0; i < 4; ++i) wr[j][i] = __ldg(wp + j * BN * 4 + i * 32);
-        uint16_t sc[GPS][4], zr[GPS][4];
+        __syncwarp();                                               // the previous k-step's readers are done
 #pragma unroll
-        for (int gi = 0; gi < GPS; ++gi)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const size_t at = (size_t)(kt * GPS + gi) * p.N + (size_t)strip * 32 + g + 8 * i;
-                sc[gi][i] = __ldg(p.scale + at);
-                zr[gi][i] = __ldg(p.zero + at);
-            }
-        // outliers: MS != 16: slot t of the bucket's first kDirectSlots packets; MS == 16: packets t and t + 4 whole
+        for (int gi = 0; gi < GPS; ++gi) {
+            // lanes 0-15: the strip's 32 scales of this group, two per lane; lanes 16-31: its zero-points
+            const uint16_t* row = (lane < 16 ? p.scale : p.zero) + (size_t)(kt * GPS + gi) * p.N + (size_t)strip * 32 + 2 * (lane & 15);
+            cp_async_4(smem_u32(szs + gi * 128 + lane * 4), row);
+        }
+        // outliers: packets t and t + 4 of the lane group's bucket, as far as it has them
         uint32_t sp_first = 0, sp_depth = 0, sp_tail = 0;
-        constexpr int NPRE = MS == 16 ? 8 : kDirectSlots;
-        uint32_t pre[NPRE];
-#pragma unroll
-        for (int d = 0; d < NPRE; ++d) pre[d] = 0;
         if (SPARSE) {
             sp_first = a + (inf & 0xffffu), sp_depth = (inf >> 16) & 0xffu, sp_tail = inf >> 24;
             if (sp_first + sp_depth + sp_tail > b) {
@@ -106,15 +108,11 @@ __global__ void __launch_bounds__(32 * WARPS, (MO == 1 && WARPS == 16) ? 2 : 1) 
                 atomicExch(p.status, (uint32_t)FQ_ERR_FORMAT);
                 sp_depth = 0, sp_tail = 0;
             }
-            if constexpr (MS == 16) {
-                const uint32_t n = sp_depth + sp_tail;
-                if ((uint32_t)t < n) { const uint4 q = __ldg(p.packed + sp_first + t); pre[0] = q.x, pre[1] = q.y, pre[2] = q.z, pre[3] = q.w; }
-                if ((uint32_t)t + 4 < n) { const uint4 q = __ldg(p.packed + sp_first + t + 4); pre[4] = q.x, pre[5] = q.y, pre[6] = q.z, pre[7] = q.w; }
-            } else {
-                const uint32_t* slot = reinterpret_cast<const uint32_t*>(p.packed + sp_first) + t;
+            const uint32_t n = sp_depth + sp_tail;
 #pragma unroll
-                for (int d = 0; d < NPRE; ++d)
-                    if ((uint32_t)d < sp_depth) pre[d] = __ldg(slot + 4 * d);
+            for (int h = 0; h < kDirectSlots / 4; ++h) {
+                const uint32_t d = t + 4 * h;
+                if (d < n) cp_async_16(smem_u32(pks + g * (kDirectSlots * 16) + ((d ^ g) & (kDirectSlots - 1)) * 16), p.packed + sp_first + d);
             }
         }
         if (!waited) {
@@ -123,7 +121,6 @@ __global__ void __launch_bounds__(32 * WARPS, (MO == 1 && WARPS == 16) ? 2 : 1) 
             waited = true;
         }
         // ---- this k-step's block of X into the warp's rows (rows beyond M are zero)
-        __syncwarp();                                               // the previous k-step's readers are done
 #pragma unroll
         for (int o = 0; o < MO; ++o)
 #pragma unroll
@@ -180,8 +177,9 @@ __global__ void __launch_bounds__(32 * WARPS, (MO == 1 && WARPS == 16) ? 2 : 1) 
             for (int cg = 0; cg < CG; ++cg)
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    const float sv = bf16_bits_to_float(sc[gi][2 * cg + h]);
-                    const float zc = -(128.0f + bf16_bits_to_float(zr[gi][2 * cg + h]));
+                    const uint16_t* szr = reinterpret_cast<const uint16_t*>(szs) + gi * 64 + g + 16 * cg + 8 * h;
+                    const float sv = bf16_bits_to_float(szr[0]);
+                    const float zc = -(128.0f + bf16_bits_to_float(szr[32]));
 #pragma unroll
                     for (int o = 0; o < MO; ++o) {
                         accf[o][cg][2 * h + 0] = fmaf(sv, fmaf(zc, ones[o][0], accg[o][cg][2 * h + 0]), accf[o][cg][2 * h + 0]);
@@ -222,16 +220,18 @@ __global__ void __launch_bounds__(32 * WARPS, (MO == 1 && WARPS == 16) ? 2 : 1) 
                     sacc[6] = fmaf(v, bf16lo(q.w), sacc[6]); sacc[7] = fmaf(v, bf16hi(q.w), sacc[7]);
                 }
             };
-            // the slots requested with the weights, as far as the longest list of the warp goes (a lane past its
-            // own list holds padding: value 0, k = 0), then the rare rest
+            // the lane's slot of the staged packets, as far as the longest list of the warp goes (a lane past its
+            // own list adds padding: value 0, k = 0), then the rare rest from global memory
             const uint32_t dmax = __reduce_max_sync(0xffffffffu, sp_depth);
+            const uint8_t* myp = pks + g * (kDirectSlots * 16) + t * 4;
 #pragma unroll
-            for (int d = 0; d < NPRE; ++d)
-                if ((uint32_t)d < dmax) add_mine(pre[d]);
+            for (int d = 0; d < kDirectSlots; ++d)
+                if ((uint32_t)d < dmax) add_mine((uint32_t)d < sp_depth ? *reinterpret_cast<const uint32_t*>(myp + ((d ^ g) & (kDirectSlots - 1)) * 16) : 0u);
             const uint32_t* slot = reinterpret_cast<const uint32_t*>(p.packed + sp_first) + t;
-            for (uint32_t d = NPRE; d < sp_depth; ++d) add_mine(__ldg(slot + 4 * d));
+            for (uint32_t d = kDirectSlots; d < sp_depth; ++d) add_mine(__ldg(slot + 4 * d));
             for (uint32_t d = sp_depth; d < sp_depth + sp_tail; ++d) {      // tail: every slot that names this lane's column
-                const uint4 q = __ldg(p.packed + sp_first + d);
+                const uint4 q = d < (uint32_t)kDirectSlots ? *reinterpret_cast<const uint4*>(pks + g * (kDirectSlots * 16) + ((d ^ g) & (kDirectSlots - 1)) * 16)
+                                                           : __ldg(p.packed + sp_first + d);
                 const uint32_t wd[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
                 for (int e = 0; e < 4; ++e)
@@ -251,21 +251,13 @@ __global__ void __launch_bounds__(32 * WARPS, (MO == 1 && WARPS == 16) ? 2 : 1) 
                         accf[o][i >> 1][2 * (i & 1) + r] = fmaf(v, bf16_bits_to_float(xbits), accf[o][i >> 1][2 * (i & 1) + r]);
                     }
             };
-            // The bucket's first eight packets sit in the four lanes of the group (requested with the weights);
-            // later ones (rare) are read when their turn comes.  The loop runs to the longest list of the warp
-            // so that the shuffles stay warp-wide; a lane group past its own list sees padding (value 0).
+            // staged packets first, later ones (rare) from global memory; past its own list a lane group adds padding
             const uint32_t n = sp_depth + sp_tail;
             const uint32_t nmax = __reduce_max_sync(0xffffffffu, n);
             for (uint32_t d = 0; d < nmax; ++d) {
-                uint4 pk;
-                if (d < 8) {
-                    const int src = (lane & ~3) | (int)(d & 3);
-                    const bool lo = d < 4;
-                    pk.x = __shfl_sync(0xffffffffu, lo ? pre[0] : pre[4], src); pk.y = __shfl_sync(0xffffffffu, lo ? pre[1] : pre[5], src);
-                    pk.z = __shfl_sync(0xffffffffu, lo ? pre[2] : pre[6], src); pk.w = __shfl_sync(0xffffffffu, lo ? pre[3] : pre[7], src);
-                } else {
-                    pk = d < n ? __ldg(p.packed + sp_first + d) : make_uint4(0, 0, 0, 0);
-                }
+                uint4 pk = make_uint4(0, 0, 0, 0);
+                if (d < n) pk = d < (uint32_t)kDirectSlots ? *reinterpret_cast<const uint4*>(pks + g * (kDirectSlots * 16) + ((d ^ g) & (kDirectSlots - 1)) * 16)
+                                                           : __ldg(p.packed + sp_first + d);
                 if (d >= sp_depth && d < n) {
                     // tail: a slot names its column; in the others it counts as padding
                     const uint32_t wd[4] = {pk.x, pk.y, pk.z, pk.w};

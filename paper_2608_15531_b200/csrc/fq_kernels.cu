@@ -729,12 +729,12 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
             const uint32_t warps = direct_warps(L, mb), nv = (mb <= 8 ? 1u : 2u) * 8u;
             cfg.gridDim = dim3(L->N / 32);
             cfg.blockDim = dim3(32 * warps);
-            // per warp: its rows of activations (2 KB per octet) and, up to 8 rows, their k-major copy (2 KB); the
-            // warps' sums reuse those bytes
-            cfg.dynamicSmemBytes = warps * 4096;
+            // per warp: rows of activations, their k-major copy, scale and zero rows, staged packets; the warps'
+            // sums reuse those bytes
+            cfg.dynamicSmemBytes = warps * kDirectWarpBytes;
             (void)nv;
             DirectFn dfn = pick_direct(mb, warps, L->group, sparse);
-            e = ensure_smem_attr((const void*)dfn, 160 * 1024);
+            e = ensure_smem_attr((const void*)dfn, 32 * kDirectWarpBytes);
             if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
             e = cudaLaunchKernelEx(&cfg, dfn, p);
         } else {

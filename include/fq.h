@@ -116,7 +116,11 @@ typedef struct fq_layout {
     uint32_t kernel_hint;      /* 0 = the library chooses the kernel of a launch from its rows and the layer's
                                   shape; 1 = never the short-job kernel (one CTA per strip of 32 columns), so
                                   that tests reach the streaming kernels on small layers too */
-    uint32_t reserved[2];
+    uint32_t slot_order;       /* read by fq_encode_tilecoo: 0 = bank-aware order of a column's outliers over its
+                                  column-slotted packets (Section 3.2.2, restated for this library's kernels:
+                                  packet d of bucket g prefers a row with k mod 4 = (g + d) mod 4); 1 = by row.
+                                  Every kernel accepts either; the arrays decode to the same set */
+    uint32_t reserved[1];
 } fq_layout_t;
 
 /* Choose tile sizes for a K x N layer.  bn_hint: 0 = library default (256 when

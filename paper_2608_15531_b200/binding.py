@@ -36,8 +36,9 @@ EXPORTS = [
 class Layout(ctypes.Structure):
     _fields_ = ([(n, ctypes.c_uint32) for n in
                  ("abi", "K", "N", "group", "BK", "BN", "buckets_per_tile", "wq_interleave", "coo_unit_bytes",
-                  "max_tile_packets", "max_bucket_packets", "max_tail_packets", "tilecoo_encoded", "kernel_hint")] +
-                [("reserved", ctypes.c_uint32 * 2)])
+                  "max_tile_packets", "max_bucket_packets", "max_tail_packets", "tilecoo_encoded", "kernel_hint",
+                  "slot_order")] +
+                [("reserved", ctypes.c_uint32 * 1)])
 
 
 class FqError(RuntimeError):

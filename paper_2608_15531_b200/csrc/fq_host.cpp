@@ -242,7 +242,8 @@ fq_status_t encode_impl(const fq_layout_t* L, const uint32_t* k, const uint32_t*
         for (size_t e = tstart[t]; e < tstart[t + 1]; ++e)
             per[bucket_of(sorted[e].c) * 4 + number_in_bucket(sorted[e].c)].push_back(sorted[e]);
         std::vector<uint32_t>& tw = tile_words[t];
-        uint32_t off = 0;
+        // depth of every bucket: its longest column, or kSlottedWithTail when that column is too long
+        std::vector<uint32_t> depths(NB);
         for (uint32_t b = 0; b < NB; ++b) {
             size_t longest = 0;
             for (uint32_t j = 0; j < 4; ++j) {
@@ -250,11 +251,88 @@ fq_status_t encode_impl(const fq_layout_t* L, const uint32_t* k, const uint32_t*
                 std::sort(col.begin(), col.end(), [](const Entry& x, const Entry& y) { return x.k < y.k; });
                 longest = std::max(longest, col.size());
             }
-            const uint32_t depth = longest > kSlottedMax ? kSlottedWithTail : (uint32_t)longest;
-            for (uint32_t i = 0; i < depth; ++i)
+            depths[b] = longest > kSlottedMax ? kSlottedWithTail : (uint32_t)longest;
+        }
+        // Which of its column-slotted packets holds which of a column's outliers is free (the sum is
+        // order-independent up to rounding).  By row: packet i holds the column's i-th.  Bank-aware (Section
+        // 3.2.2's element reordering, restated for a k-major FP32 copy of eight activation rows, 32 B per row,
+        // where rows with equal k mod 4 share banks): one load instruction of a warp reads slot j of packet d of
+        // its eight buckets and is served half a warp, i.e. four neighbouring buckets, at a time, in as many
+        // passes as the fullest bank group has different rows.  So for every four neighbouring buckets, slot j
+        // and packet number d in turn, the rows are chosen among what the four columns still have to place (or
+        // padding, row 0, where a column has places to spare) such that the passes are fewest.
+        std::vector<std::vector<uint32_t>> place(NB * 4);          // [bucket * 4 + j][d] -> index into the column + 1, 0 = padding
+        for (uint32_t b = 0; b < NB; ++b)
+            for (uint32_t j = 0; j < 4; ++j) place[b * 4 + j].assign(depths[b], 0);
+        if (L->slot_order == 1) {
+            for (uint32_t c = 0; c < NB * 4; ++c)
+                for (uint32_t d = 0; d < std::min<size_t>(per[c].size(), place[c].size()); ++d) place[c][d] = d + 1;
+        } else {
+            for (uint32_t b0 = 0; b0 < NB; b0 += 4)
+                for (uint32_t j = 0; j < 4; ++j) {
+                    uint32_t dmax = 0;
+                    std::vector<uint8_t> used[4];
+                    uint32_t todo[4];
+                    for (uint32_t q = 0; q < 4; ++q) {
+                        const uint32_t c = (b0 + q) * 4 + j;
+                        todo[q] = (uint32_t)std::min<size_t>(per[c].size(), depths[b0 + q]);
+                        used[q].assign(todo[q], 0);
+                        dmax = std::max(dmax, depths[b0 + q]);
+                    }
+                    for (uint32_t d = 0; d < dmax; ++d) {
+                        // candidates per bucket: up to four unplaced outliers (lowest rows first), padding if the
+                        // column has a place to spare; a bucket whose list has ended reads row 0 whatever happens
+                        int cand[4][5], ncand[4];
+                        for (uint32_t q = 0; q < 4; ++q) {
+                            ncand[q] = 0;
+                            const uint32_t c = (b0 + q) * 4 + j;
+                            if (d >= depths[b0 + q]) { cand[q][ncand[q]++] = -1; continue; }
+                            for (uint32_t e = 0; e < used[q].size() && ncand[q] < 4; ++e)
+                                if (!used[q][e]) cand[q][ncand[q]++] = (int)e;
+                            if (todo[q] < depths[b0 + q] - d) cand[q][ncand[q]++] = -1;
+                            (void)c;
+                        }
+                        int best[4] = {cand[0][0], cand[1][0], cand[2][0], cand[3][0]};
+                        uint32_t best_cost = 1u << 30;
+                        int pick[4];
+                        for (int i0 = 0; i0 < ncand[0]; ++i0)
+                            for (int i1 = 0; i1 < ncand[1]; ++i1)
+                                for (int i2 = 0; i2 < ncand[2]; ++i2)
+                                    for (int i3 = 0; i3 < ncand[3]; ++i3) {
+                                        pick[0] = cand[0][i0], pick[1] = cand[1][i1], pick[2] = cand[2][i2], pick[3] = cand[3][i3];
+                                        uint32_t rows[4], passes = 0, pads = 0;
+                                        for (uint32_t q = 0; q < 4; ++q) {
+                                            rows[q] = pick[q] < 0 ? 0u : per[(b0 + q) * 4 + j][pick[q]].k;
+                                            pads += pick[q] < 0 && d < depths[b0 + q];
+                                        }
+                                        for (uint32_t cls = 0; cls < 4; ++cls) {
+                                            uint32_t n = 0;
+                                            for (uint32_t q = 0; q < 4; ++q) {
+                                                if ((rows[q] & 3u) != cls) continue;
+                                                bool seen = false;
+                                                for (uint32_t r = 0; r < q; ++r) seen |= rows[r] == rows[q];
+                                                n += !seen;
+                                            }
+                                            passes = std::max(passes, n);
+                                        }
+                                        // fewest passes; then fewest paddings (outliers placed early leave later
+                                        // packets more freedom); then the first combination found (lowest rows)
+                                        const uint32_t cost = passes * 16 + pads;
+                                        if (cost < best_cost) { best_cost = cost; for (int q = 0; q < 4; ++q) best[q] = pick[q]; }
+                                    }
+                        for (uint32_t q = 0; q < 4; ++q)
+                            if (best[q] >= 0) { place[(b0 + q) * 4 + j][d] = (uint32_t)best[q] + 1; used[q][best[q]] = 1; --todo[q]; }
+                    }
+                }
+        }
+        uint32_t off = 0;
+        for (uint32_t b = 0; b < NB; ++b) {
+            const uint32_t depth = depths[b];
+            for (uint32_t d = 0; d < depth; ++d)
                 for (uint32_t j = 0; j < 4; ++j) {
                     const std::vector<Entry>& col = per[b * 4 + j];
-                    tw.push_back(i < col.size() ? entry_word(col[i].k, j, col[i].v) : entry_word(0, j, 0));
+                    const uint32_t e = place[b * 4 + j][d];
+                    tw.push_back(e ? entry_word(col[e - 1].k, j, col[e - 1].v) : entry_word(0, j, 0));
                 }
             std::vector<Entry> rest;
             for (uint32_t j = 0; j < 4; ++j) {

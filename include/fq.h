@@ -52,20 +52,24 @@
  *   columns {g, g+8, g+16, g+24} of a 32-column block share a bucket; column
  *   g + 8j is column number j of its bucket.  (These are the columns whose
  *   accumulators one group of four lanes holds after the m16n8k16 MMAs of the
- *   small-batch kernel, so a bucket is applied in registers; the paper's
+ *   kernels, so a bucket is applied in registers; the paper's
  *   load-balancing column permutation, Section 3.2.2, is replaced by this
  *   static assignment.)
  *     bucket_info[t*NB + b] = offset | depth << 16 | tail << 24  (uint16, uint8,
  *   uint8): bucket b of tile t owns depth + tail packets starting `offset`
  *   packets after the tile's first.
  *     A packet is four little-endian 32-bit slots; a slot holds one outlier:
- *   bits 16-31 the BF16 value, bits 5-11 the row inside the tile (so that
- *   slot & 0xfe0 is the row times 32), bits 12-13 the column number j, all
- *   other bits 0.  A padding slot has value bits 0x0000 and row 0.
+ *   bits 13-31 the value — an FP32 number cut to ten explicit significand
+ *   bits, which holds every BF16 and every FP16 number exactly (for a BF16
+ *   value, bits 16-31 are its bit pattern and bits 13-15 are 0); slot &
+ *   0xffffe000 is the value as FP32 —, bits 5-11 the row inside the tile (so
+ *   that slot & 0xfe0 is the row times 32), bits 3-4 the column number j, all
+ *   other bits 0.  A padding slot has value bits 0 and row 0.
  *     The first `depth` packets of a bucket are column-slotted (padding per
  *   column as in Section 4.2, with the column given by the slot's position
- *   instead of a column index per packet): slot j of packet i is the i-th
- *   outlier, by row, of column number j, or a padding slot that still names j.  If no column of
+ *   instead of a column index per packet): slot j of packet i is one of the
+ *   outliers of column number j (which one is the encoder's choice, see
+ *   slot_order below), or a padding slot that still names j.  If no column of
  *   the bucket has more than 32 outliers in the tile, depth is the longest
  *   column's count and tail is 0.  Otherwise depth is 4, and the outliers
  *   beyond the first 4 of each column follow in `tail` packets by (row,
@@ -91,7 +95,9 @@ typedef int32_t fq_status_t;
 #define FQ_ERR_TIMEOUT (-5)           /* a bounded device-side wait expired */
 #define FQ_ERR_FORMAT (-6)            /* Tile-COO validator: bad indptr / offset / index */
 
-#define FQ_ABI_VERSION 1u
+#define FQ_ABI_VERSION 2u
+#define FQ_VALUE_BF16 0u
+#define FQ_VALUE_FP16 1u
 #define FQ_MAX_M 128u
 #define FQ_BK 128u
 
@@ -120,7 +126,10 @@ typedef struct fq_layout {
                                   column-slotted packets (Section 3.2.2, restated for this library's kernels:
                                   packet d of bucket g prefers a row with k mod 4 = (g + d) mod 4); 1 = by row.
                                   Every kernel accepts either; the arrays decode to the same set */
-    uint32_t reserved[1];
+    uint32_t value_type;       /* type of the outlier values handed to fq_encode_tilecoo and returned by
+                                  fq_decode_tilecoo, 16 bits each: FQ_VALUE_BF16 (default) or FQ_VALUE_FP16 (IEEE
+                                  binary16; Table 1's value field).  The packed slots hold either exactly, and the
+                                  kernels read them the same way */
 } fq_layout_t;
 
 /* Choose tile sizes for a K x N layer.  bn_hint: 0 = library default (256 when

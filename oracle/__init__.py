@@ -89,8 +89,9 @@ def dequant(q: np.ndarray, s: np.ndarray, z: np.ndarray, g: int) -> np.ndarray:
     return out
 
 
-def fused_matmul(X: np.ndarray, q, s, z, g: int, coo_k, coo_n, coo_v, cols=None, want_abs=False):
-    """Eq. 1 in binary64.  X: uint16 (BF16 bits) MxK.  ``cols``: optional list of
+def fused_matmul(X: np.ndarray, q, s, z, g: int, coo_k, coo_n, coo_v, cols=None, want_abs=False, value_type: int = 0):
+    """Eq. 1 in binary64.  X: uint16 (BF16 bits) MxK.  ``coo_v``: uint16 value bits, BF16 (``value_type`` 0)
+    or IEEE binary16 (1).  ``cols``: optional list of
     output columns to evaluate (all when None).  Returns Y (M x ncols) and,
     when ``want_abs``, the sum of product magnitudes."""
     X = np.ascontiguousarray(X, dtype=np.uint16)
@@ -115,7 +116,7 @@ def fused_matmul(X: np.ndarray, q, s, z, g: int, coo_k, coo_n, coo_v, cols=None,
                            ctypes.c_uint32(N), ctypes.c_uint32(g), _p(q, ctypes.c_uint8),
                            _p(s, ctypes.c_uint16), _p(z, ctypes.c_uint16),
                            _p(coo_k, ctypes.c_uint32), _p(coo_n, ctypes.c_uint32),
-                           _p(coo_v, ctypes.c_uint16), ctypes.c_size_t(nnz),
+                           _p(coo_v, ctypes.c_uint16), ctypes.c_uint32(value_type), ctypes.c_size_t(nnz),
                            _p(cols, ctypes.c_uint32), ctypes.c_uint32(ncols),
                            _p(Y, ctypes.c_double), _p(Yabs, ctypes.c_double))
     return (Y, Yabs) if want_abs else Y
@@ -133,8 +134,9 @@ def decode_wq(wq: np.ndarray, K: int, N: int, BN: int) -> np.ndarray:
     return q
 
 
-def decode_tilecoo(tile_indptr, bucket_info, packed, K: int, N: int, BN: int, NB: int):
-    """Tile-COO arrays -> (k, n, value bits, bucket id) of every real entry."""
+def decode_tilecoo(tile_indptr, bucket_info, packed, K: int, N: int, BN: int, NB: int, value_type: int = 0):
+    """Tile-COO arrays -> (k, n, value bits, bucket id) of every real entry; the value bits as uint16 in the
+    given type (0: BF16, 1: IEEE binary16).  A value the type cannot hold exactly raises."""
     tile_indptr = np.ascontiguousarray(tile_indptr, dtype=np.uint32)
     bucket_info = np.ascontiguousarray(bucket_info, dtype=np.uint32)
     packed = np.ascontiguousarray(packed).view(np.uint8)
@@ -142,15 +144,27 @@ def decode_tilecoo(tile_indptr, bucket_info, packed, K: int, N: int, BN: int, NB
     cap = max(4 * npk, 1)
     k = np.empty(cap, dtype=np.uint32)
     n = np.empty(cap, dtype=np.uint32)
-    v = np.empty(cap, dtype=np.uint16)
+    v = np.empty(cap, dtype=np.uint32)
     b = np.empty(cap, dtype=np.uint32)
     cnt = ctypes.c_size_t(0)
     rc = lib().orc_decode_tilecoo(_p(tile_indptr, ctypes.c_uint32), _p(bucket_info, ctypes.c_uint32),
                                   _p(packed, ctypes.c_uint8), ctypes.c_uint32(K), ctypes.c_uint32(N),
                                   ctypes.c_uint32(BN), ctypes.c_uint32(NB), _p(k, ctypes.c_uint32),
-                                  _p(n, ctypes.c_uint32), _p(v, ctypes.c_uint16),
+                                  _p(n, ctypes.c_uint32), _p(v, ctypes.c_uint32),
                                   _p(b, ctypes.c_uint32), ctypes.byref(cnt))
     if rc != 0:
         raise ValueError(f"orc_decode_tilecoo failed: {rc}")
     c = cnt.value
-    return k[:c].copy(), n[:c].copy(), v[:c].copy(), b[:c].copy()
+    field = v[:c].copy()                                  # 19 bits: an FP32 number cut to ten fraction bits
+    if value_type == 0:
+        if (field & 7).any():
+            raise ValueError("a value does not fit BF16")
+        bits = (field >> 3).astype(np.uint16)
+    else:
+        f32 = (field << 13).view(np.float32)
+        with np.errstate(over="ignore"):
+            h = f32.astype(np.float16)
+        if not np.array_equal(h.astype(np.float32).view(np.uint32), f32.view(np.uint32)):
+            raise ValueError("a value does not fit IEEE binary16")
+        bits = h.view(np.uint16)
+    return k[:c].copy(), n[:c].copy(), bits, b[:c].copy()

@@ -139,13 +139,27 @@ void orc_dequant(const uint8_t* q, const uint16_t* scale, const uint16_t* zero, 
  *                cols[j] of X[m][k] * W_O[k][n]
  *   Yabs[m][j] = the same sums with every product replaced by its magnitude
  *                (NULL to skip); used only for condition-aware reporting.
- * X is M x K BF16 bits, row-major.  Outliers come as COO (k, n, BF16 bits).
+ * X is M x K BF16 bits, row-major.  Outliers come as COO (k, n, value bits);
+ * value_type 0: the bits are BF16, 1: IEEE binary16 (Table 1's value field
+ * allows either).
  * Y and Yabs are M x ncols binary64, row-major.
  */
+/* IEEE binary16 -> binary64, from the definition: 1 sign, 5 exponent (bias 15),
+ * 10 fraction bits; exponent 0 is subnormal (fraction * 2^-24), 31 is inf/NaN. */
+double orc_f16_to_f64(uint16_t h) {
+    const int sign = h >> 15, e = (h >> 10) & 31, f = h & 1023;
+    double mag;
+    if (e == 0) mag = ldexp((double)f, -24);
+    else if (e == 31) mag = f ? NAN : INFINITY;
+    else mag = ldexp(1.0 + (double)f / 1024.0, e - 15);
+    return sign ? -mag : mag;
+}
+
 void orc_fused_matmul(const uint16_t* X, uint32_t M, uint32_t K, uint32_t N, uint32_t g,
                       const uint8_t* q, const uint16_t* scale, const uint16_t* zero,
                       const uint32_t* coo_k, const uint32_t* coo_n, const uint16_t* coo_v,
-                      size_t nnz, const uint32_t* cols, uint32_t ncols, double* Y, double* Yabs) {
+                      uint32_t value_type, size_t nnz, const uint32_t* cols, uint32_t ncols, double* Y,
+                      double* Yabs) {
     /* dense part: X * dequant(W_Q) */
 #pragma omp parallel for schedule(static)
     for (int64_t j = 0; j < (int64_t)ncols; ++j) {
@@ -175,7 +189,7 @@ void orc_fused_matmul(const uint16_t* X, uint32_t M, uint32_t K, uint32_t N, uin
     for (size_t e = 0; e < nnz; ++e) {
         int64_t j = cols ? slot[coo_n[e]] : (int64_t)coo_n[e];
         if (j < 0) continue;
-        double v = (double)orc_bf16_to_f32(coo_v[e]);
+        double v = value_type == 1 ? orc_f16_to_f64(coo_v[e]) : (double)orc_bf16_to_f32(coo_v[e]);
         for (uint32_t m = 0; m < M; ++m) {
             double x = (double)orc_bf16_to_f32(X[(size_t)m * K + coo_k[e]]);
             Y[(size_t)m * ncols + (size_t)j] += x * v;
@@ -230,10 +244,13 @@ int orc_decode_wq(const uint32_t* wq, uint32_t K, uint32_t N, uint32_t BN, uint8
  *   (tail << 24), offset 16 bits, depth and tail 8 bits each: bucket b of
  *   tile t owns packets [tile_indptr[t] + offset, + depth + tail).  Bucket b
  *   holds the tile columns 32 * (b / 8) + b % 8 + 8 * j, j = 0..3.
- *   A packet is four little-endian 32-bit slots.  A slot: bits 16-31 a BF16
- *   value, bits 5-11 the row inside the tile, bits 12-13 the column number j,
- *   all other bits 0.  A slot whose value bits are 0x0000 is padding.  In the
- *   first `depth` packets of a bucket, slot number i names column number i.
+ *   A packet is four little-endian 32-bit slots.  A slot: bits 13-31 the
+ *   value (an FP32 number cut to ten explicit significand bits; for a BF16
+ *   value bits 13-15 are 0 and bits 16-31 are its bit pattern), bits 5-11 the
+ *   row inside the tile, bits 3-4 the column number j, all other bits 0.  A
+ *   slot whose value bits are all 0 is padding.  In the first `depth` packets
+ *   of a bucket, slot number i names column number i.  out_v receives the
+ *   19 value bits (bits 13-31 of the slot, shifted down).
  *
  * out_* must have room for 4 * (number of packets) entries; *count receives the
  * number of real entries.  Returns 0, or a negative code for a structural
@@ -242,7 +259,7 @@ int orc_decode_wq(const uint32_t* wq, uint32_t K, uint32_t N, uint32_t BN, uint8
  */
 int orc_decode_tilecoo(const uint32_t* tile_indptr, const uint32_t* bucket_info,
                        const uint8_t* packed, uint32_t K, uint32_t N, uint32_t BN, uint32_t NB,
-                       uint32_t* out_k, uint32_t* out_n, uint16_t* out_v, uint32_t* out_bucket,
+                       uint32_t* out_k, uint32_t* out_n, uint32_t* out_v, uint32_t* out_bucket,
                        size_t* count) {
     if (K % 128 != 0 || N % BN != 0) return -1;
     const uint32_t KT = K / 128, NT = N / BN;
@@ -261,9 +278,9 @@ int orc_decode_tilecoo(const uint32_t* tile_indptr, const uint32_t* bucket_info,
                     for (uint32_t sidx = 0; sidx < 4; ++sidx) {
                         uint32_t slot = (uint32_t)pk[4 * sidx] | ((uint32_t)pk[4 * sidx + 1] << 8) |
                                         ((uint32_t)pk[4 * sidx + 2] << 16) | ((uint32_t)pk[4 * sidx + 3] << 24);
-                        uint32_t kk = (slot >> 5) & 127u, j = (slot >> 12) & 3u;
-                        uint16_t v = (uint16_t)(slot >> 16);
-                        if ((slot & 0xc01fu) != 0) return -4;
+                        uint32_t kk = (slot >> 5) & 127u, j = (slot >> 3) & 3u;
+                        uint32_t v = slot >> 13;
+                        if ((slot & 0x1007u) != 0) return -4;
                         if (i < depth && j != sidx) return -4;
                         if (v == 0) continue;
                         out_k[c] = kt * 128 + kk;

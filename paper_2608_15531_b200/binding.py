@@ -23,6 +23,8 @@ FQ_ERR_CUDA = -4
 FQ_ERR_TIMEOUT = -5
 FQ_ERR_FORMAT = -6
 FQ_MAX_M = 128
+FQ_VALUE_BF16 = 0
+FQ_VALUE_FP16 = 1
 
 EXPORTS = [
     "fq_get_layout", "fq_pack_int4_sizes", "fq_pack_int4", "fq_unpack_int4", "fq_encode_tilecoo_sizes",
@@ -37,8 +39,7 @@ class Layout(ctypes.Structure):
     _fields_ = ([(n, ctypes.c_uint32) for n in
                  ("abi", "K", "N", "group", "BK", "BN", "buckets_per_tile", "wq_interleave", "coo_unit_bytes",
                   "max_tile_packets", "max_bucket_packets", "max_tail_packets", "tilecoo_encoded", "kernel_hint",
-                  "slot_order")] +
-                [("reserved", ctypes.c_uint32 * 1)])
+                  "slot_order", "value_type")])
 
 
 class FqError(RuntimeError):

@@ -204,7 +204,7 @@ __global__ void __launch_bounds__(32 * WARPS, (MO == 1 && WARPS == 16) ? 2 : 1) 
                 __syncwarp();
             }
             auto add_mine = [&](const uint32_t w) {
-                const float v = __uint_as_float(w & 0xffff0000u);
+                const float v = __uint_as_float(w & kSlotValueMask);
                 const uint32_t k = (w >> 5) & 127u;
                 if constexpr (MS == 1) {
                     sacc[0] = fmaf(v, bf16_bits_to_float(reinterpret_cast<const uint16_t*>(xrow_s)[k]), sacc[0]);
@@ -235,12 +235,12 @@ __global__ void __launch_bounds__(32 * WARPS, (MO == 1 && WARPS == 16) ? 2 : 1) 
                 const uint32_t wd[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
                 for (int e = 0; e < 4; ++e)
-                    if (((wd[e] >> 12) & 3u) == (uint32_t)t) add_mine(wd[e]);
+                    if (((wd[e] >> kSlotColShift) & 3u) == (uint32_t)t) add_mine(wd[e]);
             }
         }
         if constexpr (SPARSE && MS == 16) {
             auto add_slot = [&](const uint32_t w, const int i) {
-                const float v = __uint_as_float(w & 0xffff0000u);
+                const float v = __uint_as_float(w & kSlotValueMask);
                 const uint32_t k = (w >> 5) & 127u;
 #pragma unroll
                 for (int o = 0; o < MO; ++o)
@@ -264,7 +264,7 @@ __global__ void __launch_bounds__(32 * WARPS, (MO == 1 && WARPS == 16) ? 2 : 1) 
                     pk = make_uint4(0, 0, 0, 0);
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
-                        const uint32_t col = (wd[e] >> 12) & 3u, w = wd[e];
+                        const uint32_t col = (wd[e] >> kSlotColShift) & 3u, w = wd[e];
                         add_slot(col == 0 ? w : 0u, 0); add_slot(col == 1 ? w : 0u, 1);
                         add_slot(col == 2 ? w : 0u, 2); add_slot(col == 3 ? w : 0u, 3);
                     }

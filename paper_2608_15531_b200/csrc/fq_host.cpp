@@ -177,7 +177,7 @@ namespace {
 
 struct Entry {
     uint8_t k, c;
-    uint16_t v;
+    uint32_t v;      // the slot's 19 value bits
 };
 
 struct Encoded {
@@ -197,9 +197,39 @@ inline uint32_t bucket_of(uint32_t c) { return ((c >> 5) << 3) | (c & 7u); }
 inline uint32_t number_in_bucket(uint32_t c) { return (c >> 3) & 3u; }
 inline uint32_t column_of(uint32_t b, uint32_t j) { return ((b >> 3) << 5) | (b & 7u) | (j << 3); }
 
-// One outlier as a 32-bit word: value in the upper half, row * 32 in bits 5-11, the column's number
-// inside the bucket in bits 12-13.
-inline uint32_t entry_word(uint32_t k, uint32_t j, uint16_t v) { return ((uint32_t)v << 16) | (j << 12) | (k << 5); }
+// One outlier as a 32-bit word: the 19 value bits from bit 13 up, row * 32 in bits 5-11, the column's number
+// inside the bucket in bits 3-4.
+inline uint32_t entry_word(uint32_t k, uint32_t j, uint32_t v19) { return (v19 << fq::kSlotValueShift) | (j << fq::kSlotColShift) | (k << 5); }
+
+// IEEE binary16 bits -> the FP32 number's bits (every binary16 number is an FP32 number with at most ten fraction
+// bits), and back (exact for such numbers; `ok` says whether it was one).
+inline uint32_t f16_to_f32_bits(uint16_t h) {
+    const uint32_t sign = (uint32_t)(h & 0x8000u) << 16, e = (h >> 10) & 31u, f = h & 1023u;
+    if (e == 31) return sign | 0x7f800000u | (f << 13);
+    if (e != 0) return sign | ((e + 112u) << 23) | (f << 13);
+    if (f == 0) return sign;
+    int shift = 0;
+    uint32_t m = f;
+    while (!(m & 1024u)) m <<= 1, ++shift;                 // normalise the subnormal
+    return sign | ((uint32_t)(113 - shift) << 23) | ((m & 1023u) << 13);
+}
+inline uint16_t f32_bits_to_f16(uint32_t u, bool* ok) {
+    const uint16_t sign = (uint16_t)((u >> 16) & 0x8000u);
+    const int e = (int)((u >> 23) & 255u) - 127;
+    const uint32_t f = u & 0x7fffffu;
+    uint16_t h;
+    if (((u >> 23) & 255u) == 255u) h = (uint16_t)(sign | 0x7c00u | (f >> 13));
+    else if ((u & 0x7fffffffu) == 0) h = sign;
+    else if (e >= -14 && e <= 15) h = (uint16_t)(sign | ((uint32_t)(e + 15) << 10) | (f >> 13));
+    else if (e >= -24 && e < -14) h = (uint16_t)(sign | ((0x800000u | f) >> (13 + (-14 - e))));
+    else h = (uint16_t)(sign | 0x7c00u);                   // out of range
+    *ok = f16_to_f32_bits(h) == u;
+    return h;
+}
+// The caller's 16 value bits as the slot's 19 value bits, and back.
+inline uint32_t value_field(uint16_t v, uint32_t value_type) {
+    return value_type == FQ_VALUE_FP16 ? f16_to_f32_bits(v) >> fq::kSlotValueShift : (uint32_t)v << 3;
+}
 
 // A column with more entries than this in one tile gives its bucket a tail.
 constexpr uint32_t kSlottedMax = 32;
@@ -226,7 +256,7 @@ fq_status_t encode_impl(const fq_layout_t* L, const uint32_t* k, const uint32_t*
         for (size_t e = 0; e < nnz; ++e) {
             if ((v[e] & 0x7fffu) == 0) continue;
             size_t t = (size_t)(n[e] / BN) * KT + k[e] / FQ_BK;
-            sorted[fill[t]++] = Entry{(uint8_t)(k[e] % FQ_BK), (uint8_t)(n[e] % BN), v[e]};
+            sorted[fill[t]++] = Entry{(uint8_t)(k[e] % FQ_BK), (uint8_t)(n[e] % BN), value_field(v[e], L->value_type)};
         }
     }
     // pass 1: per tile and bucket, the column-slotted packets (packet i = entry i of each of the
@@ -432,11 +462,18 @@ fq_status_t fq_decode_tilecoo(const fq_layout_t* L, const uint32_t* indptr, cons
                 const size_t i0 = (size_t)indptr[t] + (inf & 0xffffu), cnt = ((inf >> 16) & 0xffu) + (inf >> 24);
                 for (size_t i = 0; i < cnt * 4; ++i) {
                     const uint32_t w = pw[i0 * 4 + i];
-                    if ((w >> 16) == 0) continue;
+                    if ((w & fq::kSlotValueMask) == 0) continue;
                     if (c >= cap) return fail(FQ_ERR_BUFFER_TOO_SMALL, "decode buffer holds %zu entries", cap);
                     k[c] = kt * FQ_BK + ((w >> 5) & 127u);
-                    n[c] = tn * BN + column_of(b, (w >> 12) & 3u);
-                    v[c] = (uint16_t)(w >> 16);
+                    n[c] = tn * BN + column_of(b, (w >> fq::kSlotColShift) & 3u);
+                    if (L->value_type == FQ_VALUE_FP16) {
+                        bool ok = true;
+                        v[c] = f32_bits_to_f16(w & fq::kSlotValueMask, &ok);
+                        if (!ok) return fail(FQ_ERR_FORMAT, "a value of tile %zu is not an IEEE binary16 number", t);
+                    } else {
+                        if (w & 0xe000u) return fail(FQ_ERR_FORMAT, "a value of tile %zu is not a BF16 number", t);
+                        v[c] = (uint16_t)(w >> 16);
+                    }
                     ++c;
                 }
             }
@@ -464,9 +501,16 @@ fq_status_t fq_validate_tilecoo(const fq_layout_t* L, const uint32_t* indptr, co
             if (depth > kSlottedMax) return fail(FQ_ERR_FORMAT, "bucket %u of tile %zu has %u column-slotted packets, at most %u allowed", b, t, depth, kSlottedMax);
             for (uint32_t i = 0; i < (depth + tail) * 4; ++i) {
                 const uint32_t w = pw[((size_t)indptr[t] + off) * 4 + i];
-                if (w & 0xc01fu) return fail(FQ_ERR_FORMAT, "bits outside the fields are set in a slot of bucket %u, tile %zu", b, t);
-                if (i < depth * 4 && ((w >> 12) & 3u) != (i & 3u))
-                    return fail(FQ_ERR_FORMAT, "slot %u of a column-slotted packet of bucket %u, tile %zu, names column number %u", i & 3u, b, t, (w >> 12) & 3u);
+                if (L->value_type == FQ_VALUE_FP16) {
+                    bool ok = true;
+                    f32_bits_to_f16(w & fq::kSlotValueMask, &ok);
+                    if (!ok) return fail(FQ_ERR_FORMAT, "a value in bucket %u of tile %zu is not an IEEE binary16 number", b, t);
+                } else if (w & 0xe000u) {
+                    return fail(FQ_ERR_FORMAT, "a value in bucket %u of tile %zu is not a BF16 number", b, t);
+                }
+                if (w & fq::kSlotStrayMask) return fail(FQ_ERR_FORMAT, "bits outside the fields are set in a slot of bucket %u, tile %zu", b, t);
+                if (i < depth * 4 && ((w >> fq::kSlotColShift) & 3u) != (i & 3u))
+                    return fail(FQ_ERR_FORMAT, "slot %u of a column-slotted packet of bucket %u, tile %zu, names column number %u", i & 3u, b, t, (w >> fq::kSlotColShift) & 3u);
             }
         }
     }

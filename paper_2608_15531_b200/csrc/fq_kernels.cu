@@ -240,7 +240,7 @@ constexpr int kSpmmPer = 4;       // k-steps per warp and chunk, at most
 template <int RR>
 __device__ __forceinline__ void spmm_add(float (&acc)[RR], uint32_t w, const uint8_t* xrow) {
     const uint32_t k = (w >> 5) & 127u;
-    const float v = __uint_as_float(w & 0xffff0000u);
+    const float v = __uint_as_float(w & kSlotValueMask);
     if constexpr (RR == 1) {
         acc[0] = fmaf(v, __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(xrow)[k] << 16), acc[0]);
     } else {
@@ -341,7 +341,7 @@ __global__ void __launch_bounds__(kSpmmThreads, 2) fq_spmm_kernel(const uint16_t
                 const uint32_t wd[4] = {q4.x, q4.y, q4.z, q4.w};
 #pragma unroll
                 for (int e = 0; e < 4; ++e)
-                    if (((wd[e] >> 12) & 3u) == t) spmm_add<RR>(acc, wd[e], xrow);
+                    if (((wd[e] >> kSlotColShift) & 3u) == t) spmm_add<RR>(acc, wd[e], xrow);
             }
         }
         __syncthreads();                                                  // the tile is overwritten by the next chunk

@@ -452,7 +452,7 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                             acc[R - 1] = fmaf(v, x.w, acc[R - 1]);
                         }
                     };
-                    auto apply = [&](const uint32_t w) { add(sacc, __uint_as_float(w & 0xffff0000u), w); };
+                    auto apply = [&](const uint32_t w) { add(sacc, __uint_as_float(w & kSlotValueMask), w); };
                     if (cmax > 0) apply(pk0);
                     if (cmax > 1) {
                         apply(pk1);
@@ -473,7 +473,7 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                                 const uint32_t w[4] = {pk.x, pk.y, pk.z, pk.w};
 #pragma unroll
                                 for (int e = 0; e < 4; ++e)     // a tail slot names its column
-                                    add(hacc, ((w[e] >> 12) & 3u) == (uint32_t)t ? __uint_as_float(w[e] & 0xffff0000u) : 0.0f, w[e]);
+                                    add(hacc, ((w[e] >> kSlotColShift) & 3u) == (uint32_t)t ? __uint_as_float(w[e] & kSlotValueMask) : 0.0f, w[e]);
                             }
 #pragma unroll
                             for (int ri = 0; ri < R; ++ri) {
@@ -492,7 +492,7 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                         const uint32_t w[4] = {pk.x, pk.y, pk.z, pk.w};
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            const float v = __uint_as_float(w[e] & 0xffff0000u);
+                            const float v = __uint_as_float(w[e] & kSlotValueMask);
 #pragma unroll
                             for (int o = 0; o < MO; ++o) {
                                 accf[o][e >> 1][2 * (e & 1) + 0] = fmaf(v, x2[e][o].x, accf[o][e >> 1][2 * (e & 1) + 0]);
@@ -541,8 +541,8 @@ __global__ void __launch_bounds__(32 * (1 + kActWarps + NGRP * (BN / 32)), 1) fq
                                 const uint32_t w[4] = {pk.x, pk.y, pk.z, pk.w};
 #pragma unroll
                                 for (int e = 0; e < 4; ++e) {
-                                    const uint32_t cls = (w[e] >> 12) & 3u;
-                                    const float v = __uint_as_float(w[e] & 0xffff0000u);
+                                    const uint32_t cls = (w[e] >> kSlotColShift) & 3u;
+                                    const float v = __uint_as_float(w[e] & kSlotValueMask);
 #pragma unroll
                                     for (int cg = 0; cg < CG; ++cg)
 #pragma unroll

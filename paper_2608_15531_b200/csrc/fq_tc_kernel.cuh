@@ -104,7 +104,7 @@ __device__ __forceinline__ void add_outliers(float (&acc)[RR], const uint32_t (&
 #pragma unroll
         for (int j = 0; j < NP; ++j) x[j] = *reinterpret_cast<const float*>(xtb + ((wd[j] >> 3) & 0x1fcu));
 #pragma unroll
-        for (int j = 0; j < NP; ++j) acc[0] = fmaf(__uint_as_float(wd[j] & 0xffff0000u), x[j], acc[0]);
+        for (int j = 0; j < NP; ++j) acc[0] = fmaf(__uint_as_float(wd[j] & kSlotValueMask), x[j], acc[0]);
     } else {
         float4 x[NP][RR / 4];
 #pragma unroll
@@ -117,7 +117,7 @@ __device__ __forceinline__ void add_outliers(float (&acc)[RR], const uint32_t (&
         }
 #pragma unroll
         for (int j = 0; j < NP; ++j) {
-            const float v = __uint_as_float(wd[j] & 0xffff0000u);
+            const float v = __uint_as_float(wd[j] & kSlotValueMask);
 #pragma unroll
             for (int c = 0; c < RR / 4; ++c) {
                 acc[4 * c + 0] = fmaf(v, x[j][c].x, acc[4 * c + 0]);
@@ -616,7 +616,7 @@ __global__ void __launch_bounds__(32 * (kTcFirstUnpack + (1 + epilogue_sets(RR))
 #pragma unroll
                             for (int e = 0; e < 4; ++e) {
                                 // a tail slot names its column: slots of other columns count as padding (value 0)
-                                const uint32_t mine[1] = {((wd[e] >> 12) & 3u) == t ? wd[e] : (wd[e] & 0xffffu)};
+                                const uint32_t mine[1] = {((wd[e] >> kSlotColShift) & 3u) == t ? wd[e] : (wd[e] & ~kSlotValueMask)};
                                 add_outliers<RR, 1>(hacc, mine, xtb);
                             }
                         }

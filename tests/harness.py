@@ -66,8 +66,10 @@ class Packed:
         return self._q
 
 
-def pack_layer(layer: synth.Layer, g: int, BN: int = 0, upload: bool = True) -> Packed:
+def pack_layer(layer: synth.Layer, g: int, BN: int = 0, upload: bool = True, value_type: int = 0) -> Packed:
+    """`value_type`: type of `layer.coo_v`'s 16-bit patterns (fq.FQ_VALUE_BF16 or fq.FQ_VALUE_FP16)."""
     L = fq.fq_get_layout(layer.K, layer.N, g, bn_hint=BN)
+    L.value_type = value_type
     wq, scale, zero = fq.fq_pack_int4(L, layer.W, layer.mask if layer.nnz else None)
     indptr, info, packed = fq.fq_encode_tilecoo(L, layer.coo_k, layer.coo_n, layer.coo_v)
     fq.fq_validate_tilecoo(L, indptr, info, packed)
@@ -117,7 +119,7 @@ def oracle_result(P: Packed, X_bits: np.ndarray, cols=None, dense_only=False):
         return oracle.fused_matmul(X_bits, P.q, P.scale, P.zero, P.g, e, e, np.zeros(0, dtype=np.uint16), cols=cols,
                                    want_abs=True)
     return oracle.fused_matmul(X_bits, P.q, P.scale, P.zero, P.g, lay.coo_k, lay.coo_n, lay.coo_v, cols=cols,
-                               want_abs=True)
+                               want_abs=True, value_type=P.L.value_type)
 
 
 def check_tolerances(Y_bits: np.ndarray, Yref: np.ndarray, Yabs: np.ndarray, K: int):

@@ -262,6 +262,57 @@ def test_many_units_per_cta_are_repeatable(M):
     H.check_tolerances(Y[:, cols], Yref, Yabs, K)
 
 
+def _with_fp16_values(lay, seed):
+    """The layer's outlier positions with values re-drawn as IEEE binary16 numbers (ten fraction bits in use)."""
+    rng = np.random.default_rng(seed)
+    vals = (rng.uniform(0.12, 0.4, size=lay.coo_k.size) * rng.choice([-1, 1], size=lay.coo_k.size)).astype(np.float16)
+    lay.coo_v = vals.view(np.uint16).copy()
+    lay.W[lay.coo_k, lay.coo_n] = vals.astype(np.float32)
+    return lay
+
+
+@pytest.mark.parametrize("M", [1, 4, 8, 16, 24])
+def test_fp16_outlier_values_match_the_oracle(M):
+    """Outlier values of the second type of Table 1 (IEEE binary16), every element, through every kernel that
+    serves the shape (M = 24: the tcgen05 kernel)."""
+    K, N, g = 1024, 768, 128
+    lay = _with_fp16_values(synth.layer(synth.tensor_seed(8, 11), K, N, density=0.02, layout="mixed"), 21)
+    P = H.pack_layer(lay, g, value_type=fq.FQ_VALUE_FP16)
+    X = _x(12, M, K)
+    Yref, Yabs = H.oracle_result(P, X)
+    for streaming_only in (False, True):
+        H.check_tolerances(H.run_fused(P, X, streaming_only=streaming_only), Yref, Yabs, K)
+    # the unfused pair reads the same slots; it rounds to BF16 twice (the dense result, then the sum)
+    Yref_d, _ = H.oracle_result(P, X, dense_only=True)
+    err = np.abs(H.bits_to_f64(H.run_unfused(P, X)) - Yref)
+    assert np.all(err <= 2.0 ** -8 * (np.abs(Yref_d) + np.abs(Yref)) + K * 2.0 ** -24 * Yabs)
+
+
+@pytest.mark.parametrize("M", [1, 8, 16, 24])
+def test_fp16_outlier_values_keep_their_ten_fraction_bits(M):
+    """Two outliers in one column, 1 + 2^-9 and -1, activations 512 in both rows, nothing else: Y is exactly 1.
+    With the first value cut to BF16 (eight significant bits) it would be 0."""
+    K, N, g = 256, 512, 128
+    lay = synth.layer(1, K, N, density=0.0)
+    lay.W[:] = 0.0
+    cols = np.array([5, 5, 300, 300], dtype=np.uint32)
+    rows = np.array([3, 200, 77, 130], dtype=np.uint32)
+    vals = np.array([1 + 2.0 ** -9, -1.0, -(1 + 2.0 ** -10), 1.0], dtype=np.float16)
+    mask = np.zeros((K, N), dtype=np.uint8)
+    mask[rows, cols] = 1
+    lay.mask, lay.coo_k, lay.coo_n, lay.coo_v = mask, rows, cols, vals.view(np.uint16).copy()
+    lay.W[rows, cols] = vals.astype(np.float32)
+    P = H.pack_layer(lay, g, value_type=fq.FQ_VALUE_FP16)
+    Xf = np.zeros((M, K), dtype=np.float32)
+    Xf[:, rows] = 512.0
+    X = (Xf.view(np.uint32) >> 16).astype(np.uint16)
+    for streaming_only in (False, True):
+        Y = H.bits_to_f64(H.run_fused(P, X, streaming_only=streaming_only))
+        assert np.all(Y[:, 5] == 1.0) and np.all(Y[:, 300] == -0.5)
+        Y[:, [5, 300]] = 0
+        assert not Y.any()
+
+
 def test_argument_errors_launch_nothing():
     K, N, g = 512, 512, 128
     lay = synth.layer(1, K, N, density=0.01)

@@ -157,8 +157,8 @@ def test_tilecoo_slots_and_order_inside_a_bucket():
     for bb in range(NB):
         pk = slots[off[bb]:off[bb] + depth[bb]]
         # slot j of every packet names column number j, padding included
-        assert np.array_equal((pk >> 12) & 3, np.tile(np.arange(4, dtype=np.uint32), (pk.shape[0], 1)))
-        assert not (pk & 0xc01f).any()
+        assert np.array_equal((pk >> 3) & 3, np.tile(np.arange(4, dtype=np.uint32), (pk.shape[0], 1)))
+        assert not (pk & 0x1007).any()
         for j in range(4):
             col = (bb // 8) * 32 + bb % 8 + 8 * j
             want = np.sort(Lr.coo_k[Lr.coo_n == col])
@@ -166,7 +166,7 @@ def test_tilecoo_slots_and_order_inside_a_bucket():
             # a column's outliers come first, by row; then only padding (value 0, row 0)
             assert live.sum() == want.size and live[:want.size].all()
             assert np.array_equal((pk[:want.size, j] >> 5) & 127, want)
-            assert not (pk[want.size:, j] & 0xffff0fe0).any()
+            assert not (pk[want.size:, j] & 0xffffefe0).any()
     # a hot column: its first four outliers in column-slotted packets, the rest four to a packet by row
     kk = np.arange(0, 40, dtype=np.uint32)
     nn = np.full(40, 15, dtype=np.uint32)                 # column number 1 of bucket 7
@@ -178,7 +178,7 @@ def test_tilecoo_slots_and_order_inside_a_bucket():
     assert L.max_tail_packets == 9 and L.max_bucket_packets == 13
     s2 = pk.view(np.uint32).reshape(-1, 4)
     assert np.array_equal((s2[:4, 1] >> 5) & 127, np.arange(4)) and not (s2[:4, [0, 2, 3]] >> 16).any()
-    assert np.array_equal((s2[4:].ravel() >> 5) & 127, np.arange(4, 40)) and np.all((s2[4:].ravel() >> 12) & 3 == 1)
+    assert np.array_equal((s2[4:].ravel() >> 5) & 127, np.arange(4, 40)) and np.all((s2[4:].ravel() >> 3) & 3 == 1)
     # exactly 32 in a column still has no tail
     ip, bi, pk = fq.fq_encode_tilecoo(L, kk[:32], nn[:32], vv[:32])
     assert int(bi[_bucket_of(15)]) == 0 | (32 << 16) and L.max_tail_packets == 0
@@ -239,6 +239,49 @@ def test_bank_aware_slot_order_has_fewer_conflicts_than_row_order(layout, densit
         assert (w_bank - least) < 0.8 * (w_row - least), (w_bank, w_row, least)
 
 
+def test_fp16_outlier_values_round_trip_exactly():
+    """Table 1's value field as IEEE binary16: the packed slots hold every binary16 number exactly (normal,
+    subnormal, largest), the decoders return the same bits, and a layout of the other type rejects what it
+    cannot hold."""
+    K, N = 256, 512
+    rng = np.random.default_rng(3)
+    nnz = 4000
+    pos = rng.choice(K * N, size=nnz, replace=False)
+    kk, nn = (pos // N).astype(np.uint32), (pos % N).astype(np.uint32)
+    vals = (rng.uniform(0.12, 0.4, size=nnz) * rng.choice([-1, 1], size=nnz)).astype(np.float16)
+    vb = vals.view(np.uint16).copy()
+    vb[:6] = [0x0001, 0x83ff, 0x0400, 0x7bff, 0xfbff, 0x3c01]     # subnormals, smallest normal, +-65504, 1 + 2^-10
+    L = fq.fq_get_layout(K, N, 128)
+    L.value_type = fq.FQ_VALUE_FP16
+    indptr, info, packed = fq.fq_encode_tilecoo(L, kk, nn, vb)
+    fq.fq_validate_tilecoo(L, indptr, info, packed)
+    k2, n2, v2 = fq.fq_decode_tilecoo(L, indptr, info, packed)
+    assert _as_set(k2, n2, v2) == _as_set(kk, nn, vb)
+    ko, no, vo, _ = oracle.decode_tilecoo(indptr, info, packed, K, N, L.BN, L.buckets_per_tile, value_type=1)
+    assert _as_set(ko, no, vo) == _as_set(kk, nn, vb)
+    # the slot's value field is the FP32 number itself
+    slots = packed.view(np.uint32).ravel()
+    live = slots[(slots >> 13) != 0]
+    assert sorted((live & 0xffffe000).view(np.float32).tolist()) == sorted(vb.view(np.float16).astype(np.float32).tolist())
+    # these arrays are not BF16 arrays: a BF16 layout rejects them, and the oracle's BF16 reader refuses them too
+    Lb = fq.fq_get_layout(K, N, 128)
+    Lb.max_tile_packets, Lb.max_bucket_packets, Lb.max_tail_packets, Lb.tilecoo_encoded = \
+        L.max_tile_packets, L.max_bucket_packets, L.max_tail_packets, 1
+    with pytest.raises(fq.FqError) as e:
+        fq.fq_validate_tilecoo(Lb, indptr, info, packed)
+    assert e.value.code == fq.FQ_ERR_FORMAT
+    with pytest.raises(ValueError):
+        oracle.decode_tilecoo(indptr, info, packed, K, N, L.BN, L.buckets_per_tile, value_type=0)
+    # and a BF16 value with eight significant bits and a large exponent is not a binary16 number
+    Lb2 = fq.fq_get_layout(K, N, 128)
+    ip, bi, pk = fq.fq_encode_tilecoo(Lb2, kk[:4], nn[:4], np.array([0x4780, 0x3F80, 0x0080, 0x3F81], dtype=np.uint16))
+    fq.fq_validate_tilecoo(Lb2, ip, bi, pk)
+    Lb2.value_type = fq.FQ_VALUE_FP16
+    with pytest.raises(fq.FqError) as e:
+        fq.fq_validate_tilecoo(Lb2, ip, bi, pk)          # 0x4780 = 65536 and 0x0080 = 2^-126 are out of range
+    assert e.value.code == fq.FQ_ERR_FORMAT
+
+
 def test_tilecoo_edge_cases():
     K, N, BN, NB = 256, 512, 256, 64
     L = fq.fq_get_layout(K, N, 128, bn_hint=BN)
@@ -258,7 +301,7 @@ def test_tilecoo_edge_cases():
     assert (kk.tolist(), nn.tolist(), vv.tolist()) == ([200], [300], [0x4000])
     # column 300 = tile column 44 = column number 1 of bucket 8 + 4; the other slots are padding that
     # names their own column number
-    assert packed.view(np.uint32).reshape(-1, 4)[0].tolist() == [0 << 12, (0x4000 << 16) | (1 << 12) | (72 << 5), 2 << 12, 3 << 12]
+    assert packed.view(np.uint32).reshape(-1, 4)[0].tolist() == [0 << 3, (0x4000 << 16) | (1 << 3) | (72 << 5), 2 << 3, 3 << 3]
     # one completely dense tile plus a hot row and a hot column elsewhere
     kk, nn = np.meshgrid(np.arange(128, 256), np.arange(0, 256), indexing="ij")
     k = np.concatenate([kk.ravel(), np.full(256, 3), np.arange(0, 128)]).astype(np.uint32)
@@ -296,7 +339,7 @@ def test_validator_rejects_corrupted_arrays():
     bad = info.copy(); bad[0] = (bad[0] & 0xffff) | (0xffff << 16)
     expect_format_error(indptr, bad, packed)
     slots = packed.view(np.uint32).reshape(-1, 4)
-    bad = slots.copy(); bad[0, 0] |= 1 << 14             # a bit outside the fields
+    bad = slots.copy(); bad[0, 0] |= 1 << 12             # a bit outside the fields
     expect_format_error(indptr, info, bad.view(np.uint8).reshape(-1, 16))
     bad = slots.copy(); bad[0, 2] |= 1 << 2
     expect_format_error(indptr, info, bad.view(np.uint8).reshape(-1, 16))
@@ -306,7 +349,7 @@ def test_validator_rejects_corrupted_arrays():
     assert b0 < NB and (int(info[b0]) >> 16) & 0xff > 0
     off0 = int(info[b0] & 0xffff)
     bad = slots.copy()
-    bad[off0, 1] ^= 1 << 12
+    bad[off0, 1] ^= 1 << 3
     expect_format_error(indptr, info, bad.view(np.uint8).reshape(-1, 16))
     # more column-slotted packets than the format allows
     bad = info.copy(); bad[0] = (bad[0] & 0xffff) | (33 << 16)

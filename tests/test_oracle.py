@@ -266,7 +266,7 @@ def test_decode_tilecoo_hand_built():
     slots = np.zeros((4, 4), dtype=np.uint32)
 
     def put(p, slot, k, j, bits):
-        slots[p, slot] = (bits << 16) | (j << 12) | (k << 5)
+        slots[p, slot] = (bits << 16) | (j << 3) | (k << 5)
 
     # tile 0, bucket 1 (columns 1, 9, 17, 25): two column-slotted packets
     put(0, 0, 5, 0, 0x3F80); put(0, 1, 0, 1, 0); put(0, 2, 127, 2, 0xBF80); put(0, 3, 0, 3, 0)
@@ -291,10 +291,46 @@ def test_decode_tilecoo_hand_built():
     with pytest.raises(ValueError):
         oracle.decode_tilecoo(indptr, bad, packets, K, N, BN, NB)
     wrong = slots.copy()
-    wrong[0, 1] = (0x3F80 << 16) | (2 << 12)  # a column-slotted slot that names another column
+    wrong[0, 1] = (0x3F80 << 16) | (2 << 3)  # a column-slotted slot that names another column
     with pytest.raises(ValueError):
         oracle.decode_tilecoo(indptr, info, wrong.view(np.uint8).reshape(4, 16), K, N, BN, NB)
     stray = slots.copy()
     stray[3, 0] |= 1                         # a bit outside the fields
     with pytest.raises(ValueError):
         oracle.decode_tilecoo(indptr, info, stray.view(np.uint8).reshape(4, 16), K, N, BN, NB)
+
+
+def test_binary16_conversion_matches_numpy_on_every_pattern_and_enters_the_matmul():
+    """The oracle's IEEE binary16 reader (outlier values of the second type in Table 1) against numpy's float16 for
+    all 65536 patterns, and Eq. 1 with binary16 outliers against a dense numpy matmul."""
+    import ctypes
+    lib = oracle.lib()
+    lib.orc_f16_to_f64.restype = ctypes.c_double
+    lib.orc_f16_to_f64.argtypes = [ctypes.c_uint16]
+    pats = np.arange(65536, dtype=np.uint16)
+    want = pats.view(np.float16).astype(np.float64)
+    got = np.array([lib.orc_f16_to_f64(int(p)) for p in pats])
+    assert np.array_equal(np.isnan(got), np.isnan(want))
+    ok = ~np.isnan(want)
+    assert np.array_equal(got[ok], want[ok]) and np.array_equal(np.signbit(got[ok]), np.signbit(want[ok]))
+    # Eq. 1: zero dense part (all codes equal the zero-point), outliers as binary16
+    K, N, M, g = 128, 64, 3, 128
+    rng = np.random.default_rng(11)
+    q = np.full((K, N), 5, dtype=np.uint8)
+    s = np.full((K // g, N), 0x3F80, dtype=np.uint16)            # scale 1
+    z = np.full((K // g, N), 0x40A0, dtype=np.uint16)            # zero-point 5
+    nnz = 300
+    pos = rng.choice(K * N, size=nnz, replace=False)
+    kk, nn = (pos // N).astype(np.uint32), (pos % N).astype(np.uint32)
+    vals = rng.normal(0, 1, size=nnz).astype(np.float16)
+    Xf = rng.normal(0, 1, size=(M, K)).astype(np.float32)
+    Xb = (Xf.view(np.uint32) >> 16).astype(np.uint16)
+    Xd = (Xb.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    Wd = np.zeros((K, N), dtype=np.float64)
+    Wd[kk, nn] = vals.astype(np.float64)
+    Y = oracle.fused_matmul(Xb, q, s, z, g, kk, nn, vals.view(np.uint16), value_type=1)
+    assert np.allclose(Y, Xd @ Wd, rtol=0, atol=1e-12)
+    # the same bits read as BF16 are other numbers: the type must matter
+    Yb = oracle.fused_matmul(Xb, q, s, z, g, kk, nn, vals.view(np.uint16), value_type=0)
+    assert not np.allclose(Yb, Y, rtol=1e-3, atol=1e-3)
+

@@ -159,6 +159,17 @@ fq_status_t fq_pack_int4_sizes(const fq_layout_t* L, size_t* wq_bytes, size_t* s
 fq_status_t fq_pack_int4(const fq_layout_t* L, const float* W, const uint8_t* outlier_mask, void* wq,
                          uint16_t* scale_bf16, uint16_t* zero_bf16);
 
+/* Section 3.2.1, last remark: padding slots of the packed outliers can hold original weight values.  In the
+ * column-slotted packets a bucket is as deep as its longest column, so every other column of the bucket has
+ * (depth - count) slots that cost their bytes anyway.  This host function names the weights that go there: for
+ * every tile, bucket and column, the (depth - count) non-outlier weights of the column inside the tile with the
+ * largest quantisation error |w - s (q - z)| under `mask` (larger first, lower row first among equals; never a
+ * weight whose error or whose BF16 value is 0); buckets with a column of more than 32 outliers are left alone.
+ * mask_out (K x N bytes, may not alias mask) = mask plus those; *added (may be NULL) = how many.  Packing and
+ * encoding under mask_out gives exactly as many packets as under mask.  W: K x N binary32 row-major. */
+fq_status_t fq_repurpose_pad_slots(const fq_layout_t* L, const float* W, const uint8_t* mask, uint8_t* mask_out,
+                                   uint64_t* added);
+
 /* Inverse of the nibble interleave: wq (host) -> q_canon (host, K x N, one code per byte). */
 fq_status_t fq_unpack_int4(const fq_layout_t* L, const void* wq, uint8_t* q_canon);
 

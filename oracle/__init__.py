@@ -76,6 +76,24 @@ def quantize(W: np.ndarray, mask: np.ndarray | None, g: int):
     return q, s, z
 
 
+def repurpose_pads(W: np.ndarray, mask: np.ndarray, g: int, BN: int) -> np.ndarray:
+    """Section 3.2.1's remark on padding slots: the mask with, per tile, bucket and column, as many of the
+    column's worst-quantised weights added as the column-slotted packets have padding for."""
+    W = np.ascontiguousarray(W, dtype=np.float32)
+    mask = np.ascontiguousarray(mask, dtype=np.uint8)
+    K, N = W.shape
+    q, s, z = quantize(W, mask, g)
+    out = np.empty((K, N), dtype=np.uint8)
+    lib().orc_repurpose_pads.restype = ctypes.c_int64
+    rc = lib().orc_repurpose_pads(_p(W, ctypes.c_float), _p(mask, ctypes.c_uint8), ctypes.c_uint32(K),
+                                  ctypes.c_uint32(N), ctypes.c_uint32(g), ctypes.c_uint32(BN),
+                                  _p(q, ctypes.c_uint8), _p(s, ctypes.c_uint16), _p(z, ctypes.c_uint16),
+                                  _p(out, ctypes.c_uint8))
+    if rc < 0:
+        raise ValueError(f"orc_repurpose_pads failed: {rc}")
+    return out
+
+
 def dequant(q: np.ndarray, s: np.ndarray, z: np.ndarray, g: int) -> np.ndarray:
     """Eq. 3 in binary64: What = s * (q - z)."""
     q = np.ascontiguousarray(q, dtype=np.uint8)

@@ -199,6 +199,70 @@ void orc_fused_matmul(const uint16_t* X, uint32_t M, uint32_t K, uint32_t N, uin
     free(slot);
 }
 
+/* ------------------------------------------- pad-slot repurposing */
+
+/*
+ * Section 3.2.1, last remark: padding slots of the packed outliers can hold
+ * original weight values.  In the column-slotted packets a bucket (four
+ * columns of a 128 x BN tile: tile column c belongs to bucket 8*(c/32) + c%8)
+ * is as deep as its longest column; every other column has depth - count
+ * padding slots that cost their bytes anyway.  This function names the
+ * weights that go there.  For every tile, bucket and column, taken on their
+ * own:
+ *   count = the column's outliers inside the tile (mask = 1, BF16 value not 0);
+ *   depth = the largest count of the bucket's four columns; a bucket with a
+ *           count above 32 is left alone (its packets are laid out otherwise);
+ *   the depth - count non-outlier weights of the column inside the tile with
+ *   the largest error |w - s (q - z)| of the quantisation under `mask`
+ *   (Eq. 2, Eq. 3; binary64 difference), larger error first, lower row first
+ *   among equals, error 0 or BF16 value 0 never, become outliers as well.
+ * mask_out = mask plus those.  Quantising again under mask_out and encoding
+ * gives the same packet count as under mask.  q, scale, zero: the result of
+ * orc_quantize under `mask`.  Returns the number of weights added, or -1.
+ */
+int64_t orc_repurpose_pads(const float* W, const uint8_t* mask, uint32_t K, uint32_t N, uint32_t g,
+                           uint32_t BN, const uint8_t* q, const uint16_t* scale, const uint16_t* zero,
+                           uint8_t* mask_out) {
+    if (K % 128 != 0 || N % BN != 0 || g == 0 || K % g != 0) return -1;
+    memcpy(mask_out, mask, (size_t)K * N);
+    int64_t added = 0;
+    for (uint32_t tn = 0; tn < N / BN; ++tn)
+        for (uint32_t kt = 0; kt < K / 128; ++kt)
+            for (uint32_t b = 0; b < BN / 4; ++b) {
+                uint32_t count[4], depth = 0;
+                for (uint32_t j = 0; j < 4; ++j) {
+                    const uint32_t n = tn * BN + 32 * (b / 8) + b % 8 + 8 * j;
+                    count[j] = 0;
+                    for (uint32_t r = 0; r < 128; ++r) {
+                        const size_t idx = (size_t)(kt * 128 + r) * N + n;
+                        if (mask[idx] && (orc_f32_to_bf16(W[idx]) & 0x7fffu) != 0) ++count[j];
+                    }
+                    if (count[j] > depth) depth = count[j];
+                }
+                if (depth > 32) continue;
+                for (uint32_t j = 0; j < 4; ++j) {
+                    const uint32_t n = tn * BN + 32 * (b / 8) + b % 8 + 8 * j;
+                    for (uint32_t pick = count[j]; pick < depth; ++pick) {
+                        double best = 0.0;
+                        int64_t best_r = -1;
+                        for (uint32_t r = 0; r < 128; ++r) {
+                            const uint32_t k = kt * 128 + r;
+                            const size_t idx = (size_t)k * N + n;
+                            if (mask_out[idx] || (orc_f32_to_bf16(W[idx]) & 0x7fffu) == 0) continue;
+                            const double s = (double)orc_bf16_to_f32(scale[(size_t)(k / g) * N + n]);
+                            const double z = (double)orc_bf16_to_f32(zero[(size_t)(k / g) * N + n]);
+                            const double err = fabs((double)W[idx] - s * ((double)q[idx] - z));
+                            if (err > best) best = err, best_r = (int64_t)r;   /* strict: the lowest row wins a tie */
+                        }
+                        if (best_r < 0) break;
+                        mask_out[(size_t)(kt * 128 + (uint32_t)best_r) * N + n] = 1;
+                        ++added;
+                    }
+                }
+            }
+    return added;
+}
+
 /* ------------------------------------------------------ format decoders */
 
 /*

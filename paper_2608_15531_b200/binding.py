@@ -29,6 +29,7 @@ FQ_VALUE_FP16 = 1
 EXPORTS = [
     "fq_get_layout", "fq_pack_int4_sizes", "fq_pack_int4", "fq_unpack_int4", "fq_encode_tilecoo_sizes",
     "fq_encode_tilecoo", "fq_decode_tilecoo", "fq_validate_tilecoo", "fq_workspace_bytes",
+    "fq_repurpose_pad_slots",
     "fq_fused_w4a16_outlier_gemm", "fq_fused_w4a16_outlier_gemm_noalloc", "fq_unfused_gemm", "fq_unfused_spmm", "fq_fused_host_io",
     "fq_fused_host_io_async",
     "fq_check_status", "fq_last_error",
@@ -124,6 +125,17 @@ def fq_pack_int4(L: Layout, W: np.ndarray, outlier_mask: np.ndarray | None):
     zero = np.empty((G, L.N), dtype=np.uint16)
     _check(lib().fq_pack_int4(ctypes.byref(L), _hp(W), _hp(mask), _hp(wq), _hp(scale), _hp(zero)))
     return wq, scale, zero
+
+
+def fq_repurpose_pad_slots(L: Layout, W: np.ndarray, mask: np.ndarray):
+    """Returns (mask with the worst-quantised weights added where the packets have padding, number added)."""
+    W = np.ascontiguousarray(W, dtype=np.float32)
+    mask = np.ascontiguousarray(mask, dtype=np.uint8)
+    assert W.shape == (L.K, L.N) and mask.shape == W.shape
+    out = np.empty_like(mask)
+    added = ctypes.c_uint64(0)
+    _check(lib().fq_repurpose_pad_slots(ctypes.byref(L), _hp(W), _hp(mask), _hp(out), ctypes.byref(added)))
+    return out, int(added.value)
 
 
 def fq_unpack_int4(L: Layout, wq: np.ndarray) -> np.ndarray:

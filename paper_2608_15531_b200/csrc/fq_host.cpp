@@ -67,6 +67,9 @@ fq_status_t fq_get_layout(uint32_t K, uint32_t N, uint32_t group, uint32_t bn_hi
     return FQ_OK;
 }
 
+// Tile column of column number j of bucket b (buckets are static: 8 * (c / 32) + c % 8).
+static inline uint32_t column_of_bucket(uint32_t b, uint32_t j) { return ((b >> 3) << 5) | (b & 7u) | (j << 3); }
+
 fq_status_t fq_pack_int4_sizes(const fq_layout_t* L, size_t* wq_bytes, size_t* scale_bytes, size_t* zero_bytes) {
     if (!layout_ok(L)) return fail(FQ_ERR_INVALID_ARG, "bad layout");
     if (wq_bytes) *wq_bytes = (size_t)L->K * L->N / 2;
@@ -147,6 +150,87 @@ fq_status_t fq_pack_int4(const fq_layout_t* L, const float* W, const uint8_t* ma
             }
         }
     }
+    return FQ_OK;
+}
+
+fq_status_t fq_repurpose_pad_slots(const fq_layout_t* L, const float* W, const uint8_t* mask, uint8_t* mask_out,
+                                   uint64_t* added_out) {
+    if (!layout_ok(L)) return fail(FQ_ERR_INVALID_ARG, "bad layout");
+    if (!W || !mask || !mask_out) return fail(FQ_ERR_INVALID_ARG, "fq_repurpose_pad_slots: null pointer");
+    const uint32_t K = L->K, N = L->N, g = L->group, BN = L->BN, NB = L->buckets_per_tile;
+    const uint32_t KT = K / FQ_BK, NT = N / BN, gpc = FQ_BK / g;
+    std::memcpy(mask_out, mask, (size_t)K * N);
+    uint64_t added = 0;
+#pragma omp parallel reduction(+ : added)
+    {
+        std::vector<double> err((size_t)FQ_BK * BN);          // quantisation error of every weight of the tile; < 0: not a candidate
+        std::vector<uint32_t> count(BN);
+        std::vector<std::pair<double, uint32_t>> cand;
+#pragma omp for schedule(dynamic, 4)
+        for (int64_t ch = 0; ch < (int64_t)NT * KT; ++ch) {
+            const uint32_t tn = (uint32_t)(ch / KT), kt = (uint32_t)(ch % KT);
+            const size_t n0 = (size_t)tn * BN;
+            std::fill(count.begin(), count.end(), 0u);
+            for (uint32_t gi = 0; gi < gpc; ++gi) {
+                const uint32_t k0 = kt * FQ_BK + gi * g;
+                for (uint32_t c = 0; c < BN; ++c) {
+                    // Eq. 2 for this group and column under `mask`, as in fq_pack_int4
+                    float wmin = 0.0f, wmax = 0.0f;
+                    for (uint32_t k = k0; k < k0 + g; ++k) {
+                        if (mask[(size_t)k * N + n0 + c]) continue;
+                        const float w = W[(size_t)k * N + n0 + c];
+                        wmin = std::min(wmin, w), wmax = std::max(wmax, w);
+                    }
+                    float s = bf16_to_f32(f32_to_bf16_rne((wmax - wmin) / 15.0f));
+                    int z = 0;
+                    const bool degenerate = !(s > 0.0f);
+                    if (!degenerate) {
+                        z = (int)nearbyintf(-wmin / s);
+                        z = z < 0 ? 0 : (z > 15 ? 15 : z);
+                    }
+                    for (uint32_t k = k0; k < k0 + g; ++k) {
+                        const size_t idx = (size_t)k * N + n0 + c;
+                        const float w = W[idx];
+                        const bool nonzero = (f32_to_bf16_rne(w) & 0x7fffu) != 0;
+                        double e = -1.0;
+                        if (mask[idx]) {
+                            if (nonzero) ++count[c];
+                        } else if (nonzero) {
+                            int q = 0;
+                            if (!degenerate) {
+                                q = (int)nearbyintf(w / s) + z;
+                                q = q < 0 ? 0 : (q > 15 ? 15 : q);
+                            }
+                            const double what = degenerate ? 0.0 : (double)s * ((double)q - (double)z);   // Eq. 3
+                            e = std::fabs((double)w - what);
+                        }
+                        err[(size_t)(k - kt * FQ_BK) * BN + c] = e;
+                    }
+                }
+            }
+            for (uint32_t b = 0; b < NB; ++b) {
+                uint32_t depth = 0;
+                for (uint32_t j = 0; j < 4; ++j) depth = std::max(depth, count[column_of_bucket(b, j)]);
+                if (depth > 32) continue;                      // a bucket with a tail keeps its padding
+                for (uint32_t j = 0; j < 4; ++j) {
+                    const uint32_t c = column_of_bucket(b, j), free_slots = depth - count[c];
+                    if (!free_slots) continue;
+                    cand.clear();
+                    for (uint32_t r = 0; r < FQ_BK; ++r)
+                        if (err[(size_t)r * BN + c] > 0.0) cand.emplace_back(err[(size_t)r * BN + c], r);
+                    const size_t take = std::min<size_t>(free_slots, cand.size());
+                    // larger error first, lower row first among equals
+                    std::partial_sort(cand.begin(), cand.begin() + take, cand.end(),
+                                      [](const std::pair<double, uint32_t>& x, const std::pair<double, uint32_t>& y) {
+                                          return x.first != y.first ? x.first > y.first : x.second < y.second;
+                                      });
+                    for (size_t i = 0; i < take; ++i) mask_out[(size_t)(kt * FQ_BK + cand[i].second) * N + n0 + c] = 1;
+                    added += take;
+                }
+            }
+        }
+    }
+    if (added_out) *added_out = added;
     return FQ_OK;
 }
 

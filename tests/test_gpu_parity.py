@@ -313,6 +313,27 @@ def test_fp16_outlier_values_keep_their_ten_fraction_bits(M):
         assert not Y.any()
 
 
+@pytest.mark.parametrize("M", [1, 8, 16, 24])
+def test_layer_with_repurposed_pad_slots_matches_the_oracle(M):
+    """Section 3.2.1's remark: every padding slot of the column-slotted packets holds an original weight.  Same
+    packet count, every slot live; every element against the oracle through each kernel."""
+    K, N, g = 1024, 768, 128
+    lay = synth.layer(synth.tensor_seed(8, 12), K, N, density=0.01, layout="mixed")
+    L0 = fq.fq_get_layout(K, N, g)
+    before = fq.fq_encode_tilecoo(L0, lay.coo_k, lay.coo_n, lay.coo_v)[2].shape[0]
+    mask2, added = fq.fq_repurpose_pad_slots(L0, lay.W, lay.mask)
+    assert added > 0
+    kk, nn = np.nonzero(mask2)
+    lay.mask, lay.coo_k, lay.coo_n = mask2, kk.astype(np.uint32), nn.astype(np.uint32)
+    lay.coo_v = H.f64_to_bf16_bits(lay.W[kk, nn].astype(np.float64))
+    P = H.pack_layer(lay, g)
+    assert P.packed.shape[0] == before
+    X = _x(13, M, K)
+    Yref, Yabs = H.oracle_result(P, X)
+    for streaming_only in (False, True):
+        H.check_tolerances(H.run_fused(P, X, streaming_only=streaming_only), Yref, Yabs, K)
+
+
 def test_argument_errors_launch_nothing():
     K, N, g = 512, 512, 128
     lay = synth.layer(1, K, N, density=0.01)

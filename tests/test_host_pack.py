@@ -282,6 +282,41 @@ def test_fp16_outlier_values_round_trip_exactly():
     assert e.value.code == fq.FQ_ERR_FORMAT
 
 
+@pytest.mark.parametrize("layout,BN,g", [("uniform", 256, 128), ("mixed", 128, 64), ("clustered", 256, 128)])
+def test_pad_slot_repurposing_matches_the_oracle_and_costs_no_packets(layout, BN, g):
+    """Section 3.2.1's remark on padding slots: the library picks exactly the weights the oracle picks, the packed
+    outliers take exactly as many packets as before, every padding slot of a bucket without a tail is in use, and
+    the reconstruction error drops."""
+    K, N = 512, 512
+    Lr = synth.layer(404, K, N, density=0.01, layout=layout)
+    L = fq.fq_get_layout(K, N, g, bn_hint=BN)
+    mask2, added = fq.fq_repurpose_pad_slots(L, Lr.W, Lr.mask)
+    want = oracle.repurpose_pads(Lr.W, Lr.mask, g, BN)
+    assert np.array_equal(mask2, want) and added == int(want.sum()) - int(Lr.mask.sum()) and added > 0
+    ip0, bi0, pk0 = fq.fq_encode_tilecoo(L, Lr.coo_k, Lr.coo_n, Lr.coo_v)
+    kk, nn = np.nonzero(mask2)
+    vv = ((Lr.W[kk, nn].view(np.uint32) + 0x7fff + ((Lr.W[kk, nn].view(np.uint32) >> 16) & 1)) >> 16).astype(np.uint16)
+    L2 = fq.fq_get_layout(K, N, g, bn_hint=BN)
+    ip1, bi1, pk1 = fq.fq_encode_tilecoo(L2, kk.astype(np.uint32), nn.astype(np.uint32), vv)
+    assert np.array_equal(ip0, ip1) and np.array_equal(bi0, bi1) and pk0.shape == pk1.shape
+    off, depth, tail = _fields(bi1)
+    slots = pk1.view(np.uint32).reshape(-1, 4)
+    ntile = ip1.size - 1
+    NB = L.buckets_per_tile
+    for t in range(ntile):
+        for b in range(NB):
+            i = t * NB + b
+            if tail[i] == 0:
+                assert ((slots[ip1[t] + off[i]: ip1[t] + off[i] + depth[i]] >> 13) != 0).all()
+    # the packed weights under the new mask reconstruct W more closely
+    def recon_error(m, k_, n_, v_):
+        q, s, z = oracle.quantize(Lr.W, m, g)
+        R = oracle.dequant(q, s, z, g)
+        R[k_, n_] = (v_.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+        return np.linalg.norm(Lr.W.astype(np.float64) - R)
+    assert recon_error(mask2, kk, nn, vv) < recon_error(Lr.mask, Lr.coo_k, Lr.coo_n, Lr.coo_v)
+
+
 def test_tilecoo_edge_cases():
     K, N, BN, NB = 256, 512, 256, 64
     L = fq.fq_get_layout(K, N, 128, bn_hint=BN)

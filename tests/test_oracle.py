@@ -334,3 +334,85 @@ def test_binary16_conversion_matches_numpy_on_every_pattern_and_enters_the_matmu
     Yb = oracle.fused_matmul(Xb, q, s, z, g, kk, nn, vals.view(np.uint16), value_type=0)
     assert not np.allclose(Yb, Y, rtol=1e-3, atol=1e-3)
 
+
+def _pad_case(seed, K=256, N=256, density=0.02):
+    rng = np.random.default_rng(seed)
+    W = rng.normal(0, 0.02, size=(K, N)).astype(np.float32)
+    mask = (rng.random((K, N)) < density).astype(np.uint8)
+    W = np.where(mask == 1, (rng.uniform(0.12, 0.4, size=(K, N)) * rng.choice([-1, 1], size=(K, N))).astype(np.float32), W)
+    return W, mask
+
+
+def test_pad_slot_repurposing_worked_example():
+    """Section 3.2.1's remark, on a tile small enough to check by eye.  One tile of 128 x 128, groups of 128.
+    Column 0 has two outliers, columns 8, 16 and 24 (the other three columns of bucket 0) have none: the bucket is
+    two packets deep and each of those three columns has two padding slots.  Every weight of column 8 sits
+    exactly on the quantisation grid except rows 5 and 77; column 16 is all zero; column 24 has three off-grid
+    weights.  Expected: column 8 gains rows 5 and 77, column 16 nothing (no weight with an error), column 24 its two
+    worst rows; nothing else changes."""
+    K = N = 128
+    W = np.zeros((K, N), dtype=np.float32)
+    mask = np.zeros((K, N), dtype=np.uint8)
+    W[3, 0], W[90, 0] = 0.3, -0.25
+    mask[3, 0] = mask[90, 0] = 1
+    W[10, 0] = 0.015                                      # a plain weight of column 0: range [0, 0.015]
+    # column 8: range exactly [-0.75, 0.75], scale 0.1 (BF16 of 0.1 = 0.10009765625), values on the grid s*(q-z)
+    s8 = float(np.float32(np.uint32(0x3DCD << 16).view(np.float32)))
+    W[0, 8], W[1, 8] = np.float32(-7 * s8), np.float32(8 * s8)          # z = 7
+    for r in range(2, 128):
+        W[r, 8] = np.float32(((r % 15) - 7) * s8)
+    W[5, 8] = np.float32(2.4 * s8)                        # error 0.4 s
+    W[77, 8] = np.float32(-3.3 * s8)                      # error 0.3 s
+    # column 24: scale 0x3CA4 = 0.02001953125, range exactly [-7 s, 8 s]; three off-grid weights with errors
+    # 0.009, 0.006, 0.003
+    s24 = float(np.uint32(0x3CA4 << 16).view(np.float32))
+    W[0, 24], W[1, 24] = np.float32(-7 * s24), np.float32(8 * s24)
+    W[40, 24] = np.float32(2 * s24 + 0.009)
+    W[41, 24] = np.float32(-3 * s24 - 0.006)
+    W[42, 24] = np.float32(1 * s24 + 0.003)
+    out = oracle.repurpose_pads(W, mask, 128, 128)
+    q, s, z = oracle.quantize(W, mask, 128)
+    assert s[0, 8] == 0x3DCD and oracle.bf16_to_f32(int(z[0, 8])) == 7.0
+    assert s[0, 24] == 0x3CA4 and oracle.bf16_to_f32(int(z[0, 24])) == 7.0
+    added = np.argwhere((out == 1) & (mask == 0))
+    got = {(int(r), int(c)) for r, c in added}
+    err24 = np.abs(W[:, 24].astype(np.float64) - oracle.dequant(q, s, z, 128)[:, 24])
+    worst24 = set(np.argsort(-err24, kind="stable")[:2].tolist())
+    assert worst24 == {40, 41}
+    assert got == {(5, 8), (77, 8), (40, 24), (41, 24)}
+    assert np.array_equal(out[mask == 1], mask[mask == 1])
+
+
+@pytest.mark.parametrize("seed,BN", [(1, 128), (2, 256)])
+def test_pad_slot_repurposing_invariants(seed, BN):
+    """What the definition fixes, checked with code of its own: per (tile, column) exactly depth - count weights
+    are added where that many candidates exist; they are the largest quantisation errors of the column inside the
+    tile; and the matrix reconstructed under the new mask is closer to W."""
+    K, N, g = 256, 256, 128
+    W, mask = _pad_case(seed, K, N)
+    out = oracle.repurpose_pads(W, mask, g, BN)
+    assert np.all(out[mask == 1] == 1)
+    q, s, z = oracle.quantize(W, mask, g)
+    err = np.abs(W.astype(np.float64) - oracle.dequant(q, s, z, g))
+    for tn in range(N // BN):
+        for kt in range(K // 128):
+            rows = slice(kt * 128, kt * 128 + 128)
+            cnt = mask[rows, tn * BN:(tn + 1) * BN].sum(axis=0).astype(int)
+            for b in range(BN // 4):
+                cols = [32 * (b // 8) + b % 8 + 8 * j for j in range(4)]
+                depth = max(cnt[c] for c in cols)
+                for c in cols:
+                    n = tn * BN + c
+                    new = (out[rows, n] == 1) & (mask[rows, n] == 0)
+                    assert new.sum() == depth - cnt[c]
+                    if new.any():
+                        rest = (out[rows, n] == 0)
+                        assert err[rows, n][new].min() >= err[rows, n][rest].max()
+    def recon_error(m):
+        q2, s2, z2 = oracle.quantize(W, m, g)
+        What = oracle.dequant(q2, s2, z2, g)
+        bf = ((W.view(np.uint32) + 0x7fff + ((W.view(np.uint32) >> 16) & 1)) & 0xffff0000).view(np.float32).astype(np.float64)
+        R = np.where(m == 1, bf, What)
+        return np.linalg.norm(W.astype(np.float64) - R)
+    assert recon_error(out) < recon_error(mask)
+

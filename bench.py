@@ -581,11 +581,26 @@ def run_sweep(args):
         torch.cuda.synchronize()
         return a.elapsed_time(b) / reps * 1e3
 
-    def point(cfg, tag, K, N, g, density, layout, Ms):
+    def point(cfg, tag, K, N, g, density, layout, Ms, slot_order=0, repurpose=False, extra=None):
         lay = synth.layer(synth.tensor_seed(cfg, tag), K, N, density=density, layout=layout)
         L = fq.fq_get_layout(K, N, g)
+        L.slot_order = slot_order
+        t0 = time.time()
+        if repurpose:
+            # Section 3.2.1's remark: the packets' padding slots take the column's worst-quantised weights
+            mask2, _ = fq.fq_repurpose_pad_slots(L, lay.W, lay.mask)
+            kk, nn = np.nonzero(mask2)
+            u = lay.W[kk, nn].view(np.uint32).astype(np.uint64)
+            lay.mask, lay.coo_k, lay.coo_n = mask2, kk.astype(np.uint32), nn.astype(np.uint32)
+            lay.coo_v = ((u + 0x7fff + ((u >> 16) & 1)) >> 16).astype(np.uint16)
+        t1 = time.time()
         wq, scale, zero = fq.fq_pack_int4(L, lay.W, lay.mask if lay.nnz else None)
+        t2 = time.time()
         indptr, info, packed = fq.fq_encode_tilecoo(L, lay.coo_k, lay.coo_n, lay.coo_v)
+        t3 = time.time()
+        if extra is not None:
+            extra.update(repurpose_s=round(t1 - t0, 3), pack_s=round(t2 - t1, 3), encode_s=round(t3 - t2, 3),
+                         packets=int(packed.shape[0]), stored_values=int(lay.nnz))
         if packed.shape[0] == 0:
             packed = np.zeros((8, 16), dtype=np.uint8)
         base = dict(wq=up(wq), scale=up(scale), zero=up(zero), indptr=up(indptr), info=up(info), packed=up(packed))
@@ -653,6 +668,17 @@ def run_sweep(args):
                 points += pts
                 print(f"[bench] {K}x{N} {density}: " + ", ".join(f"M={q['M']}: {q['fused_us']} us" for q in pts),
                       file=sys.stderr, flush=True)
+    elif args.sweep == "encoder":
+        # Ablation of the encoder's choices (Sec. 5.4) on the density sweep's shape at 1 % mixed outliers: order of
+        # a column's outliers over its packets (bank-aware / by row), padding slots empty / holding weights.
+        for slot_order, repurpose in ((0, False), (1, False), (0, True)):
+            extra = {}
+            pts = point(3, 10, 4096, 14336, GROUP, DENSITY, "mixed", (1, 8, 16), slot_order=slot_order,
+                        repurpose=repurpose, extra=extra)
+            for pt in pts:
+                pt.update(slot_order="bank-aware" if slot_order == 0 else "by row", pad_slots="weights" if repurpose else "empty",
+                          **extra)
+            points += pts
     elif args.sweep == "density":
         for layout in ("uniform", "clustered"):
             for density in (0.0, 0.005, 0.01, 0.02, 0.05):
@@ -712,7 +738,7 @@ def main():
                     help="skip the per-call rows of configs[0] and configs[3] (N = 1 only; the headline is unchanged)")
     ap.add_argument("--verbose", action="store_true")
     ap.add_argument("--only", default="", help="profiling aid: restrict the step to one LAYER:M, e.g. gate_up:16")
-    ap.add_argument("--sweep", default="", choices=["", "density", "batch", "paper"],
+    ap.add_argument("--sweep", default="", choices=["", "density", "batch", "paper", "encoder"],
                     help="print the density sweep, the batch transition sweep or the paper's ratio-and-batch sweep on "
                          "its largest operator shape (minutes of host time) instead of the benchmark line")
     args = ap.parse_args()

@@ -273,6 +273,8 @@ __global__ void __launch_bounds__(kSpmmThreads, 2) fq_spmm_kernel(const uint16_t
     float acc[RR];
 #pragma unroll
     for (int i = 0; i < RR; ++i) acc[i] = 0.0f;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (kt0 >= kt1) asm volatile("griddepcontrol.wait;" ::: "memory");     // a slab without k-steps still adds to Y below
 
     for (uint32_t c0 = kt0; c0 < kt1; c0 += kSpmmChunk) {
         const uint32_t nk = min((uint32_t)kSpmmChunk, kt1 - c0);
@@ -287,15 +289,6 @@ __global__ void __launch_bounds__(kSpmmThreads, 2) fq_spmm_kernel(const uint16_t
                 base[j] = __ldg(indptr + u);
             }
         }
-        // the chunk's activations: a thread takes eight consecutive k of one batch row at a time
-        constexpr int XU = RR == 1 ? 1 : RR * 16 * kSpmmChunk / kSpmmThreads;
-        uint4 xr[XU];
-#pragma unroll
-        for (int j = 0; j < XU; ++j) {
-            const uint32_t e = tid + j * kSpmmThreads, m = e % RR, o = e / RR;
-            xr[j] = make_uint4(0, 0, 0, 0);
-            if (o < 16 * nk && m < M) xr[j] = __ldg(reinterpret_cast<const uint4*>(X + (size_t)m * K + (size_t)c0 * kBK) + o);
-        }
         uint32_t w[kSpmmPer][4];
         const uint32_t* pk[kSpmmPer];
 #pragma unroll
@@ -304,6 +297,17 @@ __global__ void __launch_bounds__(kSpmmThreads, 2) fq_spmm_kernel(const uint16_t
             const uint32_t depth = (inf[j] >> 16) & 0xffu;
 #pragma unroll
             for (int d = 0; d < 4; ++d) w[j][d] = (uint32_t)d < depth ? __ldg(pk[j] + d * 4 + t) : 0u;
+        }
+        // descriptors and packets are weights; X and Y may come from the grid before this one in the stream
+        if (c0 == kt0) asm volatile("griddepcontrol.wait;" ::: "memory");
+        // the chunk's activations: a thread takes eight consecutive k of one batch row at a time
+        constexpr int XU = RR == 1 ? 1 : RR * 16 * kSpmmChunk / kSpmmThreads;
+        uint4 xr[XU];
+#pragma unroll
+        for (int j = 0; j < XU; ++j) {
+            const uint32_t e = tid + j * kSpmmThreads, m = e % RR, o = e / RR;
+            xr[j] = make_uint4(0, 0, 0, 0);
+            if (o < 16 * nk && m < M) xr[j] = __ldg(reinterpret_cast<const uint4*>(X + (size_t)m * K + (size_t)c0 * kBK) + o);
         }
 #pragma unroll
         for (int j = 0; j < XU; ++j) {
@@ -773,10 +777,13 @@ static cudaError_t launch_spmm(const fq_layout_t* L, const uint16_t* X, uint32_t
     cfg.blockDim = dim3(kSpmmThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
-    cudaLaunchAttribute at[1];
+    cudaLaunchAttribute at[2];
+    std::memset(at, 0, sizeof(at));
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = slabs, at[0].val.clusterDim.y = 1, at[0].val.clusterDim.z = 1;
-    cfg.attrs = at, cfg.numAttrs = 1;
+    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;        // as the fused launches: the descriptors
+    at[1].val.programmaticStreamSerializationAllowed = 1;                 // and first slots load during the tail of
+    cfg.attrs = at, cfg.numAttrs = 2;                                     // the kernel before (the dense half)
     return cudaLaunchKernelEx(&cfg, fq_spmm_kernel<RR>, X, (const uint32_t*)indptr, (const uint32_t*)info,
                               (const uint4*)packed, Y, M, L->K, L->N, L->BN, slabs);
 }

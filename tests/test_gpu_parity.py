@@ -334,6 +334,27 @@ def test_layer_with_repurposed_pad_slots_matches_the_oracle(M):
         H.check_tolerances(H.run_fused(P, X, streaming_only=streaming_only), Yref, Yabs, K)
 
 
+def test_column_shards_computed_one_after_the_other_give_the_full_result():
+    """The N-sharded wrapper's per-rank part on one GPU: the two ranks' shards of a layer (widths 512 and 256) are
+    packed and run one after the other, without a collective, and their slices side by side are the full Y."""
+    from paper_2608_15531_b200.sharded import ShardedLayer
+    K, N, g, M = 512, 768, 128, 8
+    lay = synth.layer(synth.tensor_seed(8, 13), K, N, density=0.01, layout="mixed")
+    X = _x(14, M, K)
+    P = H.pack_layer(lay, g)
+    Yref, Yabs = H.oracle_result(P, X)
+    Xd = H.to_dev(X)
+    parts = []
+    for rank in range(2):
+        layer = ShardedLayer(lay.W, lay.mask, lay.coo_k, lay.coo_n, lay.coo_v, g, rank, 2)
+        parts.append(H.bf16_bits(layer.local(Xd)))
+    Y = np.concatenate(parts, axis=1)
+    assert np.array_equal(Y, H.run_fused(P, X))          # same kernels, same per-column arithmetic: bit-equal
+    H.check_tolerances(Y, Yref, Yabs, K)
+    one = ShardedLayer(lay.W, lay.mask, lay.coo_k, lay.coo_n, lay.coo_v, g, 0, 1)
+    assert np.array_equal(H.bf16_bits(one.forward(Xd)), Y)
+
+
 def test_argument_errors_launch_nothing():
     K, N, g = 512, 512, 128
     lay = synth.layer(1, K, N, density=0.01)

@@ -34,10 +34,10 @@ CONFIG_ID = 2                      # the LLaMA-3-8B layer set
 REPEATS = 5                        # repetitions of the timed region (K steps each); the median is the value
 L2_COVER_BYTES = 400 << 20         # rotating copies per layer cover at least this (L2 is 126 MB)
 METRIC = "effective_hbm_gbs_fused_w4a16_outlier_gemm_m1_8_16"
-# dram__bytes_read + dram__bytes_write of the fused kernel over its algorithmic bytes, from the ncu
-# captures summarised in profiles/fq_mma_kernel_llama3_8b_decode_set.md (1.06 to 1.07 on the three
-# launches captured: the per-column padding of the packets); scaled to the average launch of the step.
-NCU_TRAFFIC_RATIO = 1.07
+# dram__bytes_read + dram__bytes_write of a fused launch over its algorithmic bytes, per layer, from the ncu captures
+# summarised in profiles/fq_kernels_llama3_8b_decode_set.md (the padding of the column-slotted packets; the ratio
+# does not depend on M).  Not measured by a bench run: `roofline.traffic` applies them to the step's launches.
+NCU_TRAFFIC_RATIO = {"gate_up": 1.072, "down": 1.053, "qkv": 1.049, "o_proj": 1.048}
 
 
 def algorithmic_bytes(K, N, g, nnz, n_tile, n_bucket, M):
@@ -441,9 +441,10 @@ def run_ours(args):
                 "ms_per_step": round(e2e_ms / args.steps, 5)},
         "gpu_launches": args.steps * len(calls),
         "roofline": {"bound": "hbm", "achieved": round(value / world, 2), "peak": peak, "unit": "GB/s",
-                     "frac": round(value / world / peak, 4), "traffic": int(NCU_TRAFFIC_RATIO * (step_bytes // len(calls))),
-                     "traffic_kind": f"constant: algorithmic bytes x {NCU_TRAFFIC_RATIO}, the DRAM/algorithmic ratio of the "
-                                     "committed captures (1.06-1.08); not measured by this run",
+                     "frac": round(value / world / peak, 4),
+                     "traffic": int(sum(NCU_TRAFFIC_RATIO.get(w["name"], 1.06) * b for w, M, b in calls) / len(calls)),
+                     "traffic_kind": "algorithmic bytes x the DRAM/algorithmic ratio of each layer's committed ncu capture "
+                                     f"{NCU_TRAFFIC_RATIO}, average launch of the step; not measured by this run",
                      "peak_kind": f"of {peak_kind}",
                      "bytes_per_launch": step_bytes // len(calls), "us_per_launch": round(ms_per_step * 1e3 / len(calls), 3),
                      # the same time against other byte counts and other denominators

@@ -175,12 +175,14 @@ fq_status_t fq_unpack_int4(const fq_layout_t* L, const void* wq, uint8_t* q_cano
 
 /*
  * Tile-COO encoder (Section 3.2.1).  Input: COO triplets on the host (k, n,
- * BF16 value bits), any order; entries whose value is +-0 are dropped.  Every
- * entry goes to the bucket of its column and is stored as "Tile-COO" above
- * says: column-slotted packets with per-column padding (Section 4.2), and a
- * tail for a bucket with a very long column.  The column and element
- * reordering of Section 3.2.2 serve a shared-memory scatter that the kernels
- * here do not have, so they are not applied.
+ * 16 value bits of the type L->value_type names), any order; entries whose
+ * value is +-0 are dropped.  Every entry goes to the bucket of its column and
+ * is stored as "Tile-COO" above says: column-slotted packets with per-column
+ * padding (Section 4.2), and a tail for a bucket with a very long column.  Of
+ * the two reorderings of Section 3.2.2 the element order is applied, restated
+ * for the kernels' shared-memory reads (L->slot_order); the column-to-bucket
+ * assignment is static (see "Tile-COO" above), so the column permutation is
+ * not.
  *
  * fq_encode_tilecoo_sizes: element counts of the three arrays (tile_indptr in
  * uint32, bucket_info in uint32, packets in 16-byte units) and the largest

@@ -205,8 +205,8 @@ def fq_fused_w4a16_outlier_gemm_noalloc(L: Layout, X, M: int, wq, scale, zero, t
                                         stream=None) -> None:
     """The fused operator without a caller-provided workspace: for callers that may not allocate
     device memory.  Uses the scratch array built into the library (one per GPU, shared by all
-    calls: do not overlap calls on different streams).  Refuses calls that need more scratch than
-    the array holds (M > 16)."""
+    calls: do not overlap calls on different streams).  Refuses calls whose ``fq_workspace_bytes`` exceeds
+    the array (FQ_ERR_BUFFER_TOO_SMALL): every call of more than 16 rows on a layer with 256-column tiles."""
     _check(lib().fq_fused_w4a16_outlier_gemm_noalloc(ctypes.byref(L), _dp(X), ctypes.c_uint32(M), _dp(wq), _dp(scale),
                                                      _dp(zero), _dp(tile_indptr), _dp(bucket_info), _dp(packed),
                                                      _dp(Y), _stream(stream)))

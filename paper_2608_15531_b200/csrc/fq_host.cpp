@@ -275,7 +275,7 @@ struct Encoded {
 
 // Bucket of a tile column: the four columns {g, g + 8, g + 16, g + 24} of a 32-column block share
 // bucket 8 * (c / 32) + c % 8.  These are the columns whose accumulators one group of four lanes
-// holds in the small-batch kernel, so a bucket's outliers are applied in registers.
+// holds in the kernels, so a bucket's outliers are applied in registers.
 inline uint32_t bucket_of(uint32_t c) { return ((c >> 5) << 3) | (c & 7u); }
 // Number of a column inside its bucket, and the way back.
 inline uint32_t number_in_bucket(uint32_t c) { return (c >> 3) & 3u; }
@@ -399,12 +399,10 @@ fq_status_t encode_impl(const fq_layout_t* L, const uint32_t* k, const uint32_t*
                         int cand[4][5], ncand[4];
                         for (uint32_t q = 0; q < 4; ++q) {
                             ncand[q] = 0;
-                            const uint32_t c = (b0 + q) * 4 + j;
                             if (d >= depths[b0 + q]) { cand[q][ncand[q]++] = -1; continue; }
                             for (uint32_t e = 0; e < used[q].size() && ncand[q] < 4; ++e)
                                 if (!used[q][e]) cand[q][ncand[q]++] = (int)e;
                             if (todo[q] < depths[b0 + q] - d) cand[q][ncand[q]++] = -1;
-                            (void)c;
                         }
                         int best[4] = {cand[0][0], cand[1][0], cand[2][0], cand[3][0]};
                         uint32_t best_cost = 1u << 30;

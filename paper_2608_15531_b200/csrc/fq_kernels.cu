@@ -513,7 +513,7 @@ static Scratch scratch_layout(const fq_layout_t* L, uint32_t rows) {
 }
 
 typedef void (*PrepFn)(const uint16_t*, uint32_t, uint32_t, uint8_t*);
-static PrepFn pick_prep(uint32_t rr, uint32_t g) { (void)rr; (void)g; return fq_prep_x_kernel<32, 128>; }
+static PrepFn pick_prep() { return fq_prep_x_kernel<32, 128>; }      // 17 to 32 rows, groups of 128: one variant
 
 typedef void (*KernelFn)(const Params);
 
@@ -525,14 +525,14 @@ struct MmaPlan {
 };
 typedef void (*MmaKernelFn)(const MmaParams);
 
-// Plan of the small-batch kernel (fq_mma_kernel): M <= 16 per launch.
+// Plan of the streaming kernel (fq_mma_kernel): M <= 16 per launch.
 static fq_status_t make_plan_mma(const fq_layout_t* L, uint32_t M, bool sparse, MmaPlan& pl) {
     const uint32_t BN = L->BN, NB = L->buckets_per_tile, GPS = kBK / L->group;
     const uint32_t MO = M <= 8 ? 1 : 2, ROWS = 8 * MO;
     const uint32_t NDW = BN / 32;
     MmaParams& p = pl.p;
     std::memset(&p, 0, sizeof(p));
-    p.M = M; p.K = L->K; p.N = L->N; p.KT = L->K / kBK; p.NT = L->N / BN; p.NB = NB; p.nsw = 0;
+    p.M = M; p.K = L->K; p.N = L->N; p.KT = L->K / kBK; p.NT = L->N / BN; p.NB = NB;
     const uint32_t w_bytes = 16 * BN * 4, sz_bytes = 2 * GPS * BN * 2;
     const uint32_t xt_bytes = sparse ? (M == 1 ? 512 : (M <= 4 ? 2048 : MO * 4096)) : 0;     // FP32 [k], [k][4] or [octet][k][8]
     // Two groups of dense warps (each takes every other unit) pay off when a CTA has enough units to
@@ -629,8 +629,7 @@ static KernelFn pick_tc_sparse(bool sparse, bool hot) {
     if (!sparse) return (KernelFn)fq_tc_kernel<BN, RR, G, false, false>;
     return hot ? (KernelFn)fq_tc_kernel<BN, RR, G, true, true> : (KernelFn)fq_tc_kernel<BN, RR, G, true, false>;
 }
-static KernelFn pick_kernel(uint32_t bn, uint32_t M, uint32_t g, bool sparse, bool hot) {
-    (void)M; (void)g;      // 17 to 32 rows, groups of 128: one variant per tile width
+static KernelFn pick_kernel(uint32_t bn, bool sparse, bool hot) {      // 17 to 32 rows, groups of 128: one variant per tile width
     return bn == 128 ? pick_tc_sparse<128, 32, 128>(sparse, hot) : pick_tc_sparse<256, 32, 128>(sparse, hot);
 }
 
@@ -708,7 +707,7 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
             p.counters = (uint32_t*)((uint8_t*)workspace + kWsHeaderBytes);
             p.partials = (float*)((uint8_t*)workspace + sc.off_partials);
             p.xblob = xb;
-            KernelFn fn = pick_kernel(L->BN, mb, L->group, sparse, pl.general);
+            KernelFn fn = pick_kernel(L->BN, sparse, pl.general);
             e = ensure_smem_attr((const void*)fn, (int)kSmemBudget);
             if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
             // the activation blocks of these rows, then the fused kernel
@@ -716,7 +715,7 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
             cfg.gridDim = dim3((warps + 3) / 4);
             cfg.blockDim = dim3(128);
             cfg.dynamicSmemBytes = 0;
-            e = cudaLaunchKernelEx(&cfg, pick_prep(rr, L->group), Xm, mb, L->K, xb);
+            e = cudaLaunchKernelEx(&cfg, pick_prep(), Xm, mb, L->K, xb);
             if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "activation preparation launch: %s", cudaGetErrorString(e));
             cfg.gridDim = dim3(pl.grid);
             cfg.blockDim = dim3(pl.threads);
@@ -730,13 +729,12 @@ static fq_status_t launch_gemm(const fq_layout_t* L, const void* X, uint32_t M, 
             p.indptr = (const uint32_t*)indptr; p.info = (const uint32_t*)info; p.packed = (const uint4*)packed;
             p.status = (uint32_t*)workspace;
             p.M = mb; p.K = L->K; p.N = L->N; p.KT = L->K / kBK; p.BN = L->BN; p.NB = L->buckets_per_tile;
-            const uint32_t warps = direct_warps(L, mb), nv = (mb <= 8 ? 1u : 2u) * 8u;
+            const uint32_t warps = direct_warps(L, mb);
             cfg.gridDim = dim3(L->N / 32);
             cfg.blockDim = dim3(32 * warps);
             // per warp: rows of activations, their k-major copy, scale and zero rows, staged packets; the warps'
             // sums reuse those bytes
             cfg.dynamicSmemBytes = warps * kDirectWarpBytes;
-            (void)nv;
             DirectFn dfn = pick_direct(mb, warps, L->group, sparse);
             e = ensure_smem_attr((const void*)dfn, 32 * kDirectWarpBytes);
             if (e != cudaSuccess) return fail(FQ_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));

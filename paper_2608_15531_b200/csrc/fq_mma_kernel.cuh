@@ -19,9 +19,8 @@ struct MmaParams {
     uint32_t* counters;
     float* partials;
     uint32_t M, K, N, KT, NT;
-    uint32_t NB, coo_cap, stages, nsw;
-    uint32_t nact;    // tcgen05 kernel: activation warps at work (the ring length is a multiple of it)
-    uint32_t split;   // small-batch kernel: 0 = units dealt out as one contiguous range per CTA (stream-K);
+    uint32_t NB, coo_cap, stages;
+    uint32_t split;   // 0 = units dealt out as one contiguous range per CTA (stream-K);
                       // c > 0 = every column tile belongs to c CTAs, CTA b takes part b mod c of tile b / c
     // shared-memory offsets (bytes); the first five are relative to a stage
     uint32_t stage_bytes, off_sz, off_xcan, off_xsum, off_info, off_coo;
@@ -57,7 +56,7 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-constexpr int kActWarps = 2;   // activation warps of the small-batch kernel
+constexpr int kActWarps = 2;   // activation warps of the streaming kernel
 // Activation row in shared memory: 256 B, its sixteen 16-byte chunks stored at chunk ^ 4 in odd rows.
 // The fragment loads of a quarter warp (rows g and g + 1, four consecutive chunks each) then touch
 // all 32 banks once.

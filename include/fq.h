@@ -220,22 +220,27 @@ fq_status_t fq_workspace_bytes(const fq_layout_t* L, uint32_t M, size_t* bytes);
 
 /*
  * The fused operator (Eq. 1; Sections 3.1 and 4.1): a launch reads X, W_Q and
- * the Tile-COO tiles through a bulk-copy/mbarrier ring, dequantises in
- * registers into tensor-core operands, applies the tile's outliers against the
- * activation tile in shared memory, and writes Y once.  Up to 16 rows of X go
- * through one launch of a kernel built on warp-level MMAs (exact integers
- * 128 + q in BF16, scale and zero-point applied per group in FP32).  Larger M
- * is served in launches of up to 32 rows by a kernel built on tcgen05.mma with
- * 8-bit integer operands (groups of 128; groups of 64 stay with launches of
- * 16 rows): its activations are block fixed point, 22 bits plus sign relative
- * to the largest |x| of each row and group, so activations more than 2^14
- * below that maximum are rounded (to 2^-22 of it).  The kernel is chosen by the
- * rows of a launch alone.
+ * the Tile-COO tiles, dequantises in registers into tensor-core operands (exact
+ * integers, scale and zero-point applied per group in FP32), adds the tile's
+ * outliers into the accumulators of their columns, and writes Y once.  Which
+ * kernel serves a launch is decided from its rows and the layer's shape alone:
+ *   - up to 16 rows: warp-level MMAs (128 + q as BF16).  Layers with so few
+ *     32-column strips and k-steps that every CTA's job would be short get one
+ *     CTA per strip, whose warps split K among themselves and read the weights
+ *     straight into registers; every other layer streams (tile, k-step) units
+ *     through a bulk-copy/mbarrier ring on persistent CTAs;
+ *   - 17 to 32 rows (a larger M is cut into such launches), groups of 128: a
+ *     kernel built on tcgen05.mma with 8-bit integer operands.  Its
+ *     activations are block fixed point, 22 bits plus sign relative to the
+ *     largest |x| of each row and group, so activations more than 2^14 below
+ *     that maximum are rounded (to 2^-22 of it).  Groups of 64 stay with
+ *     launches of 16 rows.
+ * L->kernel_hint = 1 keeps the one-CTA-per-strip kernel out (for tests).
  * X: device, M x K BF16.  M in [1, FQ_MAX_M].  Y: device, M x N BF16,
  * overwritten.  All other arrays: device copies of the host packer/encoder
- * output.  Work is split over persistent CTAs by (tile, k-step) units; tiles
- * shared by several CTAs are summed in a fixed order, so results are run-to-run
- * reproducible.
+ * output.  Partial sums of one output, whether of the warps of a CTA or of
+ * several CTAs that share a tile, are added in a fixed order, so results are
+ * run-to-run reproducible.
  *
  * Ordering.  Every kernel is launched so that it may become resident while the
  * kernel before it in the stream is still draining (programmatic dependent

@@ -355,6 +355,19 @@ def test_column_shards_computed_one_after_the_other_give_the_full_result():
     assert np.array_equal(H.bf16_bits(one.forward(Xd)), Y)
 
 
+@pytest.mark.parametrize("K,N,g", [(128, 128, 128), (128, 256, 64), (256, 128, 128), (8192, 256, 128)])
+@pytest.mark.parametrize("M", [1, 4, 7, 16])
+def test_smallest_and_thinnest_layers(K, N, g, M):
+    """One k-step (most warps of a short-job CTA have nothing to do), one column tile, one strip per CTA with 64
+    k-steps: the extremes of the short-job kernel's split, and the same shapes through the streaming kernel."""
+    lay = synth.layer(synth.tensor_seed(8, K + N), K, N, density=0.02, layout="uniform")
+    P = H.pack_layer(lay, g)
+    X = _x(15, M, K)
+    Yref, Yabs = H.oracle_result(P, X)
+    for streaming_only in (False, True):
+        H.check_tolerances(H.run_fused(P, X, streaming_only=streaming_only), Yref, Yabs, K)
+
+
 def test_argument_errors_launch_nothing():
     K, N, g = 512, 512, 128
     lay = synth.layer(1, K, N, density=0.01)
